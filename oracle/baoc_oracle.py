@@ -1,0 +1,517 @@
+"""CPU oracle for the BAOC hot path.  TEST INFRASTRUCTURE, NOT THE PRODUCT.
+
+A plain, slow, double-precision numpy restatement of what the paper's method
+computes on the path this repository accelerates: the per-block gradient
+statistics (Sec. 3.3, Eq. 3-8), their normalisation and the risk matrix
+(Appendix A, Eq. 9-21), the aggressiveness penalty (Eq. 1), the budgeted
+allocation (Eq. 2, by exhaustive enumeration) and the update rule of each
+configuration tuple of Definition 3.1 that the library offers.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this module.  It shares no code with the CUDA library and never calls it.
+Every function works on one block at a time, takes plain numpy arrays and
+carries floating-point state in float64; the 8-bit codes and their fp32
+absmax scales are the state by definition and are kept in their own types.
+
+Where the paper is silent the readings below are used (the same ones the
+library documents):
+  * coordinates are sampled densely (the sample is the whole block);
+  * EMA moments start at zero and are not bias-corrected (Eq. 3 as written);
+  * the stability EMA starts at the first available cosine; beta_rho = 0.9;
+  * quantiles use linear interpolation at position q*(n-1);
+  * the 8-bit quantiser is block-wise absmax with linear codes over 256
+    consecutive elements (signed 127 levels for first moments, unsigned 255
+    for second moments, round half to even, fp32 absmax); the 16-bit
+    quantiser rounds to bfloat16;
+  * the update direction of Eq. 8 is m/(sqrt(v)+1e-8) from the window's own
+    moments;
+  * update rules are the textbook ones for each tuple (see the step_*
+    functions).
+
+Parity unpinned: no value printed in the paper distinguishes these readings;
+each function below is pinned by closed forms, invariants, library special
+cases and brute force in the CPU test-suite instead.
+"""
+from __future__ import annotations
+
+import itertools
+import math
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+F64 = np.float64
+
+
+# ----------------------------------------------------------------------------
+# Options and configuration tuples
+# ----------------------------------------------------------------------------
+
+@dataclass
+class Opts:
+    beta_m: float = 0.9            # Eq. 3, "standard Adam values"
+    beta_v: float = 0.999
+    beta_rho: float = 0.9          # Eq. 5 smoothing factor (paper gives no value)
+    eps: float = 1e-12             # Appendix A.1
+    a_lo: float = math.log(2.0)    # Eq. 11
+    a_hi: float = math.log(10.0)
+    rho_lo: float = 0.2            # Eq. 13
+    rho_hi: float = 0.6
+    snr_lo: float = 0.0            # Eq. 15
+    snr_hi: float = 2.0
+    w: Tuple[float, float, float, float, float] = (1.0, 1.0, 1.0, 1.0, 1.0)  # w_A, w_M, w_C, w_F, w_Q
+    gamma: float = 0.1             # weight of Agg in the objective
+    use_snr: bool = True           # Eq. 17, else s_M = s_rho
+    eps_adam: float = 1e-8         # epsilon of the update direction in Eq. 8
+    qblock: int = 256              # elements per quantisation block
+
+
+@dataclass
+class Config:
+    """Definition 3.1: c = (y_a, y_m, y_d, y_f, b) plus the hyper-parameters
+    of the update rule it instantiates."""
+    adaptive: int
+    momentum: int
+    decoupled_wd: int
+    factored: int
+    bits: int
+    lr: float = 1e-3
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+    weight_decay: float = 0.0
+
+
+def default_configs() -> List[Config]:
+    """The five tuples of the hot path: fp32 AdamW, 8-bit AdamW, momentum-free
+    RMS scaling, factored second moment, SGD with momentum."""
+    return [Config(1, 1, 1, 0, 32, weight_decay=0.01),
+            Config(1, 1, 1, 0, 8, weight_decay=0.01),
+            Config(1, 0, 1, 0, 32, weight_decay=0.01),
+            Config(1, 0, 1, 1, 32, weight_decay=0.01),
+            Config(0, 1, 1, 0, 32, lr=1e-2, weight_decay=0.01)]
+
+
+# ----------------------------------------------------------------------------
+# Quantisers (the "standard quantizer" of Sec. 3.3, Precision Sensitivity)
+# ----------------------------------------------------------------------------
+
+def _blocks_view(x: np.ndarray, qblock: int):
+    """Pad x with zeros to a multiple of qblock and view it as [nq, qblock]."""
+    d = x.shape[0]
+    nq = (d + qblock - 1) // qblock
+    pad = np.zeros(nq * qblock, dtype=x.dtype)
+    pad[:d] = x
+    return pad.reshape(nq, qblock), d
+
+
+def quantize8(x: np.ndarray, signed: bool, qblock: int = 256):
+    """Block-wise absmax linear 8-bit codes.
+
+    Per quantisation block: a = fl32(max |x|); code = clamp(rne(L * x / a)) with
+    L = 127 (signed, codes in [-127, 127]) or L = 255 (unsigned, [0, 255]);
+    a == 0 gives all-zero codes.  Returns (codes, absmax fp32[nq]).
+    """
+    x = np.asarray(x, dtype=F64)
+    xb, d = _blocks_view(x, qblock)
+    a = np.max(np.abs(xb), axis=1).astype(np.float32)
+    L = 127.0 if signed else 255.0
+    a64 = a.astype(F64)
+    safe = np.where(a64 > 0.0, a64, 1.0)
+    s = np.rint(L * xb / safe[:, None])             # np.rint rounds half to even
+    s = np.clip(s, -L if signed else 0.0, L)
+    s = np.where(a64[:, None] > 0.0, s, 0.0)
+    codes = s.reshape(-1)[:d].astype(np.int8 if signed else np.uint8)
+    return codes, a
+
+
+def dequantize8(codes: np.ndarray, absmax: np.ndarray, signed: bool, qblock: int = 256) -> np.ndarray:
+    """x = code * a / L in double."""
+    L = 127.0 if signed else 255.0
+    cb, d = _blocks_view(codes.astype(F64), qblock)
+    x = cb * absmax.astype(F64)[:, None] / L
+    return x.reshape(-1)[:d]
+
+
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest bfloat16 (ties to even), returned as float64.
+
+    The value is first rounded to fp32, then its low 16 bits are rounded away.
+    """
+    f = np.asarray(x, dtype=np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    lsb = (u >> 16) & 1
+    r = ((u + 0x7FFF + lsb) >> 16) << 16
+    out = (r & 0xFFFFFFFF).astype(np.uint32).view(np.float32)
+    out = np.where(np.isfinite(f), out, f)
+    return out.astype(F64)
+
+
+# ----------------------------------------------------------------------------
+# O1. Per-step statistics (Eq. 3 and Eq. 5 left)
+# ----------------------------------------------------------------------------
+
+@dataclass
+class StatsState:
+    d: int
+    m: np.ndarray
+    v: np.ndarray
+    g_prev: Optional[np.ndarray] = None
+    rho_bar: float = 0.0
+    n_cos: int = 0
+    t: int = 0
+    last_cos: float = 0.0
+    # diagnostic only (not used by the risk): EMA of cos(g_t, m_{t-1})
+    rho_mom: float = 0.0
+    n_cos_mom: int = 0
+
+
+def stats_init(d: int) -> StatsState:
+    return StatsState(d=d, m=np.zeros(d, F64), v=np.zeros(d, F64))
+
+
+def _cosine(a: np.ndarray, b: np.ndarray, eps: float) -> float:
+    """<a,b> / (||a|| ||b|| + eps), with a non-finite result replaced by 0
+    (Appendix A.1: a NaN cosine counts as 0)."""
+    c = float(np.dot(a, b)) / (math.sqrt(float(np.dot(a, a))) * math.sqrt(float(np.dot(b, b))) + eps)
+    return c if math.isfinite(c) else 0.0
+
+
+def stats_step(st: StatsState, g: np.ndarray, o: Opts) -> None:
+    """One gradient observation of one block."""
+    g = np.asarray(g, dtype=F64)
+    st.t += 1
+    if st.g_prev is not None:
+        c = _cosine(g, st.g_prev, o.eps)                       # Eq. 5 left
+        st.last_cos = c
+        st.rho_bar = c if st.n_cos == 0 else o.beta_rho * st.rho_bar + (1.0 - o.beta_rho) * c
+        st.n_cos += 1
+        cm = _cosine(g, st.m, o.eps)                           # diagnostic
+        st.rho_mom = cm if st.n_cos_mom == 0 else o.beta_rho * st.rho_mom + (1.0 - o.beta_rho) * cm
+        st.n_cos_mom += 1
+    st.m = o.beta_m * st.m + (1.0 - o.beta_m) * g              # Eq. 3
+    st.v = o.beta_v * st.v + (1.0 - o.beta_v) * (g * g)
+    st.g_prev = g.copy()
+
+
+# ----------------------------------------------------------------------------
+# O2. Finalize (Eq. 4, Eq. 5 right, Eq. 6, Eq. 7, Eq. 8)
+# ----------------------------------------------------------------------------
+
+def quantile_linear(x: np.ndarray, q: float) -> float:
+    """q-th quantile by linear interpolation between order statistics at
+    position q*(n-1)."""
+    s = np.sort(np.asarray(x, dtype=F64))
+    n = s.shape[0]
+    pos = q * (n - 1)
+    k = int(math.floor(pos))
+    frac = pos - k
+    if k + 1 < n:
+        return float(s[k] + frac * (s[k + 1] - s[k]))
+    return float(s[k])
+
+
+def anisotropy(v: np.ndarray, eps: float) -> float:
+    """Eq. 4."""
+    return math.log((quantile_linear(v, 0.9) + eps) / (quantile_linear(v, 0.1) + eps))
+
+
+def snr(m: np.ndarray, v: np.ndarray, eps: float) -> float:
+    """Eq. 5 right: ||m||^2 / (||v||_1 + eps)."""
+    return float(np.dot(m, m)) / (float(np.sum(np.abs(v))) + eps)
+
+
+def distortion(v: np.ndarray, theta: np.ndarray, eps: float) -> float:
+    """Eq. 6 with p = 1/(sqrt(v)+eps)."""
+    theta = np.asarray(theta, dtype=F64)
+    p = 1.0 / (np.sqrt(v) + eps)
+    pbar = float(np.mean(p))
+    num = np.linalg.norm((p / pbar - 1.0) * theta)
+    return float(num / (np.linalg.norm(theta) + eps))
+
+
+def structure_residual(v: np.ndarray, rows: int, cols: int, eps: float) -> float:
+    """Eq. 7: S = v as rows x cols, rank-1 model from row and column means."""
+    if cols <= 1:
+        return 1.0          # not a matrix block: the factored configuration is not offered
+    S = np.asarray(v, dtype=F64).reshape(rows, cols)
+    a = S.mean(axis=1)
+    b = S.mean(axis=0)
+    mu = float(S.mean())
+    if mu == 0.0:
+        St = np.zeros_like(S)
+    else:
+        St = np.outer(a, b) / mu
+    return float(np.linalg.norm(S - St) / (np.linalg.norm(S) + eps))
+
+
+def precision_cosine(m: np.ndarray, v: np.ndarray, bits: int, o: Opts) -> float:
+    """Eq. 8: cosine between the full-precision direction m/(sqrt(v)+eps_adam)
+    and the one computed from quantised moments."""
+    u32 = m / (np.sqrt(v) + o.eps_adam)
+    if bits == 32:
+        mq, vq = m, v
+    elif bits == 16:
+        mq, vq = round_bf16(m), round_bf16(v)
+    elif bits == 8:
+        cm, am = quantize8(m, True, o.qblock)
+        cv, av = quantize8(v, False, o.qblock)
+        mq = dequantize8(cm, am, True, o.qblock)
+        vq = dequantize8(cv, av, False, o.qblock)
+    else:
+        raise ValueError("bits must be 8, 16 or 32")
+    ub = mq / (np.sqrt(vq) + o.eps_adam)
+    return _cosine(u32, ub, o.eps)
+
+
+def quant_rel_error(x: np.ndarray, bits: int, signed: bool, o: Opts) -> float:
+    """Diagnostic: ||x - Q_b(x)|| / ||x|| (0 for a zero vector)."""
+    if bits == 16:
+        xq = round_bf16(x)
+    else:
+        c, a = quantize8(x, signed, o.qblock)
+        xq = dequantize8(c, a, signed, o.qblock)
+    n = float(np.linalg.norm(x))
+    return float(np.linalg.norm(x - xq)) / n if n > 0.0 else 0.0
+
+
+def stats_finalize(st: StatsState, theta: np.ndarray, rows: int, cols: int, o: Opts) -> Dict[str, float]:
+    """Raw diagnostics z_i of one block at the end of the window."""
+    return {
+        "A": anisotropy(st.v, o.eps),
+        "rho_bar": st.rho_bar,
+        "snr": snr(st.m, st.v, o.eps),
+        "C": distortion(st.v, theta, o.eps),
+        "F": structure_residual(st.v, rows, cols, o.eps),
+        "Q32": precision_cosine(st.m, st.v, 32, o),
+        "Q16": precision_cosine(st.m, st.v, 16, o),
+        "Q8": precision_cosine(st.m, st.v, 8, o),
+        "q10": quantile_linear(st.v, 0.1),
+        "q90": quantile_linear(st.v, 0.9),
+        "rho_mom": st.rho_mom,
+        "err_m8": quant_rel_error(st.m, 8, True, o),
+        "err_v8": quant_rel_error(st.v, 8, False, o),
+        "err_m16": quant_rel_error(st.m, 16, True, o),
+        "err_v16": quant_rel_error(st.v, 16, False, o),
+    }
+
+
+# ----------------------------------------------------------------------------
+# O3. Normalisation (Appendix A, Eq. 10-20)
+# ----------------------------------------------------------------------------
+
+def _clip(x: float, lo: float, hi: float) -> float:
+    return min(max(x, lo), hi)
+
+
+def normalise(raw: Dict[str, float], o: Opts) -> Dict[str, float]:
+    s_A = _clip((raw["A"] - o.a_lo) / (o.a_hi - o.a_lo), 0.0, 1.0)                     # Eq. 12
+    s_rho = _clip((raw["rho_bar"] - o.rho_lo) / (o.rho_hi - o.rho_lo), 0.0, 1.0)       # Eq. 14
+    s_snr = _clip((math.log(1.0 + raw["snr"]) - o.snr_lo) / (o.snr_hi - o.snr_lo), 0.0, 1.0)  # Eq. 16
+    s_M = s_rho * s_snr if o.use_snr else s_rho                                        # Eq. 17
+    C_t = math.log(1.0 + raw["C"])                                                     # Eq. 18
+    s_F = _clip(raw["F"], 0.0, 1.0)                                                    # Eq. 19
+    out = {"s_A": s_A, "s_rho": s_rho, "s_snr": s_snr, "s_M": s_M, "C_tilde": C_t, "s_F": s_F}
+    for b in (32, 16, 8):
+        Q = _clip(raw[f"Q{b}"], o.eps, 1.0)                                            # Eq. 10
+        out[f"lQ{b}"] = -math.log(Q + o.eps)                                           # Eq. 20
+    return out
+
+
+# ----------------------------------------------------------------------------
+# O4. Risk, aggressiveness, objective (Eq. 9/21, Eq. 1)
+# ----------------------------------------------------------------------------
+
+def risk(z: Dict[str, float], c: Config, o: Opts) -> float:
+    wA, wM, wC, wF, wQ = o.w
+    return (wA * z["s_A"] * (1 - c.adaptive) + wM * z["s_M"] * (1 - c.momentum)
+            + wC * z["C_tilde"] * (1 - c.decoupled_wd) + wF * z["s_F"] * c.factored
+            + wQ * z[f"lQ{c.bits}"])
+
+
+def agg(c: Config) -> float:
+    return (1 - c.adaptive) + (1 - c.momentum) + (1 - c.decoupled_wd) + c.factored + 32.0 / c.bits - 1.0
+
+
+def objective(R: float, c: Config, o: Opts, pref: float = 0.0) -> float:
+    """Phi = (R - pref) + gamma * Agg."""
+    return (R - pref) + o.gamma * agg(c)
+
+
+# ----------------------------------------------------------------------------
+# Cost model (StateMem definition, Sec. 3.1) and fixed point of the allocator
+# ----------------------------------------------------------------------------
+
+def state_bytes(c: Config, numel: int, rows: int, cols: int, qblock: int = 256) -> int:
+    """M_{i,c}: bytes of persistent optimizer state of one block."""
+    nq = (numel + qblock - 1) // qblock
+    def per_tensor():
+        if c.bits == 32:
+            return 4 * numel
+        if c.bits == 16:
+            return 2 * numel
+        return numel + 4 * nq           # 1-byte codes + one fp32 absmax per quantisation block
+    total = 0
+    if c.momentum:
+        total += per_tensor()
+    if c.adaptive:
+        if c.factored:
+            total += 4 * (rows + cols)
+        else:
+            total += per_tensor()
+    return total
+
+
+PHI_SCALE = 2.0 ** 30
+R_SCALE = 2.0 ** 20
+
+
+def phi_fixed(phi: float) -> int:
+    return int(np.rint(phi * PHI_SCALE))
+
+
+def ratio_fixed(r: float) -> int:
+    return int(np.rint(r * R_SCALE))
+
+
+def time_cap_fixed(n_blocks: int, b_time: float) -> int:
+    return int(math.floor(n_blocks * b_time * R_SCALE))
+
+
+# ----------------------------------------------------------------------------
+# O5. Allocation by exhaustive enumeration (Eq. 2)
+# ----------------------------------------------------------------------------
+
+def allocate_bruteforce(phi_fx: Sequence[Sequence[int]], mem: Sequence[Sequence[int]],
+                        r_fx: Sequence[Sequence[int]], b_mem: int, r_cap: int,
+                        forbid: Optional[Sequence[Sequence[int]]] = None):
+    """Enumerate every assignment in lexicographic order (block 0 slowest,
+    lower configuration index first) and keep the first one of minimum total
+    objective among those within both budgets and free of forbidden pairs.
+    Returns (assignment list, objective) or (None, None) when infeasible."""
+    n = len(phi_fx)
+    k = len(phi_fx[0])
+    best, best_val = None, None
+    for asg in itertools.product(range(k), repeat=n):
+        if forbid is not None and any(forbid[i][c] for i, c in enumerate(asg)):
+            continue
+        if sum(mem[i][c] for i, c in enumerate(asg)) > b_mem:
+            continue
+        if sum(r_fx[i][c] for i, c in enumerate(asg)) > r_cap:
+            continue
+        val = sum(phi_fx[i][c] for i, c in enumerate(asg))
+        if best_val is None or val < best_val:
+            best, best_val = list(asg), val
+    return best, best_val
+
+
+# ----------------------------------------------------------------------------
+# O6. Update rules (Definition 3.1 tuples)
+# ----------------------------------------------------------------------------
+
+def _prologue(theta: np.ndarray, g: np.ndarray, c: Config):
+    """Weight decay: decoupled (theta shrinks first) or coupled (added to g)."""
+    if c.weight_decay != 0.0:
+        if c.decoupled_wd:
+            theta = theta * (1.0 - c.lr * c.weight_decay)
+        else:
+            g = g + c.weight_decay * theta
+    return theta, g
+
+
+def _adam_apply(theta, m, v, c: Config, t: int, use_m: bool):
+    bc2 = 1.0 - c.beta2 ** t
+    denom = np.sqrt(v / bc2) + c.eps
+    if use_m:
+        bc1 = 1.0 - c.beta1 ** t
+        return theta - c.lr * (m / bc1) / denom
+    return theta - c.lr * m / denom
+
+
+@dataclass
+class StepState:
+    """Optimizer state of one block under one configuration."""
+    kind: str
+    t: int = 0
+    m: Optional[np.ndarray] = None
+    v: Optional[np.ndarray] = None
+    qm: Optional[np.ndarray] = None
+    qv: Optional[np.ndarray] = None
+    am: Optional[np.ndarray] = None
+    av: Optional[np.ndarray] = None
+    r: Optional[np.ndarray] = None
+    c: Optional[np.ndarray] = None
+
+
+def config_kind(c: Config) -> str:
+    """Which of the five update paths a tuple selects."""
+    if c.adaptive and c.momentum and not c.factored:
+        return "A32" if c.bits == 32 else ("A8" if c.bits == 8 else "unsupported")
+    if c.adaptive and not c.momentum and not c.factored and c.bits == 32:
+        return "R"
+    if c.adaptive and not c.momentum and c.factored and c.bits == 32:
+        return "F"
+    if not c.adaptive and c.momentum and not c.factored and c.bits == 32:
+        return "S"
+    return "unsupported"
+
+
+def step_init(c: Config, numel: int, rows: int, cols: int, qblock: int = 256) -> StepState:
+    kind = config_kind(c)
+    nq = (numel + qblock - 1) // qblock
+    if kind == "A32":
+        return StepState(kind, m=np.zeros(numel, F64), v=np.zeros(numel, F64))
+    if kind == "A8":
+        return StepState(kind, qm=np.zeros(numel, np.int8), qv=np.zeros(numel, np.uint8),
+                         am=np.zeros(nq, np.float32), av=np.zeros(nq, np.float32))
+    if kind == "R":
+        return StepState(kind, v=np.zeros(numel, F64))
+    if kind == "F":
+        if cols <= 1:
+            raise ValueError("the factored configuration needs a matrix block")
+        return StepState(kind, r=np.zeros(rows, F64), c=np.zeros(cols, F64))
+    if kind == "S":
+        return StepState(kind, m=np.zeros(numel, F64))
+    raise ValueError("unsupported configuration tuple")
+
+
+def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, cols: int,
+         qblock: int = 256) -> np.ndarray:
+    """One optimizer step of one block; returns the new parameters (float64)
+    and updates ``st`` in place.  ``st.t`` counts steps from 1."""
+    theta = np.asarray(theta, dtype=F64)
+    g = np.asarray(g, dtype=F64)
+    st.t += 1
+    t = st.t
+    theta, g = _prologue(theta, g, c)
+    if st.kind == "A32":
+        st.m = c.beta1 * st.m + (1.0 - c.beta1) * g
+        st.v = c.beta2 * st.v + (1.0 - c.beta2) * g * g
+        return _adam_apply(theta, st.m, st.v, c, t, True)
+    if st.kind == "A8":
+        m = dequantize8(st.qm, st.am, True, qblock)
+        v = dequantize8(st.qv, st.av, False, qblock)
+        m = c.beta1 * m + (1.0 - c.beta1) * g
+        v = c.beta2 * v + (1.0 - c.beta2) * g * g
+        theta = _adam_apply(theta, m, v, c, t, True)      # uses the un-requantised moments
+        st.qm, st.am = quantize8(m, True, qblock)
+        st.qv, st.av = quantize8(v, False, qblock)
+        return theta
+    if st.kind == "R":
+        st.v = c.beta2 * st.v + (1.0 - c.beta2) * g * g
+        return _adam_apply(theta, g, st.v, c, t, False)
+    if st.kind == "F":
+        G2 = (g * g).reshape(rows, cols)
+        st.r = c.beta2 * st.r + (1.0 - c.beta2) * G2.mean(axis=1)
+        st.c = c.beta2 * st.c + (1.0 - c.beta2) * G2.mean(axis=0)
+        rm = float(st.r.mean())
+        if rm == 0.0:
+            v = np.zeros(rows * cols, F64)
+        else:
+            v = (np.outer(st.r, st.c) / rm).reshape(-1)
+        return _adam_apply(theta, g, v, c, t, False)
+    if st.kind == "S":
+        st.m = c.beta1 * st.m + g
+        return theta - c.lr * st.m
+    raise ValueError("unsupported configuration tuple")

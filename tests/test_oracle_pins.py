@@ -1,0 +1,543 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+Each test checks one function of ``oracle/baoc_oracle.py`` against a closed
+form, an invariant, a library routine that a special case reduces to, or
+brute force, chosen so that a dropped term, a wrong sign or a transposed
+operand fails at least one of them.  No GPU is needed.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import baoc_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden", "paper_constants.txt")
+
+
+def _gold():
+    out = {}
+    for line in open(GOLD):
+        line = line.split("#")[0].strip()
+        if line:
+            k, v = line.split()
+            out[k] = float(v)
+    return out
+
+
+RNG = np.random.default_rng(1234)
+
+
+def _run_window(gs, o=None):
+    o = o or O.Opts()
+    st = O.stats_init(gs[0].shape[0])
+    for g in gs:
+        O.stats_step(st, g, o)
+    return st
+
+
+# ---------------------------------------------------------------- constants
+
+def test_defaults_match_paper_constants():
+    g, o = _gold(), O.Opts()
+    assert o.eps == g["eps"]
+    assert o.a_lo == math.log(g["A_low_ratio"]) and o.a_hi == math.log(g["A_high_ratio"])
+    assert (o.rho_lo, o.rho_hi, o.snr_lo, o.snr_hi) == (g["rho_low"], g["rho_high"], g["snr_low"], g["snr_high"])
+    assert o.gamma == g["gamma"]
+    assert o.w == (1.0,) * 5 and (o.beta_m, o.beta_v) == (0.9, 0.999)
+
+
+# ---------------------------------------------------------------- P1 stability (Eq. 5 left)
+
+def test_stability_identical_gradients_is_one():
+    g = RNG.standard_normal(1000)
+    st = _run_window([g] * 6)
+    assert abs(st.rho_bar - 1.0) <= 1e-12 / np.dot(g, g) + 1e-15
+    assert st.n_cos == 5
+
+
+def test_stability_sign_flip_and_zero():
+    g = RNG.standard_normal(513)
+    st = _run_window([g, -g, g, -g])
+    assert abs(st.rho_bar + 1.0) < 1e-12
+    st = _run_window([np.zeros(64)] * 4)
+    assert st.rho_bar == 0.0
+    st = _run_window([g])                     # a window of one step has no cosine
+    assert st.rho_bar == 0.0 and st.n_cos == 0
+
+
+def test_stability_orthogonal_and_ema_recursion():
+    e0, e1 = np.eye(4)[0], np.eye(4)[1]
+    d = (e0 + e1) / math.sqrt(2.0)
+    # cosines in order: <e1,e0>=0, <d,e1>=1/sqrt2, <d,d>=1
+    st = _run_window([e0, e1, d, d])
+    c = [0.0, 1 / math.sqrt(2.0), 1.0]
+    want = c[0]
+    for x in c[1:]:
+        want = 0.9 * want + 0.1 * x
+    assert abs(st.rho_bar - want) < 1e-12
+    assert abs(st.last_cos - 1.0) < 1e-11
+
+
+def test_cosine_is_scale_invariant_and_uses_both_norms():
+    a, b = RNG.standard_normal(300), RNG.standard_normal(300)
+    st1 = _run_window([a, b])
+    st2 = _run_window([7.0 * a, 0.01 * b])
+    assert abs(st1.rho_bar - st2.rho_bar) < 1e-9
+    ref = float(a @ b / (np.linalg.norm(a) * np.linalg.norm(b)))
+    assert abs(st1.rho_bar - ref) < 1e-9
+
+
+def test_momentum_cosine_uses_previous_moment():
+    a, b = RNG.standard_normal(100), RNG.standard_normal(100)
+    st = _run_window([a, b])
+    # m after step 1 is 0.1*a, so cos(b, m_prev) = cos(b, a)
+    assert abs(st.rho_mom - st.rho_bar) < 1e-9
+
+
+# ---------------------------------------------------------------- P2 moments and SNR (Eq. 3, Eq. 5 right)
+
+@pytest.mark.parametrize("T", [1, 5, 32])
+def test_constant_gradient_closed_forms(T):
+    o = O.Opts()
+    g = RNG.standard_normal(257)
+    st = _run_window([g] * T, o)
+    np.testing.assert_allclose(st.m, (1 - o.beta_m ** T) * g, rtol=1e-12)
+    np.testing.assert_allclose(st.v, (1 - o.beta_v ** T) * g * g, rtol=1e-12)
+    want = (1 - o.beta_m ** T) ** 2 / (1 - o.beta_v ** T)
+    assert abs(O.snr(st.m, st.v, o.eps) / want - 1.0) < 1e-9
+
+
+def test_moments_match_explicit_weighted_sums():
+    o = O.Opts()
+    gs = [RNG.standard_normal(50) for _ in range(7)]
+    st = _run_window(gs, o)
+    T = len(gs)
+    m = sum((1 - o.beta_m) * o.beta_m ** (T - 1 - k) * gs[k] for k in range(T))
+    v = sum((1 - o.beta_v) * o.beta_v ** (T - 1 - k) * gs[k] ** 2 for k in range(T))
+    np.testing.assert_allclose(st.m, m, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(st.v, v, rtol=1e-12, atol=1e-15)
+
+
+def test_snr_uses_l1_of_v_and_squared_l2_of_m():
+    m = np.array([3.0, -4.0])
+    v = np.array([2.0, 6.0])
+    assert abs(O.snr(m, v, 0.0) - 25.0 / 8.0) < 1e-15
+
+
+# ---------------------------------------------------------------- P3 anisotropy and quantiles (Eq. 4)
+
+def test_isotropic_gradient_has_zero_anisotropy():
+    o = O.Opts()
+    s = RNG.choice([-1.0, 1.0], size=999) * 0.37
+    st = _run_window([s, -s, s], o)
+    assert abs(O.anisotropy(st.v, o.eps)) < 1e-9
+
+
+def test_two_level_vector_gives_log_ratio():
+    v = np.concatenate([np.full(500, 2.0), np.full(500, 32.0)])
+    RNG.shuffle(v)
+    assert abs(O.anisotropy(v, 0.0) - math.log(16.0)) < 1e-12
+    # eps enters both numerator and denominator
+    assert abs(O.anisotropy(np.array([0.0, 0.0, 1.0, 1.0]), 0.5) - math.log(1.5 / 0.5)) < 1e-12
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 10, 11, 257, 1000])
+@pytest.mark.parametrize("q", [0.1, 0.9, 0.5])
+def test_quantile_matches_numpy_and_torch(n, q):
+    x = RNG.standard_normal(n) ** 2
+    assert abs(O.quantile_linear(x, q) - np.quantile(x, q)) <= 1e-12 * max(1.0, abs(np.quantile(x, q)))
+    tq = torch.quantile(torch.from_numpy(x), q).item()
+    assert abs(O.quantile_linear(x, q) - tq) <= 1e-12 * max(1.0, abs(tq))
+
+
+def test_quantile_hand_example():
+    # positions 0.1*4 = 0.4 and 0.9*4 = 3.6 over the sorted values 1 2 3 4 5
+    x = np.array([5.0, 1.0, 4.0, 2.0, 3.0])
+    assert abs(O.quantile_linear(x, 0.1) - 1.4) < 1e-12
+    assert abs(O.quantile_linear(x, 0.9) - 4.6) < 1e-12
+
+
+# ---------------------------------------------------------------- distortion (Eq. 6)
+
+def test_distortion_zero_for_constant_preconditioner():
+    theta = RNG.standard_normal(400)
+    assert O.distortion(np.full(400, 0.3), theta, 1e-12) < 1e-12
+
+
+def test_distortion_hand_example():
+    # sqrt(v) = (1, 3) -> p = (1, 1/3), mean 2/3, p/pbar - 1 = (1/2, -1/2)
+    v = np.array([1.0, 9.0])
+    theta = np.array([2.0, -4.0])
+    want = math.sqrt(1.0 + 4.0) / math.sqrt(20.0)
+    assert abs(O.distortion(v, theta, 0.0) - want) < 1e-12
+
+
+def test_distortion_is_invariant_to_scaling_theta_and_v():
+    v = RNG.standard_normal(300) ** 2 + 0.1
+    th = RNG.standard_normal(300)
+    a = O.distortion(v, th, 0.0)
+    assert abs(O.distortion(16.0 * v, 3.0 * th, 0.0) - a) < 1e-12
+
+
+# ---------------------------------------------------------------- P4 structure residual (Eq. 7)
+
+def test_rank_one_second_moment_has_zero_residual():
+    x, y = RNG.random(37) + 0.1, RNG.random(53) + 0.1
+    assert O.structure_residual(np.outer(x, y).reshape(-1), 37, 53, 1e-12) < 1e-12
+
+
+def test_identity_like_residual_closed_form():
+    # S = I_n: row and column means 1/n, mu = 1/n, so S~ = (1/n)(1/n)/(1/n) = 1/n everywhere.
+    n = 6
+    want = math.sqrt(n * (1 - 1 / n) ** 2 + (n * n - n) / n ** 2) / math.sqrt(n)
+    assert abs(O.structure_residual(np.eye(n).reshape(-1), n, n, 0.0) - want) < 1e-12
+
+
+def test_structure_residual_depends_on_shape_orientation():
+    S = RNG.random((8, 12))
+    S[2, 5] += 5.0
+    a = O.structure_residual(S.reshape(-1), 8, 12, 0.0)
+    b = O.structure_residual(S.T.copy().reshape(-1), 12, 8, 0.0)
+    assert abs(a - b) < 1e-12                       # transposing the matrix AND the shape: same residual
+    c = O.structure_residual(S.reshape(-1), 12, 8, 0.0)
+    assert abs(a - c) > 1e-3                        # wrong shape for the same buffer: different
+    assert O.structure_residual(RNG.random(10), 10, 1, 0.0) == 1.0
+
+
+# ---------------------------------------------------------------- P8 quantisers and precision cosine (Eq. 8)
+
+def test_quantize8_roundtrip_of_representable_values_is_exact():
+    a = np.float32(0.7316)
+    codes = RNG.integers(-127, 128, size=700)
+    codes[5] = 127                                   # make the absmax of every block equal to a
+    codes[300] = -127
+    codes[600] = 127
+    x = codes.astype(np.float64) * float(a) / 127.0
+    c, am = O.quantize8(x, True)
+    np.testing.assert_array_equal(c, codes.astype(np.int8))
+    np.testing.assert_array_equal(am, np.full(3, a, np.float32))
+    np.testing.assert_allclose(O.dequantize8(c, am, True), x, rtol=0, atol=0)
+    cu = RNG.integers(0, 256, size=512)
+    cu[0] = 255
+    cu[256] = 255
+    xu = cu.astype(np.float64) * float(a) / 255.0
+    c2, a2 = O.quantize8(xu, False)
+    np.testing.assert_array_equal(c2, cu.astype(np.uint8))
+    np.testing.assert_allclose(O.dequantize8(c2, a2, False), xu, rtol=0, atol=0)
+
+
+def test_quantize8_error_bound_and_ragged_tail():
+    x = RNG.standard_normal(1000)
+    c, a = O.quantize8(x, True)
+    assert a.shape == (4,) and c.dtype == np.int8
+    xr = O.dequantize8(c, a, True)
+    bound = np.repeat(a.astype(np.float64), 256)[:1000] / 254.0
+    assert np.all(np.abs(x - xr) <= bound * (1 + 1e-6))
+    v = x * x
+    cv, av = O.quantize8(v, False)
+    vr = O.dequantize8(cv, av, False)
+    boundv = np.repeat(av.astype(np.float64), 256)[:1000] / 510.0
+    assert np.all(np.abs(v - vr) <= boundv * (1 + 1e-6))
+    # absmax is per block of 256 consecutive elements, the last one short
+    assert a[3] == np.float32(np.max(np.abs(x[768:])))
+
+
+def test_quantize8_rounds_half_to_even_and_handles_zero_block():
+    a = 127.0
+    x = np.array([a, 0.5, 1.5, 2.5, -0.5, -1.5])
+    c, _ = O.quantize8(x, True)
+    np.testing.assert_array_equal(c, np.array([127, 0, 2, 2, 0, -2], np.int8))
+    c0, a0 = O.quantize8(np.zeros(300), False)
+    assert not c0.any() and not a0.any()
+    np.testing.assert_array_equal(O.dequantize8(c0, a0, False), np.zeros(300))
+
+
+def test_round_bf16_matches_torch():
+    x = np.concatenate([RNG.standard_normal(5000) * 10.0 ** RNG.integers(-20, 20, 5000),
+                        np.array([0.0, 1.0, 1.00390625, 1.01171875, -3.0])])
+    ref = torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16).double().numpy()
+    np.testing.assert_array_equal(O.round_bf16(x), ref)
+
+
+def test_precision_cosine_pins():
+    o = O.Opts()
+    m = RNG.standard_normal(2000) * 1e-3
+    v = (RNG.standard_normal(2000) * 1e-3) ** 2 + 1e-8
+    assert abs(O.precision_cosine(m, v, 32, o) - 1.0) < 1e-9
+    q16, q8 = O.precision_cosine(m, v, 16, o), O.precision_cosine(m, v, 8, o)
+    assert 0.0 < q8 <= q16 <= 1.0 + 1e-12 and q16 > 0.9999
+    # exactly representable states: quantisation changes nothing, so Q(8) = 1
+    a = np.float32(0.25)
+    cm = RNG.integers(-127, 128, 512); cm[0] = 127; cm[256] = -127
+    cv = RNG.integers(1, 256, 512); cv[0] = 255; cv[256] = 255
+    mm = cm * float(a) / 127.0
+    vv = cv * float(a) / 255.0
+    assert abs(O.precision_cosine(mm, vv, 8, o) - 1.0) < 1e-9
+    assert O.quant_rel_error(mm, 8, True, o) == 0.0 and O.quant_rel_error(vv, 8, False, o) == 0.0
+
+
+def test_precision_cosine_explicit_small_case():
+    # one quantisation block of 4: write Eq. 8 out by hand
+    o = O.Opts(qblock=4, eps_adam=0.0, eps=0.0)
+    m = np.array([1.0, -0.5, 0.26, 0.0])
+    v = np.array([4.0, 1.0, 0.25, 2.0])
+    mq = np.rint(127 * m / 1.0) / 127.0
+    vq = np.rint(255 * v / 4.0) * 4.0 / 255.0
+    u32, u8 = m / np.sqrt(v), mq / np.sqrt(vq)
+    want = u32 @ u8 / (np.linalg.norm(u32) * np.linalg.norm(u8))
+    assert abs(O.precision_cosine(m, v, 8, o) - want) < 1e-12
+
+
+# ---------------------------------------------------------------- P6 normalisation (Eq. 10-20)
+
+def _raw(**kw):
+    base = dict(A=0.0, rho_bar=0.0, snr=0.0, C=0.0, F=0.0, Q32=1.0, Q16=1.0, Q8=1.0)
+    base.update(kw)
+    return base
+
+
+def test_normalisation_anchor_values():
+    o = O.Opts()
+    z = O.normalise(_raw(A=math.log(2.0)), o); assert z["s_A"] == 0.0
+    z = O.normalise(_raw(A=math.log(10.0)), o); assert abs(z["s_A"] - 1.0) < 1e-15
+    z = O.normalise(_raw(A=0.5 * (math.log(2.0) + math.log(10.0))), o); assert abs(z["s_A"] - 0.5) < 1e-15
+    z = O.normalise(_raw(A=5.0), o); assert z["s_A"] == 1.0
+    z = O.normalise(_raw(A=-1.0), o); assert z["s_A"] == 0.0
+    for rho, want in [(0.2, 0.0), (0.4, 0.5), (0.6, 1.0), (0.9, 1.0), (-0.5, 0.0)]:
+        assert abs(O.normalise(_raw(rho_bar=rho), o)["s_rho"] - want) < 1e-15
+    for s, want in [(0.0, 0.0), (math.e - 1.0, 0.5), (math.e ** 2 - 1.0, 1.0), (1e9, 1.0)]:
+        assert abs(O.normalise(_raw(snr=s), o)["s_snr"] - want) < 1e-15
+    z = O.normalise(_raw(rho_bar=0.4, snr=math.e - 1.0), o)
+    assert abs(z["s_M"] - 0.25) < 1e-15
+    assert abs(O.normalise(_raw(rho_bar=0.4, snr=math.e - 1.0), O.Opts(use_snr=False))["s_M"] - 0.5) < 1e-15
+    assert abs(O.normalise(_raw(C=math.e - 1.0), o)["C_tilde"] - 1.0) < 1e-15
+    assert O.normalise(_raw(F=1.7), o)["s_F"] == 1.0 and O.normalise(_raw(F=0.3), o)["s_F"] == 0.3
+    z = O.normalise(_raw(Q8=0.5, Q16=-0.2, Q32=1.0), o)
+    assert abs(z["lQ8"] - (-math.log(0.5 + 1e-12))) < 1e-15
+    assert abs(z["lQ16"] - (-math.log(2e-12))) < 1e-12          # clipped to eps first (Eq. 10)
+    assert abs(z["lQ32"] - (-math.log(1.0 + 1e-12))) < 1e-15
+
+
+# ---------------------------------------------------------------- P7 risk and Agg (Eq. 1, Eq. 9)
+
+def test_agg_of_the_five_configurations():
+    assert [O.agg(c) for c in O.default_configs()] == [0.0, 3.0, 1.0, 2.0, 1.0]
+    assert O.agg(O.Config(0, 0, 0, 1, 8)) == 7.0 and O.agg(O.Config(1, 1, 1, 0, 16)) == 1.0
+
+
+def test_risk_is_linear_in_switches_with_distinct_terms():
+    o = O.Opts(w=(2.0, 3.0, 5.0, 7.0, 11.0))
+    z = dict(s_A=0.1, s_M=0.2, C_tilde=0.3, s_F=0.4, lQ32=0.0, lQ16=0.01, lQ8=0.05)
+    assert abs(O.risk(z, O.Config(1, 1, 1, 0, 32), o)) < 1e-15
+    assert abs(O.risk(z, O.Config(0, 1, 1, 0, 32), o) - 0.2) < 1e-15
+    assert abs(O.risk(z, O.Config(1, 0, 1, 0, 32), o) - 0.6) < 1e-15
+    assert abs(O.risk(z, O.Config(1, 1, 0, 0, 32), o) - 1.5) < 1e-15
+    assert abs(O.risk(z, O.Config(1, 1, 1, 1, 32), o) - 2.8) < 1e-15
+    assert abs(O.risk(z, O.Config(1, 1, 1, 0, 8), o) - 0.55) < 1e-15
+    assert abs(O.risk(z, O.Config(0, 0, 0, 1, 16), o) - (0.2 + 0.6 + 1.5 + 2.8 + 0.11)) < 1e-12
+    c = O.Config(1, 0, 1, 1, 32)
+    assert abs(O.objective(1.0, c, O.Opts(), pref=0.25) - (0.75 + 0.1 * 2.0)) < 1e-15
+
+
+# ---------------------------------------------------------------- P5 memory model
+
+def test_state_bytes_model_and_paper_tables():
+    cfg = O.default_configs()
+    d, r, c = 1024 * 300, 1024, 300
+    assert [O.state_bytes(k, d, r, c) for k in cfg] == [8 * d, 2 * d + 8 * (d // 256), 4 * d, 4 * (r + c), 4 * d]
+    assert O.state_bytes(cfg[1], 257, 257, 1) == 2 * 257 + 8 * 2
+    assert O.state_bytes(O.Config(1, 1, 1, 0, 16), d, r, c) == 4 * d
+    g = _gold()
+    per_param = 2.0 + 8.0 / 256.0
+    for name in ("llama1b", "llama3b", "unet", "gpt2", "vit"):
+        ratio = g[f"statemem_{name}_adamw8"] / g[f"statemem_{name}_adamw16"]
+        # AdamW16 keeps 4 bytes of state per parameter; the tables' 8-bit rows then imply
+        # 2 code bytes + two fp32 absmax per 256 elements (small tensors round up, hence the slack)
+        assert abs(ratio * 4.0 - per_param) < 0.02, name
+    assert abs(g["statemem_llama1b_adamw8"] / g["statemem_llama1b_adamw16"] * 4.0 - per_param) < 1e-3
+
+
+# ---------------------------------------------------------------- P9 brute-force allocation (Eq. 2)
+
+def test_bruteforce_hand_example_and_tie_break():
+    phi = [[0, 5], [0, 5], [0, 5]]
+    mem = [[4, 1], [4, 1], [4, 1]]
+    r = [[1, 1]] * 3
+    asg, val = O.allocate_bruteforce(phi, mem, r, 9, 100)
+    assert asg == [0, 0, 1] and val == 5            # equal optima: lexicographically smallest wins
+    asg, val = O.allocate_bruteforce(phi, mem, r, 12, 100)
+    assert asg == [0, 0, 0] and val == 0
+    asg, val = O.allocate_bruteforce(phi, mem, r, 2, 100)
+    assert asg is None
+    asg, val = O.allocate_bruteforce(phi, mem, [[3, 1]] * 3, 12, 5)   # time budget binds instead
+    assert asg == [0, 1, 1] and val == 10
+    asg, val = O.allocate_bruteforce(phi, mem, r, 12, 100, forbid=[[1, 0], [0, 0], [0, 0]])
+    assert asg == [1, 0, 0]
+
+
+def test_bruteforce_feasibility_and_monotonicity():
+    rng = np.random.default_rng(5)
+    for _ in range(20):
+        n, k = 5, 3
+        phi = rng.integers(0, 50, (n, k)).tolist()
+        mem = rng.integers(1, 20, (n, k)).tolist()
+        r = rng.integers(1, 10, (n, k)).tolist()
+        prev = None
+        for b in range(5, 100, 7):
+            asg, val = O.allocate_bruteforce(phi, mem, r, b, 30)
+            if asg is None:
+                assert prev is None
+                continue
+            assert sum(mem[i][c] for i, c in enumerate(asg)) <= b
+            assert sum(r[i][c] for i, c in enumerate(asg)) <= 30
+            assert prev is None or val <= prev        # optimum never worsens as the budget grows
+            prev = val
+
+
+def test_fixed_point_helpers():
+    assert O.phi_fixed(1.0) == 2 ** 30 and O.phi_fixed(-0.5) == -(2 ** 29)
+    assert O.phi_fixed(1.5 / 2 ** 30) == 2 and O.phi_fixed(2.5 / 2 ** 30) == 2     # ties to even
+    assert O.ratio_fixed(1.25) == 5 * 2 ** 18
+    assert O.time_cap_fixed(3, 1.1) == math.floor(3 * 1.1 * 2 ** 20)
+
+
+# ---------------------------------------------------------------- P10 update rules vs torch.optim (float64)
+
+def _torch_run(opt_ctor, theta0, grads):
+    p = torch.nn.Parameter(torch.from_numpy(theta0.copy()))
+    opt = opt_ctor([p])
+    for g in grads:
+        p.grad = torch.from_numpy(g.copy())
+        opt.step()
+    return p.detach().numpy()
+
+
+def _oracle_run(cfg, theta0, grads, rows, cols):
+    st = O.step_init(cfg, theta0.shape[0], rows, cols)
+    th = theta0.copy()
+    for g in grads:
+        th = O.step(th, g, st, cfg, rows, cols)
+    return th, st
+
+
+@pytest.mark.parametrize("wd,decoupled", [(0.0, 1), (0.05, 1), (0.05, 0)])
+def test_fp32_adam_path_matches_torch(wd, decoupled):
+    th0 = RNG.standard_normal(300)
+    gs = [RNG.standard_normal(300) for _ in range(6)]
+    cfg = O.Config(1, 1, decoupled, 0, 32, lr=3e-3, beta1=0.85, beta2=0.97, eps=1e-6, weight_decay=wd)
+    if decoupled:
+        ctor = lambda ps: torch.optim.AdamW(ps, lr=3e-3, betas=(0.85, 0.97), eps=1e-6, weight_decay=wd)
+    else:
+        ctor = lambda ps: torch.optim.Adam(ps, lr=3e-3, betas=(0.85, 0.97), eps=1e-6, weight_decay=wd)
+    got, _ = _oracle_run(cfg, th0, gs, 300, 1)
+    ref = _torch_run(ctor, th0, gs)
+    # torch folds the bias corrections into the step size and the denominator; same value up to rounding
+    np.testing.assert_allclose(got, ref, rtol=1e-10, atol=1e-13)
+
+
+def test_sgd_momentum_path_matches_torch():
+    th0 = RNG.standard_normal(200)
+    gs = [RNG.standard_normal(200) for _ in range(5)]
+    cfg = O.Config(0, 1, 0, 0, 32, lr=0.05, beta1=0.8, weight_decay=0.01)
+    got, _ = _oracle_run(cfg, th0, gs, 200, 1)
+    ref = _torch_run(lambda ps: torch.optim.SGD(ps, lr=0.05, momentum=0.8, weight_decay=0.01), th0, gs)
+    np.testing.assert_allclose(got, ref, rtol=1e-12, atol=1e-14)
+    # decoupled decay: theta shrinks by (1 - lr*wd) before the momentum step
+    cfg2 = O.Config(0, 1, 1, 0, 32, lr=0.05, beta1=0.8, weight_decay=0.01)
+    got2, _ = _oracle_run(cfg2, th0, gs[:1], 200, 1)
+    np.testing.assert_allclose(got2, th0 * (1 - 0.05 * 0.01) - 0.05 * gs[0], rtol=1e-13)
+
+
+def test_rms_path_is_adam_with_beta1_zero():
+    th0 = RNG.standard_normal(128)
+    gs = [RNG.standard_normal(128) for _ in range(5)]
+    cfg = O.Config(1, 0, 1, 0, 32, lr=1e-3, beta2=0.99, eps=1e-7, weight_decay=0.02)
+    got, st = _oracle_run(cfg, th0, gs, 128, 1)
+    ref = _torch_run(lambda ps: torch.optim.AdamW(ps, lr=1e-3, betas=(0.0, 0.99), eps=1e-7, weight_decay=0.02), th0, gs)
+    np.testing.assert_allclose(got, ref, rtol=1e-10, atol=1e-13)
+    assert st.m is None                                   # no first moment is stored
+
+
+# ---------------------------------------------------------------- P11 factored path
+
+def test_factored_equals_rms_when_squares_are_rank_one():
+    rows, cols = 24, 40
+    th0 = RNG.standard_normal(rows * cols)
+    x, y = RNG.random(rows) + 0.5, RNG.random(cols) + 0.5
+    gs = []
+    for _ in range(5):
+        sign = RNG.choice([-1.0, 1.0], size=(rows, cols))
+        gs.append((sign * np.outer(x, y)).reshape(-1))       # g^2 is the same rank-1 matrix each step
+    f = O.Config(1, 0, 1, 1, 32, lr=2e-3, beta2=0.98, eps=1e-9, weight_decay=0.01)
+    r = O.Config(1, 0, 1, 0, 32, lr=2e-3, beta2=0.98, eps=1e-9, weight_decay=0.01)
+    a, st = _oracle_run(f, th0, gs, rows, cols)
+    b, _ = _oracle_run(r, th0, gs, rows, cols)
+    np.testing.assert_allclose(a, b, rtol=1e-10, atol=1e-13)
+    assert st.r.shape == (rows,) and st.c.shape == (cols,)
+    with pytest.raises(ValueError):
+        O.step_init(f, 10, 10, 1)
+
+
+def test_factored_hand_example():
+    # one step, beta2 = 0: r = row means of g^2, c = column means, v = r c^T / mean(r)
+    g = np.array([[1.0, 2.0], [3.0, 4.0]])
+    cfg = O.Config(1, 0, 1, 1, 32, lr=1.0, beta2=0.0, eps=0.0, weight_decay=0.0)
+    th, st = _oracle_run(cfg, np.zeros(4), [g.reshape(-1)], 2, 2)
+    r = np.array([2.5, 12.5]); c = np.array([5.0, 10.0])
+    v = np.outer(r, c) / 7.5
+    np.testing.assert_allclose(st.r, r); np.testing.assert_allclose(st.c, c)
+    np.testing.assert_allclose(th, (-g / np.sqrt(v)).reshape(-1), rtol=1e-13)
+
+
+# ---------------------------------------------------------------- P12 8-bit path
+
+def test_int8_path_zero_gradient_decay_and_lr_zero():
+    n = 600
+    a = np.float32(0.5)
+    cfg = O.Config(1, 1, 1, 0, 8, lr=0.0, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
+    st = O.step_init(cfg, n, n, 1)
+    qm = RNG.integers(-127, 128, n); qm[0] = 127; qm[256] = 127; qm[512] = -127
+    qv = RNG.integers(0, 256, n); qv[0] = 255; qv[256] = 255; qv[512] = 255
+    st.qm, st.qv = qm.astype(np.int8), qv.astype(np.uint8)
+    st.am = np.full(3, a, np.float32); st.av = np.full(3, a, np.float32)
+    th0 = RNG.standard_normal(n)
+    th = O.step(th0, np.zeros(n), st, cfg, n, 1)
+    np.testing.assert_array_equal(th, th0)                           # lr = 0 leaves theta alone
+    # m -> 0.9 m; the new absmax is 0.9 a (rounded to fp32), so the codes are unchanged
+    np.testing.assert_array_equal(st.qm, qm.astype(np.int8))
+    np.testing.assert_array_equal(st.qv, qv.astype(np.uint8))
+    np.testing.assert_array_equal(st.am, np.full(3, np.float32(0.9 * float(a)), np.float32))
+    np.testing.assert_array_equal(st.av, np.full(3, np.float32(0.999 * float(a)), np.float32))
+
+
+def test_int8_path_tracks_fp32_path_within_one_code():
+    n = 2048
+    th0 = RNG.standard_normal(n) * 0.02
+    gs = [RNG.standard_normal(n) * 1e-2 for _ in range(4)]
+    c8 = O.Config(1, 1, 1, 0, 8, lr=1e-4, weight_decay=0.0)
+    c32 = O.Config(1, 1, 1, 0, 32, lr=1e-4, weight_decay=0.0)
+    # a single step from zero state: the 8-bit states are the quantised fp32 states exactly
+    _, s8 = _oracle_run(c8, th0, gs[:1], n, 1)
+    t32, s32 = _oracle_run(c32, th0, gs[:1], n, 1)
+    t8, _ = _oracle_run(c8, th0, gs[:1], n, 1)
+    np.testing.assert_allclose(t8, t32, rtol=1e-13)                  # theta uses un-requantised moments
+    qm, am = O.quantize8(s32.m, True); qv, av = O.quantize8(s32.v, False)
+    np.testing.assert_array_equal(s8.qm, qm); np.testing.assert_array_equal(s8.qv, qv)
+    np.testing.assert_array_equal(s8.am, am); np.testing.assert_array_equal(s8.av, av)
+    # second step: hand-computed from the dequantised state
+    m1 = O.dequantize8(qm, am, True); v1 = O.dequantize8(qv, av, False)
+    m2 = 0.9 * m1 + 0.1 * gs[1]; v2 = 0.999 * v1 + 0.001 * gs[1] ** 2
+    th2 = t8 - 1e-4 * (m2 / (1 - 0.9 ** 2)) / (np.sqrt(v2 / (1 - 0.999 ** 2)) + 1e-8)
+    got, s8b = _oracle_run(c8, th0, gs[:2], n, 1)
+    np.testing.assert_allclose(got, th2, rtol=1e-12)
+    q2, a2 = O.quantize8(m2, True)
+    np.testing.assert_array_equal(s8b.qm, q2); np.testing.assert_array_equal(s8b.am, a2)
+
+
+def test_config_kind_dispatch():
+    kinds = [O.config_kind(c) for c in O.default_configs()]
+    assert kinds == ["A32", "A8", "R", "F", "S"]
+    assert O.config_kind(O.Config(0, 0, 1, 0, 32)) == "unsupported"
