@@ -1,0 +1,245 @@
+/*
+ * baoc.h -- C ABI of the B200 (sm_100a) library for the data-parallel hot path
+ * of BAOC, the Budget-Aware Optimizer Configurator.
+ *
+ * The path: during a sampling window every parameter block's gradient is
+ * streamed once per step to update the block's statistics (Sec. 3.3, Eq. 3-8);
+ * at the end of the window the statistics are reduced to a risk matrix
+ * (Eq. 9, Appendix A Eq. 10-21); a budgeted allocation picks one configuration
+ * per block (Eq. 1-2); from then on one fused step updates every block under
+ * its own configuration (Definition 3.1, Algorithm 1 "Training").
+ *
+ * Conventions
+ *   - Every function returns an int status: 0 = BAOC_OK, negative = error,
+ *     positive = warning (result still valid).  baoc_last_error() returns a
+ *     message for the last non-zero status of a handle.
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA
+ *     global memory of the current device.  The library never allocates device
+ *     memory: it reports sizes, the caller allocates and passes pointers, and
+ *     keeps them alive while the handle uses them.
+ *   - Device pointers must be 16-byte aligned (BAOC_E_ALIGN otherwise).  Block
+ *     element counts are arbitrary (>= 1).
+ *   - All GPU work is queued on the caller's stream (a cudaStream_t passed as
+ *     baoc_stream_t; NULL is the default stream).  Only baoc_risk(),
+ *     baoc_read_stats() and baoc_nonfinite() wait for the stream, because they
+ *     return data to the host.
+ *   - A handle is not thread-safe.  Invalid arguments are rejected on the host
+ *     before anything is launched; no call can fault the device on bad input
+ *     that the host can see (null pointers, bad sizes, wrong call order).
+ *   - Gradients are bfloat16, parameters fp32, one contiguous array per block.
+ */
+#ifndef BAOC_H
+#define BAOC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct baoc_handle baoc_t;
+typedef void* baoc_stream_t;          /* a cudaStream_t */
+
+enum {
+    BAOC_OK = 0,
+    BAOC_E_INVALID = -1,     /* null pointer, bad size, bad value */
+    BAOC_E_ALIGN = -2,       /* a device pointer is not 16-byte aligned */
+    BAOC_E_STATE = -3,       /* call order: e.g. step before configure */
+    BAOC_E_INFEASIBLE = -4,  /* no assignment satisfies both budgets and the mask */
+    BAOC_E_CUDA = -5,        /* a CUDA runtime call failed (message has the reason) */
+    BAOC_E_NONFINITE = -6,   /* reserved */
+    BAOC_E_WORKSPACE = -7,   /* workspace or state buffer too small */
+    BAOC_W_NODE_LIMIT = 1    /* allocator hit its node limit: assignment feasible, optimality not proven */
+};
+
+/* One parameter block B_i (Sec. 3.1): numel = d_i parameters viewed as a
+ * rows x cols row-major matrix.  A vector has rows = numel, cols = 1; tensors
+ * of more than two dimensions are flattened to (dim0, rest). rows*cols == numel. */
+typedef struct {
+    int64_t numel;
+    int32_t rows, cols;
+} baoc_block_t;
+
+/* A configuration tuple c = (y_a, y_m, y_d, y_f, b) of Definition 3.1 and the
+ * hyper-parameters of the update rule it selects.  Tuples the library can
+ * instantiate:  (1,1,*,0,32) fp32 Adam/AdamW;  (1,1,*,0,8) Adam/AdamW with
+ * block-wise absmax 8-bit states;  (1,0,*,0,32) momentum-free RMS scaling;
+ * (1,0,*,1,32) factored second moment (matrix blocks only);  (0,1,*,0,32) SGD
+ * with momentum (beta1 is the momentum coefficient).  Other tuples may appear
+ * in the candidate set for risk and cost queries but cannot be assigned. */
+typedef struct {
+    uint8_t adaptive, momentum, decoupled_wd, factored, bits;
+    uint8_t reserved[3];
+    float lr, beta1, beta2, eps, weight_decay;
+} baoc_config_t;
+
+/* Options of the statistics, normalisation and allocation (defaults from
+ * baoc_default_opts: Eq. 3 "standard Adam values", Appendix A anchors,
+ * gamma = 0.1).  qblock must be 256. */
+typedef struct {
+    double beta_m, beta_v;        /* Eq. 3 */
+    double beta_rho;              /* Eq. 5 smoothing factor */
+    double eps;                   /* Appendix A.1: 1e-12 */
+    double a_lo, a_hi;            /* Eq. 11 */
+    double rho_lo, rho_hi;        /* Eq. 13 */
+    double snr_lo, snr_hi;        /* Eq. 15 */
+    double w[5];                  /* user weights W: w_A, w_M, w_C, w_F, w_Q */
+    double gamma;                 /* weight of Agg(c) in the objective */
+    double eps_adam;              /* epsilon of the update direction in Eq. 8 */
+    int32_t use_snr;              /* Eq. 17; 0 selects s_M = s_rho */
+    int32_t qblock;               /* elements per 8-bit quantisation block */
+    int64_t node_limit;           /* allocator search-node limit (0 = default) */
+} baoc_opts_t;
+
+/* Per-block diagnostics z_i: raw (Eq. 4-8), normalised (Eq. 10-20) and a few
+ * extras that are not used by the risk. */
+typedef struct {
+    double A, rho_bar, snr, C, F, Q32, Q16, Q8;
+    double q10, q90;              /* the two quantiles of Eq. 4 */
+    double rho_mom;               /* EMA of cos(g_t, m_{t-1}) */
+    double err_m8, err_v8, err_m16, err_v16;   /* ||x - Q_b(x)|| / ||x|| */
+    double s_A, s_rho, s_snr, s_M, C_tilde, s_F, lQ32, lQ16, lQ8;
+    double last_cos;              /* cosine of the last step */
+    int64_t n_cos;                /* number of cosines averaged into rho_bar */
+} baoc_block_stats_t;
+
+typedef struct {
+    int32_t n_blocks, n_cfg;
+    int64_t numel;                /* sum of d_i */
+    int64_t n_tiles;              /* tiles of the statistics pass */
+    int64_t stats_steps;          /* gradient observations so far in this window */
+    int64_t state_bytes;          /* StateMem of the configured assignment (0 before configure) */
+    int64_t kernel_launches;      /* kernels this handle has launched so far */
+    int64_t stats_bytes_per_call; /* algorithmic HBM bytes of one baoc_sample_stats */
+    int64_t step_bytes_per_call;  /* algorithmic HBM bytes of one baoc_step under the assignment */
+} baoc_info_t;
+
+/* Fill *o with the defaults.  Host only. */
+void baoc_default_opts(baoc_opts_t* o);
+
+/* Create a handle for n_blocks blocks and n_cfg candidate configurations
+ * (Algorithm 1 inputs).  Copies all arrays.  opts may be NULL (defaults).
+ * Host only; touches no GPU.  Errors: BAOC_E_INVALID (null, n <= 0,
+ * rows*cols != numel, n_cfg > 32, bits not in {8,16,32}, qblock != 256). */
+int baoc_create(baoc_t** h, int n_blocks, const baoc_block_t* blocks,
+                int n_cfg, const baoc_config_t* cfgs, const baoc_opts_t* opts);
+
+/* Free the handle (host memory only; device buffers belong to the caller). */
+void baoc_destroy(baoc_t* h);
+
+/* Message of the last error on this handle ("" if none).  Never NULL. */
+const char* baoc_last_error(const baoc_t* h);
+
+/* Fill *info.  Host only. */
+int baoc_query(const baoc_t* h, baoc_info_t* info);
+
+/* ---- sampling window (Algorithm 1 "Warmup and diagnostics") -------------- */
+
+/* Bytes of device workspace the statistics need: the EMA moments of Eq. 3
+ * (fp32), the previous gradient (bf16), per-tile partial sums, per-block
+ * accumulators, tables and the scratch of the finalize pass. */
+int baoc_stats_workspace_bytes(const baoc_t* h, size_t* bytes);
+
+/* Give the handle its statistics workspace (device, >= the size above,
+ * 256-byte aligned).  Queues the zero-fill of the moments and the upload of
+ * the tile tables on the stream and starts a new window. */
+int baoc_bind_stats_workspace(baoc_t* h, void* dev, size_t bytes, baoc_stream_t stream);
+
+/* One gradient observation of every block (Eq. 3 and the cosine of Eq. 5).
+ * grads: host array of n_blocks device pointers to bf16 gradients (block i has
+ * numel_i elements).  The sample is dense: every coordinate of every block.
+ * Queues one streaming kernel and one small combine kernel; does not wait. */
+int baoc_sample_stats(baoc_t* h, const void* const* grads, baoc_stream_t stream);
+
+/* Copy the running per-block values of the window (rho_bar, last_cos, n_cos,
+ * rho_mom; other fields zero) to host stats_out[n_blocks].  Waits. */
+int baoc_read_stats(baoc_t* h, baoc_block_stats_t* stats_out, baoc_stream_t stream);
+
+/* End of the window: finalize the diagnostics (Eq. 4-8) on the device, copy
+ * them to the host, normalise them (Eq. 10-20) and fill the risk matrix
+ * R_i(c) (Eq. 9).  params: host array of n_blocks device pointers to fp32
+ * parameters (used by Eq. 6).  risk_out: host [n_blocks*n_cfg], row-major by
+ * block.  stats_out: host [n_blocks] or NULL.  Waits for the stream.
+ * BAOC_E_STATE if no gradient has been observed. */
+int baoc_risk(baoc_t* h, const float* const* params, double* risk_out,
+              baoc_block_stats_t* stats_out, baoc_stream_t stream);
+
+/* Host-only part of baoc_risk: read the raw fields of stats[i] (A, rho_bar,
+ * snr, C, F, Q32, Q16, Q8), fill their normalised fields in place and write
+ * risk_out[n_blocks*n_cfg].  No GPU needed. */
+int baoc_risk_from_raw(const baoc_t* h, baoc_block_stats_t* stats, double* risk_out);
+
+/* ---- allocation (Algorithm 1 "Allocation", Eq. 1-2) ---------------------- */
+
+/* Cost model.  mem_bytes[i*n_cfg+c] = M_{i,c}, the persistent state bytes of
+ * block i under configuration c (StateMem definition, Sec. 3.1; padding
+ * excluded).  time_ratio[i*n_cfg+c] = algorithmic HBM bytes per parameter of
+ * c divided by those of fp32 Adam, a stand-in for the measured r_{i,c}.
+ * Either output may be NULL.  Host only. */
+int baoc_cost_model(const baoc_t* h, int64_t* mem_bytes, double* time_ratio);
+
+/* Solve Eq. 2 exactly on the host: minimise sum_i Phi_{i,c_i} with
+ * Phi = (R - pref) + gamma*Agg(c) subject to sum M <= b_mem and
+ * (1/N) sum r <= b_time, one configuration per block.  Arithmetic is fixed
+ * point: Phi -> rne(Phi*2^30), r -> rne(r*2^20), time cap floor(N*b_time*2^20);
+ * among optimal assignments the lexicographically smallest (block 0 first,
+ * lower configuration index first) is returned.  forbid[i*n_cfg+c] != 0
+ * excludes a pair (hard constraint); pairs the library cannot instantiate
+ * (factored on a vector block, unsupported tuples) are excluded as well.
+ * forbid, pref, objective_out may be NULL.  All arrays host.  Returns
+ * BAOC_E_INFEASIBLE when nothing fits, BAOC_W_NODE_LIMIT when the search
+ * stopped early (assignment feasible but not proven optimal). */
+int baoc_allocate(baoc_t* h, const double* risk, const int64_t* mem_bytes,
+                  const double* time_ratio, int64_t b_mem, double b_time,
+                  const uint8_t* forbid, const double* pref,
+                  int32_t* assign_out, double* objective_out);
+
+/* ---- training (Algorithm 1 "Training") ----------------------------------- */
+
+/* Bytes of device memory the optimizer state of this assignment needs
+ * (states plus alignment padding, tables and the scratch of the factored
+ * path).  assign: host [n_blocks]. */
+int baoc_state_bytes(const baoc_t* h, const int32_t* assign, size_t* bytes);
+
+/* Instantiate the optimizer O({c_i}): lay the states out in state_dev
+ * (device, 256-byte aligned, >= baoc_state_bytes), queue their zero-fill and
+ * the upload of the tile table.  The step counter restarts. */
+int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes,
+                   baoc_stream_t stream);
+
+/* One training step of every block under its configuration.  grads / params:
+ * host arrays of n_blocks device pointers (bf16 / fp32).  step_t: 1-based step
+ * number (bias corrections).  Queues the fused update kernel (preceded by the
+ * row/column reduction kernels when some block is factored); does not wait. */
+int baoc_step(baoc_t* h, const void* const* grads, float* const* params,
+              int64_t step_t, baoc_stream_t stream);
+
+/* End-to-end convenience for callers whose gradients live in host memory:
+ * copies block i's bf16 gradient from host_grads[i] (pinned memory advised) to
+ * the device buffer dev_grads[i], then does baoc_sample_stats (if do_stats)
+ * and baoc_step (if step_t > 0) on the same stream.  Does not wait. */
+int baoc_step_from_host(baoc_t* h, const void* const* host_grads, void* const* dev_grads,
+                        float* const* params, int do_stats, int64_t step_t,
+                        baoc_stream_t stream);
+
+/* Where a block's window or optimizer state lives, for inspection,
+ * checkpointing and tests.  which: 0 = EMA first moment (fp32), 1 = EMA second
+ * moment (fp32), 2 = previous gradient (bf16) of the statistics workspace;
+ * 10..13 = the block's optimizer state tensors under the configured
+ * assignment: fp32 Adam m, v; 8-bit Adam codes of m (int8), codes of v (uint8),
+ * absmax of m (fp32), absmax of v (fp32); RMS v; SGD m; factored r (rows), c
+ * (cols).  Writes the device pointer, the element count and the element size
+ * in bytes; BAOC_E_INVALID if the block has no such tensor, BAOC_E_STATE if the
+ * buffer is not bound yet.  Host only. */
+int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* count, int32_t* elem_bytes);
+
+/* Number of blocks whose last fused step saw a non-finite gradient or
+ * produced a non-finite parameter; flags[n_blocks] (host, may be NULL) gets
+ * one byte per block.  Waits. */
+int baoc_nonfinite(baoc_t* h, uint8_t* flags, int32_t* count, baoc_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BAOC_H */

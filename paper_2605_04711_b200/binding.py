@@ -1,0 +1,277 @@
+"""Thin Python binding of the C ABI in ``include/baoc.h``.
+
+Argument marshalling only: every step of the path runs in the CUDA library.
+PyTorch supplies device memory and the stream.  The names follow the C entry
+points (``baoc_create`` -> ``Baoc(...)``, ``baoc_sample_stats`` ->
+``Baoc.sample_stats`` and so on).  There is no CPU fallback: if the shared
+library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbaoc.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build the CUDA library first "
+        "(python -m paper_2605_04711_b200.build); there is no fallback path")
+
+_lib = C.CDLL(LIB_PATH)
+
+OK, E_INVALID, E_ALIGN, E_STATE, E_INFEASIBLE, E_CUDA, E_NONFINITE, E_WORKSPACE = 0, -1, -2, -3, -4, -5, -6, -7
+W_NODE_LIMIT = 1
+
+
+class BaocError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"baoc error {code}: {msg}")
+        self.code = code
+
+
+class Block(C.Structure):
+    _fields_ = [("numel", C.c_int64), ("rows", C.c_int32), ("cols", C.c_int32)]
+
+
+class Config(C.Structure):
+    _fields_ = [("adaptive", C.c_uint8), ("momentum", C.c_uint8), ("decoupled_wd", C.c_uint8),
+                ("factored", C.c_uint8), ("bits", C.c_uint8), ("reserved", C.c_uint8 * 3),
+                ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float)]
+
+
+class Opts(C.Structure):
+    _fields_ = [("beta_m", C.c_double), ("beta_v", C.c_double), ("beta_rho", C.c_double), ("eps", C.c_double),
+                ("a_lo", C.c_double), ("a_hi", C.c_double), ("rho_lo", C.c_double), ("rho_hi", C.c_double),
+                ("snr_lo", C.c_double), ("snr_hi", C.c_double), ("w", C.c_double * 5), ("gamma", C.c_double),
+                ("eps_adam", C.c_double), ("use_snr", C.c_int32), ("qblock", C.c_int32), ("node_limit", C.c_int64)]
+
+
+class BlockStats(C.Structure):
+    _fields_ = [(n, C.c_double) for n in
+                ("A", "rho_bar", "snr", "C", "F", "Q32", "Q16", "Q8", "q10", "q90", "rho_mom",
+                 "err_m8", "err_v8", "err_m16", "err_v16",
+                 "s_A", "s_rho", "s_snr", "s_M", "C_tilde", "s_F", "lQ32", "lQ16", "lQ8", "last_cos")] + \
+               [("n_cos", C.c_int64)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class Info(C.Structure):
+    _fields_ = [("n_blocks", C.c_int32), ("n_cfg", C.c_int32), ("numel", C.c_int64), ("n_tiles", C.c_int64),
+                ("stats_steps", C.c_int64), ("state_bytes", C.c_int64), ("kernel_launches", C.c_int64),
+                ("stats_bytes_per_call", C.c_int64), ("step_bytes_per_call", C.c_int64)]
+
+
+EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error", "baoc_query",
+           "baoc_stats_workspace_bytes", "baoc_bind_stats_workspace", "baoc_sample_stats", "baoc_read_stats",
+           "baoc_risk", "baoc_risk_from_raw", "baoc_cost_model", "baoc_allocate", "baoc_state_bytes",
+           "baoc_configure", "baoc_step", "baoc_step_from_host", "baoc_view", "baoc_nonfinite"]
+
+_vp = C.c_void_p
+_lib.baoc_default_opts.argtypes = [C.POINTER(Opts)]
+_lib.baoc_default_opts.restype = None
+_lib.baoc_create.argtypes = [C.POINTER(_vp), C.c_int, C.POINTER(Block), C.c_int, C.POINTER(Config), C.POINTER(Opts)]
+_lib.baoc_destroy.argtypes = [_vp]
+_lib.baoc_destroy.restype = None
+_lib.baoc_last_error.argtypes = [_vp]
+_lib.baoc_last_error.restype = C.c_char_p
+_lib.baoc_query.argtypes = [_vp, C.POINTER(Info)]
+_lib.baoc_stats_workspace_bytes.argtypes = [_vp, C.POINTER(C.c_size_t)]
+_lib.baoc_bind_stats_workspace.argtypes = [_vp, _vp, C.c_size_t, _vp]
+_lib.baoc_sample_stats.argtypes = [_vp, _vp, _vp]
+_lib.baoc_read_stats.argtypes = [_vp, C.POINTER(BlockStats), _vp]
+_lib.baoc_risk.argtypes = [_vp, _vp, _vp, C.POINTER(BlockStats), _vp]
+_lib.baoc_risk_from_raw.argtypes = [_vp, C.POINTER(BlockStats), _vp]
+_lib.baoc_cost_model.argtypes = [_vp, _vp, _vp]
+_lib.baoc_allocate.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_double, _vp, _vp, _vp, C.POINTER(C.c_double)]
+_lib.baoc_state_bytes.argtypes = [_vp, _vp, C.POINTER(C.c_size_t)]
+_lib.baoc_configure.argtypes = [_vp, _vp, _vp, C.c_size_t, _vp]
+_lib.baoc_step.argtypes = [_vp, _vp, _vp, C.c_int64, _vp]
+_lib.baoc_step_from_host.argtypes = [_vp, _vp, _vp, _vp, C.c_int, C.c_int64, _vp]
+_lib.baoc_view.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(_vp), C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
+_lib.baoc_nonfinite.argtypes = [_vp, _vp, C.POINTER(C.c_int32), _vp]
+
+
+def default_opts() -> Opts:
+    o = Opts()
+    _lib.baoc_default_opts(C.byref(o))
+    return o
+
+
+def make_config(adaptive, momentum, decoupled_wd, factored, bits, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8,
+                weight_decay=0.0) -> Config:
+    return Config(adaptive, momentum, decoupled_wd, factored, bits, (C.c_uint8 * 3)(), lr, beta1, beta2, eps,
+                  weight_decay)
+
+
+def default_configs() -> List[Config]:
+    """fp32 AdamW, 8-bit AdamW, momentum-free RMS scaling, factored second moment, SGD with momentum."""
+    return [make_config(1, 1, 1, 0, 32, weight_decay=0.01), make_config(1, 1, 1, 0, 8, weight_decay=0.01),
+            make_config(1, 0, 1, 0, 32, weight_decay=0.01), make_config(1, 0, 1, 1, 32, weight_decay=0.01),
+            make_config(0, 1, 1, 0, 32, lr=1e-2, weight_decay=0.01)]
+
+
+def pointer_table(tensors: Sequence[torch.Tensor]):
+    """Host array of the tensors' data pointers, in the layout the C calls take."""
+    return (C.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else 0
+
+
+def _np_ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data
+
+
+class Baoc:
+    """One handle of the library (``baoc_create`` .. ``baoc_destroy``)."""
+
+    def __init__(self, blocks: Sequence, configs: Sequence[Config], opts: Optional[Opts] = None):
+        """blocks: objects with ``numel``, ``rows``, ``cols`` (or 3-tuples)."""
+        bl = []
+        for b in blocks:
+            if isinstance(b, (tuple, list)):
+                bl.append(Block(*b))
+            else:
+                bl.append(Block(b.numel, b.rows, b.cols))
+        self.n_blocks, self.n_cfg = len(bl), len(configs)
+        self._blocks = (Block * len(bl))(*bl)
+        self._cfgs = (Config * len(configs))(*configs)
+        self._h = _vp()
+        self._keep = []            # device buffers the handle points into
+        rc = _lib.baoc_create(C.byref(self._h), len(bl), self._blocks, len(configs), self._cfgs,
+                              C.byref(opts) if opts is not None else None)
+        if rc != 0:
+            raise BaocError(rc, "baoc_create rejected its arguments")
+
+    def close(self):
+        if getattr(self, "_h", None) and _lib is not None:
+            _lib.baoc_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def _check(self, rc: int) -> int:
+        if rc < 0:
+            raise BaocError(rc, _lib.baoc_last_error(self._h).decode())
+        return rc
+
+    def last_error(self) -> str:
+        return _lib.baoc_last_error(self._h).decode()
+
+    def query(self) -> Info:
+        info = Info()
+        self._check(_lib.baoc_query(self._h, C.byref(info)))
+        return info
+
+    # ---- sampling window --------------------------------------------------
+    def stats_workspace_bytes(self) -> int:
+        n = C.c_size_t()
+        self._check(_lib.baoc_stats_workspace_bytes(self._h, C.byref(n)))
+        return n.value
+
+    def bind_stats_workspace(self, ws: torch.Tensor):
+        self._check(_lib.baoc_bind_stats_workspace(self._h, ws.data_ptr(), ws.numel() * ws.element_size(), _stream()))
+        self._keep.append(ws)
+
+    def sample_stats(self, grads):
+        """grads: list of bf16 device tensors, or a table from ``pointer_table``."""
+        tab = grads if isinstance(grads, C.Array) else pointer_table(grads)
+        self._check(_lib.baoc_sample_stats(self._h, tab, _stream()))
+
+    def read_stats(self) -> List[dict]:
+        out = (BlockStats * self.n_blocks)()
+        self._check(_lib.baoc_read_stats(self._h, out, _stream()))
+        return [s.as_dict() for s in out]
+
+    def risk(self, params):
+        """Returns (risk [n_blocks, n_cfg] float64, list of per-block stats dicts)."""
+        tab = params if isinstance(params, C.Array) else pointer_table(params)
+        risk = np.zeros((self.n_blocks, self.n_cfg), np.float64)
+        st = (BlockStats * self.n_blocks)()
+        self._check(_lib.baoc_risk(self._h, tab, risk.ctypes.data, st, _stream()))
+        return risk, [s.as_dict() for s in st]
+
+    def risk_from_raw(self, raw: Sequence[dict]):
+        st = (BlockStats * self.n_blocks)()
+        for i, r in enumerate(raw):
+            for k in ("A", "rho_bar", "snr", "C", "F", "Q32", "Q16", "Q8"):
+                setattr(st[i], k, float(r[k]))
+        risk = np.zeros((self.n_blocks, self.n_cfg), np.float64)
+        self._check(_lib.baoc_risk_from_raw(self._h, st, risk.ctypes.data))
+        return risk, [s.as_dict() for s in st]
+
+    # ---- allocation -------------------------------------------------------
+    def cost_model(self):
+        mem = np.zeros((self.n_blocks, self.n_cfg), np.int64)
+        ratio = np.zeros((self.n_blocks, self.n_cfg), np.float64)
+        self._check(_lib.baoc_cost_model(self._h, mem.ctypes.data, ratio.ctypes.data))
+        return mem, ratio
+
+    def allocate(self, risk, mem, ratio, b_mem: int, b_time: float, forbid=None, pref=None):
+        """Returns (assignment int32[n_blocks], objective, status) with status 0 or W_NODE_LIMIT."""
+        risk = np.ascontiguousarray(risk, np.float64)
+        mem = np.ascontiguousarray(mem, np.int64)
+        ratio = np.ascontiguousarray(ratio, np.float64)
+        forbid = None if forbid is None else np.ascontiguousarray(forbid, np.uint8)
+        pref = None if pref is None else np.ascontiguousarray(pref, np.float64)
+        asg = np.zeros(self.n_blocks, np.int32)
+        obj = C.c_double()
+        rc = self._check(_lib.baoc_allocate(self._h, risk.ctypes.data, mem.ctypes.data, ratio.ctypes.data, int(b_mem),
+                                            float(b_time), _np_ptr(forbid), _np_ptr(pref), asg.ctypes.data, C.byref(obj)))
+        return asg, obj.value, rc
+
+    # ---- training ---------------------------------------------------------
+    def state_bytes(self, assign) -> int:
+        a = np.ascontiguousarray(assign, np.int32)
+        n = C.c_size_t()
+        self._check(_lib.baoc_state_bytes(self._h, a.ctypes.data, C.byref(n)))
+        return n.value
+
+    def configure(self, assign, state: torch.Tensor):
+        a = np.ascontiguousarray(assign, np.int32)
+        self._check(_lib.baoc_configure(self._h, a.ctypes.data, state.data_ptr(), state.numel() * state.element_size(),
+                                        _stream()))
+        self._keep.append(state)
+
+    def step(self, grads, params, step_t: int):
+        g = grads if isinstance(grads, C.Array) else pointer_table(grads)
+        p = params if isinstance(params, C.Array) else pointer_table(params)
+        self._check(_lib.baoc_step(self._h, g, p, int(step_t), _stream()))
+
+    def step_from_host(self, host_grads, dev_grads, params, do_stats: bool, step_t: int):
+        hg = host_grads if isinstance(host_grads, C.Array) else pointer_table(host_grads)
+        dg = dev_grads if isinstance(dev_grads, C.Array) else pointer_table(dev_grads)
+        p = None if params is None else (params if isinstance(params, C.Array) else pointer_table(params))
+        self._check(_lib.baoc_step_from_host(self._h, hg, dg, p, int(bool(do_stats)), int(step_t), _stream()))
+
+    def view(self, block: int, which: int):
+        """(device pointer, element count, element bytes) of a state tensor (see ``baoc_view``)."""
+        p, n, eb = _vp(), C.c_int64(), C.c_int32()
+        self._check(_lib.baoc_view(self._h, block, which, C.byref(p), C.byref(n), C.byref(eb)))
+        return p.value, n.value, eb.value
+
+    def view_tensor(self, block: int, which: int, dtype: torch.dtype) -> torch.Tensor:
+        """A state tensor as a torch view (no copy) into the buffer the caller bound."""
+        p, n, eb = self.view(block, which)
+        for buf in self._keep:
+            base = buf.data_ptr()
+            if base <= p < base + buf.numel() * buf.element_size():
+                flat = buf.view(torch.uint8).reshape(-1)
+                return flat[p - base: p - base + n * eb].view(dtype)
+        raise BaocError(E_STATE, "the tensor lies in no buffer bound through this object")
+
+    def nonfinite(self):
+        flags = np.zeros(self.n_blocks, np.uint8)
+        cnt = C.c_int32()
+        self._check(_lib.baoc_nonfinite(self._h, flags.ctypes.data, C.byref(cnt), _stream()))
+        return cnt.value, flags

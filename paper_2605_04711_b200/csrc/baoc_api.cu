@@ -1,0 +1,408 @@
+// GPU-facing entry points of the C ABI: workspace binding, the sampling-window
+// calls, the end-of-window risk, optimizer instantiation and the fused step.
+// Every argument is validated on the host before anything is queued.
+#include <cmath>
+#include <cstring>
+#include <cuda_runtime.h>
+
+#include "baoc_internal.h"
+
+using namespace baoc;
+
+namespace {
+
+int cuda_fail(const Handle* h, const char* what, cudaError_t e) {
+    return fail(h, BAOC_E_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+int launch_fail(const Handle* h, const char* what, int code) {
+    return fail(h, BAOC_E_CUDA, std::string(what) + ": " + cudaGetErrorString(cudaError_t(code)));
+}
+
+#define CU(call, what)                                        \
+    do {                                                      \
+        cudaError_t e_ = (call);                              \
+        if (e_ != cudaSuccess) return cuda_fail(h, what, e_); \
+    } while (0)
+#define LAUNCH(call, what)                              \
+    do {                                                \
+        int r_ = (call);                                \
+        if (r_ != 0) return launch_fail(h, what, r_);   \
+    } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Check a host array of device pointers; upload it when it differs from the
+// copy the device already has.
+int sync_pointer_table(Handle* h, const void* const* ptrs, std::vector<const void*>* cache, void* dev_table,
+                       cudaStream_t s, const char* what) {
+    const int n = h->n_blocks;
+    for (int i = 0; i < n; ++i) {
+        if (!ptrs[i]) return fail(h, BAOC_E_INVALID, std::string(what) + ": null block pointer");
+        if (!aligned16(ptrs[i])) return fail(h, BAOC_E_ALIGN, std::string(what) + ": block pointer not 16-byte aligned");
+    }
+    if (cache->size() == size_t(n) && std::memcmp(cache->data(), ptrs, sizeof(void*) * n) == 0) return BAOC_OK;
+    cache->assign(ptrs, ptrs + n);
+    CU(cudaMemcpyAsync(dev_table, cache->data(), sizeof(void*) * n, cudaMemcpyHostToDevice, s), what);
+    return BAOC_OK;
+}
+
+template <typename T>
+T* at(char* base, size_t off) { return reinterpret_cast<T*>(base + off); }
+
+int do_sample_stats(Handle* h, const void* const* grads, cudaStream_t s) {
+    int rc = sync_pointer_table(h, grads, &h->last_stat_grads, h->ws + h->sl.grads, s, "baoc_sample_stats");
+    if (rc) return rc;
+    const auto& L = h->sl;
+    LAUNCH(launch_stats_step(at<StatBlock>(h->ws, L.blocks), at<Tile>(h->ws, L.tiles),
+                             at<const void*>(h->ws, L.grads), at<double>(h->ws, L.partials), h->n_stat_tiles,
+                             float(h->opts.beta_m), float(h->opts.beta_v), s), "stats_step_kernel");
+    LAUNCH(launch_stats_combine(at<StatBlock>(h->ws, L.blocks), at<double>(h->ws, L.partials), at<double>(h->ws, L.acc),
+                                h->n_blocks, h->stats_steps > 0 ? 1 : 0, h->opts.beta_rho, h->opts.eps, s),
+           "stats_combine_kernel");
+    h->launches += 2;
+    h->stats_steps += 1;
+    return BAOC_OK;
+}
+
+void fill_step_params(const Handle* h, int64_t t, StepParams* P) {
+    std::memset(P, 0, sizeof(*P));
+    for (int c = 0; c < h->n_cfg; ++c) {
+        const baoc_config_t& k = h->cfgs[c];
+        CfgStep& o = P->c[c];
+        o.lr = k.lr; o.beta1 = k.beta1; o.beta2 = k.beta2; o.eps = k.eps; o.wd = k.weight_decay;
+        const bool has_wd = k.weight_decay != 0.0f;
+        o.coupled = (has_wd && !k.decoupled_wd) ? 1 : 0;
+        o.decay = (has_wd && k.decoupled_wd) ? -float(double(k.lr) * double(k.weight_decay)) : 0.0f;
+        o.bc1 = float(1.0 - std::pow(double(k.beta1), double(t)));
+        o.bc2 = float(1.0 - std::pow(double(k.beta2), double(t)));
+        o.beta1_d = double(k.beta1); o.beta2_d = double(k.beta2);
+    }
+}
+
+int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t, cudaStream_t s) {
+    int rc = sync_pointer_table(h, grads, &h->last_step_grads, h->st + h->tl.grads, s, "baoc_step (grads)");
+    if (rc) return rc;
+    rc = sync_pointer_table(h, reinterpret_cast<const void* const*>(params), &h->last_step_params, h->st + h->tl.params, s,
+                            "baoc_step (params)");
+    if (rc) return rc;
+    StepParams P;
+    fill_step_params(h, t, &P);
+    const auto& L = h->tl;
+    CU(cudaMemsetAsync(h->st + L.flags, 0, 4 * size_t(h->n_blocks), s), "baoc_step (flags)");
+    if (h->n_factored > 0) {
+        LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles),
+                                      at<int32_t>(h->st, L.f_ids), at<const void*>(h->st, L.grads), h->n_step_red_tiles,
+                                      h->n_factored, P, s), "factored_reduce_kernel");
+        h->launches += 2;
+    }
+    LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles), at<const void*>(h->st, L.grads),
+                             at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), h->n_step_tiles, P, s),
+           "fused_step_kernel");
+    h->launches += 1;
+    return BAOC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int baoc_stats_workspace_bytes(const baoc_t* h, size_t* bytes) {
+    if (!h || !bytes) return BAOC_E_INVALID;
+    *bytes = h->sl.total;
+    return BAOC_OK;
+}
+
+int baoc_bind_stats_workspace(baoc_t* h, void* dev, size_t bytes, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!dev) return fail(h, BAOC_E_INVALID, "baoc_bind_stats_workspace: null workspace");
+    if (reinterpret_cast<uintptr_t>(dev) & 255u) return fail(h, BAOC_E_ALIGN, "baoc_bind_stats_workspace: workspace not 256-byte aligned");
+    if (bytes < h->sl.total) return fail(h, BAOC_E_WORKSPACE, "baoc_bind_stats_workspace: workspace too small");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const auto& L = h->sl;
+    char* ws = static_cast<char*>(dev);
+    const int n = h->n_blocks;
+
+    std::vector<StatBlock> sb = h->h_stat_blocks;
+    std::vector<Tile> tiles;
+    std::vector<RedTile> red;
+    std::vector<int32_t> ids;
+    tiles.reserve(size_t(h->n_stat_tiles));
+    for (int i = 0; i < n; ++i) {
+        StatBlock& b = sb[i];
+        b.m = reinterpret_cast<float*>(ws + L.m + reinterpret_cast<size_t>(b.m));
+        b.v = reinterpret_cast<float*>(ws + L.v + reinterpret_cast<size_t>(b.v));
+        b.gprev = reinterpret_cast<uint16_t*>(ws + L.gprev + reinterpret_cast<size_t>(b.gprev));
+        for (int k = 0; k < b.ntiles; ++k) tiles.push_back(Tile{uint32_t(i), uint32_t(k)});
+        if (b.cols > 1) {
+            b.rowsum = reinterpret_cast<double*>(ws + L.rowsum + reinterpret_cast<size_t>(b.rowsum));
+            b.colsum = reinterpret_cast<double*>(ws + L.colsum + reinterpret_cast<size_t>(b.colsum));
+            b.red.rowpart = reinterpret_cast<double*>(ws + L.redpart + reinterpret_cast<size_t>(b.red.rowpart));
+            b.red.colpart = reinterpret_cast<double*>(ws + L.redpart + reinterpret_cast<size_t>(b.red.colpart));
+            for (int ch = 0; ch < b.red.chunks; ++ch)
+                for (int st = 0; st < b.red.strips; ++st) red.push_back(RedTile{uint32_t(i), uint32_t(ch), uint32_t(st), 0});
+            ids.push_back(i);
+        }
+    }
+    h->n_matrix = int(ids.size());
+    CU(cudaMemcpyAsync(ws + L.blocks, sb.data(), sizeof(StatBlock) * n, cudaMemcpyHostToDevice, s), "upload block table");
+    CU(cudaMemcpyAsync(ws + L.tiles, tiles.data(), sizeof(Tile) * tiles.size(), cudaMemcpyHostToDevice, s), "upload tile table");
+    if (!red.empty())
+        CU(cudaMemcpyAsync(ws + L.red_tiles, red.data(), sizeof(RedTile) * red.size(), cudaMemcpyHostToDevice, s), "upload reduction table");
+    if (!ids.empty())
+        CU(cudaMemcpyAsync(ws + L.matrix_ids, ids.data(), 4 * ids.size(), cudaMemcpyHostToDevice, s), "upload matrix ids");
+    // moments, previous gradient and running values start at zero
+    CU(cudaMemsetAsync(ws + L.m, 0, L.partials - L.m, s), "zero moments");
+    CU(cudaMemsetAsync(ws + L.acc, 0, 8 * size_t(kBlockAcc) * n, s), "zero accumulators");
+    h->ws = ws; h->ws_bytes = bytes; h->ws_bound = true;
+    h->stats_steps = 0;
+    h->last_stat_grads.clear(); h->last_stat_params.clear();
+    return BAOC_OK;
+}
+
+int baoc_sample_stats(baoc_t* h, const void* const* grads, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!grads) return fail(h, BAOC_E_INVALID, "baoc_sample_stats: null gradient table");
+    if (!h->ws_bound) return fail(h, BAOC_E_STATE, "baoc_sample_stats: no statistics workspace bound");
+    return do_sample_stats(h, grads, static_cast<cudaStream_t>(stream));
+}
+
+int baoc_read_stats(baoc_t* h, baoc_block_stats_t* out, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!out) return fail(h, BAOC_E_INVALID, "baoc_read_stats: null output");
+    if (!h->ws_bound) return fail(h, BAOC_E_STATE, "baoc_read_stats: no statistics workspace bound");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<double> acc(size_t(kBlockAcc) * h->n_blocks);
+    CU(cudaMemcpyAsync(acc.data(), h->ws + h->sl.acc, 8 * acc.size(), cudaMemcpyDeviceToHost, s), "baoc_read_stats");
+    CU(cudaStreamSynchronize(s), "baoc_read_stats");
+    for (int i = 0; i < h->n_blocks; ++i) {
+        std::memset(&out[i], 0, sizeof(out[i]));
+        const double* a = &acc[size_t(i) * kBlockAcc];
+        out[i].rho_bar = a[0]; out[i].n_cos = int64_t(a[1]); out[i].last_cos = a[3]; out[i].rho_mom = a[4];
+    }
+    return BAOC_OK;
+}
+
+int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_block_stats_t* stats_out, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!params || !risk_out) return fail(h, BAOC_E_INVALID, "baoc_risk: null argument");
+    if (!h->ws_bound) return fail(h, BAOC_E_STATE, "baoc_risk: no statistics workspace bound");
+    if (h->stats_steps <= 0) return fail(h, BAOC_E_STATE, "baoc_risk: no gradient has been observed in this window");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n = h->n_blocks;
+    int rc = sync_pointer_table(h, reinterpret_cast<const void* const*>(params), &h->last_stat_params, h->ws + h->sl.params, s, "baoc_risk (params)");
+    if (rc) return rc;
+    const auto& L = h->sl;
+    char* ws = h->ws;
+    const StatBlock* blocks = at<StatBlock>(ws, L.blocks);
+    const Tile* tiles = at<Tile>(ws, L.tiles);
+    const float* const* dparams = at<const float*>(ws, L.params);
+    LAUNCH(launch_final_sums(blocks, tiles, dparams, at<double>(ws, L.fin), at<double>(ws, L.fin_out), h->n_stat_tiles, n,
+                             h->opts.eps, float(h->opts.eps_adam), s), "stats_final_sums_kernel");
+    h->launches += 2;
+    if (h->n_matrix > 0) {
+        LAUNCH(launch_moment_reduce(blocks, at<RedTile>(ws, L.red_tiles), at<int32_t>(ws, L.matrix_ids), h->n_red_tiles,
+                                    h->n_matrix, s), "moment_reduce_kernel");
+        h->launches += 2;
+    }
+    LAUNCH(launch_final_resid(blocks, tiles, dparams, at<double>(ws, L.fin), at<double>(ws, L.fin_out), h->n_stat_tiles, n,
+                              h->opts.eps, s), "stats_final_resid_kernel");
+    h->launches += 2;
+    LAUNCH(launch_select(blocks, tiles, at<RankSel>(ws, L.sel), at<uint32_t>(ws, L.hist), h->n_stat_tiles, n, s),
+           "select kernels");
+    h->launches += 9;
+    LAUNCH(launch_gather(at<RankSel>(ws, L.sel), at<double>(ws, L.acc), at<double>(ws, L.fin_out), n, s), "stats_gather_kernel");
+    h->launches += 1;
+
+    std::vector<double> out(size_t(kFinOut) * n);
+    CU(cudaMemcpyAsync(out.data(), ws + L.fin_out, 8 * out.size(), cudaMemcpyDeviceToHost, s), "baoc_risk (copy back)");
+    CU(cudaStreamSynchronize(s), "baoc_risk (wait)");
+
+    std::vector<baoc_block_stats_t> tmp;
+    baoc_block_stats_t* st = stats_out;
+    if (!st) { tmp.resize(n); st = tmp.data(); }
+    const double eps = h->opts.eps;
+    auto cosine = [&](double dot, double na2, double nb2) {
+        const double c = dot / (std::sqrt(na2) * std::sqrt(nb2) + eps);
+        return std::isfinite(c) ? c : 0.0;
+    };
+    auto rel = [](double err2, double ref2) { return ref2 > 0.0 ? std::sqrt(err2) / std::sqrt(ref2) : 0.0; };
+    for (int i = 0; i < n; ++i) {
+        const double* o = &out[size_t(i) * kFinOut];
+        const baoc_block_t& b = h->blocks[i];
+        baoc_block_stats_t& z = st[i];
+        std::memset(&z, 0, sizeof(z));
+        // Eq. 4: quantiles by linear interpolation at position q (n - 1)
+        const double qs[2] = {0.1, 0.9};
+        double qv[2];
+        for (int k = 0; k < 2; ++k) {
+            const double pos = qs[k] * double(b.numel - 1);
+            const double frac = pos - std::floor(pos);
+            const double lo = o[16 + 2 * k], hi = o[16 + 2 * k + 1];
+            qv[k] = lo + frac * (hi - lo);
+        }
+        z.q10 = qv[0]; z.q90 = qv[1];
+        z.A = std::log((qv[1] + eps) / (qv[0] + eps));
+        z.rho_bar = o[20]; z.n_cos = int64_t(o[21]); z.last_cos = o[23]; z.rho_mom = o[24];
+        z.snr = o[0] / (o[1] + eps);                                        // Eq. 5 right
+        z.C = std::sqrt(o[14]) / (std::sqrt(o[4]) + eps);                   // Eq. 6
+        z.F = b.cols > 1 ? std::sqrt(o[15]) / (std::sqrt(o[2]) + eps) : 1.0;   // Eq. 7
+        z.Q32 = cosine(o[5], o[5], o[5]);                                   // Eq. 8
+        z.Q16 = cosine(o[9], o[5], o[8]);
+        z.Q8 = cosine(o[7], o[5], o[6]);
+        z.err_m8 = rel(o[10], o[0]); z.err_v8 = rel(o[11], o[2]);
+        z.err_m16 = rel(o[12], o[0]); z.err_v16 = rel(o[13], o[2]);
+    }
+    return baoc_risk_from_raw(h, st, risk_out);
+}
+
+int baoc_state_bytes(const baoc_t* h, const int32_t* assign, size_t* bytes) {
+    if (!h) return BAOC_E_INVALID;
+    if (!assign || !bytes) return fail(h, BAOC_E_INVALID, "baoc_state_bytes: null argument");
+    Handle::StepLayout L{};
+    int rc = compute_step_layout(h, assign, &L, nullptr, nullptr, nullptr, nullptr, nullptr);
+    if (rc) return rc;
+    *bytes = L.total;
+    return BAOC_OK;
+}
+
+int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!assign || !state_dev) return fail(h, BAOC_E_INVALID, "baoc_configure: null argument");
+    if (reinterpret_cast<uintptr_t>(state_dev) & 255u) return fail(h, BAOC_E_ALIGN, "baoc_configure: state buffer not 256-byte aligned");
+    Handle::StepLayout L{};
+    std::vector<StepBlock> sb;
+    std::vector<Tile> tiles;
+    std::vector<RedTile> red;
+    int64_t mem = 0, traffic = 0;
+    int rc = compute_step_layout(h, assign, &L, &sb, &tiles, &red, &mem, &traffic);
+    if (rc) return rc;
+    if (bytes < L.total) return fail(h, BAOC_E_WORKSPACE, "baoc_configure: state buffer too small");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char* st = static_cast<char*>(state_dev);
+    const int n = h->n_blocks;
+    std::vector<int32_t> ids;
+    for (int i = 0; i < n; ++i) {
+        StepBlock& b = sb[i];
+        auto fix = [&](void* p) { return static_cast<void*>(st + L.states + reinterpret_cast<size_t>(p)); };
+        if (b.path == kPathA32 || b.path == kPathA8 || b.path == kPathF) { b.s0 = fix(b.s0); b.s1 = fix(b.s1); }
+        else b.s0 = fix(b.s0);
+        if (b.path == kPathA8) { b.a0 = static_cast<float*>(fix(b.a0)); b.a1 = static_cast<float*>(fix(b.a1)); }
+        if (b.path == kPathF) {
+            b.a0 = static_cast<float*>(fix(b.a0));
+            b.red.rowpart = reinterpret_cast<double*>(st + L.redpart + reinterpret_cast<size_t>(b.red.rowpart));
+            b.red.colpart = reinterpret_cast<double*>(st + L.redpart + reinterpret_cast<size_t>(b.red.colpart));
+            ids.push_back(i);
+        }
+    }
+    CU(cudaMemcpyAsync(st + L.blocks, sb.data(), sizeof(StepBlock) * n, cudaMemcpyHostToDevice, s), "upload step block table");
+    CU(cudaMemcpyAsync(st + L.tiles, tiles.data(), sizeof(Tile) * tiles.size(), cudaMemcpyHostToDevice, s), "upload step tile table");
+    if (!red.empty())
+        CU(cudaMemcpyAsync(st + L.red_tiles, red.data(), sizeof(RedTile) * red.size(), cudaMemcpyHostToDevice, s), "upload step reduction table");
+    if (!ids.empty())
+        CU(cudaMemcpyAsync(st + L.f_ids, ids.data(), 4 * ids.size(), cudaMemcpyHostToDevice, s), "upload factored ids");
+    CU(cudaMemsetAsync(st + L.flags, 0, L.total - L.flags, s), "zero optimizer state");
+    h->st = st; h->st_bytes = bytes; h->tl = L; h->configured = true;
+    h->assign.assign(assign, assign + n);
+    h->h_step_blocks = sb;
+    h->n_step_tiles = int64_t(tiles.size()); h->n_step_red_tiles = int64_t(red.size());
+    h->n_factored = int(ids.size());
+    h->state_mem = mem; h->step_bytes = traffic;
+    h->last_step_grads.clear(); h->last_step_params.clear();
+    return BAOC_OK;
+}
+
+int baoc_step(baoc_t* h, const void* const* grads, float* const* params, int64_t step_t, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!grads || !params) return fail(h, BAOC_E_INVALID, "baoc_step: null pointer table");
+    if (step_t < 1) return fail(h, BAOC_E_INVALID, "baoc_step: step numbers start at 1");
+    if (!h->configured) return fail(h, BAOC_E_STATE, "baoc_step: no assignment configured");
+    return do_step(h, grads, params, step_t, static_cast<cudaStream_t>(stream));
+}
+
+int baoc_step_from_host(baoc_t* h, const void* const* host_grads, void* const* dev_grads, float* const* params,
+                        int do_stats, int64_t step_t, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!host_grads || !dev_grads) return fail(h, BAOC_E_INVALID, "baoc_step_from_host: null pointer table");
+    if (do_stats && !h->ws_bound) return fail(h, BAOC_E_STATE, "baoc_step_from_host: no statistics workspace bound");
+    if (step_t > 0 && (!h->configured || !params)) return fail(h, BAOC_E_STATE, "baoc_step_from_host: no assignment configured");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < h->n_blocks; ++i) {
+        if (!host_grads[i] || !dev_grads[i]) return fail(h, BAOC_E_INVALID, "baoc_step_from_host: null block pointer");
+        if (!aligned16(dev_grads[i])) return fail(h, BAOC_E_ALIGN, "baoc_step_from_host: block pointer not 16-byte aligned");
+    }
+    // blocks that are contiguous on both sides travel in one copy
+    int i = 0;
+    while (i < h->n_blocks) {
+        int j = i;
+        size_t bytes = 2 * size_t(h->blocks[i].numel);
+        while (j + 1 < h->n_blocks &&
+               static_cast<const char*>(host_grads[j + 1]) == static_cast<const char*>(host_grads[i]) + bytes &&
+               static_cast<const char*>(dev_grads[j + 1]) == static_cast<const char*>(dev_grads[i]) + bytes) {
+            ++j;
+            bytes += 2 * size_t(h->blocks[j].numel);
+        }
+        CU(cudaMemcpyAsync(dev_grads[i], host_grads[i], bytes, cudaMemcpyHostToDevice, s), "baoc_step_from_host (copy)");
+        i = j + 1;
+    }
+    const void* const* dg = reinterpret_cast<const void* const*>(dev_grads);
+    if (do_stats) {
+        int rc = do_sample_stats(h, dg, s);
+        if (rc) return rc;
+    }
+    if (step_t > 0) return do_step(h, dg, params, step_t, s);
+    return BAOC_OK;
+}
+
+int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* count, int32_t* elem_bytes) {
+    if (!h) return BAOC_E_INVALID;
+    if (!dev_ptr || !count || !elem_bytes || block < 0 || block >= h->n_blocks) return fail(h, BAOC_E_INVALID, "baoc_view: bad argument");
+    const baoc_block_t& b = h->blocks[block];
+    if (which >= 0 && which <= 2) {
+        if (!h->ws_bound) return fail(h, BAOC_E_STATE, "baoc_view: no statistics workspace bound");
+        const StatBlock& s = h->h_stat_blocks[block];
+        const size_t off = reinterpret_cast<size_t>(which == 2 ? static_cast<void*>(s.gprev) : static_cast<void*>(which == 0 ? s.m : s.v));
+        const size_t region = which == 0 ? h->sl.m : (which == 1 ? h->sl.v : h->sl.gprev);
+        *dev_ptr = h->ws + region + off; *count = b.numel; *elem_bytes = which == 2 ? 2 : 4;
+        return BAOC_OK;
+    }
+    if (which >= 10 && which <= 13) {
+        if (!h->configured) return fail(h, BAOC_E_STATE, "baoc_view: no assignment configured");
+        const StepBlock& s = h->h_step_blocks[block];
+        const int k = which - 10;
+        const int64_t nq = ceil_div(b.numel, kQBlock);
+        void* p = nullptr; int64_t n = 0; int32_t eb = 4;
+        switch (s.path) {
+            case kPathA32: if (k == 0) { p = s.s0; n = b.numel; } else if (k == 1) { p = s.s1; n = b.numel; } break;
+            case kPathA8:
+                if (k == 0) { p = s.s0; n = b.numel; eb = 1; } else if (k == 1) { p = s.s1; n = b.numel; eb = 1; }
+                else if (k == 2) { p = s.a0; n = nq; } else { p = s.a1; n = nq; }
+                break;
+            case kPathR: case kPathS: if (k == 0) { p = s.s0; n = b.numel; } break;
+            case kPathF: if (k == 0) { p = s.s0; n = b.rows; } else if (k == 1) { p = s.s1; n = b.cols; } break;
+            default: break;
+        }
+        if (!p) return fail(h, BAOC_E_INVALID, "baoc_view: the block has no such state tensor");
+        *dev_ptr = p; *count = n; *elem_bytes = eb;
+        return BAOC_OK;
+    }
+    return fail(h, BAOC_E_INVALID, "baoc_view: unknown tensor id");
+}
+
+int baoc_nonfinite(baoc_t* h, uint8_t* flags, int32_t* count, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!count) return fail(h, BAOC_E_INVALID, "baoc_nonfinite: null count");
+    if (!h->configured) return fail(h, BAOC_E_STATE, "baoc_nonfinite: no assignment configured");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<uint32_t> f(h->n_blocks);
+    CU(cudaMemcpyAsync(f.data(), h->st + h->tl.flags, 4 * f.size(), cudaMemcpyDeviceToHost, s), "baoc_nonfinite");
+    CU(cudaStreamSynchronize(s), "baoc_nonfinite");
+    int32_t c = 0;
+    for (int i = 0; i < h->n_blocks; ++i) {
+        if (flags) flags[i] = f[i] ? 1 : 0;
+        c += f[i] ? 1 : 0;
+    }
+    *count = c;
+    return BAOC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,128 @@
+// Device helpers shared by the statistics and step kernels: vector loads and
+// stores with streaming cache hints, bf16 unpacking, deterministic CTA
+// reductions, and the 8-bit block-wise absmax code arithmetic.
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "baoc_internal.h"
+
+namespace baoc {
+
+__device__ __forceinline__ int64_t min64(int64_t a, int64_t b) { return a < b ? a : b; }
+__device__ __forceinline__ int64_t max64(int64_t a, int64_t b) { return a > b ? a : b; }
+
+// ---- 128-bit streaming loads / stores ---------------------------------------
+// Every array on this path is touched once per launch, so loads bypass L1
+// allocation and stores are marked evict-first.
+
+__device__ __forceinline__ uint4 ld_stream_u4(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ float4 ld_stream_f4(const void* p) {
+    float4 r;
+    asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ uint2 ld_stream_u2(const void* p) {
+    uint2 r;
+    asm volatile("ld.global.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ void st_stream_f4(void* p, float4 v) {
+    asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_stream_u4(void* p, uint4 v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_stream_u2(void* p, uint2 v) {
+    asm volatile("st.global.cs.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(v.x), "r"(v.y) : "memory");
+}
+
+// ---- bf16 ------------------------------------------------------------------
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float(uint32_t(b) << 16); }
+
+// Unpack 8 bf16 values held in a uint4 into floats.
+__device__ __forceinline__ void unpack8(const uint4& w, float (&x)[8]) {
+    x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
+    x[4] = bf16_lo(w.z); x[5] = bf16_hi(w.z); x[6] = bf16_lo(w.w); x[7] = bf16_hi(w.w);
+}
+
+// A float that holds a bf16 value, widened to double without a conversion
+// instruction (the conversion pipe is narrow): re-bias the exponent with
+// integer arithmetic.  Zeros, subnormals, infinities and NaNs take the
+// ordinary conversion.
+__device__ __forceinline__ double widen_bf16_float(float x) {
+    const uint32_t u = __float_as_uint(x);
+    const uint32_t e = u & 0x7f800000u;
+    if (e == 0u || e == 0x7f800000u) return double(x);
+    const uint32_t hi = (u & 0x80000000u) | (((u & 0x7fffffffu) >> 3) + (896u << 20));
+    return __hiloint2double(int(hi), 0);
+}
+
+// Small integer (|q| < 2^31) to double, exact, without a conversion instruction.
+__device__ __forceinline__ double int_to_double(int q) {
+    return __hiloint2double(0x43300000, int(uint32_t(q) ^ 0x80000000u)) - 4503601774854144.0;   // 2^52 + 2^31
+}
+// Small integer (|q| < 2^22) to float, exact.
+__device__ __forceinline__ float int_to_float(int q) {
+    return __int_as_float(0x4B400000 + q) - 12582912.0f;                                         // 1.5 * 2^23
+}
+// Round a double of magnitude < 2^31 to the nearest integer, ties to even.
+__device__ __forceinline__ int round_to_int(double x) {
+    return __double2loint(x + 6755399441055744.0);                                               // 1.5 * 2^52
+}
+
+// ---- deterministic CTA reduction ---------------------------------------------
+// Sums K values per thread over the CTA in a fixed order (butterfly inside a
+// warp, then warps in index order) and lets thread 0 store the K results.
+template <int K>
+__device__ __forceinline__ void cta_reduce_store(double (&val)[K], double* out) {
+    __shared__ double sh[kThreads / 32][K];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        double x = val[k];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        if (lane == 0) sh[warp][k] = x;
+    }
+    __syncthreads();
+    if (threadIdx.x < K) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) s += sh[w][threadIdx.x];
+        out[threadIdx.x] = s;
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+
+// ---- 8-bit block-wise absmax codes -----------------------------------------------
+// code = clamp(rne(L * x / a)), x ~ code * a / L, with L = 127 (signed) or 255
+// (unsigned) and a the fp32 absmax of the 256-element quantisation block.  The
+// scaling and rounding are done in double so that the decision agrees with a
+// double-precision evaluation of the same formula.
+__device__ __forceinline__ double code_scale(float absmax, double levels) {
+    return absmax > 0.0f ? levels / double(absmax) : 0.0;
+}
+__device__ __forceinline__ int encode_signed(double x, double scale) {
+    return max(-127, min(127, round_to_int(x * scale)));
+}
+__device__ __forceinline__ int encode_unsigned(double x, double scale) {
+    return max(0, min(255, round_to_int(x * scale)));
+}
+
+}  // namespace baoc

@@ -1,0 +1,197 @@
+// Internal declarations shared by the host and CUDA translation units of the
+// library.  Nothing here is part of the public ABI (see include/baoc.h).
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "baoc.h"
+
+struct CUstream_st;
+typedef CUstream_st* cudaStream_t;
+
+namespace baoc {
+
+constexpr int kMaxCfg = 32;
+constexpr int kQBlock = 256;          // elements per 8-bit quantisation block
+constexpr int kTile = 4096;           // elements per tile of the streaming kernels
+constexpr int kThreads = 256;         // threads per CTA of the streaming kernels
+constexpr int kStatPartials = 4;      // doubles per tile written by the per-step statistics kernel
+constexpr int kFinalSums = 14;        // doubles per tile written by the first finalize sweep
+constexpr int kResidSums = 2;         // doubles per tile written by the second finalize sweep
+constexpr int kBlockAcc = 8;          // doubles per block of running window values
+constexpr int kRanks = 4;             // order statistics per block for the two quantiles
+constexpr int kFinOut = 32;           // doubles per block copied to the host at the end of the window
+constexpr int kRedRows = 64;          // rows per CTA of the row/column reduction kernel
+constexpr int kRedCols = 512;         // columns per CTA of the row/column reduction kernel
+
+// Update paths of the fused step.
+enum Path : int32_t { kPathA32 = 0, kPathA8 = 1, kPathR = 2, kPathF = 3, kPathS = 4, kPathNone = -1 };
+
+inline Path path_of(const baoc_config_t& c) {
+    if (c.adaptive && c.momentum && !c.factored) return c.bits == 32 ? kPathA32 : (c.bits == 8 ? kPathA8 : kPathNone);
+    if (c.adaptive && !c.momentum && !c.factored && c.bits == 32) return kPathR;
+    if (c.adaptive && !c.momentum && c.factored && c.bits == 32) return kPathF;
+    if (!c.adaptive && c.momentum && !c.factored && c.bits == 32) return kPathS;
+    return kPathNone;
+}
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
+
+// One tile of a streaming kernel: which block, and which kTile-sized piece of it.
+struct Tile {
+    uint32_t block;
+    uint32_t piece;
+};
+
+// Geometry of the row/column reduction of one matrix block.  The matrix is cut
+// into chunks of 64*L rows and strips of kRedCols columns; one CTA reduces one
+// (chunk, strip) piece and writes its row sums to rowpart[strip][row] and its
+// column sums to colpart[chunk][col].
+struct RedGeom {
+    double* rowpart;
+    double* colpart;
+    int32_t red0;        // index of the block's first reduction CTA (-1: no reduction for this block)
+    int32_t chunks, strips, L;
+};
+
+// Per-block record of the statistics pass (device copy lives in the workspace).
+struct StatBlock {
+    float* m;            // EMA first moment (Eq. 3)
+    float* v;            // EMA second moment
+    uint16_t* gprev;     // previous gradient, bf16 bits
+    double* rowsum;      // row sums of v (matrix blocks), length rows
+    double* colsum;      // column sums of v, length cols
+    int64_t numel;
+    int64_t tile0;       // index of the block's first tile
+    int32_t rows, cols;
+    int32_t ntiles, pad;
+    RedGeom red;
+};
+
+// Per-block record of the fused step (device copy lives in the state buffer).
+struct StepBlock {
+    void* s0;            // A32: m   A8: codes of m   R: v   F: r (rows)   S: m
+    void* s1;            // A32: v   A8: codes of v          F: c (cols)
+    float* a0;           // A8: absmax of m per quantisation block;  F: [0] = mean of r
+    float* a1;           // A8: absmax of v per quantisation block
+    int64_t numel;
+    int32_t rows, cols;
+    int32_t cfg;
+    int32_t path;
+    RedGeom red;
+};
+
+// State of one radix select: the bits found so far and the rank still to find
+// among the elements that share them.
+struct RankSel {
+    uint32_t prefix;
+    int32_t leader;      // first rank of the block with the same prefix (its histogram is shared)
+    int64_t remaining;
+};
+
+// One CTA of the row/column reduction: a kRedRows x kRedCols piece of a matrix block.
+struct RedTile {
+    uint32_t block;
+    uint32_t chunk;      // row chunk
+    uint32_t strip;      // column strip
+    uint32_t pad;
+};
+
+// Per-configuration scalars of one step, passed to the kernel by value.
+struct CfgStep {
+    float lr, beta1, beta2, eps;
+    float wd;            // weight decay coefficient
+    float decay;         // -lr*wd when the decay is decoupled, else 0
+    float bc1, bc2;      // 1 - beta1^t, 1 - beta2^t
+    double beta1_d, beta2_d;   // the same coefficients widened, for the 8-bit path
+    int32_t coupled;     // 1: add wd*theta to the gradient
+    int32_t pad;
+};
+struct StepParams {
+    CfgStep c[kMaxCfg];
+};
+
+struct Handle {
+    int n_blocks = 0, n_cfg = 0;
+    std::vector<baoc_block_t> blocks;
+    std::vector<baoc_config_t> cfgs;
+    baoc_opts_t opts{};
+    mutable std::string err;
+    int64_t numel = 0;
+    int64_t launches = 0;
+
+    // statistics workspace
+    char* ws = nullptr;
+    size_t ws_bytes = 0;
+    bool ws_bound = false;
+    int64_t stats_steps = 0;
+    int64_t n_stat_tiles = 0;
+    int64_t n_red_tiles = 0;         // reduction CTAs over all matrix blocks
+    int n_matrix = 0;                // blocks with cols > 1
+    std::vector<StatBlock> h_stat_blocks;
+    std::vector<const void*> last_stat_grads;
+    std::vector<const void*> last_stat_params;
+    struct StatLayout {
+        size_t blocks, tiles, red_tiles, matrix_ids, grads, params, m, v, gprev, partials, acc, fin, fin_out, hist, sel,
+               rowsum, colsum, redpart, total;
+    } sl{};
+
+    // optimizer state
+    char* st = nullptr;
+    size_t st_bytes = 0;
+    bool configured = false;
+    std::vector<int32_t> assign;
+    std::vector<StepBlock> h_step_blocks;
+    int64_t n_step_tiles = 0;
+    int64_t n_step_red_tiles = 0;
+    int n_factored = 0;              // blocks on the factored path
+    int64_t state_mem = 0;           // StateMem of the assignment (sum of M_{i,c_i})
+    int64_t step_bytes = 0;          // algorithmic bytes of one step
+    std::vector<const void*> last_step_grads;
+    std::vector<const void*> last_step_params;
+    struct StepLayout {
+        size_t blocks, tiles, red_tiles, f_ids, grads, params, flags, redpart, states, total;
+    } tl{};
+};
+
+int fail(const Handle* h, int code, const std::string& msg);
+
+// Reduction geometry of a rows x cols matrix (pointers left null).
+RedGeom red_geometry(int32_t rows, int32_t cols);
+
+// M_{i,c}: bytes of persistent state of one block under one configuration.
+int64_t state_mem_bytes(const baoc_config_t& c, const baoc_block_t& b);
+// Algorithmic HBM bytes per step of one block under one configuration.
+double step_traffic_bytes(const baoc_config_t& c, const baoc_block_t& b);
+
+void compute_stat_layout(Handle* h);
+
+// Kernel launchers (defined in the .cu files).  Each returns 0 or a cudaError_t value.
+int launch_stats_step(const StatBlock* blocks, const Tile* tiles, const void* const* grads, double* partials,
+                      int64_t n_tiles, float beta_m, float beta_v, cudaStream_t s);
+int launch_stats_combine(const StatBlock* blocks, const double* partials, double* acc, int n_blocks, int has_prev,
+                         double beta_rho, double eps, cudaStream_t s);
+int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
+                      double* fin_out, int64_t n_tiles, int n_blocks, double eps, float eps_adam, cudaStream_t s);
+int launch_final_resid(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
+                       double* fin_out, int64_t n_tiles, int n_blocks, double eps, cudaStream_t s);
+int launch_select(const StatBlock* blocks, const Tile* tiles, RankSel* sel, uint32_t* hist, int64_t n_tiles,
+                  int n_blocks, cudaStream_t s);
+int launch_gather(const RankSel* sel, const double* acc, double* fin_out, int n_blocks, cudaStream_t s);
+int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const int32_t* ids, int64_t n_red, int n_matrix,
+                         cudaStream_t s);
+int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const int32_t* ids, const void* const* grads,
+                           int64_t n_red, int n_factored, const StepParams& P, cudaStream_t s);
+int launch_fused_step(const StepBlock* blocks, const Tile* tiles, const void* const* grads, float* const* params,
+                      uint32_t* flags, int64_t n_tiles, const StepParams& P, cudaStream_t s);
+int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayout* out,
+                        std::vector<StepBlock>* blocks, std::vector<Tile>* tiles,
+                        std::vector<RedTile>* red, int64_t* state_mem, int64_t* step_bytes);
+
+}  // namespace baoc
+
+struct baoc_handle : public baoc::Handle {};

@@ -1,0 +1,434 @@
+// Kernels of the sampling window (Sec. 3.3): the per-step streaming pass that
+// updates the EMA moments (Eq. 3) and the sums behind the direction-stability
+// cosine (Eq. 5), its combine, and the end-of-window finalize sweeps that
+// produce the sums behind Eq. 4-8.
+#include "baoc_device.cuh"
+
+namespace baoc {
+
+// ============================================================================
+// Per-step pass.  One CTA per tile of kTile elements of one block; every thread
+// owns 8 consecutive elements per 2048-element slice.  Reads g_t, g_{t-1}
+// (bf16), m, v (fp32); writes m, v, g_{t-1}; leaves 4 partial sums per tile:
+// <g_t, g_{t-1}>, ||g_t||^2, <g_t, m_{t-1}>, ||m_{t-1}||^2.
+// ============================================================================
+__global__ void __launch_bounds__(kThreads)
+stats_step_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
+                  const void* const* __restrict__ grads, double* __restrict__ partials, float beta_m, float beta_v) {
+    const Tile t = tiles[blockIdx.x];
+    const StatBlock* b = blocks + t.block;
+    const int64_t numel = b->numel;
+    const uint16_t* __restrict__ g = static_cast<const uint16_t*>(grads[t.block]);
+    uint16_t* __restrict__ gp = b->gprev;
+    float* __restrict__ m = b->m;
+    float* __restrict__ v = b->v;
+    const int64_t base = int64_t(t.piece) * kTile;
+    const float om = 1.0f - beta_m, ov = 1.0f - beta_v;
+    constexpr int kSlices = kTile / (kThreads * 8);
+
+    float a_dot = 0.f, a_n2 = 0.f, a_dm = 0.f, a_m2 = 0.f;
+
+    uint4 wg[kSlices], wp[kSlices];
+    float4 m0[kSlices], m1[kSlices], v0[kSlices], v1[kSlices];
+    bool full[kSlices];
+#pragma unroll
+    for (int s = 0; s < kSlices; ++s) {
+        const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+        full[s] = e + 8 <= numel;
+        if (full[s]) {
+            wg[s] = ld_stream_u4(g + e);
+            wp[s] = ld_stream_u4(gp + e);
+            m0[s] = ld_stream_f4(m + e); m1[s] = ld_stream_f4(m + e + 4);
+            v0[s] = ld_stream_f4(v + e); v1[s] = ld_stream_f4(v + e + 4);
+        }
+    }
+#pragma unroll
+    for (int s = 0; s < kSlices; ++s) {
+        const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+        if (full[s]) {
+            float x[8], p[8];
+            unpack8(wg[s], x); unpack8(wp[s], p);
+            float mm[8] = {m0[s].x, m0[s].y, m0[s].z, m0[s].w, m1[s].x, m1[s].y, m1[s].z, m1[s].w};
+            float vv[8] = {v0[s].x, v0[s].y, v0[s].z, v0[s].w, v1[s].x, v1[s].y, v1[s].z, v1[s].w};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                a_dot = fmaf(x[j], p[j], a_dot);
+                a_n2 = fmaf(x[j], x[j], a_n2);
+                a_dm = fmaf(x[j], mm[j], a_dm);
+                a_m2 = fmaf(mm[j], mm[j], a_m2);
+                mm[j] = fmaf(beta_m, mm[j], om * x[j]);
+                vv[j] = fmaf(beta_v, vv[j], ov * (x[j] * x[j]));
+            }
+            st_stream_f4(m + e, make_float4(mm[0], mm[1], mm[2], mm[3]));
+            st_stream_f4(m + e + 4, make_float4(mm[4], mm[5], mm[6], mm[7]));
+            st_stream_f4(v + e, make_float4(vv[0], vv[1], vv[2], vv[3]));
+            st_stream_f4(v + e + 4, make_float4(vv[4], vv[5], vv[6], vv[7]));
+            st_stream_u4(gp + e, wg[s]);
+        } else if (e < numel) {
+            const int cnt = int(numel - e);
+            for (int j = 0; j < cnt; ++j) {
+                const uint16_t gb = g[e + j];
+                const float x = bf16_bits_to_float(gb), p = bf16_bits_to_float(gp[e + j]);
+                const float mm = m[e + j], vv = v[e + j];
+                a_dot = fmaf(x, p, a_dot); a_n2 = fmaf(x, x, a_n2);
+                a_dm = fmaf(x, mm, a_dm); a_m2 = fmaf(mm, mm, a_m2);
+                m[e + j] = fmaf(beta_m, mm, om * x);
+                v[e + j] = fmaf(beta_v, vv, ov * (x * x));
+                gp[e + j] = gb;
+            }
+        }
+    }
+    double acc[kStatPartials] = {double(a_dot), double(a_n2), double(a_dm), double(a_m2)};
+    cta_reduce_store<kStatPartials>(acc, partials + size_t(blockIdx.x) * kStatPartials);
+}
+
+// Sum K doubles per tile over the tiles of one block in a fixed order: thread
+// t takes tiles t, t+T, ..., then the CTA reduces.  out[K] per block.
+template <int K>
+__device__ __forceinline__ void block_tiles_sum(const double* __restrict__ part, int64_t tile0, int ntiles, double* out) {
+    double acc[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) acc[k] = 0.0;
+    for (int i = threadIdx.x; i < ntiles; i += kThreads) {
+        const double* p = part + size_t(tile0 + i) * K;
+#pragma unroll
+        for (int k = 0; k < K; ++k) acc[k] += p[k];
+    }
+    cta_reduce_store<K>(acc, out);
+}
+
+__device__ __forceinline__ double safe_cos(double dot, double n2a, double n2b, double eps) {
+    const double c = dot / (sqrt(n2a) * sqrt(n2b) + eps);
+    return isfinite(c) ? c : 0.0;          // a cosine that is not a number counts as 0
+}
+
+// Combine: one CTA per block.  acc[block] = {rho_bar, n_cos, ||g_{t-1}||^2,
+// last_cos, rho_mom, n_cos_mom, -, -}.
+__global__ void __launch_bounds__(kThreads)
+stats_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ partials,
+                     double* __restrict__ acc_all, int has_prev, double beta_rho, double eps) {
+    __shared__ double s[kStatPartials];
+    const StatBlock* b = blocks + blockIdx.x;
+    block_tiles_sum<kStatPartials>(partials, b->tile0, b->ntiles, s);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double* acc = acc_all + size_t(blockIdx.x) * kBlockAcc;
+        const double dot = s[0], n2 = s[1], dm = s[2], m2 = s[3];
+        if (has_prev) {
+            const double c = safe_cos(dot, n2, acc[2], eps);
+            acc[3] = c;
+            acc[0] = acc[1] == 0.0 ? c : beta_rho * acc[0] + (1.0 - beta_rho) * c;
+            acc[1] += 1.0;
+            const double cm = safe_cos(dm, n2, m2, eps);
+            acc[4] = acc[5] == 0.0 ? cm : beta_rho * acc[4] + (1.0 - beta_rho) * cm;
+            acc[5] += 1.0;
+        }
+        acc[2] = n2;
+    }
+}
+
+// ============================================================================
+// Finalize sweep 1: per tile, 14 sums over the window's moments (fp32), the
+// parameters and the quantised moments.  A warp owns one 256-element
+// quantisation block per slice, so the absmax is a warp reduction.
+//   0 sum m^2      1 sum v        2 sum v^2       3 sum p, p = 1/(sqrt(v)+eps)
+//   4 sum theta^2  5 sum u32^2    6 sum u8^2      7 sum u32*u8
+//   8 sum u16^2    9 sum u32*u16  10 sum (m-m8)^2 11 sum (v-v8)^2
+//   12 sum (m-m16)^2              13 sum (v-v16)^2
+// with u = m/(sqrt(v)+eps_adam) from full-precision, 8-bit and bf16 moments.
+// ============================================================================
+__device__ __forceinline__ float round_to_bf16(float x) {
+    uint32_t u = __float_as_uint(x);
+    if ((u & 0x7f800000u) == 0x7f800000u) return x;
+    u = (u + 0x7fffu + ((u >> 16) & 1u)) & 0xffff0000u;
+    return __uint_as_float(u);
+}
+
+__global__ void __launch_bounds__(kThreads)
+stats_final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
+                        const float* const* __restrict__ params, double* __restrict__ fin, double eps, float eps_adam) {
+    const Tile t = tiles[blockIdx.x];
+    const StatBlock* b = blocks + t.block;
+    const int64_t numel = b->numel;
+    const float* __restrict__ m = b->m;
+    const float* __restrict__ v = b->v;
+    const float* __restrict__ th = params[t.block];
+    const int64_t base = int64_t(t.piece) * kTile;
+    double acc[kFinalSums];
+#pragma unroll
+    for (int k = 0; k < kFinalSums; ++k) acc[k] = 0.0;
+
+    for (int s = 0; s < kTile / (kThreads * 8); ++s) {
+        const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+        float mm[8], vv[8], tt[8];
+        int cnt = 0;
+        if (e < numel) cnt = int(min64(8, numel - e));
+        // m and v are padded to whole quantisation blocks (zeros), theta is not
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const bool in = j < cnt;
+            mm[j] = in ? m[e + j] : 0.f;
+            vv[j] = in ? v[e + j] : 0.f;
+            tt[j] = in ? th[e + j] : 0.f;
+        }
+        float am = 0.f, av = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { am = fmaxf(am, fabsf(mm[j])); av = fmaxf(av, vv[j]); }
+        am = warp_max(am); av = warp_max(av);
+        const double sm = code_scale(am, 127.0), sv = code_scale(av, 255.0);
+        const float dm = am / 127.0f, dv = av / 255.0f;
+        float f[kFinalSums];
+#pragma unroll
+        for (int k = 0; k < kFinalSums; ++k) f[k] = 0.f;
+        double psum = 0.0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (j < cnt) {
+                const float mj = mm[j], vj = vv[j];
+                const float m8 = float(encode_signed(double(mj), sm)) * dm;
+                const float v8 = float(encode_unsigned(double(vj), sv)) * dv;
+                const float m16 = round_to_bf16(mj), v16 = round_to_bf16(vj);
+                const float u32 = mj / (sqrtf(vj) + eps_adam);
+                const float u8 = m8 / (sqrtf(v8) + eps_adam);
+                const float u16 = m16 / (sqrtf(v16) + eps_adam);
+                psum += 1.0 / (sqrt(double(vj)) + eps);
+                f[0] = fmaf(mj, mj, f[0]); f[1] += vj; f[2] = fmaf(vj, vj, f[2]);
+                f[4] = fmaf(tt[j], tt[j], f[4]);
+                f[5] = fmaf(u32, u32, f[5]); f[6] = fmaf(u8, u8, f[6]); f[7] = fmaf(u32, u8, f[7]);
+                f[8] = fmaf(u16, u16, f[8]); f[9] = fmaf(u32, u16, f[9]);
+                f[10] = fmaf(mj - m8, mj - m8, f[10]); f[11] = fmaf(vj - v8, vj - v8, f[11]);
+                f[12] = fmaf(mj - m16, mj - m16, f[12]); f[13] = fmaf(vj - v16, vj - v16, f[13]);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kFinalSums; ++k) acc[k] += double(f[k]);
+        acc[3] += psum;
+    }
+    cta_reduce_store<kFinalSums>(acc, fin + size_t(blockIdx.x) * kFinalSums);
+}
+
+// Per-block combine of sweep 1: fin_out[block][0..13] = the 14 sums.
+__global__ void __launch_bounds__(kThreads)
+stats_final_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ fin, double* __restrict__ fin_out) {
+    const StatBlock* b = blocks + blockIdx.x;
+    block_tiles_sum<kFinalSums>(fin, b->tile0, b->ntiles, fin_out + size_t(blockIdx.x) * kFinOut);
+}
+
+// ============================================================================
+// Finalize sweep 2: residual sums that need block-level means first.
+//   0 sum ((p/pbar - 1) * theta)^2            (Eq. 6 numerator)
+//   1 sum (S_ij - a_i b_j / mu)^2             (Eq. 7 numerator, matrix blocks)
+// Differences of nearly equal numbers: all in double.
+// ============================================================================
+__global__ void __launch_bounds__(kThreads)
+stats_final_resid_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
+                         const float* const* __restrict__ params, const double* __restrict__ fin_out,
+                         double* __restrict__ fin, double eps) {
+    const Tile t = tiles[blockIdx.x];
+    const StatBlock* b = blocks + t.block;
+    const int64_t numel = b->numel;
+    const int cols = b->cols, rows = b->rows;
+    const float* __restrict__ v = b->v;
+    const float* __restrict__ th = params[t.block];
+    const double* __restrict__ rowsum = b->rowsum;
+    const double* __restrict__ colsum = b->colsum;
+    const double* sums = fin_out + size_t(t.block) * kFinOut;
+    const double pbar = sums[3] / double(numel);
+    const double inv_pbar = pbar > 0.0 ? 1.0 / pbar : 0.0;
+    const bool matrix = cols > 1;
+    // a_i b_j / mu = rowsum_i * colsum_j / total
+    const double total = sums[1];
+    const double inv_total = (matrix && total > 0.0) ? 1.0 / total : 0.0;
+    const int64_t base = int64_t(t.piece) * kTile;
+    double acc[kResidSums] = {0.0, 0.0};
+    for (int s = 0; s < kTile / (kThreads * 8); ++s) {
+        const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+        if (e >= numel) continue;
+        const int cnt = int(min64(8, numel - e));
+        int64_t r = matrix ? e / cols : 0;
+        int c = matrix ? int(e - r * cols) : 0;
+        for (int j = 0; j < cnt; ++j) {
+            const double vj = double(v[e + j]);
+            const double p = 1.0 / (sqrt(vj) + eps);
+            const double d = (p * inv_pbar - 1.0) * double(th[e + j]);
+            acc[0] += d * d;
+            if (matrix) {
+                const double fit = rowsum[r] * colsum[c] * inv_total;
+                acc[1] += (vj - fit) * (vj - fit);
+                if (++c == cols) { c = 0; ++r; }
+            }
+        }
+    }
+    (void)rows;
+    cta_reduce_store<kResidSums>(acc, fin + size_t(blockIdx.x) * kResidSums);
+}
+
+__global__ void __launch_bounds__(kThreads)
+stats_resid_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ fin, double* __restrict__ fin_out) {
+    const StatBlock* b = blocks + blockIdx.x;
+    block_tiles_sum<kResidSums>(fin, b->tile0, b->ntiles, fin_out + size_t(blockIdx.x) * kFinOut + kFinalSums);
+}
+
+// ============================================================================
+// Exact quantiles of v by radix select on the fp32 bit patterns (v >= 0, so the
+// unsigned order of the patterns is the numeric order).  Four ranks per block
+// (the two order statistics around each of the two quantile positions), eight
+// bits per pass.  Ranks that still share a prefix share one histogram.
+// ============================================================================
+__global__ void __launch_bounds__(kThreads)
+select_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
+                   const RankSel* __restrict__ sel, uint32_t* __restrict__ hist, int shift) {
+    __shared__ uint32_t sh[kRanks][256];
+    const Tile t = tiles[blockIdx.x];
+    const StatBlock* b = blocks + t.block;
+    const int64_t numel = b->numel;
+    const uint32_t* __restrict__ v = reinterpret_cast<const uint32_t*>(b->v);
+    for (int i = threadIdx.x; i < kRanks * 256; i += kThreads) (&sh[0][0])[i] = 0u;
+    uint32_t prefix[kRanks];
+    bool lead[kRanks];
+#pragma unroll
+    for (int r = 0; r < kRanks; ++r) {
+        const RankSel s = sel[size_t(t.block) * kRanks + r];
+        prefix[r] = s.prefix; lead[r] = s.leader == r;
+    }
+    __syncthreads();
+    const int64_t base = int64_t(t.piece) * kTile;
+    const uint32_t high_mask = shift >= 24 ? 0u : (0xffffffffu << (shift + 8));
+    for (int i = threadIdx.x; i < kTile; i += kThreads) {
+        const int64_t e = base + i;
+        if (e < numel) {
+            const uint32_t u = v[e];
+            const uint32_t digit = (u >> shift) & 255u;
+#pragma unroll
+            for (int r = 0; r < kRanks; ++r)
+                if (lead[r] && ((u ^ prefix[r]) & high_mask) == 0u) atomicAdd(&sh[r][digit], 1u);
+        }
+    }
+    __syncthreads();
+    uint32_t* out = hist + size_t(t.block) * kRanks * 256;
+    for (int i = threadIdx.x; i < kRanks * 256; i += kThreads) {
+        const uint32_t c = (&sh[0][0])[i];
+        if (c) atomicAdd(out + i, c);
+    }
+}
+
+// One thread per (block, rank): pick the digit that holds the rank, extend the
+// prefix, and recompute which ranks still share a prefix.  Clears the
+// histograms for the next pass.
+__global__ void select_pick_kernel(RankSel* __restrict__ sel, uint32_t* __restrict__ hist, int n_blocks, int shift) {
+    const int blk = blockIdx.x * blockDim.x + threadIdx.x;
+    if (blk >= n_blocks) return;
+    RankSel s[kRanks];
+    for (int r = 0; r < kRanks; ++r) s[r] = sel[size_t(blk) * kRanks + r];
+    for (int r = 0; r < kRanks; ++r) {
+        const uint32_t* hh = hist + (size_t(blk) * kRanks + s[r].leader) * 256;
+        int64_t rem = s[r].remaining;
+        int d = 0;
+        for (; d < 255; ++d) {
+            const int64_t c = hh[d];
+            if (rem < c) break;
+            rem -= c;
+        }
+        s[r].remaining = rem;
+        s[r].prefix |= uint32_t(d) << shift;
+    }
+    for (int r = 0; r < kRanks; ++r) {
+        int leader = r;
+        for (int q = 0; q < r; ++q)
+            if (s[q].prefix == s[r].prefix) { leader = q; break; }
+        s[r].leader = leader;
+    }
+    for (int r = 0; r < kRanks; ++r) sel[size_t(blk) * kRanks + r] = s[r];
+    for (int i = 0; i < kRanks * 256; ++i) hist[size_t(blk) * kRanks * 256 + i] = 0u;
+}
+
+// Start of a select: ranks floor(q (n-1)) and the next one for q = 0.1, 0.9.
+__global__ void select_init_kernel(const StatBlock* __restrict__ blocks, RankSel* __restrict__ sel,
+                                   uint32_t* __restrict__ hist, int n_blocks) {
+    const int blk = blockIdx.x * blockDim.x + threadIdx.x;
+    if (blk >= n_blocks) return;
+    const int64_t n = blocks[blk].numel;
+    const double qs[2] = {0.1, 0.9};
+    for (int k = 0; k < 2; ++k) {
+        const double pos = qs[k] * double(n - 1);
+        const int64_t lo = int64_t(floor(pos));
+        const int64_t hi = min64(lo + 1, n - 1);
+        sel[size_t(blk) * kRanks + 2 * k] = RankSel{0u, 0, lo};
+        sel[size_t(blk) * kRanks + 2 * k + 1] = RankSel{0u, 0, hi};
+    }
+    for (int i = 0; i < kRanks * 256; ++i) hist[size_t(blk) * kRanks * 256 + i] = 0u;
+}
+
+// End of the window: gather everything the host needs into fin_out[block]:
+//   [0..13] sweep-1 sums, [14..15] sweep-2 sums, [16..19] the four order
+//   statistics (as doubles), [20..27] the running window values.
+__global__ void stats_gather_kernel(const RankSel* __restrict__ sel, const double* __restrict__ acc,
+                                    double* __restrict__ fin_out, int n_blocks) {
+    const int blk = blockIdx.x * blockDim.x + threadIdx.x;
+    if (blk >= n_blocks) return;
+    double* o = fin_out + size_t(blk) * kFinOut;
+    for (int r = 0; r < kRanks; ++r) o[16 + r] = double(__uint_as_float(sel[size_t(blk) * kRanks + r].prefix));
+    for (int k = 0; k < kBlockAcc; ++k) o[20 + k] = acc[size_t(blk) * kBlockAcc + k];
+}
+
+// ---- launchers ------------------------------------------------------------------
+#define BAOC_LAUNCH_CHECK()                                   \
+    do {                                                      \
+        cudaError_t e_ = cudaGetLastError();                  \
+        if (e_ != cudaSuccess) return int(e_);                \
+    } while (0)
+
+int launch_stats_step(const StatBlock* blocks, const Tile* tiles, const void* const* grads, double* partials,
+                      int64_t n_tiles, float beta_m, float beta_v, cudaStream_t s) {
+    stats_step_kernel<<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, grads, partials, beta_m, beta_v);
+    BAOC_LAUNCH_CHECK();
+    return 0;
+}
+
+int launch_stats_combine(const StatBlock* blocks, const double* partials, double* acc, int n_blocks, int has_prev,
+                         double beta_rho, double eps, cudaStream_t s) {
+    stats_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, partials, acc, has_prev, beta_rho, eps);
+    BAOC_LAUNCH_CHECK();
+    return 0;
+}
+
+int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
+                      double* fin_out, int64_t n_tiles, int n_blocks, double eps, float eps_adam, cudaStream_t s) {
+    stats_final_sums_kernel<<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, params, fin, eps, eps_adam);
+    BAOC_LAUNCH_CHECK();
+    stats_final_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out);
+    BAOC_LAUNCH_CHECK();
+    return 0;
+}
+
+int launch_final_resid(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
+                       double* fin_out, int64_t n_tiles, int n_blocks, double eps, cudaStream_t s) {
+    stats_final_resid_kernel<<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, params, fin_out, fin, eps);
+    BAOC_LAUNCH_CHECK();
+    stats_resid_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out);
+    BAOC_LAUNCH_CHECK();
+    return 0;
+}
+
+int launch_select(const StatBlock* blocks, const Tile* tiles, RankSel* sel, uint32_t* hist, int64_t n_tiles,
+                  int n_blocks, cudaStream_t s) {
+    const int tb = 128, gb = (n_blocks + tb - 1) / tb;
+    select_init_kernel<<<gb, tb, 0, s>>>(blocks, sel, hist, n_blocks);
+    BAOC_LAUNCH_CHECK();
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        select_hist_kernel<<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, sel, hist, shift);
+        BAOC_LAUNCH_CHECK();
+        select_pick_kernel<<<gb, tb, 0, s>>>(sel, hist, n_blocks, shift);
+        BAOC_LAUNCH_CHECK();
+    }
+    return 0;
+}
+
+int launch_gather(const RankSel* sel, const double* acc, double* fin_out, int n_blocks, cudaStream_t s) {
+    const int tb = 128, gb = (n_blocks + tb - 1) / tb;
+    stats_gather_kernel<<<gb, tb, 0, s>>>(sel, acc, fin_out, n_blocks);
+    BAOC_LAUNCH_CHECK();
+    return 0;
+}
+
+}  // namespace baoc
