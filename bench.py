@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the BAOC hot path on B200.
+
+One "step" is one pass of the whole per-step path over one batch of synthetic
+gradients: the statistics pass (streaming kernel + combine) followed by the
+fused mixed-configuration optimizer step under an assignment that the library
+itself produced (short sampling window -> finalize -> risk -> budgeted
+allocation).  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama_1b] [--impl ours|reference]
+
+``--impl reference`` times the CPU oracle (a deliberately plain double-precision
+program) on a bounded sample of the same workload, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "hot-path throughput: statistics pass + mixed-config optimizer step"
+UNIT = "params/s"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index = index
+        self.rows = []
+        self._halt = threading.Event()
+
+    def run(self):
+        while not self._halt.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                parts = [x.strip() for x in out.strip().split(",")]
+                if len(parts) >= 7:
+                    self.rows.append(parts)
+            except Exception:
+                pass
+            self._halt.wait(0.2)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=6)
+
+    def summary(self):
+        if not self.rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = [float(r[0]) for r in self.rows if r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for k, n in enumerate(names) if any(r[3 + k].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.rows)}
+
+
+# ----------------------------------------------------------------------------
+# CPU oracle timing (the reference arm and the cpu_baseline leg)
+# ----------------------------------------------------------------------------
+
+def _sample_blocks(wl, target_params):
+    """A bounded sample of the workload: blocks in order (skipping any larger than the target) until the target is met."""
+    picked, total = [], 0
+    for i, b in enumerate(wl.blocks):
+        if b.numel > target_params:
+            continue
+        picked.append(i)
+        total += b.numel
+        if total >= target_params:
+            break
+    return picked, total
+
+
+def time_oracle(wl, assign, steps, warmup, target_params):
+    """Time the oracle's statistics step + optimizer step on a sample of blocks.  Returns (params/s, info)."""
+    import numpy as np
+    from threadpoolctl import threadpool_limits
+    from oracle import baoc_oracle as O
+    from paper_2605_04711_b200 import workloads as W
+
+    cfgs = O.default_configs()
+    # same hyper-parameter values as the library's fp32 fields
+    for c in cfgs:
+        for k in ("lr", "beta1", "beta2", "eps", "weight_decay"):
+            setattr(c, k, float(np.float32(getattr(c, k))))
+    picked, total = _sample_blocks(wl, target_params)
+    opts = O.Opts()
+    with threadpool_limits(limits=1):
+        grads = [[W.block_grad(wl, i, t).double().numpy() for i in picked] for t in (1, 2)]
+        theta = [W.block_param(wl, i).double().numpy() for i in picked]
+        sstates = [O.stats_init(wl.blocks[i].numel) for i in picked]
+        ostates = []
+        for j, i in enumerate(picked):
+            b = wl.blocks[i]
+            c = int(assign[i]) if assign is not None else (j % 5)
+            if O.config_kind(cfgs[c]) == "F" and b.cols <= 1:
+                c = 2
+            ostates.append((c, O.step_init(cfgs[c], b.numel, b.rows, b.cols)))
+        times = []
+        for s in range(warmup + steps):
+            t0 = time.perf_counter()
+            for j, i in enumerate(picked):
+                b = wl.blocks[i]
+                g = grads[s % 2][j]
+                O.stats_step(sstates[j], g, opts)
+                c, st = ostates[j]
+                theta[j] = O.step(theta[j], g, st, cfgs[c], b.rows, b.cols)
+            dt = time.perf_counter() - t0
+            if s >= warmup:
+                times.append(dt)
+    sec = sum(times) / len(times)
+    info = {"kind": "oracle", "cores": 1, "unit": UNIT, "value": total / sec,
+            "sample": f"{len(picked)} blocks / {total} params of {wl.name} (first blocks up to {target_params} params), "
+                      f"one statistics step + one optimizer step per timed step, {len(times)} timed steps, numpy float64, 1 thread",
+            "ms_per_step": sec * 1e3}
+    return total / sec, info
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2605_04711_b200 import workloads as W
+    wl = W.make_workload(args.workload, seed=0)
+    # size the sample so that warmup + steps stay within a few minutes on one core
+    target = max(1 << 20, int(6.0e7 / max(args.steps + args.warmup, 1)))
+    value, info = time_oracle(wl, None, args.steps, args.warmup, target)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": info["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": info["sample"]},
+            "cpu_baseline": {k: info[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------
+# The CUDA arm
+# ----------------------------------------------------------------------------
+
+def run_ours(args):
+    import numpy as np
+    import torch
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    from paper_2605_04711_b200 import build
+    build.build()
+    from paper_2605_04711_b200 import harness, workloads as W
+
+    wl = W.make_workload(args.workload, seed=rank)           # replicas: every rank streams its own copy of the workload
+    sess = harness.Session(wl, n_grad_sets=2, device=f"cuda:{local}", pinned_host_grads=True)
+    sess.init_params()
+    for t in (1, 2):
+        k = sess.fill_grads(t)
+        sess.host_copy_of_grads(k)
+    sess._fixed_cache.clear()
+    torch.cuda.synchronize()
+
+    # short sampling window -> risk -> allocation -> configure (set-up, timed separately)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for t in range(1, args.window + 1):
+        sess.sample_stats(t % 2)
+    e0, e1 = ev(), ev()
+    e0.record()
+    risk, stats = sess.risk()
+    e1.record()
+    torch.cuda.synchronize()
+    finalize_ms = e0.elapsed_time(e1)
+    t0 = time.perf_counter()
+    assign, objective, rc = sess.allocate(risk)
+    alloc_ms = (time.perf_counter() - t0) * 1e3
+    sess.configure(assign)
+    info = sess.h.query()
+    stats_bytes, step_bytes = info.stats_bytes_per_call, info.step_bytes_per_call
+    counts = np.bincount(assign, minlength=len(sess.configs)).tolist()
+    params_by_cfg = [int(sum(b.numel for b, a in zip(wl.blocks, assign) if a == c)) for c in range(len(sess.configs))]
+
+    def one_step(s, t):
+        sess.sample_stats(s % 2)
+        sess.step(s % 2, t)
+
+    step_t = 0
+    for s in range(args.warmup):
+        step_t += 1
+        one_step(s, step_t)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    launches0 = sess.h.query().kernel_launches
+    sampler = ClockSampler(local)
+    sampler.start()
+    marks = [ev() for _ in range(2 * args.steps + 1)]
+    marks[0].record()
+    for s in range(args.steps):
+        step_t += 1
+        sess.sample_stats(s % 2)
+        marks[2 * s + 1].record()
+        sess.step(s % 2, step_t)
+        marks[2 * s + 2].record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+        torch.cuda.synchronize()
+    sampler.stop()
+    launches = sess.h.query().kernel_launches - launches0
+
+    total_ms = marks[0].elapsed_time(marks[-1])
+    stats_ms = sum(marks[2 * s].elapsed_time(marks[2 * s + 1]) for s in range(args.steps)) / args.steps
+    step_ms = sum(marks[2 * s + 1].elapsed_time(marks[2 * s + 2]) for s in range(args.steps)) / args.steps
+    t_max = torch.tensor([total_ms], dtype=torch.float64, device=f"cuda:{local}")
+    if dist is not None:
+        dist.all_reduce(t_max, op=dist.ReduceOp.MAX)
+    total_ms_max = float(t_max.item())
+    ms_per_step = total_ms_max / args.steps
+    value = world * wl.numel / (ms_per_step * 1e-3)
+    cnt, _ = sess.h.nonfinite()
+
+    # end to end: gradients start in pinned host memory, the per-block running statistics come back
+    e2e_steps = max(1, min(args.e2e_steps, args.steps))
+    d2h = 0
+    torch.cuda.synchronize()
+    ea, eb = ev(), ev()
+    ea.record()
+    for s in range(e2e_steps):
+        step_t += 1
+        sess.step_from_host(s % 2, True, step_t)
+        running = sess.h.read_stats()
+    eb.record()
+    torch.cuda.synchronize()
+    e2e_ms = ea.elapsed_time(eb) / e2e_steps
+    t_e2e = torch.tensor([e2e_ms], dtype=torch.float64, device=f"cuda:{local}")
+    if dist is not None:
+        dist.all_reduce(t_e2e, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t_e2e.item())
+    d2h = 8 * 8 * len(wl.blocks)
+    h2d = 2 * wl.numel
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = _peaks()
+    stats_gbs = stats_bytes / (stats_ms * 1e-3) / 1e9
+    step_gbs = step_bytes / (step_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "params": wl.numel, "blocks": len(wl.blocks), "grad_dtype": "bf16",
+                   "param_dtype": "f32", "candidate_configs": ["adamw32", "adamw8", "rms", "factored", "sgdm"],
+                   "assignment_blocks_per_config": counts, "assignment_params_per_config": params_by_cfg,
+                   "mem_budget_frac_of_fp32_adam": wl.mem_budget_frac, "state_bytes": int(info.state_bytes),
+                   "window_steps_before_timing": args.window, "l2": "inputs (>10 GB per step) far exceed the 126 MB L2",
+                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                   "allocator_status": int(rc), "nonfinite_blocks": int(cnt)},
+        "clocks": sampler.summary(),
+        "gpu_launches": int(launches),
+        "e2e": {"value": world * wl.numel / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps},
+        "roofline": {"kernel": "stats_step_kernel (+ its microsecond combine)", "bound": "hbm", "achieved": stats_gbs,
+                     "peak": peak, "unit": "GB/s", "frac": stats_gbs / peak, "peak_kind": peak_kind,
+                     "frac_of_8TBs": stats_gbs / 8000.0, "bytes_per_launch": int(stats_bytes), "ms": stats_ms,
+                     "traffic": args.traffic_stats},
+        "roofline_step": {"kernel": "fused_step_kernel (+ factored row/column kernels)", "bound": "hbm",
+                          "achieved": step_gbs, "peak": peak, "unit": "GB/s", "frac": step_gbs / peak,
+                          "frac_of_8TBs": step_gbs / 8000.0, "bytes_per_launch": int(step_bytes), "ms": step_ms,
+                          "params_per_s": wl.numel / (step_ms * 1e-3), "traffic": args.traffic_step},
+        "stats_pass": {"ms": stats_ms, "GBps": stats_gbs, "params_per_s": wl.numel / (stats_ms * 1e-3)},
+        "mixed_step": {"ms": step_ms, "GBps": step_gbs, "params_per_s": wl.numel / (step_ms * 1e-3)},
+        "once_per_window": {"finalize_and_risk_ms": finalize_ms, "allocate_ms": alloc_ms, "objective": objective},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        _, cb = time_oracle(wl, assign, 2, 1, args.cpu_sample_params)
+        line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama_1b")
+    ap.add_argument("--window", type=int, default=4, help="statistics steps before the finalize that feeds the allocation")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-sample-params", type=int, default=40_000_000)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic-stats", type=float, default=None, help="ncu DRAM bytes per launch of the statistics kernel, if known")
+    ap.add_argument("--traffic-step", type=float, default=None)
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

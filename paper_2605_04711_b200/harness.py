@@ -1,0 +1,102 @@
+"""Device-side plumbing shared by the tests, the smoke check and the benchmark.
+
+Allocates the flat parameter / gradient buffers and the library's workspaces
+with PyTorch, fills them from the seeded generators in ``workloads`` and drives
+the C ABI through ``binding``.  No arithmetic of the method lives here.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import workloads as W
+
+
+class Session:
+    """One workload resident on one GPU.
+
+    params: one flat fp32 buffer, block i at ``offs[i]`` (128-element aligned).
+    grads:  ``n_grad_sets`` flat bf16 buffers with the same offsets; set k holds
+    the gradients of step t for t % n_grad_sets == k once ``fill_grads(t)`` ran.
+    """
+
+    def __init__(self, wl: W.Workload, configs: Optional[Sequence[B.Config]] = None, opts: Optional[B.Opts] = None,
+                 n_grad_sets: int = 2, device: str = "cuda:0", pinned_host_grads: bool = False):
+        self.wl = wl
+        self.device = torch.device(device)
+        self.configs = list(configs) if configs is not None else B.default_configs()
+        self.h = B.Baoc(wl.blocks, self.configs, opts)
+        self.offs, self.total = W.flat_layout(wl, 128)
+        self.n_grad_sets = n_grad_sets
+        self.params = torch.zeros(self.total, dtype=torch.float32, device=self.device)
+        self.grads = [torch.zeros(self.total, dtype=torch.bfloat16, device=self.device) for _ in range(n_grad_sets)]
+        self.param_views = [self.params[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)]
+        self.grad_views = [[g[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)] for g in self.grads]
+        self.param_table = B.pointer_table(self.param_views)
+        self.grad_tables = [B.pointer_table(v) for v in self.grad_views]
+        self.host_grads = None
+        if pinned_host_grads:
+            self.host_grads = [torch.zeros(self.total, dtype=torch.bfloat16).pin_memory() for _ in range(n_grad_sets)]
+            self.host_tables = [B.pointer_table([hg[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)])
+                                for hg in self.host_grads]
+        self.ws = torch.empty(self.h.stats_workspace_bytes(), dtype=torch.uint8, device=self.device)
+        self.h.bind_stats_workspace(self.ws)
+        self.state = None
+        self.assign = None
+        self._fixed_cache = {}
+
+    # ---- inputs -------------------------------------------------------------
+    def init_params(self):
+        for i, v in enumerate(self.param_views):
+            v.copy_(W.block_param(self.wl, i, device=self.device))
+
+    def fill_grads(self, t: int, blocks: Optional[Sequence[int]] = None, cache_fixed: bool = False):
+        """Generate the gradients of step t (1-based) into set t % n_grad_sets."""
+        k = t % self.n_grad_sets
+        for i in (range(len(self.wl.blocks)) if blocks is None else blocks):
+            fixed = None
+            if cache_fixed:
+                if i not in self._fixed_cache:
+                    self._fixed_cache[i] = W.block_fixed_parts(self.wl, i, self.device)
+                fixed = self._fixed_cache[i]
+            W.block_grad(self.wl, i, t, device=self.device, fixed=fixed, out=self.grad_views[k][i])
+        return k
+
+    def host_copy_of_grads(self, k: int):
+        if self.host_grads is not None:
+            self.host_grads[k].copy_(self.grads[k])
+
+    # ---- the path -------------------------------------------------------------
+    def sample_stats(self, k: int):
+        self.h.sample_stats(self.grad_tables[k])
+
+    def risk(self):
+        return self.h.risk(self.param_table)
+
+    def allocate(self, risk, time_ratio=None, forbid=None, pref=None):
+        mem, ratio = self.h.cost_model()
+        if time_ratio is not None:
+            ratio = np.asarray(time_ratio, np.float64)
+        b_mem = int(np.floor(self.wl.mem_budget_frac * 8.0 * self.wl.numel))
+        return self.h.allocate(risk, mem, ratio, b_mem, self.wl.time_budget, forbid, pref)
+
+    def configure(self, assign):
+        self.assign = np.asarray(assign, np.int32)
+        self.state = torch.empty(self.h.state_bytes(self.assign), dtype=torch.uint8, device=self.device)
+        self.h.configure(self.assign, self.state)
+
+    def step(self, k: int, t: int):
+        self.h.step(self.grad_tables[k], self.param_table, t)
+
+    def step_from_host(self, k: int, do_stats: bool, t: int):
+        self.h.step_from_host(self.host_tables[k], self.grad_tables[k], self.param_table, do_stats, t)
+
+    # ---- read-back for checks ---------------------------------------------------
+    def block_grad_host(self, k: int, i: int) -> np.ndarray:
+        return self.grad_views[k][i].double().cpu().numpy()
+
+    def block_param_host(self, i: int) -> np.ndarray:
+        return self.param_views[i].double().cpu().numpy()

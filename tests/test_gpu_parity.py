@@ -1,0 +1,348 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded inputs.
+
+Tolerances (from the benchmark spec):
+  * statistics: 1e-4 relative (bounded signals are compared against
+    max(|ref|, 1e-3) so that a cosine near zero is not held to 1e-4 of nothing);
+  * fp32 states and parameters after 10 steps: max|diff| <= 1e-6 * max|ref| per
+    block;
+  * 8-bit codes: identical on >= 99.99 % of the elements, within 1 code elsewhere;
+  * allocation: bit-exact.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import baoc_oracle as O
+from paper_2605_04711_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+STAT_KEYS = ("A", "rho_bar", "snr", "C", "F", "Q32", "Q16", "Q8", "q10", "q90", "rho_mom",
+             "err_m8", "err_v8", "err_m16", "err_v16")
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2605_04711_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def H():
+    from paper_2605_04711_b200 import harness
+    return harness
+
+
+def _ocfg(c):
+    return O.Config(c.adaptive, c.momentum, c.decoupled_wd, c.factored, c.bits, lr=float(c.lr), beta1=float(c.beta1),
+                    beta2=float(c.beta2), eps=float(c.eps), weight_decay=float(c.weight_decay))
+
+
+def _close(got, ref, rel=1e-4, floor=1e-3):
+    return abs(got - ref) <= rel * max(abs(ref), floor)
+
+
+def _odd_workload(seed=3, window=6):
+    shapes = [(1, 1), (7, 1), (255, 1), (256, 1), (257, 1), (4097, 1), (6149, 1), (37, 53), (64, 147), (300, 520),
+              (5000, 8), (3, 3), (4096, 1), (130, 64), (8200, 1)]
+    blocks = [W.Block(f"odd{i}", r, c) for i, (r, c) in enumerate(shapes)]
+    rng = np.random.default_rng(seed)
+    for b in blocks:
+        b.stability = float(rng.uniform(0.05, 0.95))
+        b.tau = float(rng.uniform(0.0, 2.0))
+        b.scale = float(10.0 ** rng.uniform(-3, -1))
+    blocks[5].heavy_tail = True
+    return W.Workload("odd", blocks, window=window, mem_budget_frac=0.4, time_budget=1.3, seed=seed)
+
+
+def _oracle_window(sess, T, opts=None):
+    """Run T statistics steps on GPU and oracle; returns (oracle states, per-step cosines ok)."""
+    o = opts or O.Opts()
+    wl = sess.wl
+    states = [O.stats_init(b.numel) for b in wl.blocks]
+    for t in range(1, T + 1):
+        k = sess.fill_grads(t)
+        sess.sample_stats(k)
+        for i in range(len(wl.blocks)):
+            O.stats_step(states[i], sess.block_grad_host(k, i), o)
+    return states
+
+
+def _check_stats(sess, states, opts=None, skip_small_C=True):
+    o = opts or O.Opts()
+    wl = sess.wl
+    risk, st = sess.risk()
+    cfgs = [_ocfg(c) for c in sess.configs]
+    worst = {}
+    for i, b in enumerate(wl.blocks):
+        raw = O.stats_finalize(states[i], sess.block_param_host(i), b.rows, b.cols, o)
+        for k in STAT_KEYS:
+            got, ref = st[i][k], raw[k]
+            ok = _close(got, ref)
+            worst[k] = max(worst.get(k, 0.0), abs(got - ref) / max(abs(ref), 1e-3))
+            assert ok, (b.name, k, got, ref)
+        assert st[i]["n_cos"] == states[i].n_cos
+        z = O.normalise(raw, o)
+        for c, cfg in enumerate(cfgs):
+            ref = O.risk(z, cfg, o)
+            assert abs(risk[i, c] - ref) <= 1e-4 * max(abs(ref), 1e-2), (b.name, c, risk[i, c], ref)
+    return risk, st, worst
+
+
+# ---------------------------------------------------------------- statistics pass
+
+def test_stats_window_odd_sizes(B, H):
+    wl = _odd_workload()
+    sess = H.Session(wl, n_grad_sets=2)
+    sess.init_params()
+    states = _oracle_window(sess, wl.window)
+    run = sess.h.read_stats()
+    for i in range(len(wl.blocks)):
+        assert _close(run[i]["rho_bar"], states[i].rho_bar), (i, run[i]["rho_bar"], states[i].rho_bar)
+        assert _close(run[i]["last_cos"], states[i].last_cos)
+        assert run[i]["n_cos"] == wl.window - 1
+        m = sess.h.view_tensor(i, 0, torch.float32).double().cpu().numpy()
+        v = sess.h.view_tensor(i, 1, torch.float32).double().cpu().numpy()
+        gp = sess.h.view_tensor(i, 2, torch.bfloat16).double().cpu().numpy()
+        assert np.max(np.abs(m - states[i].m)) <= 1e-6 * max(np.max(np.abs(states[i].m)), 1e-30)
+        assert np.max(np.abs(v - states[i].v)) <= 1e-6 * max(np.max(np.abs(states[i].v)), 1e-30)
+        np.testing.assert_array_equal(gp, states[i].g_prev)
+    _check_stats(sess, states)
+    info = sess.h.query()
+    assert info.stats_steps == wl.window and info.kernel_launches > 0
+
+
+def test_stats_invariants_identical_zero_and_flipped_gradients(B, H):
+    wl = _odd_workload(seed=5)
+    sess = H.Session(wl, n_grad_sets=1)
+    sess.init_params()
+    sess.fill_grads(1)
+    n = len(wl.blocks)
+    sess.grad_views[0][2].zero_()                                   # one block sees no gradient at all
+    for _ in range(4):
+        sess.sample_stats(0)
+    run = sess.h.read_stats()
+    for i in range(n):
+        want = 0.0 if i == 2 else 1.0
+        assert abs(run[i]["rho_bar"] - want) < 1e-9, (i, run[i]["rho_bar"])   # identical gradients: stability 1
+    sess.grads[0].neg_()
+    sess.sample_stats(0)
+    run = sess.h.read_stats()
+    for i in range(n):
+        if i != 2:
+            assert abs(run[i]["last_cos"] + 1.0) < 1e-9
+    # |g_j| constant over a block: isotropic second moment, anisotropy 0
+    risk, st = sess.risk()
+    wl2 = _odd_workload(seed=6)
+    sess2 = H.Session(wl2, n_grad_sets=1)
+    sess2.init_params()
+    sess2.fill_grads(1)
+    g = sess2.grads[0]
+    g.copy_(torch.where(g.float() >= 0, torch.full_like(g, 0.5), torch.full_like(g, -0.5)))
+    for _ in range(3):
+        sess2.sample_stats(0)
+    _, st2 = sess2.risk()
+    for i in range(len(wl2.blocks)):
+        assert abs(st2[i]["A"]) < 1e-9 and st2[i]["s_A"] == 0.0
+        assert abs(st2[i]["C"]) < 1e-9                               # constant preconditioner: no distortion
+        if wl2.blocks[i].cols > 1:
+            assert st2[i]["F"] < 1e-6                                # constant matrix is rank one
+
+
+def test_stats_is_deterministic(B, H):
+    wl = _odd_workload(seed=8, window=3)
+    outs = []
+    for _ in range(2):
+        sess = H.Session(wl, n_grad_sets=1)
+        sess.init_params()
+        for t in range(1, 4):
+            sess.sample_stats(sess.fill_grads(t))
+        risk, st = sess.risk()
+        outs.append((risk.copy(), [tuple(s[k] for k in STAT_KEYS) for s in st]))
+    np.testing.assert_array_equal(outs[0][0], outs[1][0])
+    assert outs[0][1] == outs[1][1]
+
+
+# ---------------------------------------------------------------- update paths
+
+def _run_steps(sess, assign, n_steps, first_t=1):
+    """Steps on GPU and oracle from zero state; returns the oracle's params and states."""
+    wl = sess.wl
+    cfgs = [_ocfg(c) for c in sess.configs]
+    sess.configure(assign)
+    th = [sess.block_param_host(i) for i in range(len(wl.blocks))]
+    sts = [O.step_init(cfgs[assign[i]], b.numel, b.rows, b.cols) for i, b in enumerate(wl.blocks)]
+    for t in range(first_t, first_t + n_steps):
+        k = sess.fill_grads(t)
+        sess.step(k, t - first_t + 1)
+        for i, b in enumerate(wl.blocks):
+            th[i] = O.step(th[i], sess.block_grad_host(k, i), sts[i], cfgs[assign[i]], b.rows, b.cols)
+    return th, sts
+
+
+def _rel_max(got, ref):
+    return float(np.max(np.abs(got - ref)) / max(float(np.max(np.abs(ref))), 1e-30))
+
+
+def _check_block(sess, i, th_ref, st_ref, code_stats):
+    got = sess.block_param_host(i)
+    assert np.all(np.isfinite(got))
+    assert _rel_max(got, th_ref) <= 1e-6, (sess.wl.blocks[i].name, st_ref.kind, _rel_max(got, th_ref))
+    kind = st_ref.kind
+    f32 = lambda w: sess.h.view_tensor(i, w, torch.float32).double().cpu().numpy()
+    if kind == "A32":
+        assert _rel_max(f32(10), st_ref.m) <= 1e-6 and _rel_max(f32(11), st_ref.v) <= 1e-6
+    elif kind == "R":
+        assert _rel_max(f32(10), st_ref.v) <= 1e-6
+    elif kind == "S":
+        assert _rel_max(f32(10), st_ref.m) <= 1e-6
+    elif kind == "F":
+        assert _rel_max(f32(10), st_ref.r) <= 1e-6 and _rel_max(f32(11), st_ref.c) <= 1e-6
+    elif kind == "A8":
+        qm = sess.h.view_tensor(i, 10, torch.int8).cpu().numpy().astype(np.int32)
+        qv = sess.h.view_tensor(i, 11, torch.uint8).cpu().numpy().astype(np.int32)
+        dm = np.abs(qm - st_ref.qm.astype(np.int32)); dv = np.abs(qv - st_ref.qv.astype(np.int32))
+        assert dm.max() <= 1 and dv.max() <= 1
+        code_stats[0] += int((dm != 0).sum() + (dv != 0).sum()); code_stats[1] += 2 * qm.size
+        assert _rel_max(f32(12), st_ref.am.astype(np.float64)) <= 1e-6
+        assert _rel_max(f32(13), st_ref.av.astype(np.float64)) <= 1e-6
+
+
+@pytest.mark.parametrize("cfg_index", [0, 1, 2, 3, 4])
+def test_each_configuration_ten_steps_odd_sizes(B, H, cfg_index):
+    wl = _odd_workload(seed=11 + cfg_index)
+    sess = H.Session(wl, n_grad_sets=2)
+    sess.init_params()
+    assign = [cfg_index if not (cfg_index == 3 and b.cols <= 1) else 2 for b in wl.blocks]
+    th, sts = _run_steps(sess, assign, 10)
+    codes = [0, 0]
+    for i in range(len(wl.blocks)):
+        _check_block(sess, i, th[i], sts[i], codes)
+    if codes[1]:
+        assert codes[0] <= 1e-4 * codes[1], codes
+    cnt, flags = sess.h.nonfinite()
+    assert cnt == 0
+    info = sess.h.query()
+    mem, _ = sess.h.cost_model()
+    assert info.state_bytes == sum(int(mem[i, c]) for i, c in enumerate(assign))
+
+
+def test_coupled_decay_and_other_hyperparameters(B, H):
+    wl = _odd_workload(seed=21)
+    cfgs = [B.make_config(1, 1, 0, 0, 32, lr=3e-3, beta1=0.8, beta2=0.95, eps=1e-6, weight_decay=0.1),
+            B.make_config(1, 1, 0, 0, 8, lr=3e-3, beta1=0.8, beta2=0.95, eps=1e-6, weight_decay=0.1),
+            B.make_config(1, 0, 0, 0, 32, lr=1e-3, beta2=0.9, eps=1e-6, weight_decay=0.1),
+            B.make_config(1, 0, 0, 1, 32, lr=1e-3, beta2=0.9, eps=1e-6, weight_decay=0.1),
+            B.make_config(0, 1, 0, 0, 32, lr=1e-2, beta1=0.5, weight_decay=0.1)]
+    sess = H.Session(wl, configs=cfgs, n_grad_sets=2)
+    sess.init_params()
+    assign = [(i % 5) if not ((i % 5) == 3 and b.cols <= 1) else 0 for i, b in enumerate(wl.blocks)]
+    th, sts = _run_steps(sess, assign, 10)
+    codes = [0, 0]
+    for i in range(len(wl.blocks)):
+        _check_block(sess, i, th[i], sts[i], codes)
+    assert codes[0] <= 1e-4 * max(codes[1], 1)
+
+
+def test_nonfinite_gradient_is_flagged_not_fatal(B, H):
+    wl = _odd_workload(seed=31)
+    sess = H.Session(wl, n_grad_sets=1)
+    sess.init_params()
+    sess.configure([0] * len(wl.blocks))
+    sess.fill_grads(1)
+    sess.grad_views[0][4][3] = float("nan")
+    sess.grad_views[0][9][17] = float("inf")
+    sess.step(0, 1)
+    cnt, flags = sess.h.nonfinite()
+    assert cnt == 2 and flags[4] == 1 and flags[9] == 1 and flags.sum() == 2
+    sess.fill_grads(2)
+    sess.step(0, 2)                                                  # the context is still usable
+
+
+def test_gpu_argument_checks(B, H):
+    wl = _odd_workload(seed=41)
+    sess = H.Session(wl, n_grad_sets=1)
+    bad = B.pointer_table(sess.grad_views[0])
+    bad[3] = bad[3] + 2                                              # misaligned device pointer
+    with pytest.raises(B.BaocError) as e:
+        sess.h.sample_stats(bad)
+    assert e.value.code == B.E_ALIGN
+    bad[3] = None
+    with pytest.raises(B.BaocError) as e:
+        sess.h.sample_stats(bad)
+    assert e.value.code == B.E_INVALID
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.BaocError) as e:
+        sess.h.bind_stats_workspace(small)
+    assert e.value.code == B.E_WORKSPACE
+    with pytest.raises(B.BaocError) as e:
+        sess.h.configure(np.zeros(len(wl.blocks), np.int32), small)
+    assert e.value.code == B.E_WORKSPACE
+    with pytest.raises(B.BaocError) as e:
+        sess.h.risk(sess.param_table)                                # no gradient observed yet
+    assert e.value.code == B.E_STATE
+
+
+# ---------------------------------------------------------------- whole pipeline
+
+def _pipeline(B, H, name, T, n_steps, time_table=None):
+    wl = W.make_workload(name, seed=0)
+    sess = H.Session(wl, n_grad_sets=2)
+    sess.init_params()
+    states = _oracle_window(sess, T)
+    risk, st, worst = _check_stats(sess, states)
+    # allocation: the library on the GPU's risk and on the oracle's risk must agree here
+    o = O.Opts()
+    cfgs = [_ocfg(c) for c in sess.configs]
+    risk_ref = np.zeros_like(risk)
+    for i, b in enumerate(wl.blocks):
+        z = O.normalise(O.stats_finalize(states[i], sess.block_param_host(i), b.rows, b.cols, o), o)
+        for c in range(len(cfgs)):
+            risk_ref[i, c] = O.risk(z, cfgs[c], o)
+    asg, obj, rc = sess.allocate(risk, time_table)
+    asg_ref, obj_ref, rc_ref = sess.allocate(risk_ref, time_table)
+    assert rc == 0 and rc_ref == 0
+    assert asg.tolist() == asg_ref.tolist(), (obj, obj_ref)
+    mem, _ = sess.h.cost_model()
+    assert sum(int(mem[i, c]) for i, c in enumerate(asg)) <= int(wl.mem_budget_frac * 8 * wl.numel)
+    th, sts = _run_steps(sess, asg.tolist(), n_steps, first_t=T + 1)
+    codes = [0, 0]
+    for i in range(len(wl.blocks)):
+        _check_block(sess, i, th[i], sts[i], codes)
+    if codes[1]:
+        assert codes[0] <= 1e-4 * codes[1], codes
+    return asg
+
+
+def test_toy_pipeline_window_risk_allocation_ten_mixed_steps(B, H):
+    asg = _pipeline(B, H, "toy", 8, 10)
+    assert len(set(asg.tolist())) >= 2                               # the budget forces a mixed assignment
+
+
+def test_toy_allocation_matches_brute_force_on_eight_blocks(B, H):
+    wl = W.make_workload("toy", seed=0)
+    wl.blocks = wl.blocks[:8]
+    sess = H.Session(wl, n_grad_sets=2)
+    sess.init_params()
+    states = _oracle_window(sess, 4)
+    risk, st, _ = _check_stats(sess, states)
+    asg, obj, rc = sess.allocate(risk)
+    o = O.Opts()
+    cfgs = [_ocfg(c) for c in sess.configs]
+    mem, ratio = sess.h.cost_model()
+    n, K = risk.shape
+    phi = [[O.phi_fixed(O.objective(risk[i, c], cfgs[c], o)) for c in range(K)] for i in range(n)]
+    rfx = [[O.ratio_fixed(ratio[i, c]) for c in range(K)] for i in range(n)]
+    forbid = [[int(O.config_kind(cfgs[c]) == "F" and wl.blocks[i].cols <= 1) for c in range(K)] for i in range(n)]
+    want, val = O.allocate_bruteforce(phi, mem.tolist(), rfx, int(math.floor(wl.mem_budget_frac * 8.0 * wl.numel)),
+                                      O.time_cap_fixed(n, wl.time_budget), forbid)
+    assert asg.tolist() == want and obj == val / 2.0 ** 30
+
+
+def test_resnet50_pipeline_with_binding_time_budget(B, H):
+    wl = W.make_workload("resnet50")
+    table = W.time_ratio_table(wl, [1.0, 1.25, 0.8, 1.5, 0.7]).numpy()
+    _pipeline(B, H, "resnet50", 4, 3, table)
