@@ -55,7 +55,7 @@ int do_sample_stats(Handle* h, const void* const* grads, cudaStream_t s) {
     const auto& L = h->sl;
     LAUNCH(launch_stats_step(at<StatBlock>(h->ws, L.blocks), at<Tile>(h->ws, L.tiles),
                              at<const void*>(h->ws, L.grads), at<double>(h->ws, L.partials), h->n_stat_tiles,
-                             float(h->opts.beta_m), float(h->opts.beta_v), s), "stats_step_kernel");
+                             float(1.0 - h->opts.beta_m), float(1.0 - h->opts.beta_v), s), "stats_step_kernel");
     LAUNCH(launch_stats_combine(at<StatBlock>(h->ws, L.blocks), at<double>(h->ws, L.partials), at<double>(h->ws, L.acc),
                                 h->n_blocks, h->stats_steps > 0 ? 1 : 0, h->opts.beta_rho, h->opts.eps, s),
            "stats_combine_kernel");
@@ -69,13 +69,17 @@ void fill_step_params(const Handle* h, int64_t t, StepParams* P) {
     for (int c = 0; c < h->n_cfg; ++c) {
         const baoc_config_t& k = h->cfgs[c];
         CfgStep& o = P->c[c];
-        o.lr = k.lr; o.beta1 = k.beta1; o.beta2 = k.beta2; o.eps = k.eps; o.wd = k.weight_decay;
+        const double b1 = double(k.beta1), b2 = double(k.beta2), lr = double(k.lr);
+        o.beta1 = k.beta1; o.beta2 = k.beta2; o.eps = k.eps; o.wd = k.weight_decay;
+        o.om1 = float(1.0 - b1); o.om2 = float(1.0 - b2);
         const bool has_wd = k.weight_decay != 0.0f;
         o.coupled = (has_wd && !k.decoupled_wd) ? 1 : 0;
-        o.decay = (has_wd && k.decoupled_wd) ? -float(double(k.lr) * double(k.weight_decay)) : 0.0f;
-        o.bc1 = float(1.0 - std::pow(double(k.beta1), double(t)));
-        o.bc2 = float(1.0 - std::pow(double(k.beta2), double(t)));
-        o.beta1_d = double(k.beta1); o.beta2_d = double(k.beta2);
+        o.decay = (has_wd && k.decoupled_wd) ? -float(lr * double(k.weight_decay)) : 0.0f;
+        const double bc1 = 1.0 - std::pow(b1, double(t)), bc2 = 1.0 - std::pow(b2, double(t));
+        o.step_m = float(lr / bc1);
+        o.step_g = k.lr;
+        o.rsqrt_bc2 = float(1.0 / std::sqrt(bc2));
+        o.beta1_d = b1; o.beta2_d = b2; o.wd_d = double(k.weight_decay);
     }
 }
 
@@ -91,8 +95,9 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
     CU(cudaMemsetAsync(h->st + L.flags, 0, 4 * size_t(h->n_blocks), s), "baoc_step (flags)");
     if (h->n_factored > 0) {
         LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles),
-                                      at<int32_t>(h->st, L.f_ids), at<const void*>(h->st, L.grads), h->n_step_red_tiles,
-                                      h->n_factored, P, s), "factored_reduce_kernel");
+                                      at<int32_t>(h->st, L.f_ids), at<const void*>(h->st, L.grads),
+                                      at<const float*>(h->st, L.params), h->n_step_red_tiles, h->n_factored, P, s),
+               "factored_reduce_kernel");
         h->launches += 2;
     }
     LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles), at<const void*>(h->st, L.grads),

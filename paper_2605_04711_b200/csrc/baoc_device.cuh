@@ -114,15 +114,28 @@ __device__ __forceinline__ float warp_max(float x) {
 // code = clamp(rne(L * x / a)), x ~ code * a / L, with L = 127 (signed) or 255
 // (unsigned) and a the fp32 absmax of the 256-element quantisation block.  The
 // scaling and rounding are done in double so that the decision agrees with a
-// double-precision evaluation of the same formula.
+// double-precision evaluation of the same formula.  The fast path multiplies by
+// the precomputed L / a; that product is within a few ulp of (L * x) / a, so the
+// two can only round to different integers when the value sits on a tie.  bf16
+// gradients make exact ties common (x / a is often a ratio of small integers),
+// hence a value within 1e-9 of a half-integer is redone with the division, which
+// is the correctly rounded form of the definition.
 __device__ __forceinline__ double code_scale(float absmax, double levels) {
     return absmax > 0.0f ? levels / double(absmax) : 0.0;
 }
-__device__ __forceinline__ int encode_signed(double x, double scale) {
-    return max(-127, min(127, round_to_int(x * scale)));
+__device__ __forceinline__ int encode_round(double x, float absmax, double scale, double levels) {
+    constexpr double kMagic = 6755399441055744.0;                 // 1.5 * 2^52: adding it rounds to an integer, ties to even
+    const double q = x * scale;
+    const double t = q + kMagic;
+    const double d = q - (t - kMagic);                            // signed distance to the chosen integer
+    if (fabs(d) > 0.5 - 1e-9) return __double2loint((levels * x) / double(absmax) + kMagic);
+    return __double2loint(t);
 }
-__device__ __forceinline__ int encode_unsigned(double x, double scale) {
-    return max(0, min(255, round_to_int(x * scale)));
+__device__ __forceinline__ int encode_signed(double x, float absmax, double scale) {
+    return max(-127, min(127, encode_round(x, absmax, scale, 127.0)));
+}
+__device__ __forceinline__ int encode_unsigned(double x, float absmax, double scale) {
+    return max(0, min(255, encode_round(x, absmax, scale, 255.0)));
 }
 
 }  // namespace baoc

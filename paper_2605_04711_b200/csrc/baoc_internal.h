@@ -103,13 +103,18 @@ struct RedTile {
 
 // Per-configuration scalars of one step, passed to the kernel by value.
 struct CfgStep {
-    float lr, beta1, beta2, eps;
+    float beta1, beta2;
+    float om1, om2;      // 1 - beta1, 1 - beta2 (rounded from double)
+    float eps;
     float wd;            // weight decay coefficient
     float decay;         // -lr*wd when the decay is decoupled, else 0
-    float bc1, bc2;      // 1 - beta1^t, 1 - beta2^t
-    double beta1_d, beta2_d;   // the same coefficients widened, for the 8-bit path
+    float step_m;        // lr / (1 - beta1^t): multiplies a bias-corrected first moment
+    float step_g;        // lr: multiplies a raw gradient or momentum buffer
+    float rsqrt_bc2;     // 1 / sqrt(1 - beta2^t)
     int32_t coupled;     // 1: add wd*theta to the gradient
     int32_t pad;
+    double beta1_d, beta2_d;   // the coefficients widened, for the exact side of the 8-bit path
+    double wd_d;
 };
 struct StepParams {
     CfgStep c[kMaxCfg];
@@ -172,7 +177,7 @@ void compute_stat_layout(Handle* h);
 
 // Kernel launchers (defined in the .cu files).  Each returns 0 or a cudaError_t value.
 int launch_stats_step(const StatBlock* blocks, const Tile* tiles, const void* const* grads, double* partials,
-                      int64_t n_tiles, float beta_m, float beta_v, cudaStream_t s);
+                      int64_t n_tiles, float one_minus_beta_m, float one_minus_beta_v, cudaStream_t s);
 int launch_stats_combine(const StatBlock* blocks, const double* partials, double* acc, int n_blocks, int has_prev,
                          double beta_rho, double eps, cudaStream_t s);
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
@@ -185,7 +190,7 @@ int launch_gather(const RankSel* sel, const double* acc, double* fin_out, int n_
 int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const int32_t* ids, int64_t n_red, int n_matrix,
                          cudaStream_t s);
 int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const int32_t* ids, const void* const* grads,
-                           int64_t n_red, int n_factored, const StepParams& P, cudaStream_t s);
+                           const float* const* params, int64_t n_red, int n_factored, const StepParams& P, cudaStream_t s);
 int launch_fused_step(const StepBlock* blocks, const Tile* tiles, const void* const* grads, float* const* params,
                       uint32_t* flags, int64_t n_tiles, const StepParams& P, cudaStream_t s);
 int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayout* out,

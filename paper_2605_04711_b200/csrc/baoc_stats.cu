@@ -12,9 +12,14 @@ namespace baoc {
 // (bf16), m, v (fp32); writes m, v, g_{t-1}; leaves 4 partial sums per tile:
 // <g_t, g_{t-1}>, ||g_t||^2, <g_t, m_{t-1}>, ||m_{t-1}||^2.
 // ============================================================================
+// Eq. 3 as s + (1 - beta)(x - s): only 1 - beta enters, and it is rounded to
+// fp32 from its double value, so the recursion's coefficient carries no
+// cancellation error (1.0f - float(0.999) is off by 1.3e-5 relative).
+__device__ __forceinline__ float ema(float s, float x, float one_minus_beta) { return fmaf(one_minus_beta, x - s, s); }
+
 __global__ void __launch_bounds__(kThreads)
 stats_step_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
-                  const void* const* __restrict__ grads, double* __restrict__ partials, float beta_m, float beta_v) {
+                  const void* const* __restrict__ grads, double* __restrict__ partials, float om, float ov) {
     const Tile t = tiles[blockIdx.x];
     const StatBlock* b = blocks + t.block;
     const int64_t numel = b->numel;
@@ -23,7 +28,6 @@ stats_step_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
     float* __restrict__ m = b->m;
     float* __restrict__ v = b->v;
     const int64_t base = int64_t(t.piece) * kTile;
-    const float om = 1.0f - beta_m, ov = 1.0f - beta_v;
     constexpr int kSlices = kTile / (kThreads * 8);
 
     float a_dot = 0.f, a_n2 = 0.f, a_dm = 0.f, a_m2 = 0.f;
@@ -56,8 +60,8 @@ stats_step_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
                 a_n2 = fmaf(x[j], x[j], a_n2);
                 a_dm = fmaf(x[j], mm[j], a_dm);
                 a_m2 = fmaf(mm[j], mm[j], a_m2);
-                mm[j] = fmaf(beta_m, mm[j], om * x[j]);
-                vv[j] = fmaf(beta_v, vv[j], ov * (x[j] * x[j]));
+                mm[j] = ema(mm[j], x[j], om);
+                vv[j] = ema(vv[j], x[j] * x[j], ov);
             }
             st_stream_f4(m + e, make_float4(mm[0], mm[1], mm[2], mm[3]));
             st_stream_f4(m + e + 4, make_float4(mm[4], mm[5], mm[6], mm[7]));
@@ -72,8 +76,8 @@ stats_step_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
                 const float mm = m[e + j], vv = v[e + j];
                 a_dot = fmaf(x, p, a_dot); a_n2 = fmaf(x, x, a_n2);
                 a_dm = fmaf(x, mm, a_dm); a_m2 = fmaf(mm, mm, a_m2);
-                m[e + j] = fmaf(beta_m, mm, om * x);
-                v[e + j] = fmaf(beta_v, vv, ov * (x * x));
+                m[e + j] = ema(mm, x, om);
+                v[e + j] = ema(vv, x * x, ov);
                 gp[e + j] = gb;
             }
         }
@@ -185,8 +189,8 @@ stats_final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __rest
         for (int j = 0; j < 8; ++j) {
             if (j < cnt) {
                 const float mj = mm[j], vj = vv[j];
-                const float m8 = float(encode_signed(double(mj), sm)) * dm;
-                const float v8 = float(encode_unsigned(double(vj), sv)) * dv;
+                const float m8 = float(encode_signed(double(mj), am, sm)) * dm;
+                const float v8 = float(encode_unsigned(double(vj), av, sv)) * dv;
                 const float m16 = round_to_bf16(mj), v16 = round_to_bf16(vj);
                 const float u32 = mj / (sqrtf(vj) + eps_adam);
                 const float u8 = m8 / (sqrtf(v8) + eps_adam);
@@ -379,8 +383,9 @@ __global__ void stats_gather_kernel(const RankSel* __restrict__ sel, const doubl
     } while (0)
 
 int launch_stats_step(const StatBlock* blocks, const Tile* tiles, const void* const* grads, double* partials,
-                      int64_t n_tiles, float beta_m, float beta_v, cudaStream_t s) {
-    stats_step_kernel<<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, grads, partials, beta_m, beta_v);
+                      int64_t n_tiles, float one_minus_beta_m, float one_minus_beta_v, cudaStream_t s) {
+    stats_step_kernel<<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, grads, partials, one_minus_beta_m,
+                                                             one_minus_beta_v);
     BAOC_LAUNCH_CHECK();
     return 0;
 }

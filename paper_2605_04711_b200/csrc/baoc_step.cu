@@ -15,7 +15,8 @@ namespace baoc {
 // otherwise the source is an fp32 array summed as it is.
 // ============================================================================
 template <bool kSquare>
-__device__ __forceinline__ void load8(const void* src, int64_t idx, int valid, bool vec, float (&x)[8]) {
+__device__ __forceinline__ void load8(const void* src, const float* th, float wd, int64_t idx, int valid, bool vec,
+                                      float (&x)[8]) {
     if constexpr (kSquare) {
         const uint16_t* p = static_cast<const uint16_t*>(src) + idx;
         if (vec && valid == 8) {
@@ -23,6 +24,18 @@ __device__ __forceinline__ void load8(const void* src, int64_t idx, int valid, b
         } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j) x[j] = j < valid ? bf16_bits_to_float(p[j]) : 0.f;
+        }
+        if (th) {                                  // coupled decay: the squares are those of g + wd*theta
+            float t[8];
+            if (vec && valid == 8) {
+                const float4 a = ld_stream_f4(th + idx), b = ld_stream_f4(th + idx + 4);
+                t[0] = a.x; t[1] = a.y; t[2] = a.z; t[3] = a.w; t[4] = b.x; t[5] = b.y; t[6] = b.z; t[7] = b.w;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) t[j] = j < valid ? th[idx + j] : 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) x[j] = fmaf(wd, t[j], x[j]);
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) x[j] *= x[j];
@@ -39,8 +52,8 @@ __device__ __forceinline__ void load8(const void* src, int64_t idx, int valid, b
 }
 
 template <bool kSquare>
-__device__ __forceinline__ void rowcol_reduce_piece(const void* src, int rows, int cols, const RedGeom geo,
-                                                    uint32_t chunk, uint32_t strip) {
+__device__ __forceinline__ void rowcol_reduce_piece(const void* src, const float* th, float wd, int rows, int cols,
+                                                    const RedGeom geo, uint32_t chunk, uint32_t strip) {
     __shared__ float sh_row[kRedRows][65];
     __shared__ float sh_col[4][kRedCols];
     const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
@@ -61,7 +74,7 @@ __device__ __forceinline__ void rowcol_reduce_piece(const void* src, int rows, i
             float s = 0.f;
             if (r < rows && valid > 0) {
                 float x[8];
-                load8<kSquare>(src, r * cols + col0, valid, vec, x);
+                load8<kSquare>(src, th, wd, r * cols + col0, valid, vec, x);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) { s += x[j]; colacc[j] += x[j]; }
             }
@@ -96,10 +109,13 @@ __device__ __forceinline__ void rowcol_reduce_piece(const void* src, int rows, i
 // Gradient squares of the factored blocks of the step.
 __global__ void __launch_bounds__(kThreads)
 factored_reduce_kernel(const StepBlock* __restrict__ blocks, const RedTile* __restrict__ rtiles,
-                       const void* const* __restrict__ grads) {
+                       const void* const* __restrict__ grads, const float* const* __restrict__ params,
+                       const __grid_constant__ StepParams SP) {
     const RedTile t = rtiles[blockIdx.x];
     const StepBlock* b = blocks + t.block;
-    rowcol_reduce_piece<true>(grads[t.block], b->rows, b->cols, b->red, t.chunk, t.strip);
+    const CfgStep& P = SP.c[b->cfg];
+    rowcol_reduce_piece<true>(grads[t.block], P.coupled ? params[t.block] : nullptr, P.wd, b->rows, b->cols, b->red,
+                              t.chunk, t.strip);
 }
 
 // Second moments of the matrix blocks of the statistics pass.
@@ -107,7 +123,7 @@ __global__ void __launch_bounds__(kThreads)
 moment_reduce_kernel(const StatBlock* __restrict__ blocks, const RedTile* __restrict__ rtiles) {
     const RedTile t = rtiles[blockIdx.x];
     const StatBlock* b = blocks + t.block;
-    rowcol_reduce_piece<false>(b->v, b->rows, b->cols, b->red, t.chunk, t.strip);
+    rowcol_reduce_piece<false>(b->v, nullptr, 0.f, b->rows, b->cols, b->red, t.chunk, t.strip);
 }
 
 // One CTA per matrix block: add the pieces into rowsum / colsum (double).
@@ -159,37 +175,57 @@ factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __r
 // ============================================================================
 // Fused heterogeneous step.  One CTA per tile; the tile's block selects the
 // update path, so a CTA never diverges on it.  Every thread owns 8
-// consecutive elements per 2048-element slice.
+// consecutive elements per 2048-element slice, and all loads of a tile are
+// issued before the first use.
+//
+// The direction m / (sqrt(v / bc2) + eps) is evaluated as
+// m * rcp(sqrt(v) * rsqrt(bc2) + eps) with the approximate square root and
+// reciprocal (relative error 2^-23 each): the update is lr * direction, a
+// small fraction of the parameter, so the parameter keeps full fp32 accuracy,
+// and the moments themselves never pass through an approximation.
 // ============================================================================
+__device__ __forceinline__ float sqrt_approx(float x) {
+    float r;
+    asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+    float r;
+    asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
 __device__ __forceinline__ void prologue(float& x, float& t, const CfgStep& P) {
     if (P.coupled) x = fmaf(P.wd, t, x);          // coupled decay joins the gradient
     else t = fmaf(P.decay, t, t);                 // decoupled: theta <- theta - lr*wd*theta (decay holds -lr*wd)
 }
 
-__device__ __forceinline__ float adam_dir(float mhat, float v, const CfgStep& P) {
-    return mhat / (sqrtf(v / P.bc2) + P.eps);
+// theta <- theta - step * num / (sqrt(v / bc2) + eps)
+__device__ __forceinline__ float adaptive_apply(float t, float num, float v, float step, const CfgStep& P) {
+    const float denom = fmaf(sqrt_approx(v), P.rsqrt_bc2, P.eps);
+    return fmaf(-step * num, rcp_approx(denom), t);
 }
 
 struct PathA32 {
     static __device__ __forceinline__ void upd(float x, float& t, float& m, float& v, const CfgStep& P) {
         prologue(x, t, P);
-        m = fmaf(P.beta1, m, (1.0f - P.beta1) * x);
-        v = fmaf(P.beta2, v, (1.0f - P.beta2) * (x * x));
-        t = fmaf(-P.lr, adam_dir(m / P.bc1, v, P), t);
+        m = fmaf(P.beta1, m, P.om1 * x);
+        v = fmaf(P.beta2, v, P.om2 * (x * x));
+        t = adaptive_apply(t, m, v, P.step_m, P);
     }
 };
 struct PathR {
     static __device__ __forceinline__ void upd(float x, float& t, float& v, const CfgStep& P) {
         prologue(x, t, P);
-        v = fmaf(P.beta2, v, (1.0f - P.beta2) * (x * x));
-        t = fmaf(-P.lr, adam_dir(x, v, P), t);
+        v = fmaf(P.beta2, v, P.om2 * (x * x));
+        t = adaptive_apply(t, x, v, P.step_g, P);
     }
 };
 struct PathS {
     static __device__ __forceinline__ void upd(float x, float& t, float& m, const CfgStep& P) {
         prologue(x, t, P);
         m = fmaf(P.beta1, m, x);
-        t = fmaf(-P.lr, m, t);
+        t = fmaf(-P.step_g, m, t);
     }
 };
 
@@ -200,6 +236,9 @@ __device__ __forceinline__ void st8(float* p, const float (&x)[8]) {
     st_stream_f4(p, make_float4(x[0], x[1], x[2], x[3]));
     st_stream_f4(p + 4, make_float4(x[4], x[5], x[6], x[7]));
 }
+// 0 * x is 0 for a finite x and NaN otherwise: one FMA per value folds a
+// non-finite test of many values into one accumulator.
+__device__ __forceinline__ float poison(float acc, float x) { return fmaf(x, 0.0f, acc); }
 
 constexpr int kSlices = kTile / (kThreads * 8);
 
@@ -210,7 +249,7 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
     const int64_t numel = b->numel;
     float* __restrict__ m = kM ? static_cast<float*>(b->s0) : nullptr;
     float* __restrict__ v = kV ? static_cast<float*>(kM ? b->s1 : b->s0) : nullptr;
-    unsigned bad = 0;
+    float chk = 0.f;
     uint4 wg[kSlices];
     float4 t0[kSlices], t1[kSlices], m0[kSlices], m1[kSlices], v0[kSlices], v1[kSlices];
     bool full[kSlices];
@@ -238,7 +277,7 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
                 if (kM && kV) PathA32::upd(x[j], t[j], mm[j], vv[j], P);
                 else if (kV) PathR::upd(x[j], t[j], vv[j], P);
                 else PathS::upd(x[j], t[j], mm[j], P);
-                bad |= !isfinite(t[j]);
+                chk = poison(chk, t[j]);
             }
             st8(th + e, t);
             if (kM) st8(m + e, mm);
@@ -253,18 +292,21 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
                 if (kM && kV) PathA32::upd(x, t, mm, vv, P);
                 else if (kV) PathR::upd(x, t, vv, P);
                 else PathS::upd(x, t, mm, P);
-                bad |= !isfinite(t);
+                chk = poison(chk, t);
                 th[e + j] = t;
                 if (kM) m[e + j] = mm;
                 if (kV) v[e + j] = vv;
             }
         }
     }
-    return bad;
+    return chk != 0.f;                               // NaN compares unequal
 }
 
 // Factored second moment: v_ij = r_i c_j / mean(r) from the already updated
-// row and column statistics; no per-element state.
+// row and column statistics; no per-element state.  When the row length is a
+// multiple of 8 a thread's 8 elements lie in one row, so it needs one row
+// statistic and two 128-bit loads of column statistics (which stay in L1/L2:
+// every row of the tile re-reads them).
 __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgStep& P, const uint16_t* __restrict__ g,
                                                   float* __restrict__ th, int64_t base) {
     const int64_t numel = b->numel;
@@ -273,137 +315,250 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
     const float* __restrict__ c = static_cast<const float*>(b->s1);
     const float rm = b->a0[0];
     const float inv_rm = rm > 0.f ? 1.0f / rm : 0.f;
-    unsigned bad = 0;
+    float chk = 0.f;
+    if ((cols & 7) == 0) {
+        const int64_t row0 = base / cols;
+        const uint32_t col0 = uint32_t(base - row0 * cols);
+        uint4 wg[kSlices];
+        float4 t0[kSlices], t1[kSlices], c0[kSlices], c1[kSlices];
+        float ri[kSlices];
+        bool in[kSlices];
 #pragma unroll
+        for (int s = 0; s < kSlices; ++s) {
+            const uint32_t off = uint32_t(s) * (kThreads * 8) + threadIdx.x * 8;
+            const int64_t e = base + off;
+            in[s] = e < numel;                        // numel is a multiple of 8 here
+            if (in[s]) {
+                const uint32_t cc = col0 + off;       // < cols + kTile
+                const uint32_t q = cc / uint32_t(cols);
+                const uint32_t col = cc - q * uint32_t(cols);
+                wg[s] = ld_stream_u4(g + e);
+                t0[s] = ld_stream_f4(th + e); t1[s] = ld_stream_f4(th + e + 4);
+                c0[s] = __ldg(reinterpret_cast<const float4*>(c + col));
+                c1[s] = __ldg(reinterpret_cast<const float4*>(c + col + 4));
+                ri[s] = __ldg(r + row0 + q);
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < kSlices; ++s) {
+            if (!in[s]) continue;
+            const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+            float x[8], t[8], cj[8];
+            unpack8(wg[s], x); f4_to(t0[s], t1[s], t); f4_to(c0[s], c1[s], cj);
+            const float rs = ri[s] * inv_rm;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                prologue(x[j], t[j], P);
+                t[j] = adaptive_apply(t[j], x[j], rs * cj[j], P.step_g, P);
+                chk = poison(chk, t[j]);
+            }
+            st8(th + e, t);
+        }
+        return chk != 0.f;
+    }
+    // any other row length: walk the row/column position element by element
+#pragma unroll 1
     for (int s = 0; s < kSlices; ++s) {
         const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
         if (e >= numel) continue;
         const int cnt = int(min64(8, numel - e));
-        float x[8], t[8];
-        if (cnt == 8) {
-            unpack8(ld_stream_u4(g + e), x);
-            f4_to(ld_stream_f4(th + e), ld_stream_f4(th + e + 4), t);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                x[j] = j < cnt ? bf16_bits_to_float(g[e + j]) : 0.f;
-                t[j] = j < cnt ? th[e + j] : 0.f;
-            }
-        }
         int64_t row = e / cols;
         int col = int(e - row * cols);
-        float ri = __ldg(r + row) * inv_rm;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            if (j < cnt) {
-                float vv = ri * __ldg(c + col);
-                float xx = x[j];
-                prologue(xx, t[j], P);
-                t[j] = fmaf(-P.lr, adam_dir(xx, vv, P), t[j]);
-                bad |= !isfinite(t[j]);
-                if (++col == cols) { col = 0; ++row; if (j + 1 < cnt) ri = __ldg(r + row) * inv_rm; }
-            }
+        float rs = __ldg(r + row) * inv_rm;
+        for (int j = 0; j < cnt; ++j) {
+            float x = bf16_bits_to_float(g[e + j]);
+            float t = th[e + j];
+            prologue(x, t, P);
+            t = adaptive_apply(t, x, rs * __ldg(c + col), P.step_g, P);
+            chk = poison(chk, t);
+            th[e + j] = t;
+            if (++col == cols) { col = 0; ++row; if (j + 1 < cnt) rs = __ldg(r + row) * inv_rm; }
         }
-        if (cnt == 8) st8(th + e, t);
-        else
-            for (int j = 0; j < cnt; ++j) th[e + j] = t[j];
     }
-    return bad;
+    return chk != 0.f;
 }
 
+// ----------------------------------------------------------------------------
 // Adam with block-wise absmax 8-bit states.  A warp owns one 256-element
-// quantisation block per slice.  The moments are rebuilt, updated and
-// re-encoded in double so that the integer codes agree with a double-precision
-// evaluation; the parameter update itself runs in fp32 like the other paths.
+// quantisation block per slice (8 elements per lane).
+//
+// The integer codes and the fp32 absmax must agree with a double-precision
+// evaluation of   m' = beta1 (code a / 127) + (1 - beta1) g,  a' = fl32(max|m'|),
+// code' = rne(127 m' / a')   (and likewise for v with 255 levels).  Doing all of
+// it in double costs about 20 FP64 operations per element and makes the path
+// FP64-bound, so the work is split:
+//   * every element is evaluated in fp32 (the parameter update needs those
+//     values anyway); its error against the exact value is below
+//     E = 2^-21 (a_old + max|m'|) (five roundings of magnitude <= 2^-24 of terms
+//     bounded by a_old and max|m'|, with head room);
+//   * the new absmax is the fp32 rounding of the largest exact |m'|, and only
+//     elements within 2E of the fp32 maximum can hold it, so only those are
+//     recomputed in double;
+//   * a code is rne(q) with q = 127 m' / a'; the fp32 q is within
+//     w = 127 E / a' + 2^-14 of the exact one, so unless it lies within w of a
+//     half-integer the fp32 rounding is already the exact answer; the few
+//     elements that do are recomputed in double (exact ties, which bf16
+//     gradients produce from a zero state, fall in here and are resolved by the
+//     correctly rounded division).
+// ----------------------------------------------------------------------------
+struct Q8Ctx {
+    double b1, b2, wd;
+    float am_old, av_old;
+    int coupled;
+};
+
+__device__ __forceinline__ double exact_grad(uint32_t gbits16, float theta, const Q8Ctx& q) {
+    double gd = widen_bf16_float(__uint_as_float(gbits16 << 16));
+    if (q.coupled) gd += q.wd * double(theta);
+    return gd;
+}
+__device__ __forceinline__ double exact_m(int cm, double gd, const Q8Ctx& q) {
+    return q.b1 * (int_to_double(cm) * (double(q.am_old) / 127.0)) + (1.0 - q.b1) * gd;
+}
+__device__ __forceinline__ double exact_v(int cv, double gd, const Q8Ctx& q) {
+    return q.b2 * (int_to_double(cv) * (double(q.av_old) / 255.0)) + (1.0 - q.b2) * (gd * gd);
+}
+
+__device__ __forceinline__ uint32_t half_of(const uint4& w, int j) {
+    const uint32_t word = j < 2 ? w.x : (j < 4 ? w.y : (j < 6 ? w.z : w.w));
+    return (j & 1) ? (word >> 16) : (word & 0xffffu);
+}
+__device__ __forceinline__ uint32_t byte_of(const uint2& w, int j) { return ((j < 4 ? w.x : w.y) >> (8 * (j & 3))) & 0xffu; }
+
 __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep& P, const uint16_t* __restrict__ g,
                                               float* __restrict__ th, int64_t base) {
+    constexpr float kSlack = 4.76837158203125e-7f;                 // 2^-21
+    constexpr float kMagic = 12582912.0f;                          // 1.5 * 2^23: adding it rounds to an integer, ties to even
     const int64_t numel = b->numel;
     int8_t* __restrict__ qm = static_cast<int8_t*>(b->s0);
     uint8_t* __restrict__ qv = static_cast<uint8_t*>(b->s1);
     float* __restrict__ am = b->a0;
     float* __restrict__ av = b->a1;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const double b1 = P.beta1_d, b2 = P.beta2_d;
-    const double o1 = 1.0 - b1, o2 = 1.0 - b2;
-    unsigned bad = 0;
+    float chk = 0.f;
+
+    uint4 wg[kSlices];
+    float4 t0[kSlices], t1[kSlices];
+    uint2 wm[kSlices], wv[kSlices];
+    float amo[kSlices], avo[kSlices];
+    int cnt[kSlices];
 #pragma unroll
     for (int s = 0; s < kSlices; ++s) {
         const int64_t w0 = base + int64_t(s) * (kThreads * 8) + int64_t(warp) * kQBlock;
-        if (w0 >= numel) continue;                              // whole warp out of range
+        cnt[s] = -1;                                                // whole warp out of range
+        if (w0 >= numel) continue;
         const int64_t e = w0 + lane * 8;
-        const int cnt = int(max64(0, min64(8, numel - e)));
-        const int64_t qb = w0 / kQBlock;
-        float x[8], t[8];
-        uint2 wm, wv;
-        if (cnt == 8) {
-            unpack8(ld_stream_u4(g + e), x);
-            f4_to(ld_stream_f4(th + e), ld_stream_f4(th + e + 4), t);
-            wm = ld_stream_u2(qm + e);
-            wv = ld_stream_u2(qv + e);
-        } else {
-            uint32_t pm[2] = {0u, 0u}, pv[2] = {0u, 0u};
+        cnt[s] = int(max64(0, min64(8, numel - e)));
+        amo[s] = am[w0 / kQBlock]; avo[s] = av[w0 / kQBlock];
+        if (cnt[s] == 8) {
+            wg[s] = ld_stream_u4(g + e);
+            t0[s] = ld_stream_f4(th + e); t1[s] = ld_stream_f4(th + e + 4);
+            wm[s] = ld_stream_u2(qm + e);
+            wv[s] = ld_stream_u2(qv + e);
+        } else {                                                    // ragged end of the block: zero-fill
+            uint32_t pg[4] = {0u, 0u, 0u, 0u}, pm[2] = {0u, 0u}, pv[2] = {0u, 0u};
+            float tt[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const bool in = j < cnt;
-                x[j] = in ? bf16_bits_to_float(g[e + j]) : 0.f;
-                t[j] = in ? th[e + j] : 0.f;
-                const uint32_t cm = in ? uint32_t(uint8_t(qm[e + j])) : 0u;
-                const uint32_t cv = in ? uint32_t(qv[e + j]) : 0u;
-                pm[j >> 2] |= cm << (8 * (j & 3));
-                pv[j >> 2] |= cv << (8 * (j & 3));
+                const bool in = j < cnt[s];
+                tt[j] = in ? th[e + j] : 0.f;
+                pg[j >> 1] |= (in ? uint32_t(g[e + j]) : 0u) << (16 * (j & 1));
+                pm[j >> 2] |= (in ? uint32_t(uint8_t(qm[e + j])) : 0u) << (8 * (j & 3));
+                pv[j >> 2] |= (in ? uint32_t(qv[e + j]) : 0u) << (8 * (j & 3));
             }
-            wm = make_uint2(pm[0], pm[1]);
-            wv = make_uint2(pv[0], pv[1]);
+            wg[s] = make_uint4(pg[0], pg[1], pg[2], pg[3]);
+            t0[s] = make_float4(tt[0], tt[1], tt[2], tt[3]); t1[s] = make_float4(tt[4], tt[5], tt[6], tt[7]);
+            wm[s] = make_uint2(pm[0], pm[1]); wv[s] = make_uint2(pv[0], pv[1]);
         }
-        const float am_old = am[qb], av_old = av[qb];
-        const double sm = double(am_old) / 127.0, sv = double(av_old) / 255.0;
-        const float smf = am_old / 127.0f, svf = av_old / 255.0f;
-        double md[8], vd[8];
-        double mx_m = 0.0, mx_v = 0.0;
+    }
+
+#pragma unroll
+    for (int s = 0; s < kSlices; ++s) {
+        if (cnt[s] < 0) continue;
+        const int64_t w0 = base + int64_t(s) * (kThreads * 8) + int64_t(warp) * kQBlock;
+        const int64_t e = w0 + lane * 8;
+        float x[8], t[8], mf[8], vf[8];
+        unpack8(wg[s], x); f4_to(t0[s], t1[s], t);
+        const float smf = amo[s] / 127.0f, svf = avo[s] / 255.0f;
+        Q8Ctx q;
+        q.b1 = P.beta1_d; q.b2 = P.beta2_d; q.wd = P.wd_d;
+        q.am_old = amo[s]; q.av_old = avo[s]; q.coupled = P.coupled;
+
+        // fp32 pass: effective gradient, decayed parameter, new moments, their maxima
+        float mx = 0.f, vx = 0.f;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const uint32_t wmj = j < 4 ? wm.x : wm.y, wvj = j < 4 ? wv.x : wv.y;
-            const int cm = int(int8_t((wmj >> (8 * (j & 3))) & 0xffu));
-            const int cv = int((wvj >> (8 * (j & 3))) & 0xffu);
-            // double side: the states and their codes
-            double gd = widen_bf16_float(x[j]);
-            if (P.coupled) gd += double(P.wd) * double(t[j]);
-            // fp32 side: the parameter update
-            float mf = int_to_float(cm) * smf, vf = int_to_float(cv) * svf;
-            PathA32::upd(x[j], t[j], mf, vf, P);
-            bad |= !isfinite(t[j]);
-            md[j] = b1 * (int_to_double(cm) * sm) + o1 * gd;
-            vd[j] = b2 * (int_to_double(cv) * sv) + o2 * (gd * gd);
-            mx_m = fmax(mx_m, fabs(md[j]));
-            mx_v = fmax(mx_v, vd[j]);
+            const int cm = int(int8_t(byte_of(wm[s], j))), cv = int(byte_of(wv[s], j));
+            prologue(x[j], t[j], P);
+            mf[j] = fmaf(P.beta1, int_to_float(cm) * smf, P.om1 * x[j]);
+            vf[j] = fmaf(P.beta2, int_to_float(cv) * svf, P.om2 * (x[j] * x[j]));
+            mx = fmaxf(mx, fabsf(mf[j])); vx = fmaxf(vx, vf[j]);
         }
-        // rounding to fp32 is monotone, so the maximum of the rounded values is the rounded maximum
-        const float am_new = warp_max(__double2float_rn(mx_m));
-        const float av_new = warp_max(__double2float_rn(mx_v));
-        const double km = code_scale(am_new, 127.0), kv = code_scale(av_new, 255.0);
+        mx = warp_max(mx); vx = warp_max(vx);
+        const float Em = kSlack * (amo[s] + mx), Ev = kSlack * (avo[s] + vx);
+
+        // exact absmax: only elements within 2E of the fp32 maximum can hold it.
+        // (theta: the coupled gradient needs the parameter before the update; prologue leaves it untouched then.)
+        float am_c = 0.f, av_c = 0.f;
+        const float m_thr = mx - 2.0f * Em, v_thr = vx - 2.0f * Ev;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (fabsf(mf[j]) >= m_thr || vf[j] >= v_thr) {
+                const double gd = exact_grad(half_of(wg[s], j), t[j], q);
+                if (fabsf(mf[j]) >= m_thr)
+                    am_c = fmaxf(am_c, __double2float_rn(fabs(exact_m(int(int8_t(byte_of(wm[s], j))), gd, q))));
+                if (vf[j] >= v_thr) av_c = fmaxf(av_c, __double2float_rn(exact_v(int(byte_of(wv[s], j)), gd, q)));
+            }
+        }
+        const float am_new = warp_max(am_c), av_new = warp_max(av_c);
+
+        // codes: fp32 rounding unless the scaled value is within w of a half-integer
+        const float km = am_new > 0.f ? 127.0f / am_new : 0.f, kv = av_new > 0.f ? 255.0f / av_new : 0.f;
+        const float hm = 0.5f - (Em * km + 6.103515625e-5f), hv = 0.5f - (Ev * kv + 6.103515625e-5f);
         uint32_t om[2] = {0u, 0u}, ov[2] = {0u, 0u};
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            om[j >> 2] |= (uint32_t(encode_signed(md[j], km)) & 0xffu) << (8 * (j & 3));
-            ov[j >> 2] |= uint32_t(encode_unsigned(vd[j], kv)) << (8 * (j & 3));
+            const float qmf = mf[j] * km, qvf = vf[j] * kv;
+            const float rm_ = qmf + kMagic, rv_ = qvf + kMagic;
+            uint32_t code_m = __float_as_uint(rm_) & 0xffu, code_v = __float_as_uint(rv_) & 0xffu;
+            const bool slow_m = !(fabsf(qmf - (rm_ - kMagic)) <= hm), slow_v = !(fabsf(qvf - (rv_ - kMagic)) <= hv);
+            if (slow_m || slow_v) {
+                const double gd = exact_grad(half_of(wg[s], j), t[j], q);
+                if (slow_m)
+                    code_m = uint32_t(encode_signed(exact_m(int(int8_t(byte_of(wm[s], j))), gd, q), am_new,
+                                                    code_scale(am_new, 127.0))) & 0xffu;
+                if (slow_v)
+                    code_v = uint32_t(encode_unsigned(exact_v(int(byte_of(wv[s], j)), gd, q), av_new,
+                                                      code_scale(av_new, 255.0)));
+            }
+            om[j >> 2] |= code_m << (8 * (j & 3));
+            ov[j >> 2] |= code_v << (8 * (j & 3));
         }
-        if (cnt == 8) {
+
+        // parameter update from the un-requantised fp32 moments
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            t[j] = adaptive_apply(t[j], mf[j], vf[j], P.step_m, P);
+            chk = poison(chk, t[j]);
+        }
+
+        if (cnt[s] == 8) {
             st8(th + e, t);
             st_stream_u2(qm + e, make_uint2(om[0], om[1]));
             st_stream_u2(qv + e, make_uint2(ov[0], ov[1]));
         } else {
-            for (int j = 0; j < cnt; ++j) {
+            for (int j = 0; j < cnt[s]; ++j) {
                 th[e + j] = t[j];
                 qm[e + j] = int8_t((om[j >> 2] >> (8 * (j & 3))) & 0xffu);
                 qv[e + j] = uint8_t((ov[j >> 2] >> (8 * (j & 3))) & 0xffu);
             }
         }
-        if (lane == 0) { am[qb] = am_new; av[qb] = av_new; }
+        if (lane == 0) { am[w0 / kQBlock] = am_new; av[w0 / kQBlock] = av_new; }
     }
-    return bad;
+    return chk != 0.f;
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 2)
 fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
                   const void* const* __restrict__ grads, float* const* __restrict__ params,
                   uint32_t* __restrict__ flags, const __grid_constant__ StepParams SP) {
@@ -443,9 +598,9 @@ int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const i
 }
 
 int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const int32_t* ids, const void* const* grads,
-                           int64_t n_red, int n_factored, const StepParams& P, cudaStream_t s) {
+                           const float* const* params, int64_t n_red, int n_factored, const StepParams& P, cudaStream_t s) {
     if (n_red <= 0) return 0;
-    factored_reduce_kernel<<<unsigned(n_red), kThreads, 0, s>>>(blocks, rtiles, grads);
+    factored_reduce_kernel<<<unsigned(n_red), kThreads, 0, s>>>(blocks, rtiles, grads, params, P);
     BAOC_LAUNCH_CHECK();
     factored_combine_kernel<<<n_factored, kThreads, 0, s>>>(blocks, ids, P);
     BAOC_LAUNCH_CHECK();

@@ -45,6 +45,15 @@ def _close(got, ref, rel=1e-4, floor=1e-3):
     return abs(got - ref) <= rel * max(abs(ref), floor)
 
 
+def _stat_close(key, got, ref, n_steps):
+    """1e-4 relative.  The err_* diagnostics are ||x - Q(x)|| / ||x|| of the window moments; the library keeps
+    those moments in fp32 (one rounding per window step, so x is off by at most n_steps * 2^-24 relative) while
+    the oracle keeps them in double, and that perturbation passes straight into the distance: on a block of a
+    few elements it does not average out, so it is allowed on top of the relative tolerance."""
+    extra = n_steps * 2.0 ** -23 if key.startswith("err_") else 0.0
+    return abs(got - ref) <= 1e-4 * max(abs(ref), 1e-3) + extra
+
+
 def _odd_workload(seed=3, window=6):
     shapes = [(1, 1), (7, 1), (255, 1), (256, 1), (257, 1), (4097, 1), (6149, 1), (37, 53), (64, 147), (300, 520),
               (5000, 8), (3, 3), (4096, 1), (130, 64), (8200, 1)]
@@ -71,9 +80,10 @@ def _oracle_window(sess, T, opts=None):
     return states
 
 
-def _check_stats(sess, states, opts=None, skip_small_C=True):
+def _check_stats(sess, states, opts=None):
     o = opts or O.Opts()
     wl = sess.wl
+    n_steps = sess.h.query().stats_steps
     risk, st = sess.risk()
     cfgs = [_ocfg(c) for c in sess.configs]
     worst = {}
@@ -81,7 +91,7 @@ def _check_stats(sess, states, opts=None, skip_small_C=True):
         raw = O.stats_finalize(states[i], sess.block_param_host(i), b.rows, b.cols, o)
         for k in STAT_KEYS:
             got, ref = st[i][k], raw[k]
-            ok = _close(got, ref)
+            ok = _stat_close(k, got, ref, n_steps)
             worst[k] = max(worst.get(k, 0.0), abs(got - ref) / max(abs(ref), 1e-3))
             assert ok, (b.name, k, got, ref)
         assert st[i]["n_cos"] == states[i].n_cos
@@ -125,15 +135,19 @@ def test_stats_invariants_identical_zero_and_flipped_gradients(B, H):
     for _ in range(4):
         sess.sample_stats(0)
     run = sess.h.read_stats()
+    # identical gradients: stability 1, up to the eps of Eq. 5's denominator, which pulls the cosine of a
+    # block with squared norm n2 down to n2 / (n2 + eps)
+    slack = [1e-9 + 1e-12 / max(float(np.sum(sess.block_grad_host(0, i) ** 2)), 1e-300) for i in range(n)]
     for i in range(n):
         want = 0.0 if i == 2 else 1.0
-        assert abs(run[i]["rho_bar"] - want) < 1e-9, (i, run[i]["rho_bar"])   # identical gradients: stability 1
+        assert abs(run[i]["rho_bar"] - want) <= (0.0 if i == 2 else slack[i]), (i, run[i]["rho_bar"])
+        assert run[i]["rho_bar"] <= 1.0
     sess.grads[0].neg_()
     sess.sample_stats(0)
     run = sess.h.read_stats()
     for i in range(n):
         if i != 2:
-            assert abs(run[i]["last_cos"] + 1.0) < 1e-9
+            assert abs(run[i]["last_cos"] + 1.0) <= slack[i] and run[i]["last_cos"] >= -1.0
     # |g_j| constant over a block: isotropic second moment, anisotropy 0
     risk, st = sess.risk()
     wl2 = _odd_workload(seed=6)
@@ -190,7 +204,8 @@ def _rel_max(got, ref):
 def _check_block(sess, i, th_ref, st_ref, code_stats):
     got = sess.block_param_host(i)
     assert np.all(np.isfinite(got))
-    assert _rel_max(got, th_ref) <= 1e-6, (sess.wl.blocks[i].name, st_ref.kind, _rel_max(got, th_ref))
+    if th_ref is not None:
+        assert _rel_max(got, th_ref) <= 1e-6, (sess.wl.blocks[i].name, st_ref.kind, _rel_max(got, th_ref))
     kind = st_ref.kind
     f32 = lambda w: sess.h.view_tensor(i, w, torch.float32).double().cpu().numpy()
     if kind == "A32":
@@ -230,7 +245,45 @@ def test_each_configuration_ten_steps_odd_sizes(B, H, cfg_index):
     assert info.state_bytes == sum(int(mem[i, c]) for i, c in enumerate(assign))
 
 
-def test_coupled_decay_and_other_hyperparameters(B, H):
+def _round_state_to_storage(th, st):
+    """Round what the library stores in fp32 (parameters and the fp32 state tensors) to fp32, in place on the
+    oracle's side.  Codes and absmax already have their storage types."""
+    th = th.astype(np.float32).astype(np.float64)
+    for name in ("m", "v", "r", "c"):
+        a = getattr(st, name)
+        if a is not None:
+            setattr(st, name, a.astype(np.float32).astype(np.float64))
+    return th
+
+
+def _push_state(sess, i, th, st):
+    """Write the oracle's parameters and state of block i into the device buffers."""
+    dev = sess.device
+    sess.param_views[i].copy_(torch.from_numpy(th.astype(np.float32)).to(dev))
+    put = lambda which, dt, a: sess.h.view_tensor(i, which, dt).copy_(torch.from_numpy(np.ascontiguousarray(a)).to(dev))
+    if st.kind == "A32":
+        put(10, torch.float32, st.m.astype(np.float32)); put(11, torch.float32, st.v.astype(np.float32))
+    elif st.kind == "A8":
+        put(10, torch.int8, st.qm); put(11, torch.uint8, st.qv)
+        put(12, torch.float32, st.am); put(13, torch.float32, st.av)
+    elif st.kind == "R":
+        put(10, torch.float32, st.v.astype(np.float32))
+    elif st.kind == "S":
+        put(10, torch.float32, st.m.astype(np.float32))
+    elif st.kind == "F":
+        put(10, torch.float32, st.r.astype(np.float32)); put(11, torch.float32, st.c.astype(np.float32))
+
+
+def test_coupled_decay_and_other_hyperparameters_step_by_step(B, H):
+    """Ten single steps, each from a state both sides share.
+
+    With coupled decay the effective gradient g + wd*theta can cancel, and under the 8-bit configuration a small
+    second moment whose code is 0 makes the direction m/(sqrt(v)+eps) large, so the map from (theta, state) to
+    the next theta is ill-conditioned on some coordinates: the fp32 storage rounding of theta alone (which the
+    oracle, carrying theta in double, does not have) then grows over free-running steps.  The kernel's own
+    arithmetic is what is under test, so before every step the oracle's parameters and fp32 states are rounded
+    to their storage type and written to the device, and both sides take one step from there.  A coordinate may
+    be off by 1e-6 of the block's largest parameter plus 1e-5 of its own update."""
     wl = _odd_workload(seed=21)
     cfgs = [B.make_config(1, 1, 0, 0, 32, lr=3e-3, beta1=0.8, beta2=0.95, eps=1e-6, weight_decay=0.1),
             B.make_config(1, 1, 0, 0, 8, lr=3e-3, beta1=0.8, beta2=0.95, eps=1e-6, weight_decay=0.1),
@@ -239,12 +292,28 @@ def test_coupled_decay_and_other_hyperparameters(B, H):
             B.make_config(0, 1, 0, 0, 32, lr=1e-2, beta1=0.5, weight_decay=0.1)]
     sess = H.Session(wl, configs=cfgs, n_grad_sets=2)
     sess.init_params()
-    assign = [(i % 5) if not ((i % 5) == 3 and b.cols <= 1) else 0 for i, b in enumerate(wl.blocks)]
-    th, sts = _run_steps(sess, assign, 10)
+    n = len(wl.blocks)
+    assign = [(i % 5) if not ((i % 5) == 3 and b.cols <= 1) else 1 for i, b in enumerate(wl.blocks)]
+    assign[9] = 1                                                     # the 300 x 520 matrix takes the 8-bit path too
+    ocfgs = [_ocfg(c) for c in cfgs]
+    sess.configure(assign)
+    th = [sess.block_param_host(i) for i in range(n)]
+    sts = [O.step_init(ocfgs[assign[i]], b.numel, b.rows, b.cols) for i, b in enumerate(wl.blocks)]
     codes = [0, 0]
-    for i in range(len(wl.blocks)):
-        _check_block(sess, i, th[i], sts[i], codes)
-    assert codes[0] <= 1e-4 * max(codes[1], 1)
+    for t in range(1, 11):
+        k = sess.fill_grads(t)
+        for i in range(n):
+            th[i] = _round_state_to_storage(th[i], sts[i])
+            _push_state(sess, i, th[i], sts[i])
+        before = [x.copy() for x in th]
+        sess.step(k, t)
+        for i, b in enumerate(wl.blocks):
+            th[i] = O.step(th[i], sess.block_grad_host(k, i), sts[i], ocfgs[assign[i]], b.rows, b.cols)
+            got = sess.block_param_host(i)
+            tol = 1e-6 * np.max(np.abs(th[i])) + 1e-5 * np.abs(th[i] - before[i])
+            assert np.all(np.abs(got - th[i]) <= tol), (t, b.name, sts[i].kind, float(np.max(np.abs(got - th[i]) / tol)))
+            _check_block(sess, i, None, sts[i], codes)
+    assert codes[1] > 0 and codes[0] <= 1e-4 * codes[1], codes
 
 
 def test_nonfinite_gradient_is_flagged_not_fatal(B, H):
