@@ -27,6 +27,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+CONFIG_NAMES = ["adamw32", "adamw8", "rms", "factored", "sgdm"]
 METRIC = "hot-path throughput: statistics pass + mixed-config optimizer step"
 UNIT = "params/s"
 
@@ -208,6 +209,10 @@ def run_ours(args):
     t0 = time.perf_counter()
     assign, objective, rc = sess.allocate(risk)
     alloc_ms = (time.perf_counter() - t0) * 1e3
+    if args.assign != "auto":
+        # one configuration for every block (vectors cannot be factored: they take the momentum-free one)
+        c = CONFIG_NAMES.index(args.assign)
+        assign = np.asarray([c if not (c == 3 and b.cols <= 1) else 2 for b in wl.blocks], np.int32)
     sess.configure(assign)
     info = sess.h.query()
     stats_bytes, step_bytes = info.stats_bytes_per_call, info.step_bytes_per_call
@@ -289,7 +294,7 @@ def run_ours(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "params": wl.numel, "blocks": len(wl.blocks), "grad_dtype": "bf16",
-                   "param_dtype": "f32", "candidate_configs": ["adamw32", "adamw8", "rms", "factored", "sgdm"],
+                   "param_dtype": "f32", "candidate_configs": CONFIG_NAMES, "assignment": args.assign,
                    "assignment_blocks_per_config": counts, "assignment_params_per_config": params_by_cfg,
                    "mem_budget_frac_of_fp32_adam": wl.mem_budget_frac, "state_bytes": int(info.state_bytes),
                    "window_steps_before_timing": args.window, "l2": "inputs (>10 GB per step) far exceed the 126 MB L2",
@@ -326,6 +331,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama_1b")
+    ap.add_argument("--assign", default="auto", choices=["auto"] + CONFIG_NAMES,
+                    help="auto: the library's own budgeted allocation; else every block under that one configuration")
     ap.add_argument("--window", type=int, default=4, help="statistics steps before the finalize that feeds the allocation")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample-params", type=int, default=40_000_000)

@@ -296,6 +296,7 @@ int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t byt
             b.a0 = static_cast<float*>(fix(b.a0));
             b.red.rowpart = reinterpret_cast<double*>(st + L.redpart + reinterpret_cast<size_t>(b.red.rowpart));
             b.red.colpart = reinterpret_cast<double*>(st + L.redpart + reinterpret_cast<size_t>(b.red.colpart));
+            b.mean_part = reinterpret_cast<double*>(st + L.redpart + reinterpret_cast<size_t>(b.mean_part));
             ids.push_back(i);
         }
     }

@@ -151,6 +151,8 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
                 redpart += 8 * size_t(s.red.strips) * b.rows;
                 s.red.colpart = reinterpret_cast<double*>(redpart);
                 redpart += 8 * size_t(s.red.chunks) * b.cols;
+                s.mean_part = reinterpret_cast<double*>(redpart);
+                redpart += 8 * size_t(kCombineSlabs + 1);
                 break;
             }
             default: break;
@@ -163,7 +165,7 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
     for (int p : order)
         for (int i = 0; i < n; ++i)
             if (sb[i].path == p) {
-                const int64_t nt = ceil_div(sb[i].numel, kTile);
+                const int64_t nt = ceil_div(sb[i].numel, step_tile_elems(p));
                 for (int64_t k = 0; k < nt; ++k) tl.push_back(Tile{uint32_t(i), uint32_t(k)});
             }
     size_t cur = 0;

@@ -26,6 +26,8 @@ constexpr int kRanks = 4;             // order statistics per block for the two 
 constexpr int kFinOut = 32;           // doubles per block copied to the host at the end of the window
 constexpr int kRedRows = 64;          // rows per CTA of the row/column reduction kernel
 constexpr int kRedCols = 512;         // columns per CTA of the row/column reduction kernel
+constexpr int kTileF = 8192;          // elements per tile of the factored path (10 bytes per element: more elements keep as many bytes in flight)
+constexpr int kCombineSlabs = 32;     // CTAs per factored block of the row/column combine
 
 // Update paths of the fused step.
 enum Path : int32_t { kPathA32 = 0, kPathA8 = 1, kPathR = 2, kPathF = 3, kPathS = 4, kPathNone = -1 };
@@ -37,6 +39,9 @@ inline Path path_of(const baoc_config_t& c) {
     if (!c.adaptive && c.momentum && !c.factored && c.bits == 32) return kPathS;
     return kPathNone;
 }
+
+// Elements per tile of the fused step, by update path.
+inline int64_t step_tile_elems(int path) { return path == kPathF ? kTileF : kTile; }
 
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
@@ -78,6 +83,7 @@ struct StepBlock {
     void* s1;            // A32: v   A8: codes of v          F: c (cols)
     float* a0;           // A8: absmax of m per quantisation block;  F: [0] = mean of r
     float* a1;           // A8: absmax of v per quantisation block
+    double* mean_part;   // F: kCombineSlabs partial sums of the new r, then one ticket counter (uint32)
     int64_t numel;
     int32_t rows, cols;
     int32_t cfg;

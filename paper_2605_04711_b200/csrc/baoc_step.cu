@@ -143,19 +143,23 @@ moment_reduce_combine_kernel(const StatBlock* __restrict__ blocks, const int32_t
     }
 }
 
-// One CTA per factored block: r_i <- beta2 r_i + (1-beta2) mean_j g_ij^2,
-// c_j likewise over rows, then the mean of the new r.
+// kCombineSlabs CTAs per factored block, each owning a slab of the rows and of
+// the columns: r_i <- beta2 r_i + (1-beta2) mean_j g_ij^2, c_j likewise over rows.
+// Every CTA leaves the sum of its new r_i; the CTA that takes the last ticket of
+// the block adds the slab sums in index order and stores the mean of r (no CTA
+// waits for another).
 __global__ void __launch_bounds__(kThreads)
 factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __restrict__ ids,
                         const __grid_constant__ StepParams P) {
     __shared__ double total[1];
     const StepBlock* b = blocks + ids[blockIdx.x];
-    const int rows = b->rows, cols = b->cols;
+    const int rows = b->rows, cols = b->cols, slab = blockIdx.y;
     const double beta2 = P.c[b->cfg].beta2_d;
     float* __restrict__ r = static_cast<float*>(b->s0);
     float* __restrict__ c = static_cast<float*>(b->s1);
+    const int rpc = (rows + kCombineSlabs - 1) / kCombineSlabs, cpc = (cols + kCombineSlabs - 1) / kCombineSlabs;
     double local[1] = {0.0};
-    for (int i = threadIdx.x; i < rows; i += kThreads) {
+    for (int i = slab * rpc + threadIdx.x; i < min(rows, (slab + 1) * rpc); i += kThreads) {
         double s = 0.0;
         for (int st = 0; st < b->red.strips; ++st) s += b->red.rowpart[size_t(st) * rows + i];
         const float rn = float(beta2 * double(r[i]) + (1.0 - beta2) * (s / double(cols)));
@@ -163,13 +167,25 @@ factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __r
         local[0] += double(rn);
     }
     cta_reduce_store<1>(local, total);
-    for (int j = threadIdx.x; j < cols; j += kThreads) {
+    for (int j = slab * cpc + threadIdx.x; j < min(cols, (slab + 1) * cpc); j += kThreads) {
         double s = 0.0;
+#pragma unroll 4
         for (int ch = 0; ch < b->red.chunks; ++ch) s += b->red.colpart[size_t(ch) * cols + j];
         c[j] = float(beta2 * double(c[j]) + (1.0 - beta2) * (s / double(rows)));
     }
-    __syncthreads();
-    if (threadIdx.x == 0) b->a0[0] = float(total[0] / double(rows));
+    if (threadIdx.x == 0) {
+        volatile double* part = b->mean_part;
+        unsigned int* ticket = reinterpret_cast<unsigned int*>(b->mean_part + kCombineSlabs);
+        part[slab] = total[0];
+        __threadfence();
+        if (atomicAdd(ticket, 1u) == unsigned(kCombineSlabs - 1)) {
+            __threadfence();
+            double s = 0.0;
+            for (int k = 0; k < kCombineSlabs; ++k) s += part[k];
+            b->a0[0] = float(s / double(rows));
+            *ticket = 0u;                            // ready for the next step
+        }
+    }
 }
 
 // ============================================================================
@@ -241,6 +257,7 @@ __device__ __forceinline__ void st8(float* p, const float (&x)[8]) {
 __device__ __forceinline__ float poison(float acc, float x) { return fmaf(x, 0.0f, acc); }
 
 constexpr int kSlices = kTile / (kThreads * 8);
+constexpr int kSlicesF = kTileF / (kThreads * 8);
 
 // fp32 Adam / RMS / SGD-momentum: kM = has first moment, kV = has second moment.
 template <bool kM, bool kV>
@@ -319,17 +336,17 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
     if ((cols & 7) == 0) {
         const int64_t row0 = base / cols;
         const uint32_t col0 = uint32_t(base - row0 * cols);
-        uint4 wg[kSlices];
-        float4 t0[kSlices], t1[kSlices], c0[kSlices], c1[kSlices];
-        float ri[kSlices];
-        bool in[kSlices];
+        uint4 wg[kSlicesF];
+        float4 t0[kSlicesF], t1[kSlicesF], c0[kSlicesF], c1[kSlicesF];
+        float ri[kSlicesF];
+        bool in[kSlicesF];
 #pragma unroll
-        for (int s = 0; s < kSlices; ++s) {
+        for (int s = 0; s < kSlicesF; ++s) {
             const uint32_t off = uint32_t(s) * (kThreads * 8) + threadIdx.x * 8;
             const int64_t e = base + off;
             in[s] = e < numel;                        // numel is a multiple of 8 here
             if (in[s]) {
-                const uint32_t cc = col0 + off;       // < cols + kTile
+                const uint32_t cc = col0 + off;       // < cols + kTileF
                 const uint32_t q = cc / uint32_t(cols);
                 const uint32_t col = cc - q * uint32_t(cols);
                 wg[s] = ld_stream_u4(g + e);
@@ -340,7 +357,7 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
             }
         }
 #pragma unroll
-        for (int s = 0; s < kSlices; ++s) {
+        for (int s = 0; s < kSlicesF; ++s) {
             if (!in[s]) continue;
             const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
             float x[8], t[8], cj[8];
@@ -358,7 +375,7 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
     }
     // any other row length: walk the row/column position element by element
 #pragma unroll 1
-    for (int s = 0; s < kSlices; ++s) {
+    for (int s = 0; s < kSlicesF; ++s) {
         const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
         if (e >= numel) continue;
         const int cnt = int(min64(8, numel - e));
@@ -413,10 +430,16 @@ __device__ __forceinline__ double exact_grad(uint32_t gbits16, float theta, cons
     return gd;
 }
 __device__ __forceinline__ double exact_m(int cm, double gd, const Q8Ctx& q) {
-    return q.b1 * (int_to_double(cm) * (double(q.am_old) / 127.0)) + (1.0 - q.b1) * gd;
+    return q.b1 * (int_to_double(cm) * double(q.am_old) * (1.0 / 127.0)) + (1.0 - q.b1) * gd;
 }
 __device__ __forceinline__ double exact_v(int cv, double gd, const Q8Ctx& q) {
-    return q.b2 * (int_to_double(cv) * (double(q.av_old) / 255.0)) + (1.0 - q.b2) * (gd * gd);
+    return q.b2 * (int_to_double(cv) * double(q.av_old) * (1.0 / 255.0)) + (1.0 - q.b2) * (gd * gd);
+}
+
+// clamp(rne(L * x / a)) by the correctly rounded division (a > 0 whenever this is reached with x != 0).
+__device__ __forceinline__ int encode_exact(double x, float absmax, double levels, int lo) {
+    if (!(absmax > 0.0f)) return 0;
+    return max(lo, min(int(levels), round_to_int((levels * x) / double(absmax))));
 }
 
 __device__ __forceinline__ uint32_t half_of(const uint4& w, int j) {
@@ -424,6 +447,14 @@ __device__ __forceinline__ uint32_t half_of(const uint4& w, int j) {
     return (j & 1) ? (word >> 16) : (word & 0xffffu);
 }
 __device__ __forceinline__ uint32_t byte_of(const uint2& w, int j) { return ((j < 4 ? w.x : w.y) >> (8 * (j & 3))) & 0xffu; }
+// Lowest bytes of four words, packed in order.
+__device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    return __byte_perm(__byte_perm(a, b, 0x0040u), __byte_perm(c, d, 0x0040u), 0x5410u);
+}
+// Warp maximum of non-negative floats (their bit patterns order like unsigned integers): one reduction instruction.
+__device__ __forceinline__ float warp_max_nonneg(float x) {
+    return __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(x)));
+}
 
 __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep& P, const uint16_t* __restrict__ g,
                                               float* __restrict__ th, int64_t base) {
@@ -456,19 +487,15 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
             wm[s] = ld_stream_u2(qm + e);
             wv[s] = ld_stream_u2(qv + e);
         } else {                                                    // ragged end of the block: zero-fill
-            uint32_t pg[4] = {0u, 0u, 0u, 0u}, pm[2] = {0u, 0u}, pv[2] = {0u, 0u};
-            float tt[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const bool in = j < cnt[s];
-                tt[j] = in ? th[e + j] : 0.f;
-                pg[j >> 1] |= (in ? uint32_t(g[e + j]) : 0u) << (16 * (j & 1));
-                pm[j >> 2] |= (in ? uint32_t(uint8_t(qm[e + j])) : 0u) << (8 * (j & 3));
-                pv[j >> 2] |= (in ? uint32_t(qv[e + j]) : 0u) << (8 * (j & 3));
-            }
-            wg[s] = make_uint4(pg[0], pg[1], pg[2], pg[3]);
-            t0[s] = make_float4(tt[0], tt[1], tt[2], tt[3]); t1[s] = make_float4(tt[4], tt[5], tt[6], tt[7]);
-            wm[s] = make_uint2(pm[0], pm[1]); wv[s] = make_uint2(pv[0], pv[1]);
+            const int n = cnt[s];
+            auto gg = [&](int j) { return j < n ? uint32_t(g[e + j]) : 0u; };
+            auto tt = [&](int j) { return j < n ? th[e + j] : 0.f; };
+            auto mm = [&](int j) { return j < n ? uint32_t(uint8_t(qm[e + j])) : 0u; };
+            auto vv = [&](int j) { return j < n ? uint32_t(qv[e + j]) : 0u; };
+            wg[s] = make_uint4(gg(0) | gg(1) << 16, gg(2) | gg(3) << 16, gg(4) | gg(5) << 16, gg(6) | gg(7) << 16);
+            t0[s] = make_float4(tt(0), tt(1), tt(2), tt(3)); t1[s] = make_float4(tt(4), tt(5), tt(6), tt(7));
+            wm[s] = make_uint2(mm(0) | mm(1) << 8 | mm(2) << 16 | mm(3) << 24, mm(4) | mm(5) << 8 | mm(6) << 16 | mm(7) << 24);
+            wv[s] = make_uint2(vv(0) | vv(1) << 8 | vv(2) << 16 | vv(3) << 24, vv(4) | vv(5) << 8 | vv(6) << 16 | vv(7) << 24);
         }
     }
 
@@ -479,22 +506,28 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         const int64_t e = w0 + lane * 8;
         float x[8], t[8], mf[8], vf[8];
         unpack8(wg[s], x); f4_to(t0[s], t1[s], t);
-        const float smf = amo[s] / 127.0f, svf = avo[s] / 255.0f;
         Q8Ctx q;
         q.b1 = P.beta1_d; q.b2 = P.beta2_d; q.wd = P.wd_d;
         q.am_old = amo[s]; q.av_old = avo[s]; q.coupled = P.coupled;
 
-        // fp32 pass: effective gradient, decayed parameter, new moments, their maxima
+        // fp32 pass: effective gradient, decayed parameter, new moments, their maxima.
+        // A code byte b is turned into the float 2^23 + b by placing it in the low
+        // mantissa byte of 0x4B000000 (signed codes are first offset by 128).
+        const float b1s = P.beta1 * (amo[s] / 127.0f), b2s = P.beta2 * (avo[s] / 255.0f);
+        const float vbias = -8388608.0f * b2s;                      // exact: a power-of-two multiple
+        const uint32_t ms[2] = {wm[s].x ^ 0x80808080u, wm[s].y ^ 0x80808080u};
+        const uint32_t vs[2] = {wv[s].x, wv[s].y};
         float mx = 0.f, vx = 0.f;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const int cm = int(int8_t(byte_of(wm[s], j))), cv = int(byte_of(wv[s], j));
+            const float fm = __uint_as_float(__byte_perm(ms[j >> 2], 0x4B000000u, 0x7440u | (j & 3))) - 8388736.0f;
+            const float fv = __uint_as_float(__byte_perm(vs[j >> 2], 0x4B000000u, 0x7440u | (j & 3)));
             prologue(x[j], t[j], P);
-            mf[j] = fmaf(P.beta1, int_to_float(cm) * smf, P.om1 * x[j]);
-            vf[j] = fmaf(P.beta2, int_to_float(cv) * svf, P.om2 * (x[j] * x[j]));
+            mf[j] = fmaf(fm, b1s, P.om1 * x[j]);
+            vf[j] = fmaf(P.om2 * x[j], x[j], fmaf(fv, b2s, vbias));
             mx = fmaxf(mx, fabsf(mf[j])); vx = fmaxf(vx, vf[j]);
         }
-        mx = warp_max(mx); vx = warp_max(vx);
+        mx = warp_max_nonneg(mx); vx = warp_max_nonneg(vx);
         const float Em = kSlack * (amo[s] + mx), Ev = kSlack * (avo[s] + vx);
 
         // exact absmax: only elements within 2E of the fp32 maximum can hold it.
@@ -503,37 +536,34 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         const float m_thr = mx - 2.0f * Em, v_thr = vx - 2.0f * Ev;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            if (fabsf(mf[j]) >= m_thr || vf[j] >= v_thr) {
+            const bool cand_m = fabsf(mf[j]) >= m_thr, cand_v = vf[j] >= v_thr;
+            if (cand_m || cand_v) {
                 const double gd = exact_grad(half_of(wg[s], j), t[j], q);
-                if (fabsf(mf[j]) >= m_thr)
-                    am_c = fmaxf(am_c, __double2float_rn(fabs(exact_m(int(int8_t(byte_of(wm[s], j))), gd, q))));
-                if (vf[j] >= v_thr) av_c = fmaxf(av_c, __double2float_rn(exact_v(int(byte_of(wv[s], j)), gd, q)));
+                if (cand_m) am_c = fmaxf(am_c, __double2float_rn(fabs(exact_m(int(int8_t(byte_of(wm[s], j))), gd, q))));
+                if (cand_v) av_c = fmaxf(av_c, __double2float_rn(exact_v(int(byte_of(wv[s], j)), gd, q)));
             }
         }
-        const float am_new = warp_max(am_c), av_new = warp_max(av_c);
+        const float am_new = warp_max_nonneg(am_c), av_new = warp_max_nonneg(av_c);
 
-        // codes: fp32 rounding unless the scaled value is within w of a half-integer
+        // codes: rne(q) = low byte of the float q + 1.5*2^23, taken from the fp32
+        // value unless it is within w of a half-integer
         const float km = am_new > 0.f ? 127.0f / am_new : 0.f, kv = av_new > 0.f ? 255.0f / av_new : 0.f;
         const float hm = 0.5f - (Em * km + 6.103515625e-5f), hv = 0.5f - (Ev * kv + 6.103515625e-5f);
-        uint32_t om[2] = {0u, 0u}, ov[2] = {0u, 0u};
+        uint32_t cmw[8], cvw[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const float qmf = mf[j] * km, qvf = vf[j] * kv;
-            const float rm_ = qmf + kMagic, rv_ = qvf + kMagic;
-            uint32_t code_m = __float_as_uint(rm_) & 0xffu, code_v = __float_as_uint(rv_) & 0xffu;
-            const bool slow_m = !(fabsf(qmf - (rm_ - kMagic)) <= hm), slow_v = !(fabsf(qvf - (rv_ - kMagic)) <= hv);
+            const float rm_ = fmaf(mf[j], km, kMagic), rv_ = fmaf(vf[j], kv, kMagic);
+            const float dm = fmaf(mf[j], km, kMagic - rm_), dv = fmaf(vf[j], kv, kMagic - rv_);
+            cmw[j] = __float_as_uint(rm_); cvw[j] = __float_as_uint(rv_);
+            const bool slow_m = !(fabsf(dm) <= hm), slow_v = !(fabsf(dv) <= hv);
             if (slow_m || slow_v) {
                 const double gd = exact_grad(half_of(wg[s], j), t[j], q);
-                if (slow_m)
-                    code_m = uint32_t(encode_signed(exact_m(int(int8_t(byte_of(wm[s], j))), gd, q), am_new,
-                                                    code_scale(am_new, 127.0))) & 0xffu;
-                if (slow_v)
-                    code_v = uint32_t(encode_unsigned(exact_v(int(byte_of(wv[s], j)), gd, q), av_new,
-                                                      code_scale(av_new, 255.0)));
+                if (slow_m) cmw[j] = uint32_t(encode_exact(exact_m(int(int8_t(byte_of(wm[s], j))), gd, q), am_new, 127.0, -127));
+                if (slow_v) cvw[j] = uint32_t(encode_exact(exact_v(int(byte_of(wv[s], j)), gd, q), av_new, 255.0, 0));
             }
-            om[j >> 2] |= code_m << (8 * (j & 3));
-            ov[j >> 2] |= code_v << (8 * (j & 3));
         }
+        const uint2 om = make_uint2(pack_low_bytes(cmw[0], cmw[1], cmw[2], cmw[3]), pack_low_bytes(cmw[4], cmw[5], cmw[6], cmw[7]));
+        const uint2 ov = make_uint2(pack_low_bytes(cvw[0], cvw[1], cvw[2], cvw[3]), pack_low_bytes(cvw[4], cvw[5], cvw[6], cvw[7]));
 
         // parameter update from the un-requantised fp32 moments
 #pragma unroll
@@ -544,13 +574,16 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
 
         if (cnt[s] == 8) {
             st8(th + e, t);
-            st_stream_u2(qm + e, make_uint2(om[0], om[1]));
-            st_stream_u2(qv + e, make_uint2(ov[0], ov[1]));
+            st_stream_u2(qm + e, om);
+            st_stream_u2(qv + e, ov);
         } else {
-            for (int j = 0; j < cnt[s]; ++j) {
-                th[e + j] = t[j];
-                qm[e + j] = int8_t((om[j >> 2] >> (8 * (j & 3))) & 0xffu);
-                qv[e + j] = uint8_t((ov[j >> 2] >> (8 * (j & 3))) & 0xffu);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {                          // static indices keep t[] in registers
+                if (j < cnt[s]) {
+                    th[e + j] = t[j];
+                    qm[e + j] = int8_t(((j < 4 ? om.x : om.y) >> (8 * (j & 3))) & 0xffu);
+                    qv[e + j] = uint8_t(((j < 4 ? ov.x : ov.y) >> (8 * (j & 3))) & 0xffu);
+                }
             }
         }
         if (lane == 0) { am[w0 / kQBlock] = am_new; av[w0 / kQBlock] = av_new; }
@@ -567,7 +600,7 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
     const CfgStep& P = SP.c[b->cfg];
     const uint16_t* g = static_cast<const uint16_t*>(grads[t.block]);
     float* th = params[t.block];
-    const int64_t base = int64_t(t.piece) * kTile;
+    const int64_t base = int64_t(t.piece) * (b->path == kPathF ? kTileF : kTile);
     unsigned bad = 0;
     switch (b->path) {
         case kPathA32: bad = tile_dense<true, true>(b, P, g, th, base); break;
@@ -602,7 +635,7 @@ int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const
     if (n_red <= 0) return 0;
     factored_reduce_kernel<<<unsigned(n_red), kThreads, 0, s>>>(blocks, rtiles, grads, params, P);
     BAOC_LAUNCH_CHECK();
-    factored_combine_kernel<<<n_factored, kThreads, 0, s>>>(blocks, ids, P);
+    factored_combine_kernel<<<dim3(unsigned(n_factored), kCombineSlabs), kThreads, 0, s>>>(blocks, ids, P);
     BAOC_LAUNCH_CHECK();
     return 0;
 }
