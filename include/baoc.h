@@ -239,6 +239,52 @@ int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* co
  * one byte per block.  Waits. */
 int baoc_nonfinite(baoc_t* h, uint8_t* flags, int32_t* count, baoc_stream_t stream);
 
+/* ---- allocation-free variant ------------------------------------------------ */
+
+/* Largest block baoc_sample_stats_noalloc accepts (64 Mi elements).  The
+ * library image carries 5 doubles of scratch per 4096 elements of this
+ * maximum: 640 KB of device memory on every GPU that loads the library, held
+ * until the process exits. */
+#define BAOC_NOALLOC_MAX_NUMEL 67108864
+
+/* The paper has no counterpart of this entry point; it exists for callers that
+ * cannot allocate device memory when they need a block's statistics: code
+ * running inside an allocator hook or an out-of-memory callback, a trainer
+ * whose caching allocator owns every free byte and must not fall through to
+ * cudaMalloc (which synchronises the device and may fail), or a host runtime
+ * with no allocator to lend a workspace from.  It needs no handle and no
+ * workspace: the per-tile partial sums live in a fixed array inside the
+ * library, and the function calls no cudaMalloc, cudaFree or other allocating
+ * routine.
+ *
+ * One gradient observation of ONE block, with the arithmetic of
+ * baoc_sample_stats (Eq. 3 and the cosine of Eq. 5):
+ *   m <- beta_m m + (1-beta_m) g,  v <- beta_v v + (1-beta_v) g*g,
+ *   out4[0] = cos(g, gprev)   with cos(a,b) = <a,b> / (||a|| ||b|| + eps), 0 if not finite,
+ *   out4[1] = ||g||^2,  out4[2] = cos(g, m before the update),  out4[3] = ||m before the update||^2,
+ *   gprev <- g.
+ * grad_bf16 (in), gprev_bf16 (in/out): device, bf16[numel]; m, v (in/out):
+ * device, fp32[numel]; all four 16-byte aligned and owned by the caller, who
+ * zero-fills gprev, m and v before the first observation (the first cosine is
+ * then 0).  out4: device, 4 doubles, written by the second of the two kernels
+ * this call queues on the stream; the call does not wait.
+ *
+ * Errors: BAOC_E_INVALID (null pointer, numel < 1, coefficient outside [0,1)),
+ * BAOC_E_ALIGN, BAOC_E_WORKSPACE when numel > BAOC_NOALLOC_MAX_NUMEL (use the
+ * handle-based path for larger blocks), BAOC_E_CUDA.  baoc_noalloc_last_error()
+ * returns the message of the calling thread's last failure.
+ *
+ * The first call on each device looks up the device address of the built-in
+ * scratch (cudaGetSymbolAddress, with that device current) and keeps it; make
+ * that first call before any stream capture begins.  Every call on a device
+ * shares the one scratch array, which keeps the previous call's contents:
+ * nothing in it needs clearing, because each call overwrites every slot it
+ * later reads, but two calls that overlap on the GPU (different streams, or
+ * different host threads) race on it, so serialise them on one stream. */
+int baoc_sample_stats_noalloc(const void* grad_bf16, void* gprev_bf16, float* m, float* v, int64_t numel,
+                              double beta_m, double beta_v, double eps, double* out4, baoc_stream_t stream);
+const char* baoc_noalloc_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

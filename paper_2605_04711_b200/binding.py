@@ -73,7 +73,8 @@ class Info(C.Structure):
 EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error", "baoc_query",
            "baoc_stats_workspace_bytes", "baoc_bind_stats_workspace", "baoc_sample_stats", "baoc_read_stats",
            "baoc_risk", "baoc_risk_from_raw", "baoc_cost_model", "baoc_allocate", "baoc_state_bytes",
-           "baoc_configure", "baoc_step", "baoc_step_from_host", "baoc_view", "baoc_nonfinite"]
+           "baoc_configure", "baoc_step", "baoc_step_from_host", "baoc_view", "baoc_nonfinite",
+           "baoc_sample_stats_noalloc", "baoc_noalloc_last_error"]
 
 _vp = C.c_void_p
 _lib.baoc_default_opts.argtypes = [C.POINTER(Opts)]
@@ -98,6 +99,23 @@ _lib.baoc_step.argtypes = [_vp, _vp, _vp, C.c_int64, _vp]
 _lib.baoc_step_from_host.argtypes = [_vp, _vp, _vp, _vp, C.c_int, C.c_int64, _vp]
 _lib.baoc_view.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(_vp), C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
 _lib.baoc_nonfinite.argtypes = [_vp, _vp, C.POINTER(C.c_int32), _vp]
+_lib.baoc_sample_stats_noalloc.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_double, C.c_double, C.c_double, _vp, _vp]
+_lib.baoc_noalloc_last_error.argtypes = []
+_lib.baoc_noalloc_last_error.restype = C.c_char_p
+NOALLOC_MAX_NUMEL = 67108864
+
+
+def sample_stats_noalloc(grad: torch.Tensor, gprev: torch.Tensor, m: torch.Tensor, v: torch.Tensor, out4: torch.Tensor,
+                         beta_m: float = 0.9, beta_v: float = 0.999, eps: float = 1e-12, numel: Optional[int] = None):
+    """``baoc_sample_stats_noalloc``: one gradient observation of one block with no handle, no workspace and no
+    allocation (for callers that cannot allocate device memory; see the header).  grad / gprev: bf16 device
+    tensors, m / v: fp32 device tensors, out4: float64 device tensor of 4 elements.  Queues two kernels on the
+    current stream and returns; calls that overlap on one GPU race on the library's built-in scratch."""
+    n = grad.numel() if numel is None else int(numel)
+    rc = _lib.baoc_sample_stats_noalloc(grad.data_ptr(), gprev.data_ptr(), m.data_ptr(), v.data_ptr(), n,
+                                        float(beta_m), float(beta_v), float(eps), out4.data_ptr(), _stream())
+    if rc < 0:
+        raise BaocError(rc, _lib.baoc_noalloc_last_error().decode())
 
 
 def default_opts() -> Opts:
