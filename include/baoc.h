@@ -239,6 +239,15 @@ int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* co
  * one byte per block.  Waits. */
 int baoc_nonfinite(baoc_t* h, uint8_t* flags, int32_t* count, baoc_stream_t stream);
 
+/* Per-kernel timing of baoc_step, for benchmarks.  With profiling on, every
+ * baoc_step records CUDA events on its stream around the factored row/column
+ * kernels and around the fused update kernel (events are created on the first
+ * enable; no device memory is involved).  baoc_profile_last waits for the last
+ * step and writes ms[0] = row/column kernels (0 when no block is factored),
+ * ms[1] = fused update kernel.  BAOC_E_STATE if profiling is off or no step ran. */
+int baoc_profile(baoc_t* h, int enable);
+int baoc_profile_last(baoc_t* h, float* ms2);
+
 /* ---- allocation-free variant ------------------------------------------------ */
 
 /* Largest block baoc_sample_stats_noalloc accepts (64 Mi elements).  The

@@ -74,7 +74,7 @@ EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error"
            "baoc_stats_workspace_bytes", "baoc_bind_stats_workspace", "baoc_sample_stats", "baoc_read_stats",
            "baoc_risk", "baoc_risk_from_raw", "baoc_cost_model", "baoc_allocate", "baoc_state_bytes",
            "baoc_configure", "baoc_step", "baoc_step_from_host", "baoc_view", "baoc_nonfinite",
-           "baoc_sample_stats_noalloc", "baoc_noalloc_last_error"]
+           "baoc_sample_stats_noalloc", "baoc_noalloc_last_error", "baoc_profile", "baoc_profile_last"]
 
 _vp = C.c_void_p
 _lib.baoc_default_opts.argtypes = [C.POINTER(Opts)]
@@ -99,6 +99,8 @@ _lib.baoc_step.argtypes = [_vp, _vp, _vp, C.c_int64, _vp]
 _lib.baoc_step_from_host.argtypes = [_vp, _vp, _vp, _vp, C.c_int, C.c_int64, _vp]
 _lib.baoc_view.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(_vp), C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
 _lib.baoc_nonfinite.argtypes = [_vp, _vp, C.POINTER(C.c_int32), _vp]
+_lib.baoc_profile.argtypes = [_vp, C.c_int]
+_lib.baoc_profile_last.argtypes = [_vp, C.POINTER(C.c_float)]
 _lib.baoc_sample_stats_noalloc.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_double, C.c_double, C.c_double, _vp, _vp]
 _lib.baoc_noalloc_last_error.argtypes = []
 _lib.baoc_noalloc_last_error.restype = C.c_char_p
@@ -287,6 +289,15 @@ class Baoc:
                 flat = buf.view(torch.uint8).reshape(-1)
                 return flat[p - base: p - base + n * eb].view(dtype)
         raise BaocError(E_STATE, "the tensor lies in no buffer bound through this object")
+
+    def profile(self, enable: bool):
+        self._check(_lib.baoc_profile(self._h, int(bool(enable))))
+
+    def profile_last(self):
+        """(ms of the factored row/column kernels, ms of the fused update kernel) of the last step."""
+        ms = (C.c_float * 2)()
+        self._check(_lib.baoc_profile_last(self._h, ms))
+        return float(ms[0]), float(ms[1])
 
     def nonfinite(self):
         flags = np.zeros(self.n_blocks, np.uint8)

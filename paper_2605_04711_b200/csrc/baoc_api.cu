@@ -93,6 +93,7 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
     fill_step_params(h, t, &P);
     const auto& L = h->tl;
     CU(cudaMemsetAsync(h->st + L.flags, 0, 4 * size_t(h->n_blocks), s), "baoc_step (flags)");
+    if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[0]), s), "baoc_step (profile)");
     if (h->n_factored > 0) {
         LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles),
                                       at<int32_t>(h->st, L.f_ids), at<const void*>(h->st, L.grads),
@@ -100,10 +101,15 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
                "factored_reduce_kernel");
         h->launches += 2;
     }
+    if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[1]), s), "baoc_step (profile)");
     LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles), at<const void*>(h->st, L.grads),
                              at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), h->n_step_tiles, P, s),
            "fused_step_kernel");
     h->launches += 1;
+    if (h->prof_on) {
+        CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[2]), s), "baoc_step (profile)");
+        h->prof_valid = true;
+    }
     return BAOC_OK;
 }
 
@@ -356,6 +362,38 @@ int baoc_step_from_host(baoc_t* h, const void* const* host_grads, void* const* d
         if (rc) return rc;
     }
     if (step_t > 0) return do_step(h, dg, params, step_t, s);
+    return BAOC_OK;
+}
+
+static void destroy_profile_events(Handle* h) {
+    for (void*& e : h->prof_ev) {
+        if (e) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+        e = nullptr;
+    }
+}
+
+int baoc_profile(baoc_t* h, int enable) {
+    if (!h) return BAOC_E_INVALID;
+    if (enable && !h->prof_ev[0]) {
+        for (void*& e : h->prof_ev) {
+            cudaEvent_t ev;
+            CU(cudaEventCreate(&ev), "baoc_profile");
+            e = ev;
+        }
+        h->cuda_cleanup = destroy_profile_events;
+    }
+    h->prof_on = enable != 0;
+    h->prof_valid = false;
+    return BAOC_OK;
+}
+
+int baoc_profile_last(baoc_t* h, float* ms2) {
+    if (!h) return BAOC_E_INVALID;
+    if (!ms2) return fail(h, BAOC_E_INVALID, "baoc_profile_last: null output");
+    if (!h->prof_on || !h->prof_valid) return fail(h, BAOC_E_STATE, "baoc_profile_last: profiling is off or no step has run");
+    CU(cudaEventSynchronize(static_cast<cudaEvent_t>(h->prof_ev[2])), "baoc_profile_last");
+    CU(cudaEventElapsedTime(&ms2[0], static_cast<cudaEvent_t>(h->prof_ev[0]), static_cast<cudaEvent_t>(h->prof_ev[1])), "baoc_profile_last");
+    CU(cudaEventElapsedTime(&ms2[1], static_cast<cudaEvent_t>(h->prof_ev[1]), static_cast<cudaEvent_t>(h->prof_ev[2])), "baoc_profile_last");
     return BAOC_OK;
 }
 

@@ -167,6 +167,12 @@ struct Handle {
     struct StepLayout {
         size_t blocks, tiles, red_tiles, f_ids, grads, params, flags, redpart, states, total;
     } tl{};
+
+    // optional per-kernel timing of the step (CUDA events, owned by the CUDA translation unit)
+    bool prof_on = false, prof_valid = false;
+    void* prof_ev[3] = {nullptr, nullptr, nullptr};
+    void (*cuda_cleanup)(Handle*) = nullptr;
+    ~Handle() { if (cuda_cleanup) cuda_cleanup(this); }
 };
 
 int fail(const Handle* h, int code, const std::string& msg);

@@ -1,0 +1,146 @@
+"""Parity at the benchmark's full size: the LLaMA-1B-shaped workload (1.14 B parameters, 146 blocks), in the
+launch configuration ``bench.py`` times (same tables, same tiles, the library's own budgeted assignment), checked
+on sampled outputs that the CPU oracle can compute one by one:
+
+  * statistics of whole sampled blocks (a vector, a 4 M and a 16.7 M matrix), and the window values plus the
+    anisotropy / signal-to-noise of the largest block (the 65.5 M-element token table);
+  * after three mixed steps, slices of element-wise blocks (fp32 Adam, RMS, SGD-m), whole quantisation blocks
+    of 8-bit blocks, and whole factored blocks (their row/column statistics need every element).
+
+Tolerances are the ones of test_gpu_parity.py.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import baoc_oracle as O
+from paper_2605_04711_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+T_WINDOW = 3
+N_STEPS = 3
+
+
+def _ocfg(c):
+    return O.Config(c.adaptive, c.momentum, c.decoupled_wd, c.factored, c.bits, lr=float(c.lr), beta1=float(c.beta1),
+                    beta2=float(c.beta2), eps=float(c.eps), weight_decay=float(c.weight_decay))
+
+
+def _close(got, ref, extra=0.0):
+    return abs(got - ref) <= 1e-4 * max(abs(ref), 1e-3) + extra
+
+
+def _slices(numel):
+    """Three 8192-element windows (multiples of 256, so they hold whole quantisation blocks): start, middle, and
+    the end of the block including its ragged tail."""
+    if numel <= 3 * 8192:
+        return [(0, numel)]
+    mid = (numel // 2) // 256 * 256
+    last = (numel - 8192 + 255) // 256 * 256
+    return [(0, 8192), (mid, mid + 8192), (last, numel)]
+
+
+def test_llama_1b_sampled_parity_in_the_benchmark_configuration():
+    from paper_2605_04711_b200 import harness as H
+    wl = W.make_workload("llama_1b", seed=0)
+    assert wl.numel == 1_139_345_408 and len(wl.blocks) == 146
+    sess = H.Session(wl, n_grad_sets=2)
+    sess.init_params()
+    o = O.Opts()
+    name_to_i = {b.name: i for i, b in enumerate(wl.blocks)}
+    full = [name_to_i["l0.norm1"], name_to_i["l3.attn.k"], name_to_i["l5.ffn.up"]]     # whole-block statistics
+    big = name_to_i["tok_emb"]                                                          # 65 536 000 elements
+    states = {i: O.stats_init(wl.blocks[i].numel) for i in full + [big]}
+    for t in range(1, T_WINDOW + 1):
+        k = sess.fill_grads(t)
+        sess.sample_stats(k)
+        for i, st in states.items():
+            O.stats_step(st, sess.block_grad_host(k, i), o)
+    run = sess.h.read_stats()
+    for i, st in states.items():
+        assert _close(run[i]["rho_bar"], st.rho_bar) and _close(run[i]["last_cos"], st.last_cos), wl.blocks[i].name
+        assert run[i]["n_cos"] == T_WINDOW - 1
+    # moments of the largest block on slices
+    mv = [sess.h.view_tensor(big, w, torch.float32) for w in (0, 1)]
+    for lo, hi in _slices(wl.blocks[big].numel):
+        for dev, ref in ((mv[0], states[big].m), (mv[1], states[big].v)):
+            got = dev[lo:hi].double().cpu().numpy()
+            assert np.max(np.abs(got - ref[lo:hi])) <= 1e-6 * np.max(np.abs(ref))
+
+    risk, st = sess.risk()
+    for i in full:
+        b = wl.blocks[i]
+        raw = O.stats_finalize(states[i], sess.block_param_host(i), b.rows, b.cols, o)
+        for key in ("A", "rho_bar", "snr", "C", "F", "Q32", "Q16", "Q8", "q10", "q90", "rho_mom",
+                    "err_m8", "err_v8", "err_m16", "err_v16"):
+            extra = T_WINDOW * 2.0 ** -23 if key.startswith("err_") else 0.0
+            assert _close(st[i][key], raw[key], extra), (b.name, key, st[i][key], raw[key])
+    # the largest block: exact quantiles over 65.5 M elements (radix select across 16 000 tiles) and the SNR
+    assert _close(st[big]["A"], O.anisotropy(states[big].v, o.eps)), (st[big]["A"],)
+    assert _close(st[big]["snr"], O.snr(states[big].m, states[big].v, o.eps))
+    del states, mv
+
+    assign, obj, rc = sess.allocate(risk)
+    assert rc == 0
+    mem, _ = sess.h.cost_model()
+    assert sum(int(mem[i, c]) for i, c in enumerate(assign)) <= int(wl.mem_budget_frac * 8 * wl.numel)
+    cfgs = [_ocfg(c) for c in sess.configs]
+    kinds = [O.config_kind(cfgs[c]) for c in assign]
+    assert len(set(kinds)) >= 3, set(kinds)                         # the 25 % budget forces a mixed assignment
+    sess.configure(assign)
+
+    # sampled blocks per path: the first, the last and the largest block that took the path
+    picks = []
+    for kind in sorted(set(kinds)):
+        ids = [i for i, k in enumerate(kinds) if k == kind]
+        if kind == "F":
+            ids = [i for i in ids if wl.blocks[i].numel <= 17_000_000] or ids
+            chosen = {ids[0], ids[-1]}
+        else:
+            chosen = {ids[0], ids[-1], max(ids, key=lambda i: wl.blocks[i].numel)}
+        picks += [(i, kind) for i in sorted(chosen)]
+    samples = []
+    for i, kind in picks:
+        b = wl.blocks[i]
+        for lo, hi in ([(0, b.numel)] if kind == "F" else _slices(b.numel)):
+            n = hi - lo
+            rows, cols = (b.rows, b.cols) if kind == "F" else (n, 1)
+            samples.append(dict(i=i, kind=kind, lo=lo, hi=hi, rows=rows, cols=cols,
+                                th=sess.param_views[i][lo:hi].double().cpu().numpy(),
+                                st=O.step_init(cfgs[assign[i]], n, rows, cols)))
+    for t in range(1, N_STEPS + 1):
+        k = sess.fill_grads(T_WINDOW + t)
+        sess.step(k, t)
+        for s in samples:
+            g = sess.grad_views[k][s["i"]][s["lo"]:s["hi"]].double().cpu().numpy()
+            s["th"] = O.step(s["th"], g, s["st"], cfgs[assign[s["i"]]], s["rows"], s["cols"])
+    torch.cuda.synchronize()
+    cnt, _ = sess.h.nonfinite()
+    assert cnt == 0
+    bad_codes, n_codes = 0, 0
+    for s in samples:
+        i, lo, hi, ref = s["i"], s["lo"], s["hi"], s["st"]
+        name = (wl.blocks[i].name, s["kind"], lo)
+        got = sess.param_views[i][lo:hi].double().cpu().numpy()
+        assert np.max(np.abs(got - s["th"])) <= 1e-6 * np.max(np.abs(s["th"])), name
+        f32 = lambda w, a, b: sess.h.view_tensor(i, w, torch.float32)[a:b].double().cpu().numpy()
+        rel = lambda x, y: float(np.max(np.abs(x - y)) / max(float(np.max(np.abs(y))), 1e-30))
+        if s["kind"] == "A32":
+            assert rel(f32(10, lo, hi), ref.m) <= 1e-6 and rel(f32(11, lo, hi), ref.v) <= 1e-6, name
+        elif s["kind"] in ("R", "S"):
+            assert rel(f32(10, lo, hi), ref.v if s["kind"] == "R" else ref.m) <= 1e-6, name
+        elif s["kind"] == "F":
+            assert rel(f32(10, 0, s["rows"]), ref.r) <= 1e-6 and rel(f32(11, 0, s["cols"]), ref.c) <= 1e-6, name
+        elif s["kind"] == "A8":
+            qm = sess.h.view_tensor(i, 10, torch.int8)[lo:hi].cpu().numpy().astype(np.int32)
+            qv = sess.h.view_tensor(i, 11, torch.uint8)[lo:hi].cpu().numpy().astype(np.int32)
+            dm, dv = np.abs(qm - ref.qm.astype(np.int32)), np.abs(qv - ref.qv.astype(np.int32))
+            assert dm.max() <= 1 and dv.max() <= 1, name
+            bad_codes += int((dm != 0).sum() + (dv != 0).sum())
+            n_codes += 2 * qm.size
+            q0, q1 = lo // 256, (hi + 255) // 256
+            assert rel(f32(12, q0, q1), ref.am.astype(np.float64)) <= 1e-6, name
+            assert rel(f32(13, q0, q1), ref.av.astype(np.float64)) <= 1e-6, name
+    if n_codes:
+        assert bad_codes <= 1e-4 * n_codes, (bad_codes, n_codes)
