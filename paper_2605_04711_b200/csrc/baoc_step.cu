@@ -337,8 +337,9 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
         const int64_t row0 = base / cols;
         const uint32_t col0 = uint32_t(base - row0 * cols);
         uint4 wg[kSlicesF];
-        float4 t0[kSlicesF], t1[kSlicesF], c0[kSlicesF], c1[kSlicesF];
+        float4 t0[kSlicesF], t1[kSlicesF];
         float ri[kSlicesF];
+        uint32_t cl[kSlicesF];
         bool in[kSlicesF];
 #pragma unroll
         for (int s = 0; s < kSlicesF; ++s) {
@@ -351,8 +352,7 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
                 const uint32_t col = cc - q * uint32_t(cols);
                 wg[s] = ld_stream_u4(g + e);
                 t0[s] = ld_stream_f4(th + e); t1[s] = ld_stream_f4(th + e + 4);
-                c0[s] = __ldg(reinterpret_cast<const float4*>(c + col));
-                c1[s] = __ldg(reinterpret_cast<const float4*>(c + col + 4));
+                cl[s] = col;
                 ri[s] = __ldg(r + row0 + q);
             }
         }
@@ -361,7 +361,8 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
             if (!in[s]) continue;
             const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
             float x[8], t[8], cj[8];
-            unpack8(wg[s], x); f4_to(t0[s], t1[s], t); f4_to(c0[s], c1[s], cj);
+            unpack8(wg[s], x); f4_to(t0[s], t1[s], t);
+            f4_to(__ldg(reinterpret_cast<const float4*>(c + cl[s])), __ldg(reinterpret_cast<const float4*>(c + cl[s] + 4)), cj);
             const float rs = ri[s] * inv_rm;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -468,55 +469,47 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float chk = 0.f;
 
-    uint4 wg[kSlices];
-    float4 t0[kSlices], t1[kSlices];
-    uint2 wm[kSlices], wv[kSlices];
-    float amo[kSlices], avo[kSlices];
-    int cnt[kSlices];
-#pragma unroll
+    // one slice at a time: the path is bound by instruction issue, not by bytes in flight, and holding the
+    // next slice's loads would push the whole kernel past 80 registers (three CTAs per SM)
+#pragma unroll 1
     for (int s = 0; s < kSlices; ++s) {
         const int64_t w0 = base + int64_t(s) * (kThreads * 8) + int64_t(warp) * kQBlock;
-        cnt[s] = -1;                                                // whole warp out of range
-        if (w0 >= numel) continue;
+        if (w0 >= numel) break;                                     // whole warp out of range (and so is the next slice)
         const int64_t e = w0 + lane * 8;
-        cnt[s] = int(max64(0, min64(8, numel - e)));
-        amo[s] = am[w0 / kQBlock]; avo[s] = av[w0 / kQBlock];
-        if (cnt[s] == 8) {
-            wg[s] = ld_stream_u4(g + e);
-            t0[s] = ld_stream_f4(th + e); t1[s] = ld_stream_f4(th + e + 4);
-            wm[s] = ld_stream_u2(qm + e);
-            wv[s] = ld_stream_u2(qv + e);
+        const int cnt = int(max64(0, min64(8, numel - e)));
+        const float amo = am[w0 / kQBlock], avo = av[w0 / kQBlock];
+        uint4 wg;
+        float4 t0, t1;
+        uint2 wm, wv;
+        if (cnt == 8) {
+            wg = ld_stream_u4(g + e);
+            t0 = ld_stream_f4(th + e); t1 = ld_stream_f4(th + e + 4);
+            wm = ld_stream_u2(qm + e);
+            wv = ld_stream_u2(qv + e);
         } else {                                                    // ragged end of the block: zero-fill
-            const int n = cnt[s];
+            const int n = cnt;
             auto gg = [&](int j) { return j < n ? uint32_t(g[e + j]) : 0u; };
             auto tt = [&](int j) { return j < n ? th[e + j] : 0.f; };
             auto mm = [&](int j) { return j < n ? uint32_t(uint8_t(qm[e + j])) : 0u; };
             auto vv = [&](int j) { return j < n ? uint32_t(qv[e + j]) : 0u; };
-            wg[s] = make_uint4(gg(0) | gg(1) << 16, gg(2) | gg(3) << 16, gg(4) | gg(5) << 16, gg(6) | gg(7) << 16);
-            t0[s] = make_float4(tt(0), tt(1), tt(2), tt(3)); t1[s] = make_float4(tt(4), tt(5), tt(6), tt(7));
-            wm[s] = make_uint2(mm(0) | mm(1) << 8 | mm(2) << 16 | mm(3) << 24, mm(4) | mm(5) << 8 | mm(6) << 16 | mm(7) << 24);
-            wv[s] = make_uint2(vv(0) | vv(1) << 8 | vv(2) << 16 | vv(3) << 24, vv(4) | vv(5) << 8 | vv(6) << 16 | vv(7) << 24);
+            wg = make_uint4(gg(0) | gg(1) << 16, gg(2) | gg(3) << 16, gg(4) | gg(5) << 16, gg(6) | gg(7) << 16);
+            t0 = make_float4(tt(0), tt(1), tt(2), tt(3)); t1 = make_float4(tt(4), tt(5), tt(6), tt(7));
+            wm = make_uint2(mm(0) | mm(1) << 8 | mm(2) << 16 | mm(3) << 24, mm(4) | mm(5) << 8 | mm(6) << 16 | mm(7) << 24);
+            wv = make_uint2(vv(0) | vv(1) << 8 | vv(2) << 16 | vv(3) << 24, vv(4) | vv(5) << 8 | vv(6) << 16 | vv(7) << 24);
         }
-    }
-
-#pragma unroll
-    for (int s = 0; s < kSlices; ++s) {
-        if (cnt[s] < 0) continue;
-        const int64_t w0 = base + int64_t(s) * (kThreads * 8) + int64_t(warp) * kQBlock;
-        const int64_t e = w0 + lane * 8;
         float x[8], t[8], mf[8], vf[8];
-        unpack8(wg[s], x); f4_to(t0[s], t1[s], t);
+        unpack8(wg, x); f4_to(t0, t1, t);
         Q8Ctx q;
         q.b1 = P.beta1_d; q.b2 = P.beta2_d; q.wd = P.wd_d;
-        q.am_old = amo[s]; q.av_old = avo[s]; q.coupled = P.coupled;
+        q.am_old = amo; q.av_old = avo; q.coupled = P.coupled;
 
         // fp32 pass: effective gradient, decayed parameter, new moments, their maxima.
         // A code byte b is turned into the float 2^23 + b by placing it in the low
         // mantissa byte of 0x4B000000 (signed codes are first offset by 128).
-        const float b1s = P.beta1 * (amo[s] / 127.0f), b2s = P.beta2 * (avo[s] / 255.0f);
+        const float b1s = P.beta1 * (amo / 127.0f), b2s = P.beta2 * (avo / 255.0f);
         const float vbias = -8388608.0f * b2s;                      // exact: a power-of-two multiple
-        const uint32_t ms[2] = {wm[s].x ^ 0x80808080u, wm[s].y ^ 0x80808080u};
-        const uint32_t vs[2] = {wv[s].x, wv[s].y};
+        const uint32_t ms[2] = {wm.x ^ 0x80808080u, wm.y ^ 0x80808080u};
+        const uint32_t vs[2] = {wv.x, wv.y};
         float mx = 0.f, vx = 0.f;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -528,7 +521,7 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
             mx = fmaxf(mx, fabsf(mf[j])); vx = fmaxf(vx, vf[j]);
         }
         mx = warp_max_nonneg(mx); vx = warp_max_nonneg(vx);
-        const float Em = kSlack * (amo[s] + mx), Ev = kSlack * (avo[s] + vx);
+        const float Em = kSlack * (amo + mx), Ev = kSlack * (avo + vx);
 
         // exact absmax: only elements within 2E of the fp32 maximum can hold it.
         // (theta: the coupled gradient needs the parameter before the update; prologue leaves it untouched then.)
@@ -538,9 +531,9 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         for (int j = 0; j < 8; ++j) {
             const bool cand_m = fabsf(mf[j]) >= m_thr, cand_v = vf[j] >= v_thr;
             if (cand_m || cand_v) {
-                const double gd = exact_grad(half_of(wg[s], j), t[j], q);
-                if (cand_m) am_c = fmaxf(am_c, __double2float_rn(fabs(exact_m(int(int8_t(byte_of(wm[s], j))), gd, q))));
-                if (cand_v) av_c = fmaxf(av_c, __double2float_rn(exact_v(int(byte_of(wv[s], j)), gd, q)));
+                const double gd = exact_grad(half_of(wg, j), t[j], q);
+                if (cand_m) am_c = fmaxf(am_c, __double2float_rn(fabs(exact_m(int(int8_t(byte_of(wm, j))), gd, q))));
+                if (cand_v) av_c = fmaxf(av_c, __double2float_rn(exact_v(int(byte_of(wv, j)), gd, q)));
             }
         }
         const float am_new = warp_max_nonneg(am_c), av_new = warp_max_nonneg(av_c);
@@ -557,9 +550,9 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
             cmw[j] = __float_as_uint(rm_); cvw[j] = __float_as_uint(rv_);
             const bool slow_m = !(fabsf(dm) <= hm), slow_v = !(fabsf(dv) <= hv);
             if (slow_m || slow_v) {
-                const double gd = exact_grad(half_of(wg[s], j), t[j], q);
-                if (slow_m) cmw[j] = uint32_t(encode_exact(exact_m(int(int8_t(byte_of(wm[s], j))), gd, q), am_new, 127.0, -127));
-                if (slow_v) cvw[j] = uint32_t(encode_exact(exact_v(int(byte_of(wv[s], j)), gd, q), av_new, 255.0, 0));
+                const double gd = exact_grad(half_of(wg, j), t[j], q);
+                if (slow_m) cmw[j] = uint32_t(encode_exact(exact_m(int(int8_t(byte_of(wm, j))), gd, q), am_new, 127.0, -127));
+                if (slow_v) cvw[j] = uint32_t(encode_exact(exact_v(int(byte_of(wv, j)), gd, q), av_new, 255.0, 0));
             }
         }
         const uint2 om = make_uint2(pack_low_bytes(cmw[0], cmw[1], cmw[2], cmw[3]), pack_low_bytes(cmw[4], cmw[5], cmw[6], cmw[7]));
@@ -572,14 +565,14 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
             chk = poison(chk, t[j]);
         }
 
-        if (cnt[s] == 8) {
+        if (cnt == 8) {
             st8(th + e, t);
             st_stream_u2(qm + e, om);
             st_stream_u2(qv + e, ov);
         } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {                          // static indices keep t[] in registers
-                if (j < cnt[s]) {
+                if (j < cnt) {
                     th[e + j] = t[j];
                     qm[e + j] = int8_t(((j < 4 ? om.x : om.y) >> (8 * (j & 3))) & 0xffu);
                     qv[e + j] = uint8_t(((j < 4 ? ov.x : ov.y) >> (8 * (j & 3))) & 0xffu);
@@ -591,7 +584,7 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
     return chk != 0.f;
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 3)
 fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
                   const void* const* __restrict__ grads, float* const* __restrict__ params,
                   uint32_t* __restrict__ flags, const __grid_constant__ StepParams SP) {
