@@ -27,6 +27,7 @@ constexpr int kFinOut = 32;           // doubles per block copied to the host at
 constexpr int kRedRows = 64;          // rows per CTA of the row/column reduction kernel
 constexpr int kRedCols = 512;         // columns per CTA of the row/column reduction kernel
 constexpr int kTileF = 8192;          // elements per tile of the factored path (10 bytes per element: more elements keep as many bytes in flight)
+constexpr int kTileQ = 16384;         // elements per tile of the 8-bit path (its slices are prefetched through shared memory)
 constexpr int kCombineSlabs = 32;     // CTAs per factored block of the row/column combine
 
 // Update paths of the fused step.
@@ -41,7 +42,7 @@ inline Path path_of(const baoc_config_t& c) {
 }
 
 // Elements per tile of the fused step, by update path.
-inline int64_t step_tile_elems(int path) { return path == kPathF ? kTileF : kTile; }
+inline int64_t step_tile_elems(int path) { return path == kPathF ? kTileF : (path == kPathA8 ? kTileQ : kTile); }
 
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }

@@ -405,49 +405,74 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
 // code' = rne(127 m' / a')   (and likewise for v with 255 levels).  Doing all of
 // it in double costs about 20 FP64 operations per element and makes the path
 // FP64-bound, so the work is split:
-//   * every element is evaluated in fp32 (the parameter update needs those
-//     values anyway); its error against the exact value is below
-//     E = 2^-21 (a_old + max|m'|) (five roundings of magnitude <= 2^-24 of terms
-//     bounded by a_old and max|m'|, with head room);
+//   * every element is evaluated in fp32, two elements per instruction (the
+//     parameter update needs those values anyway); its error against the exact
+//     value is below E = 2^-21 (a_old + max|m'|): first-order bound
+//     2^-24 (4 max|m'| + 6 a_old) from the roundings of a_old/127, beta1*that,
+//     (1-beta1)*g (with a coupled, rounded g) and the final FMA;
 //   * the new absmax is the fp32 rounding of the largest exact |m'|, and only
-//     elements within 2E of the fp32 maximum can hold it, so only those are
-//     recomputed in double;
+//     elements within 2E of the fp32 maximum can hold it.  Lanes that own such an
+//     element are visited in a warp-uniform loop: their raw inputs are broadcast
+//     and lanes 0-7 (first moment) and 8-15 (second moment) recompute the lane's
+//     eight elements in double, so the recomputation never diverges;
 //   * a code is rne(q) with q = 127 m' / a'; the fp32 q is within
 //     w = 127 E / a' + 2^-14 of the exact one, so unless it lies within w of a
-//     half-integer the fp32 rounding is already the exact answer; the few
-//     elements that do are recomputed in double (exact ties, which bf16
-//     gradients produce from a zero state, fall in here and are resolved by the
-//     correctly rounded division).
+//     half-integer the fp32 rounding is already the exact answer.  Lanes with such
+//     an element are visited the same way and get all eight codes from the
+//     correctly rounded double division (exact ties, which bf16 gradients
+//     produce from a zero state, are resolved there).
 // ----------------------------------------------------------------------------
-struct Q8Ctx {
-    double b1, b2, wd;
-    float am_old, av_old;
-    int coupled;
+__device__ __forceinline__ uint32_t pick_word(uint32_t a, uint32_t b, uint32_t c, uint32_t d, int k) {
+    return (k & 2) ? ((k & 1) ? d : c) : ((k & 1) ? b : a);
+}
+
+// Raw inputs of the 8 elements of lane `src`, as seen by lane j = lane & 7 of a helper group.
+struct Q8Raw {
+    uint32_t gbits;      // bf16 gradient of element j
+    uint32_t cm, cv;     // code bytes of element j
+    float theta;         // parameter of element j before the update (coupled decay only)
 };
 
-__device__ __forceinline__ double exact_grad(uint32_t gbits16, float theta, const Q8Ctx& q) {
-    double gd = widen_bf16_float(__uint_as_float(gbits16 << 16));
-    if (q.coupled) gd += q.wd * double(theta);
-    return gd;
-}
-__device__ __forceinline__ double exact_m(int cm, double gd, const Q8Ctx& q) {
-    return q.b1 * (int_to_double(cm) * double(q.am_old) * (1.0 / 127.0)) + (1.0 - q.b1) * gd;
-}
-__device__ __forceinline__ double exact_v(int cv, double gd, const Q8Ctx& q) {
-    return q.b2 * (int_to_double(cv) * double(q.av_old) * (1.0 / 255.0)) + (1.0 - q.b2) * (gd * gd);
+__device__ __forceinline__ Q8Raw q8_fetch(int src, int j, const uint4& wg, const uint2& wm, const uint2& wv,
+                                          const float (&t)[8], bool coupled) {
+    const unsigned full = 0xffffffffu;
+    const uint32_t gx = __shfl_sync(full, wg.x, src), gy = __shfl_sync(full, wg.y, src);
+    const uint32_t gz = __shfl_sync(full, wg.z, src), gw = __shfl_sync(full, wg.w, src);
+    const uint32_t mx = __shfl_sync(full, wm.x, src), my = __shfl_sync(full, wm.y, src);
+    const uint32_t vx = __shfl_sync(full, wv.x, src), vy = __shfl_sync(full, wv.y, src);
+    Q8Raw r;
+    const uint32_t w = pick_word(gx, gy, gz, gw, j >> 1);
+    r.gbits = (j & 1) ? (w >> 16) : (w & 0xffffu);
+    r.cm = (((j & 4) ? my : mx) >> (8 * (j & 3))) & 0xffu;
+    r.cv = (((j & 4) ? vy : vx) >> (8 * (j & 3))) & 0xffu;
+    r.theta = 0.f;
+    if (coupled) {                                                  // uniform branch
+        float tt[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) tt[k] = __shfl_sync(full, t[k], src);
+        const float a = (j & 1) ? tt[1] : tt[0], b = (j & 1) ? tt[3] : tt[2];
+        const float c = (j & 1) ? tt[5] : tt[4], d = (j & 1) ? tt[7] : tt[6];
+        r.theta = (j & 4) ? ((j & 2) ? d : c) : ((j & 2) ? b : a);
+    }
+    return r;
 }
 
-// clamp(rne(L * x / a)) by the correctly rounded division (a > 0 whenever this is reached with x != 0).
+// Exact (double) new moment of one element: first moment for group 0, second for group 1.
+__device__ __forceinline__ double q8_exact(const Q8Raw& r, bool second, float am_old, float av_old, const CfgStep& P) {
+    double gd = widen_bf16_float(__uint_as_float(r.gbits << 16));
+    if (P.coupled) gd += P.wd_d * double(r.theta);
+    const double beta = second ? P.beta2_d : P.beta1_d;
+    const int code = second ? int(r.cv) : int(int8_t(r.cm));
+    const double old = int_to_double(code) * (second ? double(av_old) * (1.0 / 255.0) : double(am_old) * (1.0 / 127.0));
+    return beta * old + (1.0 - beta) * (second ? gd * gd : gd);
+}
+
+// clamp(rne(L * x / a)) by the correctly rounded division.
 __device__ __forceinline__ int encode_exact(double x, float absmax, double levels, int lo) {
     if (!(absmax > 0.0f)) return 0;
     return max(lo, min(int(levels), round_to_int((levels * x) / double(absmax))));
 }
 
-__device__ __forceinline__ uint32_t half_of(const uint4& w, int j) {
-    const uint32_t word = j < 2 ? w.x : (j < 4 ? w.y : (j < 6 ? w.z : w.w));
-    return (j & 1) ? (word >> 16) : (word & 0xffffu);
-}
-__device__ __forceinline__ uint32_t byte_of(const uint2& w, int j) { return ((j < 4 ? w.x : w.y) >> (8 * (j & 3))) & 0xffu; }
 // Lowest bytes of four words, packed in order.
 __device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     return __byte_perm(__byte_perm(a, b, 0x0040u), __byte_perm(c, d, 0x0040u), 0x5410u);
@@ -461,31 +486,63 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
                                               float* __restrict__ th, int64_t base) {
     constexpr float kSlack = 4.76837158203125e-7f;                 // 2^-21
     constexpr float kMagic = 12582912.0f;                          // 1.5 * 2^23: adding it rounds to an integer, ties to even
+    const unsigned full = 0xffffffffu;
     const int64_t numel = b->numel;
     int8_t* __restrict__ qm = static_cast<int8_t*>(b->s0);
     uint8_t* __restrict__ qv = static_cast<uint8_t*>(b->s1);
     float* __restrict__ am = b->a0;
     float* __restrict__ av = b->a1;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float chk = 0.f;
+    const int hj = lane & 7;                                        // element handled when helping another lane
+    const bool hv_grp = (lane & 8) != 0, helper = lane < 16;       // lanes 0-7: first moment, 8-15: second moment
+    const bool coupled = P.coupled != 0;
+    f32x2 chk = pack2(0.f, 0.f);
 
-    // one slice at a time: the path is bound by instruction issue, not by bytes in flight, and holding the
-    // next slice's loads would push the whole kernel past 80 registers (three CTAs per SM)
-#pragma unroll 1
-    for (int s = 0; s < kSlices; ++s) {
+    // Slices are prefetched one ahead through shared memory: every thread copies the 64 bytes of its own next
+    // eight elements (gradient, parameters, both code words) into its own slot with cp.async and reads them back
+    // itself, so no registers are held across the long arithmetic of the current slice and no barrier is needed.
+    constexpr int kSlicesQ = kTileQ / (kThreads * 8);
+    __shared__ __align__(16) unsigned char stage[2][kThreads * 64];
+    auto slot = [&](int st, int off) { return &stage[st][0] + off; };   // off: 0 g (16 B/thread), 4096 theta (32), 12288 m codes (8), 14336 v codes (8)
+    auto prefetch = [&](int s) {
         const int64_t w0 = base + int64_t(s) * (kThreads * 8) + int64_t(warp) * kQBlock;
-        if (w0 >= numel) break;                                     // whole warp out of range (and so is the next slice)
+        const int64_t e = w0 + lane * 8;
+        if (s < kSlicesQ && e + 8 <= numel) {                      // ragged or absent elements are loaded directly later
+            const int st = s & 1;
+            cp_async16(smem_addr(slot(st, threadIdx.x * 16)), g + e);
+            cp_async16(smem_addr(slot(st, 4096 + threadIdx.x * 32)), th + e);
+            cp_async16(smem_addr(slot(st, 4096 + threadIdx.x * 32 + 16)), th + e + 4);
+            cp_async8(smem_addr(slot(st, 12288 + threadIdx.x * 8)), qm + e);
+            cp_async8(smem_addr(slot(st, 14336 + threadIdx.x * 8)), qv + e);
+        }
+        cp_async_commit();
+    };
+    prefetch(0);
+    float amo_next = 0.f, avo_next = 0.f;
+    if (base + int64_t(warp) * kQBlock < numel) { amo_next = am[(base + int64_t(warp) * kQBlock) / kQBlock]; avo_next = av[(base + int64_t(warp) * kQBlock) / kQBlock]; }
+#pragma unroll 1
+    for (int s = 0; s < kSlicesQ; ++s) {
+        const int64_t w0 = base + int64_t(s) * (kThreads * 8) + int64_t(warp) * kQBlock;
+        prefetch(s + 1);
+        const float amo = amo_next, avo = avo_next;
+        {
+            const int64_t w1 = w0 + int64_t(kThreads) * 8;
+            if (s + 1 < kSlicesQ && w1 < numel) { amo_next = am[w1 / kQBlock]; avo_next = av[w1 / kQBlock]; }
+        }
+        cp_async_wait<1>();                                         // this slice's copies have landed (the next one's may be in flight)
+        if (w0 >= numel) break;                                     // whole warp out of range (and so are the later slices)
         const int64_t e = w0 + lane * 8;
         const int cnt = int(max64(0, min64(8, numel - e)));
-        const float amo = am[w0 / kQBlock], avo = av[w0 / kQBlock];
         uint4 wg;
         float4 t0, t1;
         uint2 wm, wv;
         if (cnt == 8) {
-            wg = ld_stream_u4(g + e);
-            t0 = ld_stream_f4(th + e); t1 = ld_stream_f4(th + e + 4);
-            wm = ld_stream_u2(qm + e);
-            wv = ld_stream_u2(qv + e);
+            const int st = s & 1;
+            wg = *reinterpret_cast<const uint4*>(slot(st, threadIdx.x * 16));
+            t0 = *reinterpret_cast<const float4*>(slot(st, 4096 + threadIdx.x * 32));
+            t1 = *reinterpret_cast<const float4*>(slot(st, 4096 + threadIdx.x * 32 + 16));
+            wm = *reinterpret_cast<const uint2*>(slot(st, 12288 + threadIdx.x * 8));
+            wv = *reinterpret_cast<const uint2*>(slot(st, 14336 + threadIdx.x * 8));
         } else {                                                    // ragged end of the block: zero-fill
             const int n = cnt;
             auto gg = [&](int j) { return j < n ? uint32_t(g[e + j]) : 0u; };
@@ -497,72 +554,103 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
             wm = make_uint2(mm(0) | mm(1) << 8 | mm(2) << 16 | mm(3) << 24, mm(4) | mm(5) << 8 | mm(6) << 16 | mm(7) << 24);
             wv = make_uint2(vv(0) | vv(1) << 8 | vv(2) << 16 | vv(3) << 24, vv(4) | vv(5) << 8 | vv(6) << 16 | vv(7) << 24);
         }
-        float x[8], t[8], mf[8], vf[8];
-        unpack8(wg, x); f4_to(t0, t1, t);
-        Q8Ctx q;
-        q.b1 = P.beta1_d; q.b2 = P.beta2_d; q.wd = P.wd_d;
-        q.am_old = amo; q.av_old = avo; q.coupled = P.coupled;
+        float t[8];                                                 // parameters before the update (kept for the coupled exact side)
+        f4_to(t0, t1, t);
 
-        // fp32 pass: effective gradient, decayed parameter, new moments, their maxima.
-        // A code byte b is turned into the float 2^23 + b by placing it in the low
-        // mantissa byte of 0x4B000000 (signed codes are first offset by 128).
-        const float b1s = P.beta1 * (amo / 127.0f), b2s = P.beta2 * (avo / 255.0f);
-        const float vbias = -8388608.0f * b2s;                      // exact: a power-of-two multiple
+        // ---- fp32 pass, two elements per instruction: effective gradient, decayed parameter, new moments
+        // A code byte c becomes the float 2^23 + c by placing it in the low mantissa
+        // byte of 0x4B000000 (signed codes are first offset by 128).
+        const float b1s = P.beta1 * (amo * (1.0f / 127.0f)), b2s = P.beta2 * (avo * (1.0f / 255.0f));
+        const f32x2 B1S = splat2(b1s), B2S = splat2(b2s), VB = splat2(-8388608.0f * b2s);   // the bias is exact: a power-of-two multiple
+        const f32x2 OM1 = splat2(P.om1), OM2 = splat2(P.om2), MOFF = splat2(-8388736.0f);
+        const uint32_t gw[4] = {wg.x, wg.y, wg.z, wg.w};
         const uint32_t ms[2] = {wm.x ^ 0x80808080u, wm.y ^ 0x80808080u};
         const uint32_t vs[2] = {wv.x, wv.y};
-        float mx = 0.f, vx = 0.f;
+        f32x2 T[4], MF[4], VF[4];
+        float lm = 0.f, lv = 0.f;                                   // this lane's maxima
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float fm = __uint_as_float(__byte_perm(ms[j >> 2], 0x4B000000u, 0x7440u | (j & 3))) - 8388736.0f;
-            const float fv = __uint_as_float(__byte_perm(vs[j >> 2], 0x4B000000u, 0x7440u | (j & 3)));
-            prologue(x[j], t[j], P);
-            mf[j] = fmaf(fm, b1s, P.om1 * x[j]);
-            vf[j] = fmaf(P.om2 * x[j], x[j], fmaf(fv, b2s, vbias));
-            mx = fmaxf(mx, fabsf(mf[j])); vx = fmaxf(vx, vf[j]);
+        for (int p = 0; p < 4; ++p) {
+            f32x2 X = pack2(bf16_lo(gw[p]), bf16_hi(gw[p]));
+            T[p] = pack2(t[2 * p], t[2 * p + 1]);
+            if (coupled) X = fma2(splat2(P.wd), T[p], X);
+            else T[p] = fma2(splat2(P.decay), T[p], T[p]);
+            const uint32_t mw = ms[p >> 1], vw = vs[p >> 1];
+            const int k0 = (2 * p) & 3, k1 = (2 * p + 1) & 3;
+            const f32x2 FM = add2(pack2(__uint_as_float(__byte_perm(mw, 0x4B000000u, 0x7440u | k0)),
+                                        __uint_as_float(__byte_perm(mw, 0x4B000000u, 0x7440u | k1))), MOFF);
+            const f32x2 FV = pack2(__uint_as_float(__byte_perm(vw, 0x4B000000u, 0x7440u | k0)),
+                                   __uint_as_float(__byte_perm(vw, 0x4B000000u, 0x7440u | k1)));
+            MF[p] = fma2(FM, B1S, mul2(OM1, X));
+            VF[p] = fma2(mul2(OM2, X), X, fma2(FV, B2S, VB));
+            float a0, a1, c0, c1;
+            unpack2(MF[p], a0, a1); unpack2(VF[p], c0, c1);
+            lm = max3(lm, fabsf(a0), fabsf(a1)); lv = max3(lv, c0, c1);
         }
-        mx = warp_max_nonneg(mx); vx = warp_max_nonneg(vx);
+        const float mx = warp_max_nonneg(lm), vx = warp_max_nonneg(lv);
         const float Em = kSlack * (amo + mx), Ev = kSlack * (avo + vx);
 
-        // exact absmax: only elements within 2E of the fp32 maximum can hold it.
-        // (theta: the coupled gradient needs the parameter before the update; prologue leaves it untouched then.)
+        // ---- exact absmax
+        unsigned cand_m = __ballot_sync(full, lm >= mx - 2.0f * Em), cand_v = __ballot_sync(full, lv >= vx - 2.0f * Ev);
         float am_c = 0.f, av_c = 0.f;
-        const float m_thr = mx - 2.0f * Em, v_thr = vx - 2.0f * Ev;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const bool cand_m = fabsf(mf[j]) >= m_thr, cand_v = vf[j] >= v_thr;
-            if (cand_m || cand_v) {
-                const double gd = exact_grad(half_of(wg, j), t[j], q);
-                if (cand_m) am_c = fmaxf(am_c, __double2float_rn(fabs(exact_m(int(int8_t(byte_of(wm, j))), gd, q))));
-                if (cand_v) av_c = fmaxf(av_c, __double2float_rn(exact_v(int(byte_of(wv, j)), gd, q)));
+        while (cand_m | cand_v) {                                   // warp-uniform
+            const int Lm = cand_m ? __ffs(cand_m) - 1 : -1, Lv = cand_v ? __ffs(cand_v) - 1 : -1;
+            cand_m &= cand_m - 1u; cand_v &= cand_v - 1u;           // (0 & anything stays 0)
+            const int src = hv_grp ? Lv : Lm;
+            const Q8Raw r = q8_fetch(max(src, 0), hj, wg, wm, wv, t, coupled);
+            const float val = __double2float_rn(fabs(q8_exact(r, hv_grp, amo, avo, P)));
+            if (helper && src >= 0) {
+                if (hv_grp) av_c = fmaxf(av_c, val); else am_c = fmaxf(am_c, val);
             }
         }
         const float am_new = warp_max_nonneg(am_c), av_new = warp_max_nonneg(av_c);
 
-        // codes: rne(q) = low byte of the float q + 1.5*2^23, taken from the fp32
-        // value unless it is within w of a half-integer
+        // ---- codes: rne(q) = low byte of the float q + 1.5*2^23
         const float km = am_new > 0.f ? 127.0f / am_new : 0.f, kv = av_new > 0.f ? 255.0f / av_new : 0.f;
         const float hm = 0.5f - (Em * km + 6.103515625e-5f), hv = 0.5f - (Ev * kv + 6.103515625e-5f);
+        const f32x2 KM = splat2(km), KV = splat2(kv), MAGIC = splat2(kMagic), MINUS1 = splat2(-1.0f);
         uint32_t cmw[8], cvw[8];
+        float dm = 0.f, dv = 0.f;                                   // largest distance to the chosen integer in this lane
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float rm_ = fmaf(mf[j], km, kMagic), rv_ = fmaf(vf[j], kv, kMagic);
-            const float dm = fmaf(mf[j], km, kMagic - rm_), dv = fmaf(vf[j], kv, kMagic - rv_);
-            cmw[j] = __float_as_uint(rm_); cvw[j] = __float_as_uint(rv_);
-            const bool slow_m = !(fabsf(dm) <= hm), slow_v = !(fabsf(dv) <= hv);
-            if (slow_m || slow_v) {
-                const double gd = exact_grad(half_of(wg, j), t[j], q);
-                if (slow_m) cmw[j] = uint32_t(encode_exact(exact_m(int(int8_t(byte_of(wm, j))), gd, q), am_new, 127.0, -127));
-                if (slow_v) cvw[j] = uint32_t(encode_exact(exact_v(int(byte_of(wv, j)), gd, q), av_new, 255.0, 0));
-            }
+        for (int p = 0; p < 4; ++p) {
+            const f32x2 RM = fma2(MF[p], KM, MAGIC), RV = fma2(VF[p], KV, MAGIC);
+            const f32x2 DM = fma2(MF[p], KM, fma2(RM, MINUS1, MAGIC)), DV = fma2(VF[p], KV, fma2(RV, MINUS1, MAGIC));
+            float r0, r1, d0, d1;
+            unpack2(RM, r0, r1); unpack2(DM, d0, d1);
+            cmw[2 * p] = __float_as_uint(r0); cmw[2 * p + 1] = __float_as_uint(r1);
+            dm = max3(dm, fabsf(d0), fabsf(d1));
+            unpack2(RV, r0, r1); unpack2(DV, d0, d1);
+            cvw[2 * p] = __float_as_uint(r0); cvw[2 * p + 1] = __float_as_uint(r1);
+            dv = max3(dv, fabsf(d0), fabsf(d1));
         }
-        const uint2 om = make_uint2(pack_low_bytes(cmw[0], cmw[1], cmw[2], cmw[3]), pack_low_bytes(cmw[4], cmw[5], cmw[6], cmw[7]));
-        const uint2 ov = make_uint2(pack_low_bytes(cvw[0], cvw[1], cvw[2], cvw[3]), pack_low_bytes(cvw[4], cvw[5], cvw[6], cvw[7]));
+        uint2 om = make_uint2(pack_low_bytes(cmw[0], cmw[1], cmw[2], cmw[3]), pack_low_bytes(cmw[4], cmw[5], cmw[6], cmw[7]));
+        uint2 ov = make_uint2(pack_low_bytes(cvw[0], cvw[1], cvw[2], cvw[3]), pack_low_bytes(cvw[4], cvw[5], cvw[6], cvw[7]));
+        unsigned slow_m = __ballot_sync(full, !(dm <= hm)), slow_v = __ballot_sync(full, !(dv <= hv));
+        while (slow_m | slow_v) {                                   // warp-uniform, rare
+            const int Lm = slow_m ? __ffs(slow_m) - 1 : -1, Lv = slow_v ? __ffs(slow_v) - 1 : -1;
+            slow_m &= slow_m - 1u; slow_v &= slow_v - 1u;
+            const int src = hv_grp ? Lv : Lm;
+            const Q8Raw r = q8_fetch(max(src, 0), hj, wg, wm, wv, t, coupled);
+            const double x = q8_exact(r, hv_grp, amo, avo, P);
+            const int code = hv_grp ? encode_exact(x, av_new, 255.0, 0) : encode_exact(x, am_new, 127.0, -127);
+            const uint32_t piece = (helper && src >= 0) ? (uint32_t(code) & 0xffu) << (8 * (hj & 3)) : 0u;
+            const uint32_t mlo = __reduce_or_sync(full, (!hv_grp && hj < 4) ? piece : 0u);
+            const uint32_t mhi = __reduce_or_sync(full, (!hv_grp && hj >= 4) ? piece : 0u);
+            const uint32_t vlo = __reduce_or_sync(full, (hv_grp && hj < 4) ? piece : 0u);
+            const uint32_t vhi = __reduce_or_sync(full, (hv_grp && hj >= 4) ? piece : 0u);
+            if (lane == Lm) om = make_uint2(mlo, mhi);
+            if (lane == Lv) ov = make_uint2(vlo, vhi);
+        }
 
-        // parameter update from the un-requantised fp32 moments
+        // ---- parameter update from the un-requantised fp32 moments
+        const f32x2 RS = splat2(P.rsqrt_bc2), EPS = splat2(P.eps), NSTEP = splat2(-P.step_m), ZERO = pack2(0.f, 0.f);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            t[j] = adaptive_apply(t[j], mf[j], vf[j], P.step_m, P);
-            chk = poison(chk, t[j]);
+        for (int p = 0; p < 4; ++p) {
+            float v0, v1, q0, q1;
+            unpack2(VF[p], v0, v1);
+            unpack2(fma2(pack2(sqrt_approx(v0), sqrt_approx(v1)), RS, EPS), q0, q1);
+            T[p] = fma2(mul2(NSTEP, MF[p]), pack2(rcp_approx(q0), rcp_approx(q1)), T[p]);
+            chk = fma2(T[p], ZERO, chk);
+            unpack2(T[p], t[2 * p], t[2 * p + 1]);
         }
 
         if (cnt == 8) {
@@ -581,7 +669,10 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         }
         if (lane == 0) { am[w0 / kQBlock] = am_new; av[w0 / kQBlock] = av_new; }
     }
-    return chk != 0.f;
+    cp_async_wait<0>();
+    float c0, c1;
+    unpack2(chk, c0, c1);
+    return (c0 != 0.f) | (c1 != 0.f);
 }
 
 __global__ void __launch_bounds__(kThreads, 3)
@@ -593,7 +684,7 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
     const CfgStep& P = SP.c[b->cfg];
     const uint16_t* g = static_cast<const uint16_t*>(grads[t.block]);
     float* th = params[t.block];
-    const int64_t base = int64_t(t.piece) * (b->path == kPathF ? kTileF : kTile);
+    const int64_t base = int64_t(t.piece) * (b->path == kPathF ? kTileF : (b->path == kPathA8 ? kTileQ : kTile));
     unsigned bad = 0;
     switch (b->path) {
         case kPathA32: bad = tile_dense<true, true>(b, P, g, th, base); break;
