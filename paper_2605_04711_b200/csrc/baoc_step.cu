@@ -68,17 +68,37 @@ __device__ __forceinline__ void rowcol_reduce_piece(const void* src, const float
     for (int l = 0; l < geo.L; ++l) {
         const int64_t r0 = row_begin + int64_t(l) * kRedRows;
         float rowacc[kRedRows / 4];
+        if (kSquare && vec && valid == 8 && th == nullptr) {
+            // common case: all 16 row segments of this thread are requested before the first one is used
+            const uint16_t* p = static_cast<const uint16_t*>(src) + col0;
+            uint4 w[kRedRows / 4];
 #pragma unroll
-        for (int k = 0; k < kRedRows / 4; ++k) {
-            const int64_t r = r0 + ty + 4 * k;
-            float s = 0.f;
-            if (r < rows && valid > 0) {
-                float x[8];
-                load8<kSquare>(src, th, wd, r * cols + col0, valid, vec, x);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) { s += x[j]; colacc[j] += x[j]; }
+            for (int k = 0; k < kRedRows / 4; ++k) {
+                const int64_t r = r0 + ty + 4 * k;
+                w[k] = r < rows ? ld_stream_u4(p + r * cols) : make_uint4(0u, 0u, 0u, 0u);
             }
-            rowacc[k] = s;
+#pragma unroll
+            for (int k = 0; k < kRedRows / 4; ++k) {
+                float x[8];
+                unpack8(w[k], x);
+                float s = 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { x[j] *= x[j]; s += x[j]; colacc[j] += x[j]; }
+                rowacc[k] = s;
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < kRedRows / 4; ++k) {
+                const int64_t r = r0 + ty + 4 * k;
+                float s = 0.f;
+                if (r < rows && valid > 0) {
+                    float x[8];
+                    load8<kSquare>(src, th, wd, r * cols + col0, valid, vec, x);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { s += x[j]; colacc[j] += x[j]; }
+                }
+                rowacc[k] = s;
+            }
         }
 #pragma unroll
         for (int k = 0; k < kRedRows / 4; ++k) sh_row[ty + 4 * k][tx] = rowacc[k];
