@@ -231,7 +231,13 @@ def run_ours(args):
     build.build()
     from paper_2605_04711_b200 import harness, workloads as W
 
-    wl = W.make_workload(args.workload, seed=rank)           # replicas: every rank streams its own copy of the workload
+    if args.shard_blocks and world > 1:
+        # strong scaling: whole blocks are dealt to the ranks (balanced by fp32-Adam step bytes); no collective is needed
+        wl = W.make_workload(args.workload, seed=0)
+        part = harness.partition_blocks([26.0 * b.numel for b in wl.blocks], world)[rank]
+        wl.blocks = [wl.blocks[i] for i in part]
+    else:
+        wl = W.make_workload(args.workload, seed=rank)       # replicas: every rank streams its own copy of the workload
     sess = harness.Session(wl, n_grad_sets=2, device=f"cuda:{local}", pinned_host_grads=True)
     sess.init_params()
     for t in (1, 2):
@@ -297,12 +303,11 @@ def run_ours(args):
     total_ms = marks[0].elapsed_time(marks[-1])
     stats_ms = sum(marks[2 * s].elapsed_time(marks[2 * s + 1]) for s in range(args.steps)) / args.steps
     step_ms = sum(marks[2 * s + 1].elapsed_time(marks[2 * s + 2]) for s in range(args.steps)) / args.steps
-    t_max = torch.tensor([total_ms], dtype=torch.float64, device=f"cuda:{local}")
-    if dist is not None:
-        dist.all_reduce(t_max, op=dist.ReduceOp.MAX)
-    total_ms_max = float(t_max.item())
+    dev = f"cuda:{local}"
+    total_ms_max = harness.max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms_max / args.steps
-    value = world * wl.numel / (ms_per_step * 1e-3)
+    all_params = harness.sum_over_ranks(wl.numel, dist, dev)      # parameters all ranks processed per step
+    value = all_params / (ms_per_step * 1e-3)
     cnt, _ = sess.h.nonfinite()
 
     # per-kernel split of the step (events inside the library around the fused kernel), on a few more steps
@@ -331,10 +336,7 @@ def run_ours(args):
     eb.record()
     torch.cuda.synchronize()
     e2e_ms = ea.elapsed_time(eb) / e2e_steps
-    t_e2e = torch.tensor([e2e_ms], dtype=torch.float64, device=f"cuda:{local}")
-    if dist is not None:
-        dist.all_reduce(t_e2e, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t_e2e.item())
+    e2e_ms = harness.max_over_ranks(e2e_ms, dist, dev)
     d2h = 8 * 8 * len(wl.blocks)
     h2d = 2 * wl.numel
 
@@ -365,18 +367,19 @@ def run_ours(args):
     roofline, other = (r_fused, r_stats) if fused_ms >= stats_ms else (r_stats, r_fused)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if (args.shard_blocks and world > 1) else "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "params": wl.numel, "blocks": len(wl.blocks), "grad_dtype": "bf16",
                    "param_dtype": "f32", "candidate_configs": CONFIG_NAMES, "assignment": args.assign,
                    "assignment_blocks_per_config": counts, "assignment_params_per_config": params_by_cfg,
                    "mem_budget_frac_of_fp32_adam": wl.mem_budget_frac, "state_bytes": int(info.state_bytes),
                    "window_steps_before_timing": args.window, "l2": "inputs (>10 GB per step) far exceed the 126 MB L2",
-                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                   "parallelism": (f"whole blocks sharded over {world} GPUs, no collective" if args.shard_blocks else
+                                   f"replicas x{world}, no collective") if world > 1 else "single GPU",
                    "allocator_status": int(rc), "nonfinite_blocks": int(cnt)},
         "clocks": sampler.summary(),
         "gpu_launches": int(launches),
-        "e2e": {"value": world * wl.numel / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+        "e2e": {"value": all_params / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                 "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps},
         "roofline": roofline,
         "roofline_other": other,
@@ -401,6 +404,8 @@ def main():
     ap.add_argument("--workload", default="llama_1b")
     ap.add_argument("--assign", default="auto", choices=["auto"] + CONFIG_NAMES,
                     help="auto: the library's own budgeted allocation; else every block under that one configuration")
+    ap.add_argument("--shard-blocks", action="store_true",
+                    help="N > 1: deal whole blocks of ONE workload to the ranks (strong scaling) instead of one replica per rank")
     ap.add_argument("--window", type=int, default=4, help="statistics steps before the finalize that feeds the allocation")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample-params", type=int, default=40_000_000)

@@ -15,6 +15,42 @@ from . import binding as B
 from . import workloads as W
 
 
+def partition_blocks(weights: Sequence[float], world: int) -> List[List[int]]:
+    """Whole blocks to ranks, no block split: longest-processing-time greedy on the given per-block weights
+    (bytes a step moves for the block, say).  Deterministic: ties go to the lower block index and the lower
+    rank.  Statistics are per-block sums and every update rule is local to its block, so ranks that own whole
+    blocks need no collective on the data path."""
+    if world < 1:
+        raise ValueError("world must be at least 1")
+    order = sorted(range(len(weights)), key=lambda i: (-float(weights[i]), i))
+    load = [0.0] * world
+    parts: List[List[int]] = [[] for _ in range(world)]
+    for i in order:
+        r = min(range(world), key=lambda k: (load[k], k))
+        parts[r].append(i)
+        load[r] += float(weights[i])
+    for p in parts:
+        p.sort()
+    return parts
+
+
+def max_over_ranks(value: float, dist=None, device="cpu") -> float:
+    """The slowest rank's value (device-timed milliseconds), as every rank sees it."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(value: float, dist=None, device="cpu") -> float:
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
 class Session:
     """One workload resident on one GPU.
 
