@@ -218,16 +218,19 @@ factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __r
 // m * rcp(sqrt(v) * rsqrt(bc2) + eps) with the approximate square root and
 // reciprocal (relative error 2^-23 each): the update is lr * direction, a
 // small fraction of the parameter, so the parameter keeps full fp32 accuracy,
-// and the moments themselves never pass through an approximation.
+// and the moments themselves never pass through an approximation.  Both are
+// the flush-to-zero forms, which are single instructions (the others wrap the
+// same unit in subnormal scaling: six instructions per square root): a second
+// moment below 1.2e-38 counts as 0 under the root, far below any eps in use.
 // ============================================================================
 __device__ __forceinline__ float sqrt_approx(float x) {
     float r;
-    asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
     return r;
 }
 __device__ __forceinline__ float rcp_approx(float x) {
     float r;
-    asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
     return r;
 }
 
@@ -518,57 +521,76 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
     const bool coupled = P.coupled != 0;
     f32x2 chk = pack2(0.f, 0.f);
 
-    // Slices are prefetched one ahead through shared memory: every thread copies the 64 bytes of its own next
+    // Slices are prefetched two ahead through shared memory: every thread copies the 64 bytes of its own next
     // eight elements (gradient, parameters, both code words) into its own slot with cp.async and reads them back
     // itself, so no registers are held across the long arithmetic of the current slice and no barrier is needed.
+    // All indexing inside the tile is 32-bit and relative to the tile's first element.
     constexpr int kSlicesQ = kTileQ / (kThreads * 8);
-    __shared__ __align__(16) unsigned char stage[2][kThreads * 64];
-    auto slot = [&](int st, int off) { return &stage[st][0] + off; };   // off: 0 g (16 B/thread), 4096 theta (32), 12288 m codes (8), 14336 v codes (8)
+    constexpr int kStagesQ = 3;                                      // two slices in flight while one is consumed
+    constexpr int kStageBytes = kThreads * 64;                       // g 16 B/thread at 0, theta 32 at 4096, m codes 8 at 12288, v codes 8 at 14336
+    __shared__ __align__(16) unsigned char stage[kStagesQ * kStageBytes];
+    const int left = int(min64(numel - base, kTileQ));              // elements of the block in this tile (>= 1)
+    const uint16_t* __restrict__ gt = g + base;
+    float* __restrict__ tht = th + base;
+    int8_t* __restrict__ qmt = qm + base;
+    uint8_t* __restrict__ qvt = qv + base;
+    float* __restrict__ amt = am + base / kQBlock;                   // base is a multiple of the quantisation block
+    float* __restrict__ avt = av + base / kQBlock;
+    const int toff = threadIdx.x * 8;                                // this thread's first element within a slice
+    const uint32_t sm0 = smem_addr(stage);
+    const uint32_t sg = threadIdx.x * 16, st_ = 4096 + threadIdx.x * 32, scm = 12288 + threadIdx.x * 8, scv = 14336 + threadIdx.x * 8;
+    uint32_t fill = 0;                                               // byte offset of the stage the next prefetch fills
     auto prefetch = [&](int s) {
-        const int64_t w0 = base + int64_t(s) * (kThreads * 8) + int64_t(warp) * kQBlock;
-        const int64_t e = w0 + lane * 8;
-        if (s < kSlicesQ && e + 8 <= numel) {                      // ragged or absent elements are loaded directly later
-            const int st = s & 1;
-            cp_async16(smem_addr(slot(st, threadIdx.x * 16)), g + e);
-            cp_async16(smem_addr(slot(st, 4096 + threadIdx.x * 32)), th + e);
-            cp_async16(smem_addr(slot(st, 4096 + threadIdx.x * 32 + 16)), th + e + 4);
-            cp_async8(smem_addr(slot(st, 12288 + threadIdx.x * 8)), qm + e);
-            cp_async8(smem_addr(slot(st, 14336 + threadIdx.x * 8)), qv + e);
+        const int e = s * (kThreads * 8) + toff;
+        if (s < kSlicesQ && e + 8 <= left) {                        // ragged or absent elements are loaded directly later
+            const uint32_t d = sm0 + fill;
+            cp_async16(d + sg, gt + e);
+            cp_async16(d + st_, tht + e);
+            cp_async16(d + st_ + 16, tht + e + 4);
+            cp_async8(d + scm, qmt + e);
+            cp_async8(d + scv, qvt + e);
         }
         cp_async_commit();
+        fill = fill == (kStagesQ - 1) * kStageBytes ? 0u : fill + kStageBytes;
     };
-    prefetch(0);
-    float amo_next = 0.f, avo_next = 0.f;
-    if (base + int64_t(warp) * kQBlock < numel) { amo_next = am[(base + int64_t(warp) * kQBlock) / kQBlock]; avo_next = av[(base + int64_t(warp) * kQBlock) / kQBlock]; }
+    // the old absmax pair of a slice travels in registers, the same distance ahead
+    auto absmax_of = [&](int s, float& a_m, float& a_v) {
+        const int w = s * (kThreads * 8) + warp * kQBlock;
+        a_m = 0.f; a_v = 0.f;
+        if (s < kSlicesQ && w < left) { a_m = amt[w / kQBlock]; a_v = avt[w / kQBlock]; }
+    };
+    float amo_1, avo_1, amo_2, avo_2;
+    prefetch(0); prefetch(1);
+    absmax_of(0, amo_1, avo_1); absmax_of(1, amo_2, avo_2);
+    uint32_t take = 0;                                               // byte offset of the stage the current slice sits in
 #pragma unroll 1
     for (int s = 0; s < kSlicesQ; ++s) {
-        const int64_t w0 = base + int64_t(s) * (kThreads * 8) + int64_t(warp) * kQBlock;
-        prefetch(s + 1);
-        const float amo = amo_next, avo = avo_next;
-        {
-            const int64_t w1 = w0 + int64_t(kThreads) * 8;
-            if (s + 1 < kSlicesQ && w1 < numel) { amo_next = am[w1 / kQBlock]; avo_next = av[w1 / kQBlock]; }
-        }
-        cp_async_wait<1>();                                         // this slice's copies have landed (the next one's may be in flight)
-        if (w0 >= numel) break;                                     // whole warp out of range (and so are the later slices)
-        const int64_t e = w0 + lane * 8;
-        const int cnt = int(max64(0, min64(8, numel - e)));
+        const int w0 = s * (kThreads * 8) + warp * kQBlock;
+        prefetch(s + 2);
+        const float amo = amo_1, avo = avo_1;
+        amo_1 = amo_2; avo_1 = avo_2;
+        absmax_of(s + 2, amo_2, avo_2);
+        cp_async_wait<2>();                                         // this slice's copies have landed (the next two may be in flight)
+        if (w0 >= left) break;                                      // whole warp out of range (and so are the later slices)
+        const int e = w0 + lane * 8;
+        const int cnt = max(0, min(8, left - e));
+        const unsigned char* mine = stage + take;
+        take = take == (kStagesQ - 1) * kStageBytes ? 0u : take + kStageBytes;
         uint4 wg;
         float4 t0, t1;
         uint2 wm, wv;
         if (cnt == 8) {
-            const int st = s & 1;
-            wg = *reinterpret_cast<const uint4*>(slot(st, threadIdx.x * 16));
-            t0 = *reinterpret_cast<const float4*>(slot(st, 4096 + threadIdx.x * 32));
-            t1 = *reinterpret_cast<const float4*>(slot(st, 4096 + threadIdx.x * 32 + 16));
-            wm = *reinterpret_cast<const uint2*>(slot(st, 12288 + threadIdx.x * 8));
-            wv = *reinterpret_cast<const uint2*>(slot(st, 14336 + threadIdx.x * 8));
+            wg = *reinterpret_cast<const uint4*>(mine + sg);
+            t0 = *reinterpret_cast<const float4*>(mine + st_);
+            t1 = *reinterpret_cast<const float4*>(mine + st_ + 16);
+            wm = *reinterpret_cast<const uint2*>(mine + scm);
+            wv = *reinterpret_cast<const uint2*>(mine + scv);
         } else {                                                    // ragged end of the block: zero-fill
             const int n = cnt;
-            auto gg = [&](int j) { return j < n ? uint32_t(g[e + j]) : 0u; };
-            auto tt = [&](int j) { return j < n ? th[e + j] : 0.f; };
-            auto mm = [&](int j) { return j < n ? uint32_t(uint8_t(qm[e + j])) : 0u; };
-            auto vv = [&](int j) { return j < n ? uint32_t(qv[e + j]) : 0u; };
+            auto gg = [&](int j) { return j < n ? uint32_t(gt[e + j]) : 0u; };
+            auto tt = [&](int j) { return j < n ? tht[e + j] : 0.f; };
+            auto mm = [&](int j) { return j < n ? uint32_t(uint8_t(qmt[e + j])) : 0u; };
+            auto vv = [&](int j) { return j < n ? uint32_t(qvt[e + j]) : 0u; };
             wg = make_uint4(gg(0) | gg(1) << 16, gg(2) | gg(3) << 16, gg(4) | gg(5) << 16, gg(6) | gg(7) << 16);
             t0 = make_float4(tt(0), tt(1), tt(2), tt(3)); t1 = make_float4(tt(4), tt(5), tt(6), tt(7));
             wm = make_uint2(mm(0) | mm(1) << 8 | mm(2) << 16 | mm(3) << 24, mm(4) | mm(5) << 8 | mm(6) << 16 | mm(7) << 24);
@@ -674,20 +696,20 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         }
 
         if (cnt == 8) {
-            st8(th + e, t);
-            st_stream_u2(qm + e, om);
-            st_stream_u2(qv + e, ov);
+            st8(tht + e, t);
+            st_stream_u2(qmt + e, om);
+            st_stream_u2(qvt + e, ov);
         } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {                          // static indices keep t[] in registers
                 if (j < cnt) {
-                    th[e + j] = t[j];
-                    qm[e + j] = int8_t(((j < 4 ? om.x : om.y) >> (8 * (j & 3))) & 0xffu);
-                    qv[e + j] = uint8_t(((j < 4 ? ov.x : ov.y) >> (8 * (j & 3))) & 0xffu);
+                    tht[e + j] = t[j];
+                    qmt[e + j] = int8_t(((j < 4 ? om.x : om.y) >> (8 * (j & 3))) & 0xffu);
+                    qvt[e + j] = uint8_t(((j < 4 ? ov.x : ov.y) >> (8 * (j & 3))) & 0xffu);
                 }
             }
         }
-        if (lane == 0) { am[w0 / kQBlock] = am_new; av[w0 / kQBlock] = av_new; }
+        if (lane == 0) { amt[w0 / kQBlock] = am_new; avt[w0 / kQBlock] = av_new; }
     }
     cp_async_wait<0>();
     float c0, c1;
