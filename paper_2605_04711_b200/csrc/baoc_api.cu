@@ -79,6 +79,8 @@ void fill_step_params(const Handle* h, int64_t t, StepParams* P) {
         o.step_m = float(lr / bc1);
         o.step_g = k.lr;
         o.rsqrt_bc2 = float(1.0 / std::sqrt(bc2));
+        o.step_m_hat = float(lr / bc1 * std::sqrt(bc2));
+        o.eps_hat = float(double(k.eps) * std::sqrt(bc2));
         o.beta1_d = b1; o.beta2_d = b2; o.wd_d = double(k.weight_decay);
     }
 }

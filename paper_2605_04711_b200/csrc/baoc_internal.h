@@ -118,6 +118,8 @@ struct CfgStep {
     float step_m;        // lr / (1 - beta1^t): multiplies a bias-corrected first moment
     float step_g;        // lr: multiplies a raw gradient or momentum buffer
     float rsqrt_bc2;     // 1 / sqrt(1 - beta2^t)
+    float step_m_hat;    // step_m * sqrt(1 - beta2^t): with eps_hat the update is step_m_hat * m / (sqrt(v) + eps_hat)
+    float eps_hat;       // eps * sqrt(1 - beta2^t)
     int32_t coupled;     // 1: add wd*theta to the gradient
     int32_t pad;
     double beta1_d, beta2_d;   // the coefficients widened, for the exact side of the 8-bit path

@@ -456,8 +456,9 @@ struct Q8Raw {
     float theta;         // parameter of element j before the update (coupled decay only)
 };
 
+template <bool kCoupled>
 __device__ __forceinline__ Q8Raw q8_fetch(int src, int j, const uint4& wg, const uint2& wm, const uint2& wv,
-                                          const float (&t)[8], bool coupled) {
+                                          const float4& t0, const float4& t1) {
     const unsigned full = 0xffffffffu;
     const uint32_t gx = __shfl_sync(full, wg.x, src), gy = __shfl_sync(full, wg.y, src);
     const uint32_t gz = __shfl_sync(full, wg.z, src), gw = __shfl_sync(full, wg.w, src);
@@ -469,21 +470,22 @@ __device__ __forceinline__ Q8Raw q8_fetch(int src, int j, const uint4& wg, const
     r.cm = (((j & 4) ? my : mx) >> (8 * (j & 3))) & 0xffu;
     r.cv = (((j & 4) ? vy : vx) >> (8 * (j & 3))) & 0xffu;
     r.theta = 0.f;
-    if (coupled) {                                                  // uniform branch
-        float tt[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) tt[k] = __shfl_sync(full, t[k], src);
-        const float a = (j & 1) ? tt[1] : tt[0], b = (j & 1) ? tt[3] : tt[2];
-        const float c = (j & 1) ? tt[5] : tt[4], d = (j & 1) ? tt[7] : tt[6];
+    if (kCoupled) {                                                 // the select uses the asking lane's j, so it follows the shuffles
+        const float x0 = __shfl_sync(full, t0.x, src), x1 = __shfl_sync(full, t0.y, src);
+        const float x2 = __shfl_sync(full, t0.z, src), x3 = __shfl_sync(full, t0.w, src);
+        const float x4 = __shfl_sync(full, t1.x, src), x5 = __shfl_sync(full, t1.y, src);
+        const float x6 = __shfl_sync(full, t1.z, src), x7 = __shfl_sync(full, t1.w, src);
+        const float a = (j & 1) ? x1 : x0, b = (j & 1) ? x3 : x2, c = (j & 1) ? x5 : x4, d = (j & 1) ? x7 : x6;
         r.theta = (j & 4) ? ((j & 2) ? d : c) : ((j & 2) ? b : a);
     }
     return r;
 }
 
 // Exact (double) new moment of one element: first moment for group 0, second for group 1.
+template <bool kCoupled>
 __device__ __forceinline__ double q8_exact(const Q8Raw& r, bool second, float am_old, float av_old, const CfgStep& P) {
     double gd = widen_bf16_float(__uint_as_float(r.gbits << 16));
-    if (P.coupled) gd += P.wd_d * double(r.theta);
+    if (kCoupled) gd += P.wd_d * double(r.theta);
     const double beta = second ? P.beta2_d : P.beta1_d;
     const int code = second ? int(r.cv) : int(int8_t(r.cm));
     const double old = int_to_double(code) * (second ? double(av_old) * (1.0 / 255.0) : double(am_old) * (1.0 / 127.0));
@@ -505,8 +507,13 @@ __device__ __forceinline__ float warp_max_nonneg(float x) {
     return __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(x)));
 }
 
+constexpr int kSlicesQ = kTileQ / (kThreads * 8);
+constexpr int kStagesQ = 3;                                          // two slices in flight while one is consumed
+constexpr int kStageBytes = kThreads * 64;                           // g 16 B/thread at 0, theta 32 at 4096, m codes 8 at 12288, v codes 8 at 14336
+
+template <bool kCoupled>
 __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep& P, const uint16_t* __restrict__ g,
-                                              float* __restrict__ th, int64_t base) {
+                                              float* __restrict__ th, int64_t base, unsigned char* stage) {
     constexpr float kSlack = 4.76837158203125e-7f;                 // 2^-21
     constexpr float kMagic = 12582912.0f;                          // 1.5 * 2^23: adding it rounds to an integer, ties to even
     const unsigned full = 0xffffffffu;
@@ -518,17 +525,12 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int hj = lane & 7;                                        // element handled when helping another lane
     const bool hv_grp = (lane & 8) != 0, helper = lane < 16;       // lanes 0-7: first moment, 8-15: second moment
-    const bool coupled = P.coupled != 0;
     f32x2 chk = pack2(0.f, 0.f);
 
     // Slices are prefetched two ahead through shared memory: every thread copies the 64 bytes of its own next
     // eight elements (gradient, parameters, both code words) into its own slot with cp.async and reads them back
     // itself, so no registers are held across the long arithmetic of the current slice and no barrier is needed.
     // All indexing inside the tile is 32-bit and relative to the tile's first element.
-    constexpr int kSlicesQ = kTileQ / (kThreads * 8);
-    constexpr int kStagesQ = 3;                                      // two slices in flight while one is consumed
-    constexpr int kStageBytes = kThreads * 64;                       // g 16 B/thread at 0, theta 32 at 4096, m codes 8 at 12288, v codes 8 at 14336
-    __shared__ __align__(16) unsigned char stage[kStagesQ * kStageBytes];
     const int left = int(min64(numel - base, kTileQ));              // elements of the block in this tile (>= 1)
     const uint16_t* __restrict__ gt = g + base;
     float* __restrict__ tht = th + base;
@@ -596,8 +598,7 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
             wm = make_uint2(mm(0) | mm(1) << 8 | mm(2) << 16 | mm(3) << 24, mm(4) | mm(5) << 8 | mm(6) << 16 | mm(7) << 24);
             wv = make_uint2(vv(0) | vv(1) << 8 | vv(2) << 16 | vv(3) << 24, vv(4) | vv(5) << 8 | vv(6) << 16 | vv(7) << 24);
         }
-        float t[8];                                                 // parameters before the update (kept for the coupled exact side)
-        f4_to(t0, t1, t);
+        // t0, t1 keep the parameters before the update: the coupled exact side needs them
 
         // ---- fp32 pass, two elements per instruction: effective gradient, decayed parameter, new moments
         // A code byte c becomes the float 2^23 + c by placing it in the low mantissa
@@ -613,8 +614,8 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
             f32x2 X = pack2(bf16_lo(gw[p]), bf16_hi(gw[p]));
-            T[p] = pack2(t[2 * p], t[2 * p + 1]);
-            if (coupled) X = fma2(splat2(P.wd), T[p], X);
+            T[p] = p == 0 ? pack2(t0.x, t0.y) : (p == 1 ? pack2(t0.z, t0.w) : (p == 2 ? pack2(t1.x, t1.y) : pack2(t1.z, t1.w)));
+            if (kCoupled) X = fma2(splat2(P.wd), T[p], X);
             else T[p] = fma2(splat2(P.decay), T[p], T[p]);
             const uint32_t mw = ms[p >> 1], vw = vs[p >> 1];
             const int k0 = (2 * p) & 3, k1 = (2 * p + 1) & 3;
@@ -638,8 +639,8 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
             const int Lm = cand_m ? __ffs(cand_m) - 1 : -1, Lv = cand_v ? __ffs(cand_v) - 1 : -1;
             cand_m &= cand_m - 1u; cand_v &= cand_v - 1u;           // (0 & anything stays 0)
             const int src = hv_grp ? Lv : Lm;
-            const Q8Raw r = q8_fetch(max(src, 0), hj, wg, wm, wv, t, coupled);
-            const float val = __double2float_rn(fabs(q8_exact(r, hv_grp, amo, avo, P)));
+            const Q8Raw r = q8_fetch<kCoupled>(max(src, 0), hj, wg, wm, wv, t0, t1);
+            const float val = __double2float_rn(fabs(q8_exact<kCoupled>(r, hv_grp, amo, avo, P)));
             if (helper && src >= 0) {
                 if (hv_grp) av_c = fmaxf(av_c, val); else am_c = fmaxf(am_c, val);
             }
@@ -671,8 +672,8 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
             const int Lm = slow_m ? __ffs(slow_m) - 1 : -1, Lv = slow_v ? __ffs(slow_v) - 1 : -1;
             slow_m &= slow_m - 1u; slow_v &= slow_v - 1u;
             const int src = hv_grp ? Lv : Lm;
-            const Q8Raw r = q8_fetch(max(src, 0), hj, wg, wm, wv, t, coupled);
-            const double x = q8_exact(r, hv_grp, amo, avo, P);
+            const Q8Raw r = q8_fetch<kCoupled>(max(src, 0), hj, wg, wm, wv, t0, t1);
+            const double x = q8_exact<kCoupled>(r, hv_grp, amo, avo, P);
             const int code = hv_grp ? encode_exact(x, av_new, 255.0, 0) : encode_exact(x, am_new, 127.0, -127);
             const uint32_t piece = (helper && src >= 0) ? (uint32_t(code) & 0xffu) << (8 * (hj & 3)) : 0u;
             const uint32_t mlo = __reduce_or_sync(full, (!hv_grp && hj < 4) ? piece : 0u);
@@ -684,14 +685,16 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         }
 
         // ---- parameter update from the un-requantised fp32 moments
-        const f32x2 RS = splat2(P.rsqrt_bc2), EPS = splat2(P.eps), NSTEP = splat2(-P.step_m), ZERO = pack2(0.f, 0.f);
+        // theta <- theta - step_m_hat * m / (sqrt(v) + eps_hat), the bias correction of v folded into both constants
+        const f32x2 EPS = splat2(P.eps_hat), NSTEP = splat2(-P.step_m_hat);
+        float t[8];
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
             float v0, v1, q0, q1;
             unpack2(VF[p], v0, v1);
-            unpack2(fma2(pack2(sqrt_approx(v0), sqrt_approx(v1)), RS, EPS), q0, q1);
+            unpack2(add2(pack2(sqrt_approx(v0), sqrt_approx(v1)), EPS), q0, q1);
             T[p] = fma2(mul2(NSTEP, MF[p]), pack2(rcp_approx(q0), rcp_approx(q1)), T[p]);
-            chk = fma2(T[p], ZERO, chk);
+            chk = add2(chk, T[p]);                                  // a non-finite parameter makes the sum non-finite
             unpack2(T[p], t[2 * p], t[2 * p + 1]);
         }
 
@@ -714,7 +717,7 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
     cp_async_wait<0>();
     float c0, c1;
     unpack2(chk, c0, c1);
-    return (c0 != 0.f) | (c1 != 0.f);
+    return !isfinite(c0) | !isfinite(c1);
 }
 
 __global__ void __launch_bounds__(kThreads, 3)
@@ -727,12 +730,13 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
     const uint16_t* g = static_cast<const uint16_t*>(grads[t.block]);
     float* th = params[t.block];
     const int64_t base = int64_t(t.piece) * (b->path == kPathF ? kTileF : (b->path == kPathA8 ? kTileQ : kTile));
+    __shared__ __align__(16) unsigned char q_stage[kStagesQ * kStageBytes];   // per-thread staging of the 8-bit path
     unsigned bad = 0;
     switch (b->path) {
         case kPathA32: bad = tile_dense<true, true>(b, P, g, th, base); break;
         case kPathR: bad = tile_dense<false, true>(b, P, g, th, base); break;
         case kPathS: bad = tile_dense<true, false>(b, P, g, th, base); break;
-        case kPathA8: bad = tile_int8(b, P, g, th, base); break;
+        case kPathA8: bad = P.coupled ? tile_int8<true>(b, P, g, th, base, q_stage) : tile_int8<false>(b, P, g, th, base, q_stage); break;
         case kPathF: bad = tile_factored(b, P, g, th, base); break;
         default: break;
     }
