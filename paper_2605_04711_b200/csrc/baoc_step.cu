@@ -562,17 +562,18 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         if (s < kSlicesQ && w < left) { a_m = amt[w / kQBlock]; a_v = avt[w / kQBlock]; }
     };
     float amo_1, avo_1, amo_2, avo_2;
-    prefetch(0); prefetch(1);
+#pragma unroll
+    for (int k = 0; k < kStagesQ - 1; ++k) prefetch(k);
     absmax_of(0, amo_1, avo_1); absmax_of(1, amo_2, avo_2);
     uint32_t take = 0;                                               // byte offset of the stage the current slice sits in
 #pragma unroll 1
     for (int s = 0; s < kSlicesQ; ++s) {
         const int w0 = s * (kThreads * 8) + warp * kQBlock;
-        prefetch(s + 2);
+        prefetch(s + kStagesQ - 1);
         const float amo = amo_1, avo = avo_1;
         amo_1 = amo_2; avo_1 = avo_2;
         absmax_of(s + 2, amo_2, avo_2);
-        cp_async_wait<2>();                                         // this slice's copies have landed (the next two may be in flight)
+        cp_async_wait<kStagesQ - 1>();                              // this slice's copies have landed (the later ones may be in flight)
         if (w0 >= left) break;                                      // whole warp out of range (and so are the later slices)
         const int e = w0 + lane * 8;
         const int cnt = max(0, min(8, left - e));
