@@ -26,7 +26,7 @@ constexpr int kRanks = 4;             // order statistics per block for the two 
 constexpr int kFinOut = 32;           // doubles per block copied to the host at the end of the window
 constexpr int kRedRows = 64;          // rows per CTA of the row/column reduction kernel
 constexpr int kRedCols = 512;         // columns per CTA of the row/column reduction kernel
-constexpr int kTileF = 8192;          // elements per tile of the factored path (10 bytes per element: more elements keep as many bytes in flight)
+constexpr int kTileF = 16384;         // elements per tile of the factored path (its slices are prefetched through shared memory)
 constexpr int kTileQ = 16384;         // elements per tile of the 8-bit path (its slices are prefetched through shared memory)
 constexpr int kCombineSlabs = 32;     // CTAs per factored block of the row/column combine
 

@@ -281,6 +281,9 @@ __device__ __forceinline__ float poison(float acc, float x) { return fmaf(x, 0.0
 
 constexpr int kSlices = kTile / (kThreads * 8);
 constexpr int kSlicesF = kTileF / (kThreads * 8);
+constexpr int kSlicesQ = kTileQ / (kThreads * 8);
+constexpr int kStagesQ = 3;                                          // two slices in flight while one is consumed
+constexpr int kStageBytes = kThreads * 64;                           // g 16 B/thread at 0, theta 32 at 4096, m codes 8 at 12288, v codes 8 at 14336
 
 // fp32 Adam / RMS / SGD-momentum: kM = has first moment, kV = has second moment.
 template <bool kM, bool kV>
@@ -348,7 +351,7 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
 // statistic and two 128-bit loads of column statistics (which stay in L1/L2:
 // every row of the tile re-reads them).
 __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgStep& P, const uint16_t* __restrict__ g,
-                                                  float* __restrict__ th, int64_t base) {
+                                                  float* __restrict__ th, int64_t base, unsigned char* stage) {
     const int64_t numel = b->numel;
     const int cols = b->cols;
     const float* __restrict__ r = static_cast<const float*>(b->s0);
@@ -357,44 +360,60 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
     const float inv_rm = rm > 0.f ? 1.0f / rm : 0.f;
     float chk = 0.f;
     if ((cols & 7) == 0) {
+        // Streaming form: each thread copies the 48 bytes of its own next eight elements (gradient, parameters)
+        // into its own shared-memory slot three slices ahead with cp.async and reads them back itself: no
+        // registers are held by loads in flight and no barrier is needed.
+        constexpr int kStagesF = 4;
+        constexpr int kStageBytesF = kThreads * 48;                   // g 16 B/thread at 0, theta 32 B/thread at 4096
+        static_assert(kStagesF * kStageBytesF <= kStagesQ * kStageBytes, "the factored ring must fit the shared staging buffer");
         const int64_t row0 = base / cols;
         const uint32_t col0 = uint32_t(base - row0 * cols);
-        uint4 wg[kSlicesF];
-        float4 t0[kSlicesF], t1[kSlicesF];
-        float ri[kSlicesF];
-        uint32_t cl[kSlicesF];
-        bool in[kSlicesF];
-#pragma unroll
-        for (int s = 0; s < kSlicesF; ++s) {
-            const uint32_t off = uint32_t(s) * (kThreads * 8) + threadIdx.x * 8;
-            const int64_t e = base + off;
-            in[s] = e < numel;                        // numel is a multiple of 8 here
-            if (in[s]) {
-                const uint32_t cc = col0 + off;       // < cols + kTileF
-                const uint32_t q = cc / uint32_t(cols);
-                const uint32_t col = cc - q * uint32_t(cols);
-                wg[s] = ld_stream_u4(g + e);
-                t0[s] = ld_stream_f4(th + e); t1[s] = ld_stream_f4(th + e + 4);
-                cl[s] = col;
-                ri[s] = __ldg(r + row0 + q);
+        const int left = int(min64(numel - base, kTileF));          // a multiple of 8 here
+        const uint16_t* __restrict__ gt = g + base;
+        float* __restrict__ tht = th + base;
+        const float* __restrict__ rt = r + row0;
+        const int toff = threadIdx.x * 8;
+        const uint32_t sm0 = smem_addr(stage), sg = threadIdx.x * 16, st_ = 4096 + threadIdx.x * 32;
+        uint32_t fill = 0, take = 0;
+        auto prefetch = [&](int s) {
+            const int e = s * (kThreads * 8) + toff;
+            if (s < kSlicesF && e < left) {
+                const uint32_t d = sm0 + fill;
+                cp_async16(d + sg, gt + e);
+                cp_async16(d + st_, tht + e);
+                cp_async16(d + st_ + 16, tht + e + 4);
             }
-        }
+            cp_async_commit();
+            fill = fill == (kStagesF - 1) * kStageBytesF ? 0u : fill + kStageBytesF;
+        };
 #pragma unroll
+        for (int k = 0; k < kStagesF - 1; ++k) prefetch(k);
+#pragma unroll 1
         for (int s = 0; s < kSlicesF; ++s) {
-            if (!in[s]) continue;
-            const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
-            float x[8], t[8], cj[8];
-            unpack8(wg[s], x); f4_to(t0[s], t1[s], t);
-            f4_to(__ldg(reinterpret_cast<const float4*>(c + cl[s])), __ldg(reinterpret_cast<const float4*>(c + cl[s] + 4)), cj);
-            const float rs = ri[s] * inv_rm;
+            prefetch(s + kStagesF - 1);
+            const int e = s * (kThreads * 8) + toff;
+            if (e >= left) break;                                   // later slices are out of range too
+            const uint32_t cc = col0 + uint32_t(e);                 // < cols + kTileF
+            const uint32_t q = cc / uint32_t(cols);
+            const uint32_t col = cc - q * uint32_t(cols);
+            float cj[8];
+            f4_to(__ldg(reinterpret_cast<const float4*>(c + col)), __ldg(reinterpret_cast<const float4*>(c + col + 4)), cj);
+            const float rs = __ldg(rt + q) * inv_rm;
+            cp_async_wait<kStagesF - 1>();                          // this slice's copies have landed
+            const unsigned char* mine = stage + take;
+            take = take == (kStagesF - 1) * kStageBytesF ? 0u : take + kStageBytesF;
+            float x[8], t[8];
+            unpack8(*reinterpret_cast<const uint4*>(mine + sg), x);
+            f4_to(*reinterpret_cast<const float4*>(mine + st_), *reinterpret_cast<const float4*>(mine + st_ + 16), t);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 prologue(x[j], t[j], P);
                 t[j] = adaptive_apply(t[j], x[j], rs * cj[j], P.step_g, P);
                 chk = poison(chk, t[j]);
             }
-            st8(th + e, t);
+            st8(tht + e, t);
         }
+        cp_async_wait<0>();
         return chk != 0.f;
     }
     // any other row length: walk the row/column position element by element
@@ -506,10 +525,6 @@ __device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint3
 __device__ __forceinline__ float warp_max_nonneg(float x) {
     return __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(x)));
 }
-
-constexpr int kSlicesQ = kTileQ / (kThreads * 8);
-constexpr int kStagesQ = 3;                                          // two slices in flight while one is consumed
-constexpr int kStageBytes = kThreads * 64;                           // g 16 B/thread at 0, theta 32 at 4096, m codes 8 at 12288, v codes 8 at 14336
 
 template <bool kCoupled>
 __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep& P, const uint16_t* __restrict__ g,
@@ -731,14 +746,14 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
     const uint16_t* g = static_cast<const uint16_t*>(grads[t.block]);
     float* th = params[t.block];
     const int64_t base = int64_t(t.piece) * (b->path == kPathF ? kTileF : (b->path == kPathA8 ? kTileQ : kTile));
-    __shared__ __align__(16) unsigned char q_stage[kStagesQ * kStageBytes];   // per-thread staging of the 8-bit path
+    __shared__ __align__(16) unsigned char q_stage[kStagesQ * kStageBytes];   // per-thread staging of the 8-bit and factored paths
     unsigned bad = 0;
     switch (b->path) {
         case kPathA32: bad = tile_dense<true, true>(b, P, g, th, base); break;
         case kPathR: bad = tile_dense<false, true>(b, P, g, th, base); break;
         case kPathS: bad = tile_dense<true, false>(b, P, g, th, base); break;
         case kPathA8: bad = P.coupled ? tile_int8<true>(b, P, g, th, base, q_stage) : tile_int8<false>(b, P, g, th, base, q_stage); break;
-        case kPathF: bad = tile_factored(b, P, g, th, base); break;
+        case kPathF: bad = tile_factored(b, P, g, th, base, q_stage); break;
         default: break;
     }
     if (bad) atomicOr(flags + t.block, 1u);

@@ -148,9 +148,9 @@ def _gpt2_small_blocks() -> List[Block]:
     return out
 
 
-def _llama_1b_blocks() -> List[Block]:
-    d, ff, layers, vocab = 2048, 8192, 16, 32000
-    out = [_mat("tok_emb", vocab, d)]
+def _llama_1b_blocks(layers: int = 16, with_table: bool = True) -> List[Block]:
+    d, ff, vocab = 2048, 8192, 32000
+    out = [_mat("tok_emb", vocab, d)] if with_table else []
     for l in range(layers):
         p = f"l{l}"
         out += [_vec(p + ".norm1", d)]
@@ -237,7 +237,7 @@ def _level_of(name: str) -> int:
 
 
 def make_workload(name: str, seed: int = 0) -> Workload:
-    """Build one of: toy, resnet50, gpt2_small, unet, llama_1b."""
+    """Build one of: toy, resnet50, gpt2_small, unet, llama_1b (and llama_2l, a two-layer cut of it for profiling)."""
     if name == "toy":
         wl = Workload(name, _toy_blocks(), window=8, mem_budget_frac=0.50, time_budget=1.3, seed=seed)
     elif name == "resnet50":
@@ -248,6 +248,10 @@ def make_workload(name: str, seed: int = 0) -> Workload:
         wl = Workload(name, _unet_blocks(), window=32, mem_budget_frac=0.30, time_budget=1.05, seed=seed)
     elif name == "llama_1b":
         wl = Workload(name, _llama_1b_blocks(), window=64, mem_budget_frac=0.25, time_budget=1.3, seed=seed)
+    elif name == "llama_2l":
+        # two layers of the LLaMA-1B shape without the token table (121.6 M parameters): same matrix shapes as the
+        # full workload at a size small enough for multi-pass profiler captures
+        wl = Workload(name, _llama_1b_blocks(2, False), window=64, mem_budget_frac=0.25, time_budget=1.3, seed=seed)
     else:
         raise ValueError(f"unknown workload {name!r}")
 
@@ -255,7 +259,7 @@ def make_workload(name: str, seed: int = 0) -> Workload:
     gen = torch.Generator().manual_seed(stream_seed(seed, 1 << 19, 7))
     u = torch.rand((len(wl.blocks), 3), generator=gen, dtype=torch.float64)
     for i, b in enumerate(wl.blocks):
-        lo, hi = (0.05, 0.95) if name == "llama_1b" else (0.0, 1.0)
+        lo, hi = (0.05, 0.95) if name.startswith("llama") else (0.0, 1.0)
         b.stability = float(lo + (hi - lo) * u[i, 0])
         b.tau = float(2.0 * u[i, 1])
         b.scale = float(10.0 ** (-3.0 + 2.0 * u[i, 2]))
