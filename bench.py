@@ -43,6 +43,27 @@ def _peaks():
     return 6650.0, "fallback"
 
 
+def _ncu_traffic(kernel, algorithmic_bytes):
+    """DRAM bytes per launch of `kernel`, scaled from the recorded ncu capture of a smaller case by the algorithmic
+    bytes of this launch (traffic is proportional to the parameters processed).  None when there is no record or
+    the kernel sources have changed since the counters were taken."""
+    import glob
+    import hashlib
+    pkg = os.path.join(ROOT, "paper_2605_04711_b200")
+    try:
+        rec = json.load(open(os.path.join(pkg, "ncu_traffic.json")))
+        h = hashlib.sha256()
+        for f in sorted(glob.glob(os.path.join(pkg, "csrc", "*"))):
+            h.update(os.path.basename(f).encode())
+            h.update(open(f, "rb").read())
+        if h.hexdigest() != rec["csrc_sha256"] or kernel not in rec:
+            return None
+        k = rec[kernel]
+        return float(k["dram_bytes"]) / float(k["algorithmic_bytes"]) * float(algorithmic_bytes)
+    except Exception:
+        return None
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clocks and clock-event (throttle) reasons while the timed region runs: NVML in-process every
     10 ms where the module loads, else the nvidia-smi query every 200 ms.  Read-only."""
@@ -356,14 +377,14 @@ def run_ours(args):
                "frac": stats_gbs / peak, "peak_kind": peak_kind + " (burst copy)", "frac_of_8TBs": stats_gbs / 8000.0,
                "bytes_per_launch": int(stats_bytes), "ms": stats_ms, "bytes_per_param": 22,
                "timed": "events around baoc_sample_stats (includes its ~25 us combine kernel)",
-               "traffic": args.traffic_stats}
+               "traffic": args.traffic_stats if args.traffic_stats is not None else _ncu_traffic("stats_step_kernel", stats_bytes)}
     r_fused = {"kernel": "fused_step_kernel", "bound": "hbm", "achieved": fused_gbs, "peak": peak, "unit": "GB/s",
                "frac": fused_gbs / peak, "peak_kind": peak_kind + " (burst copy)", "frac_of_8TBs": fused_gbs / 8000.0,
                "bytes_per_launch": int(fused_bytes), "ms": fused_ms,
                "timed": "events inside baoc_step around the fused kernel alone",
                "whole_step": {"ms": step_ms, "GBps": step_gbs, "frac": step_gbs / peak, "bytes": int(step_bytes),
                               "row_col_kernels_ms": red_ms},
-               "traffic": args.traffic_step}
+               "traffic": args.traffic_step if args.traffic_step is not None else _ncu_traffic("fused_step_kernel", fused_bytes)}
     roofline, other = (r_fused, r_stats) if fused_ms >= stats_ms else (r_stats, r_fused)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
