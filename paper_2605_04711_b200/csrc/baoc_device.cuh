@@ -160,6 +160,22 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
+// ---- approximate square root and reciprocal (one instruction each, relative error 2^-23, subnormals flushed) ----
+__device__ __forceinline__ float sqrt_approx(float x) {
+    float r;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+// Warp maximum of non-negative floats (their bit patterns order like unsigned integers): one reduction instruction.
+__device__ __forceinline__ float warp_max_nonneg(float x) {
+    return __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(x)));
+}
+
 // ---- 8-bit block-wise absmax codes -----------------------------------------------
 // code = clamp(rne(L * x / a)), x ~ code * a / L, with L = 127 (signed) or 255
 // (unsigned) and a the fp32 absmax of the 256-element quantisation block.  The

@@ -223,16 +223,6 @@ factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __r
 // same unit in subnormal scaling: six instructions per square root): a second
 // moment below 1.2e-38 counts as 0 under the root, far below any eps in use.
 // ============================================================================
-__device__ __forceinline__ float sqrt_approx(float x) {
-    float r;
-    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-    return r;
-}
-__device__ __forceinline__ float rcp_approx(float x) {
-    float r;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-    return r;
-}
 
 __device__ __forceinline__ void prologue(float& x, float& t, const CfgStep& P) {
     if (P.coupled) x = fmaf(P.wd, t, x);          // coupled decay joins the gradient
@@ -520,10 +510,6 @@ __device__ __forceinline__ int encode_exact(double x, float absmax, double level
 // Lowest bytes of four words, packed in order.
 __device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     return __byte_perm(__byte_perm(a, b, 0x0040u), __byte_perm(c, d, 0x0040u), 0x5410u);
-}
-// Warp maximum of non-negative floats (their bit patterns order like unsigned integers): one reduction instruction.
-__device__ __forceinline__ float warp_max_nonneg(float x) {
-    return __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(x)));
 }
 
 template <bool kCoupled>
