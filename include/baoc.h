@@ -239,6 +239,31 @@ int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* co
  * one byte per block.  Waits. */
 int baoc_nonfinite(baoc_t* h, uint8_t* flags, int32_t* count, baoc_stream_t stream);
 
+/* ---- checkpoint / resume ---------------------------------------------------------
+ * All per-parameter state of a handle lives in the two caller-owned device
+ * buffers (statistics workspace, optimizer state); the handle itself only adds
+ * the window's step count and the configured assignment.  A checkpoint is
+ * therefore: the bytes of those buffers (copied by the caller, with the stream
+ * idle) plus the small host blob of baoc_export.  The paper only notes that
+ * re-planning needs state to be carried over (Sec. 3.1, online variant); the
+ * format is this library's own.
+ *
+ * baoc_export: writes the blob to buf (host, capacity bytes) and its length to
+ * *size; with buf == NULL only *size is written.  BAOC_E_WORKSPACE if capacity
+ * is too small.  Host only.
+ *
+ * baoc_import: h must have been created with the same blocks and the same
+ * configuration tuples (hyper-parameters may differ).  ws_dev / state_dev are
+ * device buffers that already hold the checkpointed bytes, at any 256-byte
+ * aligned address (the tables inside them are rebuilt for the new addresses and
+ * uploaded on the stream; moments, codes and accumulators are left as they
+ * are).  Either may be NULL if the checkpointed handle had none.  Afterwards
+ * the handle continues exactly where the exported one stopped.
+ * BAOC_E_INVALID for a foreign, truncated or mismatching blob. */
+int baoc_export(const baoc_t* h, void* buf, size_t capacity, size_t* size);
+int baoc_import(baoc_t* h, const void* blob, size_t size, void* ws_dev, size_t ws_bytes,
+                void* state_dev, size_t state_bytes, baoc_stream_t stream);
+
 /* Per-kernel timing of baoc_step, for benchmarks.  With profiling on, every
  * baoc_step records CUDA events on its stream around the factored row/column
  * kernels and around the fused update kernel (events are created on the first

@@ -74,7 +74,8 @@ EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error"
            "baoc_stats_workspace_bytes", "baoc_bind_stats_workspace", "baoc_sample_stats", "baoc_read_stats",
            "baoc_risk", "baoc_risk_from_raw", "baoc_cost_model", "baoc_allocate", "baoc_state_bytes",
            "baoc_configure", "baoc_step", "baoc_step_from_host", "baoc_view", "baoc_nonfinite",
-           "baoc_sample_stats_noalloc", "baoc_noalloc_last_error", "baoc_profile", "baoc_profile_last"]
+           "baoc_sample_stats_noalloc", "baoc_noalloc_last_error", "baoc_profile", "baoc_profile_last",
+           "baoc_export", "baoc_import"]
 
 _vp = C.c_void_p
 _lib.baoc_default_opts.argtypes = [C.POINTER(Opts)]
@@ -99,6 +100,8 @@ _lib.baoc_step.argtypes = [_vp, _vp, _vp, C.c_int64, _vp]
 _lib.baoc_step_from_host.argtypes = [_vp, _vp, _vp, _vp, C.c_int, C.c_int64, _vp]
 _lib.baoc_view.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(_vp), C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
 _lib.baoc_nonfinite.argtypes = [_vp, _vp, C.POINTER(C.c_int32), _vp]
+_lib.baoc_export.argtypes = [_vp, _vp, C.c_size_t, C.POINTER(C.c_size_t)]
+_lib.baoc_import.argtypes = [_vp, _vp, C.c_size_t, _vp, C.c_size_t, _vp, C.c_size_t, _vp]
 _lib.baoc_profile.argtypes = [_vp, C.c_int]
 _lib.baoc_profile_last.argtypes = [_vp, C.POINTER(C.c_float)]
 _lib.baoc_sample_stats_noalloc.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_double, C.c_double, C.c_double, _vp, _vp]
@@ -289,6 +292,24 @@ class Baoc:
                 flat = buf.view(torch.uint8).reshape(-1)
                 return flat[p - base: p - base + n * eb].view(dtype)
         raise BaocError(E_STATE, "the tensor lies in no buffer bound through this object")
+
+    def export_state(self) -> bytes:
+        """The host blob of ``baoc_export`` (window step count and assignment)."""
+        n = C.c_size_t()
+        self._check(_lib.baoc_export(self._h, None, 0, C.byref(n)))
+        buf = C.create_string_buffer(n.value)
+        self._check(_lib.baoc_export(self._h, buf, n.value, C.byref(n)))
+        return buf.raw[:n.value]
+
+    def import_state(self, blob: bytes, ws: Optional[torch.Tensor] = None, state: Optional[torch.Tensor] = None):
+        """``baoc_import``: ws / state are device buffers that already hold the checkpointed bytes."""
+        nb = lambda t: t.numel() * t.element_size()
+        self._check(_lib.baoc_import(self._h, blob, len(blob), ws.data_ptr() if ws is not None else None,
+                                     nb(ws) if ws is not None else 0, state.data_ptr() if state is not None else None,
+                                     nb(state) if state is not None else 0, _stream()))
+        for t in (ws, state):
+            if t is not None:
+                self._keep.append(t)
 
     def profile(self, enable: bool):
         self._check(_lib.baoc_profile(self._h, int(bool(enable))))

@@ -125,7 +125,7 @@ int baoc_stats_workspace_bytes(const baoc_t* h, size_t* bytes) {
     return BAOC_OK;
 }
 
-int baoc_bind_stats_workspace(baoc_t* h, void* dev, size_t bytes, baoc_stream_t stream) {
+static int bind_stats(baoc_t* h, void* dev, size_t bytes, baoc_stream_t stream, bool reset) {
     if (!h) return BAOC_E_INVALID;
     if (!dev) return fail(h, BAOC_E_INVALID, "baoc_bind_stats_workspace: null workspace");
     if (reinterpret_cast<uintptr_t>(dev) & 255u) return fail(h, BAOC_E_ALIGN, "baoc_bind_stats_workspace: workspace not 256-byte aligned");
@@ -164,12 +164,18 @@ int baoc_bind_stats_workspace(baoc_t* h, void* dev, size_t bytes, baoc_stream_t 
     if (!ids.empty())
         CU(cudaMemcpyAsync(ws + L.matrix_ids, ids.data(), 4 * ids.size(), cudaMemcpyHostToDevice, s), "upload matrix ids");
     // moments, previous gradient and running values start at zero
-    CU(cudaMemsetAsync(ws + L.m, 0, L.partials - L.m, s), "zero moments");
-    CU(cudaMemsetAsync(ws + L.acc, 0, 8 * size_t(kBlockAcc) * n, s), "zero accumulators");
+    if (reset) {
+        CU(cudaMemsetAsync(ws + L.m, 0, L.partials - L.m, s), "zero moments");
+        CU(cudaMemsetAsync(ws + L.acc, 0, 8 * size_t(kBlockAcc) * n, s), "zero accumulators");
+    }
     h->ws = ws; h->ws_bytes = bytes; h->ws_bound = true;
-    h->stats_steps = 0;
+    if (reset) h->stats_steps = 0;
     h->last_stat_grads.clear(); h->last_stat_params.clear();
     return BAOC_OK;
+}
+
+int baoc_bind_stats_workspace(baoc_t* h, void* dev, size_t bytes, baoc_stream_t stream) {
+    return bind_stats(h, dev, bytes, stream, true);
 }
 
 int baoc_sample_stats(baoc_t* h, const void* const* grads, baoc_stream_t stream) {
@@ -278,7 +284,7 @@ int baoc_state_bytes(const baoc_t* h, const int32_t* assign, size_t* bytes) {
     return BAOC_OK;
 }
 
-int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes, baoc_stream_t stream) {
+static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes, baoc_stream_t stream, bool reset) {
     if (!h) return BAOC_E_INVALID;
     if (!assign || !state_dev) return fail(h, BAOC_E_INVALID, "baoc_configure: null argument");
     if (reinterpret_cast<uintptr_t>(state_dev) & 255u) return fail(h, BAOC_E_ALIGN, "baoc_configure: state buffer not 256-byte aligned");
@@ -314,7 +320,7 @@ int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t byt
         CU(cudaMemcpyAsync(st + L.red_tiles, red.data(), sizeof(RedTile) * red.size(), cudaMemcpyHostToDevice, s), "upload step reduction table");
     if (!ids.empty())
         CU(cudaMemcpyAsync(st + L.f_ids, ids.data(), 4 * ids.size(), cudaMemcpyHostToDevice, s), "upload factored ids");
-    CU(cudaMemsetAsync(st + L.flags, 0, L.total - L.flags, s), "zero optimizer state");
+    if (reset) CU(cudaMemsetAsync(st + L.flags, 0, L.total - L.flags, s), "zero optimizer state");
     h->st = st; h->st_bytes = bytes; h->tl = L; h->configured = true;
     h->assign.assign(assign, assign + n);
     h->h_step_blocks = sb;
@@ -322,6 +328,78 @@ int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t byt
     h->n_factored = int(ids.size());
     h->state_mem = mem; h->step_bytes = traffic;
     h->last_step_grads.clear(); h->last_step_params.clear();
+    return BAOC_OK;
+}
+
+int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes, baoc_stream_t stream) {
+    return configure_state(h, assign, state_dev, bytes, stream, true);
+}
+
+// ---- checkpoint / resume ---------------------------------------------------------
+namespace {
+struct BlobHeader {
+    uint32_t magic, version;
+    int32_t n_blocks, n_cfg;
+    int64_t numel, stats_steps;
+    int32_t ws_bound, configured;
+    uint64_t shape_hash;
+};
+constexpr uint32_t kBlobMagic = 0x434f4142u;   // "BAOC"
+
+// FNV-1a over the block shapes and the configuration tuples (not their hyper-parameters, which may change on resume)
+uint64_t shape_hash(const Handle* h) {
+    uint64_t x = 1469598103934665603ull;
+    auto mix = [&](const void* p, size_t n) {
+        const unsigned char* b = static_cast<const unsigned char*>(p);
+        for (size_t i = 0; i < n; ++i) { x ^= b[i]; x *= 1099511628211ull; }
+    };
+    for (const baoc_block_t& b : h->blocks) { mix(&b.numel, 8); mix(&b.rows, 4); mix(&b.cols, 4); }
+    for (const baoc_config_t& c : h->cfgs) mix(&c.adaptive, 5);
+    return x;
+}
+}  // namespace
+
+int baoc_export(const baoc_t* h, void* buf, size_t capacity, size_t* size) {
+    if (!h) return BAOC_E_INVALID;
+    if (!size) return fail(h, BAOC_E_INVALID, "baoc_export: null size");
+    const size_t need = sizeof(BlobHeader) + (h->configured ? 4 * size_t(h->n_blocks) : 0);
+    *size = need;
+    if (!buf) return BAOC_OK;
+    if (capacity < need) return fail(h, BAOC_E_WORKSPACE, "baoc_export: buffer too small");
+    BlobHeader hd{};
+    hd.magic = kBlobMagic; hd.version = 1; hd.n_blocks = h->n_blocks; hd.n_cfg = h->n_cfg;
+    hd.numel = h->numel; hd.stats_steps = h->stats_steps;
+    hd.ws_bound = h->ws_bound ? 1 : 0; hd.configured = h->configured ? 1 : 0;
+    hd.shape_hash = shape_hash(h);
+    std::memcpy(buf, &hd, sizeof(hd));
+    if (h->configured) std::memcpy(static_cast<char*>(buf) + sizeof(hd), h->assign.data(), 4 * size_t(h->n_blocks));
+    return BAOC_OK;
+}
+
+int baoc_import(baoc_t* h, const void* blob, size_t size, void* ws_dev, size_t ws_bytes, void* state_dev,
+                size_t state_bytes, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!blob || size < sizeof(BlobHeader)) return fail(h, BAOC_E_INVALID, "baoc_import: blob missing or truncated");
+    BlobHeader hd;
+    std::memcpy(&hd, blob, sizeof(hd));
+    if (hd.magic != kBlobMagic || hd.version != 1) return fail(h, BAOC_E_INVALID, "baoc_import: not a blob of this library version");
+    if (hd.n_blocks != h->n_blocks || hd.n_cfg != h->n_cfg || hd.numel != h->numel || hd.shape_hash != shape_hash(h))
+        return fail(h, BAOC_E_INVALID, "baoc_import: the blob belongs to a different block set or candidate set");
+    if (hd.stats_steps < 0) return fail(h, BAOC_E_INVALID, "baoc_import: corrupt blob");
+    if (hd.configured && size < sizeof(BlobHeader) + 4 * size_t(h->n_blocks)) return fail(h, BAOC_E_INVALID, "baoc_import: blob truncated");
+    if (hd.ws_bound && !ws_dev) return fail(h, BAOC_E_INVALID, "baoc_import: the checkpoint had a statistics workspace; pass its copy");
+    if (hd.configured && !state_dev) return fail(h, BAOC_E_INVALID, "baoc_import: the checkpoint had optimizer state; pass its copy");
+    if (hd.ws_bound) {
+        int rc = bind_stats(h, ws_dev, ws_bytes, stream, false);
+        if (rc) return rc;
+        h->stats_steps = hd.stats_steps;
+    }
+    if (hd.configured) {
+        std::vector<int32_t> assign(h->n_blocks);
+        std::memcpy(assign.data(), static_cast<const char*>(blob) + sizeof(BlobHeader), 4 * size_t(h->n_blocks));
+        int rc = configure_state(h, assign.data(), state_dev, state_bytes, stream, false);
+        if (rc) return rc;
+    }
     return BAOC_OK;
 }
 

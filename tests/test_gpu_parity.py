@@ -355,6 +355,47 @@ def test_gpu_argument_checks(B, H):
     assert e.value.code == B.E_STATE
 
 
+def test_checkpoint_resume_continues_bit_exactly(B, H):
+    """Export after a window and some steps, move every buffer to a new address, import into a fresh handle, and
+    let both handles continue on the same gradients: parameters, states and running statistics stay identical."""
+    wl = _odd_workload(seed=51)
+    sess = H.Session(wl, n_grad_sets=2)
+    sess.init_params()
+    n = len(wl.blocks)
+    assign = [(i % 5) if not ((i % 5) == 3 and b.cols <= 1) else 1 for i, b in enumerate(wl.blocks)]
+    for t in (1, 2, 3):
+        sess.sample_stats(sess.fill_grads(t))
+    sess.configure(assign)
+    for t in (1, 2):
+        sess.step(sess.fill_grads(3 + t), t)
+    torch.cuda.synchronize()
+    blob = sess.h.export_state()
+    ws2 = torch.empty(sess.ws.numel() + 512, dtype=torch.uint8, device=sess.device)
+    ws2 = ws2[(-ws2.data_ptr()) % 256:][:sess.ws.numel()]
+    st2 = torch.empty(sess.state.numel() + 512, dtype=torch.uint8, device=sess.device)
+    st2 = st2[(-st2.data_ptr()) % 256:][:sess.state.numel()]
+    ws2.copy_(sess.ws); st2.copy_(sess.state)
+    params2 = sess.params.clone()
+    pviews2 = [params2[o:o + b.numel] for o, b in zip(sess.offs, wl.blocks)]
+    h2 = B.Baoc(wl.blocks, sess.configs)
+    h2.import_state(blob, ws2, st2)
+    assert h2.query().stats_steps == 3 and h2.query().state_bytes == sess.h.query().state_bytes
+    for t in (3, 4, 5):
+        k = sess.fill_grads(3 + t)
+        sess.sample_stats(k); sess.step(k, t)
+        h2.sample_stats(sess.grad_views[k]); h2.step(sess.grad_views[k], pviews2, t)
+    torch.cuda.synchronize()
+    assert torch.equal(params2, sess.params)
+    a, b2 = sess.h.read_stats(), h2.read_stats()
+    for i in range(n):
+        assert a[i]["rho_bar"] == b2[i]["rho_bar"] and a[i]["n_cos"] == b2[i]["n_cos"] == 5
+        for which, dt in ((0, torch.float32), (1, torch.float32), (2, torch.bfloat16)):
+            assert torch.equal(sess.h.view_tensor(i, which, dt), h2.view_tensor(i, which, dt))
+    r1, _ = sess.risk()
+    r2, _ = h2.risk(pviews2)
+    np.testing.assert_array_equal(r1, r2)
+
+
 # ---------------------------------------------------------------- whole pipeline
 
 def _pipeline(B, H, name, T, n_steps, time_table=None):

@@ -209,3 +209,23 @@ def test_allocator_time_budget_binds_and_node_limit_warns(B):
     if rc3 == B.W_NODE_LIMIT:
         assert sum(int(mem[i, c]) for i, c in enumerate(asg3)) <= int(0.4 * 8 * wl.numel)
         assert obj3 >= obj - 1e-12
+
+
+def test_export_import_blob_without_device_state(B):
+    blocks = [(64, 8, 8), (5, 5, 1)]
+    h = B.Baoc(blocks, B.default_configs())
+    blob = h.export_state()
+    assert len(blob) >= 40
+    B.Baoc(blocks, B.default_configs()).import_state(blob)                     # nothing bound, nothing configured: fine
+    other_lr = B.default_configs()
+    other_lr[0].lr = 5e-4
+    B.Baoc(blocks, other_lr).import_state(blob)                                # hyper-parameters may differ on resume
+    for bad_handle in (B.Baoc([(64, 8, 8), (6, 6, 1)], B.default_configs()),   # another block set
+                       B.Baoc(blocks, B.default_configs()[:4])):               # another candidate set
+        with pytest.raises(B.BaocError) as e:
+            bad_handle.import_state(blob)
+        assert e.value.code == B.E_INVALID
+    for bad_blob in (blob[:10], b"XXXX" + blob[4:]):                           # truncated; foreign magic
+        with pytest.raises(B.BaocError) as e:
+            B.Baoc(blocks, B.default_configs()).import_state(bad_blob)
+        assert e.value.code == B.E_INVALID
