@@ -28,6 +28,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 CONFIG_NAMES = ["adamw32", "adamw8", "rms", "factored", "sgdm"]
+EXTENDED_NAMES = CONFIG_NAMES + ["sgd", "adamw16", "rms16", "sgdm16"]
 METRIC = "hot-path throughput: statistics pass + mixed-config optimizer step"
 UNIT = "params/s"
 
@@ -259,7 +260,11 @@ def run_ours(args):
         wl.blocks = [wl.blocks[i] for i in part]
     else:
         wl = W.make_workload(args.workload, seed=rank)       # replicas: every rank streams its own copy of the workload
-    sess = harness.Session(wl, n_grad_sets=2, device=f"cuda:{local}", pinned_host_grads=True)
+    from paper_2605_04711_b200 import binding
+    extended = args.candidates == "extended" or args.assign in EXTENDED_NAMES[5:]
+    names = EXTENDED_NAMES if extended else CONFIG_NAMES
+    sess = harness.Session(wl, configs=binding.extended_configs() if extended else None, n_grad_sets=2,
+                           device=f"cuda:{local}", pinned_host_grads=True)
     sess.init_params()
     for t in (1, 2):
         k = sess.fill_grads(t)
@@ -282,7 +287,7 @@ def run_ours(args):
     alloc_ms = (time.perf_counter() - t0) * 1e3
     if args.assign != "auto":
         # one configuration for every block (vectors cannot be factored: they take the momentum-free one)
-        c = CONFIG_NAMES.index(args.assign)
+        c = names.index(args.assign)
         assign = np.asarray([c if not (c == 3 and b.cols <= 1) else 2 for b in wl.blocks], np.int32)
     sess.configure(assign)
     info = sess.h.query()
@@ -391,7 +396,7 @@ def run_ours(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if (args.shard_blocks and world > 1) else "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "params": wl.numel, "blocks": len(wl.blocks), "grad_dtype": "bf16",
-                   "param_dtype": "f32", "candidate_configs": CONFIG_NAMES, "assignment": args.assign,
+                   "param_dtype": "f32", "candidate_configs": names, "assignment": args.assign,
                    "assignment_blocks_per_config": counts, "assignment_params_per_config": params_by_cfg,
                    "mem_budget_frac_of_fp32_adam": wl.mem_budget_frac, "state_bytes": int(info.state_bytes),
                    "window_steps_before_timing": args.window, "l2": "inputs (>10 GB per step) far exceed the 126 MB L2",
@@ -423,7 +428,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama_1b")
-    ap.add_argument("--assign", default="auto", choices=["auto"] + CONFIG_NAMES,
+    ap.add_argument("--candidates", default="default", choices=["default", "extended"],
+                    help="default: the five tuples of the headline path; extended: plus sgd and the bf16-state variants")
+    ap.add_argument("--assign", default="auto", choices=["auto"] + EXTENDED_NAMES,
                     help="auto: the library's own budgeted allocation; else every block under that one configuration")
     ap.add_argument("--shard-blocks", action="store_true",
                     help="N > 1: deal whole blocks of ONE workload to the ranks (strong scaling) instead of one replica per rank")

@@ -445,23 +445,31 @@ class StepState:
 
 
 def config_kind(c: Config) -> str:
-    """Which of the five update paths a tuple selects."""
-    if c.adaptive and c.momentum and not c.factored:
-        return "A32" if c.bits == 32 else ("A8" if c.bits == 8 else "unsupported")
-    if c.adaptive and not c.momentum and not c.factored and c.bits == 32:
-        return "R"
-    if c.adaptive and not c.momentum and c.factored and c.bits == 32:
-        return "F"
-    if not c.adaptive and c.momentum and not c.factored and c.bits == 32:
-        return "S"
-    return "unsupported"
+    """Which update path a tuple selects.  A32 / A16 / A8: Adam with fp32 / bf16 / 8-bit moments; R / R16:
+    momentum-free RMS scaling; F: factored second moment; S / S16: SGD with momentum; G: plain gradient step
+    (neither mechanism, hence no state, whatever bit-width the tuple names)."""
+    if c.factored:
+        return "F" if (c.adaptive and not c.momentum and c.bits == 32) else "unsupported"
+    if c.adaptive and c.momentum:
+        return {32: "A32", 16: "A16", 8: "A8"}[c.bits]
+    if c.adaptive and not c.momentum:
+        return {32: "R", 16: "R16"}.get(c.bits, "unsupported")
+    if not c.adaptive and c.momentum:
+        return {32: "S", 16: "S16"}.get(c.bits, "unsupported")
+    return "G"
 
 
 def step_init(c: Config, numel: int, rows: int, cols: int, qblock: int = 256) -> StepState:
     kind = config_kind(c)
     nq = (numel + qblock - 1) // qblock
-    if kind == "A32":
+    if kind in ("A32", "A16"):
         return StepState(kind, m=np.zeros(numel, F64), v=np.zeros(numel, F64))
+    if kind == "R16":
+        return StepState(kind, v=np.zeros(numel, F64))
+    if kind == "S16":
+        return StepState(kind, m=np.zeros(numel, F64))
+    if kind == "G":
+        return StepState(kind)
     if kind == "A8":
         return StepState(kind, qm=np.zeros(numel, np.int8), qv=np.zeros(numel, np.uint8),
                          am=np.zeros(nq, np.float32), av=np.zeros(nq, np.float32))
@@ -489,6 +497,23 @@ def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, 
         st.m = c.beta1 * st.m + (1.0 - c.beta1) * g
         st.v = c.beta2 * st.v + (1.0 - c.beta2) * g * g
         return _adam_apply(theta, st.m, st.v, c, t, True)
+    # 16-bit states: the stored moments are bf16; the update uses the new moments before they are rounded for
+    # storage (the same convention as the 8-bit path)
+    if st.kind == "A16":
+        m = c.beta1 * st.m + (1.0 - c.beta1) * g
+        v = c.beta2 * st.v + (1.0 - c.beta2) * g * g
+        st.m, st.v = round_bf16(m), round_bf16(v)
+        return _adam_apply(theta, m, v, c, t, True)
+    if st.kind == "R16":
+        v = c.beta2 * st.v + (1.0 - c.beta2) * g * g
+        st.v = round_bf16(v)
+        return _adam_apply(theta, g, v, c, t, False)
+    if st.kind == "S16":
+        m = c.beta1 * st.m + g
+        st.m = round_bf16(m)
+        return theta - c.lr * m
+    if st.kind == "G":
+        return theta - c.lr * g
     if st.kind == "A8":
         m = dequantize8(st.qm, st.am, True, qblock)
         v = dequantize8(st.qv, st.av, False, qblock)

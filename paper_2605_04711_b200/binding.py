@@ -142,6 +142,15 @@ def default_configs() -> List[Config]:
             make_config(0, 1, 1, 0, 32, lr=1e-2, weight_decay=0.01)]
 
 
+def extended_configs() -> List[Config]:
+    """The five default tuples plus the plain gradient step and the bf16-state variants of Adam(W), RMS scaling
+    and SGD with momentum."""
+    return default_configs() + [make_config(0, 0, 1, 0, 32, lr=1e-2, weight_decay=0.01),
+                                make_config(1, 1, 1, 0, 16, weight_decay=0.01),
+                                make_config(1, 0, 1, 0, 16, weight_decay=0.01),
+                                make_config(0, 1, 1, 0, 16, lr=1e-2, weight_decay=0.01)]
+
+
 def pointer_table(tensors: Sequence[torch.Tensor]):
     """Host array of the tensors' data pointers, in the layout the C calls take."""
     return (C.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])

@@ -303,8 +303,8 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
     for (int i = 0; i < n; ++i) {
         StepBlock& b = sb[i];
         auto fix = [&](void* p) { return static_cast<void*>(st + L.states + reinterpret_cast<size_t>(p)); };
-        if (b.path == kPathA32 || b.path == kPathA8 || b.path == kPathF) { b.s0 = fix(b.s0); b.s1 = fix(b.s1); }
-        else b.s0 = fix(b.s0);
+        if (b.path == kPathA32 || b.path == kPathA8 || b.path == kPathF || b.path == kPathA16) { b.s0 = fix(b.s0); b.s1 = fix(b.s1); }
+        else if (b.path != kPathG) b.s0 = fix(b.s0);
         if (b.path == kPathA8) { b.a0 = static_cast<float*>(fix(b.a0)); b.a1 = static_cast<float*>(fix(b.a1)); }
         if (b.path == kPathF) {
             b.a0 = static_cast<float*>(fix(b.a0));
@@ -502,6 +502,8 @@ int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* co
                 else if (k == 2) { p = s.a0; n = nq; } else { p = s.a1; n = nq; }
                 break;
             case kPathR: case kPathS: if (k == 0) { p = s.s0; n = b.numel; } break;
+            case kPathA16: if (k == 0) { p = s.s0; n = b.numel; eb = 2; } else if (k == 1) { p = s.s1; n = b.numel; eb = 2; } break;
+            case kPathR16: case kPathS16: if (k == 0) { p = s.s0; n = b.numel; eb = 2; } break;
             case kPathF: if (k == 0) { p = s.s0; n = b.rows; } else if (k == 1) { p = s.s1; n = b.cols; } break;
             default: break;
         }

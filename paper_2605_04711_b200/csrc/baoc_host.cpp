@@ -141,6 +141,9 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
                 s.a0 = static_cast<float*>(place(4 * nq)); s.a1 = static_cast<float*>(place(4 * nq));
                 break;
             case kPathR: case kPathS: s.s0 = place(4 * dpad); break;
+            case kPathA16: s.s0 = place(2 * dpad); s.s1 = place(2 * dpad); break;
+            case kPathR16: case kPathS16: s.s0 = place(2 * dpad); break;
+            case kPathG: break;
             case kPathF: {
                 s.s0 = place(4 * size_t(b.rows)); s.s1 = place(4 * size_t(b.cols));
                 s.a0 = static_cast<float*>(place(16));
@@ -161,7 +164,7 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
         traffic += step_traffic_bytes(h->cfgs[c], b);
     }
     // tiles in descending bytes per element so that the light ones fill the tail of the grid
-    const int order[5] = {kPathA32, kPathR, kPathS, kPathA8, kPathF};
+    const int order[kPathCount] = {kPathA32, kPathR, kPathS, kPathA16, kPathR16, kPathS16, kPathG, kPathA8, kPathF};
     for (int p : order)
         for (int i = 0; i < n; ++i)
             if (sb[i].path == p) {

@@ -31,14 +31,22 @@ constexpr int kTileQ = 16384;         // elements per tile of the 8-bit path (it
 constexpr int kCombineSlabs = 32;     // CTAs per factored block of the row/column combine
 
 // Update paths of the fused step.
-enum Path : int32_t { kPathA32 = 0, kPathA8 = 1, kPathR = 2, kPathF = 3, kPathS = 4, kPathNone = -1 };
+enum Path : int32_t {
+    kPathA32 = 0, kPathA8 = 1, kPathR = 2, kPathF = 3, kPathS = 4,
+    kPathG = 5,          // plain gradient step (SGD / SGDW without momentum): no state
+    kPathA16 = 6,        // Adam / AdamW with bf16 moments
+    kPathR16 = 7,        // momentum-free RMS scaling with a bf16 second moment
+    kPathS16 = 8,        // SGD with a bf16 momentum buffer
+    kPathCount = 9,
+    kPathNone = -1
+};
 
 inline Path path_of(const baoc_config_t& c) {
-    if (c.adaptive && c.momentum && !c.factored) return c.bits == 32 ? kPathA32 : (c.bits == 8 ? kPathA8 : kPathNone);
-    if (c.adaptive && !c.momentum && !c.factored && c.bits == 32) return kPathR;
-    if (c.adaptive && !c.momentum && c.factored && c.bits == 32) return kPathF;
-    if (!c.adaptive && c.momentum && !c.factored && c.bits == 32) return kPathS;
-    return kPathNone;
+    if (c.factored) return (c.adaptive && !c.momentum && c.bits == 32) ? kPathF : kPathNone;
+    if (c.adaptive && c.momentum) return c.bits == 32 ? kPathA32 : (c.bits == 16 ? kPathA16 : kPathA8);
+    if (c.adaptive && !c.momentum) return c.bits == 32 ? kPathR : (c.bits == 16 ? kPathR16 : kPathNone);
+    if (!c.adaptive && c.momentum) return c.bits == 32 ? kPathS : (c.bits == 16 ? kPathS16 : kPathNone);
+    return kPathG;       // neither mechanism: stateless, whatever bit-width the tuple names
 }
 
 // Elements per tile of the fused step, by update path.

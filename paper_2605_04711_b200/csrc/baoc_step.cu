@@ -235,29 +235,6 @@ __device__ __forceinline__ float adaptive_apply(float t, float num, float v, flo
     return fmaf(-step * num, rcp_approx(denom), t);
 }
 
-struct PathA32 {
-    static __device__ __forceinline__ void upd(float x, float& t, float& m, float& v, const CfgStep& P) {
-        prologue(x, t, P);
-        m = fmaf(P.beta1, m, P.om1 * x);
-        v = fmaf(P.beta2, v, P.om2 * (x * x));
-        t = adaptive_apply(t, m, v, P.step_m, P);
-    }
-};
-struct PathR {
-    static __device__ __forceinline__ void upd(float x, float& t, float& v, const CfgStep& P) {
-        prologue(x, t, P);
-        v = fmaf(P.beta2, v, P.om2 * (x * x));
-        t = adaptive_apply(t, x, v, P.step_g, P);
-    }
-};
-struct PathS {
-    static __device__ __forceinline__ void upd(float x, float& t, float& m, const CfgStep& P) {
-        prologue(x, t, P);
-        m = fmaf(P.beta1, m, x);
-        t = fmaf(-P.step_g, m, t);
-    }
-};
-
 __device__ __forceinline__ void f4_to(const float4& a, const float4& b, float (&x)[8]) {
     x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
 }
@@ -275,16 +252,72 @@ constexpr int kSlicesQ = kTileQ / (kThreads * 8);
 constexpr int kStagesQ = 3;                                          // two slices in flight while one is consumed
 constexpr int kStageBytes = kThreads * 64;                           // g 16 B/thread at 0, theta 32 at 4096, m codes 8 at 12288, v codes 8 at 14336
 
-// fp32 Adam / RMS / SGD-momentum: kM = has first moment, kV = has second moment.
-template <bool kM, bool kV>
+// Dense paths: one streaming pass per element, state in fp32 or bf16.
+//   kM = has a first moment / momentum buffer, kV = has a second moment, kB16 = the state is stored as bf16.
+//   kM && kV: Adam;  kV only: momentum-free RMS scaling;  kM only: SGD with momentum;  neither: plain gradient step.
+// With bf16 storage the parameter update uses the un-rounded fp32 moments and the stored value is the
+// round-to-nearest-even bf16 of the new moment.  That rounding is a decision on a floating-point value, so it is
+// taken exactly: the fp32 moment is within err of the exact one, and unless it lies within err of the midpoint
+// between the two bf16 neighbours its rounding is already the exact answer; the few that do are recomputed in
+// double (and rounded double -> fp32 -> bf16).
+__device__ __forceinline__ uint32_t bf16_rne_bits(float x) {
+    const uint32_t u = __float_as_uint(x);
+    if ((u & 0x7f800000u) == 0x7f800000u) return u >> 16;           // infinities and NaNs keep their top half
+    return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
+}
+
+template <bool kM, bool kV, bool kB16>
+struct DenseElem {
+    // One element.  x: gradient, t: parameter (updated), m / v: old moments (replaced by the new fp32 ones),
+    // mb / vb: bf16 bits of the new moments when kB16.
+    static __device__ __forceinline__ void upd(float x, float& t, float& m, float& v, uint32_t& mb, uint32_t& vb,
+                                               const CfgStep& P) {
+        constexpr float kErr = 4.76837158203125e-7f;                // 2^-21: twice the first-order bound of four roundings
+        const float x_raw = x, t_old = t, m_old = m, v_old = v;
+        prologue(x, t, P);
+        float pm = 0.f, pv = 0.f;
+        if (kM) { pm = kV ? P.om1 * x : x; m = fmaf(P.beta1, m_old, pm); }
+        if (kV) { pv = P.om2 * (x * x); v = fmaf(P.beta2, v_old, pv); }
+        if (kB16) {
+            auto exact_g = [&]() { return P.coupled ? double(x_raw) + P.wd_d * double(t_old) : double(x_raw); };
+            if (kM) {
+                const float mid = __uint_as_float((__float_as_uint(m) & 0xffff0000u) | 0x8000u);
+                float r = m;
+                if (fabsf(m - mid) <= kErr * (fabsf(pm) + fabsf(m)))
+                    r = __double2float_rn(P.beta1_d * double(m_old) + (kV ? 1.0 - P.beta1_d : 1.0) * exact_g());
+                mb = bf16_rne_bits(r);
+            }
+            if (kV) {
+                const float mid = __uint_as_float((__float_as_uint(v) & 0xffff0000u) | 0x8000u);
+                float r = v;
+                if (fabsf(v - mid) <= kErr * (pv + v)) {
+                    const double gd = exact_g();
+                    r = __double2float_rn(P.beta2_d * double(v_old) + (1.0 - P.beta2_d) * (gd * gd));
+                }
+                vb = bf16_rne_bits(r);
+            }
+        }
+        if (kM && kV) t = adaptive_apply(t, m, v, P.step_m, P);
+        else if (kV) t = adaptive_apply(t, x, v, P.step_g, P);
+        else if (kM) t = fmaf(-P.step_g, m, t);
+        else t = fmaf(-P.step_g, x, t);
+    }
+};
+
+template <bool kM, bool kV, bool kB16>
 __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep& P, const uint16_t* __restrict__ g,
                                                float* __restrict__ th, int64_t base) {
     const int64_t numel = b->numel;
-    float* __restrict__ m = kM ? static_cast<float*>(b->s0) : nullptr;
-    float* __restrict__ v = kV ? static_cast<float*>(kM ? b->s1 : b->s0) : nullptr;
+    void* const mp = kM ? b->s0 : nullptr;
+    void* const vp = kV ? (kM ? b->s1 : b->s0) : nullptr;
+    float* __restrict__ m = static_cast<float*>(mp);
+    float* __restrict__ v = static_cast<float*>(vp);
+    uint16_t* __restrict__ mh = static_cast<uint16_t*>(mp);
+    uint16_t* __restrict__ vh = static_cast<uint16_t*>(vp);
     float chk = 0.f;
     uint4 wg[kSlices];
     float4 t0[kSlices], t1[kSlices], m0[kSlices], m1[kSlices], v0[kSlices], v1[kSlices];
+    uint4 mw[kSlices], vw[kSlices];
     bool full[kSlices];
 #pragma unroll
     for (int s = 0; s < kSlices; ++s) {
@@ -293,8 +326,13 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
         if (full[s]) {
             wg[s] = ld_stream_u4(g + e);
             t0[s] = ld_stream_f4(th + e); t1[s] = ld_stream_f4(th + e + 4);
-            if (kM) { m0[s] = ld_stream_f4(m + e); m1[s] = ld_stream_f4(m + e + 4); }
-            if (kV) { v0[s] = ld_stream_f4(v + e); v1[s] = ld_stream_f4(v + e + 4); }
+            if (kB16) {
+                if (kM) mw[s] = ld_stream_u4(mh + e);
+                if (kV) vw[s] = ld_stream_u4(vh + e);
+            } else {
+                if (kM) { m0[s] = ld_stream_f4(m + e); m1[s] = ld_stream_f4(m + e + 4); }
+                if (kV) { v0[s] = ld_stream_f4(v + e); v1[s] = ld_stream_f4(v + e + 4); }
+            }
         }
     }
 #pragma unroll
@@ -302,33 +340,46 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
         const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
         if (full[s]) {
             float x[8], t[8], mm[8], vv[8];
+            uint32_t mb[8], vb[8];
             unpack8(wg[s], x); f4_to(t0[s], t1[s], t);
-            if (kM) f4_to(m0[s], m1[s], mm);
-            if (kV) f4_to(v0[s], v1[s], vv);
+            if (kB16) {
+                if (kM) unpack8(mw[s], mm);
+                if (kV) unpack8(vw[s], vv);
+            } else {
+                if (kM) f4_to(m0[s], m1[s], mm);
+                if (kV) f4_to(v0[s], v1[s], vv);
+            }
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                if (kM && kV) PathA32::upd(x[j], t[j], mm[j], vv[j], P);
-                else if (kV) PathR::upd(x[j], t[j], vv[j], P);
-                else PathS::upd(x[j], t[j], mm[j], P);
+                DenseElem<kM, kV, kB16>::upd(x[j], t[j], mm[j], vv[j], mb[j], vb[j], P);
                 chk = poison(chk, t[j]);
             }
             st8(th + e, t);
-            if (kM) st8(m + e, mm);
-            if (kV) st8(v + e, vv);
+            if (kB16) {
+                if (kM) st_stream_u4(mh + e, make_uint4(mb[0] | mb[1] << 16, mb[2] | mb[3] << 16, mb[4] | mb[5] << 16, mb[6] | mb[7] << 16));
+                if (kV) st_stream_u4(vh + e, make_uint4(vb[0] | vb[1] << 16, vb[2] | vb[3] << 16, vb[4] | vb[5] << 16, vb[6] | vb[7] << 16));
+            } else {
+                if (kM) st8(m + e, mm);
+                if (kV) st8(v + e, vv);
+            }
         } else if (e < numel) {
             const int cnt = int(numel - e);
             for (int j = 0; j < cnt; ++j) {
                 const float x = bf16_bits_to_float(g[e + j]);
                 float t = th[e + j], mm = 0.f, vv = 0.f;
-                if (kM) mm = m[e + j];
-                if (kV) vv = v[e + j];
-                if (kM && kV) PathA32::upd(x, t, mm, vv, P);
-                else if (kV) PathR::upd(x, t, vv, P);
-                else PathS::upd(x, t, mm, P);
+                uint32_t mb = 0u, vb = 0u;
+                if (kM) mm = kB16 ? bf16_bits_to_float(mh[e + j]) : m[e + j];
+                if (kV) vv = kB16 ? bf16_bits_to_float(vh[e + j]) : v[e + j];
+                DenseElem<kM, kV, kB16>::upd(x, t, mm, vv, mb, vb, P);
                 chk = poison(chk, t);
                 th[e + j] = t;
-                if (kM) m[e + j] = mm;
-                if (kV) v[e + j] = vv;
+                if (kB16) {
+                    if (kM) mh[e + j] = uint16_t(mb);
+                    if (kV) vh[e + j] = uint16_t(vb);
+                } else {
+                    if (kM) m[e + j] = mm;
+                    if (kV) v[e + j] = vv;
+                }
             }
         }
     }
@@ -735,9 +786,13 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
     __shared__ __align__(16) unsigned char q_stage[kStagesQ * kStageBytes];   // per-thread staging of the 8-bit and factored paths
     unsigned bad = 0;
     switch (b->path) {
-        case kPathA32: bad = tile_dense<true, true>(b, P, g, th, base); break;
-        case kPathR: bad = tile_dense<false, true>(b, P, g, th, base); break;
-        case kPathS: bad = tile_dense<true, false>(b, P, g, th, base); break;
+        case kPathA32: bad = tile_dense<true, true, false>(b, P, g, th, base); break;
+        case kPathR: bad = tile_dense<false, true, false>(b, P, g, th, base); break;
+        case kPathS: bad = tile_dense<true, false, false>(b, P, g, th, base); break;
+        case kPathG: bad = tile_dense<false, false, false>(b, P, g, th, base); break;
+        case kPathA16: bad = tile_dense<true, true, true>(b, P, g, th, base); break;
+        case kPathR16: bad = tile_dense<false, true, true>(b, P, g, th, base); break;
+        case kPathS16: bad = tile_dense<true, false, true>(b, P, g, th, base); break;
         case kPathA8: bad = P.coupled ? tile_int8<true>(b, P, g, th, base, q_stage) : tile_int8<false>(b, P, g, th, base, q_stage); break;
         case kPathF: bad = tile_factored(b, P, g, th, base, q_stage); break;
         default: break;

@@ -216,6 +216,17 @@ def _check_block(sess, i, th_ref, st_ref, code_stats):
         assert _rel_max(f32(10), st_ref.m) <= 1e-6
     elif kind == "F":
         assert _rel_max(f32(10), st_ref.r) <= 1e-6 and _rel_max(f32(11), st_ref.c) <= 1e-6
+    elif kind in ("A16", "R16", "S16"):
+        # bf16 states: the stored bit patterns are compared (a rounding decision, taken exactly on both sides)
+        refs = {"A16": (st_ref.m, st_ref.v), "R16": (st_ref.v,), "S16": (st_ref.m,)}[kind]
+        for w, ref in enumerate(refs):
+            got = sess.h.view_tensor(i, 10 + w, torch.bfloat16).view(torch.int16).cpu().numpy().astype(np.int32)
+            want = torch.from_numpy(ref).to(torch.bfloat16).view(torch.int16).numpy().astype(np.int32)
+            d = np.abs(got - want)
+            assert d.max() <= 1, (sess.wl.blocks[i].name, kind, w, int(d.max()))
+            code_stats[0] += int((d != 0).sum()); code_stats[1] += d.size
+    elif kind == "G":
+        pass
     elif kind == "A8":
         qm = sess.h.view_tensor(i, 10, torch.int8).cpu().numpy().astype(np.int32)
         qv = sess.h.view_tensor(i, 11, torch.uint8).cpu().numpy().astype(np.int32)
@@ -314,6 +325,28 @@ def test_coupled_decay_and_other_hyperparameters_step_by_step(B, H):
             assert np.all(np.abs(got - th[i]) <= tol), (t, b.name, sts[i].kind, float(np.max(np.abs(got - th[i]) / tol)))
             _check_block(sess, i, None, sts[i], codes)
     assert codes[1] > 0 and codes[0] <= 1e-4 * codes[1], codes
+
+
+@pytest.mark.parametrize("tuple_", [(0, 0, 1, 0, 32), (0, 0, 0, 0, 8), (1, 1, 1, 0, 16), (1, 1, 0, 0, 16), (1, 0, 1, 0, 16),
+                                    (0, 1, 1, 0, 16), (0, 1, 0, 0, 16)])
+def test_stateless_and_bf16_state_configurations_ten_steps(B, H, tuple_):
+    """Plain gradient steps (no state) and Adam / RMS / SGD-momentum with bf16 states, decoupled and coupled decay."""
+    wl = _odd_workload(seed=61 + sum(tuple_))
+    lr = 1e-2 if not tuple_[0] else 1e-3
+    cfgs = [B.make_config(*tuple_, lr=lr, weight_decay=0.05)]
+    sess = H.Session(wl, configs=cfgs, n_grad_sets=2)
+    sess.init_params()
+    assign = [0] * len(wl.blocks)
+    th, sts = _run_steps(sess, assign, 10)
+    codes = [0, 0]
+    for i in range(len(wl.blocks)):
+        _check_block(sess, i, th[i], sts[i], codes)
+    if codes[1]:
+        assert codes[0] <= 1e-4 * codes[1], codes
+    assert sess.h.nonfinite()[0] == 0
+    mem, _ = sess.h.cost_model()
+    per = {32: 4, 16: 2, 8: 1}[tuple_[4]] * (tuple_[0] + tuple_[1])
+    assert sess.h.query().state_bytes == int(mem.sum()) == per * wl.numel
 
 
 def test_nonfinite_gradient_is_flagged_not_fatal(B, H):

@@ -540,4 +540,61 @@ def test_int8_path_tracks_fp32_path_within_one_code():
 def test_config_kind_dispatch():
     kinds = [O.config_kind(c) for c in O.default_configs()]
     assert kinds == ["A32", "A8", "R", "F", "S"]
-    assert O.config_kind(O.Config(0, 0, 1, 0, 32)) == "unsupported"
+    assert O.config_kind(O.Config(0, 0, 1, 0, 32)) == "G" and O.config_kind(O.Config(0, 0, 0, 0, 8)) == "G"
+    assert [O.config_kind(O.Config(1, 1, 1, 0, b)) for b in (32, 16, 8)] == ["A32", "A16", "A8"]
+    assert [O.config_kind(O.Config(1, 0, 1, 0, b)) for b in (32, 16, 8)] == ["R", "R16", "unsupported"]
+    assert [O.config_kind(O.Config(0, 1, 1, 0, b)) for b in (32, 16, 8)] == ["S", "S16", "unsupported"]
+    assert O.config_kind(O.Config(1, 1, 1, 1, 32)) == "unsupported" and O.config_kind(O.Config(1, 0, 1, 1, 16)) == "unsupported"
+
+
+def test_plain_gradient_step_matches_torch_sgd():
+    rng = np.random.default_rng(7)
+    th0 = rng.standard_normal(37)
+    for decoupled, wd in ((1, 0.0), (0, 0.1)):
+        c = O.Config(0, 0, decoupled, 0, 32, lr=0.05, weight_decay=wd)
+        st = O.step_init(c, 37, 37, 1)
+        p = torch.tensor(th0, dtype=torch.float64, requires_grad=True)
+        opt = torch.optim.SGD([p], lr=0.05, momentum=0.0, weight_decay=wd)     # torch's decay is the coupled one
+        th = th0.copy()
+        for t in range(4):
+            g = rng.standard_normal(37)
+            th = O.step(th, g, st, c, 37, 1)
+            p.grad = torch.tensor(g, dtype=torch.float64)
+            opt.step()
+        np.testing.assert_allclose(th, p.detach().numpy(), rtol=1e-13, atol=1e-15)
+    # decoupled decay: theta (1 - lr wd) - lr g, by hand
+    c = O.Config(0, 0, 1, 0, 32, lr=0.5, weight_decay=0.2)
+    np.testing.assert_allclose(O.step(np.array([2.0]), np.array([1.0]), O.step_init(c, 1, 1, 1), c, 1, 1), [2.0 * 0.9 - 0.5])
+    assert O.state_bytes(c, 100, 100, 1) == 0
+
+
+def test_bf16_state_rules_store_rounded_moments_and_update_with_unrounded_ones():
+    rng = np.random.default_rng(11)
+    n = 300
+    g_seq = [O.round_bf16(rng.standard_normal(n) * 0.01) for _ in range(5)]
+    for full, half in ((O.Config(1, 1, 1, 0, 32, weight_decay=0.01), O.Config(1, 1, 1, 0, 16, weight_decay=0.01)),
+                       (O.Config(1, 0, 1, 0, 32), O.Config(1, 0, 1, 0, 16)),
+                       (O.Config(0, 1, 0, 0, 32, lr=1e-2, weight_decay=0.1), O.Config(0, 1, 0, 0, 16, lr=1e-2, weight_decay=0.1))):
+        s32, s16 = O.step_init(full, n, n, 1), O.step_init(half, n, n, 1)
+        th32 = th16 = rng.standard_normal(n) * 0.02
+        # first step from the zero state: same update (the un-rounded moments are used), stored moments are the bf16
+        # roundings of the fp32-path moments
+        th32 = O.step(th32, g_seq[0], s32, full, n, 1)
+        th16 = O.step(th16, g_seq[0], s16, half, n, 1)
+        np.testing.assert_array_equal(th32, th16)
+        for name in ("m", "v"):
+            a32, a16 = getattr(s32, name), getattr(s16, name)
+            if a32 is not None:
+                np.testing.assert_array_equal(a16, O.round_bf16(a32))
+                assert np.all(np.abs(a16 - a32) <= np.abs(a32) * 2.0 ** -8)           # half a bf16 spacing at most
+        # later steps start from the rounded state: stays within bf16 resolution of the fp32 path, but differs
+        for g in g_seq[1:]:
+            th32 = O.step(th32, g, s32, full, n, 1)
+            th16 = O.step(th16, g, s16, half, n, 1)
+        assert 0 < np.max(np.abs(th32 - th16)) < 1e-2 * np.max(np.abs(th32))
+        for name in ("m", "v"):
+            a16 = getattr(s16, name)
+            if a16 is not None:
+                np.testing.assert_array_equal(a16, O.round_bf16(a16))                     # the state is always bf16
+    assert O.state_bytes(O.Config(1, 1, 1, 0, 16), 1000, 1000, 1) == 4000
+    assert O.state_bytes(O.Config(0, 1, 1, 0, 16), 1000, 1000, 1) == 2000
