@@ -105,7 +105,7 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
     }
     if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[1]), s), "baoc_step (profile)");
     LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles), at<const void*>(h->st, L.grads),
-                             at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), h->n_step_tiles, P, s),
+                             at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), h->n_step_tiles, h->wide_paths, P, s),
            "fused_step_kernel");
     h->launches += 1;
     if (h->prof_on) {
@@ -326,6 +326,8 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
     h->h_step_blocks = sb;
     h->n_step_tiles = int64_t(tiles.size()); h->n_step_red_tiles = int64_t(red.size());
     h->n_factored = int(ids.size());
+    h->wide_paths = false;
+    for (const StepBlock& b : sb) h->wide_paths = h->wide_paths || b.path >= kPathG;
     h->state_mem = mem; h->step_bytes = traffic;
     h->last_step_grads.clear(); h->last_step_params.clear();
     return BAOC_OK;

@@ -43,7 +43,7 @@ double step_traffic_bytes(const baoc_config_t& c, const baoc_block_t& b) {
 RedGeom red_geometry(int32_t rows, int32_t cols) {
     RedGeom g{};
     g.rowpart = nullptr; g.colpart = nullptr; g.red0 = -1;
-    g.L = int32_t(std::max<int64_t>(1, ceil_div(rows, int64_t(kRedRows) * 64)));
+    g.L = int32_t(std::max<int64_t>(1, ceil_div(rows, int64_t(kRedRows) * 16)));   // about 16 row chunks per matrix
     g.chunks = int32_t(ceil_div(rows, int64_t(kRedRows) * g.L));
     g.strips = int32_t(ceil_div(cols, kRedCols));
     return g;

@@ -171,6 +171,7 @@ struct Handle {
     int64_t n_step_tiles = 0;
     int64_t n_step_red_tiles = 0;
     int n_factored = 0;              // blocks on the factored path
+    bool wide_paths = false;         // some block is on a path outside the five headline ones
     int64_t state_mem = 0;           // StateMem of the assignment (sum of M_{i,c_i})
     int64_t step_bytes = 0;          // algorithmic bytes of one step
     std::vector<const void*> last_step_grads;
@@ -215,7 +216,7 @@ int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const i
 int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const int32_t* ids, const void* const* grads,
                            const float* const* params, int64_t n_red, int n_factored, const StepParams& P, cudaStream_t s);
 int launch_fused_step(const StepBlock* blocks, const Tile* tiles, const void* const* grads, float* const* params,
-                      uint32_t* flags, int64_t n_tiles, const StepParams& P, cudaStream_t s);
+                      uint32_t* flags, int64_t n_tiles, bool all_paths, const StepParams& P, cudaStream_t s);
 int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayout* out,
                         std::vector<StepBlock>* blocks, std::vector<Tile>* tiles,
                         std::vector<RedTile>* red, int64_t* state_mem, int64_t* step_bytes);

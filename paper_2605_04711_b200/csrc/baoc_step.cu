@@ -54,8 +54,8 @@ __device__ __forceinline__ void load8(const void* src, const float* th, float wd
 template <bool kSquare>
 __device__ __forceinline__ void rowcol_reduce_piece(const void* src, const float* th, float wd, int rows, int cols,
                                                     const RedGeom geo, uint32_t chunk, uint32_t strip) {
-    __shared__ float sh_row[kRedRows][65];
-    __shared__ float sh_col[4][kRedCols];
+    __shared__ float sh_row[2][kRedRows][65];                      // two buffers: one barrier per 64 rows, the sums of one
+    __shared__ float sh_col[4][kRedCols];                          // group overlap the loads of the next
     const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
     const int col0 = int(strip) * kRedCols + tx * 8;
     const int valid = max(0, min(8, cols - col0));
@@ -100,19 +100,19 @@ __device__ __forceinline__ void rowcol_reduce_piece(const void* src, const float
                 rowacc[k] = s;
             }
         }
+        float (*buf)[65] = sh_row[l & 1];
 #pragma unroll
-        for (int k = 0; k < kRedRows / 4; ++k) sh_row[ty + 4 * k][tx] = rowacc[k];
-        __syncthreads();
+        for (int k = 0; k < kRedRows / 4; ++k) buf[ty + 4 * k][tx] = rowacc[k];
+        __syncthreads();                                            // the buffer written two groups ago is free again by now
         if (threadIdx.x < kRedRows) {
             const int64_t r = r0 + threadIdx.x;
             if (r < rows) {
                 double s = 0.0;
 #pragma unroll 8
-                for (int j = 0; j < 64; ++j) s += double(sh_row[threadIdx.x][j]);
+                for (int j = 0; j < 64; ++j) s += double(buf[threadIdx.x][j]);
                 geo.rowpart[size_t(strip) * rows + r] = s;
             }
         }
-        __syncthreads();
     }
 #pragma unroll
     for (int j = 0; j < 8; ++j) sh_col[ty][tx * 8 + j] = colacc[j];
@@ -773,6 +773,11 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
     return !isfinite(c0) | !isfinite(c1);
 }
 
+// Two instances of the kernel: the first holds the five headline paths only, the second all paths.  Compiled next
+// to the headline paths, the bf16-state and stateless variants cost those paths registers at the 80-register budget
+// of three CTAs per SM (2-3 % of the step), so the host launches the wider instance only when the assignment uses
+// one of them.  Either way a step is one launch.
+template <bool kAllPaths>
 __global__ void __launch_bounds__(kThreads, 3)
 fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
                   const void* const* __restrict__ grads, float* const* __restrict__ params,
@@ -789,10 +794,10 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
         case kPathA32: bad = tile_dense<true, true, false>(b, P, g, th, base); break;
         case kPathR: bad = tile_dense<false, true, false>(b, P, g, th, base); break;
         case kPathS: bad = tile_dense<true, false, false>(b, P, g, th, base); break;
-        case kPathG: bad = tile_dense<false, false, false>(b, P, g, th, base); break;
-        case kPathA16: bad = tile_dense<true, true, true>(b, P, g, th, base); break;
-        case kPathR16: bad = tile_dense<false, true, true>(b, P, g, th, base); break;
-        case kPathS16: bad = tile_dense<true, false, true>(b, P, g, th, base); break;
+        case kPathG: if (kAllPaths) bad = tile_dense<false, false, false>(b, P, g, th, base); break;
+        case kPathA16: if (kAllPaths) bad = tile_dense<true, true, true>(b, P, g, th, base); break;
+        case kPathR16: if (kAllPaths) bad = tile_dense<false, true, true>(b, P, g, th, base); break;
+        case kPathS16: if (kAllPaths) bad = tile_dense<true, false, true>(b, P, g, th, base); break;
         case kPathA8: bad = P.coupled ? tile_int8<true>(b, P, g, th, base, q_stage) : tile_int8<false>(b, P, g, th, base, q_stage); break;
         case kPathF: bad = tile_factored(b, P, g, th, base, q_stage); break;
         default: break;
@@ -828,8 +833,9 @@ int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const
 }
 
 int launch_fused_step(const StepBlock* blocks, const Tile* tiles, const void* const* grads, float* const* params,
-                      uint32_t* flags, int64_t n_tiles, const StepParams& P, cudaStream_t s) {
-    fused_step_kernel<<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
+                      uint32_t* flags, int64_t n_tiles, bool all_paths, const StepParams& P, cudaStream_t s) {
+    if (all_paths) fused_step_kernel<true><<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
+    else fused_step_kernel<false><<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
     BAOC_LAUNCH_CHECK();
     return 0;
 }
