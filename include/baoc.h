@@ -185,6 +185,25 @@ int baoc_risk_from_raw(const baoc_t* h, baoc_block_stats_t* stats, double* risk_
  * Either output may be NULL.  Host only. */
 int baoc_cost_model(const baoc_t* h, int64_t* mem_bytes, double* time_ratio);
 
+/* Measured cost model (Sec. 3.1, "Time Budget Definition": r_{i,c} = t_{i,c} /
+ * t_{i,base} from a one-step timing of updating block i with configuration c on
+ * the target hardware and the same tensor shapes).  For every pair the library
+ * can instantiate, the block alone is stepped `reps` times (after one warm-up)
+ * under that configuration with the learning rate forced to 0, timed with CUDA
+ * events on the stream; time_ratio_out[i*n_cfg+c] = t_{i,c} / t_{i,base_cfg}
+ * (pairs that cannot be assigned keep the value of baoc_cost_model);
+ * time_ms_out (may be NULL) gets the milliseconds, -1 for unmeasured pairs.
+ * With lr = 0 the parameters come out bit-identical provided eps > 0 for the
+ * adaptive tuples; the handle's own statistics and optimizer state are not
+ * touched: the states of the timed steps live in scratch_dev (device, 256-byte
+ * aligned, >= baoc_time_scratch_bytes).  grads / params: host arrays of
+ * n_blocks device pointers as in baoc_step.  Waits for the stream many times; a
+ * warm-up-time helper, not part of the training loop. */
+int baoc_time_scratch_bytes(const baoc_t* h, size_t* bytes);
+int baoc_measure_time_ratios(baoc_t* h, const void* const* grads, float* const* params, void* scratch_dev,
+                             size_t scratch_bytes, int base_cfg, int reps, double* time_ratio_out,
+                             double* time_ms_out, baoc_stream_t stream);
+
 /* Solve Eq. 2 exactly on the host: minimise sum_i Phi_{i,c_i} with
  * Phi = (R - pref) + gamma*Agg(c) subject to sum M <= b_mem and
  * (1/N) sum r <= b_time, one configuration per block.  Arithmetic is fixed

@@ -75,7 +75,7 @@ EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error"
            "baoc_risk", "baoc_risk_from_raw", "baoc_cost_model", "baoc_allocate", "baoc_state_bytes",
            "baoc_configure", "baoc_step", "baoc_step_from_host", "baoc_view", "baoc_nonfinite",
            "baoc_sample_stats_noalloc", "baoc_noalloc_last_error", "baoc_profile", "baoc_profile_last",
-           "baoc_export", "baoc_import"]
+           "baoc_export", "baoc_import", "baoc_time_scratch_bytes", "baoc_measure_time_ratios"]
 
 _vp = C.c_void_p
 _lib.baoc_default_opts.argtypes = [C.POINTER(Opts)]
@@ -100,6 +100,8 @@ _lib.baoc_step.argtypes = [_vp, _vp, _vp, C.c_int64, _vp]
 _lib.baoc_step_from_host.argtypes = [_vp, _vp, _vp, _vp, C.c_int, C.c_int64, _vp]
 _lib.baoc_view.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(_vp), C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
 _lib.baoc_nonfinite.argtypes = [_vp, _vp, C.POINTER(C.c_int32), _vp]
+_lib.baoc_time_scratch_bytes.argtypes = [_vp, C.POINTER(C.c_size_t)]
+_lib.baoc_measure_time_ratios.argtypes = [_vp, _vp, _vp, _vp, C.c_size_t, C.c_int, C.c_int, _vp, _vp, _vp]
 _lib.baoc_export.argtypes = [_vp, _vp, C.c_size_t, C.POINTER(C.c_size_t)]
 _lib.baoc_import.argtypes = [_vp, _vp, C.c_size_t, _vp, C.c_size_t, _vp, C.c_size_t, _vp]
 _lib.baoc_profile.argtypes = [_vp, C.c_int]
@@ -261,6 +263,21 @@ class Baoc:
         rc = self._check(_lib.baoc_allocate(self._h, risk.ctypes.data, mem.ctypes.data, ratio.ctypes.data, int(b_mem),
                                             float(b_time), _np_ptr(forbid), _np_ptr(pref), asg.ctypes.data, C.byref(obj)))
         return asg, obj.value, rc
+
+    def time_scratch_bytes(self) -> int:
+        n = C.c_size_t()
+        self._check(_lib.baoc_time_scratch_bytes(self._h, C.byref(n)))
+        return n.value
+
+    def measure_time_ratios(self, grads, params, scratch: torch.Tensor, base_cfg: int = 0, reps: int = 3):
+        """``baoc_measure_time_ratios``: (ratio [n_blocks, n_cfg], milliseconds [n_blocks, n_cfg])."""
+        g = grads if isinstance(grads, C.Array) else pointer_table(grads)
+        p = params if isinstance(params, C.Array) else pointer_table(params)
+        ratio = np.zeros((self.n_blocks, self.n_cfg), np.float64)
+        ms = np.zeros((self.n_blocks, self.n_cfg), np.float64)
+        self._check(_lib.baoc_measure_time_ratios(self._h, g, p, scratch.data_ptr(), scratch.numel() * scratch.element_size(),
+                                                  int(base_cfg), int(reps), ratio.ctypes.data, ms.ctypes.data, _stream()))
+        return ratio, ms
 
     # ---- training ---------------------------------------------------------
     def state_bytes(self, assign) -> int:

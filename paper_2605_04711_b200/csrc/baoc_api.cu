@@ -337,6 +337,98 @@ int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t byt
     return configure_state(h, assign, state_dev, bytes, stream, true);
 }
 
+// ---- one-step timing of every (block, configuration) pair ---------------------------
+namespace {
+size_t single_block_state_bytes(const Handle* h, int block, int cfg) {
+    baoc_handle one;
+    one.n_blocks = 1; one.n_cfg = h->n_cfg; one.blocks.assign(1, h->blocks[block]); one.cfgs = h->cfgs; one.opts = h->opts;
+    one.numel = h->blocks[block].numel;
+    Handle::StepLayout L{};
+    const int32_t a = cfg;
+    if (compute_step_layout(&one, &a, &L, nullptr, nullptr, nullptr, nullptr, nullptr) != BAOC_OK) return 0;
+    return L.total;
+}
+bool assignable(const Handle* h, int block, int cfg) {
+    const Path p = path_of(h->cfgs[cfg]);
+    return p != kPathNone && !(p == kPathF && h->blocks[block].cols <= 1);
+}
+}  // namespace
+
+int baoc_time_scratch_bytes(const baoc_t* h, size_t* bytes) {
+    if (!h) return BAOC_E_INVALID;
+    if (!bytes) return fail(h, BAOC_E_INVALID, "baoc_time_scratch_bytes: null output");
+    size_t need = 0;
+    for (int i = 0; i < h->n_blocks; ++i)
+        for (int c = 0; c < h->n_cfg; ++c)
+            if (assignable(h, i, c)) need = std::max(need, single_block_state_bytes(h, i, c));
+    *bytes = need;
+    return BAOC_OK;
+}
+
+int baoc_measure_time_ratios(baoc_t* h, const void* const* grads, float* const* params, void* scratch_dev,
+                             size_t scratch_bytes, int base_cfg, int reps, double* time_ratio_out,
+                             double* time_ms_out, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!grads || !params || !scratch_dev || !time_ratio_out) return fail(h, BAOC_E_INVALID, "baoc_measure_time_ratios: null argument");
+    if (base_cfg < 0 || base_cfg >= h->n_cfg || reps < 1 || reps > 1000) return fail(h, BAOC_E_INVALID, "baoc_measure_time_ratios: bad base configuration or repetition count");
+    if (reinterpret_cast<uintptr_t>(scratch_dev) & 255u) return fail(h, BAOC_E_ALIGN, "baoc_measure_time_ratios: scratch not 256-byte aligned");
+    size_t need = 0;
+    baoc_time_scratch_bytes(h, &need);
+    if (scratch_bytes < need) return fail(h, BAOC_E_WORKSPACE, "baoc_measure_time_ratios: scratch too small");
+    for (int i = 0; i < h->n_blocks; ++i) {
+        if (!grads[i] || !params[i]) return fail(h, BAOC_E_INVALID, "baoc_measure_time_ratios: null block pointer");
+        if (!aligned16(grads[i]) || !aligned16(params[i])) return fail(h, BAOC_E_ALIGN, "baoc_measure_time_ratios: block pointer not 16-byte aligned");
+        if (!assignable(h, i, base_cfg)) return fail(h, BAOC_E_INVALID, "baoc_measure_time_ratios: the base configuration cannot be assigned to every block");
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaEvent_t e0, e1;
+    CU(cudaEventCreate(&e0), "baoc_measure_time_ratios");
+    if (cudaEventCreate(&e1) != cudaSuccess) { cudaEventDestroy(e0); return fail(h, BAOC_E_CUDA, "baoc_measure_time_ratios: event creation failed"); }
+    const int K = h->n_cfg;
+    std::vector<double> ms(size_t(h->n_blocks) * K, -1.0);
+    int rc = BAOC_OK;
+    for (int i = 0; i < h->n_blocks && rc == BAOC_OK; ++i) {
+        // a one-block handle with every learning rate at zero: the step runs at full cost, the parameters come
+        // out bit-identical (theta * (1 - 0) - 0 * direction) and only the scratch state is written
+        baoc_handle one;
+        one.n_blocks = 1; one.n_cfg = K; one.blocks.assign(1, h->blocks[i]); one.cfgs = h->cfgs; one.opts = h->opts;
+        one.numel = h->blocks[i].numel;
+        for (baoc_config_t& c : one.cfgs) c.lr = 0.0f;
+        const void* g1[1] = {grads[i]};
+        float* p1[1] = {params[i]};
+        for (int c = 0; c < K && rc == BAOC_OK; ++c) {
+            if (!assignable(h, i, c)) continue;
+            const int32_t a = c;
+            rc = configure_state(&one, &a, scratch_dev, scratch_bytes, stream, true);
+            if (rc == BAOC_OK) rc = do_step(&one, g1, p1, 1, s);                       // warm-up (also uploads the pointer tables)
+            if (rc != BAOC_OK) break;
+            cudaEventRecord(e0, s);
+            for (int r = 0; r < reps && rc == BAOC_OK; ++r) rc = do_step(&one, g1, p1, 2 + r, s);
+            cudaEventRecord(e1, s);
+            if (rc != BAOC_OK) break;
+            float t = 0.f;
+            if (cudaEventSynchronize(e1) != cudaSuccess || cudaEventElapsedTime(&t, e0, e1) != cudaSuccess) { rc = BAOC_E_CUDA; one.err = "event timing failed"; break; }
+            ms[size_t(i) * K + c] = double(t) / reps;
+        }
+        if (rc != BAOC_OK) h->err = "baoc_measure_time_ratios: " + one.err;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (rc != BAOC_OK) return rc;
+    std::vector<double> model(size_t(h->n_blocks) * K);
+    baoc_cost_model(h, nullptr, model.data());
+    for (int i = 0; i < h->n_blocks; ++i) {
+        const double base = ms[size_t(i) * K + base_cfg];
+        for (int c = 0; c < K; ++c) {
+            const size_t k = size_t(i) * K + c;
+            // pairs that cannot be assigned keep the bytes model's value (the allocator masks them anyway)
+            time_ratio_out[k] = (ms[k] >= 0.0 && base > 0.0) ? ms[k] / base : model[k];
+            if (time_ms_out) time_ms_out[k] = ms[k];
+        }
+    }
+    return BAOC_OK;
+}
+
 // ---- checkpoint / resume ---------------------------------------------------------
 namespace {
 struct BlobHeader {

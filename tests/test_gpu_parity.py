@@ -388,6 +388,45 @@ def test_gpu_argument_checks(B, H):
     assert e.value.code == B.E_STATE
 
 
+def test_measured_time_ratios_leave_parameters_and_state_alone(B, H):
+    """The one-step timing helper (Sec. 3.1, time budget): ratios are positive, 1 for the base configuration,
+    the bytes model's value where a pair cannot be assigned; parameters, window and optimizer state are untouched."""
+    blocks = [W.Block("big", 2048, 2048, stability=0.5), W.Block("wide", 512, 4096, stability=0.5),
+              W.Block("vec", 4096, 1, stability=0.5), W.Block("tiny", 7, 1, stability=0.5)]
+    wl = W.Workload("timing", blocks, window=2, mem_budget_frac=0.5, time_budget=1.3, seed=77)
+    sess = H.Session(wl, configs=B.extended_configs(), n_grad_sets=1)
+    sess.init_params()
+    sess.fill_grads(1)
+    sess.sample_stats(0)
+    sess.configure([0, 1, 2, 4])
+    sess.step(0, 1)
+    torch.cuda.synchronize()
+    before = (sess.params.clone(), sess.ws.clone(), sess.state.clone())
+    scratch = torch.empty(sess.h.time_scratch_bytes(), dtype=torch.uint8, device=sess.device)
+    ratio, ms = sess.h.measure_time_ratios(sess.grad_tables[0], sess.param_table, scratch, base_cfg=0, reps=3)
+    torch.cuda.synchronize()
+    assert torch.equal(before[0], sess.params) and torch.equal(before[1], sess.ws) and torch.equal(before[2], sess.state)
+    _, model = sess.h.cost_model()
+    n_cfg = len(sess.configs)
+    for i, b in enumerate(blocks):
+        assert ratio[i, 0] == 1.0
+        for c in range(n_cfg):
+            if c == 3 and b.cols <= 1:                               # factored on a vector: not measurable
+                assert ms[i, c] == -1.0 and ratio[i, c] == model[i, c]
+            else:
+                assert ms[i, c] > 0.0 and 0.05 < ratio[i, c] < 20.0
+    # on the 4 M-element matrix the step is bandwidth-bound: lighter configurations are measurably cheaper
+    assert ratio[0, 5] < 0.8 and ratio[0, 4] < 0.95 and ratio[0, 2] < 0.95          # plain SGD, SGD-m, RMS vs fp32 Adam
+    # the measured table is a valid input of the allocator
+    risk = np.zeros((len(blocks), n_cfg))
+    mem, _ = sess.h.cost_model()
+    asg, _, rc = sess.h.allocate(risk, mem, ratio, int(8 * wl.numel), 1.3)
+    assert rc == 0 and len(asg) == len(blocks)
+    with pytest.raises(B.BaocError) as e:
+        sess.h.measure_time_ratios(sess.grad_tables[0], sess.param_table, scratch, base_cfg=3)   # cannot be the base: vectors
+    assert e.value.code == B.E_INVALID
+
+
 def test_checkpoint_resume_continues_bit_exactly(B, H):
     """Export after a window and some steps, move every buffer to a new address, import into a fresh handle, and
     let both handles continue on the same gradients: parameters, states and running statistics stay identical."""
