@@ -447,15 +447,15 @@ class StepState:
 def config_kind(c: Config) -> str:
     """Which update path a tuple selects.  A32 / A16 / A8: Adam with fp32 / bf16 / 8-bit moments; R / R16:
     momentum-free RMS scaling; F: factored second moment; S / S16: SGD with momentum; G: plain gradient step
-    (neither mechanism, hence no state, whatever bit-width the tuple names)."""
+    (neither mechanism, hence no state, whatever bit-width the tuple names); R8 / S8: the 8-bit forms of R / S."""
     if c.factored:
         return "F" if (c.adaptive and not c.momentum and c.bits == 32) else "unsupported"
     if c.adaptive and c.momentum:
         return {32: "A32", 16: "A16", 8: "A8"}[c.bits]
     if c.adaptive and not c.momentum:
-        return {32: "R", 16: "R16"}.get(c.bits, "unsupported")
+        return {32: "R", 16: "R16", 8: "R8"}[c.bits]
     if not c.adaptive and c.momentum:
-        return {32: "S", 16: "S16"}.get(c.bits, "unsupported")
+        return {32: "S", 16: "S16", 8: "S8"}[c.bits]
     return "G"
 
 
@@ -470,6 +470,10 @@ def step_init(c: Config, numel: int, rows: int, cols: int, qblock: int = 256) ->
         return StepState(kind, m=np.zeros(numel, F64))
     if kind == "G":
         return StepState(kind)
+    if kind == "R8":
+        return StepState(kind, qv=np.zeros(numel, np.uint8), av=np.zeros(nq, np.float32))
+    if kind == "S8":
+        return StepState(kind, qm=np.zeros(numel, np.int8), am=np.zeros(nq, np.float32))
     if kind == "A8":
         return StepState(kind, qm=np.zeros(numel, np.int8), qv=np.zeros(numel, np.uint8),
                          am=np.zeros(nq, np.float32), av=np.zeros(nq, np.float32))
@@ -514,6 +518,19 @@ def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, 
         return theta - c.lr * m
     if st.kind == "G":
         return theta - c.lr * g
+    # 8-bit single-moment rules: dequantise, update, use the un-requantised moment, requantise (as in A8)
+    if st.kind == "R8":
+        v = dequantize8(st.qv, st.av, False, qblock)
+        v = c.beta2 * v + (1.0 - c.beta2) * g * g
+        theta = _adam_apply(theta, g, v, c, t, False)
+        st.qv, st.av = quantize8(v, False, qblock)
+        return theta
+    if st.kind == "S8":
+        m = dequantize8(st.qm, st.am, True, qblock)
+        m = c.beta1 * m + g
+        theta = theta - c.lr * m
+        st.qm, st.am = quantize8(m, True, qblock)
+        return theta
     if st.kind == "A8":
         m = dequantize8(st.qm, st.am, True, qblock)
         v = dequantize8(st.qv, st.av, False, qblock)

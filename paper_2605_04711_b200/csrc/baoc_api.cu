@@ -80,6 +80,7 @@ void fill_step_params(const Handle* h, int64_t t, StepParams* P) {
         o.step_g = k.lr;
         o.rsqrt_bc2 = float(1.0 / std::sqrt(bc2));
         o.step_m_hat = float(lr / bc1 * std::sqrt(bc2));
+        o.step_g_hat = float(lr * std::sqrt(bc2));
         o.eps_hat = float(double(k.eps) * std::sqrt(bc2));
         o.beta1_d = b1; o.beta2_d = b2; o.wd_d = double(k.weight_decay);
     }
@@ -304,6 +305,8 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
         StepBlock& b = sb[i];
         auto fix = [&](void* p) { return static_cast<void*>(st + L.states + reinterpret_cast<size_t>(p)); };
         if (b.path == kPathA32 || b.path == kPathA8 || b.path == kPathF || b.path == kPathA16) { b.s0 = fix(b.s0); b.s1 = fix(b.s1); }
+        else if (b.path == kPathR8) { b.s1 = fix(b.s1); b.a1 = static_cast<float*>(fix(b.a1)); }
+        else if (b.path == kPathS8) { b.s0 = fix(b.s0); b.a0 = static_cast<float*>(fix(b.a0)); }
         else if (b.path != kPathG) b.s0 = fix(b.s0);
         if (b.path == kPathA8) { b.a0 = static_cast<float*>(fix(b.a0)); b.a1 = static_cast<float*>(fix(b.a1)); }
         if (b.path == kPathF) {
@@ -598,6 +601,8 @@ int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* co
             case kPathR: case kPathS: if (k == 0) { p = s.s0; n = b.numel; } break;
             case kPathA16: if (k == 0) { p = s.s0; n = b.numel; eb = 2; } else if (k == 1) { p = s.s1; n = b.numel; eb = 2; } break;
             case kPathR16: case kPathS16: if (k == 0) { p = s.s0; n = b.numel; eb = 2; } break;
+            case kPathR8: if (k == 0) { p = s.s1; n = b.numel; eb = 1; } else if (k == 1) { p = s.a1; n = nq; } break;
+            case kPathS8: if (k == 0) { p = s.s0; n = b.numel; eb = 1; } else if (k == 1) { p = s.a0; n = nq; } break;
             case kPathF: if (k == 0) { p = s.s0; n = b.rows; } else if (k == 1) { p = s.s1; n = b.cols; } break;
             default: break;
         }

@@ -143,6 +143,8 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
             case kPathR: case kPathS: s.s0 = place(4 * dpad); break;
             case kPathA16: s.s0 = place(2 * dpad); s.s1 = place(2 * dpad); break;
             case kPathR16: case kPathS16: s.s0 = place(2 * dpad); break;
+            case kPathR8: s.s1 = place(dpad); s.a1 = static_cast<float*>(place(4 * nq)); break;
+            case kPathS8: s.s0 = place(dpad); s.a0 = static_cast<float*>(place(4 * nq)); break;
             case kPathG: break;
             case kPathF: {
                 s.s0 = place(4 * size_t(b.rows)); s.s1 = place(4 * size_t(b.cols));
@@ -164,7 +166,7 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
         traffic += step_traffic_bytes(h->cfgs[c], b);
     }
     // tiles in descending bytes per element so that the light ones fill the tail of the grid
-    const int order[kPathCount] = {kPathA32, kPathR, kPathS, kPathA16, kPathR16, kPathS16, kPathG, kPathA8, kPathF};
+    const int order[kPathCount] = {kPathA32, kPathR, kPathS, kPathA16, kPathR16, kPathS16, kPathG, kPathA8, kPathR8, kPathS8, kPathF};
     for (int p : order)
         for (int i = 0; i < n; ++i)
             if (sb[i].path == p) {

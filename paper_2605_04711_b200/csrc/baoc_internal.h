@@ -37,20 +37,24 @@ enum Path : int32_t {
     kPathA16 = 6,        // Adam / AdamW with bf16 moments
     kPathR16 = 7,        // momentum-free RMS scaling with a bf16 second moment
     kPathS16 = 8,        // SGD with a bf16 momentum buffer
-    kPathCount = 9,
+    kPathR8 = 9,         // momentum-free RMS scaling with a block-wise absmax 8-bit second moment
+    kPathS8 = 10,        // SGD with a block-wise absmax 8-bit momentum buffer
+    kPathCount = 11,
     kPathNone = -1
 };
 
 inline Path path_of(const baoc_config_t& c) {
     if (c.factored) return (c.adaptive && !c.momentum && c.bits == 32) ? kPathF : kPathNone;
     if (c.adaptive && c.momentum) return c.bits == 32 ? kPathA32 : (c.bits == 16 ? kPathA16 : kPathA8);
-    if (c.adaptive && !c.momentum) return c.bits == 32 ? kPathR : (c.bits == 16 ? kPathR16 : kPathNone);
-    if (!c.adaptive && c.momentum) return c.bits == 32 ? kPathS : (c.bits == 16 ? kPathS16 : kPathNone);
+    if (c.adaptive && !c.momentum) return c.bits == 32 ? kPathR : (c.bits == 16 ? kPathR16 : kPathR8);
+    if (!c.adaptive && c.momentum) return c.bits == 32 ? kPathS : (c.bits == 16 ? kPathS16 : kPathS8);
     return kPathG;       // neither mechanism: stateless, whatever bit-width the tuple names
 }
 
 // Elements per tile of the fused step, by update path.
-inline int64_t step_tile_elems(int path) { return path == kPathF ? kTileF : (path == kPathA8 ? kTileQ : kTile); }
+inline int64_t step_tile_elems(int path) {
+    return path == kPathF ? kTileF : ((path == kPathA8 || path == kPathR8 || path == kPathS8) ? kTileQ : kTile);
+}
 
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
@@ -126,6 +130,7 @@ struct CfgStep {
     float step_m;        // lr / (1 - beta1^t): multiplies a bias-corrected first moment
     float step_g;        // lr: multiplies a raw gradient or momentum buffer
     float rsqrt_bc2;     // 1 / sqrt(1 - beta2^t)
+    float step_g_hat;    // lr * sqrt(1 - beta2^t)
     float step_m_hat;    // step_m * sqrt(1 - beta2^t): with eps_hat the update is step_m_hat * m / (sqrt(v) + eps_hat)
     float eps_hat;       // eps * sqrt(1 - beta2^t)
     int32_t coupled;     // 1: add wd*theta to the gradient

@@ -542,14 +542,15 @@ __device__ __forceinline__ Q8Raw q8_fetch(int src, int j, const uint4& wg, const
 }
 
 // Exact (double) new moment of one element: first moment for group 0, second for group 1.
-template <bool kCoupled>
+// kUnitGain: the first moment is a momentum buffer mu m + g rather than an average beta1 m + (1 - beta1) g.
+template <bool kCoupled, bool kUnitGain>
 __device__ __forceinline__ double q8_exact(const Q8Raw& r, bool second, float am_old, float av_old, const CfgStep& P) {
     double gd = widen_bf16_float(__uint_as_float(r.gbits << 16));
     if (kCoupled) gd += P.wd_d * double(r.theta);
     const double beta = second ? P.beta2_d : P.beta1_d;
     const int code = second ? int(r.cv) : int(int8_t(r.cm));
     const double old = int_to_double(code) * (second ? double(av_old) * (1.0 / 255.0) : double(am_old) * (1.0 / 127.0));
-    return beta * old + (1.0 - beta) * (second ? gd * gd : gd);
+    return beta * old + ((kUnitGain && !second) ? 1.0 : 1.0 - beta) * (second ? gd * gd : gd);
 }
 
 // clamp(rne(L * x / a)) by the correctly rounded division.
@@ -563,7 +564,8 @@ __device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint3
     return __byte_perm(__byte_perm(a, b, 0x0040u), __byte_perm(c, d, 0x0040u), 0x5410u);
 }
 
-template <bool kCoupled>
+// kM / kV: which moments the configuration keeps (both: Adam; kV only: RMS scaling; kM only: SGD with momentum).
+template <bool kCoupled, bool kM, bool kV>
 __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep& P, const uint16_t* __restrict__ g,
                                               float* __restrict__ th, int64_t base, unsigned char* stage) {
     constexpr float kSlack = 4.76837158203125e-7f;                 // 2^-21
@@ -601,8 +603,8 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
             cp_async16(d + sg, gt + e);
             cp_async16(d + st_, tht + e);
             cp_async16(d + st_ + 16, tht + e + 4);
-            cp_async8(d + scm, qmt + e);
-            cp_async8(d + scv, qvt + e);
+            if (kM) cp_async8(d + scm, qmt + e);
+            if (kV) cp_async8(d + scv, qvt + e);
         }
         cp_async_commit();
         fill = fill == (kStagesQ - 1) * kStageBytes ? 0u : fill + kStageBytes;
@@ -611,7 +613,10 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
     auto absmax_of = [&](int s, float& a_m, float& a_v) {
         const int w = s * (kThreads * 8) + warp * kQBlock;
         a_m = 0.f; a_v = 0.f;
-        if (s < kSlicesQ && w < left) { a_m = amt[w / kQBlock]; a_v = avt[w / kQBlock]; }
+        if (s < kSlicesQ && w < left) {
+            if (kM) a_m = amt[w / kQBlock];
+            if (kV) a_v = avt[w / kQBlock];
+        }
     };
     float amo_1, avo_1, amo_2, avo_2;
 #pragma unroll
@@ -638,14 +643,14 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
             wg = *reinterpret_cast<const uint4*>(mine + sg);
             t0 = *reinterpret_cast<const float4*>(mine + st_);
             t1 = *reinterpret_cast<const float4*>(mine + st_ + 16);
-            wm = *reinterpret_cast<const uint2*>(mine + scm);
-            wv = *reinterpret_cast<const uint2*>(mine + scv);
+            wm = kM ? *reinterpret_cast<const uint2*>(mine + scm) : make_uint2(0u, 0u);
+            wv = kV ? *reinterpret_cast<const uint2*>(mine + scv) : make_uint2(0u, 0u);
         } else {                                                    // ragged end of the block: zero-fill
             const int n = cnt;
             auto gg = [&](int j) { return j < n ? uint32_t(gt[e + j]) : 0u; };
             auto tt = [&](int j) { return j < n ? tht[e + j] : 0.f; };
-            auto mm = [&](int j) { return j < n ? uint32_t(uint8_t(qmt[e + j])) : 0u; };
-            auto vv = [&](int j) { return j < n ? uint32_t(qvt[e + j]) : 0u; };
+            auto mm = [&](int j) { return (kM && j < n) ? uint32_t(uint8_t(qmt[e + j])) : 0u; };
+            auto vv = [&](int j) { return (kV && j < n) ? uint32_t(qvt[e + j]) : 0u; };
             wg = make_uint4(gg(0) | gg(1) << 16, gg(2) | gg(3) << 16, gg(4) | gg(5) << 16, gg(6) | gg(7) << 16);
             t0 = make_float4(tt(0), tt(1), tt(2), tt(3)); t1 = make_float4(tt(4), tt(5), tt(6), tt(7));
             wm = make_uint2(mm(0) | mm(1) << 8 | mm(2) << 16 | mm(3) << 24, mm(4) | mm(5) << 8 | mm(6) << 16 | mm(7) << 24);
@@ -662,7 +667,7 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         const uint32_t gw[4] = {wg.x, wg.y, wg.z, wg.w};
         const uint32_t ms[2] = {wm.x ^ 0x80808080u, wm.y ^ 0x80808080u};
         const uint32_t vs[2] = {wv.x, wv.y};
-        f32x2 T[4], MF[4], VF[4];
+        f32x2 T[4], MF[4], VF[4], XE[4];                             // XE: effective gradients, kept only when they are the numerator
         float lm = 0.f, lv = 0.f;                                   // this lane's maxima
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
@@ -676,29 +681,37 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
                                         __uint_as_float(__byte_perm(mw, 0x4B000000u, 0x7440u | k1))), MOFF);
             const f32x2 FV = pack2(__uint_as_float(__byte_perm(vw, 0x4B000000u, 0x7440u | k0)),
                                    __uint_as_float(__byte_perm(vw, 0x4B000000u, 0x7440u | k1)));
-            MF[p] = fma2(FM, B1S, mul2(OM1, X));
-            VF[p] = fma2(mul2(OM2, X), X, fma2(FV, B2S, VB));
-            float a0, a1, c0, c1;
-            unpack2(MF[p], a0, a1); unpack2(VF[p], c0, c1);
-            lm = max3(lm, fabsf(a0), fabsf(a1)); lv = max3(lv, c0, c1);
+            float a0, a1;
+            if (kM) {                                               // Adam: beta1 m + (1 - beta1) g;  momentum SGD: mu m + g
+                MF[p] = fma2(FM, B1S, kV ? mul2(OM1, X) : X);
+                unpack2(MF[p], a0, a1);
+                lm = max3(lm, fabsf(a0), fabsf(a1));
+            }
+            if (kV) {
+                VF[p] = fma2(mul2(OM2, X), X, fma2(FV, B2S, VB));
+                unpack2(VF[p], a0, a1);
+                lv = max3(lv, a0, a1);
+                if (!kM) XE[p] = X;
+            }
         }
-        const float mx = warp_max_nonneg(lm), vx = warp_max_nonneg(lv);
+        const float mx = kM ? warp_max_nonneg(lm) : 0.f, vx = kV ? warp_max_nonneg(lv) : 0.f;
         const float Em = kSlack * (amo + mx), Ev = kSlack * (avo + vx);
 
         // ---- exact absmax
-        unsigned cand_m = __ballot_sync(full, lm >= mx - 2.0f * Em), cand_v = __ballot_sync(full, lv >= vx - 2.0f * Ev);
+        unsigned cand_m = kM ? __ballot_sync(full, lm >= mx - 2.0f * Em) : 0u;
+        unsigned cand_v = kV ? __ballot_sync(full, lv >= vx - 2.0f * Ev) : 0u;
         float am_c = 0.f, av_c = 0.f;
         while (cand_m | cand_v) {                                   // warp-uniform
             const int Lm = cand_m ? __ffs(cand_m) - 1 : -1, Lv = cand_v ? __ffs(cand_v) - 1 : -1;
             cand_m &= cand_m - 1u; cand_v &= cand_v - 1u;           // (0 & anything stays 0)
             const int src = hv_grp ? Lv : Lm;
             const Q8Raw r = q8_fetch<kCoupled>(max(src, 0), hj, wg, wm, wv, t0, t1);
-            const float val = __double2float_rn(fabs(q8_exact<kCoupled>(r, hv_grp, amo, avo, P)));
+            const float val = __double2float_rn(fabs(q8_exact<kCoupled, kM && !kV>(r, hv_grp, amo, avo, P)));
             if (helper && src >= 0) {
                 if (hv_grp) av_c = fmaxf(av_c, val); else am_c = fmaxf(am_c, val);
             }
         }
-        const float am_new = warp_max_nonneg(am_c), av_new = warp_max_nonneg(av_c);
+        const float am_new = kM ? warp_max_nonneg(am_c) : 0.f, av_new = kV ? warp_max_nonneg(av_c) : 0.f;
 
         // ---- codes: rne(q) = low byte of the float q + 1.5*2^23
         const float km = am_new > 0.f ? 127.0f / am_new : 0.f, kv = av_new > 0.f ? 255.0f / av_new : 0.f;
@@ -708,25 +721,32 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         float dm = 0.f, dv = 0.f;                                   // largest distance to the chosen integer in this lane
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
-            const f32x2 RM = fma2(MF[p], KM, MAGIC), RV = fma2(VF[p], KV, MAGIC);
-            const f32x2 DM = fma2(MF[p], KM, fma2(RM, MINUS1, MAGIC)), DV = fma2(VF[p], KV, fma2(RV, MINUS1, MAGIC));
             float r0, r1, d0, d1;
-            unpack2(RM, r0, r1); unpack2(DM, d0, d1);
-            cmw[2 * p] = __float_as_uint(r0); cmw[2 * p + 1] = __float_as_uint(r1);
-            dm = max3(dm, fabsf(d0), fabsf(d1));
-            unpack2(RV, r0, r1); unpack2(DV, d0, d1);
-            cvw[2 * p] = __float_as_uint(r0); cvw[2 * p + 1] = __float_as_uint(r1);
-            dv = max3(dv, fabsf(d0), fabsf(d1));
+            cmw[2 * p] = cmw[2 * p + 1] = cvw[2 * p] = cvw[2 * p + 1] = 0u;
+            if (kM) {
+                const f32x2 RM = fma2(MF[p], KM, MAGIC);
+                const f32x2 DM = fma2(MF[p], KM, fma2(RM, MINUS1, MAGIC));
+                unpack2(RM, r0, r1); unpack2(DM, d0, d1);
+                cmw[2 * p] = __float_as_uint(r0); cmw[2 * p + 1] = __float_as_uint(r1);
+                dm = max3(dm, fabsf(d0), fabsf(d1));
+            }
+            if (kV) {
+                const f32x2 RV = fma2(VF[p], KV, MAGIC);
+                const f32x2 DV = fma2(VF[p], KV, fma2(RV, MINUS1, MAGIC));
+                unpack2(RV, r0, r1); unpack2(DV, d0, d1);
+                cvw[2 * p] = __float_as_uint(r0); cvw[2 * p + 1] = __float_as_uint(r1);
+                dv = max3(dv, fabsf(d0), fabsf(d1));
+            }
         }
         uint2 om = make_uint2(pack_low_bytes(cmw[0], cmw[1], cmw[2], cmw[3]), pack_low_bytes(cmw[4], cmw[5], cmw[6], cmw[7]));
         uint2 ov = make_uint2(pack_low_bytes(cvw[0], cvw[1], cvw[2], cvw[3]), pack_low_bytes(cvw[4], cvw[5], cvw[6], cvw[7]));
-        unsigned slow_m = __ballot_sync(full, !(dm <= hm)), slow_v = __ballot_sync(full, !(dv <= hv));
+        unsigned slow_m = kM ? __ballot_sync(full, !(dm <= hm)) : 0u, slow_v = kV ? __ballot_sync(full, !(dv <= hv)) : 0u;
         while (slow_m | slow_v) {                                   // warp-uniform, rare
             const int Lm = slow_m ? __ffs(slow_m) - 1 : -1, Lv = slow_v ? __ffs(slow_v) - 1 : -1;
             slow_m &= slow_m - 1u; slow_v &= slow_v - 1u;
             const int src = hv_grp ? Lv : Lm;
             const Q8Raw r = q8_fetch<kCoupled>(max(src, 0), hj, wg, wm, wv, t0, t1);
-            const double x = q8_exact<kCoupled>(r, hv_grp, amo, avo, P);
+            const double x = q8_exact<kCoupled, kM && !kV>(r, hv_grp, amo, avo, P);
             const int code = hv_grp ? encode_exact(x, av_new, 255.0, 0) : encode_exact(x, am_new, 127.0, -127);
             const uint32_t piece = (helper && src >= 0) ? (uint32_t(code) & 0xffu) << (8 * (hj & 3)) : 0u;
             const uint32_t mlo = __reduce_or_sync(full, (!hv_grp && hj < 4) ? piece : 0u);
@@ -738,34 +758,42 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         }
 
         // ---- parameter update from the un-requantised fp32 moments
-        // theta <- theta - step_m_hat * m / (sqrt(v) + eps_hat), the bias correction of v folded into both constants
-        const f32x2 EPS = splat2(P.eps_hat), NSTEP = splat2(-P.step_m_hat);
+        // Adam: theta <- theta - step_m_hat * m / (sqrt(v) + eps_hat), the bias correction of v folded into both
+        // constants;  RMS scaling: the same with the effective gradient and step_g_hat;  momentum SGD: theta - lr * m
+        const f32x2 EPS = splat2(P.eps_hat), NSTEP = splat2(kV ? (kM ? -P.step_m_hat : -P.step_g_hat) : -P.step_g);
         float t[8];
 #pragma unroll
         for (int p = 0; p < 4; ++p) {
-            float v0, v1, q0, q1;
-            unpack2(VF[p], v0, v1);
-            unpack2(add2(pack2(sqrt_approx(v0), sqrt_approx(v1)), EPS), q0, q1);
-            T[p] = fma2(mul2(NSTEP, MF[p]), pack2(rcp_approx(q0), rcp_approx(q1)), T[p]);
+            if (kV) {
+                float v0, v1, q0, q1;
+                unpack2(VF[p], v0, v1);
+                unpack2(add2(pack2(sqrt_approx(v0), sqrt_approx(v1)), EPS), q0, q1);
+                T[p] = fma2(mul2(NSTEP, kM ? MF[p] : XE[p]), pack2(rcp_approx(q0), rcp_approx(q1)), T[p]);
+            } else {
+                T[p] = fma2(NSTEP, MF[p], T[p]);
+            }
             chk = add2(chk, T[p]);                                  // a non-finite parameter makes the sum non-finite
             unpack2(T[p], t[2 * p], t[2 * p + 1]);
         }
 
         if (cnt == 8) {
             st8(tht + e, t);
-            st_stream_u2(qmt + e, om);
-            st_stream_u2(qvt + e, ov);
+            if (kM) st_stream_u2(qmt + e, om);
+            if (kV) st_stream_u2(qvt + e, ov);
         } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {                          // static indices keep t[] in registers
                 if (j < cnt) {
                     tht[e + j] = t[j];
-                    qmt[e + j] = int8_t(((j < 4 ? om.x : om.y) >> (8 * (j & 3))) & 0xffu);
-                    qvt[e + j] = uint8_t(((j < 4 ? ov.x : ov.y) >> (8 * (j & 3))) & 0xffu);
+                    if (kM) qmt[e + j] = int8_t(((j < 4 ? om.x : om.y) >> (8 * (j & 3))) & 0xffu);
+                    if (kV) qvt[e + j] = uint8_t(((j < 4 ? ov.x : ov.y) >> (8 * (j & 3))) & 0xffu);
                 }
             }
         }
-        if (lane == 0) { amt[w0 / kQBlock] = am_new; avt[w0 / kQBlock] = av_new; }
+        if (lane == 0) {
+            if (kM) amt[w0 / kQBlock] = am_new;
+            if (kV) avt[w0 / kQBlock] = av_new;
+        }
     }
     cp_async_wait<0>();
     float c0, c1;
@@ -787,7 +815,7 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
     const CfgStep& P = SP.c[b->cfg];
     const uint16_t* g = static_cast<const uint16_t*>(grads[t.block]);
     float* th = params[t.block];
-    const int64_t base = int64_t(t.piece) * (b->path == kPathF ? kTileF : (b->path == kPathA8 ? kTileQ : kTile));
+    const int64_t base = int64_t(t.piece) * (b->path == kPathF ? kTileF : ((b->path == kPathA8 || b->path == kPathR8 || b->path == kPathS8) ? kTileQ : kTile));
     __shared__ __align__(16) unsigned char q_stage[kStagesQ * kStageBytes];   // per-thread staging of the 8-bit and factored paths
     unsigned bad = 0;
     switch (b->path) {
@@ -798,7 +826,9 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
         case kPathA16: if (kAllPaths) bad = tile_dense<true, true, true>(b, P, g, th, base); break;
         case kPathR16: if (kAllPaths) bad = tile_dense<false, true, true>(b, P, g, th, base); break;
         case kPathS16: if (kAllPaths) bad = tile_dense<true, false, true>(b, P, g, th, base); break;
-        case kPathA8: bad = P.coupled ? tile_int8<true>(b, P, g, th, base, q_stage) : tile_int8<false>(b, P, g, th, base, q_stage); break;
+        case kPathA8: bad = P.coupled ? tile_int8<true, true, true>(b, P, g, th, base, q_stage) : tile_int8<false, true, true>(b, P, g, th, base, q_stage); break;
+        case kPathR8: if (kAllPaths) bad = P.coupled ? tile_int8<true, false, true>(b, P, g, th, base, q_stage) : tile_int8<false, false, true>(b, P, g, th, base, q_stage); break;
+        case kPathS8: if (kAllPaths) bad = P.coupled ? tile_int8<true, true, false>(b, P, g, th, base, q_stage) : tile_int8<false, true, false>(b, P, g, th, base, q_stage); break;
         case kPathF: bad = tile_factored(b, P, g, th, base, q_stage); break;
         default: break;
     }

@@ -227,6 +227,13 @@ def _check_block(sess, i, th_ref, st_ref, code_stats):
             code_stats[0] += int((d != 0).sum()); code_stats[1] += d.size
     elif kind == "G":
         pass
+    elif kind in ("R8", "S8"):
+        dt, ref_q, ref_a = (torch.uint8, st_ref.qv, st_ref.av) if kind == "R8" else (torch.int8, st_ref.qm, st_ref.am)
+        q = sess.h.view_tensor(i, 10, dt).cpu().numpy().astype(np.int32)
+        d = np.abs(q - ref_q.astype(np.int32))
+        assert d.max() <= 1
+        code_stats[0] += int((d != 0).sum()); code_stats[1] += q.size
+        assert _rel_max(f32(11), ref_a.astype(np.float64)) <= 1e-6
     elif kind == "A8":
         qm = sess.h.view_tensor(i, 10, torch.int8).cpu().numpy().astype(np.int32)
         qv = sess.h.view_tensor(i, 11, torch.uint8).cpu().numpy().astype(np.int32)
@@ -283,6 +290,37 @@ def _push_state(sess, i, th, st):
         put(10, torch.float32, st.m.astype(np.float32))
     elif st.kind == "F":
         put(10, torch.float32, st.r.astype(np.float32)); put(11, torch.float32, st.c.astype(np.float32))
+    elif st.kind == "R8":
+        put(10, torch.uint8, st.qv); put(11, torch.float32, st.av)
+    elif st.kind == "S8":
+        put(10, torch.int8, st.qm); put(11, torch.float32, st.am)
+
+
+def _run_steps_from_shared_state(sess, assign, ocfgs, n_steps=10):
+    """Each step starts from a state both sides share: the oracle's parameters and fp32 states are rounded to their
+    storage type and written to the device (oracle -> device, never the other way), both sides take one step, and a
+    coordinate may be off by 1e-6 of the block's largest parameter plus 1e-5 of its own update.  Returns the
+    [mismatching, total] count of stored codes."""
+    wl = sess.wl
+    n = len(wl.blocks)
+    sess.configure(assign)
+    th = [sess.block_param_host(i) for i in range(n)]
+    sts = [O.step_init(ocfgs[assign[i]], b.numel, b.rows, b.cols) for i, b in enumerate(wl.blocks)]
+    codes = [0, 0]
+    for t in range(1, n_steps + 1):
+        k = sess.fill_grads(t)
+        for i in range(n):
+            th[i] = _round_state_to_storage(th[i], sts[i])
+            _push_state(sess, i, th[i], sts[i])
+        before = [x.copy() for x in th]
+        sess.step(k, t)
+        for i, b in enumerate(wl.blocks):
+            th[i] = O.step(th[i], sess.block_grad_host(k, i), sts[i], ocfgs[assign[i]], b.rows, b.cols)
+            got = sess.block_param_host(i)
+            tol = 1e-6 * np.max(np.abs(th[i])) + 1e-5 * np.abs(th[i] - before[i])
+            assert np.all(np.abs(got - th[i]) <= tol), (t, b.name, sts[i].kind, float(np.max(np.abs(got - th[i]) / tol)))
+            _check_block(sess, i, None, sts[i], codes)
+    return codes
 
 
 def test_coupled_decay_and_other_hyperparameters_step_by_step(B, H):
@@ -307,46 +345,38 @@ def test_coupled_decay_and_other_hyperparameters_step_by_step(B, H):
     assign = [(i % 5) if not ((i % 5) == 3 and b.cols <= 1) else 1 for i, b in enumerate(wl.blocks)]
     assign[9] = 1                                                     # the 300 x 520 matrix takes the 8-bit path too
     ocfgs = [_ocfg(c) for c in cfgs]
-    sess.configure(assign)
-    th = [sess.block_param_host(i) for i in range(n)]
-    sts = [O.step_init(ocfgs[assign[i]], b.numel, b.rows, b.cols) for i, b in enumerate(wl.blocks)]
-    codes = [0, 0]
-    for t in range(1, 11):
-        k = sess.fill_grads(t)
-        for i in range(n):
-            th[i] = _round_state_to_storage(th[i], sts[i])
-            _push_state(sess, i, th[i], sts[i])
-        before = [x.copy() for x in th]
-        sess.step(k, t)
-        for i, b in enumerate(wl.blocks):
-            th[i] = O.step(th[i], sess.block_grad_host(k, i), sts[i], ocfgs[assign[i]], b.rows, b.cols)
-            got = sess.block_param_host(i)
-            tol = 1e-6 * np.max(np.abs(th[i])) + 1e-5 * np.abs(th[i] - before[i])
-            assert np.all(np.abs(got - th[i]) <= tol), (t, b.name, sts[i].kind, float(np.max(np.abs(got - th[i]) / tol)))
-            _check_block(sess, i, None, sts[i], codes)
+    codes = _run_steps_from_shared_state(sess, assign, ocfgs)
     assert codes[1] > 0 and codes[0] <= 1e-4 * codes[1], codes
 
 
 @pytest.mark.parametrize("tuple_", [(0, 0, 1, 0, 32), (0, 0, 0, 0, 8), (1, 1, 1, 0, 16), (1, 1, 0, 0, 16), (1, 0, 1, 0, 16),
-                                    (0, 1, 1, 0, 16), (0, 1, 0, 0, 16)])
-def test_stateless_and_bf16_state_configurations_ten_steps(B, H, tuple_):
-    """Plain gradient steps (no state) and Adam / RMS / SGD-momentum with bf16 states, decoupled and coupled decay."""
+                                    (0, 1, 1, 0, 16), (0, 1, 0, 0, 16), (1, 0, 1, 0, 8), (1, 0, 0, 0, 8), (0, 1, 1, 0, 8),
+                                    (0, 1, 0, 0, 8)])
+def test_stateless_bf16_state_and_single_moment_int8_configurations_ten_steps(B, H, tuple_):
+    """Plain gradient steps (no state), Adam / RMS / SGD-momentum with bf16 states, RMS / SGD-momentum with 8-bit
+    states; decoupled and coupled decay."""
     wl = _odd_workload(seed=61 + sum(tuple_))
     lr = 1e-2 if not tuple_[0] else 1e-3
     cfgs = [B.make_config(*tuple_, lr=lr, weight_decay=0.05)]
     sess = H.Session(wl, configs=cfgs, n_grad_sets=2)
     sess.init_params()
     assign = [0] * len(wl.blocks)
-    th, sts = _run_steps(sess, assign, 10)
-    codes = [0, 0]
-    for i in range(len(wl.blocks)):
-        _check_block(sess, i, th[i], sts[i], codes)
+    if tuple_[2] == 0 and tuple_[4] == 8:
+        # coupled decay on 8-bit states: g + wd*theta can cancel while the second moment's code is 0, and the
+        # free-running trajectory is then ill-conditioned (see the step-by-step test above); step from shared state
+        codes = _run_steps_from_shared_state(sess, assign, [_ocfg(c) for c in cfgs])
+    else:
+        th, sts = _run_steps(sess, assign, 10)
+        codes = [0, 0]
+        for i in range(len(wl.blocks)):
+            _check_block(sess, i, th[i], sts[i], codes)
     if codes[1]:
         assert codes[0] <= 1e-4 * codes[1], codes
     assert sess.h.nonfinite()[0] == 0
     mem, _ = sess.h.cost_model()
     per = {32: 4, 16: 2, 8: 1}[tuple_[4]] * (tuple_[0] + tuple_[1])
-    assert sess.h.query().state_bytes == int(mem.sum()) == per * wl.numel
+    absmax = sum(4 * ((b.numel + 255) // 256) for b in wl.blocks) * (tuple_[0] + tuple_[1]) if tuple_[4] == 8 else 0
+    assert sess.h.query().state_bytes == int(mem.sum()) == per * wl.numel + absmax
 
 
 def test_nonfinite_gradient_is_flagged_not_fatal(B, H):

@@ -542,8 +542,8 @@ def test_config_kind_dispatch():
     assert kinds == ["A32", "A8", "R", "F", "S"]
     assert O.config_kind(O.Config(0, 0, 1, 0, 32)) == "G" and O.config_kind(O.Config(0, 0, 0, 0, 8)) == "G"
     assert [O.config_kind(O.Config(1, 1, 1, 0, b)) for b in (32, 16, 8)] == ["A32", "A16", "A8"]
-    assert [O.config_kind(O.Config(1, 0, 1, 0, b)) for b in (32, 16, 8)] == ["R", "R16", "unsupported"]
-    assert [O.config_kind(O.Config(0, 1, 1, 0, b)) for b in (32, 16, 8)] == ["S", "S16", "unsupported"]
+    assert [O.config_kind(O.Config(1, 0, 1, 0, b)) for b in (32, 16, 8)] == ["R", "R16", "R8"]
+    assert [O.config_kind(O.Config(0, 1, 1, 0, b)) for b in (32, 16, 8)] == ["S", "S16", "S8"]
     assert O.config_kind(O.Config(1, 1, 1, 1, 32)) == "unsupported" and O.config_kind(O.Config(1, 0, 1, 1, 16)) == "unsupported"
 
 
@@ -598,3 +598,28 @@ def test_bf16_state_rules_store_rounded_moments_and_update_with_unrounded_ones()
                 np.testing.assert_array_equal(a16, O.round_bf16(a16))                     # the state is always bf16
     assert O.state_bytes(O.Config(1, 1, 1, 0, 16), 1000, 1000, 1) == 4000
     assert O.state_bytes(O.Config(0, 1, 1, 0, 16), 1000, 1000, 1) == 2000
+
+
+def test_int8_single_moment_rules_follow_their_fp32_forms():
+    rng = np.random.default_rng(13)
+    n = 700                                                       # three quantisation blocks, the last one ragged
+    g0 = O.round_bf16(rng.standard_normal(n) * 0.01)
+    th0 = rng.standard_normal(n) * 0.02
+    for full, q, name, signed in ((O.Config(1, 0, 1, 0, 32), O.Config(1, 0, 1, 0, 8), "v", False),
+                                  (O.Config(0, 1, 0, 0, 32, lr=1e-2, weight_decay=0.1), O.Config(0, 1, 0, 0, 8, lr=1e-2, weight_decay=0.1), "m", True)):
+        s32, s8 = O.step_init(full, n, n, 1), O.step_init(q, n, n, 1)
+        a = O.step(th0, g0, s32, full, n, 1)
+        b = O.step(th0, g0, s8, q, n, 1)
+        np.testing.assert_array_equal(a, b)                       # from the zero state the un-requantised moment is the fp32 one
+        codes, absmax = O.quantize8(getattr(s32, name), signed)
+        np.testing.assert_array_equal(getattr(s8, "q" + name), codes)
+        np.testing.assert_array_equal(getattr(s8, "a" + name), absmax)
+        # zero gradient, no decay: the state only decays; the codes move by rne(beta * code) up to the new absmax
+        z = O.Config(q.adaptive, q.momentum, 1, 0, 8, lr=0.0, beta1=0.5, beta2=0.5)
+        before = getattr(s8, "q" + name).astype(np.int32).copy()
+        th = O.step(b, np.zeros(n), s8, z, n, 1)
+        np.testing.assert_array_equal(th, b)                      # lr = 0: parameters unchanged
+        after = getattr(s8, "q" + name).astype(np.int32)
+        assert np.all(np.abs(after - before) <= 1)                # rescaling by the decayed absmax keeps the codes
+    assert O.state_bytes(O.Config(1, 0, 1, 0, 8), 700, 700, 1) == 700 + 4 * 3
+    assert O.state_bytes(O.Config(0, 1, 1, 0, 8), 700, 700, 1) == 700 + 4 * 3
