@@ -28,7 +28,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 CONFIG_NAMES = ["adamw32", "adamw8", "rms", "factored", "sgdm"]
-EXTENDED_NAMES = CONFIG_NAMES + ["sgd", "adamw16", "rms16", "sgdm16"]
+EXTENDED_NAMES = CONFIG_NAMES + ["sgd", "adamw16", "rms16", "sgdm16", "rms8", "sgdm8"]
 METRIC = "hot-path throughput: statistics pass + mixed-config optimizer step"
 UNIT = "params/s"
 
