@@ -152,10 +152,34 @@ int baoc_stats_workspace_bytes(const baoc_t* h, size_t* bytes);
  * the tile tables on the stream and starts a new window. */
 int baoc_bind_stats_workspace(baoc_t* h, void* dev, size_t bytes, baoc_stream_t stream);
 
+/* Coordinate sampling (Sec. 3.1: the statistics are computed on a fixed sample
+ * Omega_i of each block's coordinates, |Omega_i| = ceil(s d_i), s = 0.1 % by
+ * default, drawn once).  By default this library observes every coordinate
+ * (s = 1).  With a sample set, block i is observed on the sub-grid
+ * rows[0..n_rows) x cols[0..n_cols) of its rows x cols matrix, so that the
+ * "matrix form of the sampled gradients" of Eq. 7 exists (a vector block has
+ * n_cols = 1 and cols = NULL); n_rows * n_cols plays the role of |Omega_i|.
+ * Indices are host arrays, in range and strictly increasing; the library copies
+ * them.  The draw itself is the caller's (it is an input, like the gradients).
+ * Every per-parameter quantity of the window (moments, previous gradient,
+ * quantiles, Eq. 6's parameters) then lives on the sample: each observation
+ * first gathers g[Omega] into the workspace, baoc_risk gathers theta[Omega].
+ * Call before baoc_bind_stats_workspace (the workspace size changes; a bound
+ * workspace must be bound again); samples == NULL returns to the dense sample.
+ * BAOC_E_STATE once the window has observations. */
+typedef struct {
+    int64_t n_rows;
+    int32_t n_cols;
+    const int64_t* rows;
+    const int32_t* cols;
+} baoc_sample_t;
+int baoc_set_sampling(baoc_t* h, const baoc_sample_t* samples /* [n_blocks] or NULL */);
+
 /* One gradient observation of every block (Eq. 3 and the cosine of Eq. 5).
  * grads: host array of n_blocks device pointers to bf16 gradients (block i has
- * numel_i elements).  The sample is dense: every coordinate of every block.
- * Queues one streaming kernel and one small combine kernel; does not wait. */
+ * numel_i elements).  The sample is dense (every coordinate of every block)
+ * unless baoc_set_sampling chose a sub-grid.  Queues one streaming kernel and
+ * one small combine kernel (after a gather kernel when sampling); does not wait. */
 int baoc_sample_stats(baoc_t* h, const void* const* grads, baoc_stream_t stream);
 
 /* Copy the running per-block values of the window (rho_bar, last_cos, n_cos,

@@ -64,6 +64,10 @@ class BlockStats(C.Structure):
         return {n: getattr(self, n) for n, _ in self._fields_}
 
 
+class Sample(C.Structure):
+    _fields_ = [("n_rows", C.c_int64), ("n_cols", C.c_int32), ("rows", C.c_void_p), ("cols", C.c_void_p)]
+
+
 class Info(C.Structure):
     _fields_ = [("n_blocks", C.c_int32), ("n_cfg", C.c_int32), ("numel", C.c_int64), ("n_tiles", C.c_int64),
                 ("stats_steps", C.c_int64), ("state_bytes", C.c_int64), ("kernel_launches", C.c_int64),
@@ -75,7 +79,8 @@ EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error"
            "baoc_risk", "baoc_risk_from_raw", "baoc_cost_model", "baoc_allocate", "baoc_state_bytes",
            "baoc_configure", "baoc_step", "baoc_step_from_host", "baoc_view", "baoc_nonfinite",
            "baoc_sample_stats_noalloc", "baoc_noalloc_last_error", "baoc_profile", "baoc_profile_last",
-           "baoc_export", "baoc_import", "baoc_time_scratch_bytes", "baoc_measure_time_ratios"]
+           "baoc_export", "baoc_import", "baoc_time_scratch_bytes", "baoc_measure_time_ratios",
+           "baoc_set_sampling"]
 
 _vp = C.c_void_p
 _lib.baoc_default_opts.argtypes = [C.POINTER(Opts)]
@@ -100,6 +105,7 @@ _lib.baoc_step.argtypes = [_vp, _vp, _vp, C.c_int64, _vp]
 _lib.baoc_step_from_host.argtypes = [_vp, _vp, _vp, _vp, C.c_int, C.c_int64, _vp]
 _lib.baoc_view.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(_vp), C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
 _lib.baoc_nonfinite.argtypes = [_vp, _vp, C.POINTER(C.c_int32), _vp]
+_lib.baoc_set_sampling.argtypes = [_vp, C.POINTER(Sample)]
 _lib.baoc_time_scratch_bytes.argtypes = [_vp, C.POINTER(C.c_size_t)]
 _lib.baoc_measure_time_ratios.argtypes = [_vp, _vp, _vp, _vp, C.c_size_t, C.c_int, C.c_int, _vp, _vp, _vp]
 _lib.baoc_export.argtypes = [_vp, _vp, C.c_size_t, C.POINTER(C.c_size_t)]
@@ -210,6 +216,25 @@ class Baoc:
         return info
 
     # ---- sampling window --------------------------------------------------
+    def set_sampling(self, samples):
+        """``baoc_set_sampling``.  samples: None (dense), or one (rows, cols) pair of integer index arrays per block
+        (cols is None for a vector block).  Call before ``bind_stats_workspace``."""
+        if samples is None:
+            self._check(_lib.baoc_set_sampling(self._h, None))
+            return
+        keep, arr = [], (Sample * self.n_blocks)()
+        for i, (rows, cols) in enumerate(samples):
+            r = np.ascontiguousarray(rows, np.int64)
+            keep.append(r)
+            arr[i].n_rows, arr[i].rows = r.size, r.ctypes.data
+            if cols is None:
+                arr[i].n_cols, arr[i].cols = 1, None
+            else:
+                c = np.ascontiguousarray(cols, np.int32)
+                keep.append(c)
+                arr[i].n_cols, arr[i].cols = c.size, c.ctypes.data
+        self._check(_lib.baoc_set_sampling(self._h, arr))
+
     def stats_workspace_bytes(self) -> int:
         n = C.c_size_t()
         self._check(_lib.baoc_stats_workspace_bytes(self._h, C.byref(n)))

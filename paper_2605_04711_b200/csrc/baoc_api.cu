@@ -53,8 +53,13 @@ int do_sample_stats(Handle* h, const void* const* grads, cudaStream_t s) {
     int rc = sync_pointer_table(h, grads, &h->last_stat_grads, h->ws + h->sl.grads, s, "baoc_sample_stats");
     if (rc) return rc;
     const auto& L = h->sl;
+    if (h->sampled) {
+        LAUNCH(launch_sample_gather(at<StatBlock>(h->ws, L.blocks), at<Tile>(h->ws, L.tiles), at<const void*>(h->ws, L.grads),
+                                    h->n_stat_tiles, 0, s), "sample_gather_kernel");
+        h->launches += 1;
+    }
     LAUNCH(launch_stats_step(at<StatBlock>(h->ws, L.blocks), at<Tile>(h->ws, L.tiles),
-                             at<const void*>(h->ws, L.grads), at<double>(h->ws, L.partials), h->n_stat_tiles,
+                             at<const void*>(h->ws, h->sampled ? L.sgrads : L.grads), at<double>(h->ws, L.partials), h->n_stat_tiles,
                              float(1.0 - h->opts.beta_m), float(1.0 - h->opts.beta_v), s), "stats_step_kernel");
     LAUNCH(launch_stats_combine(at<StatBlock>(h->ws, L.blocks), at<double>(h->ws, L.partials), at<double>(h->ws, L.acc),
                                 h->n_blocks, h->stats_steps > 0 ? 1 : 0, h->opts.beta_rho, h->opts.eps, s),
@@ -146,6 +151,12 @@ static int bind_stats(baoc_t* h, void* dev, size_t bytes, baoc_stream_t stream, 
         b.m = reinterpret_cast<float*>(ws + L.m + reinterpret_cast<size_t>(b.m));
         b.v = reinterpret_cast<float*>(ws + L.v + reinterpret_cast<size_t>(b.v));
         b.gprev = reinterpret_cast<uint16_t*>(ws + L.gprev + reinterpret_cast<size_t>(b.gprev));
+        if (h->sampled) {
+            b.ridx = reinterpret_cast<const int64_t*>(ws + L.ridx + reinterpret_cast<size_t>(b.ridx));
+            b.cidx = reinterpret_cast<const int32_t*>(ws + L.cidx + reinterpret_cast<size_t>(b.cidx));
+            b.gsample = reinterpret_cast<uint16_t*>(ws + L.gsample + reinterpret_cast<size_t>(b.gsample));
+            b.psample = reinterpret_cast<float*>(ws + L.psample + reinterpret_cast<size_t>(b.psample));
+        }
         for (int k = 0; k < b.ntiles; ++k) tiles.push_back(Tile{uint32_t(i), uint32_t(k)});
         if (b.cols > 1) {
             b.rowsum = reinterpret_cast<double*>(ws + L.rowsum + reinterpret_cast<size_t>(b.rowsum));
@@ -158,6 +169,22 @@ static int bind_stats(baoc_t* h, void* dev, size_t bytes, baoc_stream_t stream, 
         }
     }
     h->n_matrix = int(ids.size());
+    if (h->sampled) {
+        // index lists and the tables of sample-buffer pointers (the host vectors outlive the copies: they belong to the handle)
+        h->sample_tables.clear();
+        std::vector<int64_t>& ri = h->flat_ridx; std::vector<int32_t>& ci = h->flat_cidx;
+        ri.clear(); ci.clear();
+        for (int i = 0; i < n; ++i) {
+            ri.insert(ri.end(), h->s_rows[i].begin(), h->s_rows[i].end());
+            ci.insert(ci.end(), h->s_cols[i].begin(), h->s_cols[i].end());
+            h->sample_tables.push_back(sb[i].gsample);
+        }
+        for (int i = 0; i < n; ++i) h->sample_tables.push_back(sb[i].psample);
+        CU(cudaMemcpyAsync(ws + L.ridx, ri.data(), 8 * ri.size(), cudaMemcpyHostToDevice, s), "upload sample rows");
+        CU(cudaMemcpyAsync(ws + L.cidx, ci.data(), 4 * ci.size(), cudaMemcpyHostToDevice, s), "upload sample columns");
+        CU(cudaMemcpyAsync(ws + L.sgrads, h->sample_tables.data(), 8 * size_t(n), cudaMemcpyHostToDevice, s), "upload sample gradient table");
+        CU(cudaMemcpyAsync(ws + L.sparams, h->sample_tables.data() + n, 8 * size_t(n), cudaMemcpyHostToDevice, s), "upload sample parameter table");
+    }
     CU(cudaMemcpyAsync(ws + L.blocks, sb.data(), sizeof(StatBlock) * n, cudaMemcpyHostToDevice, s), "upload block table");
     CU(cudaMemcpyAsync(ws + L.tiles, tiles.data(), sizeof(Tile) * tiles.size(), cudaMemcpyHostToDevice, s), "upload tile table");
     if (!red.empty())
@@ -215,7 +242,11 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
     char* ws = h->ws;
     const StatBlock* blocks = at<StatBlock>(ws, L.blocks);
     const Tile* tiles = at<Tile>(ws, L.tiles);
-    const float* const* dparams = at<const float*>(ws, L.params);
+    const float* const* dparams = at<const float*>(ws, h->sampled ? L.sparams : L.params);
+    if (h->sampled) {
+        LAUNCH(launch_sample_gather(blocks, tiles, at<const void*>(ws, L.params), h->n_stat_tiles, 1, s), "sample_gather_kernel");
+        h->launches += 1;
+    }
     LAUNCH(launch_final_sums(blocks, tiles, dparams, at<double>(ws, L.fin), at<double>(ws, L.fin_out), h->n_stat_tiles, n,
                              h->opts.eps, float(h->opts.eps_adam), s), "stats_final_sums_kernel");
     h->launches += 2;
@@ -248,7 +279,7 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
     auto rel = [](double err2, double ref2) { return ref2 > 0.0 ? std::sqrt(err2) / std::sqrt(ref2) : 0.0; };
     for (int i = 0; i < n; ++i) {
         const double* o = &out[size_t(i) * kFinOut];
-        const baoc_block_t& b = h->blocks[i];
+        const baoc_block_t& b = h->stat_shapes[i];           // the block, or its sample
         baoc_block_stats_t& z = st[i];
         std::memset(&z, 0, sizeof(z));
         // Eq. 4: quantiles by linear interpolation at position q (n - 1)
@@ -583,7 +614,7 @@ int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* co
         const StatBlock& s = h->h_stat_blocks[block];
         const size_t off = reinterpret_cast<size_t>(which == 2 ? static_cast<void*>(s.gprev) : static_cast<void*>(which == 0 ? s.m : s.v));
         const size_t region = which == 0 ? h->sl.m : (which == 1 ? h->sl.v : h->sl.gprev);
-        *dev_ptr = h->ws + region + off; *count = b.numel; *elem_bytes = which == 2 ? 2 : 4;
+        *dev_ptr = h->ws + region + off; *count = h->stat_shapes[block].numel; *elem_bytes = which == 2 ? 2 : 4;
         return BAOC_OK;
     }
     if (which >= 10 && which <= 13) {

@@ -60,11 +60,20 @@ static size_t take(size_t* cur, size_t bytes) {
 // h_stat_blocks are offsets from a null base until a workspace is bound.
 void compute_stat_layout(Handle* h) {
     const int n = h->n_blocks;
-    int64_t tiles = 0, red = 0, padded = 0, sum_rows = 0, sum_cols = 0, redpart = 0;
+    int64_t tiles = 0, red = 0, padded = 0, sum_rows = 0, sum_cols = 0, redpart = 0, n_ridx = 0, n_cidx = 0;
     h->h_stat_blocks.assign(n, StatBlock{});
+    if (!h->sampled) h->stat_shapes = h->blocks;
     for (int i = 0; i < n; ++i) {
-        const baoc_block_t& b = h->blocks[i];
+        const baoc_block_t& b = h->stat_shapes[i];
         StatBlock& s = h->h_stat_blocks[i];
+        s.full_cols = h->blocks[i].cols;
+        if (h->sampled) {
+            s.ridx = reinterpret_cast<const int64_t*>(size_t(n_ridx) * 8);
+            s.cidx = reinterpret_cast<const int32_t*>(size_t(n_cidx) * 4);
+            s.gsample = reinterpret_cast<uint16_t*>(size_t(padded) * 2);
+            s.psample = reinterpret_cast<float*>(size_t(padded) * 4);
+            n_ridx += int64_t(h->s_rows[i].size()); n_cidx += int64_t(h->s_cols[i].size());
+        }
         s.numel = b.numel; s.rows = b.rows; s.cols = b.cols;
         s.tile0 = tiles; s.ntiles = int32_t(ceil_div(b.numel, kTile));
         tiles += s.ntiles;
@@ -106,6 +115,15 @@ void compute_stat_layout(Handle* h) {
     L.rowsum = take(&cur, 8 * size_t(std::max<int64_t>(sum_rows, 1)));
     L.colsum = take(&cur, 8 * size_t(std::max<int64_t>(sum_cols, 1)));
     L.redpart = take(&cur, 8 * size_t(std::max<int64_t>(redpart, 1)));
+    L.ridx = L.cidx = L.gsample = L.psample = L.sgrads = L.sparams = cur;
+    if (h->sampled) {
+        L.ridx = take(&cur, 8 * size_t(std::max<int64_t>(n_ridx, 1)));
+        L.cidx = take(&cur, 4 * size_t(std::max<int64_t>(n_cidx, 1)));
+        L.gsample = take(&cur, 2 * size_t(padded));
+        L.psample = take(&cur, 4 * size_t(padded));
+        L.sgrads = take(&cur, 8 * size_t(n));
+        L.sparams = take(&cur, 8 * size_t(n));
+    }
     L.total = cur;
 }
 
@@ -499,13 +517,53 @@ void baoc_destroy(baoc_t* h) { delete h; }
 
 const char* baoc_last_error(const baoc_t* h) { return h ? h->err.c_str() : "null handle"; }
 
+int baoc_set_sampling(baoc_t* h, const baoc_sample_t* samples) {
+    if (!h) return BAOC_E_INVALID;
+    if (h->ws_bound && h->stats_steps > 0) return fail(h, BAOC_E_STATE, "baoc_set_sampling: the window has started; set the sample before the first observation");
+    if (!samples) {                                        // back to the dense sample
+        h->sampled = false; h->s_rows.clear(); h->s_cols.clear();
+        compute_stat_layout(h);
+        h->ws_bound = false;
+        return BAOC_OK;
+    }
+    const int n = h->n_blocks;
+    std::vector<std::vector<int64_t>> rows(n);
+    std::vector<std::vector<int32_t>> cols(n);
+    std::vector<baoc_block_t> shapes(n);
+    for (int i = 0; i < n; ++i) {
+        const baoc_block_t& b = h->blocks[i];
+        const baoc_sample_t& sm = samples[i];
+        const bool vec = b.cols <= 1;
+        if (!sm.rows || sm.n_rows < 1 || sm.n_rows > b.rows) return fail(h, BAOC_E_INVALID, "baoc_set_sampling: bad row sample");
+        if (vec ? (sm.n_cols != 1) : (!sm.cols || sm.n_cols < 1 || sm.n_cols > b.cols)) return fail(h, BAOC_E_INVALID, "baoc_set_sampling: bad column sample");
+        rows[i].assign(sm.rows, sm.rows + sm.n_rows);
+        if (vec) cols[i].assign(1, 0); else cols[i].assign(sm.cols, sm.cols + sm.n_cols);
+        for (size_t k = 0; k < rows[i].size(); ++k)
+            if (rows[i][k] < 0 || rows[i][k] >= b.rows || (k && rows[i][k] <= rows[i][k - 1]))
+                return fail(h, BAOC_E_INVALID, "baoc_set_sampling: row indices must be in range and strictly increasing");
+        for (size_t k = 0; k < cols[i].size(); ++k)
+            if (cols[i][k] < 0 || cols[i][k] >= b.cols || (k && cols[i][k] <= cols[i][k - 1]))
+                return fail(h, BAOC_E_INVALID, "baoc_set_sampling: column indices must be in range and strictly increasing");
+        shapes[i].rows = int32_t(rows[i].size()); shapes[i].cols = int32_t(cols[i].size());
+        shapes[i].numel = int64_t(shapes[i].rows) * shapes[i].cols;
+    }
+    h->sampled = true; h->s_rows.swap(rows); h->s_cols.swap(cols); h->stat_shapes.swap(shapes);
+    compute_stat_layout(h);
+    h->ws_bound = false;                                   // the workspace has a new size and layout: bind again
+    return BAOC_OK;
+}
+
 int baoc_query(const baoc_t* h, baoc_info_t* info) {
     if (!h || !info) return BAOC_E_INVALID;
     info->n_blocks = h->n_blocks; info->n_cfg = h->n_cfg; info->numel = h->numel;
     info->n_tiles = h->n_stat_tiles; info->stats_steps = h->stats_steps;
     info->state_bytes = h->configured ? h->state_mem : 0;
     info->kernel_launches = h->launches;
-    info->stats_bytes_per_call = 22 * h->numel;      // g_t, g_{t-1}, m, v read; m, v, g_{t-1} written
+    {   // g_t, g_{t-1}, m, v read; m, v, g_{t-1} written, over what the statistics see (+ the gather of a sample)
+        int64_t seen = 0;
+        for (const baoc_block_t& b : (h->sampled ? h->stat_shapes : h->blocks)) seen += b.numel;
+        info->stats_bytes_per_call = (h->sampled ? 26 : 22) * seen;
+    }
     info->step_bytes_per_call = h->configured ? h->step_bytes : 0;
     return BAOC_OK;
 }

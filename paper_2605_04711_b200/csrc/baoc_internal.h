@@ -88,6 +88,12 @@ struct StatBlock {
     int32_t rows, cols;
     int32_t ntiles, pad;
     RedGeom red;
+    // coordinate sampling: the statistics see the sub-grid rows[ridx] x cols[cidx] of the block (null: the whole block)
+    const int64_t* ridx;
+    const int32_t* cidx;
+    uint16_t* gsample;   // gathered gradient of the current step, bf16 bits
+    float* psample;      // gathered parameters (finalize)
+    int64_t full_cols;   // row length of the whole block
 };
 
 // Per-block record of the fused step (device copy lives in the state buffer).
@@ -160,11 +166,18 @@ struct Handle {
     int64_t n_red_tiles = 0;         // reduction CTAs over all matrix blocks
     int n_matrix = 0;                // blocks with cols > 1
     std::vector<StatBlock> h_stat_blocks;
+    bool sampled = false;                                  // statistics on a sampled sub-grid of every block
+    std::vector<baoc_block_t> stat_shapes;                 // what the statistics see: the blocks, or their samples
+    std::vector<std::vector<int64_t>> s_rows;
+    std::vector<std::vector<int32_t>> s_cols;
+    std::vector<int64_t> flat_ridx;                        // staging of the uploads (must outlive the async copies)
+    std::vector<int32_t> flat_cidx;
+    std::vector<const void*> sample_tables;
     std::vector<const void*> last_stat_grads;
     std::vector<const void*> last_stat_params;
     struct StatLayout {
         size_t blocks, tiles, red_tiles, matrix_ids, grads, params, m, v, gprev, partials, acc, fin, fin_out, hist, sel,
-               rowsum, colsum, redpart, total;
+               rowsum, colsum, redpart, ridx, cidx, gsample, psample, sgrads, sparams, total;
     } sl{};
 
     // optimizer state
@@ -215,6 +228,8 @@ int launch_final_resid(const StatBlock* blocks, const Tile* tiles, const float* 
                        double* fin_out, int64_t n_tiles, int n_blocks, double eps, cudaStream_t s);
 int launch_select(const StatBlock* blocks, const Tile* tiles, RankSel* sel, uint32_t* hist, int64_t n_tiles,
                   int n_blocks, cudaStream_t s);
+int launch_sample_gather(const StatBlock* blocks, const Tile* tiles, const void* const* src, int64_t n_tiles, int fp32,
+                         cudaStream_t s);
 int launch_gather(const RankSel* sel, const double* acc, double* fin_out, int n_blocks, cudaStream_t s);
 int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const int32_t* ids, int64_t n_red, int n_matrix,
                          cudaStream_t s);

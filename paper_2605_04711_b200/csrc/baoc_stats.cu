@@ -452,6 +452,36 @@ __global__ void stats_gather_kernel(const RankSel* __restrict__ sel, const doubl
     for (int k = 0; k < kBlockAcc; ++k) o[20 + k] = acc[size_t(blk) * kBlockAcc + k];
 }
 
+// ============================================================================
+// Coordinate sampling: gather the sub-grid rows[ridx] x cols[cidx] of every block
+// into its compact sample buffer (bf16 gradients each step, fp32 parameters at
+// the end of the window).  One CTA per tile of the sample; element k of the
+// sample is (ridx[k / n_cols], cidx[k % n_cols]).  Padding up to the next
+// quantisation block is zero-filled so that the streaming kernels may read it.
+// ============================================================================
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+sample_gather_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const void* const* __restrict__ src) {
+    const Tile t = tiles[blockIdx.x];
+    const StatBlock* b = blocks + t.block;
+    const int64_t numel = b->numel, padded = (numel + kQBlock - 1) / kQBlock * kQBlock;
+    const int cols = b->cols;
+    const T* __restrict__ in = static_cast<const T*>(src[t.block]);
+    T* __restrict__ out = sizeof(T) == 2 ? reinterpret_cast<T*>(b->gsample) : reinterpret_cast<T*>(b->psample);
+    const int64_t base = int64_t(t.piece) * kTile;
+    for (int i = threadIdx.x; i < kTile; i += kThreads) {
+        const int64_t k = base + i;
+        if (k >= padded) break;
+        T val = T(0);
+        if (k < numel) {
+            const int64_t r = k / cols;
+            const int c = int(k - r * cols);
+            val = in[b->ridx[r] * b->full_cols + b->cidx[c]];
+        }
+        out[k] = val;
+    }
+}
+
 // ---- launchers ------------------------------------------------------------------
 #define BAOC_LAUNCH_CHECK()                                   \
     do {                                                      \
@@ -503,6 +533,14 @@ int launch_select(const StatBlock* blocks, const Tile* tiles, RankSel* sel, uint
         select_pick_kernel<<<gb, tb, 0, s>>>(sel, hist, n_blocks, shift);
         BAOC_LAUNCH_CHECK();
     }
+    return 0;
+}
+
+int launch_sample_gather(const StatBlock* blocks, const Tile* tiles, const void* const* src, int64_t n_tiles, int fp32,
+                         cudaStream_t s) {
+    if (fp32) sample_gather_kernel<float><<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, src);
+    else sample_gather_kernel<uint16_t><<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, src);
+    BAOC_LAUNCH_CHECK();
     return 0;
 }
 

@@ -60,7 +60,7 @@ class Session:
     """
 
     def __init__(self, wl: W.Workload, configs: Optional[Sequence[B.Config]] = None, opts: Optional[B.Opts] = None,
-                 n_grad_sets: int = 2, device: str = "cuda:0", pinned_host_grads: bool = False):
+                 n_grad_sets: int = 2, device: str = "cuda:0", pinned_host_grads: bool = False, samples=None):
         self.wl = wl
         self.device = torch.device(device)
         self.configs = list(configs) if configs is not None else B.default_configs()
@@ -78,6 +78,9 @@ class Session:
             self.host_grads = [torch.zeros(self.total, dtype=torch.bfloat16).pin_memory() for _ in range(n_grad_sets)]
             self.host_tables = [B.pointer_table([hg[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)])
                                 for hg in self.host_grads]
+        self.samples = samples
+        if samples is not None:
+            self.h.set_sampling(samples)
         self.ws = torch.empty(self.h.stats_workspace_bytes(), dtype=torch.uint8, device=self.device)
         self.h.bind_stats_workspace(self.ws)
         self.state = None
@@ -136,3 +139,11 @@ class Session:
 
     def block_param_host(self, i: int) -> np.ndarray:
         return self.param_views[i].double().cpu().numpy()
+
+    def sampled(self, i: int, full: np.ndarray) -> np.ndarray:
+        """The entries of block i's flat array that the statistics see (all of them without sampling)."""
+        if self.samples is None:
+            return full
+        rows, cols = self.samples[i]
+        b = self.wl.blocks[i]
+        return full[rows] if cols is None else full.reshape(b.rows, b.cols)[np.ix_(rows, cols)].reshape(-1)

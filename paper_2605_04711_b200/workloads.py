@@ -328,6 +328,27 @@ def time_ratio_table(wl: Workload, base_ratios: Sequence[float], jitter: float =
     return base[None, :] * (1.0 + jitter * (2.0 * u - 1.0))
 
 
+def sample_subgrids(wl: Workload, s_frac: float):
+    """A seeded sub-grid sample of every block's coordinates: about ``s_frac`` of them.  A vector block gets
+    ceil(s d) sorted distinct indices; a rows x cols block gets ceil(sqrt(s) rows) rows and ceil(sqrt(s) cols) columns
+    (their product is at least ceil(s d)).  Returns one (rows, cols-or-None) pair of int64 / int32 numpy arrays per
+    block, drawn once per (seed, block)."""
+    out = []
+    for i, b in enumerate(wl.blocks):
+        g = torch.Generator().manual_seed(stream_seed(wl.seed, i, 3))
+        if b.cols <= 1:
+            n = max(1, math.ceil(s_frac * b.rows))
+            rows = torch.randperm(b.rows, generator=g)[:n].sort().values
+            out.append((rows.numpy().astype("int64"), None))
+        else:
+            nr = max(1, min(b.rows, math.ceil(math.sqrt(s_frac) * b.rows)))
+            nc = max(1, min(b.cols, math.ceil(math.sqrt(s_frac) * b.cols)))
+            rows = torch.randperm(b.rows, generator=g)[:nr].sort().values
+            cols = torch.randperm(b.cols, generator=g)[:nc].sort().values
+            out.append((rows.numpy().astype("int64"), cols.numpy().astype("int32")))
+    return out
+
+
 def flat_layout(wl: Workload, align_elems: int = 128):
     """Element offset of every block in one flat buffer, each start aligned to
     ``align_elems`` elements, and the total length."""

@@ -166,6 +166,51 @@ def test_stats_invariants_identical_zero_and_flipped_gradients(B, H):
             assert st2[i]["F"] < 1e-6                                # constant matrix is rank one
 
 
+def test_sampled_statistics_match_the_oracle_on_the_sample(B, H):
+    """Coordinate sampling (Sec. 3.1): every block is observed on a fixed sub-grid; the oracle gets the same entries."""
+    wl = _odd_workload(seed=71, window=5)
+    samples = W.sample_subgrids(wl, 0.3)
+    sess = H.Session(wl, n_grad_sets=2, samples=samples)
+    sess.init_params()
+    o = O.Opts()
+    shapes = [(len(r), 1 if c is None else len(c)) for r, c in samples]
+    states = [O.stats_init(nr * nc) for nr, nc in shapes]
+    for t in range(1, wl.window + 1):
+        k = sess.fill_grads(t)
+        sess.sample_stats(k)
+        for i in range(len(wl.blocks)):
+            O.stats_step(states[i], sess.sampled(i, sess.block_grad_host(k, i)), o)
+    risk, st = sess.risk()
+    cfgs = [_ocfg(c) for c in sess.configs]
+    for i, b in enumerate(wl.blocks):
+        m = sess.h.view_tensor(i, 0, torch.float32).double().cpu().numpy()
+        assert m.shape == states[i].m.shape and np.max(np.abs(m - states[i].m)) <= 1e-6 * max(np.max(np.abs(states[i].m)), 1e-30)
+        raw = O.stats_finalize(states[i], sess.sampled(i, sess.block_param_host(i)), shapes[i][0], shapes[i][1], o)
+        for k in STAT_KEYS:
+            assert _stat_close(k, st[i][k], raw[k], wl.window), (b.name, k, st[i][k], raw[k])
+        z = O.normalise(raw, o)
+        for c, cfg in enumerate(cfgs):
+            ref = O.risk(z, cfg, o)
+            assert abs(risk[i, c] - ref) <= 1e-4 * max(abs(ref), 1e-2)
+    info = sess.h.query()
+    assert info.stats_bytes_per_call == 26 * sum(nr * nc for nr, nc in shapes)
+
+
+def test_a_sample_of_every_coordinate_equals_the_dense_pass_bit_for_bit(B, H):
+    wl = _odd_workload(seed=72, window=3)
+    full = [(np.arange(b.rows), None if b.cols <= 1 else np.arange(b.cols)) for b in wl.blocks]
+    outs = []
+    for samples in (None, full):
+        sess = H.Session(wl, n_grad_sets=1, samples=samples)
+        sess.init_params()
+        for t in range(1, 4):
+            sess.sample_stats(sess.fill_grads(t))
+        risk, st = sess.risk()
+        outs.append((risk.copy(), [tuple(s[k] for k in STAT_KEYS) for s in st]))
+    np.testing.assert_array_equal(outs[0][0], outs[1][0])
+    assert outs[0][1] == outs[1][1]
+
+
 def test_stats_is_deterministic(B, H):
     wl = _odd_workload(seed=8, window=3)
     outs = []

@@ -229,3 +229,23 @@ def test_export_import_blob_without_device_state(B):
         with pytest.raises(B.BaocError) as e:
             B.Baoc(blocks, B.default_configs()).import_state(bad_blob)
         assert e.value.code == B.E_INVALID
+
+
+def test_set_sampling_validates_indices_and_shrinks_the_workspace(B):
+    blocks = [(4096 * 8, 256, 128), (1000, 1000, 1)]
+    h = B.Baoc(blocks, B.default_configs())
+    dense = h.stats_workspace_bytes()
+    rows0, cols0 = np.arange(0, 256, 8), np.arange(0, 128, 4)
+    h.set_sampling([(rows0, cols0), (np.arange(0, 1000, 10), None)])
+    assert h.stats_workspace_bytes() < dense // 4 and h.query().n_tiles == 2
+    assert h.query().stats_bytes_per_call == 26 * (32 * 32 + 100)
+    bad = [([0, 0, 3], cols0), ([5, 3], cols0), ([256], cols0), (rows0, [128]), (rows0, None), ([], cols0)]
+    for rows, cols in bad:
+        with pytest.raises(B.BaocError) as e:
+            h.set_sampling([(rows, cols), (np.arange(10), None)])
+        assert e.value.code == B.E_INVALID
+    with pytest.raises(B.BaocError) as e:
+        h.set_sampling([(rows0, cols0), (np.arange(10), np.arange(2))])          # a vector block has one column
+    assert e.value.code == B.E_INVALID
+    h.set_sampling(None)
+    assert h.stats_workspace_bytes() == dense
