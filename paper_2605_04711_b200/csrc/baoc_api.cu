@@ -29,6 +29,20 @@ int launch_fail(const Handle* h, const char* what, int code) {
         if (r_ != 0) return launch_fail(h, what, r_);   \
     } while (0)
 
+// Events and the copy stream a handle may own (created on first use, destroyed with the handle).
+void destroy_cuda_objects(Handle* h) {
+    for (void*& e : h->prof_ev) {
+        if (e) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+        e = nullptr;
+    }
+    for (void*& e : h->copy_ev) {
+        if (e) cudaEventDestroy(static_cast<cudaEvent_t>(e));
+        e = nullptr;
+    }
+    if (h->copy_stream) cudaStreamDestroy(static_cast<cudaStream_t>(h->copy_stream));
+    h->copy_stream = nullptr;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Check a host array of device pointers; upload it when it differs from the
@@ -49,24 +63,41 @@ int sync_pointer_table(Handle* h, const void* const* ptrs, std::vector<const voi
 template <typename T>
 T* at(char* base, size_t off) { return reinterpret_cast<T*>(base + off); }
 
-int do_sample_stats(Handle* h, const void* const* grads, cudaStream_t s) {
-    int rc = sync_pointer_table(h, grads, &h->last_stat_grads, h->ws + h->sl.grads, s, "baoc_sample_stats");
-    if (rc) return rc;
+// The streaming part of one observation for the blocks [b0, b1): their tiles are contiguous in the tile table.
+int stats_step_range(Handle* h, int b0, int b1, cudaStream_t s) {
     const auto& L = h->sl;
+    const int64_t t0 = h->h_stat_blocks[b0].tile0;
+    const int64_t t1 = b1 < h->n_blocks ? h->h_stat_blocks[b1].tile0 : h->n_stat_tiles;
+    if (t1 <= t0) return BAOC_OK;
     if (h->sampled) {
-        LAUNCH(launch_sample_gather(at<StatBlock>(h->ws, L.blocks), at<Tile>(h->ws, L.tiles), at<const void*>(h->ws, L.grads),
-                                    h->n_stat_tiles, 0, s), "sample_gather_kernel");
+        LAUNCH(launch_sample_gather(at<StatBlock>(h->ws, L.blocks), at<Tile>(h->ws, L.tiles) + t0, at<const void*>(h->ws, L.grads),
+                                    t1 - t0, 0, s), "sample_gather_kernel");
         h->launches += 1;
     }
-    LAUNCH(launch_stats_step(at<StatBlock>(h->ws, L.blocks), at<Tile>(h->ws, L.tiles),
-                             at<const void*>(h->ws, h->sampled ? L.sgrads : L.grads), at<double>(h->ws, L.partials), h->n_stat_tiles,
+    LAUNCH(launch_stats_step(at<StatBlock>(h->ws, L.blocks), at<Tile>(h->ws, L.tiles) + t0,
+                             at<const void*>(h->ws, h->sampled ? L.sgrads : L.grads),
+                             at<double>(h->ws, L.partials) + size_t(t0) * kStatPartials, t1 - t0,
                              float(1.0 - h->opts.beta_m), float(1.0 - h->opts.beta_v), s), "stats_step_kernel");
+    h->launches += 1;
+    return BAOC_OK;
+}
+
+int stats_combine_all(Handle* h, cudaStream_t s) {
+    const auto& L = h->sl;
     LAUNCH(launch_stats_combine(at<StatBlock>(h->ws, L.blocks), at<double>(h->ws, L.partials), at<double>(h->ws, L.acc),
                                 h->n_blocks, h->stats_steps > 0 ? 1 : 0, h->opts.beta_rho, h->opts.eps, s),
            "stats_combine_kernel");
-    h->launches += 2;
+    h->launches += 1;
     h->stats_steps += 1;
     return BAOC_OK;
+}
+
+int do_sample_stats(Handle* h, const void* const* grads, cudaStream_t s) {
+    int rc = sync_pointer_table(h, grads, &h->last_stat_grads, h->ws + h->sl.grads, s, "baoc_sample_stats");
+    if (rc) return rc;
+    rc = stats_step_range(h, 0, h->n_blocks, s);
+    if (rc) return rc;
+    return stats_combine_all(h, s);
 }
 
 void fill_step_params(const Handle* h, int64_t t, StepParams* P) {
@@ -550,35 +581,70 @@ int baoc_step_from_host(baoc_t* h, const void* const* host_grads, void* const* d
         if (!host_grads[i] || !dev_grads[i]) return fail(h, BAOC_E_INVALID, "baoc_step_from_host: null block pointer");
         if (!aligned16(dev_grads[i])) return fail(h, BAOC_E_ALIGN, "baoc_step_from_host: block pointer not 16-byte aligned");
     }
-    // blocks that are contiguous on both sides travel in one copy
-    int i = 0;
-    while (i < h->n_blocks) {
-        int j = i;
-        size_t bytes = 2 * size_t(h->blocks[i].numel);
-        while (j + 1 < h->n_blocks &&
-               static_cast<const char*>(host_grads[j + 1]) == static_cast<const char*>(host_grads[i]) + bytes &&
-               static_cast<const char*>(dev_grads[j + 1]) == static_cast<const char*>(dev_grads[i]) + bytes) {
-            ++j;
-            bytes += 2 * size_t(h->blocks[j].numel);
-        }
-        CU(cudaMemcpyAsync(dev_grads[i], host_grads[i], bytes, cudaMemcpyHostToDevice, s), "baoc_step_from_host (copy)");
-        i = j + 1;
-    }
     const void* const* dg = reinterpret_cast<const void* const*>(dev_grads);
-    if (do_stats) {
-        int rc = do_sample_stats(h, dg, s);
-        if (rc) return rc;
+    // copy blocks [b0, b1); blocks that are contiguous on both sides travel in one copy
+    auto copy_range = [&](int b0, int b1, cudaStream_t cs) -> cudaError_t {
+        int i = b0;
+        while (i < b1) {
+            int j = i;
+            size_t bytes = 2 * size_t(h->blocks[i].numel);
+            while (j + 1 < b1 &&
+                   static_cast<const char*>(host_grads[j + 1]) == static_cast<const char*>(host_grads[i]) + bytes &&
+                   static_cast<const char*>(dev_grads[j + 1]) == static_cast<const char*>(dev_grads[i]) + bytes) {
+                ++j;
+                bytes += 2 * size_t(h->blocks[j].numel);
+            }
+            cudaError_t e = cudaMemcpyAsync(dev_grads[i], host_grads[i], bytes, cudaMemcpyHostToDevice, cs);
+            if (e != cudaSuccess) return e;
+            i = j + 1;
+        }
+        return cudaSuccess;
+    };
+    if (!do_stats) {
+        CU(copy_range(0, h->n_blocks, s), "baoc_step_from_host (copy)");
+        if (step_t > 0) return do_step(h, dg, params, step_t, s);
+        return BAOC_OK;
     }
+    // With statistics: the copy runs on an internal stream in up to kCopyGroups groups of whole blocks, and the
+    // caller's stream observes a group as soon as it has landed, so the statistics pass hides behind the transfer.
+    if (!h->copy_stream) {
+        cudaStream_t cs;
+        CU(cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking), "baoc_step_from_host (copy stream)");
+        h->copy_stream = cs;
+        for (void*& e : h->copy_ev) {
+            cudaEvent_t ev;
+            CU(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming), "baoc_step_from_host (event)");
+            e = ev;
+        }
+        h->cuda_cleanup = destroy_cuda_objects;
+    }
+    cudaStream_t cs = static_cast<cudaStream_t>(h->copy_stream);
+    int rc = sync_pointer_table(h, dg, &h->last_stat_grads, h->ws + h->sl.grads, s, "baoc_step_from_host");
+    if (rc) return rc;
+    // the copies must not overtake earlier work of the caller's stream that still reads the device gradients
+    CU(cudaEventRecord(static_cast<cudaEvent_t>(h->copy_ev[Handle::kCopyGroups]), s), "baoc_step_from_host");
+    CU(cudaStreamWaitEvent(cs, static_cast<cudaEvent_t>(h->copy_ev[Handle::kCopyGroups]), 0), "baoc_step_from_host");
+    const int64_t per_group = (h->numel + Handle::kCopyGroups - 1) / Handle::kCopyGroups;
+    int b0 = 0, g = 0;
+    while (b0 < h->n_blocks) {
+        int b1 = b0;
+        int64_t acc = 0;
+        while (b1 < h->n_blocks && (acc < per_group || g == Handle::kCopyGroups - 1)) acc += h->blocks[b1++].numel;
+        CU(copy_range(b0, b1, cs), "baoc_step_from_host (copy)");
+        CU(cudaEventRecord(static_cast<cudaEvent_t>(h->copy_ev[g]), cs), "baoc_step_from_host");
+        CU(cudaStreamWaitEvent(s, static_cast<cudaEvent_t>(h->copy_ev[g]), 0), "baoc_step_from_host");
+        rc = stats_step_range(h, b0, b1, s);
+        if (rc) return rc;
+        b0 = b1;
+        ++g;
+    }
+    rc = stats_combine_all(h, s);
+    if (rc) return rc;
     if (step_t > 0) return do_step(h, dg, params, step_t, s);
     return BAOC_OK;
 }
 
-static void destroy_profile_events(Handle* h) {
-    for (void*& e : h->prof_ev) {
-        if (e) cudaEventDestroy(static_cast<cudaEvent_t>(e));
-        e = nullptr;
-    }
-}
+
 
 int baoc_profile(baoc_t* h, int enable) {
     if (!h) return BAOC_E_INVALID;
@@ -588,7 +654,7 @@ int baoc_profile(baoc_t* h, int enable) {
             CU(cudaEventCreate(&ev), "baoc_profile");
             e = ev;
         }
-        h->cuda_cleanup = destroy_profile_events;
+        h->cuda_cleanup = destroy_cuda_objects;
     }
     h->prof_on = enable != 0;
     h->prof_valid = false;

@@ -201,6 +201,10 @@ struct Handle {
     // optional per-kernel timing of the step (CUDA events, owned by the CUDA translation unit)
     bool prof_on = false, prof_valid = false;
     void* prof_ev[3] = {nullptr, nullptr, nullptr};
+    // host-to-device pipeline of baoc_step_from_host: an internal copy stream and one event per group of blocks
+    static constexpr int kCopyGroups = 8;
+    void* copy_stream = nullptr;
+    void* copy_ev[kCopyGroups + 1] = {};
     void (*cuda_cleanup)(Handle*) = nullptr;
     ~Handle() { if (cuda_cleanup) cuda_cleanup(this); }
 };

@@ -502,6 +502,35 @@ def test_measured_time_ratios_leave_parameters_and_state_alone(B, H):
     assert e.value.code == B.E_INVALID
 
 
+def test_step_from_host_equals_separate_calls_bit_for_bit(B, H):
+    """The end-to-end call (pinned host gradients, copy pipelined with the statistics pass in groups of blocks) leaves
+    exactly what baoc_sample_stats + baoc_step leave on device-resident gradients."""
+    wl = W.make_workload("resnet50", seed=3)
+    assign = [(i % 5) if not ((i % 5) == 3 and b.cols <= 1) else 1 for i, b in enumerate(wl.blocks)]
+    res = []
+    for from_host in (False, True):
+        sess = H.Session(wl, n_grad_sets=2, pinned_host_grads=from_host)
+        sess.init_params()
+        sess.configure(assign)
+        for t in (1, 2, 3):
+            k = sess.fill_grads(t)
+            if from_host:
+                sess.host_copy_of_grads(k)
+                torch.cuda.synchronize()
+                sess.grads[k].zero_()                                   # the device copy must come from the host buffer
+                sess.step_from_host(k, True, t)
+            else:
+                sess.sample_stats(k)
+                sess.step(k, t)
+        torch.cuda.synchronize()
+        res.append((sess.params.clone(), sess.ws.clone()[sess.h.view(0, 0)[0] - sess.ws.data_ptr():], sess.h.read_stats()))
+    assert torch.equal(res[0][0], res[1][0])
+    n_m = sum((b.numel + 255) // 256 * 256 for b in wl.blocks) * 4
+    assert torch.equal(res[0][1][:2 * n_m], res[1][1][:2 * n_m])      # both moment arrays
+    for a, b2 in zip(res[0][2], res[1][2]):
+        assert a["rho_bar"] == b2["rho_bar"] and a["last_cos"] == b2["last_cos"] and a["n_cos"] == b2["n_cos"] == 2
+
+
 def test_checkpoint_resume_continues_bit_exactly(B, H):
     """Export after a window and some steps, move every buffer to a new address, import into a fresh handle, and
     let both handles continue on the same gradients: parameters, states and running statistics stay identical."""
