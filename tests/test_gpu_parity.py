@@ -1,7 +1,7 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU oracle
 on the same seeded inputs.
 
-Tolerances (from the benchmark spec):
+Tolerances:
   * statistics: 1e-4 relative (bounded signals are compared against
     max(|ref|, 1e-3) so that a cosine near zero is not held to 1e-4 of nothing);
   * fp32 states and parameters after 10 steps: max|diff| <= 1e-6 * max|ref| per
