@@ -1,6 +1,7 @@
-"""Parity at the benchmark's full size: the LLaMA-1B-shaped workload (1.14 B parameters, 146 blocks), in the
-launch configuration ``bench.py`` times (same tables, same tiles, the library's own budgeted assignment), checked
-on sampled outputs that the CPU oracle can compute one by one:
+"""Parity at full size: the LLaMA-1B-shaped workload (1.14 B parameters, 146 blocks) in the launch configuration
+``bench.py`` times (same tables, same tiles, the library's own budgeted assignment), and likewise the diffusion-UNet-
+shaped (0.86 B parameters, per-level noise scales) and GPT-2-small-shaped (124 M parameters, Student-t gradients in the
+embedding and attention blocks) workloads, checked on sampled outputs that the CPU oracle can compute one by one:
 
   * statistics of whole sampled blocks (a vector, a 4 M and a 16.7 M matrix), and the window values plus the
     anisotropy / signal-to-noise of the largest block (the 65.5 M-element token table);
@@ -41,16 +42,28 @@ def _slices(numel):
     return [(0, 8192), (mid, mid + 8192), (last, numel)]
 
 
-def test_llama_1b_sampled_parity_in_the_benchmark_configuration():
+CASES = {
+    # workload: (parameter count or None, blocks with whole-block statistics, the largest block)
+    "llama_1b": (1_139_345_408, ["l0.norm1", "l3.attn.k", "l5.ffn.up"], "tok_emb"),
+    "unet": (None, ["in.b", "down1.attn0.self.q.w", "mid.attn.ff.gate.w"], "up3.res0.conv1.w"),
+    "gpt2_small": (124_439_808, ["h0.ln1.w", "h3.attn.out.w", "h7.mlp.fc.w"], "tok_emb"),
+}
+
+
+@pytest.mark.parametrize("name", ["llama_1b", "unet", "gpt2_small"])
+def test_sampled_parity_at_full_size(name):
     from paper_2605_04711_b200 import harness as H
-    wl = W.make_workload("llama_1b", seed=0)
-    assert wl.numel == 1_139_345_408 and len(wl.blocks) == 146
+    wl = W.make_workload(name, seed=0)
+    numel, full_names, big_name = CASES[name]
+    assert numel is None or wl.numel == numel
+    if name == "unet":
+        assert abs(wl.numel - 860e6) <= 0.02 * 860e6
     sess = H.Session(wl, n_grad_sets=2)
     sess.init_params()
     o = O.Opts()
     name_to_i = {b.name: i for i, b in enumerate(wl.blocks)}
-    full = [name_to_i["l0.norm1"], name_to_i["l3.attn.k"], name_to_i["l5.ffn.up"]]     # whole-block statistics
-    big = name_to_i["tok_emb"]                                                          # 65 536 000 elements
+    full = [name_to_i[n] for n in full_names]                       # whole-block statistics
+    big = name_to_i[big_name]                                       # the workload's largest block
     states = {i: O.stats_init(wl.blocks[i].numel) for i in full + [big]}
     for t in range(1, T_WINDOW + 1):
         k = sess.fill_grads(t)
@@ -76,7 +89,7 @@ def test_llama_1b_sampled_parity_in_the_benchmark_configuration():
                     "err_m8", "err_v8", "err_m16", "err_v16"):
             extra = T_WINDOW * 2.0 ** -23 if key.startswith("err_") else 0.0
             assert _close(st[i][key], raw[key], extra), (b.name, key, st[i][key], raw[key])
-    # the largest block: exact quantiles over 65.5 M elements (radix select across 16 000 tiles) and the SNR
+    # the largest block: exact quantiles (radix select across all of its tiles; 65.5 M elements for LLaMA-1B) and the SNR
     assert _close(st[big]["A"], O.anisotropy(states[big].v, o.eps)), (st[big]["A"],)
     assert _close(st[big]["snr"], O.snr(states[big].m, states[big].v, o.eps))
     del states, mv
