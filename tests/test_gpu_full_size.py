@@ -157,3 +157,58 @@ def test_sampled_parity_at_full_size(name):
             assert rel(f32(13, q0, q1), ref.av.astype(np.float64)) <= 1e-6, name
     if n_codes:
         assert bad_codes <= 1e-4 * n_codes, (bad_codes, n_codes)
+
+
+def test_one_block_beyond_two_to_the_31_elements():
+    """Indexing past 32 bits: a single 32769 x 65537 block (2^31 + 98305 elements, odd row length, ragged tail; rows
+    and columns are 32-bit in the ABI, their product is not) through the statistics pass and the fused step (SGD with
+    momentum, so there is per-element state), checked on slices at the start, around element 2^31 and at the very
+    end."""
+    from paper_2605_04711_b200 import binding as B
+    dev = torch.device("cuda:0")
+    rows, cols = 32769, 65537
+    n = rows * cols
+    assert n > 2 ** 31
+    cfgs = [B.make_config(0, 1, 1, 0, 32, lr=1e-2, beta1=0.9, weight_decay=0.01)]
+    h = B.Baoc([(n, rows, cols)], cfgs)
+    gen = torch.Generator(device=dev).manual_seed(5)
+    theta = torch.empty(n, dtype=torch.float32, device=dev)
+    grads = [torch.empty(n, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    chunk = 2 ** 27
+    for lo in range(0, n, chunk):                                      # chunked: no full-size fp32 temporaries
+        hi = min(n, lo + chunk)
+        theta[lo:hi] = 0.02 * torch.randn(hi - lo, generator=gen, device=dev)
+        for g in grads:
+            g[lo:hi] = (0.01 * torch.randn(hi - lo, generator=gen, device=dev)).to(torch.bfloat16)
+    ws = torch.empty(h.stats_workspace_bytes(), dtype=torch.uint8, device=dev)
+    h.bind_stats_workspace(ws)
+    state = torch.empty(h.state_bytes([0]), dtype=torch.uint8, device=dev)
+    h.configure([0], state)
+    windows = [(0, 8192), (2 ** 31 - 4096, 2 ** 31 + 4096), (n - 5000, n)]
+    th0 = [theta[a:b].double().cpu().numpy() for a, b in windows]
+    o = O.Opts()
+    for k in (0, 1):
+        h.sample_stats([grads[k]])
+        h.step([grads[k]], [theta], k + 1)
+    torch.cuda.synchronize()
+    run = h.read_stats()[0]
+    # the cosine of the two gradients over all 2^31 + 4100 elements, from chunked double-precision dot products
+    dot = n1 = n2 = 0.0
+    for lo in range(0, n, chunk):
+        a, b = grads[0][lo:lo + chunk].double(), grads[1][lo:lo + chunk].double()
+        dot += float(a @ b); n1 += float(a @ a); n2 += float(b @ b)
+    want = dot / (np.sqrt(n1) * np.sqrt(n2) + o.eps)
+    assert abs(run["last_cos"] - want) <= 1e-4 * max(abs(want), 1e-3) and run["n_cos"] == 1
+    c = O.Config(0, 1, 1, 0, 32, lr=float(cfgs[0].lr), beta1=float(cfgs[0].beta1), weight_decay=float(cfgs[0].weight_decay))
+    m_dev = h.view_tensor(0, 10, torch.float32)
+    mhat = h.view_tensor(0, 0, torch.float32)
+    for (a, b), t0 in zip(windows, th0):
+        st, ss, th = O.step_init(c, b - a, b - a, 1), O.stats_init(b - a), t0
+        for k in (0, 1):
+            g = grads[k][a:b].double().cpu().numpy()
+            O.stats_step(ss, g, o)
+            th = O.step(th, g, st, c, b - a, 1)
+        got = theta[a:b].double().cpu().numpy()
+        assert np.max(np.abs(got - th)) <= 1e-6 * np.max(np.abs(th)), (a, b)
+        assert np.max(np.abs(m_dev[a:b].double().cpu().numpy() - st.m)) <= 1e-6 * np.max(np.abs(st.m))
+        assert np.max(np.abs(mhat[a:b].double().cpu().numpy() - ss.m)) <= 1e-6 * np.max(np.abs(ss.m))
