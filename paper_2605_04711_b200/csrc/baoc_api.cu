@@ -102,16 +102,19 @@ int do_sample_stats(Handle* h, const void* const* grads, cudaStream_t s) {
 
 void fill_step_params(const Handle* h, int64_t t, StepParams* P) {
     std::memset(P, 0, sizeof(*P));
-    for (int c = 0; c < h->n_cfg; ++c) {
-        const baoc_config_t& k = h->cfgs[c];
-        CfgStep& o = P->c[c];
+    for (size_t sl = 0; sl < h->slots.size(); ++sl) {
+        const Handle::Slot& slot = h->slots[sl];
+        const baoc_config_t& k = h->cfgs[slot.cfg];
+        CfgStep& o = P->c[sl];
         const double b1 = double(k.beta1), b2 = double(k.beta2), lr = double(k.lr);
         o.beta1 = k.beta1; o.beta2 = k.beta2; o.eps = k.eps; o.wd = k.weight_decay;
         o.om1 = float(1.0 - b1); o.om2 = float(1.0 - b2);
         const bool has_wd = k.weight_decay != 0.0f;
         o.coupled = (has_wd && !k.decoupled_wd) ? 1 : 0;
         o.decay = (has_wd && k.decoupled_wd) ? -float(lr * double(k.weight_decay)) : 0.0f;
-        const double bc1 = 1.0 - std::pow(b1, double(t)), bc2 = 1.0 - std::pow(b2, double(t));
+        // each moment counts the gradients it has seen since it last started from zero
+        const double tm = double(std::max<int64_t>(1, t - slot.t_m0)), tv = double(std::max<int64_t>(1, t - slot.t_v0));
+        const double bc1 = 1.0 - std::pow(b1, tm), bc2 = 1.0 - std::pow(b2, tv);
         o.step_m = float(lr / bc1);
         o.step_g = k.lr;
         o.rsqrt_bc2 = float(1.0 / std::sqrt(bc2));
@@ -120,6 +123,25 @@ void fill_step_params(const Handle* h, int64_t t, StepParams* P) {
         o.eps_hat = float(double(k.eps) * std::sqrt(bc2));
         o.beta1_d = b1; o.beta2_d = b2; o.wd_d = double(k.weight_decay);
     }
+}
+
+// Group the blocks into slots by (configuration, moment start steps); writes the slot index into the block records.
+int build_slots(Handle* h, const int32_t* assign, std::vector<StepBlock>* sb) {
+    h->slots.clear();
+    h->slot_of.assign(h->n_blocks, 0);
+    for (int i = 0; i < h->n_blocks; ++i) {
+        const Handle::Slot want{assign[i], h->t_m0[i], h->t_v0[i]};
+        size_t k = 0;
+        for (; k < h->slots.size(); ++k)
+            if (h->slots[k].cfg == want.cfg && h->slots[k].t_m0 == want.t_m0 && h->slots[k].t_v0 == want.t_v0) break;
+        if (k == h->slots.size()) {
+            if (k == size_t(kMaxSlots)) return fail(h, BAOC_E_INVALID, "too many distinct (configuration, moment start step) combinations for one step");
+            h->slots.push_back(want);
+        }
+        h->slot_of[i] = int32_t(k);
+        (*sb)[i].cfg = int32_t(k);
+    }
+    return BAOC_OK;
 }
 
 int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t, cudaStream_t s) {
@@ -359,6 +381,9 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
     int rc = compute_step_layout(h, assign, &L, &sb, &tiles, &red, &mem, &traffic);
     if (rc) return rc;
     if (bytes < L.total) return fail(h, BAOC_E_WORKSPACE, "baoc_configure: state buffer too small");
+    if (reset || h->t_m0.size() != size_t(h->n_blocks)) { h->t_m0.assign(h->n_blocks, 0); h->t_v0.assign(h->n_blocks, 0); }
+    rc = build_slots(h, assign, &sb);
+    if (rc) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* st = static_cast<char*>(state_dev);
     const int n = h->n_blocks;
@@ -521,17 +546,23 @@ uint64_t shape_hash(const Handle* h) {
 int baoc_export(const baoc_t* h, void* buf, size_t capacity, size_t* size) {
     if (!h) return BAOC_E_INVALID;
     if (!size) return fail(h, BAOC_E_INVALID, "baoc_export: null size");
-    const size_t need = sizeof(BlobHeader) + (h->configured ? 4 * size_t(h->n_blocks) : 0);
+    const size_t need = sizeof(BlobHeader) + (h->configured ? (4 + 16) * size_t(h->n_blocks) : 0);
     *size = need;
     if (!buf) return BAOC_OK;
     if (capacity < need) return fail(h, BAOC_E_WORKSPACE, "baoc_export: buffer too small");
     BlobHeader hd{};
-    hd.magic = kBlobMagic; hd.version = 1; hd.n_blocks = h->n_blocks; hd.n_cfg = h->n_cfg;
+    hd.magic = kBlobMagic; hd.version = 2; hd.n_blocks = h->n_blocks; hd.n_cfg = h->n_cfg;
     hd.numel = h->numel; hd.stats_steps = h->stats_steps;
     hd.ws_bound = h->ws_bound ? 1 : 0; hd.configured = h->configured ? 1 : 0;
     hd.shape_hash = shape_hash(h);
     std::memcpy(buf, &hd, sizeof(hd));
-    if (h->configured) std::memcpy(static_cast<char*>(buf) + sizeof(hd), h->assign.data(), 4 * size_t(h->n_blocks));
+    if (h->configured) {                                   // assignment, then the moment start steps of every block
+        char* p = static_cast<char*>(buf) + sizeof(hd);
+        const size_t n = size_t(h->n_blocks);
+        std::memcpy(p, h->assign.data(), 4 * n);
+        std::memcpy(p + 4 * n, h->t_m0.data(), 8 * n);
+        std::memcpy(p + 12 * n, h->t_v0.data(), 8 * n);
+    }
     return BAOC_OK;
 }
 
@@ -541,11 +572,11 @@ int baoc_import(baoc_t* h, const void* blob, size_t size, void* ws_dev, size_t w
     if (!blob || size < sizeof(BlobHeader)) return fail(h, BAOC_E_INVALID, "baoc_import: blob missing or truncated");
     BlobHeader hd;
     std::memcpy(&hd, blob, sizeof(hd));
-    if (hd.magic != kBlobMagic || hd.version != 1) return fail(h, BAOC_E_INVALID, "baoc_import: not a blob of this library version");
+    if (hd.magic != kBlobMagic || hd.version != 2) return fail(h, BAOC_E_INVALID, "baoc_import: not a blob of this library version");
     if (hd.n_blocks != h->n_blocks || hd.n_cfg != h->n_cfg || hd.numel != h->numel || hd.shape_hash != shape_hash(h))
         return fail(h, BAOC_E_INVALID, "baoc_import: the blob belongs to a different block set or candidate set");
     if (hd.stats_steps < 0) return fail(h, BAOC_E_INVALID, "baoc_import: corrupt blob");
-    if (hd.configured && size < sizeof(BlobHeader) + 4 * size_t(h->n_blocks)) return fail(h, BAOC_E_INVALID, "baoc_import: blob truncated");
+    if (hd.configured && size < sizeof(BlobHeader) + 20 * size_t(h->n_blocks)) return fail(h, BAOC_E_INVALID, "baoc_import: blob truncated");
     if (hd.ws_bound && !ws_dev) return fail(h, BAOC_E_INVALID, "baoc_import: the checkpoint had a statistics workspace; pass its copy");
     if (hd.configured && !state_dev) return fail(h, BAOC_E_INVALID, "baoc_import: the checkpoint had optimizer state; pass its copy");
     if (hd.ws_bound) {
@@ -556,6 +587,10 @@ int baoc_import(baoc_t* h, const void* blob, size_t size, void* ws_dev, size_t w
     if (hd.configured) {
         std::vector<int32_t> assign(h->n_blocks);
         std::memcpy(assign.data(), static_cast<const char*>(blob) + sizeof(BlobHeader), 4 * size_t(h->n_blocks));
+        const char* p = static_cast<const char*>(blob) + sizeof(BlobHeader) + 4 * size_t(h->n_blocks);
+        h->t_m0.resize(h->n_blocks); h->t_v0.resize(h->n_blocks);
+        std::memcpy(h->t_m0.data(), p, 8 * size_t(h->n_blocks));
+        std::memcpy(h->t_v0.data(), p + 8 * size_t(h->n_blocks), 8 * size_t(h->n_blocks));
         int rc = configure_state(h, assign.data(), state_dev, state_bytes, stream, false);
         if (rc) return rc;
     }

@@ -15,6 +15,7 @@ typedef CUstream_st* cudaStream_t;
 namespace baoc {
 
 constexpr int kMaxCfg = 32;
+constexpr int kMaxSlots = 48;         // distinct (configuration, moment start steps) combinations one step can carry
 constexpr int kQBlock = 256;          // elements per 8-bit quantisation block
 constexpr int kTile = 4096;           // elements per tile of the streaming kernels
 constexpr int kThreads = 256;         // threads per CTA of the streaming kernels
@@ -105,7 +106,8 @@ struct StepBlock {
     double* mean_part;   // F: kCombineSlabs partial sums of the new r, then one ticket counter (uint32)
     int64_t numel;
     int32_t rows, cols;
-    int32_t cfg;
+    int32_t cfg;         // slot of the step's parameter table: the configuration together with the steps at which the
+                         // block's moments last started from zero (they set the bias corrections)
     int32_t path;
     RedGeom red;
 };
@@ -145,7 +147,7 @@ struct CfgStep {
     double wd_d;
 };
 struct StepParams {
-    CfgStep c[kMaxCfg];
+    CfgStep c[kMaxSlots];
 };
 
 struct Handle {
@@ -190,6 +192,13 @@ struct Handle {
     int64_t n_step_red_tiles = 0;
     int n_factored = 0;              // blocks on the factored path
     bool wide_paths = false;         // some block is on a path outside the five headline ones
+    // Bias corrections count the gradients a moment has seen.  A re-configuration may restart some moments, so every
+    // block carries the step counts at which its first and second moment last started from zero; blocks that share a
+    // configuration and both counts share a slot of the step's parameter table.
+    struct Slot { int32_t cfg; int64_t t_m0, t_v0; };
+    std::vector<int64_t> t_m0, t_v0;
+    std::vector<Slot> slots;
+    std::vector<int32_t> slot_of;
     int64_t state_mem = 0;           // StateMem of the assignment (sum of M_{i,c_i})
     int64_t step_bytes = 0;          // algorithmic bytes of one step
     std::vector<const void*> last_step_grads;
