@@ -257,6 +257,29 @@ int baoc_state_bytes(const baoc_t* h, const int32_t* assign, size_t* bytes);
 int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes,
                    baoc_stream_t stream);
 
+/* Online re-configuration with optimizer-state inheritance (Sec. 3.1, remark on
+ * re-planning; appendix study "online reallocation with state inheritance").
+ * The paper says only that compatible states are migrated when possible; this
+ * library's rule, with inherit != 0:
+ *   - a first moment is kept between tuples of the same family (Adam-type
+ *     averages, or momentum buffers of SGD), re-stored in the new precision;
+ *   - an element-wise second moment (Adam, RMS scaling) is kept by any tuple
+ *     with an element-wise second moment, and becomes its row and column means
+ *     under the factored tuple; a factored one becomes r_i c_j / mean(r)
+ *     element-wise;
+ *   - every other moment of the new tuple starts from zero, and its bias
+ *     correction restarts: it counts steps from steps_done.
+ * With inherit == 0 every moment restarts.  new_assign: host [n_blocks].
+ * new_state_dev: device, 256-byte aligned, >= baoc_state_bytes(new_assign), and
+ * NOT overlapping the current state buffer, which is read while the new one is
+ * written (the transient memory the paper's remark mentions); once the stream
+ * has passed this call the old buffer may be freed.  steps_done: the number of
+ * baoc_step calls made so far (the next call passes steps_done + 1).  Queues
+ * the zero-fill, the table uploads and the migration kernels; does not wait.
+ * BAOC_E_STATE before the first baoc_configure. */
+int baoc_reconfigure(baoc_t* h, const int32_t* new_assign, void* new_state_dev, size_t bytes,
+                     int64_t steps_done, int inherit, baoc_stream_t stream);
+
 /* One training step of every block under its configuration.  grads / params:
  * host arrays of n_blocks device pointers (bf16 / fp32).  step_t: 1-based step
  * number (bias corrections).  Queues the fused update kernel (preceded by the

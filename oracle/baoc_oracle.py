@@ -420,11 +420,14 @@ def _prologue(theta: np.ndarray, g: np.ndarray, c: Config):
     return theta, g
 
 
-def _adam_apply(theta, m, v, c: Config, t: int, use_m: bool):
-    bc2 = 1.0 - c.beta2 ** t
+def _adam_apply(theta, m, v, c: Config, t, use_m: bool):
+    """t: the step count, or a pair (t_m, t_v) when the two moments have been accumulating for different numbers of
+    steps (after a re-configuration that restarted one of them)."""
+    t_m, t_v = t if isinstance(t, tuple) else (t, t)
+    bc2 = 1.0 - c.beta2 ** t_v
     denom = np.sqrt(v / bc2) + c.eps
     if use_m:
-        bc1 = 1.0 - c.beta1 ** t
+        bc1 = 1.0 - c.beta1 ** t_m
         return theta - c.lr * (m / bc1) / denom
     return theta - c.lr * m / denom
 
@@ -434,6 +437,8 @@ class StepState:
     """Optimizer state of one block under one configuration."""
     kind: str
     t: int = 0
+    t_m0: int = 0      # step counts at which the first / second moment last started from zero
+    t_v0: int = 0
     m: Optional[np.ndarray] = None
     v: Optional[np.ndarray] = None
     qm: Optional[np.ndarray] = None
@@ -495,7 +500,7 @@ def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, 
     theta = np.asarray(theta, dtype=F64)
     g = np.asarray(g, dtype=F64)
     st.t += 1
-    t = st.t
+    t = (max(1, st.t - st.t_m0), max(1, st.t - st.t_v0))     # gradients each moment has seen, this one included
     theta, g = _prologue(theta, g, c)
     if st.kind == "A32":
         st.m = c.beta1 * st.m + (1.0 - c.beta1) * g
@@ -557,3 +562,69 @@ def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, 
         st.m = c.beta1 * st.m + g
         return theta - c.lr * st.m
     raise ValueError("unsupported configuration tuple")
+
+
+# ----------------------------------------------------------------------------
+# Re-configuration with state inheritance (online variant, Sec. 3.1 remark and
+# the appendix study "online reallocation with state inheritance").  The paper
+# says only that compatible optimizer states are migrated when possible; the
+# reading here:
+#   * a first moment is inherited between configurations of the same family
+#     (Adam-type averages A32 / A16 / A8, or momentum buffers S / S16 / S8);
+#   * an element-wise second moment (A*, R*) is inherited by any configuration
+#     with an element-wise second moment; by a factored one as its row and
+#     column means; a factored one becomes r_i c_j / mean(r) element-wise;
+#   * the value is re-stored in the new precision (fp32, bf16, 8-bit codes);
+#   * a moment that cannot be inherited starts from zero, and its bias
+#     correction restarts (its start step becomes the current step count).
+# ----------------------------------------------------------------------------
+
+_M_FAMILY = {"A32": "avg", "A16": "avg", "A8": "avg", "S": "sum", "S16": "sum", "S8": "sum"}
+_V_FAMILY = {"A32": "full", "A16": "full", "A8": "full", "R": "full", "R16": "full", "R8": "full", "F": "factored"}
+_BITS = {"A32": 32, "A16": 16, "A8": 8, "R": 32, "R16": 16, "R8": 8, "S": 32, "S16": 16, "S8": 8, "F": 32, "G": 32}
+
+
+def _moment_value(st: StepState, which: str, rows: int, cols: int, qblock: int) -> Optional[np.ndarray]:
+    """The moment as the old configuration holds it, in double (None if it has none)."""
+    if which == "m":
+        if st.kind in ("A8", "S8"):
+            return dequantize8(st.qm, st.am, True, qblock)
+        return None if st.m is None else np.asarray(st.m, F64)
+    if st.kind in ("A8", "R8"):
+        return dequantize8(st.qv, st.av, False, qblock)
+    if st.kind == "F":
+        rm = float(np.mean(st.r))
+        return np.zeros(rows * cols, F64) if rm == 0.0 else (np.outer(st.r, st.c) / rm).reshape(-1)
+    return None if st.v is None else np.asarray(st.v, F64)
+
+
+def reconfigure(st: StepState, c_new: Config, rows: int, cols: int, inherit: bool = True, qblock: int = 256) -> StepState:
+    """The state of one block under ``c_new``, given its state ``st`` under the old configuration after ``st.t`` steps."""
+    numel = rows * cols
+    kind = config_kind(c_new)
+    new = step_init(c_new, numel, rows, cols, qblock)
+    new.t = st.t
+    new.t_m0 = new.t_v0 = st.t                                   # until inherited below
+    old_m = _moment_value(st, "m", rows, cols, qblock) if inherit and _M_FAMILY.get(st.kind) == _M_FAMILY.get(kind) else None
+    old_v = _moment_value(st, "v", rows, cols, qblock) if inherit and st.kind in _V_FAMILY and kind in _V_FAMILY else None
+    bits = _BITS[kind]
+    if kind in _M_FAMILY and old_m is not None:
+        new.t_m0 = st.t_m0
+        if bits == 8:
+            new.qm, new.am = quantize8(old_m, True, qblock)
+        else:
+            new.m = round_bf16(old_m) if bits == 16 else old_m.astype(np.float32).astype(F64)
+    if kind in _V_FAMILY and old_v is not None:
+        new.t_v0 = st.t_v0
+        if kind == "F":
+            if st.kind == "F":
+                new.r, new.c = st.r.copy(), st.c.copy()
+            else:
+                V = old_v.reshape(rows, cols)
+                new.r = V.mean(axis=1).astype(np.float32).astype(F64)
+                new.c = V.mean(axis=0).astype(np.float32).astype(F64)
+        elif bits == 8:
+            new.qv, new.av = quantize8(old_v, False, qblock)
+        else:
+            new.v = round_bf16(old_v) if bits == 16 else old_v.astype(np.float32).astype(F64)
+    return new

@@ -369,7 +369,10 @@ int baoc_state_bytes(const baoc_t* h, const int32_t* assign, size_t* bytes) {
     return BAOC_OK;
 }
 
-static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes, baoc_stream_t stream, bool reset) {
+// reset: zero the state and restart every moment's step count;  zero_only: zero the state, keep the counts the
+// caller has just set (re-configuration);  neither: leave both alone (resume from a checkpoint).
+static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes, baoc_stream_t stream, bool reset,
+                           bool zero_only = false) {
     if (!h) return BAOC_E_INVALID;
     if (!assign || !state_dev) return fail(h, BAOC_E_INVALID, "baoc_configure: null argument");
     if (reinterpret_cast<uintptr_t>(state_dev) & 255u) return fail(h, BAOC_E_ALIGN, "baoc_configure: state buffer not 256-byte aligned");
@@ -410,7 +413,7 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
         CU(cudaMemcpyAsync(st + L.red_tiles, red.data(), sizeof(RedTile) * red.size(), cudaMemcpyHostToDevice, s), "upload step reduction table");
     if (!ids.empty())
         CU(cudaMemcpyAsync(st + L.f_ids, ids.data(), 4 * ids.size(), cudaMemcpyHostToDevice, s), "upload factored ids");
-    if (reset) CU(cudaMemsetAsync(st + L.flags, 0, L.total - L.flags, s), "zero optimizer state");
+    if (reset || zero_only) CU(cudaMemsetAsync(st + L.flags, 0, L.total - L.flags, s), "zero optimizer state");
     h->st = st; h->st_bytes = bytes; h->tl = L; h->configured = true;
     h->assign.assign(assign, assign + n);
     h->h_step_blocks = sb;
@@ -425,6 +428,85 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
 
 int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes, baoc_stream_t stream) {
     return configure_state(h, assign, state_dev, bytes, stream, true);
+}
+
+// ---- online re-configuration with state inheritance ----------------------------------
+namespace {
+// Which family a path's first moment belongs to (1: Adam-type average, 2: momentum buffer, 0: none).
+int m_family(int path) {
+    switch (path) {
+        case kPathA32: case kPathA16: case kPathA8: return 1;
+        case kPathS: case kPathS16: case kPathS8: return 2;
+        default: return 0;
+    }
+}
+MomentRef first_moment(const StepBlock& b) {
+    MomentRef r{};
+    r.rows = b.rows; r.cols = b.cols;
+    switch (b.path) {
+        case kPathA32: case kPathS: r.data = b.s0; r.kind = kMomF32; break;
+        case kPathA16: case kPathS16: r.data = b.s0; r.kind = kMomBF16; break;
+        case kPathA8: case kPathS8: r.data = b.s0; r.absmax = b.a0; r.kind = kMomI8; break;
+        default: r.kind = kMomNone; break;
+    }
+    return r;
+}
+MomentRef second_moment(const StepBlock& b) {
+    MomentRef r{};
+    r.rows = b.rows; r.cols = b.cols;
+    switch (b.path) {
+        case kPathA32: r.data = b.s1; r.kind = kMomF32; break;
+        case kPathA16: r.data = b.s1; r.kind = kMomBF16; break;
+        case kPathA8: case kPathR8: r.data = b.s1; r.absmax = b.a1; r.kind = kMomU8; break;
+        case kPathR: r.data = b.s0; r.kind = kMomF32; break;
+        case kPathR16: r.data = b.s0; r.kind = kMomBF16; break;
+        case kPathF: r.r = static_cast<const float*>(b.s0); r.c = static_cast<const float*>(b.s1); r.kind = kMomFactored; break;
+        default: r.kind = kMomNone; break;
+    }
+    return r;
+}
+}  // namespace
+
+int baoc_reconfigure(baoc_t* h, const int32_t* new_assign, void* new_state_dev, size_t bytes, int64_t steps_done,
+                     int inherit, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!new_assign || !new_state_dev) return fail(h, BAOC_E_INVALID, "baoc_reconfigure: null argument");
+    if (!h->configured) return fail(h, BAOC_E_STATE, "baoc_reconfigure: no assignment configured yet");
+    if (steps_done < 0) return fail(h, BAOC_E_INVALID, "baoc_reconfigure: negative step count");
+    {   // the new buffer must not overlap the old one: the old state is read while the new one is written
+        const char* a = h->st; const char* b = static_cast<const char*>(new_state_dev);
+        if (b < a + h->tl.total && a < b + bytes) return fail(h, BAOC_E_INVALID, "baoc_reconfigure: the new state buffer overlaps the current one");
+    }
+    const int n = h->n_blocks;
+    const std::vector<StepBlock> old_blocks = h->h_step_blocks;
+    const std::vector<int64_t> old_tm = h->t_m0, old_tv = h->t_v0;
+    // which moments are inherited, and from there the start steps of the new moments
+    std::vector<char> keep_m(n, 0), keep_v(n, 0);
+    for (int i = 0; i < n; ++i) {
+        if (new_assign[i] < 0 || new_assign[i] >= h->n_cfg) return fail(h, BAOC_E_INVALID, "baoc_reconfigure: assignment names a configuration that does not exist");
+        const Path pn = path_of(h->cfgs[new_assign[i]]);
+        const int po = old_blocks[i].path;
+        keep_m[i] = inherit && m_family(pn) != 0 && m_family(pn) == m_family(po);
+        keep_v[i] = inherit && second_moment(old_blocks[i]).kind != kMomNone &&
+                    (pn == kPathA32 || pn == kPathA16 || pn == kPathA8 || pn == kPathR || pn == kPathR16 || pn == kPathR8 || pn == kPathF);
+        h->t_m0[i] = keep_m[i] ? old_tm[i] : steps_done;
+        h->t_v0[i] = keep_v[i] ? old_tv[i] : steps_done;
+    }
+    int rc = configure_state(h, new_assign, new_state_dev, bytes, stream, false, true);
+    if (rc) { h->t_m0 = old_tm; h->t_v0 = old_tv; return rc; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < n; ++i) {
+        const StepBlock& nb = h->h_step_blocks[i];
+        if (keep_m[i]) {
+            LAUNCH(launch_convert_moment(first_moment(old_blocks[i]), first_moment(nb), nb.numel, s), "convert_moment_kernel");
+            h->launches += 1;
+        }
+        if (keep_v[i]) {
+            LAUNCH(launch_convert_moment(second_moment(old_blocks[i]), second_moment(nb), nb.numel, s), "convert_moment_kernel");
+            h->launches += 1;
+        }
+    }
+    return BAOC_OK;
 }
 
 // ---- one-step timing of every (block, configuration) pair ---------------------------

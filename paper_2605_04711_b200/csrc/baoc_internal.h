@@ -112,6 +112,18 @@ struct StepBlock {
     RedGeom red;
 };
 
+// A stored moment, for the migration kernels of a re-configuration.
+enum MomentKind : int32_t { kMomNone = 0, kMomF32 = 1, kMomBF16 = 2, kMomI8 = 3, kMomU8 = 4, kMomFactored = 5 };
+struct MomentRef {
+    void* data;          // fp32 / bf16 values or 8-bit codes
+    float* absmax;       // one fp32 per 256 codes (8-bit kinds)
+    const float* r;      // factored: row statistics
+    const float* c;      // factored: column statistics
+    int32_t kind;
+    int32_t rows, cols;  // the block's shape
+    int32_t pad;
+};
+
 // State of one radix select: the bits found so far and the rank still to find
 // among the elements that share them.
 struct RankSel {
@@ -250,6 +262,7 @@ int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const
                            const float* const* params, int64_t n_red, int n_factored, const StepParams& P, cudaStream_t s);
 int launch_fused_step(const StepBlock* blocks, const Tile* tiles, const void* const* grads, float* const* params,
                       uint32_t* flags, int64_t n_tiles, bool all_paths, const StepParams& P, cudaStream_t s);
+int launch_convert_moment(const MomentRef& src, const MomentRef& dst, int64_t numel, cudaStream_t s);
 int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayout* out,
                         std::vector<StepBlock>* blocks, std::vector<Tile>* tiles,
                         std::vector<RedTile>* red, int64_t* state_mem, int64_t* step_bytes);

@@ -127,6 +127,13 @@ class Session:
         self.state = torch.empty(self.h.state_bytes(self.assign), dtype=torch.uint8, device=self.device)
         self.h.configure(self.assign, self.state)
 
+    def reconfigure(self, assign, steps_done: int, inherit: bool = True):
+        """Move to a new assignment in a fresh state buffer (the old one stays alive until the stream has passed)."""
+        self.assign = np.asarray(assign, np.int32)
+        new_state = torch.empty(self.h.state_bytes(self.assign), dtype=torch.uint8, device=self.device)
+        self.h.reconfigure(self.assign, new_state, steps_done, inherit)
+        self.state = new_state
+
     def step(self, k: int, t: int):
         self.h.step(self.grad_tables[k], self.param_table, t)
 

@@ -323,7 +323,8 @@ def _push_state(sess, i, th, st):
     """Write the oracle's parameters and state of block i into the device buffers."""
     dev = sess.device
     sess.param_views[i].copy_(torch.from_numpy(th.astype(np.float32)).to(dev))
-    put = lambda which, dt, a: sess.h.view_tensor(i, which, dt).copy_(torch.from_numpy(np.ascontiguousarray(a)).to(dev))
+    put = lambda which, dt, a: sess.h.view_tensor(i, which, dt).copy_(
+        (a if torch.is_tensor(a) else torch.from_numpy(np.ascontiguousarray(a))).to(dev))
     if st.kind == "A32":
         put(10, torch.float32, st.m.astype(np.float32)); put(11, torch.float32, st.v.astype(np.float32))
     elif st.kind == "A8":
@@ -335,6 +336,12 @@ def _push_state(sess, i, th, st):
         put(10, torch.float32, st.m.astype(np.float32))
     elif st.kind == "F":
         put(10, torch.float32, st.r.astype(np.float32)); put(11, torch.float32, st.c.astype(np.float32))
+    elif st.kind == "A16":
+        put(10, torch.bfloat16, torch.from_numpy(st.m).to(torch.bfloat16)); put(11, torch.bfloat16, torch.from_numpy(st.v).to(torch.bfloat16))
+    elif st.kind == "R16":
+        put(10, torch.bfloat16, torch.from_numpy(st.v).to(torch.bfloat16))
+    elif st.kind == "S16":
+        put(10, torch.bfloat16, torch.from_numpy(st.m).to(torch.bfloat16))
     elif st.kind == "R8":
         put(10, torch.uint8, st.qv); put(11, torch.float32, st.av)
     elif st.kind == "S8":
@@ -529,6 +536,63 @@ def test_step_from_host_equals_separate_calls_bit_for_bit(B, H):
     assert torch.equal(res[0][1][:2 * n_m], res[1][1][:2 * n_m])      # both moment arrays
     for a, b2 in zip(res[0][2], res[1][2]):
         assert a["rho_bar"] == b2["rho_bar"] and a["last_cos"] == b2["last_cos"] and a["n_cos"] == b2["n_cos"] == 2
+
+
+@pytest.mark.parametrize("inherit", [True, False])
+def test_reconfigure_migrates_states_like_the_oracle(B, H, inherit):
+    """Online re-configuration: three steps under one assignment, a move to another one (every pair of families and
+    precisions occurs), three more steps.  The states are synchronised oracle -> device before the move and before each
+    later step, so the migration itself and the per-moment bias corrections are what is compared."""
+    wl = _odd_workload(seed=81)
+    cfgs = B.extended_configs()                                     # 0 A32, 1 A8, 2 R, 3 F, 4 S, 5 G, 6 A16, 7 R16, 8 S16, 9 R8, 10 S8
+    sess = H.Session(wl, configs=cfgs, n_grad_sets=2)
+    sess.init_params()
+    n = len(wl.blocks)
+    ocfgs = [_ocfg(c) for c in cfgs]
+    old = [0, 1, 6, 2, 9, 4, 10, 0, 3, 3, 1, 8, 5, 7, 0]
+    new = [1, 0, 1, 0, 2, 8, 4, 4, 2, 3, 3, 10, 0, 6, 5]
+    assert len(old) == len(new) == n
+    for a in (old, new):                                            # the factored tuple only on matrices
+        for i, b in enumerate(wl.blocks):
+            if a[i] == 3 and b.cols <= 1:
+                a[i] = 2
+    sess.configure(old)
+    th = [sess.block_param_host(i) for i in range(n)]
+    sts = [O.step_init(ocfgs[old[i]], b.numel, b.rows, b.cols) for i, b in enumerate(wl.blocks)]
+
+    def shared_step(t, assign):
+        k = sess.fill_grads(t)
+        for i in range(n):
+            th[i] = _round_state_to_storage(th[i], sts[i])
+            _push_state(sess, i, th[i], sts[i])
+        before = [x.copy() for x in th]
+        sess.step(k, t)
+        for i, b in enumerate(wl.blocks):
+            th[i] = O.step(th[i], sess.block_grad_host(k, i), sts[i], ocfgs[assign[i]], b.rows, b.cols)
+            got = sess.block_param_host(i)
+            tol = 1e-6 * np.max(np.abs(th[i])) + 1e-5 * np.abs(th[i] - before[i])
+            assert np.all(np.abs(got - th[i]) <= tol), (t, b.name, sts[i].kind, float(np.max(np.abs(got - th[i]) / tol)))
+
+    for t in (1, 2, 3):
+        shared_step(t, old)
+    for i in range(n):                                              # both sides migrate from the same stored state
+        th[i] = _round_state_to_storage(th[i], sts[i])
+        _push_state(sess, i, th[i], sts[i])
+    sess.reconfigure(new, steps_done=3, inherit=inherit)
+    codes = [0, 0]
+    for i, b in enumerate(wl.blocks):
+        sts[i] = O.reconfigure(sts[i], ocfgs[new[i]], b.rows, b.cols, inherit=inherit)
+        _check_block(sess, i, None, sts[i], codes)                  # the migrated states, before any further step
+    assert codes[0] <= 1e-4 * max(codes[1], 1), codes
+    mem, _ = sess.h.cost_model()
+    assert sess.h.query().state_bytes == sum(int(mem[i, c]) for i, c in enumerate(new))
+    for t in (4, 5, 6):
+        shared_step(t, new)
+    codes = [0, 0]
+    for i in range(n):
+        _check_block(sess, i, None, sts[i], codes)
+    assert codes[0] <= 1e-4 * max(codes[1], 1), codes
+    assert sess.h.nonfinite()[0] == 0
 
 
 def test_checkpoint_resume_continues_bit_exactly(B, H):

@@ -623,3 +623,53 @@ def test_int8_single_moment_rules_follow_their_fp32_forms():
         assert np.all(np.abs(after - before) <= 1)                # rescaling by the decayed absmax keeps the codes
     assert O.state_bytes(O.Config(1, 0, 1, 0, 8), 700, 700, 1) == 700 + 4 * 3
     assert O.state_bytes(O.Config(0, 1, 1, 0, 8), 700, 700, 1) == 700 + 4 * 3
+
+
+def test_reconfigure_inherits_compatible_moments_and_restarts_the_rest():
+    rng = np.random.default_rng(17)
+    rows, cols = 24, 32
+    n = rows * cols
+    a32 = O.Config(1, 1, 1, 0, 32)
+    st = O.step_init(a32, n, rows, cols)
+    th = rng.standard_normal(n) * 0.02
+    for _ in range(3):
+        th = O.step(th, O.round_bf16(rng.standard_normal(n) * 0.01), st, a32, rows, cols)
+    m, v = st.m.copy(), st.v.copy()
+    # same tuple: nothing changes but the storage rounding to fp32
+    same = O.reconfigure(st, a32, rows, cols)
+    np.testing.assert_array_equal(same.m, m.astype(np.float32).astype(np.float64))
+    assert (same.t, same.t_m0, same.t_v0) == (3, 0, 0)
+    # Adam fp32 -> 8-bit: the codes are the quantisation of the moments; -> bf16: their rounding
+    a8 = O.reconfigure(st, O.Config(1, 1, 1, 0, 8), rows, cols)
+    q, a = O.quantize8(m, True)
+    np.testing.assert_array_equal(a8.qm, q); np.testing.assert_array_equal(a8.am, a)
+    q, a = O.quantize8(v, False)
+    np.testing.assert_array_equal(a8.qv, q); np.testing.assert_array_equal(a8.av, a)
+    a16 = O.reconfigure(st, O.Config(1, 1, 1, 0, 16), rows, cols)
+    np.testing.assert_array_equal(a16.v, O.round_bf16(v))
+    # 8-bit -> fp32: the dequantised values, within half a code of the originals
+    back = O.reconfigure(a8, a32, rows, cols)
+    assert np.max(np.abs(back.m - m)) <= np.max(np.abs(m)) / 254 * 1.0001 and (back.t_m0, back.t_v0) == (0, 0)
+    # Adam -> RMS keeps v and drops m; Adam -> SGD-momentum keeps nothing (another family) and restarts the buffer
+    r = O.reconfigure(st, O.Config(1, 0, 1, 0, 32), rows, cols)
+    np.testing.assert_array_equal(r.v, v.astype(np.float32).astype(np.float64)); assert r.m is None and r.t_v0 == 0
+    s = O.reconfigure(st, O.Config(0, 1, 1, 0, 32), rows, cols)
+    assert not s.m.any() and s.t_m0 == 3
+    # RMS -> Adam: v continues with its age, m starts from zero with a fresh bias correction
+    back2 = O.reconfigure(r, a32, rows, cols)
+    assert not back2.m.any() and (back2.t_m0, back2.t_v0) == (3, 0)
+    g = O.round_bf16(rng.standard_normal(n) * 0.01)
+    th2 = O.step(th, g, back2, a32, rows, cols)                      # step 4: m has seen 1 gradient, v has seen 4
+    m1 = (1 - a32.beta1) * g
+    v4 = a32.beta2 * r.v + (1 - a32.beta2) * g * g
+    want = th * (1 - a32.lr * a32.weight_decay) - a32.lr * (m1 / (1 - a32.beta1)) / (np.sqrt(v4 / (1 - a32.beta2 ** 4)) + a32.eps)
+    np.testing.assert_allclose(th2, want, rtol=1e-12, atol=1e-15)
+    # element-wise -> factored: row and column means; factored -> element-wise: r_i c_j / mean(r)
+    f = O.reconfigure(st, O.Config(1, 0, 1, 1, 32), rows, cols)
+    V = v.reshape(rows, cols)
+    np.testing.assert_allclose(f.r, V.mean(axis=1), rtol=1e-7); np.testing.assert_allclose(f.c, V.mean(axis=0), rtol=1e-7)
+    full = O.reconfigure(f, O.Config(1, 0, 1, 0, 32), rows, cols)
+    np.testing.assert_allclose(full.v, (np.outer(f.r, f.c) / f.r.mean()).reshape(-1), rtol=1e-7)
+    # without inheritance everything restarts
+    z = O.reconfigure(st, O.Config(1, 1, 1, 0, 32), rows, cols, inherit=False)
+    assert not z.m.any() and not z.v.any() and (z.t_m0, z.t_v0) == (3, 3)
