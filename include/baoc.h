@@ -280,6 +280,31 @@ int baoc_configure(baoc_t* h, const int32_t* assign, void* state_dev, size_t byt
 int baoc_reconfigure(baoc_t* h, const int32_t* new_assign, void* new_state_dev, size_t bytes,
                      int64_t steps_done, int inherit, baoc_stream_t stream);
 
+/* baoc_configure with a warm start: the moments the sampling window has built
+ * (Eq. 3) become the optimizer's initial moments instead of zeros (Algorithm 1
+ * hands over from "Warmup and diagnostics" to "Training" without saying what
+ * the new optimizer starts from; the same appendix study shows that dropped
+ * states cost quality).  The rule, per block, with T_w observations in the
+ * window:
+ *   - a tuple with an Adam-type first moment whose beta1 equals the window's
+ *     beta_m (compared as fp32) starts from m_hat; an SGD momentum buffer with
+ *     that coefficient starts from m_hat / (1 - beta_m), which is the buffer
+ *     m <- beta*m + g would have built from the same gradients;
+ *   - a tuple with a second moment whose beta2 equals the window's beta_v
+ *     starts from v_hat (element-wise, or its row and column means when
+ *     factored);
+ *   - each value is stored in the tuple's precision; a moment that is started
+ *     this way has seen T_w gradients, so at step t its bias correction uses
+ *     the exponent t + T_w; any other moment starts from zero as in
+ *     baoc_configure.
+ * Needs a bound workspace with at least one observation and a dense window
+ * (BAOC_E_STATE otherwise: a sampled sub-grid does not cover the block).
+ * state_dev as for baoc_configure; it must not overlap the workspace.  The
+ * step counter restarts: the next baoc_step passes 1.  Queues the zero-fill,
+ * the table uploads and the conversion kernels; does not wait. */
+int baoc_configure_from_window(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes,
+                               baoc_stream_t stream);
+
 /* One training step of every block under its configuration.  grads / params:
  * host arrays of n_blocks device pointers (bf16 / fp32).  step_t: 1-based step
  * number (bias corrections).  Queues the fused update kernel (preceded by the

@@ -628,3 +628,30 @@ def reconfigure(st: StepState, c_new: Config, rows: int, cols: int, inherit: boo
         else:
             new.v = round_bf16(old_v) if bits == 16 else old_v.astype(np.float32).astype(F64)
     return new
+
+
+# ----------------------------------------------------------------------------
+# Hand-over from the sampling window with its moments (Algorithm 1 moves from
+# "Warmup and diagnostics" to "Training" without saying what the new optimizer
+# starts from).  Reading, per block, with T_w observations in the window:
+#   * an Adam-type first moment whose beta1 equals the window's beta_m (as
+#     fp32 numbers) starts from m_hat; an SGD momentum buffer with that
+#     coefficient starts from m_hat / (1 - beta_m): what m <- beta*m + g would
+#     have built from the same gradients;
+#   * a second moment whose beta2 equals the window's beta_v starts from v_hat;
+#   * such a moment has seen T_w gradients (its start step is -T_w); storage
+#     and every other moment as in a re-configuration.
+# ----------------------------------------------------------------------------
+
+def warm_start(win: StatsState, c: Config, rows: int, cols: int, o: Opts, qblock: int = 256) -> StepState:
+    """The initial state of one block under ``c`` when the window's moments are carried into training."""
+    kind = config_kind(c)
+    same_m = np.float32(c.beta1) == np.float32(o.beta_m)
+    same_v = np.float32(c.beta2) == np.float32(o.beta_v)
+    if _M_FAMILY.get(kind) == "sum":
+        held = StepState("S", m=win.m / (1.0 - o.beta_m) if same_m else None)
+    else:
+        held = StepState("A32", m=win.m.copy() if same_m else None, v=win.v.copy() if same_v else None)
+    held.t = 0
+    held.t_m0 = held.t_v0 = -win.t
+    return reconfigure(held, c, rows, cols, True, qblock)

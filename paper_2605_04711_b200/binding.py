@@ -80,7 +80,7 @@ EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error"
            "baoc_configure", "baoc_step", "baoc_step_from_host", "baoc_view", "baoc_nonfinite",
            "baoc_sample_stats_noalloc", "baoc_noalloc_last_error", "baoc_profile", "baoc_profile_last",
            "baoc_export", "baoc_import", "baoc_time_scratch_bytes", "baoc_measure_time_ratios",
-           "baoc_set_sampling", "baoc_reconfigure"]
+           "baoc_set_sampling", "baoc_reconfigure", "baoc_configure_from_window"]
 
 _vp = C.c_void_p
 _lib.baoc_default_opts.argtypes = [C.POINTER(Opts)]
@@ -106,6 +106,7 @@ _lib.baoc_step_from_host.argtypes = [_vp, _vp, _vp, _vp, C.c_int, C.c_int64, _vp
 _lib.baoc_view.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(_vp), C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
 _lib.baoc_nonfinite.argtypes = [_vp, _vp, C.POINTER(C.c_int32), _vp]
 _lib.baoc_reconfigure.argtypes = [_vp, _vp, _vp, C.c_size_t, C.c_int64, C.c_int, _vp]
+_lib.baoc_configure_from_window.argtypes = [_vp, _vp, _vp, C.c_size_t, _vp]
 _lib.baoc_set_sampling.argtypes = [_vp, C.POINTER(Sample)]
 _lib.baoc_time_scratch_bytes.argtypes = [_vp, C.POINTER(C.c_size_t)]
 _lib.baoc_measure_time_ratios.argtypes = [_vp, _vp, _vp, _vp, C.c_size_t, C.c_int, C.c_int, _vp, _vp, _vp]
@@ -325,6 +326,13 @@ class Baoc:
         a = np.ascontiguousarray(assign, np.int32)
         self._check(_lib.baoc_reconfigure(self._h, a.ctypes.data, state.data_ptr(), state.numel() * state.element_size(),
                                           int(steps_done), int(bool(inherit)), _stream()))
+        self._keep.append(state)
+
+    def configure_from_window(self, assign, state: torch.Tensor):
+        """``baoc_configure_from_window``: instantiate the optimizer with the window's moments as its initial moments."""
+        a = np.ascontiguousarray(assign, np.int32)
+        self._check(_lib.baoc_configure_from_window(self._h, a.ctypes.data, state.data_ptr(),
+                                                    state.numel() * state.element_size(), _stream()))
         self._keep.append(state)
 
     def step(self, grads, params, step_t: int):

@@ -509,6 +509,54 @@ int baoc_reconfigure(baoc_t* h, const int32_t* new_assign, void* new_state_dev, 
     return BAOC_OK;
 }
 
+// ---- hand-over from the sampling window with its moments ------------------------------
+int baoc_configure_from_window(baoc_t* h, const int32_t* assign, void* state_dev, size_t bytes, baoc_stream_t stream) {
+    if (!h) return BAOC_E_INVALID;
+    if (!assign || !state_dev) return fail(h, BAOC_E_INVALID, "baoc_configure_from_window: null argument");
+    if (!h->ws_bound || h->stats_steps < 1) return fail(h, BAOC_E_STATE, "baoc_configure_from_window: the window holds no observation");
+    if (h->sampled) return fail(h, BAOC_E_STATE, "baoc_configure_from_window: the window saw a sampled sub-grid, not every coordinate");
+    {
+        const char* a = h->ws; const char* b = static_cast<const char*>(state_dev);
+        if (b < a + h->ws_bytes && a < b + bytes) return fail(h, BAOC_E_INVALID, "baoc_configure_from_window: the state buffer overlaps the statistics workspace");
+    }
+    const int n = h->n_blocks;
+    const float bm = float(h->opts.beta_m), bv = float(h->opts.beta_v);
+    std::vector<char> keep_m(n, 0), keep_v(n, 0);
+    std::vector<int64_t> tm(n, 0), tv(n, 0);
+    for (int i = 0; i < n; ++i) {
+        if (assign[i] < 0 || assign[i] >= h->n_cfg) return fail(h, BAOC_E_INVALID, "baoc_configure_from_window: assignment names a configuration that does not exist");
+        const baoc_config_t& c = h->cfgs[assign[i]];
+        const Path p = path_of(c);
+        keep_m[i] = m_family(p) != 0 && c.beta1 == bm;
+        keep_v[i] = (p == kPathA32 || p == kPathA16 || p == kPathA8 || p == kPathR || p == kPathR16 || p == kPathR8 || p == kPathF) && c.beta2 == bv;
+        tm[i] = keep_m[i] ? -h->stats_steps : 0;
+        tv[i] = keep_v[i] ? -h->stats_steps : 0;
+    }
+    const std::vector<int64_t> old_tm = h->t_m0, old_tv = h->t_v0;
+    h->t_m0 = tm; h->t_v0 = tv;
+    int rc = configure_state(h, assign, state_dev, bytes, stream, false, true);
+    if (rc) { h->t_m0 = old_tm; h->t_v0 = old_tv; return rc; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < n; ++i) {
+        const StepBlock& nb = h->h_step_blocks[i];
+        const StatBlock& wb = h->h_stat_blocks[i];
+        MomentRef src{};
+        src.rows = nb.rows; src.cols = nb.cols; src.kind = kMomF32;
+        if (keep_m[i]) {
+            src.data = h->ws + h->sl.m + reinterpret_cast<size_t>(wb.m);        // the handle's table holds offsets
+            src.divisor = m_family(nb.path) == 2 ? 1.0 - h->opts.beta_m : 0.0;   // a momentum buffer sums what the window averaged
+            LAUNCH(launch_convert_moment(src, first_moment(nb), nb.numel, s), "convert_moment_kernel");
+            h->launches += 1;
+        }
+        if (keep_v[i]) {
+            src.data = h->ws + h->sl.v + reinterpret_cast<size_t>(wb.v); src.divisor = 0.0;
+            LAUNCH(launch_convert_moment(src, second_moment(nb), nb.numel, s), "convert_moment_kernel");
+            h->launches += 1;
+        }
+    }
+    return BAOC_OK;
+}
+
 // ---- one-step timing of every (block, configuration) pair ---------------------------
 namespace {
 size_t single_block_state_bytes(const Handle* h, int block, int cfg) {

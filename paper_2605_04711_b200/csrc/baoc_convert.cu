@@ -9,7 +9,10 @@ namespace baoc {
 // Decode element e of a stored moment.
 __device__ __forceinline__ double moment_at(const MomentRef& s, int64_t e, double inv_mean_r) {
     switch (s.kind) {
-        case kMomF32: return double(static_cast<const float*>(s.data)[e]);
+        case kMomF32: {
+            const double x = double(static_cast<const float*>(s.data)[e]);
+            return s.divisor != 0.0 ? x / s.divisor : x;
+        }
         case kMomBF16: return double(bf16_bits_to_float(static_cast<const uint16_t*>(s.data)[e]));
         case kMomI8: return (double(static_cast<const int8_t*>(s.data)[e]) * double(s.absmax[e / kQBlock])) / 127.0;
         case kMomU8: return (double(static_cast<const uint8_t*>(s.data)[e]) * double(s.absmax[e / kQBlock])) / 255.0;

@@ -122,6 +122,7 @@ struct MomentRef {
     int32_t kind;
     int32_t rows, cols;  // the block's shape
     int32_t pad;
+    double divisor;      // fp32 sources only: the value read is data[e] / divisor (0: no division)
 };
 
 // State of one radix select: the bits found so far and the rank still to find

@@ -127,6 +127,12 @@ class Session:
         self.state = torch.empty(self.h.state_bytes(self.assign), dtype=torch.uint8, device=self.device)
         self.h.configure(self.assign, self.state)
 
+    def configure_from_window(self, assign):
+        """Instantiate the optimizer with the window's moments as its initial moments."""
+        self.assign = np.asarray(assign, np.int32)
+        self.state = torch.empty(self.h.state_bytes(self.assign), dtype=torch.uint8, device=self.device)
+        self.h.configure_from_window(self.assign, self.state)
+
     def reconfigure(self, assign, steps_done: int, inherit: bool = True):
         """Move to a new assignment in a fresh state buffer (the old one stays alive until the stream has passed)."""
         self.assign = np.asarray(assign, np.int32)

@@ -595,6 +595,58 @@ def test_reconfigure_migrates_states_like_the_oracle(B, H, inherit):
     assert sess.h.nonfinite()[0] == 0
 
 
+def test_configure_from_window_starts_from_the_windows_moments(B, H):
+    """Hand-over with a warm start: after three observations both sides hold the same window moments (the oracle's,
+    rounded to fp32 and written to the device), the optimizer is instantiated from them under every tuple (one with a
+    first-moment coefficient that differs from the window's), and three steps follow from shared states."""
+    wl = _odd_workload(seed=83)
+    cfgs = B.extended_configs() + [B.make_config(1, 1, 1, 0, 32, beta1=0.8, weight_decay=0.01)]
+    sess = H.Session(wl, configs=cfgs, n_grad_sets=2)
+    sess.init_params()
+    n = len(wl.blocks)
+    ocfgs = [_ocfg(c) for c in cfgs]
+    assign = [0, 1, 6, 2, 9, 4, 10, 11, 3, 3, 1, 8, 5, 7, 3]
+    assert len(assign) == n
+    for i, b in enumerate(wl.blocks):
+        if assign[i] == 3 and b.cols <= 1:
+            assign[i] = 11
+    o = O.Opts()
+    wins = _oracle_window(sess, 3, o)
+    for i in range(n):
+        wins[i].m = wins[i].m.astype(np.float32).astype(np.float64)
+        wins[i].v = wins[i].v.astype(np.float32).astype(np.float64)
+        sess.h.view_tensor(i, 0, torch.float32).copy_(torch.from_numpy(wins[i].m.astype(np.float32)).to(sess.device))
+        sess.h.view_tensor(i, 1, torch.float32).copy_(torch.from_numpy(wins[i].v.astype(np.float32)).to(sess.device))
+    sess.configure_from_window(assign)
+    sts = [O.warm_start(wins[i], ocfgs[assign[i]], b.rows, b.cols, o) for i, b in enumerate(wl.blocks)]
+    assert sts[7].t_m0 == 0 and sts[7].t_v0 == -3 and sts[0].t_m0 == -3
+    codes = [0, 0]
+    for i in range(n):
+        _check_block(sess, i, None, sts[i], codes)
+    assert codes[0] <= 1e-4 * max(codes[1], 1), codes
+    th = [sess.block_param_host(i) for i in range(n)]
+    for t in (1, 2, 3):
+        k = sess.fill_grads(10 + t)
+        for i in range(n):
+            th[i] = _round_state_to_storage(th[i], sts[i])
+            _push_state(sess, i, th[i], sts[i])
+        before = [x.copy() for x in th]
+        sess.step(k, t)
+        for i, b in enumerate(wl.blocks):
+            th[i] = O.step(th[i], sess.block_grad_host(k, i), sts[i], ocfgs[assign[i]], b.rows, b.cols)
+            got = sess.block_param_host(i)
+            tol = 1e-6 * np.max(np.abs(th[i])) + 1e-5 * np.abs(th[i] - before[i])
+            assert np.all(np.abs(got - th[i]) <= tol), (t, b.name, sts[i].kind, float(np.max(np.abs(got - th[i]) / tol)))
+    codes = [0, 0]
+    for i in range(n):
+        _check_block(sess, i, None, sts[i], codes)
+    assert codes[0] <= 1e-4 * max(codes[1], 1), codes
+    # a sampled window cannot be carried over, nor an empty one
+    fresh = H.Session(wl, configs=cfgs, n_grad_sets=1)
+    with pytest.raises(B.BaocError):
+        fresh.configure_from_window(assign)
+
+
 def test_checkpoint_resume_continues_bit_exactly(B, H):
     """Export after a window and some steps, move every buffer to a new address, import into a fresh handle, and
     let both handles continue on the same gradients: parameters, states and running statistics stay identical."""

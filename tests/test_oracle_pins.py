@@ -673,3 +673,53 @@ def test_reconfigure_inherits_compatible_moments_and_restarts_the_rest():
     # without inheritance everything restarts
     z = O.reconfigure(st, O.Config(1, 1, 1, 0, 32), rows, cols, inherit=False)
     assert not z.m.any() and not z.v.any() and (z.t_m0, z.t_v0) == (3, 3)
+
+
+def test_warm_start_equals_training_that_held_the_parameters_still_during_the_window():
+    """Carrying the window's moments into training must give what the optimizer itself would hold had it run through
+    the window with a zero learning rate: same moments, same ages in the bias corrections."""
+    import dataclasses
+    rng = np.random.default_rng(23)
+    rows, cols, T_w = 12, 32, 4
+    n = rows * cols
+    o = O.Opts()
+    win = O.stats_init(n)
+    gs = [O.round_bf16(rng.standard_normal(n) * 0.01) for _ in range(T_w + 2)]
+    for g in gs[:T_w]:
+        O.stats_step(win, g, o)
+    th0 = rng.standard_normal(n) * 0.02
+    for c in (O.Config(1, 1, 1, 0, 32), O.Config(1, 0, 0, 0, 32), O.Config(0, 1, 1, 0, 32, lr=1e-2), O.Config(1, 0, 1, 1, 32)):
+        still = dataclasses.replace(c, lr=0.0, weight_decay=0.0)
+        ref = O.step_init(c, n, rows, cols)
+        th_ref = th0.copy()
+        for g in gs[:T_w]:
+            th_ref = O.step(th_ref, g, ref, still, rows, cols)
+        np.testing.assert_array_equal(th_ref, th0)
+        ws = O.warm_start(win, c, rows, cols, o)
+        assert ws.t == 0
+        if ws.m is not None:
+            np.testing.assert_allclose(ws.m, ref.m, rtol=1e-7, atol=1e-30)
+            assert ws.t_m0 == -T_w
+        if ws.v is not None:
+            np.testing.assert_allclose(ws.v, ref.v, rtol=1e-7, atol=1e-30)
+        if ws.r is not None:
+            # the factored statistics of the window's v_hat are the EMAs of the row and column means of g^2
+            np.testing.assert_allclose(ws.r, ref.r, rtol=1e-6); np.testing.assert_allclose(ws.c, ref.c, rtol=1e-6)
+        th_ws = th0.copy()
+        for g in gs[T_w:]:
+            th_ref = O.step(th_ref, g, ref, c, rows, cols)
+            th_ws = O.step(th_ws, g, ws, c, rows, cols)
+        np.testing.assert_allclose(th_ws, th_ref, rtol=2e-6, atol=1e-12)
+    # a coefficient that differs from the window's: that moment starts from zero with a fresh bias correction
+    c = O.Config(1, 1, 1, 0, 32, beta1=0.8)
+    ws = O.warm_start(win, c, rows, cols, o)
+    assert not ws.m.any() and (ws.t_m0, ws.t_v0) == (0, -T_w)
+    np.testing.assert_array_equal(ws.v, win.v.astype(np.float32).astype(np.float64))
+    # 8-bit and bf16 tuples store the window's moments in their own precision
+    a8 = O.warm_start(win, O.Config(1, 1, 1, 0, 8), rows, cols, o)
+    q, a = O.quantize8(win.m, True)
+    np.testing.assert_array_equal(a8.qm, q); np.testing.assert_array_equal(a8.am, a)
+    s16 = O.warm_start(win, O.Config(0, 1, 1, 0, 16), rows, cols, o)
+    np.testing.assert_array_equal(s16.m, O.round_bf16(win.m / (1.0 - o.beta_m)))
+    # the plain gradient step has nothing to carry
+    assert O.warm_start(win, O.Config(0, 0, 1, 0, 32), rows, cols, o).m is None
