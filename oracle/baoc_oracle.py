@@ -357,7 +357,13 @@ def state_bytes(c: Config, numel: int, rows: int, cols: int, qblock: int = 256) 
         total += per_tensor()
     if c.adaptive:
         if c.factored:
-            total += 4 * (rows + cols)
+            # row and column statistics in the tuple's precision (8-bit: each vector in its own quantisation blocks)
+            if c.bits == 32:
+                total += 4 * (rows + cols)
+            elif c.bits == 16:
+                total += 2 * (rows + cols)
+            else:
+                total += rows + cols + 4 * ((rows + qblock - 1) // qblock + (cols + qblock - 1) // qblock)
         else:
             total += per_tensor()
     return total
@@ -447,14 +453,19 @@ class StepState:
     av: Optional[np.ndarray] = None
     r: Optional[np.ndarray] = None
     c: Optional[np.ndarray] = None
+    qr: Optional[np.ndarray] = None     # F8: codes and absmax of the row / column statistics
+    qc: Optional[np.ndarray] = None
+    ar: Optional[np.ndarray] = None
+    ac: Optional[np.ndarray] = None
 
 
 def config_kind(c: Config) -> str:
     """Which update path a tuple selects.  A32 / A16 / A8: Adam with fp32 / bf16 / 8-bit moments; R / R16:
     momentum-free RMS scaling; F: factored second moment; S / S16: SGD with momentum; G: plain gradient step
-    (neither mechanism, hence no state, whatever bit-width the tuple names); R8 / S8: the 8-bit forms of R / S."""
+    (neither mechanism, hence no state, whatever bit-width the tuple names); R8 / S8: the 8-bit forms of R / S;
+    F16 / F8: factored with bf16 / 8-bit row and column statistics."""
     if c.factored:
-        return "F" if (c.adaptive and not c.momentum and c.bits == 32) else "unsupported"
+        return {32: "F", 16: "F16", 8: "F8"}[c.bits] if (c.adaptive and not c.momentum) else "unsupported"
     if c.adaptive and c.momentum:
         return {32: "A32", 16: "A16", 8: "A8"}[c.bits]
     if c.adaptive and not c.momentum:
@@ -484,13 +495,24 @@ def step_init(c: Config, numel: int, rows: int, cols: int, qblock: int = 256) ->
                          am=np.zeros(nq, np.float32), av=np.zeros(nq, np.float32))
     if kind == "R":
         return StepState(kind, v=np.zeros(numel, F64))
-    if kind == "F":
+    if kind in ("F", "F16", "F8"):
         if cols <= 1:
             raise ValueError("the factored configuration needs a matrix block")
+        if kind == "F8":
+            return StepState(kind, qr=np.zeros(rows, np.uint8), qc=np.zeros(cols, np.uint8),
+                             ar=np.zeros((rows + qblock - 1) // qblock, np.float32),
+                             ac=np.zeros((cols + qblock - 1) // qblock, np.float32))
         return StepState(kind, r=np.zeros(rows, F64), c=np.zeros(cols, F64))
     if kind == "S":
         return StepState(kind, m=np.zeros(numel, F64))
     raise ValueError("unsupported configuration tuple")
+
+
+def _factored_stored(st: StepState, qblock: int):
+    """Row and column statistics of a factored state as they are stored, in double."""
+    if st.kind == "F8":
+        return dequantize8(st.qr, st.ar, False, qblock), dequantize8(st.qc, st.ac, False, qblock)
+    return np.asarray(st.r, F64), np.asarray(st.c, F64)
 
 
 def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, cols: int,
@@ -548,15 +570,25 @@ def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, 
     if st.kind == "R":
         st.v = c.beta2 * st.v + (1.0 - c.beta2) * g * g
         return _adam_apply(theta, g, st.v, c, t, False)
-    if st.kind == "F":
+    if st.kind in ("F", "F16", "F8"):
+        # the row and column statistics are read as stored; the update uses the new ones before they are rounded for
+        # storage (the convention of every reduced-precision state here)
+        r_old, c_old = _factored_stored(st, qblock)
         G2 = (g * g).reshape(rows, cols)
-        st.r = c.beta2 * st.r + (1.0 - c.beta2) * G2.mean(axis=1)
-        st.c = c.beta2 * st.c + (1.0 - c.beta2) * G2.mean(axis=0)
-        rm = float(st.r.mean())
+        r = c.beta2 * r_old + (1.0 - c.beta2) * G2.mean(axis=1)
+        cc = c.beta2 * c_old + (1.0 - c.beta2) * G2.mean(axis=0)
+        rm = float(r.mean())
         if rm == 0.0:
             v = np.zeros(rows * cols, F64)
         else:
-            v = (np.outer(st.r, st.c) / rm).reshape(-1)
+            v = (np.outer(r, cc) / rm).reshape(-1)
+        if st.kind == "F":
+            st.r, st.c = r, cc
+        elif st.kind == "F16":
+            st.r, st.c = round_bf16(r), round_bf16(cc)
+        else:
+            st.qr, st.ar = quantize8(r, False, qblock)
+            st.qc, st.ac = quantize8(cc, False, qblock)
         return _adam_apply(theta, g, v, c, t, False)
     if st.kind == "S":
         st.m = c.beta1 * st.m + g
@@ -580,8 +612,10 @@ def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, 
 # ----------------------------------------------------------------------------
 
 _M_FAMILY = {"A32": "avg", "A16": "avg", "A8": "avg", "S": "sum", "S16": "sum", "S8": "sum"}
-_V_FAMILY = {"A32": "full", "A16": "full", "A8": "full", "R": "full", "R16": "full", "R8": "full", "F": "factored"}
-_BITS = {"A32": 32, "A16": 16, "A8": 8, "R": 32, "R16": 16, "R8": 8, "S": 32, "S16": 16, "S8": 8, "F": 32, "G": 32}
+_V_FAMILY = {"A32": "full", "A16": "full", "A8": "full", "R": "full", "R16": "full", "R8": "full",
+             "F": "factored", "F16": "factored", "F8": "factored"}
+_BITS = {"A32": 32, "A16": 16, "A8": 8, "R": 32, "R16": 16, "R8": 8, "S": 32, "S16": 16, "S8": 8,
+         "F": 32, "F16": 16, "F8": 8, "G": 32}
 
 
 def _moment_value(st: StepState, which: str, rows: int, cols: int, qblock: int) -> Optional[np.ndarray]:
@@ -592,9 +626,10 @@ def _moment_value(st: StepState, which: str, rows: int, cols: int, qblock: int) 
         return None if st.m is None else np.asarray(st.m, F64)
     if st.kind in ("A8", "R8"):
         return dequantize8(st.qv, st.av, False, qblock)
-    if st.kind == "F":
-        rm = float(np.mean(st.r))
-        return np.zeros(rows * cols, F64) if rm == 0.0 else (np.outer(st.r, st.c) / rm).reshape(-1)
+    if _V_FAMILY.get(st.kind) == "factored":
+        r, c = _factored_stored(st, qblock)
+        rm = float(np.mean(r))
+        return np.zeros(rows * cols, F64) if rm == 0.0 else (np.outer(r, c) / rm).reshape(-1)
     return None if st.v is None else np.asarray(st.v, F64)
 
 
@@ -616,13 +651,19 @@ def reconfigure(st: StepState, c_new: Config, rows: int, cols: int, inherit: boo
             new.m = round_bf16(old_m) if bits == 16 else old_m.astype(np.float32).astype(F64)
     if kind in _V_FAMILY and old_v is not None:
         new.t_v0 = st.t_v0
-        if kind == "F":
-            if st.kind == "F":
-                new.r, new.c = st.r.copy(), st.c.copy()
+        if _V_FAMILY[kind] == "factored":
+            if _V_FAMILY[st.kind] == "factored":
+                r, c = _factored_stored(st, qblock)                 # factored -> factored: the statistics themselves
             else:
                 V = old_v.reshape(rows, cols)
-                new.r = V.mean(axis=1).astype(np.float32).astype(F64)
-                new.c = V.mean(axis=0).astype(np.float32).astype(F64)
+                r, c = V.mean(axis=1), V.mean(axis=0)
+            if bits == 8:
+                new.qr, new.ar = quantize8(r, False, qblock)
+                new.qc, new.ac = quantize8(c, False, qblock)
+            elif bits == 16:
+                new.r, new.c = round_bf16(r), round_bf16(c)
+            else:
+                new.r, new.c = r.astype(np.float32).astype(F64), c.astype(np.float32).astype(F64)
         elif bits == 8:
             new.qv, new.av = quantize8(old_v, False, qblock)
         else:

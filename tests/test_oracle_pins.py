@@ -544,7 +544,8 @@ def test_config_kind_dispatch():
     assert [O.config_kind(O.Config(1, 1, 1, 0, b)) for b in (32, 16, 8)] == ["A32", "A16", "A8"]
     assert [O.config_kind(O.Config(1, 0, 1, 0, b)) for b in (32, 16, 8)] == ["R", "R16", "R8"]
     assert [O.config_kind(O.Config(0, 1, 1, 0, b)) for b in (32, 16, 8)] == ["S", "S16", "S8"]
-    assert O.config_kind(O.Config(1, 1, 1, 1, 32)) == "unsupported" and O.config_kind(O.Config(1, 0, 1, 1, 16)) == "unsupported"
+    assert [O.config_kind(O.Config(1, 0, 1, 1, b)) for b in (32, 16, 8)] == ["F", "F16", "F8"]
+    assert O.config_kind(O.Config(1, 1, 1, 1, 32)) == "unsupported" and O.config_kind(O.Config(0, 0, 1, 1, 16)) == "unsupported"
 
 
 def test_plain_gradient_step_matches_torch_sgd():
@@ -723,3 +724,58 @@ def test_warm_start_equals_training_that_held_the_parameters_still_during_the_wi
     np.testing.assert_array_equal(s16.m, O.round_bf16(win.m / (1.0 - o.beta_m)))
     # the plain gradient step has nothing to carry
     assert O.warm_start(win, O.Config(0, 0, 1, 0, 32), rows, cols, o).m is None
+
+
+def test_factored_states_in_reduced_precision():
+    """Factored second moment with bf16 / 8-bit row and column statistics: the first step equals the fp32 one (the
+    update uses the new statistics before they are rounded), what is stored is the rounding / the codes of them, the
+    next step starts from the stored values, and the trajectories stay within the storage error of the fp32 one."""
+    rng = np.random.default_rng(29)
+    rows, cols = 300, 70                                   # more than one quantisation block of rows, a ragged one
+    n = rows * cols
+    f32, f16, f8 = (O.Config(1, 0, 1, 1, b) for b in (32, 16, 8))
+    assert O.state_bytes(f32, n, rows, cols) == 4 * (rows + cols)
+    assert O.state_bytes(f16, n, rows, cols) == 2 * (rows + cols)
+    assert O.state_bytes(f8, n, rows, cols) == rows + cols + 4 * (2 + 1)
+    th0 = rng.standard_normal(n) * 0.02
+    g1 = O.round_bf16(rng.standard_normal(n) * 0.01 * (1 + np.arange(n) % 7))
+    sts = {k: O.step_init(c, n, rows, cols) for k, c in (("F", f32), ("F16", f16), ("F8", f8))}
+    out = {k: O.step(th0, g1, sts[k], c, rows, cols) for k, c in (("F", f32), ("F16", f16), ("F8", f8))}
+    np.testing.assert_array_equal(out["F16"], out["F"])
+    np.testing.assert_array_equal(out["F8"], out["F"])
+    np.testing.assert_array_equal(sts["F16"].r, O.round_bf16(sts["F"].r))
+    q, a = O.quantize8(sts["F"].c, False)
+    np.testing.assert_array_equal(sts["F8"].qc, q); np.testing.assert_array_equal(sts["F8"].ac, a)
+    assert sts["F8"].ar.shape == (2,) and sts["F8"].ac.shape == (1,)
+    # second step by hand from the stored bf16 values
+    g2 = O.round_bf16(rng.standard_normal(n) * 0.01)
+    r_old, c_old = sts["F16"].r.copy(), sts["F16"].c.copy()
+    th2 = O.step(out["F16"], g2, sts["F16"], f16, rows, cols)
+    G2 = (g2 * g2).reshape(rows, cols)
+    r = f16.beta2 * r_old + (1 - f16.beta2) * G2.mean(axis=1)
+    c = f16.beta2 * c_old + (1 - f16.beta2) * G2.mean(axis=0)
+    v = (np.outer(r, c) / r.mean()).reshape(-1)
+    want = out["F16"] * (1 - f16.lr * f16.weight_decay) - f16.lr * g2 / (np.sqrt(v / (1 - f16.beta2 ** 2)) + f16.eps)
+    np.testing.assert_allclose(th2, want, rtol=1e-13, atol=1e-16)
+    np.testing.assert_array_equal(sts["F16"].r, O.round_bf16(r))
+    # a few more steps: the reduced-precision runs track the fp32 one within the storage error of sqrt(v)
+    th = {k: out[k] for k in out}
+    th["F16"] = th2
+    th["F"] = O.step(th["F"], g2, sts["F"], f32, rows, cols)
+    th["F8"] = O.step(th["F8"], g2, sts["F8"], f8, rows, cols)
+    for _ in range(4):
+        g = O.round_bf16(rng.standard_normal(n) * 0.01)
+        for k, c_ in (("F", f32), ("F16", f16), ("F8", f8)):
+            th[k] = O.step(th[k], g, sts[k], c_, rows, cols)
+    moved = np.max(np.abs(th["F"] - th0))
+    assert np.max(np.abs(th["F16"] - th["F"])) <= 0.01 * moved
+    assert np.max(np.abs(th["F8"] - th["F"])) <= 0.05 * moved
+    assert np.max(np.abs(th["F8"] - th["F"])) > 0
+    # migration between the precisions: decode, then store in the new form
+    back = O.reconfigure(sts["F8"], f32, rows, cols)
+    np.testing.assert_array_equal(back.r, O.dequantize8(sts["F8"].qr, sts["F8"].ar, False).astype(np.float32).astype(np.float64))
+    down = O.reconfigure(sts["F"], f8, rows, cols)
+    q, a = O.quantize8(sts["F"].r, False)
+    np.testing.assert_array_equal(down.qr, q); np.testing.assert_array_equal(down.ar, a)
+    full = O.reconfigure(sts["F16"], O.Config(1, 0, 1, 0, 32), rows, cols)
+    np.testing.assert_allclose(full.v, (np.outer(sts["F16"].r, sts["F16"].c) / sts["F16"].r.mean()).reshape(-1), rtol=1e-7)
