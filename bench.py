@@ -28,7 +28,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 CONFIG_NAMES = ["adamw32", "adamw8", "rms", "factored", "sgdm"]
-EXTENDED_NAMES = CONFIG_NAMES + ["sgd", "adamw16", "rms16", "sgdm16", "rms8", "sgdm8"]
+EXTENDED_NAMES = CONFIG_NAMES + ["sgd", "adamw16", "rms16", "sgdm16", "rms8", "sgdm8", "factored16", "factored8"]
 METRIC = "hot-path throughput: statistics pass + mixed-config optimizer step"
 UNIT = "params/s"
 
@@ -166,18 +166,23 @@ def _sample_blocks(wl, target_params):
     return picked, total
 
 
-def time_oracle(wl, assign, steps, warmup, target_params):
-    """Time the oracle's statistics step + optimizer step on a sample of blocks.  Returns (params/s, info)."""
+def time_oracle(wl, assign, steps, warmup, target_params, configs=None):
+    """Time the oracle's statistics step + optimizer step on a sample of blocks.  Returns (params/s, info).
+    configs: the candidate tuples ``assign`` indexes (the binding's structs); default: the oracle's five."""
     import numpy as np
     from threadpoolctl import threadpool_limits
     from oracle import baoc_oracle as O
     from paper_2605_04711_b200 import workloads as W
 
-    cfgs = O.default_configs()
-    # same hyper-parameter values as the library's fp32 fields
-    for c in cfgs:
-        for k in ("lr", "beta1", "beta2", "eps", "weight_decay"):
-            setattr(c, k, float(np.float32(getattr(c, k))))
+    if configs is None:
+        cfgs = O.default_configs()
+        # same hyper-parameter values as the library's fp32 fields
+        for c in cfgs:
+            for k in ("lr", "beta1", "beta2", "eps", "weight_decay"):
+                setattr(c, k, float(np.float32(getattr(c, k))))
+    else:
+        cfgs = [O.Config(c.adaptive, c.momentum, c.decoupled_wd, c.factored, c.bits, lr=float(c.lr), beta1=float(c.beta1),
+                         beta2=float(c.beta2), eps=float(c.eps), weight_decay=float(c.weight_decay)) for c in configs]
     picked, total = _sample_blocks(wl, target_params)
     opts = O.Opts()
     with threadpool_limits(limits=1):
@@ -188,7 +193,7 @@ def time_oracle(wl, assign, steps, warmup, target_params):
         for j, i in enumerate(picked):
             b = wl.blocks[i]
             c = int(assign[i]) if assign is not None else (j % 5)
-            if O.config_kind(cfgs[c]) == "F" and b.cols <= 1:
+            if cfgs[c].factored and b.cols <= 1:
                 c = 2
             ostates.append((c, O.step_init(cfgs[c], b.numel, b.rows, b.cols)))
         times = []
@@ -286,9 +291,11 @@ def run_ours(args):
     assign, objective, rc = sess.allocate(risk)
     alloc_ms = (time.perf_counter() - t0) * 1e3
     if args.assign != "auto":
-        # one configuration for every block (vectors cannot be factored: they take the momentum-free one)
+        # one configuration for every block (vectors cannot be factored: they take the momentum-free one of the same width)
         c = names.index(args.assign)
-        assign = np.asarray([c if not (c == 3 and b.cols <= 1) else 2 for b in wl.blocks], np.int32)
+        vec = {"factored": "rms", "factored16": "rms16", "factored8": "rms8"}
+        assign = np.asarray([names.index(vec[args.assign]) if (args.assign in vec and b.cols <= 1) else c for b in wl.blocks],
+                            np.int32)
     sess.configure(assign)
     info = sess.h.query()
     stats_bytes, step_bytes = info.stats_bytes_per_call, info.step_bytes_per_call
@@ -414,7 +421,7 @@ def run_ours(args):
         "once_per_window": {"finalize_and_risk_ms": finalize_ms, "allocate_ms": alloc_ms, "objective": objective},
     }
     if world == 1 and not args.no_cpu_baseline:
-        _, cb = time_oracle(wl, assign, 2, 1, args.cpu_sample_params)
+        _, cb = time_oracle(wl, assign, 2, 1, args.cpu_sample_params, sess.configs)
         line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
     print(json.dumps(line), flush=True)
     if dist is not None:

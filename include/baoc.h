@@ -66,14 +66,15 @@ typedef struct {
  * instantiate (Sec. 4.1 lists the mechanisms, each at 8/16/32-bit states):
  *   (1,1,*,0,32|16|8)  Adam / AdamW with fp32, bf16 or block-wise absmax 8-bit moments;
  *   (1,0,*,0,32|16|8)  momentum-free RMS scaling with an fp32, bf16 or 8-bit second moment;
- *   (1,0,*,1,32)       factored second moment (matrix blocks only);
+ *   (1,0,*,1,32|16|8)  factored second moment (matrix blocks only), its row and column statistics kept
+ *                      in fp32, in bf16 or as block-wise absmax 8-bit codes;
  *   (0,1,*,0,32|16|8)  SGD with momentum (beta1 is the momentum coefficient), fp32, bf16 or 8-bit buffer;
  *   (0,0,*,0,any)      plain gradient step (SGD / SGDW): no state, so the bit-width only enters Agg(c).
  * y_d selects decoupled (1) or coupled (0) weight decay in all of them.  With
  * bf16 or 8-bit states the parameter update uses the new moments before they are
- * rounded for storage.  Other tuples (factored at 8 or 16 bits, factored with
- * momentum or without adaptive scaling) may appear in the candidate set for risk
- * and cost queries but cannot be assigned. */
+ * rounded for storage.  Other tuples (factored with momentum or without
+ * adaptive scaling) may appear in the candidate set for risk and cost queries
+ * but cannot be assigned. */
 typedef struct {
     uint8_t adaptive, momentum, decoupled_wd, factored, bits;
     uint8_t reserved[3];
@@ -327,7 +328,8 @@ int baoc_step_from_host(baoc_t* h, const void* const* host_grads, void* const* d
  * assignment: Adam m, v (fp32 or bf16); 8-bit Adam codes of m (int8), codes of v
  * (uint8), absmax of m (fp32), absmax of v (fp32); RMS v; SGD m (fp32 or bf16);
  * 8-bit RMS / SGD-momentum: codes, then their absmax; factored r (rows), c
- * (cols); nothing for the plain gradient step.  Writes the device pointer, the element count and the element size
+ * (cols) as fp32 or bf16, or as uint8 codes followed by the absmax of r and
+ * of c (one fp32 per 256 codes); nothing for the plain gradient step.  Writes the device pointer, the element count and the element size
  * in bytes; BAOC_E_INVALID if the block has no such tensor, BAOC_E_STATE if the
  * buffer is not bound yet.  Host only. */
 int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* count, int32_t* elem_bytes);

@@ -154,13 +154,16 @@ def default_configs() -> List[Config]:
 
 def extended_configs() -> List[Config]:
     """The five default tuples plus the plain gradient step, the bf16-state variants of Adam(W), RMS scaling and
-    SGD with momentum, and the 8-bit variants of RMS scaling and SGD with momentum."""
+    SGD with momentum, the 8-bit variants of RMS scaling and SGD with momentum, and the factored second moment with
+    bf16 and 8-bit row / column statistics (indices 11 and 12)."""
     return default_configs() + [make_config(0, 0, 1, 0, 32, lr=1e-2, weight_decay=0.01),
                                 make_config(1, 1, 1, 0, 16, weight_decay=0.01),
                                 make_config(1, 0, 1, 0, 16, weight_decay=0.01),
                                 make_config(0, 1, 1, 0, 16, lr=1e-2, weight_decay=0.01),
                                 make_config(1, 0, 1, 0, 8, weight_decay=0.01),
-                                make_config(0, 1, 1, 0, 8, lr=1e-2, weight_decay=0.01)]
+                                make_config(0, 1, 1, 0, 8, lr=1e-2, weight_decay=0.01),
+                                make_config(1, 0, 1, 1, 16, weight_decay=0.01),
+                                make_config(1, 0, 1, 1, 8, weight_decay=0.01)]
 
 
 def pointer_table(tensors: Sequence[torch.Tensor]):

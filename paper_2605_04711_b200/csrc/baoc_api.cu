@@ -394,7 +394,12 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
     for (int i = 0; i < n; ++i) {
         StepBlock& b = sb[i];
         auto fix = [&](void* p) { return static_cast<void*>(st + L.states + reinterpret_cast<size_t>(p)); };
-        if (b.path == kPathA32 || b.path == kPathA8 || b.path == kPathF || b.path == kPathA16) { b.s0 = fix(b.s0); b.s1 = fix(b.s1); }
+        auto fix_scratch = [&](void* p) { return static_cast<void*>(st + L.redpart + reinterpret_cast<size_t>(p)); };
+        if (b.path == kPathF && b.fbits != 32) {
+            b.s0 = fix_scratch(b.s0); b.s1 = fix_scratch(b.s1);
+            b.f0 = fix(b.f0); b.f1 = fix(b.f1);
+            if (b.fbits == 8) { b.fa0 = static_cast<float*>(fix(b.fa0)); b.fa1 = static_cast<float*>(fix(b.fa1)); }
+        } else if (b.path == kPathA32 || b.path == kPathA8 || b.path == kPathF || b.path == kPathA16) { b.s0 = fix(b.s0); b.s1 = fix(b.s1); }
         else if (b.path == kPathR8) { b.s1 = fix(b.s1); b.a1 = static_cast<float*>(fix(b.a1)); }
         else if (b.path == kPathS8) { b.s0 = fix(b.s0); b.a0 = static_cast<float*>(fix(b.a0)); }
         else if (b.path != kPathG) b.s0 = fix(b.s0);
@@ -460,7 +465,12 @@ MomentRef second_moment(const StepBlock& b) {
         case kPathA8: case kPathR8: r.data = b.s1; r.absmax = b.a1; r.kind = kMomU8; break;
         case kPathR: r.data = b.s0; r.kind = kMomF32; break;
         case kPathR16: r.data = b.s0; r.kind = kMomBF16; break;
-        case kPathF: r.r = static_cast<const float*>(b.s0); r.c = static_cast<const float*>(b.s1); r.kind = kMomFactored; break;
+        case kPathF:
+            r.kind = kMomFactored; r.fbits = b.fbits;
+            r.wr = static_cast<float*>(b.s0); r.wc = static_cast<float*>(b.s1);
+            if (b.fbits == 32) { r.r = b.s0; r.c = b.s1; }
+            else { r.r = b.f0; r.c = b.f1; r.ar = b.fa0; r.ac = b.fa1; }
+            break;
         default: r.kind = kMomNone; break;
     }
     return r;
@@ -865,7 +875,15 @@ int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* co
             case kPathR16: case kPathS16: if (k == 0) { p = s.s0; n = b.numel; eb = 2; } break;
             case kPathR8: if (k == 0) { p = s.s1; n = b.numel; eb = 1; } else if (k == 1) { p = s.a1; n = nq; } break;
             case kPathS8: if (k == 0) { p = s.s0; n = b.numel; eb = 1; } else if (k == 1) { p = s.a0; n = nq; } break;
-            case kPathF: if (k == 0) { p = s.s0; n = b.rows; } else if (k == 1) { p = s.s1; n = b.cols; } break;
+            case kPathF:
+                if (s.fbits == 32) { if (k == 0) { p = s.s0; n = b.rows; } else if (k == 1) { p = s.s1; n = b.cols; } }
+                else {
+                    const int32_t e = s.fbits == 16 ? 2 : 1;
+                    if (k == 0) { p = s.f0; n = b.rows; eb = e; } else if (k == 1) { p = s.f1; n = b.cols; eb = e; }
+                    else if (s.fbits == 8 && k == 2) { p = s.fa0; n = ceil_div(b.rows, kQBlock); }
+                    else if (s.fbits == 8 && k == 3) { p = s.fa1; n = ceil_div(b.cols, kQBlock); }
+                }
+                break;
             default: break;
         }
         if (!p) return fail(h, BAOC_E_INVALID, "baoc_view: the block has no such state tensor");

@@ -6,6 +6,16 @@
 
 namespace baoc {
 
+// Entry i of a factored state's row (kRow) or column statistics, decoded from its stored form.
+template <bool kRow>
+__device__ __forceinline__ double factor_at(const MomentRef& s, int64_t i) {
+    const void* p = kRow ? s.r : s.c;
+    if (s.fbits == 32) return double(static_cast<const float*>(p)[i]);
+    if (s.fbits == 16) return double(bf16_bits_to_float(static_cast<const uint16_t*>(p)[i]));
+    const float* a = kRow ? s.ar : s.ac;
+    return (double(static_cast<const uint8_t*>(p)[i]) * double(a[i / kQBlock])) / 255.0;
+}
+
 // Decode element e of a stored moment.
 __device__ __forceinline__ double moment_at(const MomentRef& s, int64_t e, double inv_mean_r) {
     switch (s.kind) {
@@ -19,7 +29,7 @@ __device__ __forceinline__ double moment_at(const MomentRef& s, int64_t e, doubl
         case kMomFactored: {
             const int64_t row = e / s.cols;
             const int col = int(e - row * s.cols);
-            return double(s.r[row]) * double(s.c[col]) * inv_mean_r;
+            return factor_at<true>(s, row) * factor_at<false>(s, col) * inv_mean_r;
         }
         default: return 0.0;
     }
@@ -29,17 +39,10 @@ __device__ __forceinline__ double moment_at(const MomentRef& s, int64_t e, doubl
 __device__ __forceinline__ double inv_mean_of_rows(const MomentRef& s) {
     __shared__ double total[1];
     double local[1] = {0.0};
-    for (int i = threadIdx.x; i < s.rows; i += kThreads) local[0] += double(s.r[i]);
+    for (int i = threadIdx.x; i < s.rows; i += kThreads) local[0] += factor_at<true>(s, i);
     cta_reduce_store<1>(local, total);
     const double mean = total[0] / double(s.rows);
     return mean != 0.0 ? 1.0 / mean : 0.0;
-}
-
-__device__ __forceinline__ uint16_t bf16_from_double(double x) {
-    const float f = __double2float_rn(x);
-    const uint32_t u = __float_as_uint(f);
-    if ((u & 0x7f800000u) == 0x7f800000u) return uint16_t(u >> 16);
-    return uint16_t((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
 }
 
 // Element-wise source -> element-wise destination.  A warp owns one 256-element quantisation block per pass.
@@ -96,10 +99,11 @@ factor_cols_kernel(const MomentRef src, float* __restrict__ c) {
     c[col] = __double2float_rn(s / double(src.rows));
 }
 
-// Factored -> factored (same shape): plain copies.
-__global__ void copy_floats_kernel(const float* __restrict__ a, float* __restrict__ b, int64_t n) {
+// Factored -> factored (same shape): the statistics themselves, decoded into the destination's fp32 arrays.
+__global__ void factor_copy_kernel(const MomentRef src, float* __restrict__ r, float* __restrict__ c) {
     const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (i < n) b[i] = a[i];
+    if (i < src.rows) r[i] = __double2float_rn(factor_at<true>(src, i));
+    if (i < src.cols) c[i] = __double2float_rn(factor_at<false>(src, i));
 }
 
 #define BAOC_LAUNCH_CHECK()                                   \
@@ -108,25 +112,37 @@ __global__ void copy_floats_kernel(const float* __restrict__ a, float* __restric
         if (e_ != cudaSuccess) return int(e_);                \
     } while (0)
 
-int launch_convert_moment(const MomentRef& src, const MomentRef& dst, int64_t numel, cudaStream_t s) {
-    if (dst.kind == kMomFactored) {
-        if (src.kind == kMomFactored) {
-            copy_floats_kernel<<<unsigned((src.rows + 255) / 256), 256, 0, s>>>(src.r, const_cast<float*>(dst.r), src.rows);
-            BAOC_LAUNCH_CHECK();
-            copy_floats_kernel<<<unsigned((src.cols + 255) / 256), 256, 0, s>>>(src.c, const_cast<float*>(dst.c), src.cols);
-            BAOC_LAUNCH_CHECK();
-            return 0;
-        }
-        factor_rows_kernel<<<unsigned(src.rows), kThreads, 0, s>>>(src, const_cast<float*>(dst.r));
-        BAOC_LAUNCH_CHECK();
-        factor_cols_kernel<<<unsigned((src.cols + kThreads - 1) / kThreads), kThreads, 0, s>>>(src, const_cast<float*>(dst.c));
-        BAOC_LAUNCH_CHECK();
-        return 0;
-    }
+static int launch_vector_convert(const MomentRef& src, const MomentRef& dst, int64_t numel, cudaStream_t s) {
     const int64_t per_cta = int64_t(kThreads / 32) * kQBlock;
     convert_moment_kernel<<<unsigned((numel + per_cta - 1) / per_cta), kThreads, 0, s>>>(src, dst, numel);
     BAOC_LAUNCH_CHECK();
     return 0;
+}
+
+int launch_convert_moment(const MomentRef& src, const MomentRef& dst, int64_t numel, cudaStream_t s) {
+    if (dst.kind == kMomFactored) {
+        // first the fp32 arrays of the destination (its state when it keeps fp32, else its working copies) ...
+        if (src.kind == kMomFactored) {
+            const int64_t n = src.rows > src.cols ? src.rows : src.cols;
+            factor_copy_kernel<<<unsigned((n + 255) / 256), 256, 0, s>>>(src, dst.wr, dst.wc);
+            BAOC_LAUNCH_CHECK();
+        } else {
+            factor_rows_kernel<<<unsigned(src.rows), kThreads, 0, s>>>(src, dst.wr);
+            BAOC_LAUNCH_CHECK();
+            factor_cols_kernel<<<unsigned((src.cols + kThreads - 1) / kThreads), kThreads, 0, s>>>(src, dst.wc);
+            BAOC_LAUNCH_CHECK();
+        }
+        if (dst.fbits == 32) return 0;
+        // ... then their bf16 rounding or 8-bit codes, as two plain vectors
+        MomentRef from{}, to{};
+        from.kind = kMomF32; to.kind = dst.fbits == 16 ? kMomBF16 : kMomU8;
+        from.data = dst.wr; to.data = dst.r; to.absmax = dst.ar;
+        int rc = launch_vector_convert(from, to, dst.rows, s);
+        if (rc) return rc;
+        from.data = dst.wc; to.data = dst.c; to.absmax = dst.ac;
+        return launch_vector_convert(from, to, dst.cols, s);
+    }
+    return launch_vector_convert(src, dst, numel, s);
 }
 
 }  // namespace baoc

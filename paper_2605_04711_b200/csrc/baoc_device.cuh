@@ -64,6 +64,14 @@ __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w 
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float(uint32_t(b) << 16); }
 
+// double -> fp32 -> bf16, round to nearest even at both roundings (non-finite values keep their upper half).
+__device__ __forceinline__ uint16_t bf16_from_double(double x) {
+    const float f = __double2float_rn(x);
+    const uint32_t u = __float_as_uint(f);
+    if ((u & 0x7f800000u) == 0x7f800000u) return uint16_t(u >> 16);
+    return uint16_t((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
+}
+
 // Unpack 8 bf16 values held in a uint4 into floats.
 __device__ __forceinline__ void unpack8(const uint4& w, float (&x)[8]) {
     x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);

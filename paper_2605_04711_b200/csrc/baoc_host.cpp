@@ -27,7 +27,16 @@ int64_t state_mem_bytes(const baoc_config_t& c, const baoc_block_t& b) {
     };
     int64_t total = 0;
     if (c.momentum) total += per_tensor();
-    if (c.adaptive) total += c.factored ? 4 * (int64_t(b.rows) + int64_t(b.cols)) : per_tensor();
+    if (c.adaptive) {
+        if (!c.factored) total += per_tensor();
+        else {
+            // row and column statistics in the tuple's precision; as 8-bit codes each vector has its own quantisation blocks
+            const int64_t rc = int64_t(b.rows) + int64_t(b.cols);
+            if (c.bits == 32) total += 4 * rc;
+            else if (c.bits == 16) total += 2 * rc;
+            else total += rc + 4 * (ceil_div(b.rows, kQBlock) + ceil_div(b.cols, kQBlock));
+        }
+    }
     return total;
 }
 
@@ -165,7 +174,19 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
             case kPathS8: s.s0 = place(dpad); s.a0 = static_cast<float*>(place(4 * nq)); break;
             case kPathG: break;
             case kPathF: {
-                s.s0 = place(4 * size_t(b.rows)); s.s1 = place(4 * size_t(b.cols));
+                s.fbits = h->cfgs[c].bits;
+                if (s.fbits == 32) { s.s0 = place(4 * size_t(b.rows)); s.s1 = place(4 * size_t(b.cols)); }
+                else {
+                    // the fp32 working copies live in the scratch region (offsets from its base), the stored form in the states
+                    s.s0 = reinterpret_cast<void*>(take(&redpart, 4 * size_t(b.rows)));
+                    s.s1 = reinterpret_cast<void*>(take(&redpart, 4 * size_t(b.cols)));
+                    const size_t eb = s.fbits == 16 ? 2 : 1;
+                    s.f0 = place(eb * size_t(b.rows)); s.f1 = place(eb * size_t(b.cols));
+                    if (s.fbits == 8) {
+                        s.fa0 = static_cast<float*>(place(4 * size_t(ceil_div(b.rows, kQBlock))));
+                        s.fa1 = static_cast<float*>(place(4 * size_t(ceil_div(b.cols, kQBlock))));
+                    }
+                }
                 s.a0 = static_cast<float*>(place(16));
                 s.red.red0 = int32_t(rt.size());
                 for (int ch = 0; ch < s.red.chunks; ++ch)

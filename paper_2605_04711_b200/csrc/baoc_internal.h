@@ -45,7 +45,7 @@ enum Path : int32_t {
 };
 
 inline Path path_of(const baoc_config_t& c) {
-    if (c.factored) return (c.adaptive && !c.momentum && c.bits == 32) ? kPathF : kPathNone;
+    if (c.factored) return (c.adaptive && !c.momentum) ? kPathF : kPathNone;   // row/column statistics in fp32, bf16 or 8-bit codes
     if (c.adaptive && c.momentum) return c.bits == 32 ? kPathA32 : (c.bits == 16 ? kPathA16 : kPathA8);
     if (c.adaptive && !c.momentum) return c.bits == 32 ? kPathR : (c.bits == 16 ? kPathR16 : kPathR8);
     if (!c.adaptive && c.momentum) return c.bits == 32 ? kPathS : (c.bits == 16 ? kPathS16 : kPathS8);
@@ -110,6 +110,14 @@ struct StepBlock {
                          // block's moments last started from zero (they set the bias corrections)
     int32_t path;
     RedGeom red;
+    // Factored path with bf16 or 8-bit statistics: s0 / s1 are then fp32 working copies in the scratch region (what
+    // the update kernel reads: the new, un-rounded statistics) and the state proper is stored here.
+    void* f0;            // stored row statistics: bf16 values or 8-bit codes (null when the state is fp32)
+    void* f1;            // stored column statistics
+    float* fa0;          // 8-bit: absmax of the row statistics per quantisation block
+    float* fa1;          // 8-bit: absmax of the column statistics
+    int32_t fbits;       // 32, 16 or 8 (factored blocks; 0 otherwise)
+    int32_t pad2;
 };
 
 // A stored moment, for the migration kernels of a re-configuration.
@@ -117,11 +125,15 @@ enum MomentKind : int32_t { kMomNone = 0, kMomF32 = 1, kMomBF16 = 2, kMomI8 = 3,
 struct MomentRef {
     void* data;          // fp32 / bf16 values or 8-bit codes
     float* absmax;       // one fp32 per 256 codes (8-bit kinds)
-    const float* r;      // factored: row statistics
-    const float* c;      // factored: column statistics
+    void* r;             // factored: row statistics as stored (fp32, bf16 or 8-bit codes, by fbits)
+    void* c;             // factored: column statistics as stored
+    float* ar;           // factored, 8-bit: absmax of r / of c per 256 codes
+    float* ac;
+    float* wr;           // factored destination: the fp32 arrays the update kernel reads (r, c themselves when fbits == 32)
+    float* wc;
     int32_t kind;
     int32_t rows, cols;  // the block's shape
-    int32_t pad;
+    int32_t fbits;       // factored: 32, 16 or 8
     double divisor;      // fp32 sources only: the value read is data[e] / divisor (0: no division)
 };
 

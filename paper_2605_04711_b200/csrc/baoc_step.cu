@@ -168,6 +168,63 @@ moment_reduce_combine_kernel(const StatBlock* __restrict__ blocks, const int32_t
 // Every CTA leaves the sum of its new r_i; the CTA that takes the last ticket of
 // the block adds the slab sums in index order and stores the mean of r (no CTA
 // waits for another).
+// Row (kRow) or column statistics kept as bf16 values or 8-bit codes: a warp owns one 256-element quantisation block at
+// a time.  The stored value is read, the new one is written un-rounded (fp32) to the working copy the update kernel
+// reads, and its rounding / its code is what is stored.  Returns the thread's share of the sum of the new values.
+template <bool kRow>
+__device__ __forceinline__ double combine_reduced(const StepBlock* b, double beta2, int slab) {
+    const int n = kRow ? b->rows : b->cols, other = kRow ? b->cols : b->rows;
+    const int parts = kRow ? b->red.strips : b->red.chunks;
+    const double* __restrict__ part = kRow ? b->red.rowpart : b->red.colpart;
+    float* __restrict__ work = static_cast<float*>(kRow ? b->s0 : b->s1);
+    void* stored = kRow ? b->f0 : b->f1;
+    float* __restrict__ amax_io = kRow ? b->fa0 : b->fa1;
+    const bool codes = b->fbits == 8;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nblk = (n + kQBlock - 1) / kQBlock;
+    const int bpc = (nblk + kCombineSlabs - 1) / kCombineSlabs;
+    double sum = 0.0;
+    for (int q = slab * bpc + warp; q < min(nblk, (slab + 1) * bpc); q += kThreads / 32) {
+        const double a_old = codes ? double(amax_io[q]) : 0.0;
+        double x[8];
+        float amax = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = q * kQBlock + lane * 8 + j;
+            x[j] = 0.0;
+            if (i < n) {
+                double s = 0.0;
+                for (int p = 0; p < parts; ++p) s += part[size_t(p) * n + i];
+                const double old = codes ? (double(static_cast<const uint8_t*>(stored)[i]) * a_old) / 255.0
+                                         : double(bf16_bits_to_float(static_cast<const uint16_t*>(stored)[i]));
+                x[j] = beta2 * old + (1.0 - beta2) * (s / double(other));
+                const float xf = __double2float_rn(x[j]);
+                work[i] = xf;
+                sum += double(xf);
+                amax = fmaxf(amax, xf);                      // x >= 0; rounding is monotone, so this is the rounded maximum
+            }
+        }
+        if (codes) {
+            __syncwarp();                                    // every lane has read the old absmax before lane 0 replaces it
+            amax = warp_max(amax);
+            const double scale = code_scale(amax, 255.0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = q * kQBlock + lane * 8 + j;
+                if (i < n) static_cast<uint8_t*>(stored)[i] = uint8_t(encode_unsigned(x[j], amax, scale));
+            }
+            if (lane == 0) amax_io[q] = amax;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = q * kQBlock + lane * 8 + j;
+                if (i < n) static_cast<uint16_t*>(stored)[i] = bf16_from_double(x[j]);
+            }
+        }
+    }
+    return sum;
+}
+
 __global__ void __launch_bounds__(kThreads)
 factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __restrict__ ids,
                         const __grid_constant__ StepParams P) {
@@ -175,23 +232,29 @@ factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __r
     const StepBlock* b = blocks + ids[blockIdx.x];
     const int rows = b->rows, cols = b->cols, slab = blockIdx.y;
     const double beta2 = P.c[b->cfg].beta2_d;
-    float* __restrict__ r = static_cast<float*>(b->s0);
-    float* __restrict__ c = static_cast<float*>(b->s1);
-    const int rpc = (rows + kCombineSlabs - 1) / kCombineSlabs, cpc = (cols + kCombineSlabs - 1) / kCombineSlabs;
     double local[1] = {0.0};
-    for (int i = slab * rpc + threadIdx.x; i < min(rows, (slab + 1) * rpc); i += kThreads) {
-        double s = 0.0;
-        for (int st = 0; st < b->red.strips; ++st) s += b->red.rowpart[size_t(st) * rows + i];
-        const float rn = float(beta2 * double(r[i]) + (1.0 - beta2) * (s / double(cols)));
-        r[i] = rn;
-        local[0] += double(rn);
-    }
-    cta_reduce_store<1>(local, total);
-    for (int j = slab * cpc + threadIdx.x; j < min(cols, (slab + 1) * cpc); j += kThreads) {
-        double s = 0.0;
+    if (b->fbits != 32) {
+        local[0] = combine_reduced<true>(b, beta2, slab);
+        cta_reduce_store<1>(local, total);
+        combine_reduced<false>(b, beta2, slab);
+    } else {
+        float* __restrict__ r = static_cast<float*>(b->s0);
+        float* __restrict__ c = static_cast<float*>(b->s1);
+        const int rpc = (rows + kCombineSlabs - 1) / kCombineSlabs, cpc = (cols + kCombineSlabs - 1) / kCombineSlabs;
+        for (int i = slab * rpc + threadIdx.x; i < min(rows, (slab + 1) * rpc); i += kThreads) {
+            double s = 0.0;
+            for (int st = 0; st < b->red.strips; ++st) s += b->red.rowpart[size_t(st) * rows + i];
+            const float rn = float(beta2 * double(r[i]) + (1.0 - beta2) * (s / double(cols)));
+            r[i] = rn;
+            local[0] += double(rn);
+        }
+        cta_reduce_store<1>(local, total);
+        for (int j = slab * cpc + threadIdx.x; j < min(cols, (slab + 1) * cpc); j += kThreads) {
+            double s = 0.0;
 #pragma unroll 4
-        for (int ch = 0; ch < b->red.chunks; ++ch) s += b->red.colpart[size_t(ch) * cols + j];
-        c[j] = float(beta2 * double(c[j]) + (1.0 - beta2) * (s / double(rows)));
+            for (int ch = 0; ch < b->red.chunks; ++ch) s += b->red.colpart[size_t(ch) * cols + j];
+            c[j] = float(beta2 * double(c[j]) + (1.0 - beta2) * (s / double(rows)));
+        }
     }
     if (threadIdx.x == 0) {
         volatile double* part = b->mean_part;

@@ -261,9 +261,16 @@ def _check_block(sess, i, th_ref, st_ref, code_stats):
         assert _rel_max(f32(10), st_ref.m) <= 1e-6
     elif kind == "F":
         assert _rel_max(f32(10), st_ref.r) <= 1e-6 and _rel_max(f32(11), st_ref.c) <= 1e-6
-    elif kind in ("A16", "R16", "S16"):
+    elif kind == "F8":
+        for w, (ref_q, ref_a) in enumerate(((st_ref.qr, st_ref.ar), (st_ref.qc, st_ref.ac))):
+            q = sess.h.view_tensor(i, 10 + w, torch.uint8).cpu().numpy().astype(np.int32)
+            d = np.abs(q - ref_q.astype(np.int32))
+            assert d.max() <= 1
+            code_stats[0] += int((d != 0).sum()); code_stats[1] += q.size
+            assert _rel_max(f32(12 + w), ref_a.astype(np.float64)) <= 1e-6
+    elif kind in ("A16", "R16", "S16", "F16"):
         # bf16 states: the stored bit patterns are compared (a rounding decision, taken exactly on both sides)
-        refs = {"A16": (st_ref.m, st_ref.v), "R16": (st_ref.v,), "S16": (st_ref.m,)}[kind]
+        refs = {"A16": (st_ref.m, st_ref.v), "R16": (st_ref.v,), "S16": (st_ref.m,), "F16": (st_ref.r, st_ref.c)}[kind]
         for w, ref in enumerate(refs):
             got = sess.h.view_tensor(i, 10 + w, torch.bfloat16).view(torch.int16).cpu().numpy().astype(np.int32)
             want = torch.from_numpy(ref).to(torch.bfloat16).view(torch.int16).numpy().astype(np.int32)
@@ -342,6 +349,11 @@ def _push_state(sess, i, th, st):
         put(10, torch.bfloat16, torch.from_numpy(st.v).to(torch.bfloat16))
     elif st.kind == "S16":
         put(10, torch.bfloat16, torch.from_numpy(st.m).to(torch.bfloat16))
+    elif st.kind == "F16":
+        put(10, torch.bfloat16, torch.from_numpy(st.r).to(torch.bfloat16)); put(11, torch.bfloat16, torch.from_numpy(st.c).to(torch.bfloat16))
+    elif st.kind == "F8":
+        put(10, torch.uint8, st.qr); put(11, torch.uint8, st.qc)
+        put(12, torch.float32, st.ar); put(13, torch.float32, st.ac)
     elif st.kind == "R8":
         put(10, torch.uint8, st.qv); put(11, torch.float32, st.av)
     elif st.kind == "S8":
@@ -431,6 +443,44 @@ def test_stateless_bf16_state_and_single_moment_int8_configurations_ten_steps(B,
     assert sess.h.query().state_bytes == int(mem.sum()) == per * wl.numel + absmax
 
 
+@pytest.mark.parametrize("tuple_", [(1, 0, 1, 1, 16), (1, 0, 0, 1, 16), (1, 0, 1, 1, 8), (1, 0, 0, 1, 8)])
+def test_factored_with_bf16_and_int8_statistics_ten_steps(B, H, tuple_):
+    """Factored second moment whose row and column statistics are stored as bf16 values or 8-bit codes, on the matrix
+    blocks (the vectors take RMS scaling at the same precision); decoupled and coupled decay.  Steps start from shared
+    states, so each step's reading of the stored statistics and its re-storing are what is compared."""
+    wl = _odd_workload(seed=91 + sum(tuple_))
+    cfgs = [B.make_config(*tuple_, weight_decay=0.05), B.make_config(1, 0, tuple_[2], 0, tuple_[4], weight_decay=0.05)]
+    sess = H.Session(wl, configs=cfgs, n_grad_sets=2)
+    sess.init_params()
+    assign = [0 if b.cols > 1 else 1 for b in wl.blocks]
+    codes = _run_steps_from_shared_state(sess, assign, [_ocfg(c) for c in cfgs])
+    assert codes[1] > 0 and codes[0] <= 1e-4 * codes[1], codes
+    assert sess.h.nonfinite()[0] == 0
+    mem, _ = sess.h.cost_model()
+    want = 0
+    for b in wl.blocks:
+        if b.cols > 1:
+            rc = b.rows + b.cols
+            want += 2 * rc if tuple_[4] == 16 else rc + 4 * ((b.rows + 255) // 256 + (b.cols + 255) // 256)
+        else:
+            want += 2 * b.numel if tuple_[4] == 16 else b.numel + 4 * ((b.numel + 255) // 256)
+    assert sess.h.query().state_bytes == sum(int(mem[i, a]) for i, a in enumerate(assign)) == want
+
+
+def test_factored_bf16_statistics_free_running_ten_steps(B, H):
+    """Ten free-running steps (no state sharing) of the factored tuple with bf16 statistics."""
+    wl = _odd_workload(seed=97)
+    cfgs = [B.make_config(1, 0, 1, 1, 16, weight_decay=0.05), B.make_config(1, 0, 1, 0, 16, weight_decay=0.05)]
+    sess = H.Session(wl, configs=cfgs, n_grad_sets=2)
+    sess.init_params()
+    assign = [0 if b.cols > 1 else 1 for b in wl.blocks]
+    th, sts = _run_steps(sess, assign, 10)
+    codes = [0, 0]
+    for i in range(len(wl.blocks)):
+        _check_block(sess, i, th[i], sts[i], codes)
+    assert codes[0] <= 1e-4 * codes[1], codes
+
+
 def test_nonfinite_gradient_is_flagged_not_fatal(B, H):
     wl = _odd_workload(seed=31)
     sess = H.Session(wl, n_grad_sets=1)
@@ -493,7 +543,7 @@ def test_measured_time_ratios_leave_parameters_and_state_alone(B, H):
     for i, b in enumerate(blocks):
         assert ratio[i, 0] == 1.0
         for c in range(n_cfg):
-            if c == 3 and b.cols <= 1:                               # factored on a vector: not measurable
+            if c in (3, 11, 12) and b.cols <= 1:                     # factored on a vector: not measurable
                 assert ms[i, c] == -1.0 and ratio[i, c] == model[i, c]
             else:
                 assert ms[i, c] > 0.0 and 0.05 < ratio[i, c] < 20.0
@@ -538,23 +588,28 @@ def test_step_from_host_equals_separate_calls_bit_for_bit(B, H):
         assert a["rho_bar"] == b2["rho_bar"] and a["last_cos"] == b2["last_cos"] and a["n_cos"] == b2["n_cos"] == 2
 
 
+@pytest.mark.parametrize("variant", [0, 1])
 @pytest.mark.parametrize("inherit", [True, False])
-def test_reconfigure_migrates_states_like_the_oracle(B, H, inherit):
+def test_reconfigure_migrates_states_like_the_oracle(B, H, inherit, variant):
     """Online re-configuration: three steps under one assignment, a move to another one (every pair of families and
     precisions occurs), three more steps.  The states are synchronised oracle -> device before the move and before each
     later step, so the migration itself and the per-moment bias corrections are what is compared."""
     wl = _odd_workload(seed=81)
-    cfgs = B.extended_configs()                                     # 0 A32, 1 A8, 2 R, 3 F, 4 S, 5 G, 6 A16, 7 R16, 8 S16, 9 R8, 10 S8
+    cfgs = B.extended_configs()              # 0 A32, 1 A8, 2 R, 3 F, 4 S, 5 G, 6 A16, 7 R16, 8 S16, 9 R8, 10 S8, 11 F16, 12 F8
     sess = H.Session(wl, configs=cfgs, n_grad_sets=2)
     sess.init_params()
     n = len(wl.blocks)
     ocfgs = [_ocfg(c) for c in cfgs]
-    old = [0, 1, 6, 2, 9, 4, 10, 0, 3, 3, 1, 8, 5, 7, 0]
-    new = [1, 0, 1, 0, 2, 8, 4, 4, 2, 3, 3, 10, 0, 6, 5]
+    if variant == 0:
+        old = [0, 1, 6, 2, 9, 4, 10, 0, 3, 3, 1, 8, 5, 7, 0]
+        new = [1, 0, 1, 0, 2, 8, 4, 4, 2, 3, 3, 10, 0, 6, 5]
+    else:                                    # the factored precisions: blocks 7..11 and 13 are matrices
+        old = [0, 1, 6, 2, 9, 4, 10, 0, 11, 12, 12, 11, 5, 7, 0]
+        new = [1, 0, 1, 0, 2, 8, 4, 12, 12, 0, 3, 2, 0, 11, 5]
     assert len(old) == len(new) == n
-    for a in (old, new):                                            # the factored tuple only on matrices
+    for a in (old, new):                                            # the factored tuples only on matrices
         for i, b in enumerate(wl.blocks):
-            if a[i] == 3 and b.cols <= 1:
+            if a[i] in (3, 11, 12) and b.cols <= 1:
                 a[i] = 2
     sess.configure(old)
     th = [sess.block_param_host(i) for i in range(n)]
@@ -605,11 +660,12 @@ def test_configure_from_window_starts_from_the_windows_moments(B, H):
     sess.init_params()
     n = len(wl.blocks)
     ocfgs = [_ocfg(c) for c in cfgs]
-    assign = [0, 1, 6, 2, 9, 4, 10, 11, 3, 3, 1, 8, 5, 7, 3]
+    odd = len(cfgs) - 1                                             # the tuple whose beta1 differs from the window's
+    assign = [0, 1, 6, 2, 9, 4, 10, odd, 3, 12, 1, 8, 5, 11, 3]
     assert len(assign) == n
     for i, b in enumerate(wl.blocks):
         if assign[i] == 3 and b.cols <= 1:
-            assign[i] = 11
+            assign[i] = odd
     o = O.Opts()
     wins = _oracle_window(sess, 3, o)
     for i in range(n):
