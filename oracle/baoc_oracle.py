@@ -696,3 +696,107 @@ def warm_start(win: StatsState, c: Config, rows: int, cols: int, o: Opts, qblock
     held.t = 0
     held.t_m0 = held.t_v0 = -win.t
     return reconfigure(held, c, rows, cols, True, qblock)
+
+
+# ----------------------------------------------------------------------------
+# O7. Block partitioning (Appendix on block partitioning, Algorithm 2).
+#
+# Input: candidate units in forward order, with parameter counts n_j and
+# normalised diagnostic vectors z_j; weights w_k; n_min = alpha * |Theta|; the
+# statistic-difference threshold tau (None: the upper quartile of all pairwise
+# Delta among the candidate units, as the paper's implementation sets it).
+# Delta(U_a, U_b) = max_k w_k |z_{a,k} - z_{b,k}|.
+#
+# The algorithm's verbs are loose; the reading taken here, step by step:
+#   * every gap between adjacent units is a candidate boundary;
+#   * a temporary block made of several units has the size-weighted mean of
+#     their z as its diagnostic vector;
+#   * minimum-size filtering: while some temporary block is smaller than n_min
+#     (and more than one block is left), the first such block is merged into
+#     the adjacent block with the smaller Delta to it (ties: the smaller
+#     neighbour, then the left one);
+#   * block formation: a boundary between adjacent temporary blocks survives
+#     iff their Delta exceeds tau (both satisfy the size constraint after the
+#     filtering); each decision is taken on the temporary blocks as the
+#     filtering left them, so the result does not depend on scan order;
+#   * post-processing, split: a block made of several temporary blocks is cut
+#     where the Delta between the weighted means of its two sides is largest,
+#     provided that Delta exceeds tau and both sides reach n_min; repeated on
+#     both halves;
+#   * post-processing, re-merge: the minimum-size filtering once more.
+# Returns (block index of every unit, tau used).
+# ----------------------------------------------------------------------------
+
+def partition_delta(za: np.ndarray, zb: np.ndarray, w: np.ndarray) -> float:
+    return float(np.max(w * np.abs(za - zb)))
+
+
+def _mean_z(sizes: Sequence[int], Z: np.ndarray, members: Sequence[int]) -> np.ndarray:
+    """Size-weighted mean of the members' vectors, accumulated in member order as offsets from the first member's
+    vector (so that units with identical statistics average to exactly that vector)."""
+    first = Z[members[0]]
+    acc = np.zeros(Z.shape[1], F64)
+    tot = 0.0
+    for j in members:
+        acc = acc + float(sizes[j]) * (Z[j] - first)
+        tot += float(sizes[j])
+    return first + acc / tot
+
+
+def _size_filter(blocks: List[List[int]], sizes: Sequence[int], Z: np.ndarray, w: np.ndarray, n_min: float) -> List[List[int]]:
+    blocks = [list(b) for b in blocks]
+    while len(blocks) > 1:
+        small = next((i for i, b in enumerate(blocks) if sum(sizes[j] for j in b) < n_min), None)
+        if small is None:
+            break
+        zs = _mean_z(sizes, Z, blocks[small])
+        cands = []
+        for nb in (small - 1, small + 1):
+            if 0 <= nb < len(blocks):
+                cands.append((partition_delta(zs, _mean_z(sizes, Z, blocks[nb]), w), sum(sizes[j] for j in blocks[nb]), nb))
+        cands.sort()                                   # smaller Delta, then smaller neighbour, then the left one
+        nb = cands[0][2]
+        lo, hi = min(small, nb), max(small, nb)
+        blocks[lo:hi + 1] = [blocks[lo] + blocks[hi]]
+    return blocks
+
+
+def partition_blocks(sizes: Sequence[int], Z: np.ndarray, w: Optional[Sequence[float]] = None, alpha: float = 0.0,
+                     tau: Optional[float] = None):
+    Z = np.asarray(Z, F64)
+    m, K = Z.shape
+    w = np.ones(K, F64) if w is None else np.asarray(w, F64)
+    n_min = alpha * float(sum(sizes))
+    if tau is None:
+        pair = [partition_delta(Z[a], Z[b], w) for a in range(m) for b in range(a + 1, m)]
+        tau = quantile_linear(np.asarray(pair, F64), 0.75) if pair else 0.0
+    # minimum-size filtering on the candidate units
+    temp = _size_filter([[j] for j in range(m)], sizes, Z, w, n_min)
+    # block formation
+    formed: List[List[List[int]]] = [[temp[0]]]
+    for a in range(len(temp) - 1):
+        if partition_delta(_mean_z(sizes, Z, temp[a]), _mean_z(sizes, Z, temp[a + 1]), w) > tau:
+            formed.append([temp[a + 1]])
+        else:
+            formed[-1].append(temp[a + 1])
+    # post-processing: split where the two sides are clearly separated
+    def split(parts: List[List[int]]) -> List[List[List[int]]]:
+        best, best_cut = -1.0, -1
+        for cut in range(1, len(parts)):
+            left = [j for p in parts[:cut] for j in p]
+            right = [j for p in parts[cut:] for j in p]
+            if sum(sizes[j] for j in left) < n_min or sum(sizes[j] for j in right) < n_min:
+                continue
+            d = partition_delta(_mean_z(sizes, Z, left), _mean_z(sizes, Z, right), w)
+            if d > best:
+                best, best_cut = d, cut
+        if best_cut < 0 or not best > tau:
+            return [parts]
+        return split(parts[:best_cut]) + split(parts[best_cut:])
+    final = [[j for p in blk for j in p] for f in formed for blk in split(f)]
+    # post-processing: re-merge what is still too small
+    final = _size_filter(final, sizes, Z, w, n_min)
+    ids = np.zeros(m, np.int32)
+    for b, members in enumerate(final):
+        ids[members] = b
+    return ids, float(tau)

@@ -779,3 +779,80 @@ def test_factored_states_in_reduced_precision():
     np.testing.assert_array_equal(down.qr, q); np.testing.assert_array_equal(down.ar, a)
     full = O.reconfigure(sts["F16"], O.Config(1, 0, 1, 0, 32), rows, cols)
     np.testing.assert_allclose(full.v, (np.outer(sts["F16"].r, sts["F16"].c) / sts["F16"].r.mean()).reshape(-1), rtol=1e-7)
+
+
+# ---------------------------------------------------------------- block partitioning (Algorithm 2)
+
+def test_partition_threshold_is_the_upper_quartile_of_pairwise_differences():
+    Z = np.array([[0.0], [1.0], [3.0]])
+    ids, tau = O.partition_blocks([10, 10, 10], Z)
+    assert tau == 2.5                                       # differences 1, 2, 3: position 0.75 * 2 = 1.5
+    Zr = RNG.random((9, 5))
+    w = np.array([1.0, 2.0, 0.5, 1.0, 3.0])
+    pair = [np.max(w * np.abs(Zr[a] - Zr[b])) for a in range(9) for b in range(a + 1, 9)]
+    assert abs(O.partition_blocks([5] * 9, Zr, w)[1] - np.quantile(pair, 0.75)) < 1e-15
+    assert O.partition_delta(np.array([0.0, 1.0]), np.array([0.5, 0.0]), np.array([4.0, 1.0])) == 2.0
+
+
+def test_partition_identical_units_form_one_block_and_clusters_split_at_their_edge():
+    ids, tau = O.partition_blocks([7] * 6, np.full((6, 3), 0.4))
+    assert tau == 0.0 and ids.tolist() == [0] * 6
+    Z = np.array([[0.1, 0.2]] * 3 + [[0.9, 0.2]] * 4 + [[0.9, 0.8]] * 2)
+    ids, _ = O.partition_blocks([10] * 9, Z, tau=0.5)
+    assert ids.tolist() == [0, 0, 0, 1, 1, 1, 1, 2, 2]
+    # the weights enter the difference: with the first diagnostic switched off only the second edge remains
+    ids, _ = O.partition_blocks([10] * 9, Z, w=[0.0, 1.0], tau=0.5)
+    assert ids.tolist() == [0] * 7 + [1, 1]
+
+
+def test_partition_small_units_join_their_statistically_closest_neighbour():
+    Z = np.array([[0.0], [0.9], [1.0]])
+    ids, _ = O.partition_blocks([100, 1, 100], Z, alpha=5 / 201, tau=0.5)
+    assert ids.tolist() == [0, 1, 1]
+    ids, _ = O.partition_blocks([100, 1, 100], np.array([[0.0], [0.1], [1.0]]), alpha=5 / 201, tau=0.5)
+    assert ids.tolist() == [0, 0, 1]
+    # equal differences: the smaller neighbour takes it
+    ids, _ = O.partition_blocks([100, 1, 50], np.array([[0.0], [0.5], [1.0]]), alpha=5 / 151, tau=0.3)
+    assert ids.tolist() == [0, 1, 1]
+    # a unit below the minimum never stays alone, whatever its statistics
+    ids, _ = O.partition_blocks([50, 2, 50, 3], np.array([[0.0], [9.0], [0.0], [-9.0]]), alpha=0.05, tau=0.1)
+    sizes = np.bincount(ids, weights=[50, 2, 50, 3])
+    assert np.all(sizes >= 0.05 * 105)
+
+
+def test_partition_splits_a_chain_of_small_steps_where_its_sides_differ():
+    # adjacent differences 0.3, 0.6, 0.3 <= tau, so block formation merges everything; the means of the two sides
+    # differ by 0.8, 0.9, 0.8 at the three cuts: the middle one wins and exceeds tau, the halves stay whole (0.3)
+    Z = np.array([[0.0], [0.3], [0.9], [1.2]])
+    ids, _ = O.partition_blocks([10] * 4, Z, tau=0.7)
+    assert ids.tolist() == [0, 0, 1, 1]
+    # the cut respects the minimum size: with n_min = 25 neither side of the middle cut fits
+    ids, _ = O.partition_blocks([10] * 4, Z, alpha=15 / 40, tau=0.7)
+    assert ids.tolist() == [0, 0, 1, 1]
+    ids, _ = O.partition_blocks([10] * 4, Z, alpha=25 / 40, tau=0.7)
+    assert ids.tolist() == [0, 0, 0, 0]
+    # weighted means: the heavy third unit pulls its side to 0.9, so the cut after the first unit separates most
+    # (0 against 0.897; the middle cut gives 0.15 against 0.903), and the rest holds together (0.3 against 0.903)
+    ids, _ = O.partition_blocks([10, 10, 1000, 10], Z, tau=0.7)
+    assert ids.tolist() == [0, 1, 1, 1]
+
+
+def test_partition_invariants_on_random_inputs():
+    rng = np.random.default_rng(5)
+    for trial in range(40):
+        m = int(rng.integers(1, 30))
+        sizes = rng.integers(1, 1000, size=m).tolist()
+        Z = rng.random((m, 5))
+        alpha = float(rng.choice([0.0, 0.01, 0.05, 0.2]))
+        ids, tau = O.partition_blocks(sizes, Z, alpha=alpha)
+        assert ids[0] == 0 and np.all(np.diff(ids) >= 0) and np.all(np.diff(ids) <= 1)     # contiguous, in order
+        per = np.bincount(ids, weights=sizes)
+        assert len(per) == 1 or np.all(per >= alpha * sum(sizes))
+        # a boundary that survived separates blocks whose statistics differ by more than tau, or was forced by nothing:
+        # merging two adjacent final blocks must not be something block formation would have done
+        if alpha == 0.0:
+            for b in range(len(per) - 1):
+                za = O._mean_z(sizes, Z, np.nonzero(ids == b)[0]); zb = O._mean_z(sizes, Z, np.nonzero(ids == b + 1)[0])
+                members_a, members_b = np.nonzero(ids == b)[0], np.nonzero(ids == b + 1)[0]
+                edge = O.partition_delta(Z[members_a[-1]], Z[members_b[0]], np.ones(5))
+                assert edge > tau or O.partition_delta(za, zb, np.ones(5)) > tau
