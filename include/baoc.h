@@ -245,6 +245,32 @@ int baoc_allocate(baoc_t* h, const double* risk, const int64_t* mem_bytes,
                   const uint8_t* forbid, const double* pref,
                   int32_t* assign_out, double* objective_out);
 
+/* ---- block partitioning (appendix on block partitioning, Algorithm 2) ----- */
+
+/* From candidate units to blocks.  The units come in forward order (the
+ * structural scan of the model is the caller's); numel[j] = n_j parameters;
+ * z: row-major [n_units][k] normalised diagnostic vectors (for instance s_A,
+ * s_M, C~, s_F, l_Q of baoc_block_stats_t after a window run with the units
+ * as blocks); w: k non-negative weights or NULL for w_k = 1; alpha: the
+ * minimum block size as a fraction of all parameters (n_min = alpha*|Theta|);
+ * tau: the statistic-difference threshold, negative for the paper's choice,
+ * the upper quartile of Delta(U_a,U_b) = max_k w_k |z_a,k - z_b,k| over all
+ * pairs of units.  The algorithm's steps are stated loosely; this library's
+ * reading: every gap between adjacent units is a candidate boundary; a group
+ * of units has the size-weighted mean of their vectors; a unit or group below
+ * n_min joins the adjacent group with the smaller Delta (ties: the smaller
+ * neighbour, then the left one); a boundary between adjacent groups survives
+ * iff their Delta exceeds tau; a formed block is cut again where the means of
+ * its two sides differ most, if by more than tau and both sides reach n_min;
+ * what is still below n_min is merged as before.  Blocks are runs of
+ * consecutive units: block_of_unit[j] (out, [n_units]) is non-decreasing from
+ * 0.  n_blocks and tau_used may be NULL.  Host only, no handle, no GPU.
+ * BAOC_E_INVALID: null, n_units < 1, k outside 1..64, numel < 1, alpha outside
+ * [0,1], a negative weight, a non-finite z or w, tau NaN. */
+int baoc_partition(int n_units, const int64_t* numel, const double* z, int k, const double* w,
+                   double alpha, double tau, int32_t* block_of_unit, int32_t* n_blocks,
+                   double* tau_used);
+
 /* ---- training (Algorithm 1 "Training") ----------------------------------- */
 
 /* Bytes of device memory the optimizer state of this assignment needs

@@ -80,7 +80,7 @@ EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error"
            "baoc_configure", "baoc_step", "baoc_step_from_host", "baoc_view", "baoc_nonfinite",
            "baoc_sample_stats_noalloc", "baoc_noalloc_last_error", "baoc_profile", "baoc_profile_last",
            "baoc_export", "baoc_import", "baoc_time_scratch_bytes", "baoc_measure_time_ratios",
-           "baoc_set_sampling", "baoc_reconfigure", "baoc_configure_from_window"]
+           "baoc_set_sampling", "baoc_reconfigure", "baoc_configure_from_window", "baoc_partition"]
 
 _vp = C.c_void_p
 _lib.baoc_default_opts.argtypes = [C.POINTER(Opts)]
@@ -107,6 +107,7 @@ _lib.baoc_view.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(_vp), C.POINTER(C.c_
 _lib.baoc_nonfinite.argtypes = [_vp, _vp, C.POINTER(C.c_int32), _vp]
 _lib.baoc_reconfigure.argtypes = [_vp, _vp, _vp, C.c_size_t, C.c_int64, C.c_int, _vp]
 _lib.baoc_configure_from_window.argtypes = [_vp, _vp, _vp, C.c_size_t, _vp]
+_lib.baoc_partition.argtypes = [C.c_int, _vp, _vp, C.c_int, _vp, C.c_double, C.c_double, _vp, _vp, _vp]
 _lib.baoc_set_sampling.argtypes = [_vp, C.POINTER(Sample)]
 _lib.baoc_time_scratch_bytes.argtypes = [_vp, C.POINTER(C.c_size_t)]
 _lib.baoc_measure_time_ratios.argtypes = [_vp, _vp, _vp, _vp, C.c_size_t, C.c_int, C.c_int, _vp, _vp, _vp]
@@ -131,6 +132,31 @@ def sample_stats_noalloc(grad: torch.Tensor, gprev: torch.Tensor, m: torch.Tenso
                                         float(beta_m), float(beta_v), float(eps), out4.data_ptr(), _stream())
     if rc < 0:
         raise BaocError(rc, _lib.baoc_noalloc_last_error().decode())
+
+
+def partition(numel, z, w=None, alpha: float = 0.0, tau: Optional[float] = None):
+    """``baoc_partition`` (Algorithm 2): candidate units in forward order -> (block index of every unit, tau used).
+    z: [n_units, k] normalised diagnostic vectors; tau None = the upper quartile of the pairwise differences."""
+    n = np.ascontiguousarray(numel, np.int64)
+    Z = np.ascontiguousarray(z, np.float64)
+    if Z.ndim != 2 or Z.shape[0] != n.shape[0]:
+        raise ValueError("z must be [n_units, k]")
+    ww = None if w is None else np.ascontiguousarray(w, np.float64)
+    if ww is not None and ww.shape != (Z.shape[1],):
+        raise ValueError("w must have k entries")
+    out = np.zeros(n.shape[0], np.int32)
+    nb, tu = C.c_int32(), C.c_double()
+    rc = _lib.baoc_partition(n.shape[0], n.ctypes.data, Z.ctypes.data, Z.shape[1], _np_ptr(ww), float(alpha),
+                             -1.0 if tau is None else float(tau), out.ctypes.data, C.addressof(nb), C.addressof(tu))
+    if rc < 0:
+        raise BaocError(rc, "baoc_partition: invalid argument")
+    return out, tu.value
+
+
+def unit_diagnostics(stats) -> np.ndarray:
+    """[n, 5] normalised diagnostic vectors (s_A, s_M, C~, s_F, l_Q at 8 bits) from ``Baoc.risk``'s per-block records:
+    the z_j that ``partition`` takes when the candidate units were run through a window as blocks."""
+    return np.asarray([[s.s_A, s.s_M, s.C_tilde, s.s_F, s.lQ8] for s in stats], np.float64)
 
 
 def default_opts() -> Opts:

@@ -249,3 +249,39 @@ def test_set_sampling_validates_indices_and_shrinks_the_workspace(B):
     assert e.value.code == B.E_INVALID
     h.set_sampling(None)
     assert h.stats_workspace_bytes() == dense
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_partition_equals_the_oracle(B, seed):
+    """Algorithm 2 in the library against the oracle: the block of every unit and the threshold, bit for bit."""
+    rng = np.random.default_rng(100 + seed)
+    for trial in range(30):
+        m = int(rng.integers(1, 40))
+        k = int(rng.integers(1, 6))
+        sizes = rng.integers(1, 5000, size=m)
+        Z = rng.random((m, k))
+        if trial % 3 == 0:                                          # smooth drifts plus jumps: formation merges, the split cuts
+            Z = np.cumsum(rng.random((m, k)) * 0.08, axis=0) + (rng.random((m, 1)) < 0.15).cumsum(axis=0) * 0.5
+        if trial % 5 == 0:
+            Z[rng.integers(0, m)] = Z[0]                            # identical units
+        w = None if trial % 2 else rng.random(k) * 2
+        alpha = float(rng.choice([0.0, 0.005, 0.03, 0.1, 0.3]))
+        tau = None if trial % 4 else float(rng.random() * 0.6)
+        want, tau_want = O.partition_blocks(sizes.tolist(), Z, w, alpha, tau)
+        got, tau_got = B.partition(sizes, Z, w, alpha, tau)
+        assert tau_got == tau_want
+        assert got.tolist() == want.tolist(), (seed, trial)
+
+
+def test_partition_rejects_bad_arguments(B):
+    Z = np.zeros((3, 2))
+    for bad in (dict(numel=[1, 0, 2]), dict(alpha=-0.1), dict(alpha=1.5), dict(w=[1.0, -1.0]), dict(tau=float("nan"))):
+        args = dict(numel=[4, 5, 6], z=Z, w=None, alpha=0.0, tau=None)
+        args.update(bad)
+        with pytest.raises(B.BaocError):
+            B.partition(**args)
+    Zbad = Z.copy(); Zbad[1, 1] = np.inf
+    with pytest.raises(B.BaocError):
+        B.partition([4, 5, 6], Zbad)
+    ids, tau = B.partition([7], np.ones((1, 5)))
+    assert ids.tolist() == [0] and tau == 0.0
