@@ -34,6 +34,13 @@ __device__ __forceinline__ uint2 ld_stream_u2(const void* p) {
     asm volatile("ld.global.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));
     return r;
 }
+// A load that stays where it is written: the compiler may neither delay it to its first use nor repeat it there.  For
+// values fetched well ahead of their use (a register prefetch), where sinking the load would expose its full latency.
+__device__ __forceinline__ float ld_pinned_f32(const float* p) {
+    float v;
+    asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
 __device__ __forceinline__ void st_stream_f4(void* p, float4 v) {
     asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }

@@ -672,27 +672,25 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         cp_async_commit();
         fill = fill == (kStagesQ - 1) * kStageBytes ? 0u : fill + kStageBytes;
     };
-    // the old absmax pair of a slice travels in registers, the same distance ahead
-    auto absmax_of = [&](int s, float& a_m, float& a_v) {
-        const int w = s * (kThreads * 8) + warp * kQBlock;
-        a_m = 0.f; a_v = 0.f;
-        if (s < kSlicesQ && w < left) {
-            if (kM) a_m = amt[w / kQBlock];
-            if (kV) a_v = avt[w / kQBlock];
-        }
-    };
-    float amo_1, avo_1, amo_2, avo_2;
+    // The old absmax values of the whole tile are fetched once, before the first wait: lane l < 8 of a warp holds the
+    // first moment's absmax of the warp's quantisation block in slice l, lane 8 + l the second moment's.  (Fetched
+    // slice by slice they arrived late: a plain load queues behind the copies in flight and takes longer than a slice.)
+    static_assert(kSlicesQ <= 8, "one lane per slice and moment");
+    float amax_old = 0.f;
+    {
+        const int sl = lane & 7, w = sl * (kThreads * 8) + warp * kQBlock;
+        const bool second = (lane & 8) != 0;
+        if (lane < 16 && sl < kSlicesQ && w < left && (second ? kV : kM))
+            amax_old = ld_pinned_f32((second ? avt : amt) + w / kQBlock);
+    }
 #pragma unroll
     for (int k = 0; k < kStagesQ - 1; ++k) prefetch(k);
-    absmax_of(0, amo_1, avo_1); absmax_of(1, amo_2, avo_2);
     uint32_t take = 0;                                               // byte offset of the stage the current slice sits in
 #pragma unroll 1
     for (int s = 0; s < kSlicesQ; ++s) {
         const int w0 = s * (kThreads * 8) + warp * kQBlock;
         prefetch(s + kStagesQ - 1);
-        const float amo = amo_1, avo = avo_1;
-        amo_1 = amo_2; avo_1 = avo_2;
-        absmax_of(s + 2, amo_2, avo_2);
+        const float amo = kM ? __shfl_sync(full, amax_old, s) : 0.f, avo = kV ? __shfl_sync(full, amax_old, 8 + s) : 0.f;
         cp_async_wait<kStagesQ - 1>();                              // this slice's copies have landed (the later ones may be in flight)
         if (w0 >= left) break;                                      // whole warp out of range (and so are the later slices)
         const int e = w0 + lane * 8;
