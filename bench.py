@@ -48,16 +48,15 @@ def _ncu_traffic(kernel, algorithmic_bytes):
     """DRAM bytes per launch of `kernel`, scaled from the recorded ncu capture of a smaller case by the algorithmic
     bytes of this launch (traffic is proportional to the parameters processed).  None when there is no record or
     the kernel sources have changed since the counters were taken."""
-    import glob
     import hashlib
     pkg = os.path.join(ROOT, "paper_2605_04711_b200")
     try:
         rec = json.load(open(os.path.join(pkg, "ncu_traffic.json")))
         h = hashlib.sha256()
-        for f in sorted(glob.glob(os.path.join(pkg, "csrc", "*"))):
-            h.update(os.path.basename(f).encode())
-            h.update(open(f, "rb").read())
-        if h.hexdigest() != rec["csrc_sha256"] or kernel not in rec:
+        for name in rec["kernel_sources"]:               # the files that define the two kernels and what they include
+            h.update(name.encode())
+            h.update(open(os.path.join(pkg, "csrc", name), "rb").read())
+        if h.hexdigest() != rec["kernel_sources_sha256"] or kernel not in rec:
             return None
         k = rec[kernel]
         return float(k["dram_bytes"]) / float(k["algorithmic_bytes"]) * float(algorithmic_bytes)

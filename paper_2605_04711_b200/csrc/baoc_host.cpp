@@ -49,13 +49,24 @@ double step_traffic_bytes(const baoc_config_t& c, const baoc_block_t& b) {
     return bytes;
 }
 
-RedGeom red_geometry(int32_t rows, int32_t cols) {
+// About 16 * refine row chunks per matrix (never finer than one group of 64 rows).
+RedGeom red_geometry(int32_t rows, int32_t cols, int refine) {
     RedGeom g{};
     g.rowpart = nullptr; g.colpart = nullptr; g.red0 = -1;
-    g.L = int32_t(std::max<int64_t>(1, ceil_div(rows, int64_t(kRedRows) * 16)));   // about 16 row chunks per matrix
+    const int64_t groups = ceil_div(rows, kRedRows);
+    g.L = int32_t(std::max<int64_t>(1, ceil_div(groups, std::min<int64_t>(16 * int64_t(refine), groups))));
     g.chunks = int32_t(ceil_div(rows, int64_t(kRedRows) * g.L));
     g.strips = int32_t(ceil_div(cols, kRedCols));
     return g;
+}
+
+// How much finer than 16 row chunks per matrix the reduction has to cut so that all the matrices together give about
+// four CTAs per SM: coarse chunks move the fewest partial sums, but a few narrow matrices alone (an embedding table
+// of 768 columns is two strips) would leave most of the GPU idle.
+static int red_refinement(int64_t ctas_at_16_chunks) {
+    constexpr int64_t kWant = 4 * 148;
+    if (ctas_at_16_chunks <= 0 || ctas_at_16_chunks >= kWant) return 1;
+    return int(std::min<int64_t>(64, ceil_div(kWant, ctas_at_16_chunks)));
 }
 
 static size_t take(size_t* cur, size_t bytes) {
@@ -72,6 +83,12 @@ void compute_stat_layout(Handle* h) {
     int64_t tiles = 0, red = 0, padded = 0, sum_rows = 0, sum_cols = 0, redpart = 0, n_ridx = 0, n_cidx = 0;
     h->h_stat_blocks.assign(n, StatBlock{});
     if (!h->sampled) h->stat_shapes = h->blocks;
+    int64_t coarse = 0;
+    for (int i = 0; i < n; ++i) {
+        const baoc_block_t& b = h->stat_shapes[i];
+        if (b.cols > 1) { const RedGeom g = red_geometry(b.rows, b.cols, 1); coarse += int64_t(g.chunks) * g.strips; }
+    }
+    const int refine = red_refinement(coarse);
     for (int i = 0; i < n; ++i) {
         const baoc_block_t& b = h->stat_shapes[i];
         StatBlock& s = h->h_stat_blocks[i];
@@ -90,7 +107,7 @@ void compute_stat_layout(Handle* h) {
         s.v = reinterpret_cast<float*>(size_t(padded) * 4);
         s.gprev = reinterpret_cast<uint16_t*>(size_t(padded) * 2);
         padded += round_up(b.numel, kQBlock);
-        s.red = red_geometry(b.rows, b.cols);
+        s.red = red_geometry(b.rows, b.cols, refine);
         if (b.cols > 1) {
             s.red.red0 = int32_t(red);
             red += int64_t(s.red.chunks) * s.red.strips;
@@ -147,6 +164,13 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
     size_t states = 0, redpart = 0;
     int64_t mem = 0;
     double traffic = 0;
+    int64_t coarse = 0;
+    for (int i = 0; i < n; ++i)
+        if (assign[i] >= 0 && assign[i] < h->n_cfg && path_of(h->cfgs[assign[i]]) == kPathF) {
+            const RedGeom g = red_geometry(h->blocks[i].rows, h->blocks[i].cols, 1);
+            coarse += int64_t(g.chunks) * g.strips;
+        }
+    const int refine = red_refinement(coarse);
     for (int i = 0; i < n; ++i) {
         const int c = assign[i];
         if (c < 0 || c >= h->n_cfg) return fail(h, BAOC_E_INVALID, "assignment names a configuration that does not exist");
@@ -157,7 +181,7 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
         StepBlock& s = sb[i];
         s = StepBlock{};
         s.numel = b.numel; s.rows = b.rows; s.cols = b.cols; s.cfg = c; s.path = p;
-        s.red = red_geometry(b.rows, b.cols);
+        s.red = red_geometry(b.rows, b.cols, refine);
         const size_t dpad = size_t(round_up(b.numel, kQBlock));
         const size_t nq = size_t(ceil_div(b.numel, kQBlock));
         auto place = [&](size_t bytes) { return reinterpret_cast<void*>(take(&states, bytes)); };

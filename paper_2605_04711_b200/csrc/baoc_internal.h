@@ -246,7 +246,7 @@ struct Handle {
 int fail(const Handle* h, int code, const std::string& msg);
 
 // Reduction geometry of a rows x cols matrix (pointers left null).
-RedGeom red_geometry(int32_t rows, int32_t cols);
+RedGeom red_geometry(int32_t rows, int32_t cols, int refine);
 
 // M_{i,c}: bytes of persistent state of one block under one configuration.
 int64_t state_mem_bytes(const baoc_config_t& c, const baoc_block_t& b);
