@@ -163,10 +163,15 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
         h->launches += 2;
     }
     if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[1]), s), "baoc_step (profile)");
-    LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles), at<const void*>(h->st, L.grads),
-                             at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), h->n_step_tiles, h->wide_paths, P, s),
-           "fused_step_kernel");
-    h->launches += 1;
+    int64_t first = 0;
+    for (int fam = 0; fam < kFamCount; ++fam) {                     // one launch per path family present
+        if (h->fam_tiles[fam] == 0) continue;
+        LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles) + first, at<const void*>(h->st, L.grads),
+                                 at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), h->fam_tiles[fam], fam, P, s),
+               "fused_step_kernel");
+        h->launches += 1;
+        first += h->fam_tiles[fam];
+    }
     if (h->prof_on) {
         CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[2]), s), "baoc_step (profile)");
         h->prof_valid = true;
@@ -424,8 +429,8 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
     h->h_step_blocks = sb;
     h->n_step_tiles = int64_t(tiles.size()); h->n_step_red_tiles = int64_t(red.size());
     h->n_factored = int(ids.size());
-    h->wide_paths = false;
-    for (const StepBlock& b : sb) h->wide_paths = h->wide_paths || b.path >= kPathG;
+    for (int64_t& c : h->fam_tiles) c = 0;
+    for (const StepBlock& b : sb) h->fam_tiles[family_of(b.path)] += ceil_div(b.numel, step_tile_elems(b.path));
     h->state_mem = mem; h->step_bytes = traffic;
     h->last_step_grads.clear(); h->last_step_params.clear();
     return BAOC_OK;

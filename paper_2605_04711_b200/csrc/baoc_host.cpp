@@ -228,8 +228,9 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
         mem += state_mem_bytes(h->cfgs[c], b);
         traffic += step_traffic_bytes(h->cfgs[c], b);
     }
-    // tiles in descending bytes per element so that the light ones fill the tail of the grid
-    const int order[kPathCount] = {kPathA32, kPathR, kPathS, kPathA16, kPathR16, kPathS16, kPathG, kPathA8, kPathR8, kPathS8, kPathF};
+    // the tiles of one path family after another (each family has its own kernel instance); within a family in
+    // descending bytes per element, so that the light tiles fill the tail of the grid
+    const int order[kPathCount] = {kPathA32, kPathR, kPathS, kPathA8, kPathF, kPathA16, kPathR16, kPathS16, kPathG, kPathR8, kPathS8};
     for (int p : order)
         for (int i = 0; i < n; ++i)
             if (sb[i].path == p) {

@@ -9,6 +9,12 @@
 
 #include "baoc.h"
 
+#ifdef __CUDACC__
+#define BAOC_HD __host__ __device__
+#else
+#define BAOC_HD
+#endif
+
 struct CUstream_st;
 typedef CUstream_st* cudaStream_t;
 
@@ -52,8 +58,18 @@ inline Path path_of(const baoc_config_t& c) {
     return kPathG;       // neither mechanism: stateless, whatever bit-width the tuple names
 }
 
+// Families of update paths: each has its own instance of the fused kernel and its own stretch of the tile table.
+enum Family : int32_t { kFamHead = 0, kFamDense = 1, kFamQ8 = 2, kFamCount = 3 };
+inline int family_of(int path) {
+    switch (path) {
+        case kPathG: case kPathA16: case kPathR16: case kPathS16: return kFamDense;
+        case kPathR8: case kPathS8: return kFamQ8;
+        default: return kFamHead;
+    }
+}
+
 // Elements per tile of the fused step, by update path.
-inline int64_t step_tile_elems(int path) {
+BAOC_HD inline int64_t step_tile_elems(int path) {
     return path == kPathF ? kTileF : ((path == kPathA8 || path == kPathR8 || path == kPathS8) ? kTileQ : kTile);
 }
 
@@ -216,7 +232,7 @@ struct Handle {
     int64_t n_step_tiles = 0;
     int64_t n_step_red_tiles = 0;
     int n_factored = 0;              // blocks on the factored path
-    bool wide_paths = false;         // some block is on a path outside the five headline ones
+    int64_t fam_tiles[kFamCount] = {0, 0, 0};   // tiles of each path family; the tile table holds the families one after another
     // Bias corrections count the gradients a moment has seen.  A re-configuration may restart some moments, so every
     // block carries the step counts at which its first and second moment last started from zero; blocks that share a
     // configuration and both counts share a slot of the step's parameter table.
@@ -274,7 +290,7 @@ int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const i
 int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const int32_t* ids, const void* const* grads,
                            const float* const* params, int64_t n_red, int n_factored, const StepParams& P, cudaStream_t s);
 int launch_fused_step(const StepBlock* blocks, const Tile* tiles, const void* const* grads, float* const* params,
-                      uint32_t* flags, int64_t n_tiles, bool all_paths, const StepParams& P, cudaStream_t s);
+                      uint32_t* flags, int64_t n_tiles, int family, const StepParams& P, cudaStream_t s);
 int launch_convert_moment(const MomentRef& src, const MomentRef& dst, int64_t numel, cudaStream_t s);
 int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayout* out,
                         std::vector<StepBlock>* blocks, std::vector<Tile>* tiles,

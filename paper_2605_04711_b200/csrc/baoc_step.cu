@@ -323,19 +323,23 @@ constexpr int kStageBytes = kThreads * 64;                           // g 16 B/t
 // taken exactly: the fp32 moment is within err of the exact one, and unless it lies within err of the midpoint
 // between the two bf16 neighbours its rounding is already the exact answer; the few that do are recomputed in
 // double (and rounded double -> fp32 -> bf16).
-__device__ __forceinline__ uint32_t bf16_rne_bits(float x) {
-    const uint32_t u = __float_as_uint(x);
-    if ((u & 0x7f800000u) == 0x7f800000u) return u >> 16;           // infinities and NaNs keep their top half
-    return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
+// Two floats rounded to bf16 (nearest, ties to even) and packed, `lo` in the low half: one instruction.
+__device__ __forceinline__ uint32_t pack_bf16x2_rne(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
 }
 
 template <bool kM, bool kV, bool kB16>
 struct DenseElem {
     // One element.  x: gradient, t: parameter (updated), m / v: old moments (replaced by the new fp32 ones),
-    // mb / vb: bf16 bits of the new moments when kB16.
-    static __device__ __forceinline__ void upd(float x, float& t, float& m, float& v, uint32_t& mb, uint32_t& vb,
+    // mr / vr (kB16): the values whose bf16 rounding is to be stored: the new moments, or their exact recomputation.
+    static __device__ __forceinline__ void upd(float x, float& t, float& m, float& v, float& mr, float& vr,
                                                const CfgStep& P) {
-        constexpr float kErr = 4.76837158203125e-7f;                // 2^-21: twice the first-order bound of four roundings
+        // The fp32 moment differs from the exact one by at most 2^-24 (2 |p| + |m|) (p: the gradient term, rounded once
+        // as a product and once through the rounded coefficient; m: the final FMA), plus as much again through p when
+        // a coupled decay has rounded the gradient first: 2^-22 (|p| + |m|) covers the first, 2^-21 both.
+        const float kErr = P.coupled ? 4.76837158203125e-7f : 2.384185791015625e-7f;
         const float x_raw = x, t_old = t, m_old = m, v_old = v;
         prologue(x, t, P);
         float pm = 0.f, pv = 0.f;
@@ -345,19 +349,17 @@ struct DenseElem {
             auto exact_g = [&]() { return P.coupled ? double(x_raw) + P.wd_d * double(t_old) : double(x_raw); };
             if (kM) {
                 const float mid = __uint_as_float((__float_as_uint(m) & 0xffff0000u) | 0x8000u);
-                float r = m;
+                mr = m;
                 if (fabsf(m - mid) <= kErr * (fabsf(pm) + fabsf(m)))
-                    r = __double2float_rn(P.beta1_d * double(m_old) + (kV ? 1.0 - P.beta1_d : 1.0) * exact_g());
-                mb = bf16_rne_bits(r);
+                    mr = __double2float_rn(P.beta1_d * double(m_old) + (kV ? 1.0 - P.beta1_d : 1.0) * exact_g());
             }
             if (kV) {
                 const float mid = __uint_as_float((__float_as_uint(v) & 0xffff0000u) | 0x8000u);
-                float r = v;
+                vr = v;
                 if (fabsf(v - mid) <= kErr * (pv + v)) {
                     const double gd = exact_g();
-                    r = __double2float_rn(P.beta2_d * double(v_old) + (1.0 - P.beta2_d) * (gd * gd));
+                    vr = __double2float_rn(P.beta2_d * double(v_old) + (1.0 - P.beta2_d) * (gd * gd));
                 }
-                vb = bf16_rne_bits(r);
             }
         }
         if (kM && kV) t = adaptive_apply(t, m, v, P.step_m, P);
@@ -403,7 +405,7 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
         const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
         if (full[s]) {
             float x[8], t[8], mm[8], vv[8];
-            uint32_t mb[8], vb[8];
+            float mb[8], vb[8];
             unpack8(wg[s], x); f4_to(t0[s], t1[s], t);
             if (kB16) {
                 if (kM) unpack8(mw[s], mm);
@@ -419,8 +421,10 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
             }
             st8(th + e, t);
             if (kB16) {
-                if (kM) st_stream_u4(mh + e, make_uint4(mb[0] | mb[1] << 16, mb[2] | mb[3] << 16, mb[4] | mb[5] << 16, mb[6] | mb[7] << 16));
-                if (kV) st_stream_u4(vh + e, make_uint4(vb[0] | vb[1] << 16, vb[2] | vb[3] << 16, vb[4] | vb[5] << 16, vb[6] | vb[7] << 16));
+                if (kM) st_stream_u4(mh + e, make_uint4(pack_bf16x2_rne(mb[0], mb[1]), pack_bf16x2_rne(mb[2], mb[3]),
+                                                        pack_bf16x2_rne(mb[4], mb[5]), pack_bf16x2_rne(mb[6], mb[7])));
+                if (kV) st_stream_u4(vh + e, make_uint4(pack_bf16x2_rne(vb[0], vb[1]), pack_bf16x2_rne(vb[2], vb[3]),
+                                                        pack_bf16x2_rne(vb[4], vb[5]), pack_bf16x2_rne(vb[6], vb[7])));
             } else {
                 if (kM) st8(m + e, mm);
                 if (kV) st8(v + e, vv);
@@ -430,15 +434,15 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
             for (int j = 0; j < cnt; ++j) {
                 const float x = bf16_bits_to_float(g[e + j]);
                 float t = th[e + j], mm = 0.f, vv = 0.f;
-                uint32_t mb = 0u, vb = 0u;
+                float mb = 0.f, vb = 0.f;
                 if (kM) mm = kB16 ? bf16_bits_to_float(mh[e + j]) : m[e + j];
                 if (kV) vv = kB16 ? bf16_bits_to_float(vh[e + j]) : v[e + j];
                 DenseElem<kM, kV, kB16>::upd(x, t, mm, vv, mb, vb, P);
                 chk = poison(chk, t);
                 th[e + j] = t;
                 if (kB16) {
-                    if (kM) mh[e + j] = uint16_t(mb);
-                    if (kV) vh[e + j] = uint16_t(vb);
+                    if (kM) mh[e + j] = uint16_t(pack_bf16x2_rne(mb, 0.f));
+                    if (kV) vh[e + j] = uint16_t(pack_bf16x2_rne(vb, 0.f));
                 } else {
                     if (kM) m[e + j] = mm;
                     if (kV) v[e + j] = vv;
@@ -862,12 +866,16 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
     return !isfinite(c0) | !isfinite(c1);
 }
 
-// Two instances of the kernel: the first holds the five headline paths only, the second all paths.  Compiled next
-// to the headline paths, the bf16-state and stateless variants cost those paths registers at the 80-register budget
-// of three CTAs per SM (2-3 % of the step), so the host launches the wider instance only when the assignment uses
-// one of them.  Either way a step is one launch.
-template <bool kAllPaths>
-__global__ void __launch_bounds__(kThreads, 3)
+// Three instances of the kernel, one per family of update paths, each over its own stretch of the tile table:
+//   kFamHead   the five headline paths (fp32 Adam / RMS / SGD-momentum, 8-bit Adam, factored): 80 registers, three
+//              CTAs per SM, 48 KB of shared memory for the cp.async rings;
+//   kFamDense  the stateless and bf16-state dense paths: no shared memory, 64 registers, four CTAs per SM (these
+//              paths keep fewer bytes per thread in flight, so they want the extra CTA);
+//   kFamQ8     8-bit RMS scaling and 8-bit SGD-momentum: as the headline 8-bit path.
+// Compiled into one kernel, the extra paths cost the headline ones registers at the 80-register budget (about 9 % on
+// the factored tiles), so a step is one launch when the assignment stays within one family and up to three otherwise.
+template <int kFam>
+__global__ void __launch_bounds__(kThreads, kFam == kFamDense ? 4 : 3)
 fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
                   const void* const* __restrict__ grads, float* const* __restrict__ params,
                   uint32_t* __restrict__ flags, const __grid_constant__ StepParams SP) {
@@ -876,22 +884,34 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
     const CfgStep& P = SP.c[b->cfg];
     const uint16_t* g = static_cast<const uint16_t*>(grads[t.block]);
     float* th = params[t.block];
-    const int64_t base = int64_t(t.piece) * (b->path == kPathF ? kTileF : ((b->path == kPathA8 || b->path == kPathR8 || b->path == kPathS8) ? kTileQ : kTile));
-    __shared__ __align__(16) unsigned char q_stage[kStagesQ * kStageBytes];   // per-thread staging of the 8-bit and factored paths
+    const int64_t base = int64_t(t.piece) * step_tile_elems(b->path);
     unsigned bad = 0;
-    switch (b->path) {
-        case kPathA32: bad = tile_dense<true, true, false>(b, P, g, th, base); break;
-        case kPathR: bad = tile_dense<false, true, false>(b, P, g, th, base); break;
-        case kPathS: bad = tile_dense<true, false, false>(b, P, g, th, base); break;
-        case kPathG: if (kAllPaths) bad = tile_dense<false, false, false>(b, P, g, th, base); break;
-        case kPathA16: if (kAllPaths) bad = tile_dense<true, true, true>(b, P, g, th, base); break;
-        case kPathR16: if (kAllPaths) bad = tile_dense<false, true, true>(b, P, g, th, base); break;
-        case kPathS16: if (kAllPaths) bad = tile_dense<true, false, true>(b, P, g, th, base); break;
-        case kPathA8: bad = P.coupled ? tile_int8<true, true, true>(b, P, g, th, base, q_stage) : tile_int8<false, true, true>(b, P, g, th, base, q_stage); break;
-        case kPathR8: if (kAllPaths) bad = P.coupled ? tile_int8<true, false, true>(b, P, g, th, base, q_stage) : tile_int8<false, false, true>(b, P, g, th, base, q_stage); break;
-        case kPathS8: if (kAllPaths) bad = P.coupled ? tile_int8<true, true, false>(b, P, g, th, base, q_stage) : tile_int8<false, true, false>(b, P, g, th, base, q_stage); break;
-        case kPathF: bad = tile_factored(b, P, g, th, base, q_stage); break;
-        default: break;
+    if (kFam == kFamDense) {
+        switch (b->path) {
+            case kPathG: bad = tile_dense<false, false, false>(b, P, g, th, base); break;
+            case kPathA16: bad = tile_dense<true, true, true>(b, P, g, th, base); break;
+            case kPathR16: bad = tile_dense<false, true, true>(b, P, g, th, base); break;
+            case kPathS16: bad = tile_dense<true, false, true>(b, P, g, th, base); break;
+            default: break;
+        }
+    } else {
+        __shared__ __align__(16) unsigned char q_stage[kStagesQ * kStageBytes];   // per-thread staging of the 8-bit and factored paths
+        if (kFam == kFamHead) {
+            switch (b->path) {
+                case kPathA32: bad = tile_dense<true, true, false>(b, P, g, th, base); break;
+                case kPathR: bad = tile_dense<false, true, false>(b, P, g, th, base); break;
+                case kPathS: bad = tile_dense<true, false, false>(b, P, g, th, base); break;
+                case kPathA8: bad = P.coupled ? tile_int8<true, true, true>(b, P, g, th, base, q_stage) : tile_int8<false, true, true>(b, P, g, th, base, q_stage); break;
+                case kPathF: bad = tile_factored(b, P, g, th, base, q_stage); break;
+                default: break;
+            }
+        } else {
+            switch (b->path) {
+                case kPathR8: bad = P.coupled ? tile_int8<true, false, true>(b, P, g, th, base, q_stage) : tile_int8<false, false, true>(b, P, g, th, base, q_stage); break;
+                case kPathS8: bad = P.coupled ? tile_int8<true, true, false>(b, P, g, th, base, q_stage) : tile_int8<false, true, false>(b, P, g, th, base, q_stage); break;
+                default: break;
+            }
+        }
     }
     if (bad) atomicOr(flags + t.block, 1u);
 }
@@ -924,9 +944,12 @@ int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const
 }
 
 int launch_fused_step(const StepBlock* blocks, const Tile* tiles, const void* const* grads, float* const* params,
-                      uint32_t* flags, int64_t n_tiles, bool all_paths, const StepParams& P, cudaStream_t s) {
-    if (all_paths) fused_step_kernel<true><<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
-    else fused_step_kernel<false><<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
+                      uint32_t* flags, int64_t n_tiles, int family, const StepParams& P, cudaStream_t s) {
+    if (n_tiles <= 0) return 0;
+    const unsigned grid = unsigned(n_tiles);
+    if (family == kFamHead) fused_step_kernel<kFamHead><<<grid, kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
+    else if (family == kFamDense) fused_step_kernel<kFamDense><<<grid, kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
+    else fused_step_kernel<kFamQ8><<<grid, kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
     BAOC_LAUNCH_CHECK();
     return 0;
 }
