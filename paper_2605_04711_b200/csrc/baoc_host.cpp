@@ -113,7 +113,7 @@ void compute_stat_layout(Handle* h) {
             red += int64_t(s.red.chunks) * s.red.strips;
             s.rowsum = reinterpret_cast<double*>(size_t(sum_rows) * 8);
             s.colsum = reinterpret_cast<double*>(size_t(sum_cols) * 8);
-            sum_rows += b.rows; sum_cols += b.cols;
+            sum_rows += b.rows; sum_cols += round_up(b.cols, 2);   // column sums start 16-byte aligned (read in pairs)
             s.red.rowpart = reinterpret_cast<double*>(size_t(redpart) * 8);
             redpart += int64_t(s.red.strips) * b.rows;
             s.red.colpart = reinterpret_cast<double*>(size_t(redpart) * 8);

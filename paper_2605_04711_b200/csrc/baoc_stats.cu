@@ -210,10 +210,11 @@ stats_final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __rest
             const float m8 = (fmaf(mj, km, kMagic) - kMagic) * dm;
             const float v8 = (fmaf(vj, kv, kMagic) - kMagic) * dv;
             const float m16 = round_to_bf16(mj), v16 = round_to_bf16(vj);
-            const float u32 = mj * rcp_approx(sqrt_approx(vj) + eps_adam);
+            const float sq = __fsqrt_rn(vj);                        // shared by the direction and by p (precond_of's own value)
+            const float u32 = mj * rcp_approx(sq + eps_adam);
             const float u8 = m8 * rcp_approx(sqrt_approx(v8) + eps_adam);
             const float u16 = m16 * rcp_approx(sqrt_approx(v16) + eps_adam);
-            pj[j] = in ? precond_of(vj, eps_f) : 0.f;
+            pj[j] = in ? __fdiv_rn(1.0f, sq + eps_f) : 0.f;
             f[0] = fmaf(mj, mj, f[0]); f[1] += vj; f[2] = fmaf(vj, vj, f[2]);
             f[4] = fmaf(tt[j], tt[j], f[4]);
             f[5] = fmaf(u32, u32, f[5]); f[6] = fmaf(u8, u8, f[6]); f[7] = fmaf(u32, u8, f[7]);
@@ -285,6 +286,27 @@ stats_final_resid_kernel(const StatBlock* __restrict__ blocks, const Tile* __res
         int64_t r = matrix ? e / cols : 0;
         int c = matrix ? int(e - r * cols) : 0;
         double rs = matrix ? __ldg(rowsum + r) * inv_total : 0.0;
+        if (cnt == 8 && (!matrix || (cols & 7) == 0)) {
+            // the eight elements lie in one row (or the block is a vector): one row sum, four 16-byte loads of column sums
+            double cs[8];
+            if (matrix) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const double2 w = __ldg(reinterpret_cast<const double2*>(colsum + c) + q);
+                    cs[2 * q] = w.x; cs[2 * q + 1] = w.y;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const double d = (double(precond_of(vv[j], eps_f)) * inv_pbar - 1.0) * double(tt[j]);
+                acc[0] += d * d;
+                if (matrix) {
+                    const double diff = double(vv[j]) - rs * cs[j];
+                    acc[1] += diff * diff;
+                }
+            }
+            continue;
+        }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             if (j < cnt) {
