@@ -212,3 +212,102 @@ def test_one_block_beyond_two_to_the_31_elements():
         assert np.max(np.abs(got - th)) <= 1e-6 * np.max(np.abs(th)), (a, b)
         assert np.max(np.abs(m_dev[a:b].double().cpu().numpy() - st.m)) <= 1e-6 * np.max(np.abs(st.m))
         assert np.max(np.abs(mhat[a:b].double().cpu().numpy() - ss.m)) <= 1e-6 * np.max(np.abs(ss.m))
+
+
+def test_every_tuple_family_in_one_step_at_full_size():
+    """All thirteen instantiable tuples dealt round-robin over the blocks of the LLaMA-1B-shaped workload, so that one
+    step launches every kernel instance (headline paths, stateless / bf16 dense paths, 8-bit single-moment paths) over
+    its stretch of the tile table; three steps, checked on slices (whole blocks for the factored ones)."""
+    from paper_2605_04711_b200 import binding as B, harness as H
+    wl = W.make_workload("llama_1b", seed=1)
+    bcfgs = B.extended_configs()
+    sess = H.Session(wl, configs=bcfgs, n_grad_sets=2)
+    sess.init_params()
+    cfgs = [_ocfg(c) for c in bcfgs]
+    factored = {3: 2, 11: 7, 12: 9}                                  # vectors take RMS scaling at the same precision
+    assign = []
+    for i, b in enumerate(wl.blocks):
+        c = i % len(bcfgs)
+        assign.append(factored[c] if (c in factored and b.cols <= 1) else c)
+    kinds = [O.config_kind(cfgs[c]) for c in assign]
+    assert set(kinds) == {"A32", "A8", "R", "F", "S", "G", "A16", "R16", "S16", "R8", "S8", "F16", "F8"}
+    sess.configure(assign)
+    mem, _ = sess.h.cost_model()
+    assert sess.h.query().state_bytes == sum(int(mem[i, c]) for i, c in enumerate(assign))
+    picks = []
+    for kind in sorted(set(kinds)):
+        ids = [i for i, k in enumerate(kinds) if k == kind]
+        if kind.startswith("F"):
+            ids = [i for i in ids if wl.blocks[i].numel <= 17_000_000] or ids
+            picks += [(ids[0], kind)]
+        else:
+            picks += [(i, kind) for i in sorted({ids[0], max(ids, key=lambda i: wl.blocks[i].numel)})]
+    samples = []
+    for i, kind in picks:
+        b = wl.blocks[i]
+        whole = kind.startswith("F")
+        for lo, hi in ([(0, b.numel)] if whole else _slices(b.numel)):
+            n = hi - lo
+            rows, cols = (b.rows, b.cols) if whole else (n, 1)
+            samples.append(dict(i=i, kind=kind, lo=lo, hi=hi, rows=rows, cols=cols,
+                                th=sess.param_views[i][lo:hi].double().cpu().numpy(),
+                                st=O.step_init(cfgs[assign[i]], n, rows, cols)))
+    launches0 = sess.h.query().kernel_launches
+    for t in range(1, N_STEPS + 1):
+        k = sess.fill_grads(t)
+        sess.step(k, t)
+        for s in samples:
+            g = sess.grad_views[k][s["i"]][s["lo"]:s["hi"]].double().cpu().numpy()
+            s["th"] = O.step(s["th"], g, s["st"], cfgs[assign[s["i"]]], s["rows"], s["cols"])
+    torch.cuda.synchronize()
+    assert sess.h.query().kernel_launches - launches0 == N_STEPS * 5    # row/column reduce + combine, three instances
+    assert sess.h.nonfinite()[0] == 0
+    bad, total = 0, 0
+    rel = lambda x, y: float(np.max(np.abs(x - y)) / max(float(np.max(np.abs(y))), 1e-30))
+    for s in samples:
+        i, lo, hi, ref, kind = s["i"], s["lo"], s["hi"], s["st"], s["kind"]
+        name = (wl.blocks[i].name, kind, lo)
+        got = sess.param_views[i][lo:hi].double().cpu().numpy()
+        assert np.max(np.abs(got - s["th"])) <= 1e-6 * np.max(np.abs(s["th"])), name
+        view = lambda w, dt, a, b: sess.h.view_tensor(i, w, dt)[a:b]
+        f32 = lambda w, a, b: view(w, torch.float32, a, b).double().cpu().numpy()
+        bits = lambda w, a, b: view(w, torch.bfloat16, a, b).view(torch.int16).cpu().numpy().astype(np.int32)
+        want_bits = lambda x: torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().astype(np.int32)
+        q0, q1 = lo // 256, (hi + 255) // 256
+
+        def codes(w, dt, ref_q, a=lo, b=hi):
+            nonlocal bad, total
+            d = np.abs(view(w, dt, a, b).cpu().numpy().astype(np.int32) - ref_q.astype(np.int32))
+            assert d.max() <= 1, name
+            bad += int((d != 0).sum()); total += d.size
+
+        def patterns(w, ref_x, a=lo, b=hi):
+            nonlocal bad, total
+            d = np.abs(bits(w, a, b) - want_bits(ref_x))
+            assert d.max() <= 1, name
+            bad += int((d != 0).sum()); total += d.size
+
+        if kind == "A32":
+            assert rel(f32(10, lo, hi), ref.m) <= 1e-6 and rel(f32(11, lo, hi), ref.v) <= 1e-6, name
+        elif kind in ("R", "S"):
+            assert rel(f32(10, lo, hi), ref.v if kind == "R" else ref.m) <= 1e-6, name
+        elif kind == "F":
+            assert rel(f32(10, 0, s["rows"]), ref.r) <= 1e-6 and rel(f32(11, 0, s["cols"]), ref.c) <= 1e-6, name
+        elif kind == "F16":
+            patterns(10, ref.r, 0, s["rows"]); patterns(11, ref.c, 0, s["cols"])
+        elif kind == "F8":
+            codes(10, torch.uint8, ref.qr, 0, s["rows"]); codes(11, torch.uint8, ref.qc, 0, s["cols"])
+            assert rel(f32(12, 0, len(ref.ar)), ref.ar.astype(np.float64)) <= 1e-6, name
+            assert rel(f32(13, 0, len(ref.ac)), ref.ac.astype(np.float64)) <= 1e-6, name
+        elif kind == "A16":
+            patterns(10, ref.m); patterns(11, ref.v)
+        elif kind in ("R16", "S16"):
+            patterns(10, ref.v if kind == "R16" else ref.m)
+        elif kind == "A8":
+            codes(10, torch.int8, ref.qm); codes(11, torch.uint8, ref.qv)
+            assert rel(f32(12, q0, q1), ref.am.astype(np.float64)) <= 1e-6, name
+            assert rel(f32(13, q0, q1), ref.av.astype(np.float64)) <= 1e-6, name
+        elif kind in ("R8", "S8"):
+            codes(10, torch.uint8 if kind == "R8" else torch.int8, ref.qv if kind == "R8" else ref.qm)
+            assert rel(f32(11, q0, q1), (ref.av if kind == "R8" else ref.am).astype(np.float64)) <= 1e-6, name
+    assert total > 0 and bad <= 1e-4 * total, (bad, total)
