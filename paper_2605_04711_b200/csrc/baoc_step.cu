@@ -86,6 +86,28 @@ __device__ __forceinline__ void rowcol_reduce_piece(const void* src, const float
                 for (int j = 0; j < 8; ++j) { x[j] *= x[j]; s += x[j]; colacc[j] += x[j]; }
                 rowacc[k] = s;
             }
+        } else if (!kSquare && vec && valid == 8) {
+            // fp32 input (the window's second moments): the row segments are requested eight at a time
+            const float* p = static_cast<const float*>(src) + col0;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                float4 a[kRedRows / 8], b[kRedRows / 8];
+#pragma unroll
+                for (int k = 0; k < kRedRows / 8; ++k) {
+                    const int64_t r = r0 + ty + 4 * (h * (kRedRows / 8) + k);
+                    const bool in = r < rows;
+                    a[k] = in ? ld_stream_f4(p + r * cols) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    b[k] = in ? ld_stream_f4(p + r * cols + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int k = 0; k < kRedRows / 8; ++k) {
+                    const float x[8] = {a[k].x, a[k].y, a[k].z, a[k].w, b[k].x, b[k].y, b[k].z, b[k].w};
+                    float s = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { s += x[j]; colacc[j] += x[j]; }
+                    rowacc[h * (kRedRows / 8) + k] = s;
+                }
+            }
         } else {
 #pragma unroll
             for (int k = 0; k < kRedRows / 4; ++k) {
