@@ -334,15 +334,22 @@ int baoc_configure_from_window(baoc_t* h, const int32_t* assign, void* state_dev
 
 /* One training step of every block under its configuration.  grads / params:
  * host arrays of n_blocks device pointers (bf16 / fp32).  step_t: 1-based step
- * number (bias corrections).  Queues the fused update kernel (preceded by the
- * row/column reduction kernels when some block is factored); does not wait. */
+ * number (bias corrections).  Queues the fused update kernel, one launch per
+ * family of update paths in use (headline tuples; stateless and bf16-state
+ * tuples; 8-bit single-moment tuples), preceded by the row/column reduction
+ * kernels when some block is factored; does not wait. */
 int baoc_step(baoc_t* h, const void* const* grads, float* const* params,
               int64_t step_t, baoc_stream_t stream);
 
 /* End-to-end convenience for callers whose gradients live in host memory:
  * copies block i's bf16 gradient from host_grads[i] (pinned memory advised) to
  * the device buffer dev_grads[i], then does baoc_sample_stats (if do_stats)
- * and baoc_step (if step_t > 0) on the same stream.  Does not wait. */
+ * and baoc_step (if step_t > 0) on the same stream.  With do_stats the copy
+ * runs on an internal stream in up to eight groups of whole blocks, and each
+ * group takes its statistics step and its optimizer step as soon as it has
+ * landed, so that all but the last group's work hides behind the transfer;
+ * every block sees exactly the arithmetic of the separate calls.  Does not
+ * wait. */
 int baoc_step_from_host(baoc_t* h, const void* const* host_grads, void* const* dev_grads,
                         float* const* params, int do_stats, int64_t step_t,
                         baoc_stream_t stream);

@@ -179,6 +179,41 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
     return BAOC_OK;
 }
 
+// What do_step does before its launches: pointer tables, the step's scalars, cleared flags.
+int step_prologue(Handle* h, const void* const* grads, float* const* params, int64_t t, cudaStream_t s, StepParams* P) {
+    int rc = sync_pointer_table(h, grads, &h->last_step_grads, h->st + h->tl.grads, s, "baoc_step (grads)");
+    if (rc) return rc;
+    rc = sync_pointer_table(h, reinterpret_cast<const void* const*>(params), &h->last_step_params, h->st + h->tl.params, s,
+                            "baoc_step (params)");
+    if (rc) return rc;
+    fill_step_params(h, t, P);
+    CU(cudaMemsetAsync(h->st + h->tl.flags, 0, 4 * size_t(h->n_blocks), s), "baoc_step (flags)");
+    return BAOC_OK;
+}
+
+// The optimizer step of one copy group: its factored blocks' row/column kernels, then its tiles family by family.
+int step_group(Handle* h, const Handle::GroupStep& g, const StepParams& P, cudaStream_t s) {
+    const auto& L = h->tl;
+    if (g.n_f > 0) {
+        LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles) + g.red0,
+                                      at<int32_t>(h->st, L.f_ids) + g.f0, at<const void*>(h->st, L.grads),
+                                      at<const float*>(h->st, L.params), g.n_red, g.n_f, P, s),
+               "factored_reduce_kernel");
+        h->launches += 2;
+    }
+    int64_t first = g.tile0;
+    for (int fam = 0; fam < kFamCount; ++fam) {
+        if (g.fam_tiles[fam] == 0) continue;
+        LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles_by_group) + first,
+                                 at<const void*>(h->st, L.grads), at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags),
+                                 g.fam_tiles[fam], fam, P, s),
+               "fused_step_kernel");
+        h->launches += 1;
+        first += g.fam_tiles[fam];
+    }
+    return BAOC_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -419,6 +454,39 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
     }
     CU(cudaMemcpyAsync(st + L.blocks, sb.data(), sizeof(StepBlock) * n, cudaMemcpyHostToDevice, s), "upload step block table");
     CU(cudaMemcpyAsync(st + L.tiles, tiles.data(), sizeof(Tile) * tiles.size(), cudaMemcpyHostToDevice, s), "upload step tile table");
+    // the same tiles group by group (copy groups of the end-to-end call), within a group family by family in path order
+    std::vector<Handle::GroupStep> groups;
+    h->group_tiles.clear();
+    {
+        std::vector<int> gb0, gb1;
+        compute_copy_groups(h, &gb0, &gb1);
+        const int order[kPathCount] = {kPathA32, kPathR, kPathS, kPathA8, kPathF, kPathA16, kPathR16, kPathS16, kPathG, kPathR8, kPathS8};
+        int32_t f_seen = 0;
+        for (size_t g = 0; g < gb0.size(); ++g) {
+            Handle::GroupStep gs{};
+            gs.b0 = gb0[g]; gs.b1 = gb1[g];
+            gs.tile0 = int64_t(h->group_tiles.size());
+            for (int p : order)
+                for (int i = gs.b0; i < gs.b1; ++i)
+                    if (sb[i].path == p) {
+                        const int64_t nt = ceil_div(sb[i].numel, step_tile_elems(p));
+                        for (int64_t k = 0; k < nt; ++k) h->group_tiles.push_back(Tile{uint32_t(i), uint32_t(k)});
+                        gs.fam_tiles[family_of(p)] += nt;
+                    }
+            gs.red0 = -1; gs.f0 = f_seen;
+            for (int i = gs.b0; i < gs.b1; ++i)
+                if (sb[i].path == kPathF) {
+                    if (gs.red0 < 0) gs.red0 = sb[i].red.red0;
+                    gs.n_red += int64_t(sb[i].red.chunks) * sb[i].red.strips;
+                    gs.n_f += 1;
+                }
+            if (gs.red0 < 0) gs.red0 = 0;
+            f_seen += gs.n_f;
+            groups.push_back(gs);
+        }
+    }
+    CU(cudaMemcpyAsync(st + L.tiles_by_group, h->group_tiles.data(), sizeof(Tile) * h->group_tiles.size(), cudaMemcpyHostToDevice, s),
+       "upload step tile table (by group)");
     if (!red.empty())
         CU(cudaMemcpyAsync(st + L.red_tiles, red.data(), sizeof(RedTile) * red.size(), cudaMemcpyHostToDevice, s), "upload step reduction table");
     if (!ids.empty())
@@ -427,6 +495,7 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
     h->st = st; h->st_bytes = bytes; h->tl = L; h->configured = true;
     h->assign.assign(assign, assign + n);
     h->h_step_blocks = sb;
+    h->groups = groups;
     h->n_step_tiles = int64_t(tiles.size()); h->n_step_red_tiles = int64_t(red.size());
     h->n_factored = int(ids.size());
     for (int64_t& c : h->fam_tiles) c = 0;
@@ -804,24 +873,27 @@ int baoc_step_from_host(baoc_t* h, const void* const* host_grads, void* const* d
     // the copies must not overtake earlier work of the caller's stream that still reads the device gradients
     CU(cudaEventRecord(static_cast<cudaEvent_t>(h->copy_ev[Handle::kCopyGroups]), s), "baoc_step_from_host");
     CU(cudaStreamWaitEvent(cs, static_cast<cudaEvent_t>(h->copy_ev[Handle::kCopyGroups]), 0), "baoc_step_from_host");
-    const int64_t per_group = (h->numel + Handle::kCopyGroups - 1) / Handle::kCopyGroups;
-    int b0 = 0, g = 0;
-    while (b0 < h->n_blocks) {
-        int b1 = b0;
-        int64_t acc = 0;
-        while (b1 < h->n_blocks && (acc < per_group || g == Handle::kCopyGroups - 1)) acc += h->blocks[b1++].numel;
-        CU(copy_range(b0, b1, cs), "baoc_step_from_host (copy)");
+    // With an optimizer step as well, every group also takes its step as soon as its statistics are queued, so that
+    // only the last group's work is left when the transfer ends.  Each block sees exactly the launches of baoc_step.
+    std::vector<int> gb0, gb1;
+    compute_copy_groups(h, &gb0, &gb1);
+    StepParams P;
+    if (step_t > 0) {
+        rc = step_prologue(h, dg, params, step_t, s, &P);
+        if (rc) return rc;
+    }
+    for (size_t g = 0; g < gb0.size(); ++g) {
+        CU(copy_range(gb0[g], gb1[g], cs), "baoc_step_from_host (copy)");
         CU(cudaEventRecord(static_cast<cudaEvent_t>(h->copy_ev[g]), cs), "baoc_step_from_host");
         CU(cudaStreamWaitEvent(s, static_cast<cudaEvent_t>(h->copy_ev[g]), 0), "baoc_step_from_host");
-        rc = stats_step_range(h, b0, b1, s);
+        rc = stats_step_range(h, gb0[g], gb1[g], s);
         if (rc) return rc;
-        b0 = b1;
-        ++g;
+        if (step_t > 0) {
+            rc = step_group(h, h->groups[g], P, s);
+            if (rc) return rc;
+        }
     }
-    rc = stats_combine_all(h, s);
-    if (rc) return rc;
-    if (step_t > 0) return do_step(h, dg, params, step_t, s);
-    return BAOC_OK;
+    return stats_combine_all(h, s);
 }
 
 

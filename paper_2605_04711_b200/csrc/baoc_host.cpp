@@ -153,6 +153,20 @@ void compute_stat_layout(Handle* h) {
     L.total = cur;
 }
 
+void compute_copy_groups(const Handle* h, std::vector<int>* b0s, std::vector<int>* b1s) {
+    b0s->clear(); b1s->clear();
+    const int64_t per_group = ceil_div(h->numel, Handle::kCopyGroups);
+    int b0 = 0, g = 0;
+    while (b0 < h->n_blocks) {
+        int b1 = b0;
+        int64_t acc = 0;
+        while (b1 < h->n_blocks && (acc < per_group || g == Handle::kCopyGroups - 1)) acc += h->blocks[b1++].numel;
+        b0s->push_back(b0); b1s->push_back(b1);
+        b0 = b1;
+        ++g;
+    }
+}
+
 // Optimizer-state buffer of one assignment: tables, non-finite flags, the
 // scratch of the factored path and the states themselves.
 int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayout* out, std::vector<StepBlock>* blocks,
@@ -240,6 +254,7 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
     size_t cur = 0;
     out->blocks = take(&cur, sizeof(StepBlock) * n);
     out->tiles = take(&cur, sizeof(Tile) * tl.size());
+    out->tiles_by_group = take(&cur, sizeof(Tile) * tl.size());
     out->red_tiles = take(&cur, sizeof(RedTile) * std::max<size_t>(rt.size(), 1));
     out->f_ids = take(&cur, 4 * size_t(n));
     out->grads = take(&cur, 8 * size_t(n));

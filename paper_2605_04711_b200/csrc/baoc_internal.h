@@ -245,8 +245,20 @@ struct Handle {
     std::vector<const void*> last_step_grads;
     std::vector<const void*> last_step_params;
     struct StepLayout {
-        size_t blocks, tiles, red_tiles, f_ids, grads, params, flags, redpart, states, total;
+        size_t blocks, tiles, tiles_by_group, red_tiles, f_ids, grads, params, flags, redpart, states, total;
     } tl{};
+    // The end-to-end call copies the gradients in groups of whole blocks and lets each group take its statistics step
+    // and its optimizer step as soon as it has landed: a second tile table holds the step's tiles group by group
+    // (within a group family by family), and every group knows its stretches of the tables.
+    struct GroupStep {
+        int b0, b1;                      // blocks [b0, b1)
+        int64_t tile0;                   // first tile of the group in the by-group table
+        int64_t fam_tiles[kFamCount];    // its tiles per path family
+        int64_t red0, n_red;             // its stretch of the row/column reduction table
+        int32_t f0, n_f;                 // its stretch of the list of factored blocks
+    };
+    std::vector<GroupStep> groups;
+    std::vector<Tile> group_tiles;       // staging of the by-group table (must outlive the asynchronous upload)
 
     // optional per-kernel timing of the step (CUDA events, owned by the CUDA translation unit)
     bool prof_on = false, prof_valid = false;
@@ -292,6 +304,8 @@ int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const
 int launch_fused_step(const StepBlock* blocks, const Tile* tiles, const void* const* grads, float* const* params,
                       uint32_t* flags, int64_t n_tiles, int family, const StepParams& P, cudaStream_t s);
 int launch_convert_moment(const MomentRef& src, const MomentRef& dst, int64_t numel, cudaStream_t s);
+// Copy groups of the end-to-end call: up to Handle::kCopyGroups runs of whole blocks of about equal bytes.
+void compute_copy_groups(const Handle* h, std::vector<int>* b0, std::vector<int>* b1);
 int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayout* out,
                         std::vector<StepBlock>* blocks, std::vector<Tile>* tiles,
                         std::vector<RedTile>* red, int64_t* state_mem, int64_t* step_bytes);
