@@ -144,42 +144,7 @@ int build_slots(Handle* h, const int32_t* assign, std::vector<StepBlock>* sb) {
     return BAOC_OK;
 }
 
-int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t, cudaStream_t s) {
-    int rc = sync_pointer_table(h, grads, &h->last_step_grads, h->st + h->tl.grads, s, "baoc_step (grads)");
-    if (rc) return rc;
-    rc = sync_pointer_table(h, reinterpret_cast<const void* const*>(params), &h->last_step_params, h->st + h->tl.params, s,
-                            "baoc_step (params)");
-    if (rc) return rc;
-    StepParams P;
-    fill_step_params(h, t, &P);
-    const auto& L = h->tl;
-    CU(cudaMemsetAsync(h->st + L.flags, 0, 4 * size_t(h->n_blocks), s), "baoc_step (flags)");
-    if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[0]), s), "baoc_step (profile)");
-    if (h->n_factored > 0) {
-        LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles),
-                                      at<int32_t>(h->st, L.f_ids), at<const void*>(h->st, L.grads),
-                                      at<const float*>(h->st, L.params), h->n_step_red_tiles, h->n_factored, P, s),
-               "factored_reduce_kernel");
-        h->launches += 2;
-    }
-    if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[1]), s), "baoc_step (profile)");
-    int64_t first = 0;
-    for (int fam = 0; fam < kFamCount; ++fam) {                     // one launch per path family present
-        if (h->fam_tiles[fam] == 0) continue;
-        LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles) + first, at<const void*>(h->st, L.grads),
-                                 at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), h->fam_tiles[fam], fam, P, s),
-               "fused_step_kernel");
-        h->launches += 1;
-        first += h->fam_tiles[fam];
-    }
-    if (h->prof_on) {
-        CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[2]), s), "baoc_step (profile)");
-        h->prof_valid = true;
-    }
-    return BAOC_OK;
-}
-
-// What do_step does before its launches: pointer tables, the step's scalars, cleared flags.
+// What a step does before its launches: pointer tables, the step's scalars, cleared flags.
 int step_prologue(Handle* h, const void* const* grads, float* const* params, int64_t t, cudaStream_t s, StepParams* P) {
     int rc = sync_pointer_table(h, grads, &h->last_step_grads, h->st + h->tl.grads, s, "baoc_step (grads)");
     if (rc) return rc;
@@ -210,6 +175,37 @@ int step_group(Handle* h, const Handle::GroupStep& g, const StepParams& P, cudaS
                "fused_step_kernel");
         h->launches += 1;
         first += g.fam_tiles[fam];
+    }
+    return BAOC_OK;
+}
+
+// One step of every block: the whole tile table, one launch per path family present.
+int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t, cudaStream_t s) {
+    StepParams P;
+    int rc = step_prologue(h, grads, params, t, s, &P);
+    if (rc) return rc;
+    const auto& L = h->tl;
+    if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[0]), s), "baoc_step (profile)");
+    if (h->n_factored > 0) {
+        LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles),
+                                      at<int32_t>(h->st, L.f_ids), at<const void*>(h->st, L.grads),
+                                      at<const float*>(h->st, L.params), h->n_step_red_tiles, h->n_factored, P, s),
+               "factored_reduce_kernel");
+        h->launches += 2;
+    }
+    if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[1]), s), "baoc_step (profile)");
+    int64_t first = 0;
+    for (int fam = 0; fam < kFamCount; ++fam) {
+        if (h->fam_tiles[fam] == 0) continue;
+        LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles) + first, at<const void*>(h->st, L.grads),
+                                 at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), h->fam_tiles[fam], fam, P, s),
+               "fused_step_kernel");
+        h->launches += 1;
+        first += h->fam_tiles[fam];
+    }
+    if (h->prof_on) {
+        CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[2]), s), "baoc_step (profile)");
+        h->prof_valid = true;
     }
     return BAOC_OK;
 }
