@@ -267,8 +267,10 @@ def run_ours(args):
     from paper_2605_04711_b200 import binding
     extended = args.candidates == "extended" or args.assign in EXTENDED_NAMES[5:]
     names = EXTENDED_NAMES if extended else CONFIG_NAMES
+    # optional: the statistics see a seeded sub-grid of every block (the paper's sparse coordinate sampling)
+    samples = W.sample_subgrids(wl, args.sample_frac) if args.sample_frac < 1.0 else None
     sess = harness.Session(wl, configs=binding.extended_configs() if extended else None, n_grad_sets=2,
-                           device=f"cuda:{local}", pinned_host_grads=True)
+                           device=f"cuda:{local}", pinned_host_grads=True, samples=samples)
     sess.init_params()
     for t in (1, 2):
         k = sess.fill_grads(t)
@@ -386,9 +388,10 @@ def run_ours(args):
     fused_gbs = fused_bytes / (fused_ms * 1e-3) / 1e9
     r_stats = {"kernel": "stats_step_kernel", "bound": "hbm", "achieved": stats_gbs, "peak": peak, "unit": "GB/s",
                "frac": stats_gbs / peak, "peak_kind": peak_kind + " (burst copy)", "frac_of_8TBs": stats_gbs / 8000.0,
-               "bytes_per_launch": int(stats_bytes), "ms": stats_ms, "bytes_per_param": 22,
+               "bytes_per_launch": int(stats_bytes), "ms": stats_ms,
+               "bytes_per_param": 22 if samples is None else "26 per sampled coordinate",
                "timed": "events around baoc_sample_stats (includes its ~25 us combine kernel)",
-               "traffic": args.traffic_stats if args.traffic_stats is not None else _ncu_traffic("stats_step_kernel", stats_bytes)}
+               "traffic": args.traffic_stats if args.traffic_stats is not None else (_ncu_traffic("stats_step_kernel", stats_bytes) if samples is None else None)}
     r_fused = {"kernel": "fused_step_kernel", "bound": "hbm", "achieved": fused_gbs, "peak": peak, "unit": "GB/s",
                "frac": fused_gbs / peak, "peak_kind": peak_kind + " (burst copy)", "frac_of_8TBs": fused_gbs / 8000.0,
                "bytes_per_launch": int(fused_bytes), "ms": fused_ms,
@@ -405,7 +408,7 @@ def run_ours(args):
                    "param_dtype": "f32", "candidate_configs": names, "assignment": args.assign,
                    "assignment_blocks_per_config": counts, "assignment_params_per_config": params_by_cfg,
                    "mem_budget_frac_of_fp32_adam": wl.mem_budget_frac, "state_bytes": int(info.state_bytes),
-                   "window_steps_before_timing": args.window, "l2": "inputs (>10 GB per step) far exceed the 126 MB L2",
+                   "window_steps_before_timing": args.window, "stats_sample_frac": args.sample_frac, "l2": "inputs (>10 GB per step) far exceed the 126 MB L2",
                    "parallelism": (f"whole blocks sharded over {world} GPUs, no collective" if args.shard_blocks else
                                    f"replicas x{world}, no collective") if world > 1 else "single GPU",
                    "allocator_status": int(rc), "nonfinite_blocks": int(cnt)},
@@ -440,6 +443,9 @@ def main():
                     help="auto: the library's own budgeted allocation; else every block under that one configuration")
     ap.add_argument("--shard-blocks", action="store_true",
                     help="N > 1: deal whole blocks of ONE workload to the ranks (strong scaling) instead of one replica per rank")
+    ap.add_argument("--sample-frac", type=float, default=1.0,
+                    help="fraction of every block's coordinates the statistics see (1 = dense, the default; the paper's own "
+                         "default is 0.001)")
     ap.add_argument("--window", type=int, default=4, help="statistics steps before the finalize that feeds the allocation")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample-params", type=int, default=40_000_000)
