@@ -383,7 +383,7 @@ def run_ours(args):
     stats_gbs = stats_bytes / (stats_ms * 1e-3) / 1e9
     step_gbs = step_bytes / (step_ms * 1e-3) / 1e9
     # the dominant kernel of the step gets the `roofline` object, the other one `roofline_other`
-    n_factored = params_by_cfg[3]
+    n_factored = sum(n for n, c in zip(params_by_cfg, sess.configs) if c.factored)   # at any precision of their statistics
     fused_bytes = step_bytes - 2 * n_factored              # the row/column kernels read the factored blocks' gradients once
     fused_gbs = fused_bytes / (fused_ms * 1e-3) / 1e9
     r_stats = {"kernel": "stats_step_kernel", "bound": "hbm", "achieved": stats_gbs, "peak": peak, "unit": "GB/s",
