@@ -559,14 +559,33 @@ def test_measured_time_ratios_leave_parameters_and_state_alone(B, H):
     assert e.value.code == B.E_INVALID
 
 
-def test_step_from_host_equals_separate_calls_bit_for_bit(B, H):
-    """The end-to-end call (pinned host gradients, copy pipelined with the statistics pass in groups of blocks) leaves
-    exactly what baoc_sample_stats + baoc_step leave on device-resident gradients."""
+def _state_tensors(sess, B):
+    """Every optimizer-state tensor of every block, as raw bytes."""
+    out = []
+    for i in range(len(sess.wl.blocks)):
+        for which in (10, 11, 12, 13):
+            try:
+                ptr, n, eb = sess.h.view(i, which)
+            except B.BaocError:
+                continue
+            out.append(sess.h.view_tensor(i, which, {1: torch.uint8, 2: torch.int16, 4: torch.int32}[eb]).clone())
+    return out
+
+
+@pytest.mark.parametrize("extended", [False, True])
+def test_step_from_host_equals_separate_calls_bit_for_bit(B, H, extended):
+    """The end-to-end call (pinned host gradients; the copy runs in groups of blocks and every group takes its
+    statistics step and its optimizer step as soon as it has landed) leaves exactly what baoc_sample_stats + baoc_step
+    leave on device-resident gradients: parameters, window moments, running statistics and every state tensor.  With
+    the extended candidates every tuple occurs, so every group launches all three kernel instances."""
     wl = W.make_workload("resnet50", seed=3)
-    assign = [(i % 5) if not ((i % 5) == 3 and b.cols <= 1) else 1 for i, b in enumerate(wl.blocks)]
+    cfgs = B.extended_configs() if extended else None
+    k_cfg = 13 if extended else 5
+    vec = {3: 1, 11: 7, 12: 9}
+    assign = [(vec[i % k_cfg] if ((i % k_cfg) in vec and b.cols <= 1) else i % k_cfg) for i, b in enumerate(wl.blocks)]
     res = []
     for from_host in (False, True):
-        sess = H.Session(wl, n_grad_sets=2, pinned_host_grads=from_host)
+        sess = H.Session(wl, configs=cfgs, n_grad_sets=2, pinned_host_grads=from_host)
         sess.init_params()
         sess.configure(assign)
         for t in (1, 2, 3):
@@ -580,12 +599,17 @@ def test_step_from_host_equals_separate_calls_bit_for_bit(B, H):
                 sess.sample_stats(k)
                 sess.step(k, t)
         torch.cuda.synchronize()
-        res.append((sess.params.clone(), sess.ws.clone()[sess.h.view(0, 0)[0] - sess.ws.data_ptr():], sess.h.read_stats()))
+        res.append((sess.params.clone(), sess.ws.clone()[sess.h.view(0, 0)[0] - sess.ws.data_ptr():], sess.h.read_stats(),
+                    _state_tensors(sess, B), sess.h.nonfinite()[0]))
     assert torch.equal(res[0][0], res[1][0])
     n_m = sum((b.numel + 255) // 256 * 256 for b in wl.blocks) * 4
     assert torch.equal(res[0][1][:2 * n_m], res[1][1][:2 * n_m])      # both moment arrays
     for a, b2 in zip(res[0][2], res[1][2]):
         assert a["rho_bar"] == b2["rho_bar"] and a["last_cos"] == b2["last_cos"] and a["n_cos"] == b2["n_cos"] == 2
+    assert len(res[0][3]) == len(res[1][3]) > 0
+    for x, y in zip(res[0][3], res[1][3]):
+        assert torch.equal(x, y)
+    assert res[0][4] == res[1][4] == 0
 
 
 @pytest.mark.parametrize("variant", [0, 1])
