@@ -801,7 +801,12 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         const float am_new = kM ? warp_max_nonneg(am_c) : 0.f, av_new = kV ? warp_max_nonneg(av_c) : 0.f;
 
         // ---- codes: rne(q) = low byte of the float q + 1.5*2^23
-        const float km = am_new > 0.f ? 127.0f / am_new : 0.f, kv = av_new > 0.f ? 255.0f / av_new : 0.f;
+        // L / a' from the approximate reciprocal and one Newton step: within about one ulp (2^-23) of the quotient, so
+        // q = m' * (L / a') is off by at most L * 2^-23 = 3.0e-5 on that account, inside the 2^-14 of the window below
+        // (a subnormal a' flushes to an infinite scale; the non-finite distance then sends the lane to the exact side)
+        const float rm0 = rcp_approx(am_new), rv0 = rcp_approx(av_new);
+        const float km = am_new > 0.f ? 127.0f * (rm0 * fmaf(-am_new, rm0, 2.0f)) : 0.f;
+        const float kv = av_new > 0.f ? 255.0f * (rv0 * fmaf(-av_new, rv0, 2.0f)) : 0.f;
         const float hm = 0.5f - (Em * km + 6.103515625e-5f), hv = 0.5f - (Ev * kv + 6.103515625e-5f);
         const f32x2 KM = splat2(km), KV = splat2(kv), MAGIC = splat2(kMagic), MINUS1 = splat2(-1.0f);
         uint32_t cmw[8], cvw[8];
