@@ -126,14 +126,15 @@ __device__ __forceinline__ void rowcol_reduce_piece(const void* src, const float
 #pragma unroll
         for (int k = 0; k < kRedRows / 4; ++k) buf[ty + 4 * k][tx] = rowacc[k];
         __syncthreads();                                            // the buffer written two groups ago is free again by now
-        if (threadIdx.x < kRedRows) {
-            const int64_t r = r0 + threadIdx.x;
-            if (r < rows) {
-                double s = 0.0;
-#pragma unroll 8
-                for (int j = 0; j < 64; ++j) s += double(buf[threadIdx.x][j]);
-                geo.rowpart[size_t(strip) * rows + r] = s;
-            }
+        {   // four threads per row: 16 of the 64 per-thread sums each, then two exchanges (a fixed order)
+            const int row = threadIdx.x >> 2, part = threadIdx.x & 3;
+            double s = 0.0;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) s += double(buf[row][part * 16 + j]);
+            s += __shfl_xor_sync(0xffffffffu, s, 1);
+            s += __shfl_xor_sync(0xffffffffu, s, 2);
+            const int64_t r = r0 + row;
+            if (part == 0 && r < rows) geo.rowpart[size_t(strip) * rows + r] = s;
         }
     }
 #pragma unroll
@@ -149,7 +150,7 @@ __device__ __forceinline__ void rowcol_reduce_piece(const void* src, const float
 }
 
 // Gradient squares of the factored blocks of the step.
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 factored_reduce_kernel(const StepBlock* __restrict__ blocks, const RedTile* __restrict__ rtiles,
                        const void* const* __restrict__ grads, const float* const* __restrict__ params,
                        const __grid_constant__ StepParams SP) {
