@@ -423,7 +423,7 @@ def run_ours(args):
         "once_per_window": {"finalize_and_risk_ms": finalize_ms, "allocate_ms": alloc_ms, "objective": objective},
     }
     if world == 1 and not args.no_cpu_baseline:
-        _, cb = time_oracle(wl, assign, 2, 1, args.cpu_sample_params, sess.configs)
+        _, cb = time_oracle(wl, assign, 3, 1, args.cpu_sample_params, sess.configs)   # about 15 s of CPU work
         line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
     print(json.dumps(line), flush=True)
     if dist is not None:
@@ -448,7 +448,7 @@ def main():
                          "default is 0.001)")
     ap.add_argument("--window", type=int, default=4, help="statistics steps before the finalize that feeds the allocation")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-sample-params", type=int, default=40_000_000)
+    ap.add_argument("--cpu-sample-params", type=int, default=100_000_000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--traffic-stats", type=float, default=None, help="ncu DRAM bytes per launch of the statistics kernel, if known")
     ap.add_argument("--traffic-step", type=float, default=None)
