@@ -291,6 +291,64 @@ def test_precision_cosine_explicit_small_case():
     assert abs(O.precision_cosine(m, v, 8, o) - want) < 1e-12
 
 
+def test_precision_cosine_sixteen_bits_by_hand():
+    """Eq. 8 at b = 16 on four elements whose bfloat16 neighbours are written out as literals (8 significant bits:
+    a spacing of 2^-7 in [1, 2), 2^-9 in [1/4, 1/2), 2^-11 in [1/16, 1/8)), with two exact ties.  The value must
+    also tell apart the mistakes that leave a moment un-rounded."""
+    o = O.Opts(eps_adam=0.0, eps=0.0)
+    m = np.array([1.00390625, -0.3, 1.01171875, 3.0])      # 1 + 2^-8: tie, to the even 1.0;  1 + 3*2^-8: tie, to 1 + 2^-6
+    v = np.array([4.0, 0.1, 1.0078125, 2.0])               # 1 + 2^-7 is a bfloat16 already
+    m16 = np.array([1.0, -0.30078125, 1.015625, 3.0])      # 0.3 = 1.2 * 2^-2 -> (1 + 26/128) / 4
+    v16 = np.array([4.0, 0.10009765625, 1.0078125, 2.0])   # 0.1 = 1.6 * 2^-4 -> (1 + 77/128) / 16
+    u32, u16 = m / np.sqrt(v), m16 / np.sqrt(v16)
+    want = u32 @ u16 / (np.linalg.norm(u32) * np.linalg.norm(u16))
+    got = O.precision_cosine(m, v, 16, o)
+    assert abs(got - want) < 1e-14
+    assert want < 1.0 - 1e-7                                # the rounding is visible in the value
+    for mq, vq in ((m, v), (m16, v), (m, v16)):             # nothing rounded, only m, only v: all distinguishable
+        ub = mq / np.sqrt(vq)
+        wrong = u32 @ ub / (np.linalg.norm(u32) * np.linalg.norm(ub))
+        assert abs(got - wrong) > 1e-8
+
+
+def test_quant_rel_error_by_hand_at_eight_and_sixteen_bits():
+    """||x - Q_b(x)|| / ||x|| on one quantisation block of four, every code and rounded value written out."""
+    o = O.Opts(qblock=4)
+    # signed 8-bit, absmax 1: 127 x = 127, -63.5 (tie, to the even 64), 33.02, 0
+    x = np.array([1.0, -0.5, 0.26, 0.0])
+    xq = np.array([127.0, -64.0, 33.0, 0.0]) / 127.0
+    want = math.sqrt(float(np.sum((x - xq) ** 2))) / math.sqrt(1.0 + 0.25 + 0.26 ** 2)
+    got = O.quant_rel_error(x, 8, True, o)
+    assert want > 1e-3 and abs(got - want) < 1e-15
+    assert abs(got - math.sqrt(float(np.sum((x - xq) ** 2))) / float(np.linalg.norm(xq))) > 1e-7   # not divided by ||Q(x)||
+    # unsigned 8-bit, absmax 4: 255 v / 4 = 255, 63.75, 15.9375, 127.5 (tie, to the even 128)
+    v = np.array([4.0, 1.0, 0.25, 2.0])
+    vq = np.array([255.0, 64.0, 16.0, 128.0]) * 4.0 / 255.0
+    want_v = math.sqrt(float(np.sum((v - vq) ** 2))) / math.sqrt(16.0 + 1.0 + 0.0625 + 4.0)
+    assert want_v > 1e-3 and abs(O.quant_rel_error(v, 8, False, o) - want_v) < 1e-15
+    # 16 bits: the bfloat16 literals of the test above (signedness does not enter)
+    y = np.array([1.00390625, -0.3, 1.01171875, 0.1])
+    yq = np.array([1.0, -0.30078125, 1.015625, 0.10009765625])
+    want_y = math.sqrt(float(np.sum((y - yq) ** 2))) / math.sqrt(float(np.sum(y * y)))
+    for signed in (True, False):
+        assert abs(O.quant_rel_error(y, 16, signed, o) - want_y) < 1e-15
+    assert want_y > 1e-3
+    assert O.quant_rel_error(np.zeros(4), 8, True, o) == 0.0 and O.quant_rel_error(np.zeros(4), 16, True, o) == 0.0
+
+
+def test_stats_finalize_reports_the_pinned_diagnostics():
+    """The finalize record carries exactly the pinned functions' values (a wiring check: no swapped keys)."""
+    o = O.Opts(qblock=4, eps_adam=0.0)
+    st = O.stats_init(4)
+    st.m = np.array([1.00390625, -0.3, 1.01171875, 0.1])
+    st.v = np.array([4.0, 1.0, 0.25, 2.0])
+    raw = O.stats_finalize(st, np.ones(4), 4, 1, o)
+    assert raw["Q16"] == O.precision_cosine(st.m, st.v, 16, o) and raw["Q8"] == O.precision_cosine(st.m, st.v, 8, o)
+    assert raw["err_m8"] == O.quant_rel_error(st.m, 8, True, o) and raw["err_v8"] == O.quant_rel_error(st.v, 8, False, o)
+    assert raw["err_m16"] == O.quant_rel_error(st.m, 16, True, o) and raw["err_v16"] == O.quant_rel_error(st.v, 16, False, o)
+    assert len({raw["err_m8"], raw["err_v8"], raw["err_m16"], raw["err_v16"]}) == 4
+
+
 # ---------------------------------------------------------------- P6 normalisation (Eq. 10-20)
 
 def _raw(**kw):
