@@ -443,7 +443,14 @@ int baoc_profile_last(baoc_t* h, float* ms2);
  *
  * The first call on each device looks up the device address of the built-in
  * scratch (cudaGetSymbolAddress, with that device current) and keeps it; make
- * that first call before any stream capture begins.  Every call on a device
+ * that first call before any stream capture begins.  Make it at start-up, as a
+ * warm-up on a small block, while allocation is still allowed: the CUDA runtime
+ * may load the library's device code lazily, so the first call is also the one
+ * that places the scratch array and the two kernels on the device (it can fail
+ * with BAOC_E_CUDA when memory is already exhausted); from the second call on a
+ * device nothing is loaded or placed any more.  The address that is kept does
+ * not survive cudaDeviceReset: a process that resets a device must not call
+ * this function on it afterwards.  Every call on a device
  * shares the one scratch array, which keeps the previous call's contents:
  * nothing in it needs clearing, because each call overwrites every slot it
  * later reads, but two calls that overlap on the GPU (different streams, or

@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libbaoc.so")
-SOURCES = ["baoc_host.cpp", "baoc_partition.cpp", "baoc_api.cu", "baoc_stats.cu", "baoc_step.cu", "baoc_noalloc.cu",
+SOURCES = ["baoc_host.cpp", "baoc_partition.cpp", "baoc_api.cu", "baoc_stats.cu", "baoc_finalize.cu", "baoc_step.cu", "baoc_noalloc.cu",
            "baoc_convert.cu"]
 HEADERS = [os.path.join(ROOT, "include", "baoc.h"), os.path.join(CSRC, "baoc_internal.h"),
            os.path.join(CSRC, "baoc_device.cuh")]

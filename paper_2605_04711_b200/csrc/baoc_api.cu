@@ -336,22 +336,19 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
         LAUNCH(launch_sample_gather(blocks, tiles, at<const void*>(ws, L.params), h->n_stat_tiles, 1, s), "sample_gather_kernel");
         h->launches += 1;
     }
-    LAUNCH(launch_final_sums(blocks, tiles, dparams, at<double>(ws, L.fin), at<double>(ws, L.fin_out), h->n_stat_tiles, n,
-                             h->opts.eps, float(h->opts.eps_adam), s), "stats_final_sums_kernel");
-    h->launches += 2;
+    LAUNCH(launch_final_sums(blocks, tiles, dparams, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<uint32_t>(ws, L.hist),
+                             at<RankSel>(ws, L.sel), h->n_stat_tiles, n, h->opts.eps, float(h->opts.eps_adam), s),
+           "final_sums_kernel");
+    h->launches += 5;
     if (h->n_matrix > 0) {
         LAUNCH(launch_moment_reduce(blocks, at<RedTile>(ws, L.red_tiles), at<int32_t>(ws, L.matrix_ids), h->n_red_tiles,
                                     h->n_matrix, s), "moment_reduce_kernel");
-        h->launches += 2;
+        h->launches += 3;
     }
-    LAUNCH(launch_final_resid(blocks, tiles, dparams, at<double>(ws, L.fin), at<double>(ws, L.fin_out), h->n_stat_tiles, n,
-                              h->opts.eps, s), "stats_final_resid_kernel");
-    h->launches += 2;
-    LAUNCH(launch_select(blocks, tiles, at<RankSel>(ws, L.sel), at<uint32_t>(ws, L.hist), h->n_stat_tiles, n, s),
-           "select kernels");
-    h->launches += 9;
-    LAUNCH(launch_gather(at<RankSel>(ws, L.sel), at<double>(ws, L.acc), at<double>(ws, L.fin_out), n, s), "stats_gather_kernel");
-    h->launches += 1;
+    LAUNCH(launch_final_resid_select(blocks, tiles, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<RankSel>(ws, L.sel),
+                                     at<uint32_t>(ws, L.hist), at<double>(ws, L.acc), h->n_stat_tiles, n, s),
+           "final_hist_kernel");
+    h->launches += 6;
 
     std::vector<double> out(size_t(kFinOut) * n);
     CU(cudaMemcpyAsync(out.data(), ws + L.fin_out, 8 * out.size(), cudaMemcpyDeviceToHost, s), "baoc_risk (copy back)");
@@ -377,15 +374,20 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
         for (int k = 0; k < 2; ++k) {
             const double pos = qs[k] * double(b.numel - 1);
             const double frac = pos - std::floor(pos);
-            const double lo = o[16 + 2 * k], hi = o[16 + 2 * k + 1];
+            const double lo = o[kFinRanks + 2 * k], hi = o[kFinRanks + 2 * k + 1];
             qv[k] = lo + frac * (hi - lo);
         }
         z.q10 = qv[0]; z.q90 = qv[1];
         z.A = std::log((qv[1] + eps) / (qv[0] + eps));
-        z.rho_bar = o[20]; z.n_cos = int64_t(o[21]); z.last_cos = o[23]; z.rho_mom = o[24];
+        z.rho_bar = o[kFinAcc]; z.n_cos = int64_t(o[kFinAcc + 1]); z.last_cos = o[kFinAcc + 3]; z.rho_mom = o[kFinAcc + 4];
         z.snr = o[0] / (o[1] + eps);                                        // Eq. 5 right
-        z.C = std::sqrt(o[14]) / (std::sqrt(o[4]) + eps);                   // Eq. 6
-        z.F = b.cols > 1 ? std::sqrt(o[15]) / (std::sqrt(o[2]) + eps) : 1.0;   // Eq. 7
+        {   // Eq. 6 from the sums of the deviations d = p - p0 from the pilot value: with delta = pbar - p0,
+            // sum ((p / pbar - 1) theta)^2 = (sum d^2 theta^2 - 2 delta sum d theta^2 + delta^2 sum theta^2) / pbar^2
+            const double delta = o[3] / double(b.numel), pbar = o[kFinPilot] + delta;
+            const double num2 = std::max(0.0, o[15] - 2.0 * delta * o[14] + delta * delta * o[4]);
+            z.C = pbar > 0.0 ? (std::sqrt(num2) / pbar) / (std::sqrt(o[4]) + eps) : 0.0;
+        }
+        z.F = b.cols > 1 ? std::sqrt(o[kFinResid]) / (std::sqrt(o[2]) + eps) : 1.0;   // Eq. 7
         z.Q32 = cosine(o[5], o[5], o[5]);                                   // Eq. 8
         z.Q16 = cosine(o[9], o[5], o[8]);
         z.Q8 = cosine(o[7], o[5], o[6]);
@@ -866,28 +868,40 @@ int baoc_step_from_host(baoc_t* h, const void* const* host_grads, void* const* d
     cudaStream_t cs = static_cast<cudaStream_t>(h->copy_stream);
     int rc = sync_pointer_table(h, dg, &h->last_stat_grads, h->ws + h->sl.grads, s, "baoc_step_from_host");
     if (rc) return rc;
-    // the copies must not overtake earlier work of the caller's stream that still reads the device gradients
-    CU(cudaEventRecord(static_cast<cudaEvent_t>(h->copy_ev[Handle::kCopyGroups]), s), "baoc_step_from_host");
-    CU(cudaStreamWaitEvent(cs, static_cast<cudaEvent_t>(h->copy_ev[Handle::kCopyGroups]), 0), "baoc_step_from_host");
+    // Everything that can fail on the host alone comes before the copy stream is forked from the caller's stream.
     // With an optimizer step as well, every group also takes its step as soon as its statistics are queued, so that
     // only the last group's work is left when the transfer ends.  Each block sees exactly the launches of baoc_step.
     std::vector<int> gb0, gb1;
     compute_copy_groups(h, &gb0, &gb1);
+    if (gb0.size() > size_t(Handle::kCopyGroups)) return fail(h, BAOC_E_INVALID, "baoc_step_from_host: more copy groups than events");
+    if (step_t > 0) {                                       // the by-group tile table was laid out for these very groups
+        bool same = h->groups.size() == gb0.size();
+        for (size_t g = 0; same && g < gb0.size(); ++g) same = h->groups[g].b0 == gb0[g] && h->groups[g].b1 == gb1[g];
+        if (!same) return fail(h, BAOC_E_STATE, "baoc_step_from_host: the configured state was laid out for other copy groups");
+    }
     StepParams P;
     if (step_t > 0) {
         rc = step_prologue(h, dg, params, step_t, s, &P);
         if (rc) return rc;
     }
+    // the copies must not overtake earlier work of the caller's stream that still reads the device gradients
+    CU(cudaEventRecord(static_cast<cudaEvent_t>(h->copy_ev[Handle::kCopyGroups]), s), "baoc_step_from_host");
+    CU(cudaStreamWaitEvent(cs, static_cast<cudaEvent_t>(h->copy_ev[Handle::kCopyGroups]), 0), "baoc_step_from_host");
+    // From here on the copy stream runs ahead of the caller's stream.  Whatever goes wrong, the caller's stream is
+    // joined to the copies already queued before the call returns, so that a retry or any later work on that stream
+    // cannot race with a transfer still in flight.
+    auto join = [&]() {
+        if (cudaEventRecord(static_cast<cudaEvent_t>(h->copy_ev[Handle::kCopyGroups]), cs) == cudaSuccess)
+            cudaStreamWaitEvent(s, static_cast<cudaEvent_t>(h->copy_ev[Handle::kCopyGroups]), 0);
+    };
     for (size_t g = 0; g < gb0.size(); ++g) {
-        CU(copy_range(gb0[g], gb1[g], cs), "baoc_step_from_host (copy)");
-        CU(cudaEventRecord(static_cast<cudaEvent_t>(h->copy_ev[g]), cs), "baoc_step_from_host");
-        CU(cudaStreamWaitEvent(s, static_cast<cudaEvent_t>(h->copy_ev[g]), 0), "baoc_step_from_host");
+        cudaError_t e = copy_range(gb0[g], gb1[g], cs);
+        if (e == cudaSuccess) e = cudaEventRecord(static_cast<cudaEvent_t>(h->copy_ev[g]), cs);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s, static_cast<cudaEvent_t>(h->copy_ev[g]), 0);
+        if (e != cudaSuccess) { join(); return cuda_fail(h, "baoc_step_from_host (copy)", e); }
         rc = stats_step_range(h, gb0[g], gb1[g], s);
-        if (rc) return rc;
-        if (step_t > 0) {
-            rc = step_group(h, h->groups[g], P, s);
-            if (rc) return rc;
-        }
+        if (rc == BAOC_OK && step_t > 0) rc = step_group(h, h->groups[g], P, s);
+        if (rc) { join(); return rc; }
     }
     return stats_combine_all(h, s);
 }

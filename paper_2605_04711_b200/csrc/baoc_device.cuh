@@ -85,6 +85,11 @@ __device__ __forceinline__ void unpack8(const uint4& w, float (&x)[8]) {
     x[4] = bf16_lo(w.z); x[5] = bf16_hi(w.z); x[6] = bf16_lo(w.w); x[7] = bf16_hi(w.w);
 }
 
+// Two float4 as an array of eight floats.
+__device__ __forceinline__ void f4_to8(const float4& a, const float4& b, float (&x)[8]) {
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+
 // A float that holds a bf16 value, widened to double without a conversion
 // instruction (the conversion pipe is narrow): re-bias the exponent with
 // integer arithmetic.  Zeros, subnormals, infinities and NaNs take the
@@ -132,6 +137,21 @@ __device__ __forceinline__ void cta_reduce_store(double (&val)[K], double* out) 
         out[threadIdx.x] = s;
     }
     __syncthreads();
+}
+
+// Sum K doubles per tile slot over the tiles of one block in a fixed order: thread
+// t takes tiles t, t+T, ..., then the CTA reduces.  out[K] per block.
+template <int K>
+__device__ __forceinline__ void block_tiles_sum(const double* __restrict__ part, int64_t tile0, int ntiles, double* out) {
+    double acc[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) acc[k] = 0.0;
+    for (int i = threadIdx.x; i < ntiles; i += kThreads) {
+        const double* p = part + size_t(tile0 + i) * K;
+#pragma unroll
+        for (int k = 0; k < K; ++k) acc[k] += p[k];
+    }
+    cta_reduce_store<K>(acc, out);
 }
 
 __device__ __forceinline__ float warp_max(float x) {

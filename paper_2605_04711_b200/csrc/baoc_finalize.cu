@@ -1,0 +1,550 @@
+// End-of-window finalize of the sampling window (Sec. 3.3): the sums behind the
+// signal-to-noise ratio (Eq. 5), the distortion (Eq. 6), the structure residual
+// (Eq. 7) and the precision cosines (Eq. 8), and the exact quantiles behind the
+// anisotropy (Eq. 4).  Three sweeps over the window's moments:
+//   1. final_sums_kernel   reads m, v, theta: 16 sums per block, and the histogram of the top byte of v
+//   2. final_hist_kernel<true>   reads v: Eq. 7 residual (after the row/column sums), histogram of the next 12 bits
+//   3. final_hist_kernel<false>  reads v: histogram of the last 12 bits
+// A CTA works through a run of consecutive tiles, keeps its partial sums and
+// histograms on chip while the tiles belong to one block, and hands them over
+// once per block (a deterministic, fixed partition of the work).
+#include "baoc_device.cuh"
+
+namespace baoc {
+
+// ============================================================================
+// Pilot value of the preconditioner p = 1/(sqrt(v)+eps) of Eq. 6: the mean of p
+// over up to 1024 evenly spaced elements of the block.  Eq. 6 needs
+// sum ((p/pbar - 1) theta)^2, which a single sweep can only form from sums that
+// do not involve pbar; sums of the deviations p - p0 from a pilot value close
+// to pbar do that without cancellation (p0 = pbar would be exact), and for a
+// block whose p are all equal p0 is exactly that value and every deviation 0.
+// ============================================================================
+__device__ __forceinline__ float precond_of(float v, float eps) { return rcp_approx(sqrt_approx(v) + eps); }
+
+__global__ void __launch_bounds__(kThreads)
+final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, double* __restrict__ fin_out) {
+    __shared__ double total[1];
+    const StatBlock* b = blocks + blockIdx.x;
+    const int64_t numel = b->numel;
+    const int64_t n = min64(numel, 1024);
+    const int64_t stride = numel / n;
+    double acc[1] = {0.0};
+    for (int64_t k = threadIdx.x; k < n; k += kThreads) acc[0] += double(precond_of(b->v[k * stride], eps));
+    cta_reduce_store<1>(acc, total);
+    // n identical fp32 values sum exactly in double, and the correctly rounded quotient is that value again
+    if (threadIdx.x == 0) fin_out[size_t(blockIdx.x) * kFinOut + kFinPilot] = double(float(total[0] / double(n)));
+}
+
+// ============================================================================
+// Sweep 1.  Per block, 16 sums over the window's moments (fp32), the parameters
+// and the quantised moments:
+//   0 sum m^2      1 sum v        2 sum v^2       3 sum (p - p0)
+//   4 sum theta^2  5 sum u32^2    6 sum u8^2      7 sum u32*u8
+//   8 sum u16^2    9 sum u32*u16  10 sum (m-m8)^2 11 sum (v-v8)^2
+//   12 sum (m-m16)^2              13 sum (v-v16)^2
+//   14 sum (p - p0) theta^2       15 sum (p - p0)^2 theta^2
+// with u = m/(sqrt(v)+eps_adam) from full-precision, 8-bit and bf16 moments and
+// p0 the block's pilot value.  A warp owns one 256-element quantisation block per
+// slice, so the absmax is a warp reduction.
+//
+// Everything is evaluated in fp32, two elements per instruction: the sums are
+// compared at 1e-4, far above fp32 rounding, and a code that lands on the other
+// side of a rounding tie moves a cosine by less than 1e-8.  Square roots and
+// reciprocals are the approximate ones (2^-23).  The bf16 round trip is a
+// Veltkamp split (x*(2^16+1) - (x*(2^16+1) - x) keeps the upper 8 significant
+// bits, rounded to nearest), which runs on the FMA pipe instead of the narrow
+// conversion pipe.  A thread keeps its partial sums in fp32 for at most
+// kFinRunTiles tiles (128 elements per thread) and widens them to double for the
+// reduction across the CTA.
+//
+// The slices are staged through shared memory by per-thread cp.async copies two
+// slices ahead (96 bytes per thread and slice: m, v, theta), so loads in flight
+// hold no registers during the long arithmetic of the current slice.
+// ============================================================================
+constexpr int kFsStageBytes = kThreads * 96;                 // m 32 B/thread at 0, v at 8192, theta at 16384
+constexpr int kFsStages = 3;
+constexpr int kHistCopies = 8;                               // replicas of the top-byte histogram (one per lane & 7)
+constexpr int kFsSmemBytes = kFsStages * kFsStageBytes + kHistCopies * 256 * 4;
+
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { return fma2(b, splat2(-1.0f), a); }
+
+__global__ void __launch_bounds__(kThreads, 2)
+final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
+                  const float* const* __restrict__ params, double* __restrict__ fin,
+                  const double* __restrict__ fin_out, uint32_t* __restrict__ hist, int64_t n_tiles,
+                  int tiles_per_cta, float eps_f, float eps_adam) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    unsigned char* stage = dyn;
+    uint32_t (*sh)[256] = reinterpret_cast<uint32_t (*)[256]>(dyn + kFsStages * kFsStageBytes);
+    constexpr float kMagic = 12582912.0f;                    // 1.5 * 2^23: adding it rounds to an integer, ties to even
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int copy = threadIdx.x & (kHistCopies - 1);
+    const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
+    const int nsl = int(last - first) * (kTile / (kThreads * 8));     // slices of this CTA
+    const uint32_t sm0 = smem_addr(stage);
+    const uint32_t om = threadIdx.x * 32, ov = 8192 + threadIdx.x * 32, ot = 16384 + threadIdx.x * 32;
+
+    for (int i = threadIdx.x; i < kHistCopies * 256; i += kThreads) (&sh[0][0])[i] = 0u;
+    __syncthreads();
+
+    f32x2 F[kFinalSums];
+#pragma unroll
+    for (int k = 0; k < kFinalSums; ++k) F[k] = pack2(0.f, 0.f);
+
+    // hand the finished run of tiles [t_begin, t_end) of block blk over: its sums go to the slot of its first tile
+    // (zeros to the others, the per-block combine adds all slots), its histogram to the block's global one
+    auto flush = [&](int blk, int64_t t_begin, int64_t t_end) {
+        double acc[kFinalSums];
+#pragma unroll
+        for (int k = 0; k < kFinalSums; ++k) {
+            float lo, hi;
+            unpack2(F[k], lo, hi);
+            acc[k] = double(lo) + double(hi);
+            F[k] = pack2(0.f, 0.f);
+        }
+        cta_reduce_store<kFinalSums>(acc, fin + size_t(t_begin) * kFinalSums);
+        double* rest = fin + size_t(t_begin + 1) * kFinalSums;
+        for (int64_t i = threadIdx.x; i < (t_end - t_begin - 1) * kFinalSums; i += kThreads) rest[i] = 0.0;
+        uint32_t* out = hist + size_t(blk) * kRanks * kSelBins;
+        for (int d = threadIdx.x; d < 256; d += kThreads) {
+            uint32_t cnt = 0u;
+#pragma unroll
+            for (int c = 0; c < kHistCopies; ++c) { cnt += sh[c][d]; sh[c][d] = 0u; }
+            if (cnt) atomicAdd(out + d, cnt);
+        }
+        __syncthreads();
+    };
+
+    uint32_t fill = 0, take = 0;
+    auto prefetch = [&](int k) {
+        if (k < nsl) {
+            const Tile t = tiles[first + (k >> 1)];
+            const StatBlock* b = blocks + t.block;
+            const int64_t numel = b->numel;
+            const int64_t e = int64_t(t.piece) * kTile + int64_t(k & 1) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+            // m and v are padded with zeros to whole quantisation blocks: in bounds whenever the warp's block starts
+            // inside the array; theta is not padded
+            if (e - lane * 8 < numel) {
+                const uint32_t d = sm0 + fill;
+                cp_async16(d + om, b->m + e); cp_async16(d + om + 16, b->m + e + 4);
+                cp_async16(d + ov, b->v + e); cp_async16(d + ov + 16, b->v + e + 4);
+                if (e + 8 <= numel) {
+                    const float* th = params[t.block];
+                    cp_async16(d + ot, th + e); cp_async16(d + ot + 16, th + e + 4);
+                }
+            }
+        }
+        cp_async_commit();
+        fill = fill == (kFsStages - 1) * kFsStageBytes ? 0u : fill + kFsStageBytes;
+    };
+#pragma unroll
+    for (int k = 0; k < kFsStages - 1; ++k) prefetch(k);
+
+    int cur_block = -1;
+    int64_t run_first = first;
+    float p0 = 0.f;
+    const f32x2 MAGIC = splat2(kMagic), NMAGIC = splat2(-kMagic), C16 = splat2(65537.0f), EA = splat2(eps_adam),
+                EPS = splat2(eps_f);
+#pragma unroll 1
+    for (int k = 0; k < nsl; ++k) {
+        prefetch(k + kFsStages - 1);
+        cp_async_wait<kFsStages - 1>();                      // this slice's copies have landed
+        const int64_t ti = first + (k >> 1);
+        const Tile t = tiles[ti];
+        if (int(t.block) != cur_block) {                     // uniform over the CTA; only at a tile boundary
+            if (cur_block >= 0) flush(cur_block, run_first, ti);
+            cur_block = int(t.block);
+            run_first = ti;
+            p0 = float(fin_out[size_t(t.block) * kFinOut + kFinPilot]);
+        }
+        const unsigned char* mine = stage + take;
+        take = take == (kFsStages - 1) * kFsStageBytes ? 0u : take + kFsStageBytes;
+        const StatBlock* b = blocks + t.block;
+        const int64_t numel = b->numel;
+        const int64_t w0 = int64_t(t.piece) * kTile + int64_t(k & 1) * (kThreads * 8) + int64_t(warp) * kQBlock;
+        if (w0 >= numel) continue;                           // whole warp out of range
+        const int64_t e = w0 + lane * 8;
+        const int cnt = int(max64(0, min64(8, numel - e)));
+        float mm[8], vv[8], tt[8];
+        f4_to8(*reinterpret_cast<const float4*>(mine + om), *reinterpret_cast<const float4*>(mine + om + 16), mm);
+        f4_to8(*reinterpret_cast<const float4*>(mine + ov), *reinterpret_cast<const float4*>(mine + ov + 16), vv);
+        if (cnt == 8) {
+            f4_to8(*reinterpret_cast<const float4*>(mine + ot), *reinterpret_cast<const float4*>(mine + ot + 16), tt);
+        } else {
+            const float* th = params[t.block];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) tt[j] = j < cnt ? th[e + j] : 0.f;
+        }
+
+        // ---- absmax of the warp's quantisation block, code scales
+        float am = 0.f, av = 0.f;
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            am = max3(am, fabsf(mm[2 * p]), fabsf(mm[2 * p + 1]));
+            av = max3(av, vv[2 * p], vv[2 * p + 1]);
+        }
+        am = warp_max_nonneg(am); av = warp_max_nonneg(av);
+        const float rm0 = rcp_approx(am), rv0 = rcp_approx(av);      // L / a from the reciprocal and one Newton step
+        const f32x2 KM = splat2(am > 0.f ? 127.0f * (rm0 * fmaf(-am, rm0, 2.0f)) : 0.f);
+        const f32x2 KV = splat2(av > 0.f ? 255.0f * (rv0 * fmaf(-av, rv0, 2.0f)) : 0.f);
+        // a / L in two parts (the second one the exact remainder of the first, divided by L), so that code * a / L comes
+        // out correctly rounded and the block's largest element, whose code is L, is reproduced exactly
+        const float dmh = am * (1.0f / 127.0f), dvh = av * (1.0f / 255.0f);
+        const f32x2 DM = splat2(dmh), DV = splat2(dvh);
+        const f32x2 DML = splat2(fmaf(-127.0f, dmh, am) * (1.0f / 127.0f)), DVL = splat2(fmaf(-255.0f, dvh, av) * (1.0f / 255.0f));
+
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const f32x2 M = pack2(mm[2 * p], mm[2 * p + 1]), V = pack2(vv[2 * p], vv[2 * p + 1]);
+            const f32x2 T = pack2(tt[2 * p], tt[2 * p + 1]);
+            // 8-bit round trips: code = rne(x L / a) by the magic-number addition, value = code a / L
+            const f32x2 QM = add2(fma2(M, KM, MAGIC), NMAGIC), QV = add2(fma2(V, KV, MAGIC), NMAGIC);
+            const f32x2 M8 = fma2(QM, DM, mul2(QM, DML)), V8 = fma2(QV, DV, mul2(QV, DVL));
+            // bf16 round trips
+            const f32x2 CM = mul2(M, C16), CV = mul2(V, C16);
+            const f32x2 M16 = sub2(CM, sub2(CM, M)), V16 = sub2(CV, sub2(CV, V));
+            // directions and the preconditioner (padding: m = v = 0 gives zeros everywhere but in p, which is masked)
+            float a0, a1, b0, b1, c0, c1;
+            const f32x2 S = pack2(sqrt_approx(vv[2 * p]), sqrt_approx(vv[2 * p + 1]));
+            unpack2(add2(S, EA), a0, a1);
+            const f32x2 U32 = mul2(M, pack2(rcp_approx(a0), rcp_approx(a1)));
+            unpack2(add2(S, EPS), a0, a1);
+            const f32x2 PD = pack2(2 * p < cnt ? rcp_approx(a0) - p0 : 0.f, 2 * p + 1 < cnt ? rcp_approx(a1) - p0 : 0.f);
+            unpack2(V8, b0, b1);
+            unpack2(add2(pack2(sqrt_approx(b0), sqrt_approx(b1)), EA), b0, b1);
+            const f32x2 U8 = mul2(M8, pack2(rcp_approx(b0), rcp_approx(b1)));
+            unpack2(V16, c0, c1);
+            unpack2(add2(pack2(sqrt_approx(c0), sqrt_approx(c1)), EA), c0, c1);
+            const f32x2 U16 = mul2(M16, pack2(rcp_approx(c0), rcp_approx(c1)));
+            // the sums
+            F[0] = fma2(M, M, F[0]); F[1] = add2(F[1], V); F[2] = fma2(V, V, F[2]); F[3] = add2(F[3], PD);
+            const f32x2 T2 = mul2(T, T), PT = mul2(PD, T2);
+            F[4] = add2(F[4], T2); F[14] = add2(F[14], PT); F[15] = fma2(PD, PT, F[15]);
+            F[5] = fma2(U32, U32, F[5]); F[6] = fma2(U8, U8, F[6]); F[7] = fma2(U32, U8, F[7]);
+            F[8] = fma2(U16, U16, F[8]); F[9] = fma2(U32, U16, F[9]);
+            const f32x2 E0 = sub2(M, M8), E1 = sub2(V, V8), E2 = sub2(M, M16), E3 = sub2(V, V16);
+            F[10] = fma2(E0, E0, F[10]); F[11] = fma2(E1, E1, F[11]); F[12] = fma2(E2, E2, F[12]); F[13] = fma2(E3, E3, F[13]);
+        }
+
+        // ---- first radix pass of the quantile select: the top byte of v's bit pattern (sign and upper exponent bits).
+        // Nearly all elements of a block share it, so a thread adds runs of equal bytes, into one of eight replicas.
+        {
+            int cur = -1;
+            uint32_t n = 0u;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (j < cnt) {
+                    const int d = int(__float_as_uint(vv[j]) >> 24);
+                    if (d == cur) {
+                        ++n;
+                    } else {
+                        if (n) atomicAdd(&sh[copy][cur], n);
+                        cur = d; n = 1u;
+                    }
+                }
+            }
+            if (n) atomicAdd(&sh[copy][cur], n);
+        }
+    }
+    cp_async_wait<0>();
+    if (cur_block >= 0) flush(cur_block, run_first, last);
+}
+
+// Per-block combines of the sweeps: the sums over the block's tile slots, in tile order.
+__global__ void __launch_bounds__(kThreads)
+final_sums_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ fin, double* __restrict__ fin_out) {
+    const StatBlock* b = blocks + blockIdx.x;
+    block_tiles_sum<kFinalSums>(fin, b->tile0, b->ntiles, fin_out + size_t(blockIdx.x) * kFinOut);
+}
+
+__global__ void __launch_bounds__(kThreads)
+final_resid_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ fin, double* __restrict__ fin_out) {
+    const StatBlock* b = blocks + blockIdx.x;
+    block_tiles_sum<kResidSums>(fin, b->tile0, b->ntiles, fin_out + size_t(blockIdx.x) * kFinOut + kFinResid);
+}
+
+// ============================================================================
+// Sweeps 2 and 3: radix passes of the exact quantile select over the fp32 bit
+// patterns of v (v >= 0, so the unsigned order of the patterns is the numeric
+// order): four ranks per block (the two order statistics around each of the two
+// quantile positions); ranks that still share a prefix share one histogram (the
+// "leader" rank's).  A pass looks at the 12 bits [shift, shift + 12) of the
+// elements whose higher bits equal the prefix found so far.
+// kResid: the same sweep also forms the Eq. 7 numerator
+//   sum (S_ij - a_i b_j / mu)^2 = sum (v_ij - rowsum_i colsum_j / total)^2
+// of matrix blocks, in double (a difference of nearly equal numbers).
+// ============================================================================
+template <bool kResid>
+__global__ void __launch_bounds__(kThreads, 3)
+final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const RankSel* __restrict__ sel,
+                  double* __restrict__ fin, uint32_t* __restrict__ hist, int64_t n_tiles, int tiles_per_cta, int shift) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    uint32_t (*sh)[kSelBins] = reinterpret_cast<uint32_t (*)[kSelBins]>(dyn);      // one histogram per rank slot
+    const uint32_t high_mask = ~((1u << (shift + kSelBits)) - 1u);
+    const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
+    uint32_t prefix[kRanks];
+    bool lead[kRanks];
+    int cur_block = -1;
+    int64_t run_first = first;
+    double acc[kResidSums] = {0.0};
+
+    auto flush = [&](int blk, int64_t t_begin, int64_t t_end) {
+        if (kResid) {
+            cta_reduce_store<kResidSums>(acc, fin + size_t(t_begin) * kResidSums);
+            double* rest = fin + size_t(t_begin + 1) * kResidSums;
+            for (int64_t i = threadIdx.x; i < (t_end - t_begin - 1) * kResidSums; i += kThreads) rest[i] = 0.0;
+            acc[0] = 0.0;
+        } else {
+            __syncthreads();
+        }
+#pragma unroll
+        for (int r = 0; r < kRanks; ++r) {
+            if (!lead[r]) continue;                           // uniform over the CTA
+            uint32_t* out = hist + (size_t(blk) * kRanks + r) * kSelBins;
+            for (int d = threadIdx.x; d < kSelBins; d += kThreads) {
+                const uint32_t cnt = sh[r][d];
+                if (cnt) { atomicAdd(out + d, cnt); sh[r][d] = 0u; }
+            }
+        }
+        __syncthreads();
+    };
+
+    for (int i = threadIdx.x; i < kRanks * kSelBins; i += kThreads) (&sh[0][0])[i] = 0u;
+    __syncthreads();
+
+#pragma unroll 1
+    for (int64_t ti = first; ti < last; ++ti) {
+        const Tile t = tiles[ti];
+        if (int(t.block) != cur_block) {                      // uniform over the CTA
+            if (cur_block >= 0) flush(cur_block, run_first, ti);
+            cur_block = int(t.block);
+            run_first = ti;
+#pragma unroll
+            for (int r = 0; r < kRanks; ++r) {
+                const RankSel s = sel[size_t(t.block) * kRanks + r];
+                prefix[r] = s.prefix; lead[r] = s.leader == r;
+            }
+        }
+        const StatBlock* b = blocks + t.block;
+        const int64_t numel = b->numel;
+        const uint32_t* __restrict__ v = reinterpret_cast<const uint32_t*>(b->v);
+        const int64_t base = int64_t(t.piece) * kTile;
+        constexpr int kSl = kTile / (kThreads * 8);
+        uint32_t u[8 * kSl];
+        int valid[kSl];
+#pragma unroll
+        for (int h = 0; h < kSl; ++h) {                       // v is padded to whole quantisation blocks: in bounds whenever e < numel
+            const int64_t e = base + int64_t(h) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+            valid[h] = e < numel ? int(min64(8, numel - e)) : 0;
+            uint4 a = make_uint4(0u, 0u, 0u, 0u), c = a;
+            if (valid[h] > 0) { a = ld_stream_u4(v + e); c = ld_stream_u4(v + e + 4); }
+            u[8 * h + 0] = a.x; u[8 * h + 1] = a.y; u[8 * h + 2] = a.z; u[8 * h + 3] = a.w;
+            u[8 * h + 4] = c.x; u[8 * h + 5] = c.y; u[8 * h + 6] = c.z; u[8 * h + 7] = c.w;
+        }
+        if (kResid && b->cols > 1) {
+            const int cols = b->cols;
+            const double* __restrict__ rowsum = b->rowsum;
+            const double* __restrict__ colsum = b->colsum;
+            const double total = rowsum[b->rows];             // the block's sum of v, left there by the row/column combine
+            const double inv_total = total > 0.0 ? 1.0 / total : 0.0;
+#pragma unroll
+            for (int h = 0; h < kSl; ++h) {
+                if (valid[h] == 0) continue;
+                const int64_t e = base + int64_t(h) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+                int64_t r = e / cols;
+                int c = int(e - r * cols);
+                double rs = __ldg(rowsum + r) * inv_total;
+                if (valid[h] == 8 && (cols & 7) == 0) {
+                    // the eight elements lie in one row: one row sum, four 16-byte loads of column sums
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const double2 w = __ldg(reinterpret_cast<const double2*>(colsum + c) + q);
+                        const double d0 = double(__uint_as_float(u[8 * h + 2 * q])) - rs * w.x;
+                        const double d1 = double(__uint_as_float(u[8 * h + 2 * q + 1])) - rs * w.y;
+                        acc[0] += d0 * d0;
+                        acc[0] += d1 * d1;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (j < valid[h]) {
+                            const double diff = double(__uint_as_float(u[8 * h + j])) - rs * __ldg(colsum + c);
+                            acc[0] += diff * diff;
+                            if (++c == cols) { c = 0; ++r; if (j + 1 < valid[h]) rs = __ldg(rowsum + r) * inv_total; }
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < kRanks; ++r) {
+            if (!lead[r]) continue;
+            int cur = -1;
+            uint32_t n = 0u;
+#pragma unroll
+            for (int k = 0; k < 8 * kSl; ++k) {
+                if ((k & 7) < valid[k >> 3] && ((u[k] ^ prefix[r]) & high_mask) == 0u) {
+                    const int d = int((u[k] >> shift) & uint32_t(kSelBins - 1));
+                    if (d == cur) {
+                        ++n;
+                    } else {
+                        if (n) atomicAdd(&sh[r][cur], n);
+                        cur = d; n = 1u;
+                    }
+                }
+            }
+            if (n) atomicAdd(&sh[r][cur], n);
+        }
+    }
+    if (cur_block >= 0) flush(cur_block, run_first, last);
+}
+
+// One CTA per block: for each of the four ranks find the bin of its leader's
+// histogram that holds the rank (a scan over the CTA), extend the prefix,
+// recompute which ranks still share a prefix, and clear the histograms for the
+// next pass.
+__global__ void __launch_bounds__(kThreads)
+select_pick_kernel(RankSel* __restrict__ sel, uint32_t* __restrict__ hist, int shift, int bins) {
+    __shared__ unsigned long long warp_tot[kThreads / 32];
+    __shared__ int res_d[kRanks];
+    __shared__ long long res_rem[kRanks];
+    const int blk = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    RankSel s[kRanks];
+#pragma unroll
+    for (int r = 0; r < kRanks; ++r) s[r] = sel[size_t(blk) * kRanks + r];
+    if (threadIdx.x < kRanks) { res_d[threadIdx.x] = bins - 1; res_rem[threadIdx.x] = 0; }
+    const int per = bins / kThreads;                          // 1 or 16 bins per thread
+    for (int r = 0; r < kRanks; ++r) {
+        const uint32_t* hh = hist + (size_t(blk) * kRanks + s[r].leader) * kSelBins + threadIdx.x * per;
+        unsigned long long local = 0ull;
+        for (int i = 0; i < per; ++i) local += hh[i];
+        unsigned long long incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        __syncthreads();                                      // the previous rank's readers are done with warp_tot
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        for (int w = 0; w < warp; ++w) incl += warp_tot[w];
+        const unsigned long long excl = incl - local, rem = (unsigned long long)(s[r].remaining);
+        if (excl <= rem && rem < incl) {                      // exactly one thread
+            unsigned long long left = rem - excl;
+            int d = 0;
+            for (; d < per - 1; ++d) {
+                const unsigned long long c = hh[d];
+                if (left < c) break;
+                left -= c;
+            }
+            res_d[r] = threadIdx.x * per + d;
+            res_rem[r] = (long long)(left);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int r = 0; r < kRanks; ++r) {
+            s[r].prefix |= uint32_t(res_d[r]) << shift;
+            s[r].remaining = res_rem[r];
+        }
+        for (int r = 0; r < kRanks; ++r) {
+            int leader = r;
+            for (int q = 0; q < r; ++q)
+                if (s[q].prefix == s[r].prefix) { leader = q; break; }
+            s[r].leader = leader;
+        }
+        for (int r = 0; r < kRanks; ++r) sel[size_t(blk) * kRanks + r] = s[r];
+    }
+    uint32_t* mine = hist + size_t(blk) * kRanks * kSelBins;
+    for (int i = threadIdx.x; i < kRanks * kSelBins; i += kThreads) mine[i] = 0u;
+}
+
+// Start of a select: ranks floor(q (n-1)) and the next one for q = 0.1, 0.9; all four share the empty prefix.
+__global__ void select_init_kernel(const StatBlock* __restrict__ blocks, RankSel* __restrict__ sel, int n_blocks) {
+    const int blk = blockIdx.x * blockDim.x + threadIdx.x;
+    if (blk >= n_blocks) return;
+    const int64_t n = blocks[blk].numel;
+    const double qs[2] = {0.1, 0.9};
+    for (int k = 0; k < 2; ++k) {
+        const double pos = qs[k] * double(n - 1);
+        const int64_t lo = int64_t(floor(pos));
+        const int64_t hi = min64(lo + 1, n - 1);
+        sel[size_t(blk) * kRanks + 2 * k] = RankSel{0u, 0, lo};
+        sel[size_t(blk) * kRanks + 2 * k + 1] = RankSel{0u, 0, hi};
+    }
+}
+
+// End of the window: gather what the host needs into fin_out[block]:
+//   [0..15] sweep-1 sums, [16..19] the four order statistics (as doubles),
+//   [20..27] the running window values, [28] the Eq. 7 numerator, [29] the pilot value.
+__global__ void stats_gather_kernel(const RankSel* __restrict__ sel, const double* __restrict__ acc,
+                                    double* __restrict__ fin_out, int n_blocks) {
+    const int blk = blockIdx.x * blockDim.x + threadIdx.x;
+    if (blk >= n_blocks) return;
+    double* o = fin_out + size_t(blk) * kFinOut;
+    for (int r = 0; r < kRanks; ++r) o[kFinRanks + r] = double(__uint_as_float(sel[size_t(blk) * kRanks + r].prefix));
+    for (int k = 0; k < kBlockAcc; ++k) o[kFinAcc + k] = acc[size_t(blk) * kBlockAcc + k];
+}
+
+// ---- launchers ------------------------------------------------------------------
+#define BAOC_LAUNCH_CHECK()                                   \
+    do {                                                      \
+        cudaError_t e_ = cudaGetLastError();                  \
+        if (e_ != cudaSuccess) return int(e_);                \
+    } while (0)
+
+// Tiles per CTA of a sweep: as many as `most`, fewer when the workload would then not give every SM a few CTAs.
+static int run_tiles(int64_t n_tiles, int most) {
+    const int64_t want = n_tiles / (int64_t(148) * 6);
+    return int(want < 1 ? 1 : (want > most ? most : want));
+}
+
+int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
+                      double* fin_out, uint32_t* hist, RankSel* sel, int64_t n_tiles, int n_blocks, double eps,
+                      float eps_adam, cudaStream_t s) {
+    const int tb = 128, gb = (n_blocks + tb - 1) / tb;
+    cudaError_t e = cudaMemsetAsync(hist, 0, size_t(n_blocks) * kRanks * kSelBins * sizeof(uint32_t), s);
+    if (e != cudaSuccess) return int(e);
+    select_init_kernel<<<gb, tb, 0, s>>>(blocks, sel, n_blocks);
+    BAOC_LAUNCH_CHECK();
+    final_pilot_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, float(eps), fin_out);
+    BAOC_LAUNCH_CHECK();
+    e = cudaFuncSetAttribute(final_sums_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes);
+    if (e != cudaSuccess) return int(e);
+    const int per = run_tiles(n_tiles, kFinRunTiles);
+    final_sums_kernel<<<unsigned((n_tiles + per - 1) / per), kThreads, kFsSmemBytes, s>>>(
+        blocks, tiles, params, fin, fin_out, hist, n_tiles, per, float(eps), eps_adam);
+    BAOC_LAUNCH_CHECK();
+    final_sums_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out);
+    BAOC_LAUNCH_CHECK();
+    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, 24, 256);
+    BAOC_LAUNCH_CHECK();
+    return 0;
+}
+
+int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
+                              uint32_t* hist, const double* acc, int64_t n_tiles, int n_blocks, cudaStream_t s) {
+    constexpr int kSmem = kRanks * kSelBins * int(sizeof(uint32_t));
+    cudaError_t e = cudaFuncSetAttribute(final_hist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(final_hist_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e != cudaSuccess) return int(e);
+    const int per = run_tiles(n_tiles, kSelRunTiles);
+    const unsigned grid = unsigned((n_tiles + per - 1) / per);
+    final_hist_kernel<true><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per, kSelBits);
+    BAOC_LAUNCH_CHECK();
+    final_resid_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out);
+    BAOC_LAUNCH_CHECK();
+    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, kSelBits, kSelBins);
+    BAOC_LAUNCH_CHECK();
+    final_hist_kernel<false><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per, 0);
+    BAOC_LAUNCH_CHECK();
+    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, 0, kSelBins);
+    BAOC_LAUNCH_CHECK();
+    const int tb = 128, gb = (n_blocks + tb - 1) / tb;
+    stats_gather_kernel<<<gb, tb, 0, s>>>(sel, acc, fin_out, n_blocks);
+    BAOC_LAUNCH_CHECK();
+    return 0;
+}
+
+}  // namespace baoc

@@ -113,7 +113,8 @@ void compute_stat_layout(Handle* h) {
             red += int64_t(s.red.chunks) * s.red.strips;
             s.rowsum = reinterpret_cast<double*>(size_t(sum_rows) * 8);
             s.colsum = reinterpret_cast<double*>(size_t(sum_cols) * 8);
-            sum_rows += b.rows; sum_cols += round_up(b.cols, 2);   // column sums start 16-byte aligned (read in pairs)
+            sum_rows += b.rows + 1;                                // the row sums, then their total
+            sum_cols += round_up(b.cols, 2);                       // column sums start 16-byte aligned (read in pairs)
             s.red.rowpart = reinterpret_cast<double*>(size_t(redpart) * 8);
             redpart += int64_t(s.red.strips) * b.rows;
             s.red.colpart = reinterpret_cast<double*>(size_t(redpart) * 8);
@@ -136,7 +137,7 @@ void compute_stat_layout(Handle* h) {
     L.acc = take(&cur, 8 * size_t(kBlockAcc) * n);
     L.fin = take(&cur, 8 * size_t(kFinalSums) * size_t(tiles));
     L.fin_out = take(&cur, 8 * size_t(kFinOut) * n);
-    L.hist = take(&cur, 4 * size_t(256) * kRanks * n);
+    L.hist = take(&cur, 4 * size_t(kSelBins) * kRanks * n);
     L.sel = take(&cur, sizeof(RankSel) * size_t(kRanks) * n);
     L.rowsum = take(&cur, 8 * size_t(std::max<int64_t>(sum_rows, 1)));
     L.colsum = take(&cur, 8 * size_t(std::max<int64_t>(sum_cols, 1)));

@@ -26,11 +26,19 @@ constexpr int kQBlock = 256;          // elements per 8-bit quantisation block
 constexpr int kTile = 4096;           // elements per tile of the streaming kernels
 constexpr int kThreads = 256;         // threads per CTA of the streaming kernels
 constexpr int kStatPartials = 4;      // doubles per tile written by the per-step statistics kernel
-constexpr int kFinalSums = 14;        // doubles per tile written by the first finalize sweep
-constexpr int kResidSums = 2;         // doubles per tile written by the second finalize sweep
+constexpr int kFinalSums = 16;        // doubles per tile slot written by the first finalize sweep
+constexpr int kResidSums = 1;         // doubles per tile slot written by the second finalize sweep
 constexpr int kBlockAcc = 8;          // doubles per block of running window values
 constexpr int kRanks = 4;             // order statistics per block for the two quantiles
-constexpr int kFinOut = 32;           // doubles per block copied to the host at the end of the window
+constexpr int kFinOut = 32;           // doubles per block copied to the host at the end of the window:
+constexpr int kFinRanks = 16;         //   [0..15] first-sweep sums, [16..19] the four order statistics,
+constexpr int kFinAcc = 20;           //   [20..27] the running window values,
+constexpr int kFinResid = 28;         //   [28] the Eq. 7 numerator,
+constexpr int kFinPilot = 29;         //   [29] the pilot value of the Eq. 6 preconditioner
+constexpr int kSelBits = 12;          // bits per radix pass of the quantile select after the first one (which takes the top byte)
+constexpr int kSelBins = 1 << kSelBits;
+constexpr int kFinRunTiles = 8;       // most tiles a CTA of the first finalize sweep works through (its partial sums stay in fp32 that long)
+constexpr int kSelRunTiles = 64;      // most tiles a CTA of the other two sweeps works through
 constexpr int kRedRows = 64;          // rows per CTA of the row/column reduction kernel
 constexpr int kRedCols = 512;         // columns per CTA of the row/column reduction kernel
 constexpr int kTileF = 16384;         // elements per tile of the factored path (its slices are prefetched through shared memory)
@@ -98,7 +106,7 @@ struct StatBlock {
     float* m;            // EMA first moment (Eq. 3)
     float* v;            // EMA second moment
     uint16_t* gprev;     // previous gradient, bf16 bits
-    double* rowsum;      // row sums of v (matrix blocks), length rows
+    double* rowsum;      // row sums of v (matrix blocks), length rows, followed by their total
     double* colsum;      // column sums of v, length cols
     int64_t numel;
     int64_t tile0;       // index of the block's first tile
@@ -288,15 +296,15 @@ int launch_stats_step(const StatBlock* blocks, const Tile* tiles, const void* co
                       int64_t n_tiles, float one_minus_beta_m, float one_minus_beta_v, cudaStream_t s);
 int launch_stats_combine(const StatBlock* blocks, const double* partials, double* acc, int n_blocks, int has_prev,
                          double beta_rho, double eps, cudaStream_t s);
+// First finalize sweep (with the pilot values, the start of the select and its first radix pass), then, after the
+// row/column sums of the matrix blocks, the second and third sweep and the gather of the per-block results.
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
-                      double* fin_out, int64_t n_tiles, int n_blocks, double eps, float eps_adam, cudaStream_t s);
-int launch_final_resid(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
-                       double* fin_out, int64_t n_tiles, int n_blocks, double eps, cudaStream_t s);
-int launch_select(const StatBlock* blocks, const Tile* tiles, RankSel* sel, uint32_t* hist, int64_t n_tiles,
-                  int n_blocks, cudaStream_t s);
+                      double* fin_out, uint32_t* hist, RankSel* sel, int64_t n_tiles, int n_blocks, double eps,
+                      float eps_adam, cudaStream_t s);
+int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
+                              uint32_t* hist, const double* acc, int64_t n_tiles, int n_blocks, cudaStream_t s);
 int launch_sample_gather(const StatBlock* blocks, const Tile* tiles, const void* const* src, int64_t n_tiles, int fp32,
                          cudaStream_t s);
-int launch_gather(const RankSel* sel, const double* acc, double* fin_out, int n_blocks, cudaStream_t s);
 int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const int32_t* ids, int64_t n_red, int n_matrix,
                          cudaStream_t s);
 int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const int32_t* ids, const void* const* grads,

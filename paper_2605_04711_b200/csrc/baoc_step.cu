@@ -169,21 +169,33 @@ moment_reduce_kernel(const StatBlock* __restrict__ blocks, const RedTile* __rest
     rowcol_reduce_piece<false>(b->v, nullptr, 0.f, b->rows, b->cols, b->red, t.chunk, t.strip);
 }
 
-// One CTA per matrix block: add the pieces into rowsum / colsum (double).
+// kCombineSlabs CTAs per matrix block, each owning a slab of the rows and of the columns: add the pieces into
+// rowsum / colsum (double).
 __global__ void __launch_bounds__(kThreads)
 moment_reduce_combine_kernel(const StatBlock* __restrict__ blocks, const int32_t* __restrict__ ids) {
     const StatBlock* b = blocks + ids[blockIdx.x];
-    const int rows = b->rows, cols = b->cols;
-    for (int i = threadIdx.x; i < rows; i += kThreads) {
+    const int rows = b->rows, cols = b->cols, slab = blockIdx.y;
+    const int rpc = (rows + kCombineSlabs - 1) / kCombineSlabs, cpc = (cols + kCombineSlabs - 1) / kCombineSlabs;
+    for (int i = slab * rpc + threadIdx.x; i < min(rows, (slab + 1) * rpc); i += kThreads) {
         double s = 0.0;
         for (int st = 0; st < b->red.strips; ++st) s += b->red.rowpart[size_t(st) * rows + i];
         b->rowsum[i] = s;
     }
-    for (int j = threadIdx.x; j < cols; j += kThreads) {
+    for (int j = slab * cpc + threadIdx.x; j < min(cols, (slab + 1) * cpc); j += kThreads) {
         double s = 0.0;
+#pragma unroll 4
         for (int ch = 0; ch < b->red.chunks; ++ch) s += b->red.colpart[size_t(ch) * cols + j];
         b->colsum[j] = s;
     }
+}
+
+// One CTA per matrix block: the block's total, the sum of its row sums in a fixed order, stored behind them.
+__global__ void __launch_bounds__(kThreads)
+moment_total_kernel(const StatBlock* __restrict__ blocks, const int32_t* __restrict__ ids) {
+    const StatBlock* b = blocks + ids[blockIdx.x];
+    double acc[1] = {0.0};
+    for (int i = threadIdx.x; i < b->rows; i += kThreads) acc[0] += b->rowsum[i];
+    cta_reduce_store<1>(acc, b->rowsum + b->rows);
 }
 
 // kCombineSlabs CTAs per factored block, each owning a slab of the rows and of
@@ -956,7 +968,9 @@ int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const i
     if (n_red <= 0) return 0;
     moment_reduce_kernel<<<unsigned(n_red), kThreads, 0, s>>>(blocks, rtiles);
     BAOC_LAUNCH_CHECK();
-    moment_reduce_combine_kernel<<<n_matrix, kThreads, 0, s>>>(blocks, ids);
+    moment_reduce_combine_kernel<<<dim3(unsigned(n_matrix), kCombineSlabs), kThreads, 0, s>>>(blocks, ids);
+    BAOC_LAUNCH_CHECK();
+    moment_total_kernel<<<n_matrix, kThreads, 0, s>>>(blocks, ids);
     BAOC_LAUNCH_CHECK();
     return 0;
 }

@@ -9,7 +9,9 @@ Tolerances:
   * 8-bit codes: identical on >= 99.99 % of the elements, within 1 code elsewhere;
   * allocation: bit-exact.
 """
+import json
 import math
+import os
 
 import numpy as np
 import pytest
@@ -45,12 +47,22 @@ def _close(got, ref, rel=1e-4, floor=1e-3):
     return abs(got - ref) <= rel * max(abs(ref), floor)
 
 
-def _stat_close(key, got, ref, n_steps):
-    """1e-4 relative.  The err_* diagnostics are ||x - Q(x)|| / ||x|| of the window moments; the library keeps
-    those moments in fp32 (one rounding per window step, so x is off by at most n_steps * 2^-24 relative) while
-    the oracle keeps them in double, and that perturbation passes straight into the distance: on a block of a
-    few elements it does not average out, so it is allowed on top of the relative tolerance."""
-    extra = n_steps * 2.0 ** -23 if key.startswith("err_") else 0.0
+def _carriers(x):
+    """How many elements carry the norm of x: the participation ratio (sum x^2)^2 / sum x^4, which is the element
+    count for equal magnitudes and 1 when a single element dominates.  Computed from the oracle's own moments."""
+    x2 = np.square(np.asarray(x, np.float64) / max(float(np.max(np.abs(x))), 1e-300))
+    return float(np.sum(x2)) ** 2 / max(float(np.sum(x2 * x2)), 1e-300)
+
+
+def _stat_close(key, got, ref, n_steps, carriers):
+    """1e-4 relative.  One exception: the err_* diagnostics are ||x - Q(x)|| / ||x|| of a window moment x, a function
+    of x with Lipschitz constant 1 + err in the relative norm.  The library stores x in fp32 (one rounding per window
+    step: up to n_steps * 2^-24 relative per element), the oracle in double.  Over many elements of comparable size
+    those roundings average out far below 1e-4 of err; where fewer than 256 elements carry the norm (a short block,
+    or a heavy-tailed one that a handful of coordinates dominate) they pass straight into the distance, and there,
+    and only there, the perturbation bound n_steps * 2^-23 is allowed on top.  The finalize kernels alone are held to
+    1e-4 with nothing added by the shared-state test below."""
+    extra = n_steps * 2.0 ** -23 if (key.startswith("err_") and carriers < 256.0) else 0.0
     return abs(got - ref) <= 1e-4 * max(abs(ref), 1e-3) + extra
 
 
@@ -91,7 +103,7 @@ def _check_stats(sess, states, opts=None):
         raw = O.stats_finalize(states[i], sess.block_param_host(i), b.rows, b.cols, o)
         for k in STAT_KEYS:
             got, ref = st[i][k], raw[k]
-            ok = _stat_close(k, got, ref, n_steps)
+            ok = _stat_close(k, got, ref, n_steps, _carriers(states[i].m if "_m" in k else states[i].v))
             worst[k] = max(worst.get(k, 0.0), abs(got - ref) / max(abs(ref), 1e-3))
             assert ok, (b.name, k, got, ref)
         assert st[i]["n_cos"] == states[i].n_cos
@@ -123,6 +135,29 @@ def test_stats_window_odd_sizes(B, H):
     _check_stats(sess, states)
     info = sess.h.query()
     assert info.stats_steps == wl.window and info.kernel_launches > 0
+
+
+def test_finalize_from_shared_moments_holds_every_diagnostic_to_1e_4(B, H):
+    """The finalize kernels alone: after a 12-step window the oracle's moments are rounded to fp32 (the library's
+    storage type) and written to the device (oracle -> device, never the other way), so that both sides finalize the
+    same numbers.  Every diagnostic, the quantisation errors included, then agrees within 1e-4 with nothing added."""
+    wl = _odd_workload(seed=4, window=12)
+    sess = H.Session(wl, n_grad_sets=2)
+    sess.init_params()
+    o = O.Opts()
+    states = _oracle_window(sess, wl.window, o)
+    for i in range(len(wl.blocks)):
+        states[i].m = states[i].m.astype(np.float32).astype(np.float64)
+        states[i].v = states[i].v.astype(np.float32).astype(np.float64)
+        sess.h.view_tensor(i, 0, torch.float32).copy_(torch.from_numpy(states[i].m.astype(np.float32)).to(sess.device))
+        sess.h.view_tensor(i, 1, torch.float32).copy_(torch.from_numpy(states[i].v.astype(np.float32)).to(sess.device))
+    _, st = sess.risk()
+    for i, b in enumerate(wl.blocks):
+        raw = O.stats_finalize(states[i], sess.block_param_host(i), b.rows, b.cols, o)
+        for k in STAT_KEYS:
+            if k in ("rho_bar", "rho_mom"):
+                continue                                             # running values of the per-step pass, compared elsewhere
+            assert abs(st[i][k] - raw[k]) <= 1e-4 * max(abs(raw[k]), 1e-3), (b.name, k, st[i][k], raw[k])
 
 
 def test_stats_invariants_identical_zero_and_flipped_gradients(B, H):
@@ -187,7 +222,7 @@ def test_sampled_statistics_match_the_oracle_on_the_sample(B, H):
         assert m.shape == states[i].m.shape and np.max(np.abs(m - states[i].m)) <= 1e-6 * max(np.max(np.abs(states[i].m)), 1e-30)
         raw = O.stats_finalize(states[i], sess.sampled(i, sess.block_param_host(i)), shapes[i][0], shapes[i][1], o)
         for k in STAT_KEYS:
-            assert _stat_close(k, st[i][k], raw[k], wl.window), (b.name, k, st[i][k], raw[k])
+            assert _stat_close(k, st[i][k], raw[k], wl.window, _carriers(states[i].m if "_m" in k else states[i].v)), (b.name, k, st[i][k], raw[k])
         z = O.normalise(raw, o)
         for c, cfg in enumerate(cfgs):
             ref = O.risk(z, cfg, o)
@@ -246,21 +281,56 @@ def _rel_max(got, ref):
     return float(np.max(np.abs(got - ref)) / max(float(np.max(np.abs(ref))), 1e-30))
 
 
-def _check_block(sess, i, th_ref, st_ref, code_stats):
+# Worst per-element relative error seen on the non-negative fp32 states (second moments, row and column statistics),
+# by path; written to the file BAOC_TEST_REPORT names, if set, when the module is done.
+WORST_ELEMENTWISE = {}
+
+
+def _elementwise(kind, name, got, ref):
+    """Second moments and row / column statistics are sums of non-negative terms, so every element of them (not only
+    the block's largest) must hold 1e-6 relative; first moments and parameters cancel and are held in the max norm.
+    The floor is the smallest normal fp32 number: below it fp32 itself has no 24 bits left."""
+    err = np.abs(got - ref)
+    tol = 1e-6 * np.abs(ref) + 1.2e-38
+    WORST_ELEMENTWISE[kind] = max(WORST_ELEMENTWISE.get(kind, 0.0), float(np.max(err / (np.abs(ref) + 1.2e-32))))
+    assert np.all(err <= tol), (name, kind, float(np.max(err / tol)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _report_worst():
+    yield
+    path = os.environ.get("BAOC_TEST_REPORT")
+    if path and WORST_ELEMENTWISE:
+        with open(path, "a") as f:
+            f.write(json.dumps({"worst_elementwise_relative_error": WORST_ELEMENTWISE}) + "\n")
+
+
+def _check_block(sess, i, th_ref, st_ref, code_stats, elementwise=True):
+    """elementwise: also hold every element of a non-negative fp32 state to 1e-6 of itself.  Off where both sides
+    run free under coupled decay: there the effective gradient g + wd*theta can cancel, so an element's own
+    relative error is not bounded by the arithmetic."""
     got = sess.block_param_host(i)
     assert np.all(np.isfinite(got))
+    name = sess.wl.blocks[i].name
     if th_ref is not None:
-        assert _rel_max(got, th_ref) <= 1e-6, (sess.wl.blocks[i].name, st_ref.kind, _rel_max(got, th_ref))
+        assert _rel_max(got, th_ref) <= 1e-6, (name, st_ref.kind, _rel_max(got, th_ref))
     kind = st_ref.kind
     f32 = lambda w: sess.h.view_tensor(i, w, torch.float32).double().cpu().numpy()
     if kind == "A32":
         assert _rel_max(f32(10), st_ref.m) <= 1e-6 and _rel_max(f32(11), st_ref.v) <= 1e-6
+        if elementwise:
+            _elementwise(kind, name, f32(11), st_ref.v)
     elif kind == "R":
         assert _rel_max(f32(10), st_ref.v) <= 1e-6
+        if elementwise:
+            _elementwise(kind, name, f32(10), st_ref.v)
     elif kind == "S":
         assert _rel_max(f32(10), st_ref.m) <= 1e-6
     elif kind == "F":
         assert _rel_max(f32(10), st_ref.r) <= 1e-6 and _rel_max(f32(11), st_ref.c) <= 1e-6
+        if elementwise:
+            _elementwise(kind + ".r", name, f32(10), st_ref.r)
+            _elementwise(kind + ".c", name, f32(11), st_ref.c)
     elif kind == "F8":
         for w, (ref_q, ref_a) in enumerate(((st_ref.qr, st_ref.ar), (st_ref.qc, st_ref.ac))):
             q = sess.h.view_tensor(i, 10 + w, torch.uint8).cpu().numpy().astype(np.int32)
@@ -411,6 +481,26 @@ def test_coupled_decay_and_other_hyperparameters_step_by_step(B, H):
     ocfgs = [_ocfg(c) for c in cfgs]
     codes = _run_steps_from_shared_state(sess, assign, ocfgs)
     assert codes[1] > 0 and codes[0] <= 1e-4 * codes[1], codes
+
+
+def test_coupled_decay_free_running_ten_steps_on_the_fp32_paths(B, H):
+    """Coupled weight decay (y_d = 0 in Definition 3.1) on the four fp32 headline paths (Adam, RMS scaling, factored
+    second moment, SGD with momentum): ten free-running steps from zero state, parameters and states within 1e-6 of
+    the block's largest value.  (The 8-bit tuples under coupled decay are stepped from shared states above: a second
+    moment whose code is 0 makes their free-running trajectory ill-conditioned.)"""
+    wl = _odd_workload(seed=23)
+    cfgs = [B.make_config(1, 1, 0, 0, 32, lr=3e-3, beta1=0.8, beta2=0.95, eps=1e-6, weight_decay=0.1),
+            B.make_config(1, 0, 0, 0, 32, lr=1e-3, beta2=0.9, eps=1e-6, weight_decay=0.1),
+            B.make_config(1, 0, 0, 1, 32, lr=1e-3, beta2=0.9, eps=1e-6, weight_decay=0.1),
+            B.make_config(0, 1, 0, 0, 32, lr=1e-2, beta1=0.5, weight_decay=0.1)]
+    sess = H.Session(wl, configs=cfgs, n_grad_sets=2)
+    sess.init_params()
+    assign = [(i % 4) if not ((i % 4) == 2 and b.cols <= 1) else 1 for i, b in enumerate(wl.blocks)]
+    assert {0, 1, 2, 3} <= set(assign)
+    th, sts = _run_steps(sess, assign, 10)
+    for i in range(len(wl.blocks)):
+        _check_block(sess, i, th[i], sts[i], [0, 0], elementwise=False)
+    assert sess.h.nonfinite()[0] == 0
 
 
 @pytest.mark.parametrize("tuple_", [(0, 0, 1, 0, 32), (0, 0, 0, 0, 8), (1, 1, 1, 0, 16), (1, 1, 0, 0, 16), (1, 0, 1, 0, 16),
@@ -770,7 +860,7 @@ def test_checkpoint_resume_continues_bit_exactly(B, H):
 
 # ---------------------------------------------------------------- whole pipeline
 
-def _pipeline(B, H, name, T, n_steps, time_table=None):
+def _pipeline(B, H, name, T, n_steps, time_table=None, full=False):
     wl = W.make_workload(name, seed=0)
     sess = H.Session(wl, n_grad_sets=2)
     sess.init_params()
@@ -796,7 +886,7 @@ def _pipeline(B, H, name, T, n_steps, time_table=None):
         _check_block(sess, i, th[i], sts[i], codes)
     if codes[1]:
         assert codes[0] <= 1e-4 * codes[1], codes
-    return asg
+    return (asg, risk, risk_ref, sess) if full else asg
 
 
 def test_toy_pipeline_window_risk_allocation_ten_mixed_steps(B, H):
@@ -825,6 +915,32 @@ def test_toy_allocation_matches_brute_force_on_eight_blocks(B, H):
 
 
 def test_resnet50_pipeline_with_binding_time_budget(B, H):
+    """The ResNet-50-shaped configuration as stated: a 32-step window, memory budget 40 %, a time-ratio table under
+    which B_time = 1.1 binds, then ten mixed steps."""
     wl = W.make_workload("resnet50")
+    assert wl.window == 32 and wl.time_budget == 1.1 and wl.mem_budget_frac == 0.4
     table = W.time_ratio_table(wl, [1.0, 1.25, 0.8, 1.5, 0.7]).numpy()
-    _pipeline(B, H, "resnet50", 4, 3, table)
+    asg, risk, risk_ref, sess = _pipeline(B, H, "resnet50", wl.window, 10, table, full=True)
+    mean_ratio = lambda a: float(np.mean([table[i, c] for i, c in enumerate(a)]))
+    assert mean_ratio(asg) <= 1.1 + 1e-9
+    # a time budget just below what the memory budget alone would choose does bind: the optimum moves, stays within
+    # both budgets, and is again the same from the library's risk and from the oracle's
+    mem, _ = sess.h.cost_model()
+    b_mem = int(np.floor(0.4 * 8.0 * wl.numel))
+    free, _, rc = sess.h.allocate(risk, mem, table, b_mem, 10.0)
+    assert rc == 0
+    tight = mean_ratio(free) - 0.02
+    bound, _, rc1 = sess.h.allocate(risk, mem, table, b_mem, tight)
+    bound_ref, _, rc2 = sess.h.allocate(risk_ref, mem, table, b_mem, tight)
+    assert rc1 == 0 and rc2 == 0 and bound.tolist() == bound_ref.tolist() != free.tolist()
+    assert mean_ratio(bound) <= tight + 1e-9 and sum(int(mem[i, c]) for i, c in enumerate(bound)) <= b_mem
+
+
+def test_gpt2_small_pipeline_window_risk_allocation_ten_mixed_steps(B, H):
+    """The GPT-2-small-shaped configuration (124 M parameters, Student-t gradients in the embedding and attention
+    blocks, memory budget 35 %): window, finalize and risk against the oracle on every block, the allocation from
+    the library's risk equal to the allocation from the oracle's risk, then ten mixed steps on every block."""
+    wl = W.make_workload("gpt2_small")
+    assert wl.numel == 124_439_808 and wl.mem_budget_frac == 0.35
+    asg = _pipeline(B, H, "gpt2_small", 8, 10)
+    assert len(set(asg.tolist())) >= 2
