@@ -2,12 +2,14 @@
 // signal-to-noise ratio (Eq. 5), the distortion (Eq. 6), the structure residual
 // (Eq. 7) and the precision cosines (Eq. 8), and the exact quantiles behind the
 // anisotropy (Eq. 4).  Three sweeps over the window's moments:
-//   1. final_sums_kernel   reads m, v, theta: 16 sums per block, and the histogram of the top byte of v
+//   1. final_sums_kernel   reads m, v, theta: 16 sums per block, and the histogram of the top 12 bits of v
 //   2. final_hist_kernel<true>   reads v: Eq. 7 residual (after the row/column sums), histogram of the next 12 bits
-//   3. final_hist_kernel<false>  reads v: histogram of the last 12 bits
+//   3. final_hist_kernel<false>  reads v: histogram of the last 8 bits
 // A CTA works through a run of consecutive tiles, keeps its partial sums and
 // histograms on chip while the tiles belong to one block, and hands them over
 // once per block (a deterministic, fixed partition of the work).
+#include <cstring>
+
 #include "baoc_device.cuh"
 
 namespace baoc {
@@ -64,10 +66,96 @@ final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, double* __re
 // ============================================================================
 constexpr int kFsStageBytes = kThreads * 96;                 // m 32 B/thread at 0, v at 8192, theta at 16384
 constexpr int kFsStages = 3;
-constexpr int kHistCopies = 8;                               // replicas of the top-byte histogram (one per lane & 7)
-constexpr int kFsSmemBytes = kFsStages * kFsStageBytes + kHistCopies * 256 * 4;
+constexpr int kFsSmemBytes = kFsStages * kFsStageBytes + kSelBins * 4;      // the staging ring and the histogram of the first digit
 
-__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) { return fma2(b, splat2(-1.0f), a); }
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float rsqrt_approx(float x) {
+    float r;
+    asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+// One slice of eight elements per thread (a warp: one 256-element quantisation block).  kFull: all eight elements of
+// every lane of the warp lie inside the block; otherwise cnt of them do and the padding (m = v = theta = 0) is
+// masked out of the one sum it would otherwise enter (p - p0).
+//
+// The bf16 direction costs no extra square root or reciprocal: with n = (v - v16) / v (|n| <= 2^-8),
+// sqrt(v16) - sqrt(v) = -sqrt(v) n (1/2 + n/8 + n^2/16) up to n^4, and with e that difference over (sqrt(v) + eps_adam),
+// 1 / (sqrt(v16) + eps_adam) = (1 - e + e^2 - e^3) / (sqrt(v) + eps_adam) up to e^4: both truncations are below 1e-10.
+template <bool kFull>
+__device__ __forceinline__ void fs_slice(const float (&mm)[8], const float (&vv)[8], const float (&tt)[8], int cnt,
+                                         float p0, float eps_f, float eps_adam, f32x2 (&F)[kFinalSums], uint32_t* hist1) {
+    const f32x2 P0 = splat2(p0), MAGIC = splat2(12582912.0f), C16 = splat2(65537.0f), EA = splat2(eps_adam), EPS = splat2(eps_f),
+                ONE = splat2(1.0f), MONE = splat2(-1.0f);
+    // ---- absmax of the warp's quantisation block, code scales
+    float am = 0.f, av = 0.f;
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        am = max3(am, fabsf(mm[2 * p]), fabsf(mm[2 * p + 1]));
+        av = max3(av, vv[2 * p], vv[2 * p + 1]);
+    }
+    am = warp_max_nonneg(am); av = warp_max_nonneg(av);
+    const float rm0 = rcp_approx(am), rv0 = rcp_approx(av);          // L / a from the reciprocal and one Newton step
+    const f32x2 KM = splat2(am > 0.f ? 127.0f * (rm0 * fmaf(-am, rm0, 2.0f)) : 0.f);
+    const f32x2 KV = splat2(av > 0.f ? 255.0f * (rv0 * fmaf(-av, rv0, 2.0f)) : 0.f);
+    // a / L in two parts (the second one the exact remainder of the first, divided by L), so that code * a / L comes
+    // out correctly rounded and the block's largest element, whose code is L, is reproduced exactly
+    const float dmh = am * (1.0f / 127.0f), dvh = av * (1.0f / 255.0f);
+    const f32x2 DM = splat2(dmh), DV = splat2(dvh);
+    const f32x2 DML = splat2(fmaf(-127.0f, dmh, am) * (1.0f / 127.0f)), DVL = splat2(fmaf(-255.0f, dvh, av) * (1.0f / 255.0f));
+
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        const f32x2 M = pack2(mm[2 * p], mm[2 * p + 1]), V = pack2(vv[2 * p], vv[2 * p + 1]);
+        const f32x2 T = pack2(tt[2 * p], tt[2 * p + 1]);
+        // 8-bit round trips: code = rne(x L / a) by the magic-number addition, value = code a / L
+        const f32x2 QM = sub2(fma2(M, KM, MAGIC), MAGIC), QV = sub2(fma2(V, KV, MAGIC), MAGIC);
+        const f32x2 M8 = fma2(QM, DM, mul2(QM, DML)), V8 = fma2(QV, DV, mul2(QV, DVL));
+        // bf16 round trips
+        const f32x2 CM = mul2(M, C16), CV = mul2(V, C16);
+        // (written as x*(-1) + y: a plain packed subtraction here came out as the identity, the two differences folded)
+        const f32x2 M16 = fma2(fma2(M, MONE, CM), MONE, CM), V16 = fma2(fma2(V, MONE, CV), MONE, CV);
+        const f32x2 E0 = sub2(M, M8), E1 = sub2(V, V8), E2 = sub2(M, M16), E3 = sub2(V, V16);
+        // full-precision direction and the preconditioner: sqrt(v) = v rsqrt(v) (a v below the smallest normal number
+        // counts as that number under the root: its root is far below either epsilon)
+        float a0, a1, b0, b1;
+        const f32x2 R = pack2(rsqrt_approx(fmaxf(vv[2 * p], 1.17549435e-38f)), rsqrt_approx(fmaxf(vv[2 * p + 1], 1.17549435e-38f)));
+        const f32x2 S = mul2(V, R);
+        unpack2(add2(S, EA), a0, a1);
+        const f32x2 R32 = pack2(rcp_approx(a0), rcp_approx(a1));
+        const f32x2 U32 = mul2(M, R32);
+        unpack2(add2(S, EPS), a0, a1);
+        f32x2 PD = sub2(pack2(rcp_approx(a0), rcp_approx(a1)), P0);
+        if (!kFull) PD = mul2(PD, pack2(2 * p < cnt ? 1.f : 0.f, 2 * p + 1 < cnt ? 1.f : 0.f));
+        // 8-bit direction: the quantised second moment is not close to v in relative terms, so its own root
+        unpack2(V8, b0, b1);
+        unpack2(add2(pack2(sqrt_approx(b0), sqrt_approx(b1)), EA), b0, b1);
+        const f32x2 U8 = mul2(M8, pack2(rcp_approx(b0), rcp_approx(b1)));
+        // bf16 direction from the series
+        const f32x2 N = mul2(E3, mul2(R, R));
+        const f32x2 H = mul2(N, fma2(N, fma2(N, splat2(0.0625f), splat2(0.125f)), splat2(0.5f)));
+        const f32x2 NE = mul2(mul2(S, H), R32);                                  // -(sqrt(v16) - sqrt(v)) / (sqrt(v) + eps_adam)
+        const f32x2 U16 = mul2(M16, mul2(R32, fma2(NE, fma2(NE, add2(NE, ONE), ONE), ONE)));
+        // the sums
+        F[0] = fma2(M, M, F[0]); F[1] = add2(F[1], V); F[2] = fma2(V, V, F[2]); F[3] = add2(F[3], PD);
+        const f32x2 T2 = mul2(T, T), PT = mul2(PD, T2);
+        F[4] = add2(F[4], T2); F[14] = add2(F[14], PT); F[15] = fma2(PD, PT, F[15]);
+        F[5] = fma2(U32, U32, F[5]); F[6] = fma2(U8, U8, F[6]); F[7] = fma2(U32, U8, F[7]);
+        F[8] = fma2(U16, U16, F[8]); F[9] = fma2(U32, U16, F[9]);
+        F[10] = fma2(E0, E0, F[10]); F[11] = fma2(E1, E1, F[11]); F[12] = fma2(E2, E2, F[12]); F[13] = fma2(E3, E3, F[13]);
+    }
+
+    // ---- first radix pass of the quantile select: the top 12 bits of v's bit pattern (sign, exponent, three mantissa
+    // bits).  The second moments of a block spread over many of these bins, so a plain shared-memory histogram with one
+    // atomic per element meets few collisions.
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        if (kFull || j < cnt) atomicAdd(hist1 + (__float_as_uint(vv[j]) >> (32 - kSelBits)), 1u);
+}
 
 __global__ void __launch_bounds__(kThreads, 2)
 final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
@@ -76,25 +164,24 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
                   int tiles_per_cta, float eps_f, float eps_adam) {
     extern __shared__ __align__(16) unsigned char dyn[];
     unsigned char* stage = dyn;
-    uint32_t (*sh)[256] = reinterpret_cast<uint32_t (*)[256]>(dyn + kFsStages * kFsStageBytes);
-    constexpr float kMagic = 12582912.0f;                    // 1.5 * 2^23: adding it rounds to an integer, ties to even
+    uint32_t* hist1 = reinterpret_cast<uint32_t*>(dyn + kFsStages * kFsStageBytes);      // kSelBins counters
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int copy = threadIdx.x & (kHistCopies - 1);
     const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
     const int nsl = int(last - first) * (kTile / (kThreads * 8));     // slices of this CTA
     const uint32_t sm0 = smem_addr(stage);
-    const uint32_t om = threadIdx.x * 32, ov = 8192 + threadIdx.x * 32, ot = 16384 + threadIdx.x * 32;
+    const uint32_t om = threadIdx.x * 32, ov = 8192 + om, ot = 16384 + om;
+    constexpr uint32_t kHalf = 16;                           // a thread's 32 bytes per array are contiguous
 
-    for (int i = threadIdx.x; i < kHistCopies * 256; i += kThreads) (&sh[0][0])[i] = 0u;
+    for (int i = threadIdx.x; i < kSelBins; i += kThreads) hist1[i] = 0u;
     __syncthreads();
 
     f32x2 F[kFinalSums];
 #pragma unroll
     for (int k = 0; k < kFinalSums; ++k) F[k] = pack2(0.f, 0.f);
 
-    // hand the finished run of tiles [t_begin, t_end) of block blk over: its sums go to the slot of its first tile
-    // (zeros to the others, the per-block combine adds all slots), its histogram to the block's global one
-    auto flush = [&](int blk, int64_t t_begin, int64_t t_end) {
+    // hand the finished run of tiles of block blk over: its sums go to the slot of its first tile (the per-block
+    // combine adds the slots of the runs' first tiles), its histogram to the block's global one
+    auto flush = [&](int blk, int64_t t_begin) {
         double acc[kFinalSums];
 #pragma unroll
         for (int k = 0; k < kFinalSums; ++k) {
@@ -104,18 +191,16 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
             F[k] = pack2(0.f, 0.f);
         }
         cta_reduce_store<kFinalSums>(acc, fin + size_t(t_begin) * kFinalSums);
-        double* rest = fin + size_t(t_begin + 1) * kFinalSums;
-        for (int64_t i = threadIdx.x; i < (t_end - t_begin - 1) * kFinalSums; i += kThreads) rest[i] = 0.0;
-        uint32_t* out = hist + size_t(blk) * kRanks * kSelBins;
-        for (int d = threadIdx.x; d < 256; d += kThreads) {
-            uint32_t cnt = 0u;
-#pragma unroll
-            for (int c = 0; c < kHistCopies; ++c) { cnt += sh[c][d]; sh[c][d] = 0u; }
-            if (cnt) atomicAdd(out + d, cnt);
+        uint32_t* out = hist + size_t(blk) * kRanks * kSelBins;          // all four ranks still share one histogram
+        for (int d = threadIdx.x; d < kSelBins; d += kThreads) {
+            const uint32_t cnt = hist1[d];
+            if (cnt) { atomicAdd(out + d, cnt); hist1[d] = 0u; }
         }
         __syncthreads();
     };
 
+    // Each thread copies the 32 bytes per array that hold its own eight elements, as two 16-byte copies through L1:
+    // the second copy finds its 32-byte sector there, so that L2 serves every sector once.
     uint32_t fill = 0, take = 0;
     auto prefetch = [&](int k) {
         if (k < nsl) {
@@ -127,11 +212,11 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
             // inside the array; theta is not padded
             if (e - lane * 8 < numel) {
                 const uint32_t d = sm0 + fill;
-                cp_async16(d + om, b->m + e); cp_async16(d + om + 16, b->m + e + 4);
-                cp_async16(d + ov, b->v + e); cp_async16(d + ov + 16, b->v + e + 4);
+                cp_async16_l1(d + om, b->m + e); cp_async16_l1(d + om + kHalf, b->m + e + 4);
+                cp_async16_l1(d + ov, b->v + e); cp_async16_l1(d + ov + kHalf, b->v + e + 4);
                 if (e + 8 <= numel) {
                     const float* th = params[t.block];
-                    cp_async16(d + ot, th + e); cp_async16(d + ot + 16, th + e + 4);
+                    cp_async16_l1(d + ot, th + e); cp_async16_l1(d + ot + kHalf, th + e + 4);
                 }
             }
         }
@@ -144,8 +229,6 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
     int cur_block = -1;
     int64_t run_first = first;
     float p0 = 0.f;
-    const f32x2 MAGIC = splat2(kMagic), NMAGIC = splat2(-kMagic), C16 = splat2(65537.0f), EA = splat2(eps_adam),
-                EPS = splat2(eps_f);
 #pragma unroll 1
     for (int k = 0; k < nsl; ++k) {
         prefetch(k + kFsStages - 1);
@@ -153,147 +236,116 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
         const int64_t ti = first + (k >> 1);
         const Tile t = tiles[ti];
         if (int(t.block) != cur_block) {                     // uniform over the CTA; only at a tile boundary
-            if (cur_block >= 0) flush(cur_block, run_first, ti);
+            if (cur_block >= 0) flush(cur_block, run_first);
             cur_block = int(t.block);
             run_first = ti;
             p0 = float(fin_out[size_t(t.block) * kFinOut + kFinPilot]);
         }
         const unsigned char* mine = stage + take;
         take = take == (kFsStages - 1) * kFsStageBytes ? 0u : take + kFsStageBytes;
-        const StatBlock* b = blocks + t.block;
-        const int64_t numel = b->numel;
+        const int64_t numel = blocks[t.block].numel;
         const int64_t w0 = int64_t(t.piece) * kTile + int64_t(k & 1) * (kThreads * 8) + int64_t(warp) * kQBlock;
         if (w0 >= numel) continue;                           // whole warp out of range
-        const int64_t e = w0 + lane * 8;
-        const int cnt = int(max64(0, min64(8, numel - e)));
         float mm[8], vv[8], tt[8];
-        f4_to8(*reinterpret_cast<const float4*>(mine + om), *reinterpret_cast<const float4*>(mine + om + 16), mm);
-        f4_to8(*reinterpret_cast<const float4*>(mine + ov), *reinterpret_cast<const float4*>(mine + ov + 16), vv);
-        if (cnt == 8) {
-            f4_to8(*reinterpret_cast<const float4*>(mine + ot), *reinterpret_cast<const float4*>(mine + ot + 16), tt);
+        f4_to8(*reinterpret_cast<const float4*>(mine + om), *reinterpret_cast<const float4*>(mine + om + kHalf), mm);
+        f4_to8(*reinterpret_cast<const float4*>(mine + ov), *reinterpret_cast<const float4*>(mine + ov + kHalf), vv);
+        if (w0 + kQBlock <= numel) {                         // uniform over the warp
+            f4_to8(*reinterpret_cast<const float4*>(mine + ot), *reinterpret_cast<const float4*>(mine + ot + kHalf), tt);
+            fs_slice<true>(mm, vv, tt, 8, p0, eps_f, eps_adam, F, hist1);
         } else {
-            const float* th = params[t.block];
+            const int64_t e = w0 + lane * 8;
+            const int cnt = int(max64(0, min64(8, numel - e)));
+            if (cnt == 8) {
+                f4_to8(*reinterpret_cast<const float4*>(mine + ot), *reinterpret_cast<const float4*>(mine + ot + kHalf), tt);
+            } else {
+                const float* th = params[t.block];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) tt[j] = j < cnt ? th[e + j] : 0.f;
-        }
-
-        // ---- absmax of the warp's quantisation block, code scales
-        float am = 0.f, av = 0.f;
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-            am = max3(am, fabsf(mm[2 * p]), fabsf(mm[2 * p + 1]));
-            av = max3(av, vv[2 * p], vv[2 * p + 1]);
-        }
-        am = warp_max_nonneg(am); av = warp_max_nonneg(av);
-        const float rm0 = rcp_approx(am), rv0 = rcp_approx(av);      // L / a from the reciprocal and one Newton step
-        const f32x2 KM = splat2(am > 0.f ? 127.0f * (rm0 * fmaf(-am, rm0, 2.0f)) : 0.f);
-        const f32x2 KV = splat2(av > 0.f ? 255.0f * (rv0 * fmaf(-av, rv0, 2.0f)) : 0.f);
-        // a / L in two parts (the second one the exact remainder of the first, divided by L), so that code * a / L comes
-        // out correctly rounded and the block's largest element, whose code is L, is reproduced exactly
-        const float dmh = am * (1.0f / 127.0f), dvh = av * (1.0f / 255.0f);
-        const f32x2 DM = splat2(dmh), DV = splat2(dvh);
-        const f32x2 DML = splat2(fmaf(-127.0f, dmh, am) * (1.0f / 127.0f)), DVL = splat2(fmaf(-255.0f, dvh, av) * (1.0f / 255.0f));
-
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-            const f32x2 M = pack2(mm[2 * p], mm[2 * p + 1]), V = pack2(vv[2 * p], vv[2 * p + 1]);
-            const f32x2 T = pack2(tt[2 * p], tt[2 * p + 1]);
-            // 8-bit round trips: code = rne(x L / a) by the magic-number addition, value = code a / L
-            const f32x2 QM = add2(fma2(M, KM, MAGIC), NMAGIC), QV = add2(fma2(V, KV, MAGIC), NMAGIC);
-            const f32x2 M8 = fma2(QM, DM, mul2(QM, DML)), V8 = fma2(QV, DV, mul2(QV, DVL));
-            // bf16 round trips
-            const f32x2 CM = mul2(M, C16), CV = mul2(V, C16);
-            const f32x2 M16 = sub2(CM, sub2(CM, M)), V16 = sub2(CV, sub2(CV, V));
-            // directions and the preconditioner (padding: m = v = 0 gives zeros everywhere but in p, which is masked)
-            float a0, a1, b0, b1, c0, c1;
-            const f32x2 S = pack2(sqrt_approx(vv[2 * p]), sqrt_approx(vv[2 * p + 1]));
-            unpack2(add2(S, EA), a0, a1);
-            const f32x2 U32 = mul2(M, pack2(rcp_approx(a0), rcp_approx(a1)));
-            unpack2(add2(S, EPS), a0, a1);
-            const f32x2 PD = pack2(2 * p < cnt ? rcp_approx(a0) - p0 : 0.f, 2 * p + 1 < cnt ? rcp_approx(a1) - p0 : 0.f);
-            unpack2(V8, b0, b1);
-            unpack2(add2(pack2(sqrt_approx(b0), sqrt_approx(b1)), EA), b0, b1);
-            const f32x2 U8 = mul2(M8, pack2(rcp_approx(b0), rcp_approx(b1)));
-            unpack2(V16, c0, c1);
-            unpack2(add2(pack2(sqrt_approx(c0), sqrt_approx(c1)), EA), c0, c1);
-            const f32x2 U16 = mul2(M16, pack2(rcp_approx(c0), rcp_approx(c1)));
-            // the sums
-            F[0] = fma2(M, M, F[0]); F[1] = add2(F[1], V); F[2] = fma2(V, V, F[2]); F[3] = add2(F[3], PD);
-            const f32x2 T2 = mul2(T, T), PT = mul2(PD, T2);
-            F[4] = add2(F[4], T2); F[14] = add2(F[14], PT); F[15] = fma2(PD, PT, F[15]);
-            F[5] = fma2(U32, U32, F[5]); F[6] = fma2(U8, U8, F[6]); F[7] = fma2(U32, U8, F[7]);
-            F[8] = fma2(U16, U16, F[8]); F[9] = fma2(U32, U16, F[9]);
-            const f32x2 E0 = sub2(M, M8), E1 = sub2(V, V8), E2 = sub2(M, M16), E3 = sub2(V, V16);
-            F[10] = fma2(E0, E0, F[10]); F[11] = fma2(E1, E1, F[11]); F[12] = fma2(E2, E2, F[12]); F[13] = fma2(E3, E3, F[13]);
-        }
-
-        // ---- first radix pass of the quantile select: the top byte of v's bit pattern (sign and upper exponent bits).
-        // Nearly all elements of a block share it, so a thread adds runs of equal bytes, into one of eight replicas.
-        {
-            int cur = -1;
-            uint32_t n = 0u;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (j < cnt) {
-                    const int d = int(__float_as_uint(vv[j]) >> 24);
-                    if (d == cur) {
-                        ++n;
-                    } else {
-                        if (n) atomicAdd(&sh[copy][cur], n);
-                        cur = d; n = 1u;
-                    }
-                }
+                for (int j = 0; j < 8; ++j) tt[j] = j < cnt ? th[e + j] : 0.f;
             }
-            if (n) atomicAdd(&sh[copy][cur], n);
+            fs_slice<false>(mm, vv, tt, cnt, p0, eps_f, eps_adam, F, hist1);
         }
     }
     cp_async_wait<0>();
-    if (cur_block >= 0) flush(cur_block, run_first, last);
+    if (cur_block >= 0) flush(cur_block, run_first);
 }
 
-// Per-block combines of the sweeps: the sums over the block's tile slots, in tile order.
-__global__ void __launch_bounds__(kThreads)
-final_sums_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ fin, double* __restrict__ fin_out) {
-    const StatBlock* b = blocks + blockIdx.x;
-    block_tiles_sum<kFinalSums>(fin, b->tile0, b->ntiles, fin_out + size_t(blockIdx.x) * kFinOut);
+// Per-block combines of the sweeps.  A sweep's CTA b works through the tiles [b per, (b+1) per) of the tile table and
+// leaves the sums of each run of tiles of one block in the slot of the run's first tile; the runs of a block therefore
+// start at its first tile and at every multiple of `per` inside it.  Their slots are added in tile order.
+template <int K>
+__device__ __forceinline__ void block_runs_sum(const double* __restrict__ part, int64_t tile0, int ntiles, int per, double* out) {
+    double acc[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) acc[k] = 0.0;
+    const int64_t r0 = tile0 / per;                          // the run that holds the block's first tile
+    const int nruns = int((tile0 + ntiles - 1) / per - r0) + 1;
+    for (int i = threadIdx.x; i < nruns; i += kThreads) {
+        const int64_t head = i == 0 ? tile0 : (r0 + i) * per;
+        const double* p = part + size_t(head) * K;
+#pragma unroll
+        for (int k = 0; k < K; ++k) acc[k] += p[k];
+    }
+    cta_reduce_store<K>(acc, out);
 }
 
 __global__ void __launch_bounds__(kThreads)
-final_resid_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ fin, double* __restrict__ fin_out) {
+final_sums_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ fin, double* __restrict__ fin_out, int per) {
     const StatBlock* b = blocks + blockIdx.x;
-    block_tiles_sum<kResidSums>(fin, b->tile0, b->ntiles, fin_out + size_t(blockIdx.x) * kFinOut + kFinResid);
+    block_runs_sum<kFinalSums>(fin, b->tile0, b->ntiles, per, fin_out + size_t(blockIdx.x) * kFinOut);
+}
+
+__global__ void __launch_bounds__(kThreads)
+final_resid_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ fin, double* __restrict__ fin_out, int per) {
+    const StatBlock* b = blocks + blockIdx.x;
+    block_runs_sum<kResidSums>(fin, b->tile0, b->ntiles, per, fin_out + size_t(blockIdx.x) * kFinOut + kFinResid);
 }
 
 // ============================================================================
-// Sweeps 2 and 3: radix passes of the exact quantile select over the fp32 bit
-// patterns of v (v >= 0, so the unsigned order of the patterns is the numeric
-// order): four ranks per block (the two order statistics around each of the two
-// quantile positions); ranks that still share a prefix share one histogram (the
-// "leader" rank's).  A pass looks at the 12 bits [shift, shift + 12) of the
-// elements whose higher bits equal the prefix found so far.
-// kResid: the same sweep also forms the Eq. 7 numerator
-//   sum (S_ij - a_i b_j / mu)^2 = sum (v_ij - rowsum_i colsum_j / total)^2
-// of matrix blocks, in double (a difference of nearly equal numbers).
+// Sweeps 2 and 3: the remaining radix passes of the exact quantile select over
+// the fp32 bit patterns of v (v >= 0, so the unsigned order of the patterns is
+// the numeric order): four ranks per block (the two order statistics around each
+// of the two quantile positions); ranks that still share a prefix share one
+// histogram (the "leader" rank's).  The first pass (top 12 bits) is part of the
+// first sweep; here
+//   kResid = true:  second pass, bits [8, 20) of the elements whose top 12 bits are a rank's prefix, and in the same
+//                   sweep the Eq. 7 numerator
+//                     sum (S_ij - a_i b_j / mu)^2 = sum (v_ij - rowsum_i colsum_j / total)^2
+//                   of matrix blocks, in double (a difference of nearly equal numbers);
+//   kResid = false: third pass, bits [0, 8) of the elements whose upper 24 bits are a rank's prefix.
+// Few elements match a prefix: a thread first tests whether any of its 16 does.  A thread whose 16 elements are all
+// equal (constant or untouched stretches of a tensor) adds them with one atomic.
+// The histograms count in 16 bits, two bins per word, which halves their shared memory (32 KB, so that four CTAs fit
+// an SM and keep enough loads in flight); a CTA therefore hands its histograms over after at most kSelRunTiles = 15
+// tiles (61440 elements, below 2^16).  (Staging the tiles through a cp.async ring at two CTAs per SM was slower.)
 // ============================================================================
+constexpr int kFhHistWords = kSelBins / 2;
+constexpr int kFhSmemBytes = kRanks * kFhHistWords * 4;
+static_assert(kSelRunTiles * kTile < 65536, "a 16-bit bin must hold a whole run of tiles");
+
 template <bool kResid>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, kResid ? 3 : 4)
 final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const RankSel* __restrict__ sel,
-                  double* __restrict__ fin, uint32_t* __restrict__ hist, int64_t n_tiles, int tiles_per_cta, int shift) {
+                  double* __restrict__ fin, uint32_t* __restrict__ hist, int64_t n_tiles, int tiles_per_cta) {
     extern __shared__ __align__(16) unsigned char dyn[];
-    uint32_t (*sh)[kSelBins] = reinterpret_cast<uint32_t (*)[kSelBins]>(dyn);      // one histogram per rank slot
-    const uint32_t high_mask = ~((1u << (shift + kSelBits)) - 1u);
+    uint32_t (*sh)[kFhHistWords] = reinterpret_cast<uint32_t (*)[kFhHistWords]>(dyn);
+    constexpr int kShift = kResid ? kSel3Bits : 0;            // lowest bit of this pass's digit
+    constexpr int kBits = kResid ? kSelBits : kSel3Bits;      // width of the digit
+    constexpr int kSl = kTile / (kThreads * 8);
+    static_assert(kSl == 2, "a tile is two slices of eight elements per thread");
     const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
-    uint32_t prefix[kRanks];
+    uint32_t prefix[kRanks], upper[kRanks];                   // upper: the prefix above this pass's digit
     bool lead[kRanks];
     int cur_block = -1;
     int64_t run_first = first;
     double acc[kResidSums] = {0.0};
+    // position of the current tile's first element in its matrix, kept by 32-bit arithmetic from tile to tile
+    int64_t row0 = 0;
+    uint32_t col0 = 0, cols_u = 1, magic = 0;
+    int64_t next_base = -1;
 
-    auto flush = [&](int blk, int64_t t_begin, int64_t t_end) {
+    auto flush = [&](int blk, int64_t t_begin) {
         if (kResid) {
             cta_reduce_store<kResidSums>(acc, fin + size_t(t_begin) * kResidSums);
-            double* rest = fin + size_t(t_begin + 1) * kResidSums;
-            for (int64_t i = threadIdx.x; i < (t_end - t_begin - 1) * kResidSums; i += kThreads) rest[i] = 0.0;
             acc[0] = 0.0;
         } else {
             __syncthreads();
@@ -302,35 +354,65 @@ final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
         for (int r = 0; r < kRanks; ++r) {
             if (!lead[r]) continue;                           // uniform over the CTA
             uint32_t* out = hist + (size_t(blk) * kRanks + r) * kSelBins;
-            for (int d = threadIdx.x; d < kSelBins; d += kThreads) {
-                const uint32_t cnt = sh[r][d];
-                if (cnt) { atomicAdd(out + d, cnt); sh[r][d] = 0u; }
+            for (int w = threadIdx.x; w < kFhHistWords; w += kThreads) {
+                const uint32_t x = sh[r][w];
+                if (x) {
+                    if (x & 0xffffu) atomicAdd(out + 2 * w, x & 0xffffu);
+                    if (x >> 16) atomicAdd(out + 2 * w + 1, x >> 16);
+                    sh[r][w] = 0u;
+                }
             }
         }
         __syncthreads();
     };
+    // n elements into bin d of rank slot r
+    auto count = [&](int r, uint32_t d, uint32_t n) { atomicAdd(&sh[r][d >> 1], n << ((d & 1u) * 16u)); };
+    // floor(x / cols_u) for x < 2^32 from the precomputed floor((2^32 - 1) / cols_u): the estimate is at most 2 short
+    auto divmod = [&](uint32_t x, uint32_t& rem) {
+        uint32_t q = __umulhi(x, magic);
+        rem = x - q * cols_u;
+        if (rem >= cols_u) { rem -= cols_u; ++q; }
+        if (rem >= cols_u) { rem -= cols_u; ++q; }
+        return q;
+    };
 
-    for (int i = threadIdx.x; i < kRanks * kSelBins; i += kThreads) (&sh[0][0])[i] = 0u;
+    for (int i = threadIdx.x; i < kRanks * kFhHistWords; i += kThreads) (&sh[0][0])[i] = 0u;
     __syncthreads();
 
 #pragma unroll 1
     for (int64_t ti = first; ti < last; ++ti) {
         const Tile t = tiles[ti];
+        const StatBlock* b = blocks + t.block;
+        const int64_t base = int64_t(t.piece) * kTile;
         if (int(t.block) != cur_block) {                      // uniform over the CTA
-            if (cur_block >= 0) flush(cur_block, run_first, ti);
+            if (cur_block >= 0) flush(cur_block, run_first);
             cur_block = int(t.block);
             run_first = ti;
 #pragma unroll
             for (int r = 0; r < kRanks; ++r) {
                 const RankSel s = sel[size_t(t.block) * kRanks + r];
                 prefix[r] = s.prefix; lead[r] = s.leader == r;
+                upper[r] = s.prefix >> (kShift + kBits);
+            }
+            if (kResid) {
+                cols_u = uint32_t(b->cols);
+                magic = 0xffffffffu / cols_u;
+                next_base = -1;
             }
         }
-        const StatBlock* b = blocks + t.block;
         const int64_t numel = b->numel;
+        if (kResid && cols_u > 1u) {
+            if (base == next_base) {                          // the next piece of the same matrix: advance by one tile
+                uint32_t rem;
+                row0 += divmod(col0 + uint32_t(kTile), rem);
+                col0 = rem;
+            } else {
+                row0 = base / int64_t(cols_u);
+                col0 = uint32_t(base - row0 * int64_t(cols_u));
+            }
+            next_base = base + kTile;
+        }
         const uint32_t* __restrict__ v = reinterpret_cast<const uint32_t*>(b->v);
-        const int64_t base = int64_t(t.piece) * kTile;
-        constexpr int kSl = kTile / (kThreads * 8);
         uint32_t u[8 * kSl];
         int valid[kSl];
 #pragma unroll
@@ -342,8 +424,9 @@ final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
             u[8 * h + 0] = a.x; u[8 * h + 1] = a.y; u[8 * h + 2] = a.z; u[8 * h + 3] = a.w;
             u[8 * h + 4] = c.x; u[8 * h + 5] = c.y; u[8 * h + 6] = c.z; u[8 * h + 7] = c.w;
         }
-        if (kResid && b->cols > 1) {
-            const int cols = b->cols;
+        const bool tile_full = base + kTile <= numel;         // uniform over the CTA
+
+        if (kResid && cols_u > 1u) {
             const double* __restrict__ rowsum = b->rowsum;
             const double* __restrict__ colsum = b->colsum;
             const double total = rowsum[b->rows];             // the block's sum of v, left there by the row/column combine
@@ -351,53 +434,58 @@ final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
 #pragma unroll
             for (int h = 0; h < kSl; ++h) {
                 if (valid[h] == 0) continue;
-                const int64_t e = base + int64_t(h) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
-                int64_t r = e / cols;
-                int c = int(e - r * cols);
+                uint32_t c;
+                int64_t r = row0 + divmod(col0 + uint32_t(h * (kThreads * 8) + threadIdx.x * 8), c);
                 double rs = __ldg(rowsum + r) * inv_total;
-                if (valid[h] == 8 && (cols & 7) == 0) {
+                if (valid[h] == 8 && (cols_u & 7u) == 0u) {
                     // the eight elements lie in one row: one row sum, four 16-byte loads of column sums
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const double2 w = __ldg(reinterpret_cast<const double2*>(colsum + c) + q);
-                        const double d0 = double(__uint_as_float(u[8 * h + 2 * q])) - rs * w.x;
-                        const double d1 = double(__uint_as_float(u[8 * h + 2 * q + 1])) - rs * w.y;
-                        acc[0] += d0 * d0;
-                        acc[0] += d1 * d1;
+                        const double d0 = fma(-rs, w.x, double(__uint_as_float(u[8 * h + 2 * q])));
+                        const double d1 = fma(-rs, w.y, double(__uint_as_float(u[8 * h + 2 * q + 1])));
+                        acc[0] = fma(d0, d0, acc[0]);
+                        acc[0] = fma(d1, d1, acc[0]);
                     }
                 } else {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         if (j < valid[h]) {
-                            const double diff = double(__uint_as_float(u[8 * h + j])) - rs * __ldg(colsum + c);
-                            acc[0] += diff * diff;
-                            if (++c == cols) { c = 0; ++r; if (j + 1 < valid[h]) rs = __ldg(rowsum + r) * inv_total; }
+                            const double diff = fma(-rs, __ldg(colsum + c), double(__uint_as_float(u[8 * h + j])));
+                            acc[0] = fma(diff, diff, acc[0]);
+                            if (++c == cols_u) { c = 0u; ++r; if (j + 1 < valid[h]) rs = __ldg(rowsum + r) * inv_total; }
                         }
                     }
                 }
             }
         }
+
+        // ---- the histogram of this pass's digit
+        uint32_t differ = 0u;
+        bool any = false;
 #pragma unroll
-        for (int r = 0; r < kRanks; ++r) {
-            if (!lead[r]) continue;
-            int cur = -1;
-            uint32_t n = 0u;
+        for (int j = 0; j < 8 * kSl; ++j) {
+            differ |= u[j] ^ u[0];
+            const uint32_t key = u[j] >> (kShift + kBits);
+            any |= (tile_full || (j & 7) < valid[j >> 3]) &
+                   ((key == upper[0]) | (key == upper[1]) | (key == upper[2]) | (key == upper[3]));
+        }
+        if (any) {
 #pragma unroll
-            for (int k = 0; k < 8 * kSl; ++k) {
-                if ((k & 7) < valid[k >> 3] && ((u[k] ^ prefix[r]) & high_mask) == 0u) {
-                    const int d = int((u[k] >> shift) & uint32_t(kSelBins - 1));
-                    if (d == cur) {
-                        ++n;
-                    } else {
-                        if (n) atomicAdd(&sh[r][cur], n);
-                        cur = d; n = 1u;
-                    }
+            for (int r = 0; r < kRanks; ++r) {
+                if (!lead[r]) continue;
+                if (tile_full && differ == 0u) {
+                    if ((u[0] >> (kShift + kBits)) == upper[r]) count(r, (u[0] >> kShift) & ((1u << kBits) - 1u), uint32_t(8 * kSl));
+                    continue;
                 }
+#pragma unroll
+                for (int j = 0; j < 8 * kSl; ++j)
+                    if ((tile_full || (j & 7) < valid[j >> 3]) && (u[j] >> (kShift + kBits)) == upper[r])
+                        count(r, (u[j] >> kShift) & ((1u << kBits) - 1u), 1u);
             }
-            if (n) atomicAdd(&sh[r][cur], n);
         }
     }
-    if (cur_block >= 0) flush(cur_block, run_first, last);
+    if (cur_block >= 0) flush(cur_block, run_first);
 }
 
 // One CTA per block: for each of the four ranks find the bin of its leader's
@@ -516,30 +604,30 @@ int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* c
     final_sums_kernel<<<unsigned((n_tiles + per - 1) / per), kThreads, kFsSmemBytes, s>>>(
         blocks, tiles, params, fin, fin_out, hist, n_tiles, per, float(eps), eps_adam);
     BAOC_LAUNCH_CHECK();
-    final_sums_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out);
+    final_sums_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
     BAOC_LAUNCH_CHECK();
-    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, 24, 256);
+    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, 32 - kSelBits, kSelBins);
     BAOC_LAUNCH_CHECK();
     return 0;
 }
 
 int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
                               uint32_t* hist, const double* acc, int64_t n_tiles, int n_blocks, cudaStream_t s) {
-    constexpr int kSmem = kRanks * kSelBins * int(sizeof(uint32_t));
+    constexpr int kSmem = kFhSmemBytes;
     cudaError_t e = cudaFuncSetAttribute(final_hist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(final_hist_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return int(e);
     const int per = run_tiles(n_tiles, kSelRunTiles);
     const unsigned grid = unsigned((n_tiles + per - 1) / per);
-    final_hist_kernel<true><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per, kSelBits);
+    final_hist_kernel<true><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per);
     BAOC_LAUNCH_CHECK();
-    final_resid_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out);
+    final_resid_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
     BAOC_LAUNCH_CHECK();
-    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, kSelBits, kSelBins);
+    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, kSel3Bits, kSelBins);
     BAOC_LAUNCH_CHECK();
-    final_hist_kernel<false><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per, 0);
+    final_hist_kernel<false><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per);
     BAOC_LAUNCH_CHECK();
-    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, 0, kSelBins);
+    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, 0, 1 << kSel3Bits);
     BAOC_LAUNCH_CHECK();
     const int tb = 128, gb = (n_blocks + tb - 1) / tb;
     stats_gather_kernel<<<gb, tb, 0, s>>>(sel, acc, fin_out, n_blocks);

@@ -35,10 +35,11 @@ constexpr int kFinRanks = 16;         //   [0..15] first-sweep sums, [16..19] th
 constexpr int kFinAcc = 20;           //   [20..27] the running window values,
 constexpr int kFinResid = 28;         //   [28] the Eq. 7 numerator,
 constexpr int kFinPilot = 29;         //   [29] the pilot value of the Eq. 6 preconditioner
-constexpr int kSelBits = 12;          // bits per radix pass of the quantile select after the first one (which takes the top byte)
+constexpr int kSelBits = 12;          // bits of the first and of the second radix pass of the quantile select
 constexpr int kSelBins = 1 << kSelBits;
+constexpr int kSel3Bits = 32 - 2 * kSelBits;   // bits of the third and last pass
 constexpr int kFinRunTiles = 8;       // most tiles a CTA of the first finalize sweep works through (its partial sums stay in fp32 that long)
-constexpr int kSelRunTiles = 64;      // most tiles a CTA of the other two sweeps works through
+constexpr int kSelRunTiles = 15;      // most tiles a CTA of the other two sweeps works through (their histograms count in 16 bits)
 constexpr int kRedRows = 64;          // rows per CTA of the row/column reduction kernel
 constexpr int kRedCols = 512;         // columns per CTA of the row/column reduction kernel
 constexpr int kTileF = 16384;         // elements per tile of the factored path (its slices are prefetched through shared memory)

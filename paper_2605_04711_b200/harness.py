@@ -51,6 +51,19 @@ def sum_over_ranks(value: float, dist=None, device="cpu") -> float:
     return float(t.item())
 
 
+def all_gather_params(local: torch.Tensor, out: torch.Tensor, dist) -> None:
+    """The one exchange of a whole-block sharded step when replicas hold full weights: every rank contributes its flat
+    parameter buffer ``local`` (all ranks' buffers have the same length, the longest shard's) and receives all of them
+    in ``out`` (world x that length; rank r's block that starts at offset o of its buffer lies at r * len(local) + o).
+    Queued behind the step on the current stream; NCCL on GPUs, gloo in the CPU tests."""
+    if out.numel() != local.numel() * dist.get_world_size():
+        raise ValueError("out must hold one buffer of local's length per rank")
+    try:
+        dist.all_gather_into_tensor(out, local)
+    except (RuntimeError, NotImplementedError):               # a backend without the flat form
+        dist.all_gather(list(out.view(dist.get_world_size(), -1).unbind(0)), local)
+
+
 class Session:
     """One workload resident on one GPU.
 
@@ -60,14 +73,17 @@ class Session:
     """
 
     def __init__(self, wl: W.Workload, configs: Optional[Sequence[B.Config]] = None, opts: Optional[B.Opts] = None,
-                 n_grad_sets: int = 2, device: str = "cuda:0", pinned_host_grads: bool = False, samples=None):
+                 n_grad_sets: int = 2, device: str = "cuda:0", pinned_host_grads: bool = False, samples=None,
+                 param_capacity: int = 0):
         self.wl = wl
         self.device = torch.device(device)
         self.configs = list(configs) if configs is not None else B.default_configs()
         self.h = B.Baoc(wl.blocks, self.configs, opts)
         self.offs, self.total = W.flat_layout(wl, 128)
         self.n_grad_sets = n_grad_sets
-        self.params = torch.zeros(self.total, dtype=torch.float32, device=self.device)
+        # param_capacity: allocate the parameter buffer at least this long (the longest shard's length, so that the
+        # buffers of all ranks can be all-gathered as they are)
+        self.params = torch.zeros(max(self.total, int(param_capacity)), dtype=torch.float32, device=self.device)
         self.grads = [torch.zeros(self.total, dtype=torch.bfloat16, device=self.device) for _ in range(n_grad_sets)]
         self.param_views = [self.params[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)]
         self.grad_views = [[g[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)] for g in self.grads]
