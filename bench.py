@@ -275,7 +275,8 @@ def run_ours(args):
     # optional: the statistics see a seeded sub-grid of every block (the paper's sparse coordinate sampling)
     samples = W.sample_subgrids(wl, args.sample_frac) if args.sample_frac < 1.0 else None
     sess = harness.Session(wl, configs=binding.extended_configs() if extended else None, n_grad_sets=2,
-                           device=f"cuda:{local}", pinned_host_grads=True, samples=samples, param_capacity=cap)
+                           device=f"cuda:{local}", pinned_host_grads=True, samples=samples, param_capacity=cap,
+                           factored_group_bytes=int(args.factored_group_mb * 2 ** 20))
     gathered = torch.empty(world * cap, dtype=torch.float32, device=f"cuda:{local}") if sharded else None
     # after a sharded step: all ranks receive all updated parameters
     exchange = (lambda: harness.all_gather_params(sess.params, gathered, dist)) if sharded else (lambda: None)
@@ -419,7 +420,7 @@ def run_ours(args):
                    "param_dtype": "f32", "candidate_configs": names, "assignment": args.assign,
                    "assignment_blocks_per_config": counts, "assignment_params_per_config": params_by_cfg,
                    "mem_budget_frac_of_fp32_adam": wl.mem_budget_frac, "state_bytes": int(info.state_bytes),
-                   "window_steps_before_timing": args.window, "stats_sample_frac": args.sample_frac, "l2": "inputs (>10 GB per step) far exceed the 126 MB L2",
+                   "window_steps_before_timing": args.window, "stats_sample_frac": args.sample_frac, "factored_group_mb": args.factored_group_mb, "l2": "inputs (>10 GB per step) far exceed the 126 MB L2",
                    "parallelism": (f"whole blocks sharded over {world} GPUs; no collective in the statistics pass or the update; "
                                    f"NCCL all-gather of the updated parameters ({4 * cap} bytes per rank) inside the timed region"
                                    if sharded else f"replicas x{world}, no collective") if world > 1 else "single GPU",
@@ -459,6 +460,9 @@ def main():
     ap.add_argument("--sample-frac", type=float, default=1.0,
                     help="fraction of every block's coordinates the statistics see (1 = dense, the default; the paper's own "
                          "default is 0.001)")
+    ap.add_argument("--factored-group-mb", type=float, default=0.0,
+                    help="0: one row/column reduction and one update launch for all factored blocks; > 0: factored blocks in groups "
+                         "of at most this many MiB of gradient, each reduced and updated back to back (second read from L2)")
     ap.add_argument("--window", type=int, default=4, help="statistics steps before the finalize that feeds the allocation")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-sample-params", type=int, default=100_000_000)

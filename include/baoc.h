@@ -341,6 +341,20 @@ int baoc_configure_from_window(baoc_t* h, const int32_t* assign, void* state_dev
 int baoc_step(baoc_t* h, const void* const* grads, float* const* params,
               int64_t step_t, baoc_stream_t stream);
 
+/* Schedule of the factored blocks inside baoc_step.  The factored second moment
+ * needs the row and column sums of g*g of a whole matrix before any element of
+ * that matrix can be updated, so its gradient is read twice: by the reduction,
+ * then by the update.  group_bytes == 0 (the default): one reduction over all
+ * factored blocks, then one update launch for all blocks.  group_bytes > 0:
+ * the factored blocks are taken in groups of whole blocks of at most that many
+ * bytes of gradient (a larger block forms a group alone), and every group runs
+ * its reduction, the combine and its update tiles back to back, so that the
+ * second read can be served from L2 (which holds 126 MB on B200); the results
+ * are bit-identical, the step then takes 3 launches per group.  Call before
+ * baoc_configure (BAOC_E_STATE afterwards).  Definition 3.1 fixes what is
+ * computed, not in which order the blocks are visited. */
+int baoc_set_factored_schedule(baoc_t* h, int64_t group_bytes);
+
 /* End-to-end convenience for callers whose gradients live in host memory:
  * copies block i's bf16 gradient from host_grads[i] (pinned memory advised) to
  * the device buffer dev_grads[i], then does baoc_sample_stats (if do_stats)
@@ -402,7 +416,9 @@ int baoc_import(baoc_t* h, const void* blob, size_t size, void* ws_dev, size_t w
  * kernels and around the fused update kernel (events are created on the first
  * enable; no device memory is involved).  baoc_profile_last waits for the last
  * step and writes ms[0] = row/column kernels (0 when no block is factored),
- * ms[1] = fused update kernel.  BAOC_E_STATE if profiling is off or no step ran. */
+ * ms[1] = fused update kernel (with a grouped factored schedule the kernels
+ * alternate: ms[0] = 0 and ms[1] = the whole step).  BAOC_E_STATE if profiling
+ * is off or no step ran. */
 int baoc_profile(baoc_t* h, int enable);
 int baoc_profile_last(baoc_t* h, float* ms2);
 

@@ -80,7 +80,8 @@ EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error"
            "baoc_configure", "baoc_step", "baoc_step_from_host", "baoc_view", "baoc_nonfinite",
            "baoc_sample_stats_noalloc", "baoc_noalloc_last_error", "baoc_profile", "baoc_profile_last",
            "baoc_export", "baoc_import", "baoc_time_scratch_bytes", "baoc_measure_time_ratios",
-           "baoc_set_sampling", "baoc_reconfigure", "baoc_configure_from_window", "baoc_partition"]
+           "baoc_set_sampling", "baoc_reconfigure", "baoc_configure_from_window", "baoc_partition",
+           "baoc_set_factored_schedule"]
 
 _vp = C.c_void_p
 _lib.baoc_default_opts.argtypes = [C.POINTER(Opts)]
@@ -113,6 +114,7 @@ _lib.baoc_time_scratch_bytes.argtypes = [_vp, C.POINTER(C.c_size_t)]
 _lib.baoc_measure_time_ratios.argtypes = [_vp, _vp, _vp, _vp, C.c_size_t, C.c_int, C.c_int, _vp, _vp, _vp]
 _lib.baoc_export.argtypes = [_vp, _vp, C.c_size_t, C.POINTER(C.c_size_t)]
 _lib.baoc_import.argtypes = [_vp, _vp, C.c_size_t, _vp, C.c_size_t, _vp, C.c_size_t, _vp]
+_lib.baoc_set_factored_schedule.argtypes = [_vp, C.c_int64]
 _lib.baoc_profile.argtypes = [_vp, C.c_int]
 _lib.baoc_profile_last.argtypes = [_vp, C.POINTER(C.c_float)]
 _lib.baoc_sample_stats_noalloc.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_double, C.c_double, C.c_double, _vp, _vp]
@@ -408,6 +410,11 @@ class Baoc:
         for t in (ws, state):
             if t is not None:
                 self._keep.append(t)
+
+    def set_factored_schedule(self, group_bytes: int):
+        """``baoc_set_factored_schedule``: 0 = one reduction and one update launch; > 0 = factored blocks in groups of
+        at most that many gradient bytes, each reduced and updated back to back (before ``configure``)."""
+        self._check(_lib.baoc_set_factored_schedule(self._h, int(group_bytes)))
 
     def profile(self, enable: bool):
         self._check(_lib.baoc_profile(self._h, int(bool(enable))))

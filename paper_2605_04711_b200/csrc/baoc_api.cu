@@ -185,8 +185,9 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
     int rc = step_prologue(h, grads, params, t, s, &P);
     if (rc) return rc;
     const auto& L = h->tl;
+    const bool grouped = h->factored_group_bytes > 0 && h->n_factored > 0;
     if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[0]), s), "baoc_step (profile)");
-    if (h->n_factored > 0) {
+    if (h->n_factored > 0 && !grouped) {
         LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles),
                                       at<int32_t>(h->st, L.f_ids), at<const void*>(h->st, L.grads),
                                       at<const float*>(h->st, L.params), h->n_step_red_tiles, h->n_factored, P, s),
@@ -197,10 +198,29 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
     int64_t first = 0;
     for (int fam = 0; fam < kFamCount; ++fam) {
         if (h->fam_tiles[fam] == 0) continue;
-        LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles) + first, at<const void*>(h->st, L.grads),
-                                 at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), h->fam_tiles[fam], fam, P, s),
-               "fused_step_kernel");
-        h->launches += 1;
+        // grouped schedule: the headline family's launch stops before the factored tiles, which close its stretch
+        const int64_t here = (grouped && fam == kFamHead) ? h->fam_tiles[fam] - h->n_factored_tiles : h->fam_tiles[fam];
+        if (here > 0) {
+            LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles) + first, at<const void*>(h->st, L.grads),
+                                     at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), here, fam, P, s),
+                   "fused_step_kernel");
+            h->launches += 1;
+        }
+        if (grouped && fam == kFamHead) {
+            // every group: row/column reduction, its combine, then the group's update tiles, back to back
+            const int64_t f_first = first + here;
+            for (const Handle::FactoredGroup& g : h->f_groups) {
+                LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles) + g.red0,
+                                              at<int32_t>(h->st, L.f_ids) + g.f0, at<const void*>(h->st, L.grads),
+                                              at<const float*>(h->st, L.params), g.n_red, g.n_f, P, s),
+                       "factored_reduce_kernel");
+                LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles) + f_first + g.tile0,
+                                         at<const void*>(h->st, L.grads), at<float*>(h->st, L.params),
+                                         at<uint32_t>(h->st, L.flags), g.n_tiles, kFamHead, P, s),
+                       "fused_step_kernel");
+                h->launches += 3;
+            }
+        }
         first += h->fam_tiles[fam];
     }
     if (h->prof_on) {
@@ -490,6 +510,25 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
     if (!ids.empty())
         CU(cudaMemcpyAsync(st + L.f_ids, ids.data(), 4 * ids.size(), cudaMemcpyHostToDevice, s), "upload factored ids");
     if (reset || zero_only) CU(cudaMemsetAsync(st + L.flags, 0, L.total - L.flags, s), "zero optimizer state");
+    {   // factored blocks in index order: that is their order in the tile table, the reduction table and the id list
+        h->f_groups.clear();
+        h->n_factored_tiles = 0;
+        Handle::FactoredGroup g{0, 0, 0, 0, 0, 0};
+        int64_t bytes_in_group = 0;
+        for (int i = 0; i < n; ++i) {
+            if (sb[i].path != kPathF) continue;
+            const int64_t gb = 2 * sb[i].numel, nt = ceil_div(sb[i].numel, kTileF), nr = int64_t(sb[i].red.chunks) * sb[i].red.strips;
+            if (g.n_f > 0 && bytes_in_group + gb > h->factored_group_bytes) {
+                h->f_groups.push_back(g);
+                g = Handle::FactoredGroup{g.tile0 + g.n_tiles, 0, g.red0 + g.n_red, 0, g.f0 + g.n_f, 0};
+                bytes_in_group = 0;
+            }
+            g.n_tiles += nt; g.n_red += nr; g.n_f += 1;
+            bytes_in_group += gb;
+            h->n_factored_tiles += nt;
+        }
+        if (g.n_f > 0) h->f_groups.push_back(g);
+    }
     h->st = st; h->st_bytes = bytes; h->tl = L; h->configured = true;
     h->assign.assign(assign, assign + n);
     h->h_step_blocks = sb;
@@ -907,6 +946,14 @@ int baoc_step_from_host(baoc_t* h, const void* const* host_grads, void* const* d
 }
 
 
+
+int baoc_set_factored_schedule(baoc_t* h, int64_t group_bytes) {
+    if (!h) return BAOC_E_INVALID;
+    if (group_bytes < 0) return fail(h, BAOC_E_INVALID, "baoc_set_factored_schedule: negative size");
+    if (h->configured) return fail(h, BAOC_E_STATE, "baoc_set_factored_schedule: set the schedule before baoc_configure");
+    h->factored_group_bytes = group_bytes;
+    return BAOC_OK;
+}
 
 int baoc_profile(baoc_t* h, int enable) {
     if (!h) return BAOC_E_INVALID;

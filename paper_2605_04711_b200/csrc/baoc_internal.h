@@ -268,6 +268,15 @@ struct Handle {
     };
     std::vector<GroupStep> groups;
     std::vector<Tile> group_tiles;       // staging of the by-group table (must outlive the asynchronous upload)
+    // Optional schedule of the factored blocks in baoc_step: groups of whole factored blocks of at most
+    // factored_group_bytes of gradient each take their row/column reduction, its combine and their update tiles back to
+    // back, so that the update's second read of the gradient can come from L2 (0: one reduction and one update launch
+    // for all blocks).  A group is a stretch of the reduction table, of the list of factored blocks and of the main
+    // tile table (the factored tiles close the headline family's stretch, block by block).
+    struct FactoredGroup { int64_t tile0, n_tiles, red0, n_red; int32_t f0, n_f; };
+    int64_t factored_group_bytes = 0;
+    std::vector<FactoredGroup> f_groups;
+    int64_t n_factored_tiles = 0;
 
     // optional per-kernel timing of the step (CUDA events, owned by the CUDA translation unit)
     bool prof_on = false, prof_valid = false;

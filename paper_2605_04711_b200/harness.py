@@ -74,7 +74,7 @@ class Session:
 
     def __init__(self, wl: W.Workload, configs: Optional[Sequence[B.Config]] = None, opts: Optional[B.Opts] = None,
                  n_grad_sets: int = 2, device: str = "cuda:0", pinned_host_grads: bool = False, samples=None,
-                 param_capacity: int = 0):
+                 param_capacity: int = 0, factored_group_bytes: int = 0):
         self.wl = wl
         self.device = torch.device(device)
         self.configs = list(configs) if configs is not None else B.default_configs()
@@ -94,6 +94,8 @@ class Session:
             self.host_grads = [torch.zeros(self.total, dtype=torch.bfloat16).pin_memory() for _ in range(n_grad_sets)]
             self.host_tables = [B.pointer_table([hg[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)])
                                 for hg in self.host_grads]
+        if factored_group_bytes:
+            self.h.set_factored_schedule(factored_group_bytes)
         self.samples = samples
         if samples is not None:
             self.h.set_sampling(samples)

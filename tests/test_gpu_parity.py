@@ -571,6 +571,33 @@ def test_factored_bf16_statistics_free_running_ten_steps(B, H):
     assert codes[0] <= 1e-4 * codes[1], codes
 
 
+def test_grouped_factored_schedule_is_bit_identical(B, H):
+    """baoc_set_factored_schedule: factored blocks reduced and updated group by group (so that the second read of the
+    gradient can come from L2) leave exactly what the one-reduction schedule leaves: parameters and every state tensor,
+    over three mixed steps, with groups of one block, of a few blocks, and one group for all."""
+    wl = W.make_workload("toy", seed=2)
+    assign = [3 if b.cols > 1 and i % 3 != 2 else (i % 5 if i % 5 != 3 else 0) for i, b in enumerate(wl.blocks)]
+    assert assign.count(3) >= 4
+    res = []
+    for group_bytes in (0, 1, 3 * 2 * 256 * 256, 1 << 40):
+        sess = H.Session(wl, n_grad_sets=1, factored_group_bytes=group_bytes)
+        sess.init_params()
+        sess.configure(assign)
+        launches0 = sess.h.query().kernel_launches
+        for t in (1, 2, 3):
+            sess.fill_grads(t)
+            sess.step(0, t)
+        torch.cuda.synchronize()
+        res.append((sess.params.clone(), _state_tensors(sess, B), sess.h.query().kernel_launches - launches0))
+    for other in res[1:]:
+        assert torch.equal(res[0][0], other[0])
+        assert len(res[0][1]) == len(other[1]) > 0
+        for x, y in zip(res[0][1], other[1]):
+            assert torch.equal(x, y)
+    assert res[0][2] == 3 * 3 and res[3][2] == 3 * 4                  # one group: reduce, combine, the rest, the factored tiles
+    assert res[1][2] == 3 * (1 + 3 * assign.count(3))                 # a group per factored block
+
+
 def test_nonfinite_gradient_is_flagged_not_fatal(B, H):
     wl = _odd_workload(seed=31)
     sess = H.Session(wl, n_grad_sets=1)
