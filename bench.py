@@ -152,22 +152,30 @@ class ClockSampler(threading.Thread):
 # CPU oracle timing (the reference arm and the cpu_baseline leg)
 # ----------------------------------------------------------------------------
 
-def _sample_blocks(wl, target_params):
-    """A bounded sample of the workload: blocks in order (skipping any larger than the target) until the target is met."""
+def _sample_blocks(wl, target_params, slice_rows=False):
+    """A bounded sample of the workload: blocks in order until the target is met.  Without slicing, blocks larger than
+    the target are skipped; with slicing, a matrix larger than a quarter of the target is cut to its first rows (whole
+    rows, so it stays a matrix and every path, the factored one included, can run on it).  Returns
+    ([(block index, rows, cols)], parameters)."""
     picked, total = [], 0
+    cap = max(1, target_params // 4)
     for i, b in enumerate(wl.blocks):
-        if b.numel > target_params:
+        rows, cols = b.rows, b.cols
+        if slice_rows and b.numel > cap:
+            rows = max(1, cap // cols) if cols > 1 else cap
+        elif b.numel > target_params:
             continue
-        picked.append(i)
-        total += b.numel
+        picked.append((i, rows, cols))
+        total += rows * cols
         if total >= target_params:
             break
     return picked, total
 
 
-def time_oracle(wl, assign, steps, warmup, target_params, configs=None):
+def time_oracle(wl, assign, steps, warmup, target_params, configs=None, slice_rows=False):
     """Time the oracle's statistics step + optimizer step on a sample of blocks.  Returns (params/s, info).
-    configs: the candidate tuples ``assign`` indexes (the binding's structs); default: the oracle's five."""
+    configs: the candidate tuples ``assign`` indexes (the binding's structs); default: the oracle's five.
+    assign None: the sampled blocks take the candidates in turn (vectors skip the factored one)."""
     import numpy as np
     from threadpoolctl import threadpool_limits
     from oracle import baoc_oracle as O
@@ -182,35 +190,38 @@ def time_oracle(wl, assign, steps, warmup, target_params, configs=None):
     else:
         cfgs = [O.Config(c.adaptive, c.momentum, c.decoupled_wd, c.factored, c.bits, lr=float(c.lr), beta1=float(c.beta1),
                          beta2=float(c.beta2), eps=float(c.eps), weight_decay=float(c.weight_decay)) for c in configs]
-    picked, total = _sample_blocks(wl, target_params)
+    picked, total = _sample_blocks(wl, target_params, slice_rows)
     opts = O.Opts()
+    kinds = []
     with threadpool_limits(limits=1):
-        grads = [[W.block_grad(wl, i, t).double().numpy() for i in picked] for t in (1, 2)]
-        theta = [W.block_param(wl, i).double().numpy() for i in picked]
-        sstates = [O.stats_init(wl.blocks[i].numel) for i in picked]
+        grads = [[W.block_grad(wl, i, t).double().numpy()[:r * c] for i, r, c in picked] for t in (1, 2)]
+        theta = [W.block_param(wl, i).double().numpy()[:r * c] for i, r, c in picked]
+        sstates = [O.stats_init(r * c) for _, r, c in picked]
         ostates = []
-        for j, i in enumerate(picked):
-            b = wl.blocks[i]
-            c = int(assign[i]) if assign is not None else (j % 5)
-            if cfgs[c].factored and b.cols <= 1:
+        for j, (i, r, c_) in enumerate(picked):
+            c = int(assign[i]) if assign is not None else (j % len(cfgs))
+            if cfgs[c].factored and c_ <= 1:
                 c = 2
-            ostates.append((c, O.step_init(cfgs[c], b.numel, b.rows, b.cols)))
+            ostates.append((c, O.step_init(cfgs[c], r * c_, r, c_)))
+            kinds.append(O.config_kind(cfgs[c]))
         times = []
         for s in range(warmup + steps):
             t0 = time.perf_counter()
-            for j, i in enumerate(picked):
-                b = wl.blocks[i]
+            for j, (i, r, c_) in enumerate(picked):
                 g = grads[s % 2][j]
                 O.stats_step(sstates[j], g, opts)
                 c, st = ostates[j]
-                theta[j] = O.step(theta[j], g, st, cfgs[c], b.rows, b.cols)
+                theta[j] = O.step(theta[j], g, st, cfgs[c], r, c_)
             dt = time.perf_counter() - t0
             if s >= warmup:
                 times.append(dt)
     sec = sum(times) / len(times)
+    sliced = sum(1 for i, r, c in picked if r * c < wl.blocks[i].numel)
     info = {"kind": "oracle", "cores": 1, "unit": UNIT, "value": total / sec,
-            "sample": f"{len(picked)} blocks / {total} params of {wl.name} (first blocks up to {target_params} params), "
-                      f"one statistics step + one optimizer step per timed step, {len(times)} timed steps, numpy float64, 1 thread",
+            "sample": f"{len(picked)} blocks / {total} params of {wl.name} (blocks in order up to {target_params} params"
+                      + (f", {sliced} matrices cut to their first rows" if slice_rows else ", larger blocks skipped")
+                      + f"; update paths {'/'.join(sorted(set(kinds)))}), one statistics step + one optimizer step per timed step, "
+                      f"{len(times)} timed steps, numpy float64, 1 thread",
             "ms_per_step": sec * 1e3}
     return total / sec, info
 
@@ -221,9 +232,10 @@ def run_reference(args):
         return
     from paper_2605_04711_b200 import workloads as W
     wl = W.make_workload(args.workload, seed=0)
-    # size the sample so that warmup + steps stay within a few minutes on one core
-    target = max(1 << 20, int(6.0e7 / max(args.steps + args.warmup, 1)))
-    value, info = time_oracle(wl, None, args.steps, args.warmup, target)
+    # size the sample so that warmup + steps stay within a few minutes on one core (the oracle does about 3e7 parameters
+    # per second); large matrices are cut to their first rows so that the sample holds matrices and every update path
+    target = max(1 << 20, int(6.0e8 / max(args.steps + args.warmup, 1)))
+    value, info = time_oracle(wl, None, args.steps, args.warmup, target, slice_rows=True)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": info["ms_per_step"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -326,18 +338,25 @@ def run_ours(args):
         dist.barrier()
         torch.cuda.synchronize()
 
+    # L2: a step of the large workloads streams many times the 126 MB of L2; a workload whose step moves less than
+    # 1 GB gets L2 flushed (a 256 MB buffer overwritten) before every timed step, outside the timed intervals
+    flush_l2 = (stats_bytes + step_bytes) < (1 << 30)
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=f"cuda:{local}") if flush_l2 else None
     launches0 = sess.h.query().kernel_launches
     sampler = ClockSampler(local)
     sampler.start()
-    marks = [ev() for _ in range(2 * args.steps + 1)]
-    marks[0].record()
+    marks = [(ev(), ev(), ev()) for _ in range(args.steps)]
     for s in range(args.steps):
         step_t += 1
+        if flush_l2:
+            flush_buf.fill_(s & 0xff)
+        a, b, c = marks[s]
+        a.record()
         sess.sample_stats(s % 2)
-        marks[2 * s + 1].record()
+        b.record()
         sess.step(s % 2, step_t)
         exchange()
-        marks[2 * s + 2].record()
+        c.record()
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
@@ -345,9 +364,10 @@ def run_ours(args):
     sampler.stop()
     launches = sess.h.query().kernel_launches - launches0
 
-    total_ms = marks[0].elapsed_time(marks[-1])
-    stats_ms = sum(marks[2 * s].elapsed_time(marks[2 * s + 1]) for s in range(args.steps)) / args.steps
-    step_ms = sum(marks[2 * s + 1].elapsed_time(marks[2 * s + 2]) for s in range(args.steps)) / args.steps
+    # the K steps run back to back on one stream; with the L2 flush in between only the steps themselves are counted
+    total_ms = (sum(a.elapsed_time(c) for a, b, c in marks) if flush_l2 else marks[0][0].elapsed_time(marks[-1][2]))
+    stats_ms = sum(a.elapsed_time(b) for a, b, c in marks) / args.steps
+    step_ms = sum(b.elapsed_time(c) for a, b, c in marks) / args.steps
     dev = f"cuda:{local}"
     total_ms_max = harness.max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms_max / args.steps
@@ -355,18 +375,26 @@ def run_ours(args):
     value = all_params / (ms_per_step * 1e-3)
     cnt, _ = sess.h.nonfinite()
 
-    # per-kernel split of the step (events inside the library around the fused kernel), on a few more steps
+    # per-kernel split of the step (events inside the library around the row/column kernels and the fused kernel), on a
+    # few more steps; the same loop also brackets the whole baoc_step call, so parts and whole come from one loop.  The
+    # loop reads its events back after every step (a host synchronisation), which the main timed loop does not have.
     sess.h.profile(True)
-    red_ms, fused_ms = [], []
+    red_ms, fused_ms, whole_ms = [], [], []
     for s in range(min(args.steps, 20)):
         step_t += 1
         sess.sample_stats(s % 2)
+        w0, w1 = ev(), ev()
+        w0.record()
         sess.step(s % 2, step_t)
+        w1.record()
         a, b = sess.h.profile_last()
+        torch.cuda.synchronize()
         red_ms.append(a)
         fused_ms.append(b)
+        whole_ms.append(w0.elapsed_time(w1))
     sess.h.profile(False)
     red_ms, fused_ms = sum(red_ms) / len(red_ms), sum(fused_ms) / len(fused_ms)
+    parts_whole_ms = sum(whole_ms) / len(whole_ms)
 
     # end to end: gradients start in pinned host memory, the per-block running statistics come back
     e2e_steps = max(1, min(args.e2e_steps, args.steps))
@@ -396,20 +424,32 @@ def run_ours(args):
     step_gbs = step_bytes / (step_ms * 1e-3) / 1e9
     # the dominant kernel of the step gets the `roofline` object, the other one `roofline_other`
     n_factored = sum(n for n, c in zip(params_by_cfg, sess.configs) if c.factored)   # at any precision of their statistics
-    fused_bytes = step_bytes - 2 * n_factored              # the row/column kernels read the factored blocks' gradients once
+    # the library counts what it moves: 12 B per factored parameter (the gradient is read by the row/column reduction and
+    # again by the update); the method itself needs 10 B (one read), which is also what the fused kernel alone moves
+    algo_step_bytes = step_bytes - 2 * n_factored
+    fused_bytes = algo_step_bytes
     fused_gbs = fused_bytes / (fused_ms * 1e-3) / 1e9
+    algo_step_gbs = algo_step_bytes / (step_ms * 1e-3) / 1e9
+    peak_note = peak_kind + " (burst copy, read + write; a read-dominated kernel can exceed it: the nominal 8 TB/s is the ceiling)"
     r_stats = {"kernel": "stats_step_kernel", "bound": "hbm", "achieved": stats_gbs, "peak": peak, "unit": "GB/s",
-               "frac": stats_gbs / peak, "peak_kind": peak_kind + " (burst copy)", "frac_of_8TBs": stats_gbs / 8000.0,
+               "frac": stats_gbs / peak, "peak_kind": peak_note, "frac_of_8TBs": stats_gbs / 8000.0,
                "bytes_per_launch": int(stats_bytes), "ms": stats_ms,
                "bytes_per_param": 22 if samples is None else "26 per sampled coordinate",
                "timed": "events around baoc_sample_stats (includes its ~25 us combine kernel)",
                "traffic": args.traffic_stats if args.traffic_stats is not None else (_ncu_traffic("stats_step_kernel", stats_bytes) if samples is None else None)}
     r_fused = {"kernel": "fused_step_kernel", "bound": "hbm", "achieved": fused_gbs, "peak": peak, "unit": "GB/s",
-               "frac": fused_gbs / peak, "peak_kind": peak_kind + " (burst copy)", "frac_of_8TBs": fused_gbs / 8000.0,
+               "frac": fused_gbs / peak, "peak_kind": peak_note, "frac_of_8TBs": fused_gbs / 8000.0,
                "bytes_per_launch": int(fused_bytes), "ms": fused_ms,
-               "timed": "events inside baoc_step around the fused kernel alone",
-               "whole_step": {"ms": step_ms, "GBps": step_gbs, "frac": step_gbs / peak, "bytes": int(step_bytes),
-                              "row_col_kernels_ms": red_ms},
+               "timed": "events inside baoc_step around the fused kernel alone, in the parts loop (see parts_loop)",
+               "parts_loop": {"steps": len(whole_ms), "whole_step_ms": parts_whole_ms, "row_col_kernels_ms": red_ms,
+                              "fused_kernel_ms": fused_ms,
+                              "note": "one loop with a host synchronisation after every step; the main timed loop has none"},
+               "whole_step": {"ms": step_ms, "timed": "events around baoc_step in the main timed loop",
+                              "bytes_moved": int(step_bytes), "GBps_moved": step_gbs, "frac_moved": step_gbs / peak,
+                              "bytes_algorithmic": int(algo_step_bytes), "GBps_algorithmic": algo_step_gbs,
+                              "frac_algorithmic": algo_step_gbs / peak, "frac_algorithmic_of_8TBs": algo_step_gbs / 8000.0,
+                              "note": "moved counts the factored blocks' gradient twice (12 B/param: row/column reduction, then "
+                                      "update); algorithmic counts it once (10 B/param)"},
                "traffic": args.traffic_step if args.traffic_step is not None else _ncu_traffic("fused_step_kernel", fused_bytes)}
     roofline, other = (r_fused, r_stats) if fused_ms >= stats_ms else (r_stats, r_fused)
     line = {
@@ -420,7 +460,8 @@ def run_ours(args):
                    "param_dtype": "f32", "candidate_configs": names, "assignment": args.assign,
                    "assignment_blocks_per_config": counts, "assignment_params_per_config": params_by_cfg,
                    "mem_budget_frac_of_fp32_adam": wl.mem_budget_frac, "state_bytes": int(info.state_bytes),
-                   "window_steps_before_timing": args.window, "stats_sample_frac": args.sample_frac, "factored_group_mb": args.factored_group_mb, "l2": "inputs (>10 GB per step) far exceed the 126 MB L2",
+                   "window_steps_before_timing": args.window, "stats_sample_frac": args.sample_frac, "factored_group_mb": args.factored_group_mb, "l2": ("flushed before every timed step (a 256 MB buffer overwritten, outside the timed intervals)" if flush_l2 else
+                          f"inputs ({(stats_bytes + step_bytes) / 1e9:.1f} GB per step) far exceed the 126 MB L2"),
                    "parallelism": (f"whole blocks sharded over {world} GPUs; no collective in the statistics pass or the update; "
                                    f"NCCL all-gather of the updated parameters ({4 * cap} bytes per rank) inside the timed region"
                                    if sharded else f"replicas x{world}, no collective") if world > 1 else "single GPU",
@@ -432,7 +473,7 @@ def run_ours(args):
         "roofline": roofline,
         "roofline_other": other,
         "stats_pass": {"ms": stats_ms, "GBps": stats_gbs, "params_per_s": wl.numel / (stats_ms * 1e-3)},
-        "mixed_step": {"ms": step_ms, "GBps": step_gbs, "params_per_s": wl.numel / (step_ms * 1e-3),
+        "mixed_step": {"ms": step_ms, "GBps": step_gbs, "GBps_algorithmic": algo_step_gbs, "params_per_s": wl.numel / (step_ms * 1e-3),
                        "includes_param_all_gather": sharded},
         "once_per_window": {"finalize_and_risk_ms": finalize_ms, "allocate_ms": alloc_ms, "objective": objective},
     }

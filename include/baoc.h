@@ -422,6 +422,39 @@ int baoc_import(baoc_t* h, const void* blob, size_t size, void* ws_dev, size_t w
 int baoc_profile(baoc_t* h, int enable);
 int baoc_profile_last(baoc_t* h, float* ms2);
 
+/* ---- checked build ------------------------------------------------------------
+ * The paper has no counterpart of this.  The library can be built with
+ * -DBAOC_CHECKED (libbaoc_checked.so): every CTA of the streaming kernels of the
+ * window and of the step then validates, before it touches memory, that its tile
+ * exists, names a block of the table and starts inside it, and that every range
+ * of the bound workspace or state buffer it is about to read or write lies inside
+ * that buffer.  The first violation is recorded (nothing traps, the CTA returns,
+ * the context stays usable).  It is the stand-in for a memory checker where none
+ * can be run; caller-owned arrays are covered by guard words in the test harness.
+ *
+ * baoc_check_status: waits for the device, then writes the first recorded
+ * violation since the last call to *out and clears the records.  enabled = 1 in
+ * a checked build, 0 in a normal one (where code is always 0).  code: 0 clean,
+ * 1 tile index beyond the table, 2 block index beyond the table, 3 tile start
+ * outside its block, 4 a range outside the bound buffer (a = which array,
+ * b = offset of the range in the buffer, c = its bytes, d = the buffer's
+ * bytes), 5 null pointer; kernel: 1 statistics step, 2 its combine, 3 sample
+ * gather, 4 first finalize sweep, 5 later sweeps, 6 / 7 row-column reduction of
+ * the window / of the step, 8 its combine, 9 fused step, 10 the self-test.
+ *
+ * baoc_check_selftest: queues a one-thread kernel that runs the range check on
+ * numbers that violate it (a 32-byte range that starts 16 bytes before the end
+ * of a buffer; no memory is touched), so that a test can see a violation being
+ * recorded and the context staying usable.  BAOC_E_STATE in a normal build. */
+typedef struct {
+    int32_t enabled;
+    uint32_t code, kernel;
+    int32_t reserved;
+    int64_t a, b, c, d;
+} baoc_check_t;
+int baoc_check_status(baoc_check_t* out);
+int baoc_check_selftest(baoc_stream_t stream);
+
 /* ---- allocation-free variant ------------------------------------------------ */
 
 /* Largest block baoc_sample_stats_noalloc accepts (64 Mi elements).  The

@@ -65,6 +65,7 @@ class Opts:
     use_snr: bool = True           # Eq. 17, else s_M = s_rho
     eps_adam: float = 1e-8         # epsilon of the update direction in Eq. 8
     qblock: int = 256              # elements per quantisation block
+    quantizer8: str = "linear"     # the 8-bit quantiser of Eq. 8: "linear" absmax codes or the "dynamic" codebook
 
 
 @dataclass
@@ -81,6 +82,13 @@ class Config:
     beta2: float = 0.999
     eps: float = 1e-8
     weight_decay: float = 0.0
+    quantizer: str = "linear"      # 8-bit states: "linear" absmax codes, or the non-linear "dynamic" codebook
+    # Options of the factored tuple that turn its mechanism-pure rule into the published Adafactor algorithm (the
+    # paper names Adafactor among its mechanisms without saying which of its parts are meant).  All off by default.
+    af_beta2_schedule: bool = False   # beta2_t = 1 - t^-0.8 instead of a constant, and no bias correction
+    af_clip: float = 0.0              # d > 0: the update u is divided by max(1, RMS(u) / d)
+    af_relative_step: bool = False    # step size max(1e-3, RMS(theta)) * min(1e-2, 1 / sqrt(t)) instead of lr
+    af_eps1: float = 0.0              # added to every squared gradient before the row and column means
 
 
 def default_configs() -> List[Config]:
@@ -131,6 +139,62 @@ def dequantize8(codes: np.ndarray, absmax: np.ndarray, signed: bool, qblock: int
     L = 127.0 if signed else 255.0
     cb, d = _blocks_view(codes.astype(F64), qblock)
     x = cb * absmax.astype(F64)[:, None] / L
+    return x.reshape(-1)[:d]
+
+
+# ----------------------------------------------------------------------------
+# Non-linear 8-bit codebook: the alternative reading of "a standard quantizer".
+# The block-wise 8-bit optimizers that the paper cites for its AdamW8 baseline
+# (Sec. 4.1, Baselines) describe a "dynamic" 8-bit data type: an optional sign
+# bit, then a run of zero bits whose length E is a decimal exponent, one
+# indicator bit, and the remaining F bits as a linear fraction within a decade.
+# The table below is built from that description (it is this repository's own
+# construction, no third-party table is reproduced): the magnitudes are
+#     10^-E * (0.1 + 0.9 (k + 1) / 2^F),   k = 0 .. 2^F - 1,
+# with F = B - 1 - E for E = 0 .. B - 1, where B = 7 value bits for the signed
+# type (first moments) and B = 8 for the unsigned one (second moments), plus the
+# value 0.  Decade E thus covers (10^-(E+1), 10^-E] with 2^F entries, the largest
+# entry is exactly 1 and the smallest positive one 10^-(B-1).  Signed: 127
+# magnitudes of either sign and zero, 255 entries; unsigned: 255 and zero, 256.
+# A code is the index of its entry in ascending order.  Quantisation is block-
+# wise with the fp32 absmax a: the code of x is the entry nearest to x / a (a tie
+# goes to the entry of smaller magnitude); x ~ entry * a.
+# ----------------------------------------------------------------------------
+
+def dynamic_codebook(signed: bool) -> np.ndarray:
+    bits = 7 if signed else 8
+    mags = []
+    for E in range(bits):
+        F = bits - 1 - E
+        for k in range(2 ** F):
+            mags.append(10.0 ** (-E) * (0.1 + 0.9 * (k + 1) / 2.0 ** F))
+    mags = np.sort(np.asarray(mags, F64))
+    if signed:
+        return np.concatenate([-mags[::-1], [0.0], mags])
+    return np.concatenate([[0.0], mags])
+
+
+def quantize8_dynamic(x: np.ndarray, signed: bool, qblock: int = 256):
+    """Codes (uint8 indices into ``dynamic_codebook(signed)``) and the fp32 absmax of every quantisation block."""
+    x = np.asarray(x, dtype=F64)
+    xb, d = _blocks_view(x, qblock)
+    a = np.max(np.abs(xb), axis=1).astype(np.float32)
+    a64 = a.astype(F64)
+    y = xb / np.where(a64 > 0.0, a64, 1.0)[:, None]
+    y = np.where(a64[:, None] > 0.0, y, 0.0)
+    t = dynamic_codebook(signed)
+    mid = 0.5 * (t[:-1] + t[1:])
+    toward_zero_pos = np.searchsorted(mid, y, side="left")      # y on a midpoint: the lower entry, smaller for y > 0
+    toward_zero_neg = np.searchsorted(mid, y, side="right")     # the upper entry, smaller in magnitude for y < 0
+    idx = np.where(y >= 0.0, toward_zero_pos, toward_zero_neg)
+    return idx.reshape(-1)[:d].astype(np.uint8), a
+
+
+def dequantize8_dynamic(codes: np.ndarray, absmax: np.ndarray, signed: bool, qblock: int = 256) -> np.ndarray:
+    """x = entry * a in double."""
+    t = dynamic_codebook(signed)
+    cb, d = _blocks_view(codes.astype(np.int64), qblock)
+    x = t[cb] * absmax.astype(F64)[:, None]
     return x.reshape(-1)[:d]
 
 
@@ -254,6 +318,11 @@ def precision_cosine(m: np.ndarray, v: np.ndarray, bits: int, o: Opts) -> float:
         mq, vq = m, v
     elif bits == 16:
         mq, vq = round_bf16(m), round_bf16(v)
+    elif bits == 8 and o.quantizer8 == "dynamic":
+        cm, am = quantize8_dynamic(m, True, o.qblock)
+        cv, av = quantize8_dynamic(v, False, o.qblock)
+        mq = dequantize8_dynamic(cm, am, True, o.qblock)
+        vq = dequantize8_dynamic(cv, av, False, o.qblock)
     elif bits == 8:
         cm, am = quantize8(m, True, o.qblock)
         cv, av = quantize8(v, False, o.qblock)
@@ -269,6 +338,9 @@ def quant_rel_error(x: np.ndarray, bits: int, signed: bool, o: Opts) -> float:
     """Diagnostic: ||x - Q_b(x)|| / ||x|| (0 for a zero vector)."""
     if bits == 16:
         xq = round_bf16(x)
+    elif o.quantizer8 == "dynamic":
+        c, a = quantize8_dynamic(x, signed, o.qblock)
+        xq = dequantize8_dynamic(c, a, signed, o.qblock)
     else:
         c, a = quantize8(x, signed, o.qblock)
         xq = dequantize8(c, a, signed, o.qblock)
@@ -467,6 +539,8 @@ def config_kind(c: Config) -> str:
     if c.factored:
         return {32: "F", 16: "F16", 8: "F8"}[c.bits] if (c.adaptive and not c.momentum) else "unsupported"
     if c.adaptive and c.momentum:
+        if c.bits == 8 and c.quantizer == "dynamic":
+            return "A8N"                                             # Adam with 8-bit moments in the non-linear codebook
         return {32: "A32", 16: "A16", 8: "A8"}[c.bits]
     if c.adaptive and not c.momentum:
         return {32: "R", 16: "R16", 8: "R8"}[c.bits]
@@ -492,6 +566,9 @@ def step_init(c: Config, numel: int, rows: int, cols: int, qblock: int = 256) ->
         return StepState(kind, qm=np.zeros(numel, np.int8), am=np.zeros(nq, np.float32))
     if kind == "A8":
         return StepState(kind, qm=np.zeros(numel, np.int8), qv=np.zeros(numel, np.uint8),
+                         am=np.zeros(nq, np.float32), av=np.zeros(nq, np.float32))
+    if kind == "A8N":
+        return StepState(kind, qm=np.zeros(numel, np.uint8), qv=np.zeros(numel, np.uint8),
                          am=np.zeros(nq, np.float32), av=np.zeros(nq, np.float32))
     if kind == "R":
         return StepState(kind, v=np.zeros(numel, F64))
@@ -523,6 +600,7 @@ def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, 
     g = np.asarray(g, dtype=F64)
     st.t += 1
     t = (max(1, st.t - st.t_m0), max(1, st.t - st.t_v0))     # gradients each moment has seen, this one included
+    theta_in = theta
     theta, g = _prologue(theta, g, c)
     if st.kind == "A32":
         st.m = c.beta1 * st.m + (1.0 - c.beta1) * g
@@ -567,6 +645,15 @@ def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, 
         st.qm, st.am = quantize8(m, True, qblock)
         st.qv, st.av = quantize8(v, False, qblock)
         return theta
+    if st.kind == "A8N":
+        m = dequantize8_dynamic(st.qm, st.am, True, qblock)
+        v = dequantize8_dynamic(st.qv, st.av, False, qblock)
+        m = c.beta1 * m + (1.0 - c.beta1) * g
+        v = c.beta2 * v + (1.0 - c.beta2) * g * g
+        theta = _adam_apply(theta, m, v, c, t, True)      # uses the un-requantised moments
+        st.qm, st.am = quantize8_dynamic(m, True, qblock)
+        st.qv, st.av = quantize8_dynamic(v, False, qblock)
+        return theta
     if st.kind == "R":
         st.v = c.beta2 * st.v + (1.0 - c.beta2) * g * g
         return _adam_apply(theta, g, st.v, c, t, False)
@@ -574,9 +661,11 @@ def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, 
         # the row and column statistics are read as stored; the update uses the new ones before they are rounded for
         # storage (the convention of every reduced-precision state here)
         r_old, c_old = _factored_stored(st, qblock)
-        G2 = (g * g).reshape(rows, cols)
-        r = c.beta2 * r_old + (1.0 - c.beta2) * G2.mean(axis=1)
-        cc = c.beta2 * c_old + (1.0 - c.beta2) * G2.mean(axis=0)
+        t_v = t[1]
+        beta2 = 1.0 - float(t_v) ** -0.8 if c.af_beta2_schedule else c.beta2
+        G2 = (g * g + c.af_eps1).reshape(rows, cols)
+        r = beta2 * r_old + (1.0 - beta2) * G2.mean(axis=1)
+        cc = beta2 * c_old + (1.0 - beta2) * G2.mean(axis=0)
         rm = float(r.mean())
         if rm == 0.0:
             v = np.zeros(rows * cols, F64)
@@ -589,7 +678,20 @@ def step(theta: np.ndarray, g: np.ndarray, st: StepState, c: Config, rows: int, 
         else:
             st.qr, st.ar = quantize8(r, False, qblock)
             st.qc, st.ac = quantize8(cc, False, qblock)
-        return _adam_apply(theta, g, v, c, t, False)
+        if not (c.af_beta2_schedule or c.af_clip > 0.0 or c.af_relative_step):
+            return _adam_apply(theta, g, v, c, t, False)
+        # Adafactor's remaining parts.  theta_in: the parameters before this step (the relative step size is taken from
+        # them); a decoupled decay then uses that step size in place of lr.
+        bc2 = 1.0 if c.af_beta2_schedule else 1.0 - c.beta2 ** t_v
+        u = g / (np.sqrt(v / bc2) + c.eps)
+        if c.af_clip > 0.0:
+            u = u / max(1.0, math.sqrt(float(np.mean(u * u))) / c.af_clip)
+        alpha = c.lr
+        if c.af_relative_step:
+            alpha = max(1e-3, math.sqrt(float(np.mean(theta_in * theta_in)))) * min(1e-2, 1.0 / math.sqrt(float(t_v)))
+            if c.weight_decay != 0.0 and c.decoupled_wd:
+                theta = theta_in * (1.0 - alpha * c.weight_decay)
+        return theta - alpha * u
     if st.kind == "S":
         st.m = c.beta1 * st.m + g
         return theta - c.lr * st.m

@@ -16,12 +16,15 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbaoc.so")
+# BAOC_CHECKED=1 in the environment selects the checked build of the library (in-kernel validation of every tile and
+# range, see include/baoc.h); it is a different file, so the choice is made once, at import
+CHECKED = os.environ.get("BAOC_CHECKED", "") == "1"
+LIB_PATH = os.path.join(_HERE, "libbaoc_checked.so" if CHECKED else "libbaoc.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
         f"{LIB_PATH} is missing: build the CUDA library first "
-        "(python -m paper_2605_04711_b200.build); there is no fallback path")
+        "(python -m paper_2605_04711_b200.build [--checked]); there is no fallback path")
 
 _lib = C.CDLL(LIB_PATH)
 
@@ -64,6 +67,11 @@ class BlockStats(C.Structure):
         return {n: getattr(self, n) for n, _ in self._fields_}
 
 
+class Check(C.Structure):
+    _fields_ = [("enabled", C.c_int32), ("code", C.c_uint32), ("kernel", C.c_uint32), ("reserved", C.c_int32),
+                ("a", C.c_int64), ("b", C.c_int64), ("c", C.c_int64), ("d", C.c_int64)]
+
+
 class Sample(C.Structure):
     _fields_ = [("n_rows", C.c_int64), ("n_cols", C.c_int32), ("rows", C.c_void_p), ("cols", C.c_void_p)]
 
@@ -81,7 +89,7 @@ EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error"
            "baoc_sample_stats_noalloc", "baoc_noalloc_last_error", "baoc_profile", "baoc_profile_last",
            "baoc_export", "baoc_import", "baoc_time_scratch_bytes", "baoc_measure_time_ratios",
            "baoc_set_sampling", "baoc_reconfigure", "baoc_configure_from_window", "baoc_partition",
-           "baoc_set_factored_schedule"]
+           "baoc_set_factored_schedule", "baoc_check_status", "baoc_check_selftest"]
 
 _vp = C.c_void_p
 _lib.baoc_default_opts.argtypes = [C.POINTER(Opts)]
@@ -115,6 +123,8 @@ _lib.baoc_measure_time_ratios.argtypes = [_vp, _vp, _vp, _vp, C.c_size_t, C.c_in
 _lib.baoc_export.argtypes = [_vp, _vp, C.c_size_t, C.POINTER(C.c_size_t)]
 _lib.baoc_import.argtypes = [_vp, _vp, C.c_size_t, _vp, C.c_size_t, _vp, C.c_size_t, _vp]
 _lib.baoc_set_factored_schedule.argtypes = [_vp, C.c_int64]
+_lib.baoc_check_status.argtypes = [C.POINTER(Check)]
+_lib.baoc_check_selftest.argtypes = [_vp]
 _lib.baoc_profile.argtypes = [_vp, C.c_int]
 _lib.baoc_profile_last.argtypes = [_vp, C.POINTER(C.c_float)]
 _lib.baoc_sample_stats_noalloc.argtypes = [_vp, _vp, _vp, _vp, C.c_int64, C.c_double, C.c_double, C.c_double, _vp, _vp]
@@ -134,6 +144,22 @@ def sample_stats_noalloc(grad: torch.Tensor, gprev: torch.Tensor, m: torch.Tenso
                                         float(beta_m), float(beta_v), float(eps), out4.data_ptr(), _stream())
     if rc < 0:
         raise BaocError(rc, _lib.baoc_noalloc_last_error().decode())
+
+
+def check_status() -> dict:
+    """``baoc_check_status``: the first violation the checked build's kernels recorded since the last call (and clears
+    it).  {"enabled": 0, "code": 0, ...} from a normal build."""
+    c = Check()
+    rc = _lib.baoc_check_status(C.byref(c))
+    if rc < 0:
+        raise BaocError(rc, "baoc_check_status failed")
+    return {k: getattr(c, k) for k in ("enabled", "code", "kernel", "a", "b", "c", "d")}
+
+
+def check_selftest() -> int:
+    """``baoc_check_selftest``: queue the kernel that makes the range check fail on purpose-made numbers (no memory is
+    touched).  Returns the status code (E_STATE from a normal build)."""
+    return _lib.baoc_check_selftest(_stream())
 
 
 def partition(numel, z, w=None, alpha: float = 0.0, tau: Optional[float] = None):

@@ -63,6 +63,10 @@ int sync_pointer_table(Handle* h, const void* const* ptrs, std::vector<const voi
 template <typename T>
 T* at(char* base, size_t off) { return reinterpret_cast<T*>(base + off); }
 
+// What a launch over n_tiles tiles (or reduction pieces) may touch: the statistics workspace, or the state buffer.
+CheckCtx ws_ctx(const Handle* h, int64_t n_tiles) { return CheckCtx{h->ws, h->ws + h->ws_bytes, (long long)n_tiles, h->n_blocks, 0}; }
+CheckCtx st_ctx(const Handle* h, int64_t n_tiles) { return CheckCtx{h->st, h->st + h->st_bytes, (long long)n_tiles, h->n_blocks, 0}; }
+
 // The streaming part of one observation for the blocks [b0, b1): their tiles are contiguous in the tile table.
 int stats_step_range(Handle* h, int b0, int b1, cudaStream_t s) {
     const auto& L = h->sl;
@@ -71,13 +75,13 @@ int stats_step_range(Handle* h, int b0, int b1, cudaStream_t s) {
     if (t1 <= t0) return BAOC_OK;
     if (h->sampled) {
         LAUNCH(launch_sample_gather(at<StatBlock>(h->ws, L.blocks), at<Tile>(h->ws, L.tiles) + t0, at<const void*>(h->ws, L.grads),
-                                    t1 - t0, 0, s), "sample_gather_kernel");
+                                    t1 - t0, 0, ws_ctx(h, t1 - t0), s), "sample_gather_kernel");
         h->launches += 1;
     }
     LAUNCH(launch_stats_step(at<StatBlock>(h->ws, L.blocks), at<Tile>(h->ws, L.tiles) + t0,
                              at<const void*>(h->ws, h->sampled ? L.sgrads : L.grads),
                              at<double>(h->ws, L.partials) + size_t(t0) * kStatPartials, t1 - t0,
-                             float(1.0 - h->opts.beta_m), float(1.0 - h->opts.beta_v), s), "stats_step_kernel");
+                             float(1.0 - h->opts.beta_m), float(1.0 - h->opts.beta_v), ws_ctx(h, t1 - t0), s), "stats_step_kernel");
     h->launches += 1;
     return BAOC_OK;
 }
@@ -85,7 +89,7 @@ int stats_step_range(Handle* h, int b0, int b1, cudaStream_t s) {
 int stats_combine_all(Handle* h, cudaStream_t s) {
     const auto& L = h->sl;
     LAUNCH(launch_stats_combine(at<StatBlock>(h->ws, L.blocks), at<double>(h->ws, L.partials), at<double>(h->ws, L.acc),
-                                h->n_blocks, h->stats_steps > 0 ? 1 : 0, h->opts.beta_rho, h->opts.eps, s),
+                                h->n_blocks, h->stats_steps > 0 ? 1 : 0, h->opts.beta_rho, h->opts.eps, ws_ctx(h, h->n_stat_tiles), s),
            "stats_combine_kernel");
     h->launches += 1;
     h->stats_steps += 1;
@@ -162,7 +166,7 @@ int step_group(Handle* h, const Handle::GroupStep& g, const StepParams& P, cudaS
     if (g.n_f > 0) {
         LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles) + g.red0,
                                       at<int32_t>(h->st, L.f_ids) + g.f0, at<const void*>(h->st, L.grads),
-                                      at<const float*>(h->st, L.params), g.n_red, g.n_f, P, s),
+                                      at<const float*>(h->st, L.params), g.n_red, g.n_f, P, st_ctx(h, g.n_red), s),
                "factored_reduce_kernel");
         h->launches += 2;
     }
@@ -171,7 +175,7 @@ int step_group(Handle* h, const Handle::GroupStep& g, const StepParams& P, cudaS
         if (g.fam_tiles[fam] == 0) continue;
         LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles_by_group) + first,
                                  at<const void*>(h->st, L.grads), at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags),
-                                 g.fam_tiles[fam], fam, P, s),
+                                 g.fam_tiles[fam], fam, P, st_ctx(h, g.fam_tiles[fam]), s),
                "fused_step_kernel");
         h->launches += 1;
         first += g.fam_tiles[fam];
@@ -190,7 +194,8 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
     if (h->n_factored > 0 && !grouped) {
         LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles),
                                       at<int32_t>(h->st, L.f_ids), at<const void*>(h->st, L.grads),
-                                      at<const float*>(h->st, L.params), h->n_step_red_tiles, h->n_factored, P, s),
+                                      at<const float*>(h->st, L.params), h->n_step_red_tiles, h->n_factored, P,
+                                      st_ctx(h, h->n_step_red_tiles), s),
                "factored_reduce_kernel");
         h->launches += 2;
     }
@@ -202,7 +207,7 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
         const int64_t here = (grouped && fam == kFamHead) ? h->fam_tiles[fam] - h->n_factored_tiles : h->fam_tiles[fam];
         if (here > 0) {
             LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles) + first, at<const void*>(h->st, L.grads),
-                                     at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), here, fam, P, s),
+                                     at<float*>(h->st, L.params), at<uint32_t>(h->st, L.flags), here, fam, P, st_ctx(h, here), s),
                    "fused_step_kernel");
             h->launches += 1;
         }
@@ -212,11 +217,11 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
             for (const Handle::FactoredGroup& g : h->f_groups) {
                 LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles) + g.red0,
                                               at<int32_t>(h->st, L.f_ids) + g.f0, at<const void*>(h->st, L.grads),
-                                              at<const float*>(h->st, L.params), g.n_red, g.n_f, P, s),
+                                              at<const float*>(h->st, L.params), g.n_red, g.n_f, P, st_ctx(h, g.n_red), s),
                        "factored_reduce_kernel");
                 LAUNCH(launch_fused_step(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles) + f_first + g.tile0,
                                          at<const void*>(h->st, L.grads), at<float*>(h->st, L.params),
-                                         at<uint32_t>(h->st, L.flags), g.n_tiles, kFamHead, P, s),
+                                         at<uint32_t>(h->st, L.flags), g.n_tiles, kFamHead, P, st_ctx(h, g.n_tiles), s),
                        "fused_step_kernel");
                 h->launches += 3;
             }
@@ -353,20 +358,22 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
     const Tile* tiles = at<Tile>(ws, L.tiles);
     const float* const* dparams = at<const float*>(ws, h->sampled ? L.sparams : L.params);
     if (h->sampled) {
-        LAUNCH(launch_sample_gather(blocks, tiles, at<const void*>(ws, L.params), h->n_stat_tiles, 1, s), "sample_gather_kernel");
+        LAUNCH(launch_sample_gather(blocks, tiles, at<const void*>(ws, L.params), h->n_stat_tiles, 1, ws_ctx(h, h->n_stat_tiles), s),
+               "sample_gather_kernel");
         h->launches += 1;
     }
     LAUNCH(launch_final_sums(blocks, tiles, dparams, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<uint32_t>(ws, L.hist),
-                             at<RankSel>(ws, L.sel), h->n_stat_tiles, n, h->opts.eps, float(h->opts.eps_adam), s),
+                             at<RankSel>(ws, L.sel), h->n_stat_tiles, n, h->opts.eps, float(h->opts.eps_adam),
+                             ws_ctx(h, h->n_stat_tiles), s),
            "final_sums_kernel");
     h->launches += 5;
     if (h->n_matrix > 0) {
         LAUNCH(launch_moment_reduce(blocks, at<RedTile>(ws, L.red_tiles), at<int32_t>(ws, L.matrix_ids), h->n_red_tiles,
-                                    h->n_matrix, s), "moment_reduce_kernel");
+                                    h->n_matrix, ws_ctx(h, h->n_red_tiles), s), "moment_reduce_kernel");
         h->launches += 3;
     }
     LAUNCH(launch_final_resid_select(blocks, tiles, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<RankSel>(ws, L.sel),
-                                     at<uint32_t>(ws, L.hist), at<double>(ws, L.acc), h->n_stat_tiles, n, s),
+                                     at<uint32_t>(ws, L.hist), at<double>(ws, L.acc), h->n_stat_tiles, n, ws_ctx(h, h->n_stat_tiles), s),
            "final_hist_kernel");
     h->launches += 6;
 
@@ -953,6 +960,33 @@ int baoc_set_factored_schedule(baoc_t* h, int64_t group_bytes) {
     if (h->configured) return fail(h, BAOC_E_STATE, "baoc_set_factored_schedule: set the schedule before baoc_configure");
     h->factored_group_bytes = group_bytes;
     return BAOC_OK;
+}
+
+int baoc_check_status(baoc_check_t* out) {
+    if (!out) return BAOC_E_INVALID;
+    std::memset(out, 0, sizeof(*out));
+#ifdef BAOC_CHECKED
+    out->enabled = 1;
+    if (cudaDeviceSynchronize() != cudaSuccess) return BAOC_E_CUDA;
+    int (*const fetch[])(CheckRecord*) = {stats_check_fetch, finalize_check_fetch, step_check_fetch};
+    for (auto f : fetch) {
+        CheckRecord r{};
+        if (f(&r) != 0) return BAOC_E_CUDA;
+        if (r.code != 0 && out->code == 0) {                 // every unit is fetched and cleared; the first violation is reported
+            out->code = r.code; out->kernel = r.kernel; out->a = r.a; out->b = r.b; out->c = r.c; out->d = r.d;
+        }
+    }
+#endif
+    return BAOC_OK;
+}
+
+int baoc_check_selftest(baoc_stream_t stream) {
+#ifdef BAOC_CHECKED
+    return launch_check_selftest(static_cast<cudaStream_t>(stream)) == 0 ? BAOC_OK : BAOC_E_CUDA;
+#else
+    (void)stream;
+    return BAOC_E_STATE;
+#endif
 }
 
 int baoc_profile(baoc_t* h, int enable) {

@@ -7,6 +7,7 @@
 #include <cuda_runtime.h>
 
 #include "baoc_internal.h"
+#include "baoc_check.cuh"
 
 namespace baoc {
 

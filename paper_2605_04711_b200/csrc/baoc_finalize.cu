@@ -161,7 +161,27 @@ __global__ void __launch_bounds__(kThreads, 2)
 final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
                   const float* const* __restrict__ params, double* __restrict__ fin,
                   const double* __restrict__ fin_out, uint32_t* __restrict__ hist, int64_t n_tiles,
-                  int tiles_per_cta, float eps_f, float eps_adam) {
+                  int tiles_per_cta, float eps_f, float eps_adam BAOC_CHECK_PARAM) {
+#ifdef BAOC_CHECKED
+    {   // validate every tile of this CTA's run, and the ranges of the workspace it will touch, before touching anything
+        const int64_t c0 = int64_t(blockIdx.x) * tiles_per_cta, c1 = min64(c0 + tiles_per_cta, n_tiles);
+        if (c0 >= ck.n_tiles || n_tiles != ck.n_tiles) { check_fail(kChkTileIndex, kKerFinalSums, c0, ck.n_tiles, n_tiles, 0); return; }
+        for (int64_t ti = c0; ti < c1; ++ti) {
+            const Tile ct = tiles[ti];
+            if (ct.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerFinalSums, ct.block, ck.n_blocks, ti, 0); return; }
+            const StatBlock* cb = blocks + ct.block;
+            const int64_t cbase = int64_t(ct.piece) * kTile;
+            const int64_t cpad = (cb->numel + kQBlock - 1) / kQBlock * kQBlock, cn = min64(kTile, cpad - cbase);
+            if (!check_tile(ck, kKerFinalSums, ti, ct.block, cbase, cb->numel) ||
+                !check_range(ck, kKerFinalSums, cb->m + cbase, 4 * cn, 0) || !check_range(ck, kKerFinalSums, cb->v + cbase, 4 * cn, 1) ||
+                !check_range(ck, kKerFinalSums, fin + size_t(ti) * kFinalSums, 8 * kFinalSums, 2) ||
+                !check_range(ck, kKerFinalSums, hist + size_t(ct.block) * kRanks * kSelBins, 4ll * kSelBins, 3) ||
+                !check_range(ck, kKerFinalSums, fin_out + size_t(ct.block) * kFinOut, 8 * kFinOut, 4) ||
+                !check_caller_ptr(kKerFinalSums, params[ct.block], 5))
+                return;
+        }
+    }
+#endif
     extern __shared__ __align__(16) unsigned char dyn[];
     unsigned char* stage = dyn;
     uint32_t* hist1 = reinterpret_cast<uint32_t*>(dyn + kFsStages * kFsStageBytes);      // kSelBins counters
@@ -325,7 +345,29 @@ static_assert(kSelRunTiles * kTile < 65536, "a 16-bit bin must hold a whole run 
 template <bool kResid>
 __global__ void __launch_bounds__(kThreads, kResid ? 3 : 4)
 final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const RankSel* __restrict__ sel,
-                  double* __restrict__ fin, uint32_t* __restrict__ hist, int64_t n_tiles, int tiles_per_cta) {
+                  double* __restrict__ fin, uint32_t* __restrict__ hist, int64_t n_tiles, int tiles_per_cta BAOC_CHECK_PARAM) {
+#ifdef BAOC_CHECKED
+    {
+        const int64_t c0 = int64_t(blockIdx.x) * tiles_per_cta, c1 = min64(c0 + tiles_per_cta, n_tiles);
+        if (c0 >= ck.n_tiles || n_tiles != ck.n_tiles) { check_fail(kChkTileIndex, kKerFinalHist, c0, ck.n_tiles, n_tiles, 0); return; }
+        for (int64_t ti = c0; ti < c1; ++ti) {
+            const Tile ct = tiles[ti];
+            if (ct.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerFinalHist, ct.block, ck.n_blocks, ti, 0); return; }
+            const StatBlock* cb = blocks + ct.block;
+            const int64_t cbase = int64_t(ct.piece) * kTile;
+            const int64_t cpad = (cb->numel + kQBlock - 1) / kQBlock * kQBlock, cn = min64(kTile, cpad - cbase);
+            if (!check_tile(ck, kKerFinalHist, ti, ct.block, cbase, cb->numel) ||
+                !check_range(ck, kKerFinalHist, cb->v + cbase, 4 * cn, 0) ||
+                !check_range(ck, kKerFinalHist, hist + size_t(ct.block) * kRanks * kSelBins, 4ll * kRanks * kSelBins, 1) ||
+                !check_range(ck, kKerFinalHist, sel + size_t(ct.block) * kRanks, int64_t(sizeof(RankSel)) * kRanks, 2))
+                return;
+            if (kResid && (!check_range(ck, kKerFinalHist, fin + size_t(ti) * kResidSums, 8 * kResidSums, 3) ||
+                           (cb->cols > 1 && (!check_range(ck, kKerFinalHist, cb->rowsum, 8ll * (cb->rows + 1), 4) ||
+                                             !check_range(ck, kKerFinalHist, cb->colsum, 8ll * cb->cols, 5)))))
+                return;
+        }
+    }
+#endif
     extern __shared__ __align__(16) unsigned char dyn[];
     uint32_t (*sh)[kFhHistWords] = reinterpret_cast<uint32_t (*)[kFhHistWords]>(dyn);
     constexpr int kShift = kResid ? kSel3Bits : 0;            // lowest bit of this pass's digit
@@ -582,6 +624,8 @@ __global__ void stats_gather_kernel(const RankSel* __restrict__ sel, const doubl
         if (e_ != cudaSuccess) return int(e_);                \
     } while (0)
 
+BAOC_DEFINE_CHECK_FETCH(finalize_check_fetch)
+
 // Tiles per CTA of a sweep: as many as `most`, fewer when the workload would then not give every SM a few CTAs.
 static int run_tiles(int64_t n_tiles, int most) {
     const int64_t want = n_tiles / (int64_t(148) * 6);
@@ -590,7 +634,8 @@ static int run_tiles(int64_t n_tiles, int most) {
 
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
                       double* fin_out, uint32_t* hist, RankSel* sel, int64_t n_tiles, int n_blocks, double eps,
-                      float eps_adam, cudaStream_t s) {
+                      float eps_adam, const CheckCtx& ck, cudaStream_t s) {
+    (void)ck;
     const int tb = 128, gb = (n_blocks + tb - 1) / tb;
     cudaError_t e = cudaMemsetAsync(hist, 0, size_t(n_blocks) * kRanks * kSelBins * sizeof(uint32_t), s);
     if (e != cudaSuccess) return int(e);
@@ -602,7 +647,7 @@ int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* c
     if (e != cudaSuccess) return int(e);
     const int per = run_tiles(n_tiles, kFinRunTiles);
     final_sums_kernel<<<unsigned((n_tiles + per - 1) / per), kThreads, kFsSmemBytes, s>>>(
-        blocks, tiles, params, fin, fin_out, hist, n_tiles, per, float(eps), eps_adam);
+        blocks, tiles, params, fin, fin_out, hist, n_tiles, per, float(eps), eps_adam BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     final_sums_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
     BAOC_LAUNCH_CHECK();
@@ -612,20 +657,22 @@ int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* c
 }
 
 int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                              uint32_t* hist, const double* acc, int64_t n_tiles, int n_blocks, cudaStream_t s) {
+                              uint32_t* hist, const double* acc, int64_t n_tiles, int n_blocks, const CheckCtx& ck,
+                              cudaStream_t s) {
+    (void)ck;
     constexpr int kSmem = kFhSmemBytes;
     cudaError_t e = cudaFuncSetAttribute(final_hist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(final_hist_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return int(e);
     const int per = run_tiles(n_tiles, kSelRunTiles);
     const unsigned grid = unsigned((n_tiles + per - 1) / per);
-    final_hist_kernel<true><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per);
+    final_hist_kernel<true><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     final_resid_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
     BAOC_LAUNCH_CHECK();
     select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, kSel3Bits, kSelBins);
     BAOC_LAUNCH_CHECK();
-    final_hist_kernel<false><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per);
+    final_hist_kernel<false><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, 0, 1 << kSel3Bits);
     BAOC_LAUNCH_CHECK();

@@ -85,6 +85,22 @@ BAOC_HD inline int64_t step_tile_elems(int path) {
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
 
+// Checked build (-DBAOC_CHECKED, see baoc_check.cuh): what a launch may touch (the bound buffer and the sizes of the
+// tables it indexes), and the record of the first violation a kernel found.  Plain data; a normal build passes the
+// context to the launchers too and ignores it.
+struct CheckCtx {
+    const char* lo;
+    const char* hi;
+    long long n_tiles;
+    int n_blocks;
+    int pad;
+};
+struct CheckRecord {
+    unsigned int code;       // 0: clean
+    unsigned int kernel;
+    long long a, b, c, d;    // the offending numbers (index and limit, or range and buffer bounds)
+};
+
 // One tile of a streaming kernel: which block, and which kTile-sized piece of it.
 struct Tile {
     uint32_t block;
@@ -303,24 +319,32 @@ void compute_stat_layout(Handle* h);
 
 // Kernel launchers (defined in the .cu files).  Each returns 0 or a cudaError_t value.
 int launch_stats_step(const StatBlock* blocks, const Tile* tiles, const void* const* grads, double* partials,
-                      int64_t n_tiles, float one_minus_beta_m, float one_minus_beta_v, cudaStream_t s);
+                      int64_t n_tiles, float one_minus_beta_m, float one_minus_beta_v, const CheckCtx& ck, cudaStream_t s);
 int launch_stats_combine(const StatBlock* blocks, const double* partials, double* acc, int n_blocks, int has_prev,
-                         double beta_rho, double eps, cudaStream_t s);
+                         double beta_rho, double eps, const CheckCtx& ck, cudaStream_t s);
 // First finalize sweep (with the pilot values, the start of the select and its first radix pass), then, after the
 // row/column sums of the matrix blocks, the second and third sweep and the gather of the per-block results.
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
                       double* fin_out, uint32_t* hist, RankSel* sel, int64_t n_tiles, int n_blocks, double eps,
-                      float eps_adam, cudaStream_t s);
+                      float eps_adam, const CheckCtx& ck, cudaStream_t s);
 int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                              uint32_t* hist, const double* acc, int64_t n_tiles, int n_blocks, cudaStream_t s);
+                              uint32_t* hist, const double* acc, int64_t n_tiles, int n_blocks, const CheckCtx& ck,
+                              cudaStream_t s);
 int launch_sample_gather(const StatBlock* blocks, const Tile* tiles, const void* const* src, int64_t n_tiles, int fp32,
-                         cudaStream_t s);
+                         const CheckCtx& ck, cudaStream_t s);
 int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const int32_t* ids, int64_t n_red, int n_matrix,
-                         cudaStream_t s);
+                         const CheckCtx& ck, cudaStream_t s);
 int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const int32_t* ids, const void* const* grads,
-                           const float* const* params, int64_t n_red, int n_factored, const StepParams& P, cudaStream_t s);
+                           const float* const* params, int64_t n_red, int n_factored, const StepParams& P, const CheckCtx& ck,
+                           cudaStream_t s);
 int launch_fused_step(const StepBlock* blocks, const Tile* tiles, const void* const* grads, float* const* params,
-                      uint32_t* flags, int64_t n_tiles, int family, const StepParams& P, cudaStream_t s);
+                      uint32_t* flags, int64_t n_tiles, int family, const StepParams& P, const CheckCtx& ck, cudaStream_t s);
+// Checked build: fetch (and clear) the violation record of each CUDA translation unit, and a self-test kernel that runs
+// the range check on numbers that violate it (no memory is touched).  Each returns 0 or a cudaError_t value.
+int stats_check_fetch(CheckRecord* out);
+int finalize_check_fetch(CheckRecord* out);
+int step_check_fetch(CheckRecord* out);
+int launch_check_selftest(cudaStream_t s);
 int launch_convert_moment(const MomentRef& src, const MomentRef& dst, int64_t numel, cudaStream_t s);
 // Copy groups of the end-to-end call: up to Handle::kCopyGroups runs of whole blocks of about equal bytes.
 void compute_copy_groups(const Handle* h, std::vector<int>* b0, std::vector<int>* b1);

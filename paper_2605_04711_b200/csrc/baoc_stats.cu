@@ -19,7 +19,22 @@ __device__ __forceinline__ float ema(float s, float x, float one_minus_beta) { r
 
 __global__ void __launch_bounds__(kThreads)
 stats_step_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
-                  const void* const* __restrict__ grads, double* __restrict__ partials, float om, float ov) {
+                  const void* const* __restrict__ grads, double* __restrict__ partials, float om, float ov BAOC_CHECK_PARAM) {
+#ifdef BAOC_CHECKED
+    {   // validate the tile and every range of the workspace it will touch before touching anything
+        if (int64_t(blockIdx.x) >= ck.n_tiles) { check_fail(kChkTileIndex, kKerStatsStep, blockIdx.x, ck.n_tiles, 0, 0); return; }
+        const Tile ct = tiles[blockIdx.x];
+        if (ct.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerStatsStep, ct.block, ck.n_blocks, blockIdx.x, 0); return; }
+        const StatBlock* cb = blocks + ct.block;
+        const int64_t cbase = int64_t(ct.piece) * kTile, cn = min64(kTile, cb->numel - cbase);
+        if (!check_tile(ck, kKerStatsStep, blockIdx.x, ct.block, cbase, cb->numel) ||
+            !check_range(ck, kKerStatsStep, cb->m + cbase, 4 * cn, 0) || !check_range(ck, kKerStatsStep, cb->v + cbase, 4 * cn, 1) ||
+            !check_range(ck, kKerStatsStep, cb->gprev + cbase, 2 * cn, 2) ||
+            !check_range(ck, kKerStatsStep, partials + size_t(blockIdx.x) * kStatPartials, 8 * kStatPartials, 3) ||
+            !check_caller_ptr(kKerStatsStep, grads[ct.block], 4))
+            return;
+    }
+#endif
     const Tile t = tiles[blockIdx.x];
     const StatBlock* b = blocks + t.block;
     const int64_t numel = b->numel;
@@ -95,7 +110,16 @@ __device__ __forceinline__ double safe_cos(double dot, double n2a, double n2b, d
 // last_cos, rho_mom, n_cos_mom, -, -}.
 __global__ void __launch_bounds__(kThreads)
 stats_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ partials,
-                     double* __restrict__ acc_all, int has_prev, double beta_rho, double eps) {
+                     double* __restrict__ acc_all, int has_prev, double beta_rho, double eps BAOC_CHECK_PARAM) {
+#ifdef BAOC_CHECKED
+    {
+        if (int(blockIdx.x) >= ck.n_blocks) { check_fail(kChkBlockIndex, kKerStatsCombine, blockIdx.x, ck.n_blocks, 0, 0); return; }
+        const StatBlock* cb = blocks + blockIdx.x;
+        if (!check_range(ck, kKerStatsCombine, partials + size_t(cb->tile0) * kStatPartials, 8ll * kStatPartials * cb->ntiles, 0) ||
+            !check_range(ck, kKerStatsCombine, acc_all + size_t(blockIdx.x) * kBlockAcc, 8 * kBlockAcc, 1))
+            return;
+    }
+#endif
     __shared__ double s[kStatPartials];
     const StatBlock* b = blocks + blockIdx.x;
     block_tiles_sum<kStatPartials>(partials, b->tile0, b->ntiles, s);
@@ -125,7 +149,24 @@ stats_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restr
 // ============================================================================
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
-sample_gather_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const void* const* __restrict__ src) {
+sample_gather_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const void* const* __restrict__ src
+                     BAOC_CHECK_PARAM) {
+#ifdef BAOC_CHECKED
+    {
+        if (int64_t(blockIdx.x) >= ck.n_tiles) { check_fail(kChkTileIndex, kKerSampleGather, blockIdx.x, ck.n_tiles, 0, 0); return; }
+        const Tile ct = tiles[blockIdx.x];
+        if (ct.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerSampleGather, ct.block, ck.n_blocks, blockIdx.x, 0); return; }
+        const StatBlock* cb = blocks + ct.block;
+        const int64_t cbase = int64_t(ct.piece) * kTile;
+        const int64_t cpad = (cb->numel + kQBlock - 1) / kQBlock * kQBlock, cn = min64(kTile, cpad - cbase);
+        const void* dst = sizeof(T) == 2 ? static_cast<const void*>(cb->gsample + cbase) : static_cast<const void*>(cb->psample + cbase);
+        if (!check_tile(ck, kKerSampleGather, blockIdx.x, ct.block, cbase, cb->numel) ||
+            !check_range(ck, kKerSampleGather, dst, int64_t(sizeof(T)) * cn, 0) ||
+            !check_range(ck, kKerSampleGather, cb->ridx, 8ll * cb->rows, 1) || !check_range(ck, kKerSampleGather, cb->cidx, 4ll * cb->cols, 2) ||
+            !check_caller_ptr(kKerSampleGather, src[ct.block], 3))
+            return;
+    }
+#endif
     const Tile t = tiles[blockIdx.x];
     const StatBlock* b = blocks + t.block;
     const int64_t numel = b->numel, padded = (numel + kQBlock - 1) / kQBlock * kQBlock;
@@ -153,25 +194,30 @@ sample_gather_kernel(const StatBlock* __restrict__ blocks, const Tile* __restric
         if (e_ != cudaSuccess) return int(e_);                \
     } while (0)
 
+BAOC_DEFINE_CHECK_FETCH(stats_check_fetch)
+
 int launch_stats_step(const StatBlock* blocks, const Tile* tiles, const void* const* grads, double* partials,
-                      int64_t n_tiles, float one_minus_beta_m, float one_minus_beta_v, cudaStream_t s) {
+                      int64_t n_tiles, float one_minus_beta_m, float one_minus_beta_v, const CheckCtx& ck, cudaStream_t s) {
+    (void)ck;
     stats_step_kernel<<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, grads, partials, one_minus_beta_m,
-                                                             one_minus_beta_v);
+                                                             one_minus_beta_v BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     return 0;
 }
 
 int launch_stats_combine(const StatBlock* blocks, const double* partials, double* acc, int n_blocks, int has_prev,
-                         double beta_rho, double eps, cudaStream_t s) {
-    stats_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, partials, acc, has_prev, beta_rho, eps);
+                         double beta_rho, double eps, const CheckCtx& ck, cudaStream_t s) {
+    (void)ck;
+    stats_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, partials, acc, has_prev, beta_rho, eps BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     return 0;
 }
 
 int launch_sample_gather(const StatBlock* blocks, const Tile* tiles, const void* const* src, int64_t n_tiles, int fp32,
-                         cudaStream_t s) {
-    if (fp32) sample_gather_kernel<float><<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, src);
-    else sample_gather_kernel<uint16_t><<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, src);
+                         const CheckCtx& ck, cudaStream_t s) {
+    (void)ck;
+    if (fp32) sample_gather_kernel<float><<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, src BAOC_CHECK_ARG(ck));
+    else sample_gather_kernel<uint16_t><<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, src BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     return 0;
 }

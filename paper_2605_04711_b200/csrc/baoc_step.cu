@@ -149,11 +149,35 @@ __device__ __forceinline__ void rowcol_reduce_piece(const void* src, const float
     }
 }
 
+#ifdef BAOC_CHECKED
+// A reduction CTA: its piece exists, names a block and a (chunk, strip) of that block's geometry, and the partial sums
+// it will write lie inside the bound buffer.
+__device__ __forceinline__ bool check_red_piece(const CheckCtx& ck, unsigned kernel, const RedTile& t, int rows, int cols,
+                                                const RedGeom& geo) {
+    if (int(t.chunk) >= geo.chunks || int(t.strip) >= geo.strips) return check_fail(kChkTileStart, kernel, t.chunk, geo.chunks, t.strip, geo.strips);
+    const int64_t r0 = int64_t(t.chunk) * kRedRows * geo.L, nr = min64(int64_t(kRedRows) * geo.L, rows - r0);
+    const int64_t c0 = int64_t(t.strip) * kRedCols, nc = min64(kRedCols, cols - c0);
+    return check_range(ck, kernel, geo.rowpart + size_t(t.strip) * rows + r0, 8 * nr, 0) &&
+           check_range(ck, kernel, geo.colpart + size_t(t.chunk) * cols + c0, 8 * nc, 1);
+}
+#endif
+
 // Gradient squares of the factored blocks of the step.
 __global__ void __launch_bounds__(kThreads, 4)
 factored_reduce_kernel(const StepBlock* __restrict__ blocks, const RedTile* __restrict__ rtiles,
                        const void* const* __restrict__ grads, const float* const* __restrict__ params,
-                       const __grid_constant__ StepParams SP) {
+                       const __grid_constant__ StepParams SP BAOC_CHECK_PARAM) {
+#ifdef BAOC_CHECKED
+    {
+        if (int64_t(blockIdx.x) >= ck.n_tiles) { check_fail(kChkTileIndex, kKerFactoredReduce, blockIdx.x, ck.n_tiles, 0, 0); return; }
+        const RedTile ct = rtiles[blockIdx.x];
+        if (ct.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerFactoredReduce, ct.block, ck.n_blocks, blockIdx.x, 0); return; }
+        const StepBlock* cb = blocks + ct.block;
+        if (!check_red_piece(ck, kKerFactoredReduce, ct, cb->rows, cb->cols, cb->red) ||
+            !check_caller_ptr(kKerFactoredReduce, grads[ct.block], 2))
+            return;
+    }
+#endif
     const RedTile t = rtiles[blockIdx.x];
     const StepBlock* b = blocks + t.block;
     const CfgStep& P = SP.c[b->cfg];
@@ -163,7 +187,19 @@ factored_reduce_kernel(const StepBlock* __restrict__ blocks, const RedTile* __re
 
 // Second moments of the matrix blocks of the statistics pass.
 __global__ void __launch_bounds__(kThreads)
-moment_reduce_kernel(const StatBlock* __restrict__ blocks, const RedTile* __restrict__ rtiles) {
+moment_reduce_kernel(const StatBlock* __restrict__ blocks, const RedTile* __restrict__ rtiles BAOC_CHECK_PARAM) {
+#ifdef BAOC_CHECKED
+    {
+        if (int64_t(blockIdx.x) >= ck.n_tiles) { check_fail(kChkTileIndex, kKerMomentReduce, blockIdx.x, ck.n_tiles, 0, 0); return; }
+        const RedTile ct = rtiles[blockIdx.x];
+        if (ct.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerMomentReduce, ct.block, ck.n_blocks, blockIdx.x, 0); return; }
+        const StatBlock* cb = blocks + ct.block;
+        const int64_t cpad = (cb->numel + kQBlock - 1) / kQBlock * kQBlock;
+        if (!check_red_piece(ck, kKerMomentReduce, ct, cb->rows, cb->cols, cb->red) ||
+            !check_range(ck, kKerMomentReduce, cb->v, 4 * cpad, 2))
+            return;
+    }
+#endif
     const RedTile t = rtiles[blockIdx.x];
     const StatBlock* b = blocks + t.block;
     rowcol_reduce_piece<false>(b->v, nullptr, 0.f, b->rows, b->cols, b->red, t.chunk, t.strip);
@@ -262,7 +298,27 @@ __device__ __forceinline__ double combine_reduced(const StepBlock* b, double bet
 
 __global__ void __launch_bounds__(kThreads)
 factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __restrict__ ids,
-                        const __grid_constant__ StepParams P) {
+                        const __grid_constant__ StepParams P BAOC_CHECK_PARAM) {
+#ifdef BAOC_CHECKED
+    {
+        const int cid = ids[blockIdx.x];
+        if (cid < 0 || cid >= ck.n_blocks) { check_fail(kChkBlockIndex, kKerFactoredCombine, cid, ck.n_blocks, blockIdx.x, 0); return; }
+        const StepBlock* cb = blocks + cid;
+        if (!check_range(ck, kKerFactoredCombine, cb->s0, 4ll * cb->rows, 0) || !check_range(ck, kKerFactoredCombine, cb->s1, 4ll * cb->cols, 1) ||
+            !check_range(ck, kKerFactoredCombine, cb->a0, 4, 2) ||
+            !check_range(ck, kKerFactoredCombine, cb->mean_part, 8ll * (kCombineSlabs + 1), 3) ||
+            !check_range(ck, kKerFactoredCombine, cb->red.rowpart, 8ll * cb->red.strips * cb->rows, 4) ||
+            !check_range(ck, kKerFactoredCombine, cb->red.colpart, 8ll * cb->red.chunks * cb->cols, 5))
+            return;
+        if (cb->fbits != 32) {
+            const int64_t eb = cb->fbits == 16 ? 2 : 1;
+            if (!check_range(ck, kKerFactoredCombine, cb->f0, eb * cb->rows, 6) || !check_range(ck, kKerFactoredCombine, cb->f1, eb * cb->cols, 7)) return;
+            if (cb->fbits == 8 && (!check_range(ck, kKerFactoredCombine, cb->fa0, 4ll * ((cb->rows + kQBlock - 1) / kQBlock), 8) ||
+                                   !check_range(ck, kKerFactoredCombine, cb->fa1, 4ll * ((cb->cols + kQBlock - 1) / kQBlock), 9)))
+                return;
+        }
+    }
+#endif
     __shared__ double total[1];
     const StepBlock* b = blocks + ids[blockIdx.x];
     const int rows = b->rows, cols = b->cols, slab = blockIdx.y;
@@ -918,7 +974,41 @@ template <int kFam>
 __global__ void __launch_bounds__(kThreads, kFam == kFamDense ? 4 : 3)
 fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
                   const void* const* __restrict__ grads, float* const* __restrict__ params,
-                  uint32_t* __restrict__ flags, const __grid_constant__ StepParams SP) {
+                  uint32_t* __restrict__ flags, const __grid_constant__ StepParams SP BAOC_CHECK_PARAM) {
+#ifdef BAOC_CHECKED
+    {   // validate the tile and every state range its path will touch before touching anything
+        if (int64_t(blockIdx.x) >= ck.n_tiles) { check_fail(kChkTileIndex, kKerFusedStep, blockIdx.x, ck.n_tiles, 0, 0); return; }
+        const Tile ct = tiles[blockIdx.x];
+        if (ct.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerFusedStep, ct.block, ck.n_blocks, blockIdx.x, 0); return; }
+        const StepBlock* cb = blocks + ct.block;
+        const int64_t te = step_tile_elems(cb->path), cbase = int64_t(ct.piece) * te, cn = min64(te, cb->numel - cbase);
+        if (!check_tile(ck, kKerFusedStep, blockIdx.x, ct.block, cbase, cb->numel) ||
+            !check_range(ck, kKerFusedStep, flags + ct.block, 4, 0) || cb->cfg < 0 || cb->cfg >= kMaxSlots ||
+            !check_caller_ptr(kKerFusedStep, grads[ct.block], 1) || !check_caller_ptr(kKerFusedStep, params[ct.block], 2))
+            return;
+        const int64_t q0 = cbase / kQBlock, nq = (cbase + cn + kQBlock - 1) / kQBlock - q0;
+        auto elems = [&](const void* p, int64_t bytes_per, int what) {
+            return check_range(ck, kKerFusedStep, static_cast<const char*>(p) + cbase * bytes_per, cn * bytes_per, what);
+        };
+        auto scales = [&](const float* p, int what) { return check_range(ck, kKerFusedStep, p + q0, 4 * nq, what); };
+        bool ok = true;
+        switch (cb->path) {
+            case kPathA32: ok = elems(cb->s0, 4, 10) && elems(cb->s1, 4, 11); break;
+            case kPathA16: ok = elems(cb->s0, 2, 10) && elems(cb->s1, 2, 11); break;
+            case kPathA8: ok = elems(cb->s0, 1, 10) && elems(cb->s1, 1, 11) && scales(cb->a0, 12) && scales(cb->a1, 13); break;
+            case kPathR: case kPathS: ok = elems(cb->s0, 4, 10); break;
+            case kPathR16: case kPathS16: ok = elems(cb->s0, 2, 10); break;
+            case kPathR8: ok = elems(cb->s1, 1, 11) && scales(cb->a1, 13); break;
+            case kPathS8: ok = elems(cb->s0, 1, 10) && scales(cb->a0, 12); break;
+            case kPathF:
+                ok = check_range(ck, kKerFusedStep, cb->s0, 4ll * cb->rows, 10) && check_range(ck, kKerFusedStep, cb->s1, 4ll * cb->cols, 11) &&
+                     check_range(ck, kKerFusedStep, cb->a0, 4, 12);
+                break;
+            default: break;
+        }
+        if (!ok) return;
+    }
+#endif
     const Tile t = tiles[blockIdx.x];
     const StepBlock* b = blocks + t.block;
     const CfgStep& P = SP.c[b->cfg];
@@ -963,10 +1053,31 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
         if (e_ != cudaSuccess) return int(e_);                \
     } while (0)
 
+BAOC_DEFINE_CHECK_FETCH(step_check_fetch)
+
+#ifdef BAOC_CHECKED
+// The range check run on numbers that violate it; no memory but the record is touched.
+__global__ void check_selftest_kernel(const CheckCtx ck) {
+    if (threadIdx.x == 0) check_range(ck, kKerSelfTest, ck.hi - 16, 32, 99);
+}
+#endif
+int launch_check_selftest(cudaStream_t s) {
+#ifdef BAOC_CHECKED
+    static char fake[64];                                   // a host range: only its addresses are compared, nothing dereferences them
+    const CheckCtx ck{fake, fake + 64, 0, 0, 0};
+    check_selftest_kernel<<<1, 32, 0, s>>>(ck);
+    BAOC_LAUNCH_CHECK();
+#else
+    (void)s;
+#endif
+    return 0;
+}
+
 int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const int32_t* ids, int64_t n_red, int n_matrix,
-                         cudaStream_t s) {
+                         const CheckCtx& ck, cudaStream_t s) {
+    (void)ck;
     if (n_red <= 0) return 0;
-    moment_reduce_kernel<<<unsigned(n_red), kThreads, 0, s>>>(blocks, rtiles);
+    moment_reduce_kernel<<<unsigned(n_red), kThreads, 0, s>>>(blocks, rtiles BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     moment_reduce_combine_kernel<<<dim3(unsigned(n_matrix), kCombineSlabs), kThreads, 0, s>>>(blocks, ids);
     BAOC_LAUNCH_CHECK();
@@ -976,22 +1087,25 @@ int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const i
 }
 
 int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const int32_t* ids, const void* const* grads,
-                           const float* const* params, int64_t n_red, int n_factored, const StepParams& P, cudaStream_t s) {
+                           const float* const* params, int64_t n_red, int n_factored, const StepParams& P, const CheckCtx& ck,
+                           cudaStream_t s) {
+    (void)ck;
     if (n_red <= 0) return 0;
-    factored_reduce_kernel<<<unsigned(n_red), kThreads, 0, s>>>(blocks, rtiles, grads, params, P);
+    factored_reduce_kernel<<<unsigned(n_red), kThreads, 0, s>>>(blocks, rtiles, grads, params, P BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
-    factored_combine_kernel<<<dim3(unsigned(n_factored), kCombineSlabs), kThreads, 0, s>>>(blocks, ids, P);
+    factored_combine_kernel<<<dim3(unsigned(n_factored), kCombineSlabs), kThreads, 0, s>>>(blocks, ids, P BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     return 0;
 }
 
 int launch_fused_step(const StepBlock* blocks, const Tile* tiles, const void* const* grads, float* const* params,
-                      uint32_t* flags, int64_t n_tiles, int family, const StepParams& P, cudaStream_t s) {
+                      uint32_t* flags, int64_t n_tiles, int family, const StepParams& P, const CheckCtx& ck, cudaStream_t s) {
+    (void)ck;
     if (n_tiles <= 0) return 0;
     const unsigned grid = unsigned(n_tiles);
-    if (family == kFamHead) fused_step_kernel<kFamHead><<<grid, kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
-    else if (family == kFamDense) fused_step_kernel<kFamDense><<<grid, kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
-    else fused_step_kernel<kFamQ8><<<grid, kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P);
+    if (family == kFamHead) fused_step_kernel<kFamHead><<<grid, kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P BAOC_CHECK_ARG(ck));
+    else if (family == kFamDense) fused_step_kernel<kFamDense><<<grid, kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P BAOC_CHECK_ARG(ck));
+    else fused_step_kernel<kFamQ8><<<grid, kThreads, 0, s>>>(blocks, tiles, grads, params, flags, P BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     return 0;
 }

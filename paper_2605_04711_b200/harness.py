@@ -51,6 +51,29 @@ def sum_over_ranks(value: float, dist=None, device="cpu") -> float:
     return float(t.item())
 
 
+GUARD_BYTES = 4096
+GUARD_BYTE = 0xC5
+
+
+def guarded_alloc(n_bytes: int, device, fill_zero: bool = False):
+    """A buffer of n_bytes bytes with GUARD_BYTES guard bytes of a fixed pattern before and after it, for tests of memory
+    safety where no memory checker can be run: returns (whole allocation, the usable view).  The view keeps the 256-byte
+    alignment of the allocation."""
+    whole = torch.empty(n_bytes + 2 * GUARD_BYTES, dtype=torch.uint8, device=device)
+    whole[:GUARD_BYTES] = GUARD_BYTE
+    whole[GUARD_BYTES + n_bytes:] = GUARD_BYTE
+    view = whole[GUARD_BYTES:GUARD_BYTES + n_bytes]
+    if fill_zero:
+        view.zero_()
+    return whole, view
+
+
+def guards_intact(whole: torch.Tensor) -> bool:
+    """True while nothing has written into the guard bytes around a buffer from ``guarded_alloc``."""
+    n = whole.numel() - 2 * GUARD_BYTES
+    return bool((whole[:GUARD_BYTES] == GUARD_BYTE).all().item() and (whole[GUARD_BYTES + n:] == GUARD_BYTE).all().item())
+
+
 def all_gather_params(local: torch.Tensor, out: torch.Tensor, dist) -> None:
     """The one exchange of a whole-block sharded step when replicas hold full weights: every rank contributes its flat
     parameter buffer ``local`` (all ranks' buffers have the same length, the longest shard's) and receives all of them
@@ -64,6 +87,9 @@ def all_gather_params(local: torch.Tensor, out: torch.Tensor, dist) -> None:
         dist.all_gather(list(out.view(dist.get_world_size(), -1).unbind(0)), local)
 
 
+LIVE_SESSIONS = None        # a weakref.WeakSet, created on first use: the sessions whose guards a test fixture verifies
+
+
 class Session:
     """One workload resident on one GPU.
 
@@ -75,6 +101,11 @@ class Session:
     def __init__(self, wl: W.Workload, configs: Optional[Sequence[B.Config]] = None, opts: Optional[B.Opts] = None,
                  n_grad_sets: int = 2, device: str = "cuda:0", pinned_host_grads: bool = False, samples=None,
                  param_capacity: int = 0, factored_group_bytes: int = 0):
+        global LIVE_SESSIONS
+        if LIVE_SESSIONS is None:
+            import weakref
+            LIVE_SESSIONS = weakref.WeakSet()
+        LIVE_SESSIONS.add(self)
         self.wl = wl
         self.device = torch.device(device)
         self.configs = list(configs) if configs is not None else B.default_configs()
@@ -83,8 +114,17 @@ class Session:
         self.n_grad_sets = n_grad_sets
         # param_capacity: allocate the parameter buffer at least this long (the longest shard's length, so that the
         # buffers of all ranks can be all-gathered as they are)
-        self.params = torch.zeros(max(self.total, int(param_capacity)), dtype=torch.float32, device=self.device)
-        self.grads = [torch.zeros(self.total, dtype=torch.bfloat16, device=self.device) for _ in range(n_grad_sets)]
+        # every device buffer sits between guard bytes (``verify_guards``)
+        self._guarded = []
+
+        def alloc(n_bytes, zero=False):
+            whole, view = guarded_alloc(n_bytes, self.device, zero)
+            self._guarded.append(whole)
+            return view
+
+        self._alloc = alloc
+        self.params = alloc(4 * max(self.total, int(param_capacity)), True).view(torch.float32)
+        self.grads = [alloc(2 * self.total, True).view(torch.bfloat16) for _ in range(n_grad_sets)]
         self.param_views = [self.params[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)]
         self.grad_views = [[g[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)] for g in self.grads]
         self.param_table = B.pointer_table(self.param_views)
@@ -99,11 +139,16 @@ class Session:
         self.samples = samples
         if samples is not None:
             self.h.set_sampling(samples)
-        self.ws = torch.empty(self.h.stats_workspace_bytes(), dtype=torch.uint8, device=self.device)
+        self.ws = alloc(self.h.stats_workspace_bytes())
         self.h.bind_stats_workspace(self.ws)
         self.state = None
         self.assign = None
         self._fixed_cache = {}
+
+    def verify_guards(self) -> bool:
+        """True while no kernel (or copy) has written outside any of this session's device buffers."""
+        torch.cuda.synchronize(self.device)
+        return all(guards_intact(w) for w in self._guarded)
 
     # ---- inputs -------------------------------------------------------------
     def init_params(self):
@@ -142,19 +187,19 @@ class Session:
 
     def configure(self, assign):
         self.assign = np.asarray(assign, np.int32)
-        self.state = torch.empty(self.h.state_bytes(self.assign), dtype=torch.uint8, device=self.device)
+        self.state = self._alloc(self.h.state_bytes(self.assign))
         self.h.configure(self.assign, self.state)
 
     def configure_from_window(self, assign):
         """Instantiate the optimizer with the window's moments as its initial moments."""
         self.assign = np.asarray(assign, np.int32)
-        self.state = torch.empty(self.h.state_bytes(self.assign), dtype=torch.uint8, device=self.device)
+        self.state = self._alloc(self.h.state_bytes(self.assign))
         self.h.configure_from_window(self.assign, self.state)
 
     def reconfigure(self, assign, steps_done: int, inherit: bool = True):
         """Move to a new assignment in a fresh state buffer (the old one stays alive until the stream has passed)."""
         self.assign = np.asarray(assign, np.int32)
-        new_state = torch.empty(self.h.state_bytes(self.assign), dtype=torch.uint8, device=self.device)
+        new_state = self._alloc(self.h.state_bytes(self.assign))
         self.h.reconfigure(self.assign, new_state, steps_done, inherit)
         self.state = new_state
 

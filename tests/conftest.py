@@ -24,3 +24,21 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _memory_safety(request):
+    """After every GPU test: no buffer of a live harness session has been written outside its bounds (guard bytes
+    around every device buffer), and, when the checked build of the library is loaded (BAOC_CHECKED=1), none of its
+    kernels has recorded a violation."""
+    yield
+    if "gpu" not in request.keywords:
+        return
+    B = sys.modules.get("paper_2605_04711_b200.binding")
+    H = sys.modules.get("paper_2605_04711_b200.harness")
+    if B is not None:
+        status = B.check_status()
+        assert status["code"] == 0, status
+    if H is not None and H.LIVE_SESSIONS:
+        for sess in list(H.LIVE_SESSIONS):
+            assert sess.verify_guards(), "a kernel wrote outside a device buffer of " + sess.wl.name

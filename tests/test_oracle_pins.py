@@ -914,3 +914,175 @@ def test_partition_invariants_on_random_inputs():
                 members_a, members_b = np.nonzero(ids == b)[0], np.nonzero(ids == b + 1)[0]
                 edge = O.partition_delta(Z[members_a[-1]], Z[members_b[0]], np.ones(5))
                 assert edge > tau or O.partition_delta(za, zb, np.ones(5)) > tau
+
+
+# ---------------------------------------------------------------- non-linear 8-bit codebook (alternative reading of the quantiser)
+
+def test_dynamic_codebook_entries_by_hand():
+    ts, tu = O.dynamic_codebook(True), O.dynamic_codebook(False)
+    assert ts.shape == (255,) and tu.shape == (256,)
+    assert np.all(np.diff(ts) > 0) and np.all(np.diff(tu) > 0)
+    np.testing.assert_array_equal(ts, -ts[::-1])                     # symmetric; the middle entry is zero
+    assert ts[127] == 0.0 and tu[0] == 0.0 and ts[-1] == 1.0 and ts[0] == -1.0 and tu[-1] == 1.0
+    # decade E of the signed type has 2^(6-E) entries in (10^-(E+1), 10^-E]; written out: the top decade 64 steps of
+    # 0.9/64 above 0.1, the next one 32 steps of 0.09/32 above 0.01, ..., the last one the single value 1e-6
+    pos = ts[128:]
+    assert pos.shape == (127,)
+    assert abs(pos[0] - 1e-6) < 1e-21 and abs(pos[1] - 0.55e-5) < 1e-20 and abs(pos[2] - 1e-5) < 1e-20
+    assert abs(pos[-64] - (0.1 + 0.9 / 64)) < 1e-16 and abs(pos[-65] - 0.1) < 1e-16 and abs(pos[-2] - (1.0 - 0.9 / 64)) < 1e-16
+    for E in range(7):
+        n = int(np.sum((pos > 10.0 ** -(E + 1) * (1 + 1e-12)) & (pos <= 10.0 ** -E * (1 + 1e-12))))
+        assert n == 2 ** (6 - E), (E, n)
+    # unsigned: one more fraction bit per decade and one more decade
+    upos = tu[1:]
+    assert abs(upos[0] - 1e-7) < 1e-22 and abs(upos[-128] - (0.1 + 0.9 / 128)) < 1e-16
+    for E in range(8):
+        assert int(np.sum((upos > 10.0 ** -(E + 1) * (1 + 1e-12)) & (upos <= 10.0 ** -E * (1 + 1e-12)))) == 2 ** (7 - E)
+
+
+def test_dynamic_codebook_round_trip_nearest_entry_and_ties():
+    for signed in (True, False):
+        t = O.dynamic_codebook(signed)
+        a = np.float32(0.5)                                           # a power of two: entry * a is exact
+        x = t * float(a)
+        if not signed:
+            x = x.copy()                                              # the block's absmax must be a: its last entry is 1 * a
+        codes, am = O.quantize8_dynamic(x, signed, qblock=len(t))
+        np.testing.assert_array_equal(codes, np.arange(len(t), dtype=np.uint8))
+        assert am.tolist() == [0.5]
+        np.testing.assert_array_equal(O.dequantize8_dynamic(codes, am, signed, qblock=len(t)), x)
+        # nearest entry: brute force over the table
+        y = RNG.uniform(-1.0 if signed else 0.0, 1.0, 3000)
+        y[0] = 1.0                                                    # absmax 1
+        codes, am = O.quantize8_dynamic(y, signed, qblock=3000)
+        brute = np.argmin(np.abs(y[:, None] - t[None, :]), axis=1)
+        np.testing.assert_array_equal(codes, brute.astype(np.uint8))
+        # a tie goes to the entry of smaller magnitude
+        k = len(t) - 3
+        tie = np.array([1.0, 0.5 * (t[k] + t[k + 1])])
+        assert O.quantize8_dynamic(tie, signed, qblock=2)[0][1] == k
+    ts = O.dynamic_codebook(True)
+    tie = np.array([-1.0, 0.5 * (ts[2] + ts[3])])
+    assert O.quantize8_dynamic(tie, True, qblock=2)[0][1] == 3        # negative: the upper entry is the smaller one
+    c0, a0 = O.quantize8_dynamic(np.zeros(300), True)
+    assert not a0.any() and not O.dequantize8_dynamic(c0, a0, True).any()
+
+
+def test_dynamic_codebook_keeps_small_second_moments_that_linear_codes_lose():
+    """What the non-linear table is for: a second moment 1e-4 of its block's absmax survives (relative error below 10 %)
+    where the linear code rounds it to zero."""
+    v = np.array([1.0, 1e-4, 3e-6, 0.0])
+    cl, al = O.quantize8(v, False, 4)
+    assert O.dequantize8(cl, al, False, 4)[1] == 0.0
+    cd, ad = O.quantize8_dynamic(v, False, 4)
+    vd = O.dequantize8_dynamic(cd, ad, False, 4)
+    assert abs(vd[1] - 1e-4) <= 0.1 * 1e-4 and abs(vd[2] - 3e-6) <= 0.2 * 3e-6 and vd[3] == 0.0 and vd[0] == 1.0
+
+
+def test_adam_on_the_dynamic_codebook_by_hand_and_against_fp32():
+    c = O.Config(1, 1, 1, 0, 8, lr=1e-2, beta1=0.5, beta2=0.5, eps=0.0, weight_decay=0.0, quantizer="dynamic")
+    assert O.config_kind(c) == "A8N"
+    st = O.step_init(c, 2, 2, 1, qblock=2)
+    g = np.array([1.0, -0.25])
+    th = O.step(np.zeros(2), g, st, c, 2, 1, qblock=2)
+    # m = g/2, v = g^2/2; bias corrections 1/2 each: theta = -lr * g / |g|
+    np.testing.assert_allclose(th, [-1e-2, 1e-2], rtol=0, atol=1e-15)
+    ts, tu = O.dynamic_codebook(True), O.dynamic_codebook(False)
+    assert st.am.tolist() == [0.5] and st.av.tolist() == [0.5]
+    # m / a = (1, -0.25): 0.25 lies between the entries 0.1 + 0.9 * 10/64 = 0.240625 and 0.1 + 0.9 * 11/64 = 0.2546875
+    assert ts[st.qm[0]] == 1.0 and abs(ts[st.qm[1]] + 0.2546875) < 1e-16
+    # v / a = (1, 1/16): the decade (0.01, 0.1] of the unsigned type has 64 entries 0.01 + 0.09 (k+1)/64; k + 1 = 37 is nearest
+    assert tu[st.qv[0]] == 1.0 and abs(tu[st.qv[1]] - (0.01 + 0.09 * 37 / 64)) < 1e-16
+    # ten steps stay close to the fp32 rule (the codebook's relative error is a few per cent per entry)
+    c32 = O.Config(1, 1, 1, 0, 32, lr=1e-3, weight_decay=0.01)
+    c8n = O.Config(1, 1, 1, 0, 8, lr=1e-3, weight_decay=0.01, quantizer="dynamic")
+    d = 700
+    s32, s8 = O.step_init(c32, d, d, 1), O.step_init(c8n, d, d, 1)
+    th32 = th8 = RNG.standard_normal(d) * 0.02
+    for t in range(10):
+        g = RNG.standard_normal(d) * 1e-2
+        th32, th8 = O.step(th32, g, s32, c32, d, 1), O.step(th8, g, s8, c8n, d, 1)
+    assert np.max(np.abs(th32 - th8)) < 5e-4 and np.max(np.abs(th32 - th8)) > 0.0
+    m8 = O.dequantize8_dynamic(s8.qm, s8.am, True)
+    assert np.max(np.abs(m8 - s32.m)) <= 0.08 * np.max(np.abs(s32.m))
+
+
+def test_precision_cosine_with_the_dynamic_codebook():
+    o = O.Opts(qblock=4, eps_adam=0.0, eps=0.0, quantizer8="dynamic")
+    m = np.array([1.0, -0.5, 0.26, 0.0])
+    v = np.array([4.0, 1.0, 0.25, 2.0])
+    ts, tu = O.dynamic_codebook(True), O.dynamic_codebook(False)
+    near = lambda t, y: t[np.argmin(np.abs(t - y))]
+    mq = np.array([near(ts, x / 1.0) * 1.0 for x in m])
+    vq = np.array([near(tu, x / 4.0) * 4.0 for x in v])
+    u32, u8 = m / np.sqrt(v), mq / np.sqrt(vq)
+    want = u32 @ u8 / (np.linalg.norm(u32) * np.linalg.norm(u8))
+    assert abs(O.precision_cosine(m, v, 8, o) - want) < 1e-14
+    assert abs(O.precision_cosine(m, v, 8, o) - O.precision_cosine(m, v, 8, O.Opts(qblock=4, eps_adam=0.0, eps=0.0))) > 1e-9
+    want_err = math.sqrt(float(np.sum((v - vq) ** 2))) / math.sqrt(float(np.sum(v * v)))
+    assert abs(O.quant_rel_error(v, 8, False, o) - want_err) < 1e-15
+
+
+# ---------------------------------------------------------------- Adafactor options of the factored tuple
+
+def test_adafactor_options_off_is_the_mechanism_pure_rule():
+    G = RNG.standard_normal((5, 7))
+    th0 = RNG.standard_normal(35) * 0.02
+    base = O.Config(1, 0, 1, 1, 32, lr=1e-3, beta2=0.9, weight_decay=0.01)
+    same = O.Config(1, 0, 1, 1, 32, lr=1e-3, beta2=0.9, weight_decay=0.01, af_beta2_schedule=False, af_clip=0.0,
+                    af_relative_step=False, af_eps1=0.0)
+    s1, s2 = O.step_init(base, 35, 5, 7), O.step_init(same, 35, 5, 7)
+    np.testing.assert_array_equal(O.step(th0, G.reshape(-1), s1, base, 5, 7), O.step(th0, G.reshape(-1), s2, same, 5, 7))
+
+
+def test_adafactor_beta2_schedule_clipping_and_relative_step_by_hand():
+    # a 2 x 2 block, two steps, every quantity written out
+    G1 = np.array([[3.0, 1.0], [1.0, 2.0]])
+    G2 = np.array([[1.0, -2.0], [0.5, 1.0]])
+    th0 = np.array([0.5, -0.5, 0.25, 1.0])
+    c = O.Config(1, 0, 1, 1, 32, lr=123.0, beta2=0.999, eps=0.0, weight_decay=0.0, af_beta2_schedule=True, af_clip=1.0,
+                 af_relative_step=True, af_eps1=1e-30)
+    st = O.step_init(c, 4, 2, 2)
+    th1 = O.step(th0, G1.reshape(-1), st, c, 2, 2)
+    # step 1: beta2_1 = 1 - 1^-0.8 = 0, so r and c are the row and column means of g^2 (+ eps1, invisible here)
+    r1, c1 = np.array([5.0, 2.5]), np.array([5.0, 2.5])
+    np.testing.assert_allclose(st.r, r1, rtol=1e-15); np.testing.assert_allclose(st.c, c1, rtol=1e-15)
+    v1 = np.outer(r1, c1) / 3.75
+    u1 = G1 / np.sqrt(v1)                                             # no bias correction under the schedule
+    rms1 = math.sqrt(float(np.mean(u1 ** 2)))
+    assert rms1 > 1.0
+    u1 = u1 / rms1                                                    # clipped to RMS 1 (d = 1)
+    alpha1 = max(1e-3, math.sqrt(float(np.mean(th0 ** 2)))) * min(1e-2, 1.0)
+    np.testing.assert_allclose(th1, th0 - alpha1 * u1.reshape(-1), rtol=1e-14)
+    th2 = O.step(th1, G2.reshape(-1), st, c, 2, 2)
+    b2 = 1.0 - 2.0 ** -0.8                                            # 0.42565...
+    assert abs(b2 - 0.4256508) < 1e-7
+    r2 = b2 * r1 + (1 - b2) * (G2 ** 2).mean(axis=1)
+    c2 = b2 * c1 + (1 - b2) * (G2 ** 2).mean(axis=0)
+    v2 = np.outer(r2, c2) / r2.mean()
+    u2 = G2 / np.sqrt(v2)
+    u2 = u2 / max(1.0, math.sqrt(float(np.mean(u2 ** 2))))
+    alpha2 = max(1e-3, math.sqrt(float(np.mean(th1 ** 2)))) * min(1e-2, 1.0 / math.sqrt(2.0))
+    np.testing.assert_allclose(th2, th1 - alpha2 * u2.reshape(-1), rtol=1e-13)
+    # each option alone changes the result, and the configured lr is not used under the relative step
+    for kw in (dict(af_beta2_schedule=True), dict(af_clip=1.0), dict(af_relative_step=True)):
+        ca = O.Config(1, 0, 1, 1, 32, lr=1e-3, beta2=0.9, **kw)
+        cb = O.Config(1, 0, 1, 1, 32, lr=1e-3, beta2=0.9)
+        sa, sb = O.step_init(ca, 4, 2, 2), O.step_init(cb, 4, 2, 2)
+        ta, tb = th0, th0
+        for G in (G1, G2):
+            ta, tb = O.step(ta, G.reshape(-1), sa, ca, 2, 2), O.step(tb, G.reshape(-1), sb, cb, 2, 2)
+        assert np.max(np.abs(ta - tb)) > 1e-6, kw
+    # small update: no clipping happens (the factor is max(1, .))
+    cs = O.Config(1, 0, 1, 1, 32, lr=1e-3, beta2=0.9, eps=10.0, af_clip=1.0)
+    cn = O.Config(1, 0, 1, 1, 32, lr=1e-3, beta2=0.9, eps=10.0)
+    np.testing.assert_array_equal(O.step(th0, G1.reshape(-1), O.step_init(cs, 4, 2, 2), cs, 2, 2),
+                                  O.step(th0, G1.reshape(-1), O.step_init(cn, 4, 2, 2), cn, 2, 2))
+    # relative step with a decoupled decay: the decay uses the same step size
+    cw = O.Config(1, 0, 1, 1, 32, lr=7.0, beta2=0.9, eps=0.0, weight_decay=0.5, af_relative_step=True)
+    sw = O.step_init(cw, 4, 2, 2)
+    tw = O.step(th0, G1.reshape(-1), sw, cw, 2, 2)
+    a = max(1e-3, math.sqrt(float(np.mean(th0 ** 2)))) * 1e-2
+    vw = np.outer(0.1 * r1, 0.1 * c1) / (0.1 * 3.75)
+    uw = G1 / np.sqrt(vw / (1 - 0.9))
+    np.testing.assert_allclose(tw, th0 * (1 - a * 0.5) - a * uw.reshape(-1), rtol=1e-13)
