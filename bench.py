@@ -28,7 +28,8 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 CONFIG_NAMES = ["adamw32", "adamw8", "rms", "factored", "sgdm"]
-EXTENDED_NAMES = CONFIG_NAMES + ["sgd", "adamw16", "rms16", "sgdm16", "rms8", "sgdm8", "factored16", "factored8"]
+EXTENDED_NAMES = CONFIG_NAMES + ["sgd", "adamw16", "rms16", "sgdm16", "rms8", "sgdm8", "factored16", "factored8",
+                                 "adamw8_dynamic", "adafactor"]
 METRIC = "hot-path throughput: statistics pass + mixed-config optimizer step"
 UNIT = "params/s"
 
@@ -189,7 +190,10 @@ def time_oracle(wl, assign, steps, warmup, target_params, configs=None, slice_ro
                 setattr(c, k, float(np.float32(getattr(c, k))))
     else:
         cfgs = [O.Config(c.adaptive, c.momentum, c.decoupled_wd, c.factored, c.bits, lr=float(c.lr), beta1=float(c.beta1),
-                         beta2=float(c.beta2), eps=float(c.eps), weight_decay=float(c.weight_decay)) for c in configs]
+                         beta2=float(c.beta2), eps=float(c.eps), weight_decay=float(c.weight_decay),
+                         quantizer="dynamic" if c.quantizer else "linear", af_beta2_schedule=bool(c.af_flags & 1),
+                         af_clip=1.0 if c.af_flags & 2 else 0.0, af_relative_step=bool(c.af_flags & 4),
+                         af_eps1=1e-30 if c.af_flags & 8 else 0.0) for c in configs]
     picked, total = _sample_blocks(wl, target_params, slice_rows)
     opts = O.Opts()
     kinds = []
@@ -315,7 +319,7 @@ def run_ours(args):
     if args.assign != "auto":
         # one configuration for every block (vectors cannot be factored: they take the momentum-free one of the same width)
         c = names.index(args.assign)
-        vec = {"factored": "rms", "factored16": "rms16", "factored8": "rms8"}
+        vec = {"factored": "rms", "factored16": "rms16", "factored8": "rms8", "adafactor": "rms"}
         assign = np.asarray([names.index(vec[args.assign]) if (args.assign in vec and b.cols <= 1) else c for b in wl.blocks],
                             np.int32)
     sess.configure(assign)

@@ -64,10 +64,12 @@ typedef struct {
 /* A configuration tuple c = (y_a, y_m, y_d, y_f, b) of Definition 3.1 and the
  * hyper-parameters of the update rule it selects.  Tuples the library can
  * instantiate (Sec. 4.1 lists the mechanisms, each at 8/16/32-bit states):
- *   (1,1,*,0,32|16|8)  Adam / AdamW with fp32, bf16 or block-wise absmax 8-bit moments;
+ *   (1,1,*,0,32|16|8)  Adam / AdamW with fp32, bf16 or block-wise absmax 8-bit moments (8-bit: linear codes or the
+ *                      non-linear codebook, see quantizer);
  *   (1,0,*,0,32|16|8)  momentum-free RMS scaling with an fp32, bf16 or 8-bit second moment;
  *   (1,0,*,1,32|16|8)  factored second moment (matrix blocks only), its row and column statistics kept
- *                      in fp32, in bf16 or as block-wise absmax 8-bit codes;
+ *                      in fp32, in bf16 or as block-wise absmax 8-bit codes; optionally with the remaining parts
+ *                      of Adafactor (see af_flags);
  *   (0,1,*,0,32|16|8)  SGD with momentum (beta1 is the momentum coefficient), fp32, bf16 or 8-bit buffer;
  *   (0,0,*,0,any)      plain gradient step (SGD / SGDW): no state, so the bit-width only enters Agg(c).
  * y_d selects decoupled (1) or coupled (0) weight decay in all of them.  With
@@ -77,9 +79,43 @@ typedef struct {
  * but cannot be assigned. */
 typedef struct {
     uint8_t adaptive, momentum, decoupled_wd, factored, bits;
-    uint8_t reserved[3];
+    uint8_t quantizer;   /* 8-bit Adam only: 0 = linear absmax codes, 1 = the non-linear codebook (below) */
+    uint8_t af_flags;    /* factored tuple only: Adafactor's options (below), 0 = none */
+    uint8_t reserved;    /* 0 */
     float lr, beta1, beta2, eps, weight_decay;
 } baoc_config_t;
+
+/* Two alternative readings that a configuration may select.
+ *
+ * quantizer = BAOC_Q_DYNAMIC.  The paper calls Q_b "a standard quantizer" and
+ * cites block-wise 8-bit optimizers for its AdamW8 baseline (Sec. 4.1).  Their
+ * data type is non-linear: an optional sign bit, a run of zero bits whose
+ * length E is a decimal exponent, an indicator bit, and F remaining bits as a
+ * linear fraction of the decade.  This library builds its own table from that
+ * description: magnitudes 10^-E (0.1 + 0.9 (k+1) / 2^F), k = 0 .. 2^F - 1,
+ * F = B - 1 - E, E = 0 .. B - 1, with B = 7 for first moments (signed: 255
+ * entries with zero) and B = 8 for second moments (256 entries with zero).  A
+ * code is the index of the entry nearest to x / absmax in ascending order (a
+ * tie goes to the smaller magnitude); blocks of 256 elements and fp32 absmax as
+ * for the linear codes.  Offered for the tuple (1,1,*,0,8); baoc_opts_t's
+ * quantizer8 selects it for the precision cosine of Eq. 8.
+ *
+ * af_flags.  The paper names Adafactor among its mechanisms (Sec. 4.1) without
+ * saying which parts of the published algorithm are meant; the factored tuple
+ * by default keeps only the factored second moment.  The flags add the rest:
+ *   BAOC_AF_SCHEDULE  beta2_t = 1 - t^-0.8 instead of the constant beta2, and
+ *                     no bias correction of the second moment;
+ *   BAOC_AF_CLIP      the update u = g / (sqrt(v) + eps) is divided by
+ *                     max(1, RMS(u)) (clipping threshold 1);
+ *   BAOC_AF_RELATIVE  step size max(1e-3, RMS(theta)) * min(1e-2, 1/sqrt(t))
+ *                     instead of lr, with theta before the step (a decoupled
+ *                     decay uses the same step size);
+ *   BAOC_AF_EPS1      1e-30 is added to every squared gradient before the row
+ *                     and column means.
+ * Clipping and the relative step need the norms of u and theta over the whole
+ * block: one more sweep over the block's gradient and parameters per step. */
+enum { BAOC_Q_LINEAR = 0, BAOC_Q_DYNAMIC = 1 };
+enum { BAOC_AF_SCHEDULE = 1, BAOC_AF_CLIP = 2, BAOC_AF_RELATIVE = 4, BAOC_AF_EPS1 = 8 };
 
 /* Options of the statistics, normalisation and allocation (defaults from
  * baoc_default_opts: Eq. 3 "standard Adam values", Appendix A anchors,
@@ -97,6 +133,8 @@ typedef struct {
     int32_t use_snr;              /* Eq. 17; 0 selects s_M = s_rho */
     int32_t qblock;               /* elements per 8-bit quantisation block */
     int64_t node_limit;           /* allocator search-node limit (0 = default) */
+    int32_t quantizer8;           /* the 8-bit quantiser of Eq. 8: BAOC_Q_LINEAR (default) or BAOC_Q_DYNAMIC */
+    int32_t reserved;             /* 0 */
 } baoc_opts_t;
 
 /* Per-block diagnostics z_i: raw (Eq. 4-8), normalised (Eq. 10-20) and a few
@@ -440,7 +478,8 @@ int baoc_profile_last(baoc_t* h, float* ms2);
  * b = offset of the range in the buffer, c = its bytes, d = the buffer's
  * bytes), 5 null pointer; kernel: 1 statistics step, 2 its combine, 3 sample
  * gather, 4 first finalize sweep, 5 later sweeps, 6 / 7 row-column reduction of
- * the window / of the step, 8 its combine, 9 fused step, 10 the self-test.
+ * the window / of the step, 8 its combine, 9 fused step, 10 the self-test, 11 the norms of the
+ * factored tuple's Adafactor options.
  *
  * baoc_check_selftest: queues a one-thread kernel that runs the range check on
  * numbers that violate it (a 32-byte range that starts 16 bytes before the end

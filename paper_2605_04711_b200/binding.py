@@ -44,7 +44,8 @@ class Block(C.Structure):
 
 class Config(C.Structure):
     _fields_ = [("adaptive", C.c_uint8), ("momentum", C.c_uint8), ("decoupled_wd", C.c_uint8),
-                ("factored", C.c_uint8), ("bits", C.c_uint8), ("reserved", C.c_uint8 * 3),
+                ("factored", C.c_uint8), ("bits", C.c_uint8), ("quantizer", C.c_uint8), ("af_flags", C.c_uint8),
+                ("reserved", C.c_uint8),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
                 ("weight_decay", C.c_float)]
 
@@ -53,7 +54,8 @@ class Opts(C.Structure):
     _fields_ = [("beta_m", C.c_double), ("beta_v", C.c_double), ("beta_rho", C.c_double), ("eps", C.c_double),
                 ("a_lo", C.c_double), ("a_hi", C.c_double), ("rho_lo", C.c_double), ("rho_hi", C.c_double),
                 ("snr_lo", C.c_double), ("snr_hi", C.c_double), ("w", C.c_double * 5), ("gamma", C.c_double),
-                ("eps_adam", C.c_double), ("use_snr", C.c_int32), ("qblock", C.c_int32), ("node_limit", C.c_int64)]
+                ("eps_adam", C.c_double), ("use_snr", C.c_int32), ("qblock", C.c_int32), ("node_limit", C.c_int64),
+                ("quantizer8", C.c_int32), ("reserved", C.c_int32)]
 
 
 class BlockStats(C.Structure):
@@ -193,9 +195,14 @@ def default_opts() -> Opts:
     return o
 
 
+Q_LINEAR, Q_DYNAMIC = 0, 1
+AF_SCHEDULE, AF_CLIP, AF_RELATIVE, AF_EPS1 = 1, 2, 4, 8
+
+
 def make_config(adaptive, momentum, decoupled_wd, factored, bits, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8,
-                weight_decay=0.0) -> Config:
-    return Config(adaptive, momentum, decoupled_wd, factored, bits, (C.c_uint8 * 3)(), lr, beta1, beta2, eps,
+                weight_decay=0.0, quantizer=Q_LINEAR, af_flags=0) -> Config:
+    """quantizer: Q_DYNAMIC puts 8-bit Adam on the non-linear codebook; af_flags: Adafactor's options of the factored tuple."""
+    return Config(adaptive, momentum, decoupled_wd, factored, bits, quantizer, af_flags, 0, lr, beta1, beta2, eps,
                   weight_decay)
 
 
@@ -209,7 +216,8 @@ def default_configs() -> List[Config]:
 def extended_configs() -> List[Config]:
     """The five default tuples plus the plain gradient step, the bf16-state variants of Adam(W), RMS scaling and
     SGD with momentum, the 8-bit variants of RMS scaling and SGD with momentum, and the factored second moment with
-    bf16 and 8-bit row / column statistics (indices 11 and 12)."""
+    bf16 and 8-bit row / column statistics (indices 11 and 12); then the two alternative readings: Adam on the
+    non-linear 8-bit codebook (13) and the factored tuple with all of Adafactor's options (14)."""
     return default_configs() + [make_config(0, 0, 1, 0, 32, lr=1e-2, weight_decay=0.01),
                                 make_config(1, 1, 1, 0, 16, weight_decay=0.01),
                                 make_config(1, 0, 1, 0, 16, weight_decay=0.01),
@@ -217,7 +225,10 @@ def extended_configs() -> List[Config]:
                                 make_config(1, 0, 1, 0, 8, weight_decay=0.01),
                                 make_config(0, 1, 1, 0, 8, lr=1e-2, weight_decay=0.01),
                                 make_config(1, 0, 1, 1, 16, weight_decay=0.01),
-                                make_config(1, 0, 1, 1, 8, weight_decay=0.01)]
+                                make_config(1, 0, 1, 1, 8, weight_decay=0.01),
+                                make_config(1, 1, 1, 0, 8, weight_decay=0.01, quantizer=Q_DYNAMIC),
+                                make_config(1, 0, 1, 1, 32, weight_decay=0.01,
+                                            af_flags=AF_SCHEDULE | AF_CLIP | AF_RELATIVE | AF_EPS1)]
 
 
 def pointer_table(tensors: Sequence[torch.Tensor]):

@@ -118,14 +118,23 @@ void fill_step_params(const Handle* h, int64_t t, StepParams* P) {
         o.decay = (has_wd && k.decoupled_wd) ? -float(lr * double(k.weight_decay)) : 0.0f;
         // each moment counts the gradients it has seen since it last started from zero
         const double tm = double(std::max<int64_t>(1, t - slot.t_m0)), tv = double(std::max<int64_t>(1, t - slot.t_v0));
-        const double bc1 = 1.0 - std::pow(b1, tm), bc2 = 1.0 - std::pow(b2, tv);
+        double bc2 = 1.0 - std::pow(b2, tv);
+        const double bc1 = 1.0 - std::pow(b1, tm);
+        o.af_flags = k.factored ? int32_t(k.af_flags) : 0;
+        double b2_now = b2;
+        if (o.af_flags & kAfSchedule) {                    // Adafactor: beta2_t = 1 - t^-0.8, no bias correction
+            b2_now = 1.0 - std::pow(tv, -0.8);
+            bc2 = 1.0;
+        }
+        o.eps1_d = (o.af_flags & kAfEps1) ? 1e-30 : 0.0;
+        o.rho_d = std::min(1e-2, 1.0 / std::sqrt(tv));
         o.step_m = float(lr / bc1);
         o.step_g = k.lr;
         o.rsqrt_bc2 = float(1.0 / std::sqrt(bc2));
         o.step_m_hat = float(lr / bc1 * std::sqrt(bc2));
         o.step_g_hat = float(lr * std::sqrt(bc2));
         o.eps_hat = float(double(k.eps) * std::sqrt(bc2));
-        o.beta1_d = b1; o.beta2_d = b2; o.wd_d = double(k.weight_decay);
+        o.beta1_d = b1; o.beta2_d = b2_now; o.wd_d = double(k.weight_decay);
     }
 }
 
@@ -183,13 +192,10 @@ int step_group(Handle* h, const Handle::GroupStep& g, const StepParams& P, cudaS
     return BAOC_OK;
 }
 
-// One step of every block: the whole tile table, one launch per path family present.
-int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t, cudaStream_t s) {
-    StepParams P;
-    int rc = step_prologue(h, grads, params, t, s, &P);
-    if (rc) return rc;
+// The launches of one step of every block, after the prologue: the whole tile table, one launch per path family present.
+int step_launches(Handle* h, const StepParams& P, cudaStream_t s) {
     const auto& L = h->tl;
-    const bool grouped = h->factored_group_bytes > 0 && h->n_factored > 0;
+    const bool grouped = h->factored_group_bytes > 0 && h->n_factored > 0 && h->n_fa == 0;   // blocks with Adafactor's options keep the one-reduction schedule
     if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[0]), s), "baoc_step (profile)");
     if (h->n_factored > 0 && !grouped) {
         LAUNCH(launch_factored_reduce(at<StepBlock>(h->st, L.blocks), at<RedTile>(h->st, L.red_tiles),
@@ -198,6 +204,13 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
                                       st_ctx(h, h->n_step_red_tiles), s),
                "factored_reduce_kernel");
         h->launches += 2;
+        if (h->n_fa > 0) {
+            LAUNCH(launch_factored_norms(at<StepBlock>(h->st, L.blocks), at<Tile>(h->st, L.tiles) + h->fa_tile0,
+                                         at<int32_t>(h->st, L.f_ids) + h->n_factored, at<const void*>(h->st, L.grads),
+                                         at<const float*>(h->st, L.params), h->n_fa_tiles, h->n_fa, P, st_ctx(h, h->n_fa_tiles), s),
+                   "factored_norms_kernel");
+            h->launches += 2;
+        }
     }
     if (h->prof_on) CU(cudaEventRecord(static_cast<cudaEvent_t>(h->prof_ev[1]), s), "baoc_step (profile)");
     int64_t first = 0;
@@ -233,6 +246,13 @@ int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t
         h->prof_valid = true;
     }
     return BAOC_OK;
+}
+
+int do_step(Handle* h, const void* const* grads, float* const* params, int64_t t, cudaStream_t s) {
+    StepParams P;
+    int rc = step_prologue(h, grads, params, t, s, &P);
+    if (rc) return rc;
+    return step_launches(h, P, s);
 }
 
 }  // namespace
@@ -364,7 +384,7 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
     }
     LAUNCH(launch_final_sums(blocks, tiles, dparams, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<uint32_t>(ws, L.hist),
                              at<RankSel>(ws, L.sel), h->n_stat_tiles, n, h->opts.eps, float(h->opts.eps_adam),
-                             ws_ctx(h, h->n_stat_tiles), s),
+                             h->opts.quantizer8, ws_ctx(h, h->n_stat_tiles), s),
            "final_sums_kernel");
     h->launches += 5;
     if (h->n_matrix > 0) {
@@ -460,16 +480,17 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
         StepBlock& b = sb[i];
         auto fix = [&](void* p) { return static_cast<void*>(st + L.states + reinterpret_cast<size_t>(p)); };
         auto fix_scratch = [&](void* p) { return static_cast<void*>(st + L.redpart + reinterpret_cast<size_t>(p)); };
-        if (b.path == kPathF && b.fbits != 32) {
+        if (is_factored_path(b.path) && b.fbits != 32) {
             b.s0 = fix_scratch(b.s0); b.s1 = fix_scratch(b.s1);
             b.f0 = fix(b.f0); b.f1 = fix(b.f1);
             if (b.fbits == 8) { b.fa0 = static_cast<float*>(fix(b.fa0)); b.fa1 = static_cast<float*>(fix(b.fa1)); }
-        } else if (b.path == kPathA32 || b.path == kPathA8 || b.path == kPathF || b.path == kPathA16) { b.s0 = fix(b.s0); b.s1 = fix(b.s1); }
+        } else if (b.path == kPathA32 || b.path == kPathA8 || b.path == kPathA8N || is_factored_path(b.path) || b.path == kPathA16) { b.s0 = fix(b.s0); b.s1 = fix(b.s1); }
         else if (b.path == kPathR8) { b.s1 = fix(b.s1); b.a1 = static_cast<float*>(fix(b.a1)); }
         else if (b.path == kPathS8) { b.s0 = fix(b.s0); b.a0 = static_cast<float*>(fix(b.a0)); }
         else if (b.path != kPathG) b.s0 = fix(b.s0);
-        if (b.path == kPathA8) { b.a0 = static_cast<float*>(fix(b.a0)); b.a1 = static_cast<float*>(fix(b.a1)); }
-        if (b.path == kPathF) {
+        if (b.path == kPathA8 || b.path == kPathA8N) { b.a0 = static_cast<float*>(fix(b.a0)); b.a1 = static_cast<float*>(fix(b.a1)); }
+        if (b.path == kPathFA) b.norm_part = reinterpret_cast<double*>(st + L.redpart + reinterpret_cast<size_t>(b.norm_part));
+        if (is_factored_path(b.path)) {
             b.a0 = static_cast<float*>(fix(b.a0));
             b.red.rowpart = reinterpret_cast<double*>(st + L.redpart + reinterpret_cast<size_t>(b.red.rowpart));
             b.red.colpart = reinterpret_cast<double*>(st + L.redpart + reinterpret_cast<size_t>(b.red.colpart));
@@ -485,13 +506,12 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
     {
         std::vector<int> gb0, gb1;
         compute_copy_groups(h, &gb0, &gb1);
-        const int order[kPathCount] = {kPathA32, kPathR, kPathS, kPathA8, kPathF, kPathA16, kPathR16, kPathS16, kPathG, kPathR8, kPathS8};
         int32_t f_seen = 0;
         for (size_t g = 0; g < gb0.size(); ++g) {
             Handle::GroupStep gs{};
             gs.b0 = gb0[g]; gs.b1 = gb1[g];
             gs.tile0 = int64_t(h->group_tiles.size());
-            for (int p : order)
+            for (int p : kPathOrder)
                 for (int i = gs.b0; i < gs.b1; ++i)
                     if (sb[i].path == p) {
                         const int64_t nt = ceil_div(sb[i].numel, step_tile_elems(p));
@@ -500,7 +520,7 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
                     }
             gs.red0 = -1; gs.f0 = f_seen;
             for (int i = gs.b0; i < gs.b1; ++i)
-                if (sb[i].path == kPathF) {
+                if (is_factored_path(sb[i].path)) {
                     if (gs.red0 < 0) gs.red0 = sb[i].red.red0;
                     gs.n_red += int64_t(sb[i].red.chunks) * sb[i].red.strips;
                     gs.n_f += 1;
@@ -514,8 +534,18 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
        "upload step tile table (by group)");
     if (!red.empty())
         CU(cudaMemcpyAsync(st + L.red_tiles, red.data(), sizeof(RedTile) * red.size(), cudaMemcpyHostToDevice, s), "upload step reduction table");
+    // behind the factored blocks' ids: those with Adafactor's options (their tiles close the tile table)
+    const size_t n_all_f = ids.size();
+    int64_t fa_tiles = 0;
+    for (int i = 0; i < n; ++i)
+        if (sb[i].path == kPathFA) { ids.push_back(i); fa_tiles += ceil_div(sb[i].numel, kTileF); }
+    h->n_fa = int(ids.size() - n_all_f);
+    h->n_fa_tiles = fa_tiles;
+    h->fa_tile0 = int64_t(tiles.size()) - fa_tiles;
+    h->f_id_staging = ids;
     if (!ids.empty())
-        CU(cudaMemcpyAsync(st + L.f_ids, ids.data(), 4 * ids.size(), cudaMemcpyHostToDevice, s), "upload factored ids");
+        CU(cudaMemcpyAsync(st + L.f_ids, h->f_id_staging.data(), 4 * ids.size(), cudaMemcpyHostToDevice, s), "upload factored ids");
+    ids.resize(n_all_f);
     if (reset || zero_only) CU(cudaMemsetAsync(st + L.flags, 0, L.total - L.flags, s), "zero optimizer state");
     {   // factored blocks in index order: that is their order in the tile table, the reduction table and the id list
         h->f_groups.clear();
@@ -523,7 +553,7 @@ static int configure_state(baoc_t* h, const int32_t* assign, void* state_dev, si
         Handle::FactoredGroup g{0, 0, 0, 0, 0, 0};
         int64_t bytes_in_group = 0;
         for (int i = 0; i < n; ++i) {
-            if (sb[i].path != kPathF) continue;
+            if (!is_factored_path(sb[i].path)) continue;
             const int64_t gb = 2 * sb[i].numel, nt = ceil_div(sb[i].numel, kTileF), nr = int64_t(sb[i].red.chunks) * sb[i].red.strips;
             if (g.n_f > 0 && bytes_in_group + gb > h->factored_group_bytes) {
                 h->f_groups.push_back(g);
@@ -583,7 +613,7 @@ MomentRef second_moment(const StepBlock& b) {
         case kPathA8: case kPathR8: r.data = b.s1; r.absmax = b.a1; r.kind = kMomU8; break;
         case kPathR: r.data = b.s0; r.kind = kMomF32; break;
         case kPathR16: r.data = b.s0; r.kind = kMomBF16; break;
-        case kPathF:
+        case kPathF: case kPathFA:
             r.kind = kMomFactored; r.fbits = b.fbits;
             r.wr = static_cast<float*>(b.s0); r.wc = static_cast<float*>(b.s1);
             if (b.fbits == 32) { r.r = b.s0; r.c = b.s1; }
@@ -616,7 +646,7 @@ int baoc_reconfigure(baoc_t* h, const int32_t* new_assign, void* new_state_dev, 
         const int po = old_blocks[i].path;
         keep_m[i] = inherit && m_family(pn) != 0 && m_family(pn) == m_family(po);
         keep_v[i] = inherit && second_moment(old_blocks[i]).kind != kMomNone &&
-                    (pn == kPathA32 || pn == kPathA16 || pn == kPathA8 || pn == kPathR || pn == kPathR16 || pn == kPathR8 || pn == kPathF);
+                    (pn == kPathA32 || pn == kPathA16 || pn == kPathA8 || pn == kPathR || pn == kPathR16 || pn == kPathR8 || is_factored_path(pn));
         h->t_m0[i] = keep_m[i] ? old_tm[i] : steps_done;
         h->t_v0[i] = keep_v[i] ? old_tv[i] : steps_done;
     }
@@ -656,7 +686,8 @@ int baoc_configure_from_window(baoc_t* h, const int32_t* assign, void* state_dev
         const baoc_config_t& c = h->cfgs[assign[i]];
         const Path p = path_of(c);
         keep_m[i] = m_family(p) != 0 && c.beta1 == bm;
-        keep_v[i] = (p == kPathA32 || p == kPathA16 || p == kPathA8 || p == kPathR || p == kPathR16 || p == kPathR8 || p == kPathF) && c.beta2 == bv;
+        keep_v[i] = (p == kPathA32 || p == kPathA16 || p == kPathA8 || p == kPathR || p == kPathR16 || p == kPathR8 || is_factored_path(p)) &&
+                    c.beta2 == bv && !(c.af_flags & kAfSchedule);
         tm[i] = keep_m[i] ? -h->stats_steps : 0;
         tv[i] = keep_v[i] ? -h->stats_steps : 0;
     }
@@ -698,7 +729,7 @@ size_t single_block_state_bytes(const Handle* h, int block, int cfg) {
 }
 bool assignable(const Handle* h, int block, int cfg) {
     const Path p = path_of(h->cfgs[cfg]);
-    return p != kPathNone && !(p == kPathF && h->blocks[block].cols <= 1);
+    return p != kPathNone && !(is_factored_path(p) && h->blocks[block].cols <= 1);
 }
 }  // namespace
 
@@ -741,7 +772,12 @@ int baoc_measure_time_ratios(baoc_t* h, const void* const* grads, float* const* 
         baoc_handle one;
         one.n_blocks = 1; one.n_cfg = K; one.blocks.assign(1, h->blocks[i]); one.cfgs = h->cfgs; one.opts = h->opts;
         one.numel = h->blocks[i].numel;
-        for (baoc_config_t& c : one.cfgs) c.lr = 0.0f;
+        for (baoc_config_t& c : one.cfgs) {
+            c.lr = 0.0f;
+            // Adafactor's relative step size does not come from lr: time it as update clipping, which runs the same
+            // sweep for the two norms, so that the step size stays lr = 0
+            if (c.af_flags & kAfRelative) c.af_flags = uint8_t((c.af_flags & ~kAfRelative) | kAfClip);
+        }
         const void* g1[1] = {grads[i]};
         float* p1[1] = {params[i]};
         for (int c = 0; c < K && rc == BAOC_OK; ++c) {
@@ -796,7 +832,7 @@ uint64_t shape_hash(const Handle* h) {
         for (size_t i = 0; i < n; ++i) { x ^= b[i]; x *= 1099511628211ull; }
     };
     for (const baoc_block_t& b : h->blocks) { mix(&b.numel, 8); mix(&b.rows, 4); mix(&b.cols, 4); }
-    for (const baoc_config_t& c : h->cfgs) mix(&c.adaptive, 5);
+    for (const baoc_config_t& c : h->cfgs) mix(&c.adaptive, 7);      // the tuple, the 8-bit quantiser and Adafactor's options
     return x;
 }
 }  // namespace
@@ -809,7 +845,7 @@ int baoc_export(const baoc_t* h, void* buf, size_t capacity, size_t* size) {
     if (!buf) return BAOC_OK;
     if (capacity < need) return fail(h, BAOC_E_WORKSPACE, "baoc_export: buffer too small");
     BlobHeader hd{};
-    hd.magic = kBlobMagic; hd.version = 2; hd.n_blocks = h->n_blocks; hd.n_cfg = h->n_cfg;
+    hd.magic = kBlobMagic; hd.version = 3; hd.n_blocks = h->n_blocks; hd.n_cfg = h->n_cfg;
     hd.numel = h->numel; hd.stats_steps = h->stats_steps;
     hd.ws_bound = h->ws_bound ? 1 : 0; hd.configured = h->configured ? 1 : 0;
     hd.shape_hash = shape_hash(h);
@@ -830,7 +866,7 @@ int baoc_import(baoc_t* h, const void* blob, size_t size, void* ws_dev, size_t w
     if (!blob || size < sizeof(BlobHeader)) return fail(h, BAOC_E_INVALID, "baoc_import: blob missing or truncated");
     BlobHeader hd;
     std::memcpy(&hd, blob, sizeof(hd));
-    if (hd.magic != kBlobMagic || hd.version != 2) return fail(h, BAOC_E_INVALID, "baoc_import: not a blob of this library version");
+    if (hd.magic != kBlobMagic || hd.version != 3) return fail(h, BAOC_E_INVALID, "baoc_import: not a blob of this library version");
     if (hd.n_blocks != h->n_blocks || hd.n_cfg != h->n_cfg || hd.numel != h->numel || hd.shape_hash != shape_hash(h))
         return fail(h, BAOC_E_INVALID, "baoc_import: the blob belongs to a different block set or candidate set");
     if (hd.stats_steps < 0) return fail(h, BAOC_E_INVALID, "baoc_import: corrupt blob");
@@ -946,8 +982,14 @@ int baoc_step_from_host(baoc_t* h, const void* const* host_grads, void* const* d
         if (e == cudaSuccess) e = cudaStreamWaitEvent(s, static_cast<cudaEvent_t>(h->copy_ev[g]), 0);
         if (e != cudaSuccess) { join(); return cuda_fail(h, "baoc_step_from_host (copy)", e); }
         rc = stats_step_range(h, gb0[g], gb1[g], s);
-        if (rc == BAOC_OK && step_t > 0) rc = step_group(h, h->groups[g], P, s);
+        // blocks with Adafactor's options need their norms between the reduction and the update: with such blocks the
+        // step follows the transfer as a whole instead of group by group
+        if (rc == BAOC_OK && step_t > 0 && h->n_fa == 0) rc = step_group(h, h->groups[g], P, s);
         if (rc) { join(); return rc; }
+    }
+    if (step_t > 0 && h->n_fa > 0) {
+        rc = step_launches(h, P, s);
+        if (rc) return rc;
     }
     return stats_combine_all(h, s);
 }
@@ -1034,7 +1076,7 @@ int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* co
         void* p = nullptr; int64_t n = 0; int32_t eb = 4;
         switch (s.path) {
             case kPathA32: if (k == 0) { p = s.s0; n = b.numel; } else if (k == 1) { p = s.s1; n = b.numel; } break;
-            case kPathA8:
+            case kPathA8: case kPathA8N:
                 if (k == 0) { p = s.s0; n = b.numel; eb = 1; } else if (k == 1) { p = s.s1; n = b.numel; eb = 1; }
                 else if (k == 2) { p = s.a0; n = nq; } else { p = s.a1; n = nq; }
                 break;
@@ -1043,7 +1085,7 @@ int baoc_view(const baoc_t* h, int block, int which, void** dev_ptr, int64_t* co
             case kPathR16: case kPathS16: if (k == 0) { p = s.s0; n = b.numel; eb = 2; } break;
             case kPathR8: if (k == 0) { p = s.s1; n = b.numel; eb = 1; } else if (k == 1) { p = s.a1; n = nq; } break;
             case kPathS8: if (k == 0) { p = s.s0; n = b.numel; eb = 1; } else if (k == 1) { p = s.a0; n = nq; } break;
-            case kPathF:
+            case kPathF: case kPathFA:
                 if (s.fbits == 32) { if (k == 0) { p = s.s0; n = b.rows; } else if (k == 1) { p = s.s1; n = b.cols; } }
                 else {
                     const int32_t e = s.fbits == 16 ? 2 : 1;

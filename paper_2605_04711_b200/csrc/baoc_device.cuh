@@ -244,4 +244,60 @@ __device__ __forceinline__ int encode_unsigned(double x, float absmax, double sc
     return max(0, min(255, encode_round(x, absmax, scale, 255.0)));
 }
 
+// ---- the non-linear ("dynamic") 8-bit codebook ---------------------------------------
+// Magnitudes 10^-E (0.1 + 0.9 (k+1) / 2^F), k < 2^F, F = B - 1 - E, E < B, with B = 7 value bits (signed) or 8
+// (unsigned), and zero; a code is the index of the nearest entry in ascending order.  In ascending order the positive
+// magnitude number p >= 1 has F = floor(log2 p), E = B - 1 - F, k = p - 2^F, so a CTA builds the tables in place.
+struct DynTables {
+    double ts[256], ms[256];     // signed entries (255 used) and the midpoints between neighbours (254 used), padded upwards
+    double tu[256], mu[256];     // unsigned entries and their 255 midpoints
+};
+static __constant__ double kPow10[8] = {1.0, 1e-1, 1e-2, 1e-3, 1e-4, 1e-5, 1e-6, 1e-7};
+__device__ __forceinline__ double dyn_magnitude(int p, int value_bits) {
+    const double* p10 = kPow10;
+    const int F = 31 - __clz(p), E = value_bits - 1 - F, k = p - (1 << F);
+    const double frac = __dadd_rn(0.1, __dmul_rn(__dmul_rn(0.9, double(k + 1)), 1.0 / double(1 << F)));
+    return __dmul_rn(p10[E], frac);
+}
+__device__ __forceinline__ void dyn_build(DynTables* T) {      // all kThreads = 256 threads of the CTA
+    const int i = threadIdx.x;
+    T->tu[i] = i == 0 ? 0.0 : dyn_magnitude(i, 8);
+    T->ts[i] = i == 127 ? 0.0 : (i < 127 ? -dyn_magnitude(127 - i, 7) : (i < 255 ? dyn_magnitude(i - 127, 7) : 2.0));
+    __syncthreads();
+    T->mu[i] = i < 255 ? 0.5 * (T->tu[i] + T->tu[i + 1]) : 4.0;     // the padding is above every y in [-1, 1]
+    T->ms[i] = i < 254 ? 0.5 * (T->ts[i] + T->ts[i + 1]) : 4.0;
+    __syncthreads();
+}
+// Index of the entry nearest to y: the number of midpoints below y (a tie goes to the entry of smaller magnitude).
+__device__ __forceinline__ int dyn_nearest(const double* mid, double y) {
+    int lo = 0;
+    const bool neg = y < 0.0;
+#pragma unroll
+    for (int step = 128; step > 0; step >>= 1) {
+        const double m = mid[lo + step - 1];
+        if (neg ? y >= m : y > m) lo += step;
+    }
+    return lo;
+}
+// The same tables in fp32 (for sums that are compared at 1e-4): ts, ms, tu, mu, 256 floats each.
+__device__ __forceinline__ void dyn_build_f32(float* t4) {           // all kThreads = 256 threads of the CTA
+    const int i = threadIdx.x;
+    const double u0 = i == 0 ? 0.0 : dyn_magnitude(i, 8), u1 = i < 255 ? dyn_magnitude(i + 1, 8) : 8.0;
+    auto sgn = [](int k) { return k == 127 ? 0.0 : (k < 127 ? -dyn_magnitude(127 - k, 7) : (k < 255 ? dyn_magnitude(k - 127, 7) : 8.0)); };
+    const double s0 = sgn(i), s1 = sgn(i + 1 < 256 ? i + 1 : 255);
+    t4[i] = float(s0); t4[256 + i] = i < 254 ? float(0.5 * (s0 + s1)) : 4.0f;
+    t4[512 + i] = float(u0); t4[768 + i] = i < 255 ? float(0.5 * (u0 + u1)) : 4.0f;
+    __syncthreads();
+}
+__device__ __forceinline__ int dyn_nearest_f32(const float* mid, float y) {
+    int lo = 0;
+    const bool neg = y < 0.f;
+#pragma unroll
+    for (int step = 128; step > 0; step >>= 1) {
+        const float m = mid[lo + step - 1];
+        if (neg ? y >= m : y > m) lo += step;
+    }
+    return lo;
+}
+
 }  // namespace baoc

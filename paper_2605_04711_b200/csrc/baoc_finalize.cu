@@ -66,7 +66,7 @@ final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, double* __re
 // ============================================================================
 constexpr int kFsStageBytes = kThreads * 96;                 // m 32 B/thread at 0, v at 8192, theta at 16384
 constexpr int kFsStages = 3;
-constexpr int kFsSmemBytes = kFsStages * kFsStageBytes + kSelBins * 4;      // the staging ring and the histogram of the first digit
+constexpr int kFsSmemBytes = kFsStages * kFsStageBytes + kSelBins * 4 + 4096;   // the staging ring, the histogram of the first digit, the codebook
 
 __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
     f32x2 d;
@@ -86,9 +86,12 @@ __device__ __forceinline__ float rsqrt_approx(float x) {
 // The bf16 direction costs no extra square root or reciprocal: with n = (v - v16) / v (|n| <= 2^-8),
 // sqrt(v16) - sqrt(v) = -sqrt(v) n (1/2 + n/8 + n^2/16) up to n^4, and with e that difference over (sqrt(v) + eps_adam),
 // 1 / (sqrt(v16) + eps_adam) = (1 - e + e^2 - e^3) / (sqrt(v) + eps_adam) up to e^4: both truncations are below 1e-10.
-template <bool kFull>
+// kDyn: the 8-bit round trip goes through the non-linear codebook (dyn: its fp32 tables in shared memory) instead of the
+// linear absmax codes.
+template <bool kFull, bool kDyn>
 __device__ __forceinline__ void fs_slice(const float (&mm)[8], const float (&vv)[8], const float (&tt)[8], int cnt,
-                                         float p0, float eps_f, float eps_adam, f32x2 (&F)[kFinalSums], uint32_t* hist1) {
+                                         float p0, float eps_f, float eps_adam, f32x2 (&F)[kFinalSums], uint32_t* hist1,
+                                         const float* dyn) {
     const f32x2 P0 = splat2(p0), MAGIC = splat2(12582912.0f), C16 = splat2(65537.0f), EA = splat2(eps_adam), EPS = splat2(eps_f),
                 ONE = splat2(1.0f), MONE = splat2(-1.0f);
     // ---- absmax of the warp's quantisation block, code scales
@@ -113,8 +116,15 @@ __device__ __forceinline__ void fs_slice(const float (&mm)[8], const float (&vv)
         const f32x2 M = pack2(mm[2 * p], mm[2 * p + 1]), V = pack2(vv[2 * p], vv[2 * p + 1]);
         const f32x2 T = pack2(tt[2 * p], tt[2 * p + 1]);
         // 8-bit round trips: code = rne(x L / a) by the magic-number addition, value = code a / L
-        const f32x2 QM = sub2(fma2(M, KM, MAGIC), MAGIC), QV = sub2(fma2(V, KV, MAGIC), MAGIC);
-        const f32x2 M8 = fma2(QM, DM, mul2(QM, DML)), V8 = fma2(QV, DV, mul2(QV, DVL));
+        f32x2 M8, V8;
+        if (kDyn) {
+            const float ia = am > 0.f ? rm0 : 0.f, iv = av > 0.f ? rv0 : 0.f;
+            M8 = pack2(dyn[dyn_nearest_f32(dyn + 256, mm[2 * p] * ia)] * am, dyn[dyn_nearest_f32(dyn + 256, mm[2 * p + 1] * ia)] * am);
+            V8 = pack2(dyn[512 + dyn_nearest_f32(dyn + 768, vv[2 * p] * iv)] * av, dyn[512 + dyn_nearest_f32(dyn + 768, vv[2 * p + 1] * iv)] * av);
+        } else {
+            const f32x2 QM = sub2(fma2(M, KM, MAGIC), MAGIC), QV = sub2(fma2(V, KV, MAGIC), MAGIC);
+            M8 = fma2(QM, DM, mul2(QM, DML)); V8 = fma2(QV, DV, mul2(QV, DVL));
+        }
         // bf16 round trips
         const f32x2 CM = mul2(M, C16), CV = mul2(V, C16);
         // (written as x*(-1) + y: a plain packed subtraction here came out as the identity, the two differences folded)
@@ -157,6 +167,7 @@ __device__ __forceinline__ void fs_slice(const float (&mm)[8], const float (&vv)
         if (kFull || j < cnt) atomicAdd(hist1 + (__float_as_uint(vv[j]) >> (32 - kSelBits)), 1u);
 }
 
+template <bool kDyn>
 __global__ void __launch_bounds__(kThreads, 2)
 final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
                   const float* const* __restrict__ params, double* __restrict__ fin,
@@ -185,6 +196,8 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
     extern __shared__ __align__(16) unsigned char dyn[];
     unsigned char* stage = dyn;
     uint32_t* hist1 = reinterpret_cast<uint32_t*>(dyn + kFsStages * kFsStageBytes);      // kSelBins counters
+    float* dyn_tables = reinterpret_cast<float*>(dyn + kFsStages * kFsStageBytes + kSelBins * 4);
+    if (kDyn) dyn_build_f32(dyn_tables);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
     const int nsl = int(last - first) * (kTile / (kThreads * 8));     // slices of this CTA
@@ -271,7 +284,7 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
         f4_to8(*reinterpret_cast<const float4*>(mine + ov), *reinterpret_cast<const float4*>(mine + ov + kHalf), vv);
         if (w0 + kQBlock <= numel) {                         // uniform over the warp
             f4_to8(*reinterpret_cast<const float4*>(mine + ot), *reinterpret_cast<const float4*>(mine + ot + kHalf), tt);
-            fs_slice<true>(mm, vv, tt, 8, p0, eps_f, eps_adam, F, hist1);
+            fs_slice<true, kDyn>(mm, vv, tt, 8, p0, eps_f, eps_adam, F, hist1, dyn_tables);
         } else {
             const int64_t e = w0 + lane * 8;
             const int cnt = int(max64(0, min64(8, numel - e)));
@@ -282,7 +295,7 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
 #pragma unroll
                 for (int j = 0; j < 8; ++j) tt[j] = j < cnt ? th[e + j] : 0.f;
             }
-            fs_slice<false>(mm, vv, tt, cnt, p0, eps_f, eps_adam, F, hist1);
+            fs_slice<false, kDyn>(mm, vv, tt, cnt, p0, eps_f, eps_adam, F, hist1, dyn_tables);
         }
     }
     cp_async_wait<0>();
@@ -634,7 +647,7 @@ static int run_tiles(int64_t n_tiles, int most) {
 
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
                       double* fin_out, uint32_t* hist, RankSel* sel, int64_t n_tiles, int n_blocks, double eps,
-                      float eps_adam, const CheckCtx& ck, cudaStream_t s) {
+                      float eps_adam, int quantizer8, const CheckCtx& ck, cudaStream_t s) {
     (void)ck;
     const int tb = 128, gb = (n_blocks + tb - 1) / tb;
     cudaError_t e = cudaMemsetAsync(hist, 0, size_t(n_blocks) * kRanks * kSelBins * sizeof(uint32_t), s);
@@ -643,11 +656,17 @@ int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* c
     BAOC_LAUNCH_CHECK();
     final_pilot_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, float(eps), fin_out);
     BAOC_LAUNCH_CHECK();
-    e = cudaFuncSetAttribute(final_sums_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes);
+    e = cudaFuncSetAttribute(final_sums_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(final_sums_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes);
     if (e != cudaSuccess) return int(e);
     const int per = run_tiles(n_tiles, kFinRunTiles);
-    final_sums_kernel<<<unsigned((n_tiles + per - 1) / per), kThreads, kFsSmemBytes, s>>>(
-        blocks, tiles, params, fin, fin_out, hist, n_tiles, per, float(eps), eps_adam BAOC_CHECK_ARG(ck));
+    const unsigned grid = unsigned((n_tiles + per - 1) / per);
+    if (quantizer8)
+        final_sums_kernel<true><<<grid, kThreads, kFsSmemBytes, s>>>(blocks, tiles, params, fin, fin_out, hist, n_tiles, per,
+                                                                       float(eps), eps_adam BAOC_CHECK_ARG(ck));
+    else
+        final_sums_kernel<false><<<grid, kThreads, kFsSmemBytes, s>>>(blocks, tiles, params, fin, fin_out, hist, n_tiles, per,
+                                                                        float(eps), eps_adam BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     final_sums_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
     BAOC_LAUNCH_CHECK();

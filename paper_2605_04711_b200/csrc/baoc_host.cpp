@@ -46,6 +46,7 @@ int64_t state_mem_bytes(const baoc_config_t& c, const baoc_block_t& b) {
 double step_traffic_bytes(const baoc_config_t& c, const baoc_block_t& b) {
     double bytes = 2.0 * b.numel + 8.0 * b.numel + 2.0 * double(state_mem_bytes(c, b));
     if (c.factored) bytes += 2.0 * b.numel;
+    if (c.factored && (c.af_flags & (kAfClip | kAfRelative))) bytes += 6.0 * b.numel;   // one more sweep over g and theta for the two norms
     return bytes;
 }
 
@@ -181,7 +182,7 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
     double traffic = 0;
     int64_t coarse = 0;
     for (int i = 0; i < n; ++i)
-        if (assign[i] >= 0 && assign[i] < h->n_cfg && path_of(h->cfgs[assign[i]]) == kPathF) {
+        if (assign[i] >= 0 && assign[i] < h->n_cfg && is_factored_path(path_of(h->cfgs[assign[i]]))) {
             const RedGeom g = red_geometry(h->blocks[i].rows, h->blocks[i].cols, 1);
             coarse += int64_t(g.chunks) * g.strips;
         }
@@ -192,7 +193,7 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
         const baoc_block_t& b = h->blocks[i];
         const Path p = path_of(h->cfgs[c]);
         if (p == kPathNone) return fail(h, BAOC_E_INVALID, "assignment names a configuration tuple the library cannot instantiate");
-        if (p == kPathF && b.cols <= 1) return fail(h, BAOC_E_INVALID, "the factored configuration needs a matrix block");
+        if (is_factored_path(p) && b.cols <= 1) return fail(h, BAOC_E_INVALID, "the factored configuration needs a matrix block");
         StepBlock& s = sb[i];
         s = StepBlock{};
         s.numel = b.numel; s.rows = b.rows; s.cols = b.cols; s.cfg = c; s.path = p;
@@ -202,7 +203,7 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
         auto place = [&](size_t bytes) { return reinterpret_cast<void*>(take(&states, bytes)); };
         switch (p) {
             case kPathA32: s.s0 = place(4 * dpad); s.s1 = place(4 * dpad); break;
-            case kPathA8:
+            case kPathA8: case kPathA8N:
                 s.s0 = place(dpad); s.s1 = place(dpad);
                 s.a0 = static_cast<float*>(place(4 * nq)); s.a1 = static_cast<float*>(place(4 * nq));
                 break;
@@ -212,8 +213,13 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
             case kPathR8: s.s1 = place(dpad); s.a1 = static_cast<float*>(place(4 * nq)); break;
             case kPathS8: s.s0 = place(dpad); s.a0 = static_cast<float*>(place(4 * nq)); break;
             case kPathG: break;
-            case kPathF: {
+            case kPathF: case kPathFA: {
                 s.fbits = h->cfgs[c].bits;
+                s.af_flags = h->cfgs[c].af_flags;
+                if (p == kPathFA) {
+                    s.norm_part = reinterpret_cast<double*>(redpart);
+                    redpart += 8 * 2 * size_t(ceil_div(b.numel, kTileF));
+                }
                 if (s.fbits == 32) { s.s0 = place(4 * size_t(b.rows)); s.s1 = place(4 * size_t(b.cols)); }
                 else {
                     // the fp32 working copies live in the scratch region (offsets from its base), the stored form in the states
@@ -243,10 +249,7 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
         mem += state_mem_bytes(h->cfgs[c], b);
         traffic += step_traffic_bytes(h->cfgs[c], b);
     }
-    // the tiles of one path family after another (each family has its own kernel instance); within a family in
-    // descending bytes per element, so that the light tiles fill the tail of the grid
-    const int order[kPathCount] = {kPathA32, kPathR, kPathS, kPathA8, kPathF, kPathA16, kPathR16, kPathS16, kPathG, kPathR8, kPathS8};
-    for (int p : order)
+    for (int p : kPathOrder)
         for (int i = 0; i < n; ++i)
             if (sb[i].path == p) {
                 const int64_t nt = ceil_div(sb[i].numel, step_tile_elems(p));
@@ -257,7 +260,7 @@ int compute_step_layout(const Handle* h, const int32_t* assign, Handle::StepLayo
     out->tiles = take(&cur, sizeof(Tile) * tl.size());
     out->tiles_by_group = take(&cur, sizeof(Tile) * tl.size());
     out->red_tiles = take(&cur, sizeof(RedTile) * std::max<size_t>(rt.size(), 1));
-    out->f_ids = take(&cur, 4 * size_t(n));
+    out->f_ids = take(&cur, 8 * size_t(n));               // the factored blocks, then those with Adafactor's options
     out->grads = take(&cur, 8 * size_t(n));
     out->params = take(&cur, 8 * size_t(n));
     out->flags = take(&cur, 4 * size_t(n));
@@ -546,7 +549,7 @@ int baoc_create(baoc_t** out, int n_blocks, const baoc_block_t* blocks, int n_cf
     if (!blocks || !cfgs || n_blocks <= 0 || n_cfg <= 0 || n_cfg > kMaxCfg) return BAOC_E_INVALID;
     baoc_opts_t o;
     if (opts) o = *opts; else baoc_default_opts(&o);
-    if (o.qblock != kQBlock) return BAOC_E_INVALID;
+    if (o.qblock != kQBlock || o.quantizer8 < 0 || o.quantizer8 > 1 || o.reserved != 0) return BAOC_E_INVALID;
     if (!(o.beta_m >= 0 && o.beta_m < 1 && o.beta_v >= 0 && o.beta_v < 1 && o.beta_rho >= 0 && o.beta_rho < 1)) return BAOC_E_INVALID;
     if (!(o.a_hi > o.a_lo && o.rho_hi > o.rho_lo && o.snr_hi > o.snr_lo && o.eps >= 0)) return BAOC_E_INVALID;
     int64_t total = 0;
@@ -559,6 +562,7 @@ int baoc_create(baoc_t** out, int n_blocks, const baoc_block_t* blocks, int n_cf
     for (int c = 0; c < n_cfg; ++c) {
         const baoc_config_t& k = cfgs[c];
         if (k.adaptive > 1 || k.momentum > 1 || k.decoupled_wd > 1 || k.factored > 1) return BAOC_E_INVALID;
+        if (k.quantizer > 1 || k.af_flags > 15 || k.reserved != 0) return BAOC_E_INVALID;
         if (k.bits != 8 && k.bits != 16 && k.bits != 32) return BAOC_E_INVALID;
         if (!(k.beta1 >= 0 && k.beta1 < 1 && k.beta2 >= 0 && k.beta2 < 1 && k.eps >= 0)) return BAOC_E_INVALID;
         if (!std::isfinite(k.lr) || !std::isfinite(k.weight_decay)) return BAOC_E_INVALID;
@@ -672,7 +676,7 @@ int baoc_allocate(baoc_t* h, const double* risk, const int64_t* mem_bytes, const
             if (forbid && forbid[k]) continue;
             const Path p = path_of(h->cfgs[c]);
             if (p == kPathNone) continue;
-            if (p == kPathF && h->blocks[i].cols <= 1) continue;
+            if (is_factored_path(p) && h->blocks[i].cols <= 1) continue;
             if (!std::isfinite(risk[k]) || !std::isfinite(time_ratio[k]) || time_ratio[k] < 0 || mem_bytes[k] < 0)
                 return fail(h, BAOC_E_INVALID, "baoc_allocate: non-finite or negative input");
             const double phi = (risk[k] - (pref ? pref[k] : 0.0)) + h->opts.gamma * agg(h->cfgs[c]);

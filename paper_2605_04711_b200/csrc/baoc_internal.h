@@ -55,13 +55,22 @@ enum Path : int32_t {
     kPathS16 = 8,        // SGD with a bf16 momentum buffer
     kPathR8 = 9,         // momentum-free RMS scaling with a block-wise absmax 8-bit second moment
     kPathS8 = 10,        // SGD with a block-wise absmax 8-bit momentum buffer
-    kPathCount = 11,
+    kPathA8N = 11,       // Adam / AdamW with 8-bit moments in the non-linear (dynamic) codebook
+    kPathFA = 12,        // factored second moment with Adafactor's options (beta2 schedule, update clipping, relative step)
+    kPathCount = 13,
     kPathNone = -1
 };
 
+// Bits of baoc_config_t::af_flags.
+enum AfFlags : int32_t { kAfSchedule = 1, kAfClip = 2, kAfRelative = 4, kAfEps1 = 8 };
+
+inline bool is_factored_path(int path) { return path == kPathF || path == kPathFA; }
+
 inline Path path_of(const baoc_config_t& c) {
-    if (c.factored) return (c.adaptive && !c.momentum) ? kPathF : kPathNone;   // row/column statistics in fp32, bf16 or 8-bit codes
-    if (c.adaptive && c.momentum) return c.bits == 32 ? kPathA32 : (c.bits == 16 ? kPathA16 : kPathA8);
+    if (c.af_flags != 0 && !c.factored) return kPathNone;               // Adafactor's options belong to the factored tuple
+    if (c.quantizer != 0 && !(c.bits == 8 && c.adaptive && c.momentum && !c.factored)) return kPathNone;   // the codebook is offered for 8-bit Adam
+    if (c.factored) return (c.adaptive && !c.momentum) ? (c.af_flags ? kPathFA : kPathF) : kPathNone;   // row/column statistics in fp32, bf16 or 8-bit codes
+    if (c.adaptive && c.momentum) return c.bits == 32 ? kPathA32 : (c.bits == 16 ? kPathA16 : (c.quantizer ? kPathA8N : kPathA8));
     if (c.adaptive && !c.momentum) return c.bits == 32 ? kPathR : (c.bits == 16 ? kPathR16 : kPathR8);
     if (!c.adaptive && c.momentum) return c.bits == 32 ? kPathS : (c.bits == 16 ? kPathS16 : kPathS8);
     return kPathG;       // neither mechanism: stateless, whatever bit-width the tuple names
@@ -72,15 +81,21 @@ enum Family : int32_t { kFamHead = 0, kFamDense = 1, kFamQ8 = 2, kFamCount = 3 }
 inline int family_of(int path) {
     switch (path) {
         case kPathG: case kPathA16: case kPathR16: case kPathS16: return kFamDense;
-        case kPathR8: case kPathS8: return kFamQ8;
+        case kPathR8: case kPathS8: case kPathA8N: case kPathFA: return kFamQ8;
         default: return kFamHead;
     }
 }
 
 // Elements per tile of the fused step, by update path.
 BAOC_HD inline int64_t step_tile_elems(int path) {
-    return path == kPathF ? kTileF : ((path == kPathA8 || path == kPathR8 || path == kPathS8) ? kTileQ : kTile);
+    return (path == kPathF || path == kPathFA) ? kTileF
+                                               : ((path == kPathA8 || path == kPathR8 || path == kPathS8 || path == kPathA8N) ? kTileQ : kTile);
 }
+
+// Order of the paths in the step's tile table: the families one after another (each has its own kernel instance),
+// within a family in descending bytes per element, so that the light tiles fill the tail of the grid.
+constexpr int kPathOrder[kPathCount] = {kPathA32, kPathR, kPathS, kPathA8, kPathF, kPathA16, kPathR16, kPathS16, kPathG,
+                                        kPathR8, kPathS8, kPathA8N, kPathFA};
 
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
@@ -158,7 +173,8 @@ struct StepBlock {
     float* fa0;          // 8-bit: absmax of the row statistics per quantisation block
     float* fa1;          // 8-bit: absmax of the column statistics
     int32_t fbits;       // 32, 16 or 8 (factored blocks; 0 otherwise)
-    int32_t pad2;
+    int32_t af_flags;    // Adafactor's options of the block's tuple (kPathFA)
+    double* norm_part;   // kPathFA: per tile of the block {sum u^2, sum theta^2}; a0[1] = clip factor, a0[2] = step size
 };
 
 // A stored moment, for the migration kernels of a re-configuration.
@@ -208,9 +224,11 @@ struct CfgStep {
     float step_m_hat;    // step_m * sqrt(1 - beta2^t): with eps_hat the update is step_m_hat * m / (sqrt(v) + eps_hat)
     float eps_hat;       // eps * sqrt(1 - beta2^t)
     int32_t coupled;     // 1: add wd*theta to the gradient
-    int32_t pad;
-    double beta1_d, beta2_d;   // the coefficients widened, for the exact side of the 8-bit path
+    int32_t af_flags;    // Adafactor's options (factored tuple)
+    double beta1_d, beta2_d;   // the coefficients widened, for the exact side of the 8-bit path (beta2_d: this step's value under the schedule)
     double wd_d;
+    double eps1_d;       // added to every squared gradient of the factored reduction (0 unless the tuple asks for it)
+    double rho_d;        // relative step: min(1e-2, 1 / sqrt(t))
 };
 struct StepParams {
     CfgStep c[kMaxSlots];
@@ -256,7 +274,9 @@ struct Handle {
     std::vector<StepBlock> h_step_blocks;
     int64_t n_step_tiles = 0;
     int64_t n_step_red_tiles = 0;
-    int n_factored = 0;              // blocks on the factored path
+    int n_factored = 0;              // blocks on a factored path (with or without Adafactor's options)
+    int n_fa = 0;                    // of those, blocks with Adafactor's options; their tiles close the tile table
+    int64_t fa_tile0 = 0, n_fa_tiles = 0;
     int64_t fam_tiles[kFamCount] = {0, 0, 0};   // tiles of each path family; the tile table holds the families one after another
     // Bias corrections count the gradients a moment has seen.  A re-configuration may restart some moments, so every
     // block carries the step counts at which its first and second moment last started from zero; blocks that share a
@@ -267,6 +287,7 @@ struct Handle {
     std::vector<int32_t> slot_of;
     int64_t state_mem = 0;           // StateMem of the assignment (sum of M_{i,c_i})
     int64_t step_bytes = 0;          // algorithmic bytes of one step
+    std::vector<int32_t> f_id_staging;   // staging of the id lists (must outlive the asynchronous upload)
     std::vector<const void*> last_step_grads;
     std::vector<const void*> last_step_params;
     struct StepLayout {
@@ -326,7 +347,7 @@ int launch_stats_combine(const StatBlock* blocks, const double* partials, double
 // row/column sums of the matrix blocks, the second and third sweep and the gather of the per-block results.
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
                       double* fin_out, uint32_t* hist, RankSel* sel, int64_t n_tiles, int n_blocks, double eps,
-                      float eps_adam, const CheckCtx& ck, cudaStream_t s);
+                      float eps_adam, int quantizer8, const CheckCtx& ck, cudaStream_t s);
 int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
                               uint32_t* hist, const double* acc, int64_t n_tiles, int n_blocks, const CheckCtx& ck,
                               cudaStream_t s);
@@ -345,6 +366,11 @@ int stats_check_fetch(CheckRecord* out);
 int finalize_check_fetch(CheckRecord* out);
 int step_check_fetch(CheckRecord* out);
 int launch_check_selftest(cudaStream_t s);
+// Adafactor's options: per tile of the given blocks the sums of u^2 and theta^2, then per block the clip factor and the
+// step size (ids: the blocks, n of them; tiles: their stretch of the tile table).
+int launch_factored_norms(const StepBlock* blocks, const Tile* tiles, const int32_t* ids, const void* const* grads,
+                          const float* const* params, int64_t n_tiles, int n, const StepParams& P, const CheckCtx& ck,
+                          cudaStream_t s);
 int launch_convert_moment(const MomentRef& src, const MomentRef& dst, int64_t numel, cudaStream_t s);
 // Copy groups of the end-to-end call: up to Handle::kCopyGroups runs of whole blocks of about equal bytes.
 void compute_copy_groups(const Handle* h, std::vector<int>* b0, std::vector<int>* b1);

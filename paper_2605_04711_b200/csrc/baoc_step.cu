@@ -243,7 +243,7 @@ moment_total_kernel(const StatBlock* __restrict__ blocks, const int32_t* __restr
 // a time.  The stored value is read, the new one is written un-rounded (fp32) to the working copy the update kernel
 // reads, and its rounding / its code is what is stored.  Returns the thread's share of the sum of the new values.
 template <bool kRow>
-__device__ __forceinline__ double combine_reduced(const StepBlock* b, double beta2, int slab) {
+__device__ __forceinline__ double combine_reduced(const StepBlock* b, double beta2, double eps1, int slab) {
     const int n = kRow ? b->rows : b->cols, other = kRow ? b->cols : b->rows;
     const int parts = kRow ? b->red.strips : b->red.chunks;
     const double* __restrict__ part = kRow ? b->red.rowpart : b->red.colpart;
@@ -268,7 +268,7 @@ __device__ __forceinline__ double combine_reduced(const StepBlock* b, double bet
                 for (int p = 0; p < parts; ++p) s += part[size_t(p) * n + i];
                 const double old = codes ? (double(static_cast<const uint8_t*>(stored)[i]) * a_old) / 255.0
                                          : double(bf16_bits_to_float(static_cast<const uint16_t*>(stored)[i]));
-                x[j] = beta2 * old + (1.0 - beta2) * (s / double(other));
+                x[j] = beta2 * old + (1.0 - beta2) * (s / double(other) + eps1);
                 const float xf = __double2float_rn(x[j]);
                 work[i] = xf;
                 sum += double(xf);
@@ -322,12 +322,12 @@ factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __r
     __shared__ double total[1];
     const StepBlock* b = blocks + ids[blockIdx.x];
     const int rows = b->rows, cols = b->cols, slab = blockIdx.y;
-    const double beta2 = P.c[b->cfg].beta2_d;
+    const double beta2 = P.c[b->cfg].beta2_d, eps1 = P.c[b->cfg].eps1_d;   // (the mean of g^2 + eps1 is the mean of g^2, plus eps1)
     double local[1] = {0.0};
     if (b->fbits != 32) {
-        local[0] = combine_reduced<true>(b, beta2, slab);
+        local[0] = combine_reduced<true>(b, beta2, eps1, slab);
         cta_reduce_store<1>(local, total);
-        combine_reduced<false>(b, beta2, slab);
+        combine_reduced<false>(b, beta2, eps1, slab);
     } else {
         float* __restrict__ r = static_cast<float*>(b->s0);
         float* __restrict__ c = static_cast<float*>(b->s1);
@@ -335,7 +335,7 @@ factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __r
         for (int i = slab * rpc + threadIdx.x; i < min(rows, (slab + 1) * rpc); i += kThreads) {
             double s = 0.0;
             for (int st = 0; st < b->red.strips; ++st) s += b->red.rowpart[size_t(st) * rows + i];
-            const float rn = float(beta2 * double(r[i]) + (1.0 - beta2) * (s / double(cols)));
+            const float rn = float(beta2 * double(r[i]) + (1.0 - beta2) * (s / double(cols) + eps1));
             r[i] = rn;
             local[0] += double(rn);
         }
@@ -344,7 +344,7 @@ factored_combine_kernel(const StepBlock* __restrict__ blocks, const int32_t* __r
             double s = 0.0;
 #pragma unroll 4
             for (int ch = 0; ch < b->red.chunks; ++ch) s += b->red.colpart[size_t(ch) * cols + j];
-            c[j] = float(beta2 * double(c[j]) + (1.0 - beta2) * (s / double(rows)));
+            c[j] = float(beta2 * double(c[j]) + (1.0 - beta2) * (s / double(rows) + eps1));
         }
     }
     if (threadIdx.x == 0) {
@@ -549,6 +549,9 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
 // multiple of 8 a thread's 8 elements lie in one row, so it needs one row
 // statistic and two 128-bit loads of column statistics (which stay in L1/L2:
 // every row of the tile re-reads them).
+// kOpt: the block's tuple carries Adafactor's options: the step size and the clip factor are per-block values that the
+// norms kernels have left behind the mean of r, and a decoupled decay uses that step size.
+template <bool kOpt>
 __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgStep& P, const uint16_t* __restrict__ g,
                                                   float* __restrict__ th, int64_t base, unsigned char* stage) {
     const int64_t numel = b->numel;
@@ -558,6 +561,16 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
     const float rm = b->a0[0];
     const float inv_rm = rm > 0.f ? 1.0f / rm : 0.f;
     float chk = 0.f;
+    float step = P.step_g, decay = P.decay;
+    if (kOpt) {
+        const float alpha = (P.af_flags & kAfRelative) ? b->a0[2] : P.step_g;
+        step = (P.af_flags & kAfClip) ? alpha * b->a0[1] : alpha;
+        decay = P.decay != 0.f ? -alpha * P.wd : 0.f;            // decoupled: theta <- theta (1 - alpha wd)
+    }
+    auto pro = [&](float& x, float& t) {
+        if (P.coupled) x = fmaf(P.wd, t, x);
+        else t = fmaf(decay, t, t);
+    };
     if ((cols & 7) == 0) {
         // Streaming form: each thread copies the 48 bytes of its own next eight elements (gradient, parameters)
         // into its own shared-memory slot three slices ahead with cp.async and reads them back itself: no
@@ -606,8 +619,8 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
             f4_to(*reinterpret_cast<const float4*>(mine + st_), *reinterpret_cast<const float4*>(mine + st_ + 16), t);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                prologue(x[j], t[j], P);
-                t[j] = adaptive_apply(t[j], x[j], rs * cj[j], P.step_g, P);
+                pro(x[j], t[j]);
+                t[j] = adaptive_apply(t[j], x[j], rs * cj[j], step, P);
                 chk = poison(chk, t[j]);
             }
             st8(tht + e, t);
@@ -627,8 +640,8 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
         for (int j = 0; j < cnt; ++j) {
             float x = bf16_bits_to_float(g[e + j]);
             float t = th[e + j];
-            prologue(x, t, P);
-            t = adaptive_apply(t, x, rs * __ldg(c + col), P.step_g, P);
+            pro(x, t);
+            t = adaptive_apply(t, x, rs * __ldg(c + col), step, P);
             chk = poison(chk, t);
             th[e + j] = t;
             if (++col == cols) { col = 0; ++row; if (j + 1 < cnt) rs = __ldg(r + row) * inv_rm; }
@@ -962,12 +975,165 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
     return !isfinite(c0) | !isfinite(c1);
 }
 
+// ----------------------------------------------------------------------------
+// Adam with 8-bit moments in the non-linear ("dynamic") codebook: the alternative
+// reading of the 8-bit quantiser.  Magnitudes 10^-E (0.1 + 0.9 (k+1) / 2^F), k < 2^F,
+// F = B - 1 - E, E < B, with B = 7 value bits (signed, first moments) or 8 (unsigned,
+// second moments), and zero; a code is the index of the nearest entry in ascending
+// order.  In ascending order the positive magnitude number p >= 1 has F = floor(log2 p),
+// E = B - 1 - F, k = p - 2^F, so the tables are built in place by every CTA (into
+// shared memory) and no table is stored anywhere.
+// The whole update of the moments and the choice of the codes is done in double, in
+// the order a plain double-precision evaluation takes, so that the stored codes and
+// absmax values are that evaluation's; a step of this path is bound by fp64
+// arithmetic, not by memory.  The parameter update is the fp32 one of the other paths.
+// ----------------------------------------------------------------------------
+__device__ __forceinline__ double warp_max_f64(double x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmax(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+
+template <bool kCoupled>
+__device__ __forceinline__ unsigned tile_int8_dyn(const StepBlock* b, const CfgStep& P, const uint16_t* __restrict__ g,
+                                                  float* __restrict__ th, int64_t base, unsigned char* stage) {
+    static_assert(sizeof(DynTables) <= kStagesQ * kStageBytes, "the tables must fit the shared staging buffer");
+    DynTables* T = reinterpret_cast<DynTables*>(stage);
+    dyn_build(T);
+    const int64_t numel = b->numel;
+    uint8_t* __restrict__ qm = static_cast<uint8_t*>(b->s0) + base;
+    uint8_t* __restrict__ qv = static_cast<uint8_t*>(b->s1) + base;
+    float* __restrict__ am = b->a0 + base / kQBlock;
+    float* __restrict__ av = b->a1 + base / kQBlock;
+    const uint16_t* __restrict__ gt = g + base;
+    float* __restrict__ tht = th + base;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int left = int(min64(numel - base, kTileQ));
+    const double om1 = 1.0 - P.beta1_d, om2 = 1.0 - P.beta2_d;
+    float chk = 0.f;
+#pragma unroll 1
+    for (int s = 0; s < kSlicesQ; ++s) {
+        const int w0 = s * (kThreads * 8) + warp * kQBlock;
+        if (w0 >= left) break;                                       // whole warp out of range (and so are the later slices)
+        const int e = w0 + lane * 8;
+        const int cnt = max(0, min(8, left - e));
+        const double amo = double(am[w0 / kQBlock]), avo = double(av[w0 / kQBlock]);
+        double m[8], v[8];
+        float t[8];
+        double lm = 0.0, lv = 0.0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            m[j] = 0.0; v[j] = 0.0; t[j] = 0.f;
+            if (j < cnt) {
+                double gd = double(bf16_bits_to_float(gt[e + j]));
+                t[j] = tht[e + j];
+                if (kCoupled) gd += P.wd_d * double(t[j]);
+                else t[j] = fmaf(P.decay, t[j], t[j]);
+                m[j] = P.beta1_d * (T->ts[qm[e + j]] * amo) + om1 * gd;
+                v[j] = P.beta2_d * (T->tu[qv[e + j]] * avo) + om2 * (gd * gd);
+                lm = fmax(lm, fabs(m[j])); lv = fmax(lv, v[j]);
+            }
+        }
+        const float am_new = __double2float_rn(warp_max_f64(lm)), av_new = __double2float_rn(warp_max_f64(lv));
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (j < cnt) {
+                qm[e + j] = uint8_t(dyn_nearest(T->ms, am_new > 0.f ? m[j] / double(am_new) : 0.0));
+                qv[e + j] = uint8_t(dyn_nearest(T->mu, av_new > 0.f ? v[j] / double(av_new) : 0.0));
+                t[j] = adaptive_apply(t[j], float(m[j]), float(v[j]), P.step_m, P);
+                chk = poison(chk, t[j]);
+                tht[e + j] = t[j];
+            }
+        }
+        if (lane == 0) { am[w0 / kQBlock] = am_new; av[w0 / kQBlock] = av_new; }
+    }
+    return chk != 0.f;
+}
+
+// ----------------------------------------------------------------------------
+// Adafactor's update clipping and relative step size need two norms over a whole
+// block before any of its elements is updated: RMS(u) of the update
+// u = g / (sqrt(v / bc2) + eps) with the new factored second moment, and RMS(theta)
+// of the parameters before the step.  One CTA per tile of such a block leaves
+// {sum u^2, sum theta^2} in the block's list of tile sums; one CTA per block then
+// adds them in tile order and stores the clip factor 1 / max(1, RMS(u)) and the step
+// size max(1e-3, RMS(theta)) min(1e-2, 1/sqrt(t)) behind the block's mean of r.
+// ----------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+factored_norms_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
+                      const void* const* __restrict__ grads, const float* const* __restrict__ params,
+                      const __grid_constant__ StepParams SP BAOC_CHECK_PARAM) {
+#ifdef BAOC_CHECKED
+    {
+        if (int64_t(blockIdx.x) >= ck.n_tiles) { check_fail(kChkTileIndex, kKerFactoredNorms, blockIdx.x, ck.n_tiles, 0, 0); return; }
+        const Tile ct = tiles[blockIdx.x];
+        if (ct.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerFactoredNorms, ct.block, ck.n_blocks, blockIdx.x, 0); return; }
+        const StepBlock* cb = blocks + ct.block;
+        if (!check_tile(ck, kKerFactoredNorms, blockIdx.x, ct.block, int64_t(ct.piece) * kTileF, cb->numel) ||
+            !check_range(ck, kKerFactoredNorms, cb->s0, 4ll * cb->rows, 0) || !check_range(ck, kKerFactoredNorms, cb->s1, 4ll * cb->cols, 1) ||
+            !check_range(ck, kKerFactoredNorms, cb->a0, 12, 2) || !check_range(ck, kKerFactoredNorms, cb->norm_part + 2 * size_t(ct.piece), 16, 3) ||
+            !check_caller_ptr(kKerFactoredNorms, grads[ct.block], 4) || !check_caller_ptr(kKerFactoredNorms, params[ct.block], 5))
+            return;
+    }
+#endif
+    const Tile t = tiles[blockIdx.x];
+    const StepBlock* b = blocks + t.block;
+    const CfgStep& P = SP.c[b->cfg];
+    const uint16_t* __restrict__ g = static_cast<const uint16_t*>(grads[t.block]);
+    const float* __restrict__ th = params[t.block];
+    const float* __restrict__ r = static_cast<const float*>(b->s0);
+    const float* __restrict__ c = static_cast<const float*>(b->s1);
+    const int64_t numel = b->numel, base = int64_t(t.piece) * kTileF;
+    const int cols = b->cols;
+    const float rm = b->a0[0];
+    const float inv_rm = rm > 0.f ? 1.0f / rm : 0.f;
+    double acc[2] = {0.0, 0.0};
+#pragma unroll 1
+    for (int s = 0; s < kSlicesF; ++s) {
+        const int64_t e = base + int64_t(s) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+        if (e >= numel) continue;
+        const int cnt = int(min64(8, numel - e));
+        int64_t row = e / cols;
+        int col = int(e - row * cols);
+        float rs = __ldg(r + row) * inv_rm;
+        float u2 = 0.f, t2 = 0.f;
+        for (int j = 0; j < cnt; ++j) {
+            float x = bf16_bits_to_float(g[e + j]);
+            const float tt = th[e + j];
+            if (P.coupled) x = fmaf(P.wd, tt, x);
+            const float u = x * rcp_approx(fmaf(sqrt_approx(rs * __ldg(c + col)), P.rsqrt_bc2, P.eps));
+            u2 = fmaf(u, u, u2); t2 = fmaf(tt, tt, t2);
+            if (++col == cols) { col = 0; ++row; if (j + 1 < cnt) rs = __ldg(r + row) * inv_rm; }
+        }
+        acc[0] += double(u2); acc[1] += double(t2);
+    }
+    cta_reduce_store<2>(acc, b->norm_part + 2 * size_t(t.piece));
+}
+
+__global__ void __launch_bounds__(kThreads)
+factored_scale_kernel(const StepBlock* __restrict__ blocks, const int32_t* __restrict__ ids, const __grid_constant__ StepParams SP) {
+    __shared__ double sums[2];
+    const StepBlock* b = blocks + ids[blockIdx.x];
+    const CfgStep& P = SP.c[b->cfg];
+    const int ntiles = int((b->numel + kTileF - 1) / kTileF);
+    double acc[2] = {0.0, 0.0};
+    for (int i = threadIdx.x; i < ntiles; i += kThreads) { acc[0] += b->norm_part[2 * i]; acc[1] += b->norm_part[2 * i + 1]; }
+    cta_reduce_store<2>(acc, sums);
+    if (threadIdx.x == 0) {
+        const double n = double(b->numel);
+        const double rms_u = sqrt(sums[0] / n), rms_t = sqrt(sums[1] / n);
+        b->a0[1] = float(1.0 / fmax(1.0, rms_u));
+        b->a0[2] = float(fmax(1e-3, rms_t) * P.rho_d);
+    }
+}
+
 // Three instances of the kernel, one per family of update paths, each over its own stretch of the tile table:
 //   kFamHead   the five headline paths (fp32 Adam / RMS / SGD-momentum, 8-bit Adam, factored): 80 registers, three
 //              CTAs per SM, 48 KB of shared memory for the cp.async rings;
 //   kFamDense  the stateless and bf16-state dense paths: no shared memory, 64 registers, four CTAs per SM (these
 //              paths keep fewer bytes per thread in flight, so they want the extra CTA);
-//   kFamQ8     8-bit RMS scaling and 8-bit SGD-momentum: as the headline 8-bit path.
+//   kFamQ8     8-bit RMS scaling and 8-bit SGD-momentum: as the headline 8-bit path; also the alternative readings
+//              (Adam on the non-linear 8-bit codebook, the factored tuple with Adafactor's options).
 // Compiled into one kernel, the extra paths cost the headline ones registers at the 80-register budget (about 9 % on
 // the factored tiles), so a step is one launch when the assignment stays within one family and up to three otherwise.
 template <int kFam>
@@ -995,14 +1161,14 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
         switch (cb->path) {
             case kPathA32: ok = elems(cb->s0, 4, 10) && elems(cb->s1, 4, 11); break;
             case kPathA16: ok = elems(cb->s0, 2, 10) && elems(cb->s1, 2, 11); break;
-            case kPathA8: ok = elems(cb->s0, 1, 10) && elems(cb->s1, 1, 11) && scales(cb->a0, 12) && scales(cb->a1, 13); break;
+            case kPathA8: case kPathA8N: ok = elems(cb->s0, 1, 10) && elems(cb->s1, 1, 11) && scales(cb->a0, 12) && scales(cb->a1, 13); break;
             case kPathR: case kPathS: ok = elems(cb->s0, 4, 10); break;
             case kPathR16: case kPathS16: ok = elems(cb->s0, 2, 10); break;
             case kPathR8: ok = elems(cb->s1, 1, 11) && scales(cb->a1, 13); break;
             case kPathS8: ok = elems(cb->s0, 1, 10) && scales(cb->a0, 12); break;
-            case kPathF:
+            case kPathF: case kPathFA:
                 ok = check_range(ck, kKerFusedStep, cb->s0, 4ll * cb->rows, 10) && check_range(ck, kKerFusedStep, cb->s1, 4ll * cb->cols, 11) &&
-                     check_range(ck, kKerFusedStep, cb->a0, 4, 12);
+                     check_range(ck, kKerFusedStep, cb->a0, 12, 12);
                 break;
             default: break;
         }
@@ -1032,13 +1198,15 @@ fused_step_kernel(const StepBlock* __restrict__ blocks, const Tile* __restrict__
                 case kPathR: bad = tile_dense<false, true, false>(b, P, g, th, base); break;
                 case kPathS: bad = tile_dense<true, false, false>(b, P, g, th, base); break;
                 case kPathA8: bad = P.coupled ? tile_int8<true, true, true>(b, P, g, th, base, q_stage) : tile_int8<false, true, true>(b, P, g, th, base, q_stage); break;
-                case kPathF: bad = tile_factored(b, P, g, th, base, q_stage); break;
+                case kPathF: bad = tile_factored<false>(b, P, g, th, base, q_stage); break;
                 default: break;
             }
         } else {
             switch (b->path) {
                 case kPathR8: bad = P.coupled ? tile_int8<true, false, true>(b, P, g, th, base, q_stage) : tile_int8<false, false, true>(b, P, g, th, base, q_stage); break;
                 case kPathS8: bad = P.coupled ? tile_int8<true, true, false>(b, P, g, th, base, q_stage) : tile_int8<false, true, false>(b, P, g, th, base, q_stage); break;
+                case kPathA8N: bad = P.coupled ? tile_int8_dyn<true>(b, P, g, th, base, q_stage) : tile_int8_dyn<false>(b, P, g, th, base, q_stage); break;
+                case kPathFA: bad = tile_factored<true>(b, P, g, th, base, q_stage); break;
                 default: break;
             }
         }
@@ -1094,6 +1262,18 @@ int launch_factored_reduce(const StepBlock* blocks, const RedTile* rtiles, const
     factored_reduce_kernel<<<unsigned(n_red), kThreads, 0, s>>>(blocks, rtiles, grads, params, P BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     factored_combine_kernel<<<dim3(unsigned(n_factored), kCombineSlabs), kThreads, 0, s>>>(blocks, ids, P BAOC_CHECK_ARG(ck));
+    BAOC_LAUNCH_CHECK();
+    return 0;
+}
+
+int launch_factored_norms(const StepBlock* blocks, const Tile* tiles, const int32_t* ids, const void* const* grads,
+                          const float* const* params, int64_t n_tiles, int n, const StepParams& P, const CheckCtx& ck,
+                          cudaStream_t s) {
+    (void)ck;
+    if (n_tiles <= 0 || n <= 0) return 0;
+    factored_norms_kernel<<<unsigned(n_tiles), kThreads, 0, s>>>(blocks, tiles, grads, params, P BAOC_CHECK_ARG(ck));
+    BAOC_LAUNCH_CHECK();
+    factored_scale_kernel<<<n, kThreads, 0, s>>>(blocks, ids, P);
     BAOC_LAUNCH_CHECK();
     return 0;
 }

@@ -14,7 +14,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 # the odd-size and mixed cases of the parity suite: every kernel of the window, of the finalize and of the step, every
 # update path, ragged tails, one-element blocks, sampling, re-configuration
 CASES = ("odd_sizes or each_configuration or stateless_bf16 or factored_with or finalize_from_shared or sampled_statistics "
-         "or reconfigure or configure_from_window or toy_pipeline or grouped_factored or nonfinite or coupled_decay")
+         "or reconfigure or configure_from_window or toy_pipeline or grouped_factored or nonfinite or coupled_decay "
+         "or dynamic_codebook or adafactor")
 
 
 def _child(args, timeout=1500):

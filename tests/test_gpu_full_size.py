@@ -26,7 +26,10 @@ N_STEPS = 10
 
 def _ocfg(c):
     return O.Config(c.adaptive, c.momentum, c.decoupled_wd, c.factored, c.bits, lr=float(c.lr), beta1=float(c.beta1),
-                    beta2=float(c.beta2), eps=float(c.eps), weight_decay=float(c.weight_decay))
+                    beta2=float(c.beta2), eps=float(c.eps), weight_decay=float(c.weight_decay),
+                    quantizer="dynamic" if c.quantizer else "linear", af_beta2_schedule=bool(c.af_flags & 1),
+                    af_clip=1.0 if c.af_flags & 2 else 0.0, af_relative_step=bool(c.af_flags & 4),
+                    af_eps1=1e-30 if c.af_flags & 8 else 0.0)
 
 
 def _close(got, ref):
@@ -217,7 +220,7 @@ def test_one_block_beyond_two_to_the_31_elements():
 
 
 def test_every_tuple_family_in_one_step_at_full_size():
-    """All thirteen instantiable tuples dealt round-robin over the blocks of the LLaMA-1B-shaped workload, so that one
+    """All fifteen instantiable tuples (the two alternative readings included) dealt round-robin over the blocks of the LLaMA-1B-shaped workload, so that one
     step launches every kernel instance (headline paths, stateless / bf16 dense paths, 8-bit single-moment paths) over
     its stretch of the tile table; ten steps, checked on slices (whole blocks for the factored ones)."""
     from paper_2605_04711_b200 import binding as B, harness as H
@@ -226,13 +229,14 @@ def test_every_tuple_family_in_one_step_at_full_size():
     sess = H.Session(wl, configs=bcfgs, n_grad_sets=2)
     sess.init_params()
     cfgs = [_ocfg(c) for c in bcfgs]
-    factored = {3: 2, 11: 7, 12: 9}                                  # vectors take RMS scaling at the same precision
+    factored = {3: 2, 11: 7, 12: 9, 14: 2}                           # vectors take RMS scaling at the same precision
     assign = []
     for i, b in enumerate(wl.blocks):
         c = i % len(bcfgs)
         assign.append(factored[c] if (c in factored and b.cols <= 1) else c)
     kinds = [O.config_kind(cfgs[c]) for c in assign]
-    assert set(kinds) == {"A32", "A8", "R", "F", "S", "G", "A16", "R16", "S16", "R8", "S8", "F16", "F8"}
+    assert set(kinds) == {"A32", "A8", "R", "F", "S", "G", "A16", "R16", "S16", "R8", "S8", "F16", "F8", "A8N"}
+    assert any(cfgs[c].af_clip for c in assign)                      # the factored tuple with Adafactor's options is among them
     sess.configure(assign)
     mem, _ = sess.h.cost_model()
     assert sess.h.query().state_bytes == sum(int(mem[i, c]) for i, c in enumerate(assign))
@@ -242,6 +246,8 @@ def test_every_tuple_family_in_one_step_at_full_size():
         if kind.startswith("F"):
             ids = [i for i in ids if wl.blocks[i].numel <= 17_000_000] or ids
             picks += [(ids[0], kind)]
+            with_options = [i for i in ids if cfgs[assign[i]].af_clip and i != ids[0]]
+            picks += [(with_options[0], kind)] if with_options else []
         else:
             picks += [(i, kind) for i in sorted({ids[0], max(ids, key=lambda i: wl.blocks[i].numel)})]
     samples = []
@@ -262,7 +268,7 @@ def test_every_tuple_family_in_one_step_at_full_size():
             g = sess.grad_views[k][s["i"]][s["lo"]:s["hi"]].double().cpu().numpy()
             s["th"] = O.step(s["th"], g, s["st"], cfgs[assign[s["i"]]], s["rows"], s["cols"])
     torch.cuda.synchronize()
-    assert sess.h.query().kernel_launches - launches0 == N_STEPS * 5    # row/column reduce + combine, three instances
+    assert sess.h.query().kernel_launches - launches0 == N_STEPS * 7    # row/column reduce + combine, two norms kernels, three instances
     assert sess.h.nonfinite()[0] == 0
     bad, total = 0, 0
     rel = lambda x, y: float(np.max(np.abs(x - y)) / max(float(np.max(np.abs(y))), 1e-30))
@@ -305,6 +311,10 @@ def test_every_tuple_family_in_one_step_at_full_size():
             patterns(10, ref.m); patterns(11, ref.v)
         elif kind in ("R16", "S16"):
             patterns(10, ref.v if kind == "R16" else ref.m)
+        elif kind == "A8N":
+            codes(10, torch.uint8, ref.qm); codes(11, torch.uint8, ref.qv)
+            assert rel(f32(12, q0, q1), ref.am.astype(np.float64)) <= 1e-6, name
+            assert rel(f32(13, q0, q1), ref.av.astype(np.float64)) <= 1e-6, name
         elif kind == "A8":
             codes(10, torch.int8, ref.qm); codes(11, torch.uint8, ref.qv)
             assert rel(f32(12, q0, q1), ref.am.astype(np.float64)) <= 1e-6, name
