@@ -393,8 +393,9 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
         h->launches += 3;
     }
     LAUNCH(launch_final_resid_select(blocks, tiles, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<RankSel>(ws, L.sel),
-                                     at<uint32_t>(ws, L.hist), at<double>(ws, L.acc), h->n_stat_tiles, n, ws_ctx(h, h->n_stat_tiles), s),
-           "final_hist_kernel");
+                                     at<uint32_t>(ws, L.hist), at<uint32_t>(ws, L.surv), at<uint32_t>(ws, L.surv_cnt),
+                                     at<double>(ws, L.acc), h->n_stat_tiles, n, ws_ctx(h, h->n_stat_tiles), s),
+           "final_resid_hist_kernel");
     h->launches += 6;
 
     std::vector<double> out(size_t(kFinOut) * n);

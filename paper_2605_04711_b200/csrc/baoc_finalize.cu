@@ -3,8 +3,9 @@
 // (Eq. 7) and the precision cosines (Eq. 8), and the exact quantiles behind the
 // anisotropy (Eq. 4).  Three sweeps over the window's moments:
 //   1. final_sums_kernel   reads m, v, theta: 16 sums per block, and the histogram of the top 12 bits of v
-//   2. final_hist_kernel<true>   reads v: Eq. 7 residual (after the row/column sums), histogram of the next 12 bits
-//   3. final_hist_kernel<false>  reads v: histogram of the last 8 bits
+//   2. final_resid_hist_kernel   reads v: Eq. 7 residual (after the row/column sums), histogram of the next 12 bits of
+//                                the elements that share a rank's top 12 bits, and the list of those elements
+//   3. final_last_kernel         reads that list (a tenth of v or less): histogram of the last 8 bits
 // A CTA works through a run of consecutive tiles, keeps its partial sums and
 // histograms on chip while the tiles belong to one block, and hands them over
 // once per block (a deterministic, fixed partition of the work).
@@ -339,26 +340,79 @@ final_resid_combine_kernel(const StatBlock* __restrict__ blocks, const double* _
 // the numeric order): four ranks per block (the two order statistics around each
 // of the two quantile positions); ranks that still share a prefix share one
 // histogram (the "leader" rank's).  The first pass (top 12 bits) is part of the
-// first sweep; here
-//   kResid = true:  second pass, bits [8, 20) of the elements whose top 12 bits are a rank's prefix, and in the same
-//                   sweep the Eq. 7 numerator
-//                     sum (S_ij - a_i b_j / mu)^2 = sum (v_ij - rowsum_i colsum_j / total)^2
-//                   of matrix blocks, in double (a difference of nearly equal numbers);
-//   kResid = false: third pass, bits [0, 8) of the elements whose upper 24 bits are a rank's prefix.
-// Few elements match a prefix: a thread first tests whether any of its 16 does.  A thread whose 16 elements are all
-// equal (constant or untouched stretches of a tensor) adds them with one atomic.
-// The histograms count in 16 bits, two bins per word, which halves their shared memory (32 KB, so that four CTAs fit
-// an SM and keep enough loads in flight); a CTA therefore hands its histograms over after at most kSelRunTiles = 15
-// tiles (61440 elements, below 2^16).  (Staging the tiles through a cp.async ring at two CTAs per SM was slower.)
+// first sweep.
+//
+// Sweep 2 (final_resid_hist_kernel) reads v: the second pass, bits [8, 20) of the
+// elements whose top 12 bits are a rank's prefix (the "survivors"), and in the
+// same sweep the Eq. 7 numerator
+//     sum (S_ij - a_i b_j / mu)^2 = sum (v_ij - rowsum_i colsum_j / total)^2
+// of matrix blocks, in double (a difference of nearly equal numbers).
+// Survivors are few (one bin of the first digit is an eighth of an octave), so
+// they are not counted where they are found, which would leave most lanes idle
+// around every atomic: a thread notes which of its 16 elements survive in a bit
+// mask and copies them to its warp's staging segment; the warp then counts the
+// staged values with all lanes busy (lanes holding equal values add once).  The
+// staged values also go to a survivors list in global memory, kSurvTile slots per
+// tile of the CTA's run of tiles of one block.
+//
+// Sweep 3 (final_last_kernel) reads that list instead of v: the third pass, bits
+// [0, 8) of the survivors whose upper 24 bits are a rank's prefix.  A run whose
+// survivors did not fit its slots (more than one element in eight: a constant or
+// nearly constant tensor) is marked, and the third pass reads v for that run.
+//
+// The second pass counts in 16 bits, two bins per word (32 KB of histograms, 16 KB
+// of staging); a CTA therefore hands its histograms over after at most
+// kSelRunTiles = 15 tiles (61440 elements, below 2^16).
 // ============================================================================
-constexpr int kFhHistWords = kSelBins / 2;
-constexpr int kFhSmemBytes = kRanks * kFhHistWords * 4;
+constexpr int kRhHistWords = kSelBins / 2;
+constexpr int kRhHistBytes = kRanks * kRhHistWords * 4;
+constexpr int kRhSegWords = kTile / (kThreads / 32);          // a warp's 512 elements of a tile, should all survive
+constexpr int kRhSmemBytes = kRhHistBytes + kTile * 4;
 static_assert(kSelRunTiles * kTile < 65536, "a 16-bit bin must hold a whole run of tiles");
 
-template <bool kResid>
-__global__ void __launch_bounds__(kThreads, kResid ? 3 : 4)
-final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const RankSel* __restrict__ sel,
-                  double* __restrict__ fin, uint32_t* __restrict__ hist, int64_t n_tiles, int tiles_per_cta BAOC_CHECK_PARAM) {
+// The distinct prefixes the ranks of a block still have (one per leader), padded with a value no key takes.
+struct Leaders {
+    uint32_t key[kRanks];
+    int slot[kRanks];
+    int n;
+};
+__device__ __forceinline__ Leaders leaders_of(const RankSel* __restrict__ sel, int key_shift) {
+    Leaders L;
+    L.n = 0;
+#pragma unroll
+    for (int r = 0; r < kRanks; ++r) { L.key[r] = 0xffffffffu; L.slot[r] = 0; }
+#pragma unroll
+    for (int r = 0; r < kRanks; ++r) {
+        const RankSel s = sel[r];
+        if (s.leader == r) {
+#pragma unroll
+            for (int k = 0; k < kRanks; ++k)
+                if (k == L.n) { L.key[k] = s.prefix >> key_shift; L.slot[k] = r; }
+            ++L.n;
+        }
+    }
+    return L;
+}
+
+// bit j set: element j of the thread (8 h + i: slice h, element i) is in range and its key is a leader's
+template <int kL, bool kFull, int kKeyShift>
+__device__ __forceinline__ uint32_t match_mask(const uint32_t (&u)[16], const int (&valid)[2], const Leaders& L) {
+    uint32_t mask = 0u;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const uint32_t key = u[j] >> kKeyShift;
+        bool p = (key == L.key[0]) | (key == L.key[1]);
+        if (kL > 2) p |= (key == L.key[2]) | (key == L.key[3]);
+        if (!kFull) p &= (j & 7) < valid[j >> 3];
+        if (p) mask |= 1u << j;
+    }
+    return mask;
+}
+
+__global__ void __launch_bounds__(kThreads, 3)
+final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const RankSel* __restrict__ sel,
+                        double* __restrict__ fin, uint32_t* __restrict__ hist, uint32_t* __restrict__ surv,
+                        uint32_t* __restrict__ surv_cnt, int64_t n_tiles, int tiles_per_cta BAOC_CHECK_PARAM) {
 #ifdef BAOC_CHECKED
     {
         const int64_t c0 = int64_t(blockIdx.x) * tiles_per_cta, c1 = min64(c0 + tiles_per_cta, n_tiles);
@@ -372,26 +426,32 @@ final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
             if (!check_tile(ck, kKerFinalHist, ti, ct.block, cbase, cb->numel) ||
                 !check_range(ck, kKerFinalHist, cb->v + cbase, 4 * cn, 0) ||
                 !check_range(ck, kKerFinalHist, hist + size_t(ct.block) * kRanks * kSelBins, 4ll * kRanks * kSelBins, 1) ||
-                !check_range(ck, kKerFinalHist, sel + size_t(ct.block) * kRanks, int64_t(sizeof(RankSel)) * kRanks, 2))
-                return;
-            if (kResid && (!check_range(ck, kKerFinalHist, fin + size_t(ti) * kResidSums, 8 * kResidSums, 3) ||
-                           (cb->cols > 1 && (!check_range(ck, kKerFinalHist, cb->rowsum, 8ll * (cb->rows + 1), 4) ||
-                                             !check_range(ck, kKerFinalHist, cb->colsum, 8ll * cb->cols, 5)))))
+                !check_range(ck, kKerFinalHist, sel + size_t(ct.block) * kRanks, int64_t(sizeof(RankSel)) * kRanks, 2) ||
+                !check_range(ck, kKerFinalHist, fin + size_t(ti) * kResidSums, 8 * kResidSums, 3) ||
+                !check_range(ck, kKerFinalHist, surv + size_t(ti) * kSurvTile, 4ll * kSurvTile, 6) ||
+                !check_range(ck, kKerFinalHist, surv_cnt + ti, 4, 7) ||
+                (cb->cols > 1 && (!check_range(ck, kKerFinalHist, cb->rowsum, 8ll * (cb->rows + 1), 4) ||
+                                  !check_range(ck, kKerFinalHist, cb->colsum, 8ll * cb->cols, 5))))
                 return;
         }
     }
 #endif
     extern __shared__ __align__(16) unsigned char dyn[];
-    uint32_t (*sh)[kFhHistWords] = reinterpret_cast<uint32_t (*)[kFhHistWords]>(dyn);
-    constexpr int kShift = kResid ? kSel3Bits : 0;            // lowest bit of this pass's digit
-    constexpr int kBits = kResid ? kSelBits : kSel3Bits;      // width of the digit
+    uint32_t (*sh)[kRhHistWords] = reinterpret_cast<uint32_t (*)[kRhHistWords]>(dyn);
+    uint32_t* stage = reinterpret_cast<uint32_t*>(dyn + kRhHistBytes);
+    __shared__ int wcnt[kThreads / 32];                       // survivors a warp has staged of its current tile
+    __shared__ int run_cnt, run_over;                         // survivors of the run written so far; the run outgrew its slots
+    constexpr int kKeyShift = 32 - kSelBits;                  // the first digit
     constexpr int kSl = kTile / (kThreads * 8);
     static_assert(kSl == 2, "a tile is two slices of eight elements per thread");
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
-    uint32_t prefix[kRanks], upper[kRanks];                   // upper: the prefix above this pass's digit
-    bool lead[kRanks];
+    Leaders L;
+    L.n = 0;
     int cur_block = -1;
     int64_t run_first = first;
+    int cap = 0;                                              // slots of the current run
+    uint32_t* surv_run = surv;
     double acc[kResidSums] = {0.0};
     // position of the current tile's first element in its matrix, kept by 32-bit arithmetic from tile to tile
     int64_t row0 = 0;
@@ -399,29 +459,27 @@ final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
     int64_t next_base = -1;
 
     auto flush = [&](int blk, int64_t t_begin) {
-        if (kResid) {
-            cta_reduce_store<kResidSums>(acc, fin + size_t(t_begin) * kResidSums);
-            acc[0] = 0.0;
-        } else {
-            __syncthreads();
+        cta_reduce_store<kResidSums>(acc, fin + size_t(t_begin) * kResidSums);   // (every warp has drained its last tile)
+        acc[0] = 0.0;
+        if (threadIdx.x == 0) {
+            surv_cnt[t_begin] = run_over ? kSurvOverflow : uint32_t(run_cnt);
+            run_cnt = 0; run_over = 0;
         }
 #pragma unroll
-        for (int r = 0; r < kRanks; ++r) {
-            if (!lead[r]) continue;                           // uniform over the CTA
-            uint32_t* out = hist + (size_t(blk) * kRanks + r) * kSelBins;
-            for (int w = threadIdx.x; w < kFhHistWords; w += kThreads) {
-                const uint32_t x = sh[r][w];
+        for (int k = 0; k < kRanks; ++k) {
+            if (k >= L.n) continue;                           // uniform over the CTA
+            uint32_t* out = hist + (size_t(blk) * kRanks + L.slot[k]) * kSelBins;
+            for (int w = threadIdx.x; w < kRhHistWords; w += kThreads) {
+                const uint32_t x = sh[k][w];
                 if (x) {
                     if (x & 0xffffu) atomicAdd(out + 2 * w, x & 0xffffu);
                     if (x >> 16) atomicAdd(out + 2 * w + 1, x >> 16);
-                    sh[r][w] = 0u;
+                    sh[k][w] = 0u;
                 }
             }
         }
         __syncthreads();
     };
-    // n elements into bin d of rank slot r
-    auto count = [&](int r, uint32_t d, uint32_t n) { atomicAdd(&sh[r][d >> 1], n << ((d & 1u) * 16u)); };
     // floor(x / cols_u) for x < 2^32 from the precomputed floor((2^32 - 1) / cols_u): the estimate is at most 2 short
     auto divmod = [&](uint32_t x, uint32_t& rem) {
         uint32_t q = __umulhi(x, magic);
@@ -431,7 +489,9 @@ final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
         return q;
     };
 
-    for (int i = threadIdx.x; i < kRanks * kFhHistWords; i += kThreads) (&sh[0][0])[i] = 0u;
+    for (int i = threadIdx.x; i < kRanks * kRhHistWords; i += kThreads) (&sh[0][0])[i] = 0u;
+    if (threadIdx.x < kThreads / 32) wcnt[threadIdx.x] = 0;
+    if (threadIdx.x == 0) { run_cnt = 0; run_over = 0; }
     __syncthreads();
 
 #pragma unroll 1
@@ -443,20 +503,15 @@ final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
             if (cur_block >= 0) flush(cur_block, run_first);
             cur_block = int(t.block);
             run_first = ti;
-#pragma unroll
-            for (int r = 0; r < kRanks; ++r) {
-                const RankSel s = sel[size_t(t.block) * kRanks + r];
-                prefix[r] = s.prefix; lead[r] = s.leader == r;
-                upper[r] = s.prefix >> (kShift + kBits);
-            }
-            if (kResid) {
-                cols_u = uint32_t(b->cols);
-                magic = 0xffffffffu / cols_u;
-                next_base = -1;
-            }
+            L = leaders_of(sel + size_t(t.block) * kRanks, kKeyShift);
+            cap = int(min64(last, b->tile0 + b->ntiles) - ti) * kSurvTile;
+            surv_run = surv + size_t(ti) * kSurvTile;
+            cols_u = uint32_t(b->cols);
+            magic = 0xffffffffu / cols_u;
+            next_base = -1;
         }
         const int64_t numel = b->numel;
-        if (kResid && cols_u > 1u) {
+        if (cols_u > 1u) {
             if (base == next_base) {                          // the next piece of the same matrix: advance by one tile
                 uint32_t rem;
                 row0 += divmod(col0 + uint32_t(kTile), rem);
@@ -481,7 +536,7 @@ final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
         }
         const bool tile_full = base + kTile <= numel;         // uniform over the CTA
 
-        if (kResid && cols_u > 1u) {
+        if (cols_u > 1u) {
             const double* __restrict__ rowsum = b->rowsum;
             const double* __restrict__ colsum = b->colsum;
             const double total = rowsum[b->rows];             // the block's sum of v, left there by the row/column combine
@@ -515,32 +570,138 @@ final_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
             }
         }
 
-        // ---- the histogram of this pass's digit
-        uint32_t differ = 0u;
-        bool any = false;
+        // ---- the survivors of this tile: noted, staged by warp, counted, listed
+        uint32_t mask;
+        if (tile_full) mask = L.n <= 2 ? match_mask<2, true, kKeyShift>(u, valid, L) : match_mask<4, true, kKeyShift>(u, valid, L);
+        else mask = match_mask<4, false, kKeyShift>(u, valid, L);
+        uint32_t* seg = stage + warp * kRhSegWords;
+        const int mine = __popc(mask);
+        int pos = mine ? atomicAdd(&wcnt[warp], mine) : 0;
 #pragma unroll
-        for (int j = 0; j < 8 * kSl; ++j) {
-            differ |= u[j] ^ u[0];
-            const uint32_t key = u[j] >> (kShift + kBits);
-            any |= (tile_full || (j & 7) < valid[j >> 3]) &
-                   ((key == upper[0]) | (key == upper[1]) | (key == upper[2]) | (key == upper[3]));
-        }
-        if (any) {
-#pragma unroll
-            for (int r = 0; r < kRanks; ++r) {
-                if (!lead[r]) continue;
-                if (tile_full && differ == 0u) {
-                    if ((u[0] >> (kShift + kBits)) == upper[r]) count(r, (u[0] >> kShift) & ((1u << kBits) - 1u), uint32_t(8 * kSl));
-                    continue;
-                }
-#pragma unroll
-                for (int j = 0; j < 8 * kSl; ++j)
-                    if ((tile_full || (j & 7) < valid[j >> 3]) && (u[j] >> (kShift + kBits)) == upper[r])
-                        count(r, (u[j] >> kShift) & ((1u << kBits) - 1u), 1u);
+        for (int j = 0; j < 8 * kSl; ++j)
+            if (mask & (1u << j)) seg[pos++] = u[j];
+        __syncwarp();
+        const int staged = wcnt[warp];                        // uniform over the warp
+        if (staged > 0) {
+            int off = 0;
+            if (lane == 0) {
+                off = atomicAdd(&run_cnt, staged);
+                if (off + staged > cap) run_over = 1;
             }
+            off = __shfl_sync(0xffffffffu, off, 0);
+            const bool fits = off + staged <= cap;
+            for (int i0 = 0; i0 < staged; i0 += 32) {
+                const int i = i0 + lane;
+                const bool on = i < staged;
+                const unsigned act = __ballot_sync(0xffffffffu, on);
+                if (on) {
+                    const uint32_t x = seg[i];
+                    if (fits) surv_run[off + i] = x;
+                    const unsigned same = __match_any_sync(act, x);
+                    if (lane == __ffs(int(same)) - 1) {       // one lane per distinct value adds for all of them
+                        const uint32_t key = x >> kKeyShift, d = (x >> kSel3Bits) & uint32_t(kSelBins - 1);
+                        const uint32_t n = uint32_t(__popc(same)) << ((d & 1u) * 16u);
+#pragma unroll
+                        for (int k = 0; k < kRanks; ++k)
+                            if (key == L.key[k]) atomicAdd(&sh[k][d >> 1], n);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) wcnt[warp] = 0;
+            __syncwarp();
         }
     }
     if (cur_block >= 0) flush(cur_block, run_first);
+}
+
+// Sweep 3: the last 8 bits.  Same partition of the tiles into runs as sweep 2; per run either its survivors list or, for
+// a run that was marked, the tiles of v themselves.  The histogram (256 bins of 32 bits per leader) is handed over per run.
+constexpr int kLastBins = 1 << kSel3Bits;
+
+__global__ void __launch_bounds__(kThreads)
+final_last_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const RankSel* __restrict__ sel,
+                  uint32_t* __restrict__ hist, const uint32_t* __restrict__ surv, const uint32_t* __restrict__ surv_cnt,
+                  int64_t n_tiles, int tiles_per_cta BAOC_CHECK_PARAM) {
+    __shared__ uint32_t sh[kRanks][kLastBins];
+    const int lane = threadIdx.x & 31;
+    const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
+#ifdef BAOC_CHECKED
+    if (first >= ck.n_tiles || n_tiles != ck.n_tiles) { check_fail(kChkTileIndex, kKerFinalLast, first, ck.n_tiles, n_tiles, 0); return; }
+#endif
+    for (int i = threadIdx.x; i < kRanks * kLastBins; i += kThreads) (&sh[0][0])[i] = 0u;
+    __syncthreads();
+
+    // one lane per distinct value among the lanes `act` adds for all of them
+    auto count_same = [&](unsigned act, uint32_t x, const Leaders& L) {
+        const unsigned same = __match_any_sync(act, x);
+        if (lane == __ffs(int(same)) - 1) {
+            const uint32_t key = x >> kSel3Bits, d = x & uint32_t(kLastBins - 1);
+#pragma unroll
+            for (int k = 0; k < kRanks; ++k)
+                if (key == L.key[k]) atomicAdd(&sh[k][d], uint32_t(__popc(same)));
+        }
+    };
+
+#pragma unroll 1
+    for (int64_t t_begin = first; t_begin < last;) {
+        const Tile t = tiles[t_begin];
+#ifdef BAOC_CHECKED
+        if (t.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerFinalLast, t.block, ck.n_blocks, t_begin, 0); return; }
+#endif
+        const StatBlock* b = blocks + t.block;
+        const int64_t t_end = min64(last, b->tile0 + b->ntiles);     // the run: this CTA's tiles of the block
+        const Leaders L = leaders_of(sel + size_t(t.block) * kRanks, kSel3Bits);
+        const uint32_t cnt = surv_cnt[t_begin];
+#ifdef BAOC_CHECKED
+        if (!check_range(ck, kKerFinalLast, surv_cnt + t_begin, 4, 0) ||
+            !check_range(ck, kKerFinalLast, surv + size_t(t_begin) * kSurvTile, 4ll * kSurvTile * (t_end - t_begin), 1) ||
+            !check_range(ck, kKerFinalLast, hist + size_t(t.block) * kRanks * kSelBins, 4ll * kRanks * kSelBins, 2) ||
+            (cnt != kSurvOverflow && int64_t(cnt) > int64_t(kSurvTile) * (t_end - t_begin) &&
+             !check_fail(kChkRange, kKerFinalLast, 3, cnt, t_begin, t_end)))
+            return;
+#endif
+        if (cnt != kSurvOverflow) {
+            const uint32_t* __restrict__ list = surv + size_t(t_begin) * kSurvTile;
+            for (uint32_t i0 = 0; i0 < cnt; i0 += kThreads) {             // uniform over the CTA
+                const uint32_t i = i0 + threadIdx.x;
+                const bool on = i < cnt;
+                const unsigned act = __ballot_sync(0xffffffffu, on);
+                if (on) count_same(act, list[i], L);
+            }
+        } else {
+            const uint32_t* __restrict__ v = reinterpret_cast<const uint32_t*>(b->v);
+            const int64_t e0 = int64_t(t.piece) * kTile, e1 = min64(b->numel, e0 + (t_end - t_begin) * int64_t(kTile));
+#ifdef BAOC_CHECKED
+            if (!check_range(ck, kKerFinalLast, v + e0, 4 * (e1 - e0), 4)) return;
+#endif
+            for (int64_t i0 = e0; i0 < e1; i0 += kThreads) {              // uniform over the CTA
+                const int64_t i = i0 + threadIdx.x;
+                const bool on = i < e1;
+                uint32_t x = 0u;
+                bool hit = false;
+                if (on) {
+                    x = v[i];
+                    const uint32_t key = x >> kSel3Bits;
+                    hit = (key == L.key[0]) | (key == L.key[1]) | (key == L.key[2]) | (key == L.key[3]);
+                }
+                const unsigned act = __ballot_sync(0xffffffffu, hit);
+                if (hit) count_same(act, x, L);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kRanks; ++k) {
+            if (k >= L.n) continue;                           // uniform over the CTA
+            uint32_t* out = hist + (size_t(t.block) * kRanks + L.slot[k]) * kSelBins;
+            for (int w = threadIdx.x; w < kLastBins; w += kThreads) {
+                const uint32_t x = sh[k][w];
+                if (x) { atomicAdd(out + w, x); sh[k][w] = 0u; }
+            }
+        }
+        __syncthreads();
+        t_begin = t_end;
+    }
 }
 
 // One CTA per block: for each of the four ranks find the bin of its leader's
@@ -676,22 +837,21 @@ int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* c
 }
 
 int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                              uint32_t* hist, const double* acc, int64_t n_tiles, int n_blocks, const CheckCtx& ck,
-                              cudaStream_t s) {
+                              uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc, int64_t n_tiles,
+                              int n_blocks, const CheckCtx& ck, cudaStream_t s) {
     (void)ck;
-    constexpr int kSmem = kFhSmemBytes;
-    cudaError_t e = cudaFuncSetAttribute(final_hist_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(final_hist_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    cudaError_t e = cudaFuncSetAttribute(final_resid_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRhSmemBytes);
     if (e != cudaSuccess) return int(e);
     const int per = run_tiles(n_tiles, kSelRunTiles);
     const unsigned grid = unsigned((n_tiles + per - 1) / per);
-    final_hist_kernel<true><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per BAOC_CHECK_ARG(ck));
+    final_resid_hist_kernel<<<grid, kThreads, kRhSmemBytes, s>>>(blocks, tiles, sel, fin, hist, surv, surv_cnt, n_tiles,
+                                                                per BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     final_resid_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
     BAOC_LAUNCH_CHECK();
     select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, kSel3Bits, kSelBins);
     BAOC_LAUNCH_CHECK();
-    final_hist_kernel<false><<<grid, kThreads, kSmem, s>>>(blocks, tiles, sel, fin, hist, n_tiles, per BAOC_CHECK_ARG(ck));
+    final_last_kernel<<<grid, kThreads, 0, s>>>(blocks, tiles, sel, hist, surv, surv_cnt, n_tiles, per BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, 0, 1 << kSel3Bits);
     BAOC_LAUNCH_CHECK();

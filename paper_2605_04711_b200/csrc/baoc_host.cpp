@@ -140,6 +140,8 @@ void compute_stat_layout(Handle* h) {
     L.fin_out = take(&cur, 8 * size_t(kFinOut) * n);
     L.hist = take(&cur, 4 * size_t(kSelBins) * kRanks * n);
     L.sel = take(&cur, sizeof(RankSel) * size_t(kRanks) * n);
+    L.surv = take(&cur, 4 * size_t(kSurvTile) * size_t(tiles));
+    L.surv_cnt = take(&cur, 4 * size_t(tiles));
     L.rowsum = take(&cur, 8 * size_t(std::max<int64_t>(sum_rows, 1)));
     L.colsum = take(&cur, 8 * size_t(std::max<int64_t>(sum_cols, 1)));
     L.redpart = take(&cur, 8 * size_t(std::max<int64_t>(redpart, 1)));

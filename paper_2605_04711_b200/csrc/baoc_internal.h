@@ -40,6 +40,8 @@ constexpr int kSelBins = 1 << kSelBits;
 constexpr int kSel3Bits = 32 - 2 * kSelBits;   // bits of the third and last pass
 constexpr int kFinRunTiles = 8;       // most tiles a CTA of the first finalize sweep works through (its partial sums stay in fp32 that long)
 constexpr int kSelRunTiles = 15;      // most tiles a CTA of the other two sweeps works through (their histograms count in 16 bits)
+constexpr int kSurvTile = 512;        // slots per tile in the list of the select's survivors (elements that share a rank's first digit)
+constexpr uint32_t kSurvOverflow = 0xffffffffu;   // count of a run whose survivors did not fit: the last pass reads v instead
 constexpr int kRedRows = 64;          // rows per CTA of the row/column reduction kernel
 constexpr int kRedCols = 512;         // columns per CTA of the row/column reduction kernel
 constexpr int kTileF = 16384;         // elements per tile of the factored path (its slices are prefetched through shared memory)
@@ -262,7 +264,7 @@ struct Handle {
     std::vector<const void*> last_stat_grads;
     std::vector<const void*> last_stat_params;
     struct StatLayout {
-        size_t blocks, tiles, red_tiles, matrix_ids, grads, params, m, v, gprev, partials, acc, fin, fin_out, hist, sel,
+        size_t blocks, tiles, red_tiles, matrix_ids, grads, params, m, v, gprev, partials, acc, fin, fin_out, hist, sel, surv, surv_cnt,
                rowsum, colsum, redpart, ridx, cidx, gsample, psample, sgrads, sparams, total;
     } sl{};
 
@@ -349,8 +351,8 @@ int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* c
                       double* fin_out, uint32_t* hist, RankSel* sel, int64_t n_tiles, int n_blocks, double eps,
                       float eps_adam, int quantizer8, const CheckCtx& ck, cudaStream_t s);
 int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                              uint32_t* hist, const double* acc, int64_t n_tiles, int n_blocks, const CheckCtx& ck,
-                              cudaStream_t s);
+                              uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc, int64_t n_tiles,
+                              int n_blocks, const CheckCtx& ck, cudaStream_t s);
 int launch_sample_gather(const StatBlock* blocks, const Tile* tiles, const void* const* src, int64_t n_tiles, int fp32,
                          const CheckCtx& ck, cudaStream_t s);
 int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const int32_t* ids, int64_t n_red, int n_matrix,

@@ -204,6 +204,30 @@ def test_stats_invariants_identical_zero_and_flipped_gradients(B, H):
             assert st2[i]["F"] < 1e-6                                # constant matrix is rank one
 
 
+def test_quantile_select_with_long_stretches_of_equal_values(B, H):
+    """Eq. 4's quantiles when many elements of v are equal: the leading 40 % of every block never sees a gradient
+    (v = 0 there, so the 10 % quantile is exactly 0 and its bin holds far more than one element in eight), the rest
+    does.  Tiles inside the stretch overflow their survivor slots and are re-read from v by the last radix pass,
+    tiles outside it go through the list; both must give the oracle's order statistics."""
+    wl = _odd_workload(seed=9, window=4)
+    sess = H.Session(wl, n_grad_sets=2)
+    sess.init_params()
+    o = O.Opts()
+    states = [O.stats_init(b.numel) for b in wl.blocks]
+    for t in range(1, wl.window + 1):
+        k = sess.fill_grads(t)
+        for i, b in enumerate(wl.blocks):
+            sess.grad_views[k][i].view(-1)[: (2 * b.numel) // 5].zero_()
+        sess.sample_stats(k)
+        for i in range(len(wl.blocks)):
+            O.stats_step(states[i], sess.block_grad_host(k, i), o)
+    _, st, _ = _check_stats(sess, states, o)
+    for i, b in enumerate(wl.blocks):
+        if b.numel >= 10:
+            raw = O.stats_finalize(states[i], sess.block_param_host(i), b.rows, b.cols, o)
+            assert st[i]["A"] == pytest.approx(raw["A"], rel=1e-6), (b.name, st[i]["A"], raw["A"])
+
+
 def test_sampled_statistics_match_the_oracle_on_the_sample(B, H):
     """Coordinate sampling (Sec. 3.1): every block is observed on a fixed sub-grid; the oracle gets the same entries."""
     wl = _odd_workload(seed=71, window=5)
