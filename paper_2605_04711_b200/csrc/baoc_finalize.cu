@@ -448,7 +448,14 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __rest
     const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
     Leaders L;
     L.n = 0;
+    // what the tiles of one block share, fetched once when the CTA enters the block (nothing a tile needs then hangs on
+    // a chain of dependent loads): its extent in the tile table, v, the row/column sums, 1 / total
     int cur_block = -1;
+    int64_t blk_end = first, tile0 = 0, numel = 0;
+    const uint32_t* __restrict__ v = nullptr;
+    const double* __restrict__ rowsum = nullptr;
+    const double* __restrict__ colsum = nullptr;
+    double inv_total = 0.0;
     int64_t run_first = first;
     int cap = 0;                                              // slots of the current run
     uint32_t* surv_run = surv;
@@ -496,21 +503,29 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __rest
 
 #pragma unroll 1
     for (int64_t ti = first; ti < last; ++ti) {
-        const Tile t = tiles[ti];
-        const StatBlock* b = blocks + t.block;
-        const int64_t base = int64_t(t.piece) * kTile;
-        if (int(t.block) != cur_block) {                      // uniform over the CTA
+        if (ti == blk_end) {                                  // uniform over the CTA: the first tile of the next block
             if (cur_block >= 0) flush(cur_block, run_first);
+            const Tile t = tiles[ti];
+            const StatBlock* b = blocks + t.block;
             cur_block = int(t.block);
             run_first = ti;
+            tile0 = b->tile0;                                 // the block's tiles are tile0 + piece, piece = 0, 1, ...
+            blk_end = min64(last, tile0 + b->ntiles);
+            numel = b->numel;
+            v = reinterpret_cast<const uint32_t*>(b->v);
             L = leaders_of(sel + size_t(t.block) * kRanks, kKeyShift);
-            cap = int(min64(last, b->tile0 + b->ntiles) - ti) * kSurvTile;
+            cap = int(blk_end - ti) * kSurvTile;
             surv_run = surv + size_t(ti) * kSurvTile;
             cols_u = uint32_t(b->cols);
             magic = 0xffffffffu / cols_u;
             next_base = -1;
+            if (cols_u > 1u) {
+                rowsum = b->rowsum; colsum = b->colsum;
+                const double total = rowsum[b->rows];         // the block's sum of v, left there by the row/column combine
+                inv_total = total > 0.0 ? 1.0 / total : 0.0;
+            }
         }
-        const int64_t numel = b->numel;
+        const int64_t base = (ti - tile0) * kTile;
         if (cols_u > 1u) {
             if (base == next_base) {                          // the next piece of the same matrix: advance by one tile
                 uint32_t rem;
@@ -522,25 +537,31 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __rest
             }
             next_base = base + kTile;
         }
-        const uint32_t* __restrict__ v = reinterpret_cast<const uint32_t*>(b->v);
+        const bool tile_full = base + kTile <= numel;         // uniform over the CTA
+        const uint32_t* __restrict__ vt = v + base + threadIdx.x * 8;
         uint32_t u[8 * kSl];
         int valid[kSl];
+        if (tile_full) {
 #pragma unroll
-        for (int h = 0; h < kSl; ++h) {                       // v is padded to whole quantisation blocks: in bounds whenever e < numel
-            const int64_t e = base + int64_t(h) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
-            valid[h] = e < numel ? int(min64(8, numel - e)) : 0;
-            uint4 a = make_uint4(0u, 0u, 0u, 0u), c = a;
-            if (valid[h] > 0) { a = ld_stream_u4(v + e); c = ld_stream_u4(v + e + 4); }
-            u[8 * h + 0] = a.x; u[8 * h + 1] = a.y; u[8 * h + 2] = a.z; u[8 * h + 3] = a.w;
-            u[8 * h + 4] = c.x; u[8 * h + 5] = c.y; u[8 * h + 6] = c.z; u[8 * h + 7] = c.w;
+            for (int h = 0; h < kSl; ++h) {
+                const uint4 a = ld_stream_u4(vt + h * (kThreads * 8)), c = ld_stream_u4(vt + h * (kThreads * 8) + 4);
+                valid[h] = 8;
+                u[8 * h + 0] = a.x; u[8 * h + 1] = a.y; u[8 * h + 2] = a.z; u[8 * h + 3] = a.w;
+                u[8 * h + 4] = c.x; u[8 * h + 5] = c.y; u[8 * h + 6] = c.z; u[8 * h + 7] = c.w;
+            }
+        } else {
+#pragma unroll
+            for (int h = 0; h < kSl; ++h) {                   // v is padded to whole quantisation blocks: in bounds whenever e < numel
+                const int64_t e = base + int64_t(h) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+                valid[h] = e < numel ? int(min64(8, numel - e)) : 0;
+                uint4 a = make_uint4(0u, 0u, 0u, 0u), c = a;
+                if (valid[h] > 0) { a = ld_stream_u4(vt + h * (kThreads * 8)); c = ld_stream_u4(vt + h * (kThreads * 8) + 4); }
+                u[8 * h + 0] = a.x; u[8 * h + 1] = a.y; u[8 * h + 2] = a.z; u[8 * h + 3] = a.w;
+                u[8 * h + 4] = c.x; u[8 * h + 5] = c.y; u[8 * h + 6] = c.z; u[8 * h + 7] = c.w;
+            }
         }
-        const bool tile_full = base + kTile <= numel;         // uniform over the CTA
 
         if (cols_u > 1u) {
-            const double* __restrict__ rowsum = b->rowsum;
-            const double* __restrict__ colsum = b->colsum;
-            const double total = rowsum[b->rows];             // the block's sum of v, left there by the row/column combine
-            const double inv_total = total > 0.0 ? 1.0 / total : 0.0;
 #pragma unroll
             for (int h = 0; h < kSl; ++h) {
                 if (valid[h] == 0) continue;
