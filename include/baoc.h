@@ -158,6 +158,9 @@ typedef struct {
     int64_t kernel_launches;      /* kernels this handle has launched so far */
     int64_t stats_bytes_per_call; /* algorithmic HBM bytes of one baoc_sample_stats */
     int64_t step_bytes_per_call;  /* algorithmic HBM bytes of one baoc_step under the assignment */
+    int64_t select_retries;       /* blocks whose quantile select (Eq. 4) the last baoc_risk had to repeat over the
+                                   * full value range because an order statistic lay outside the range of the
+                                   * block's sample; 0 in the usual case */
 } baoc_info_t;
 
 /* Fill *o with the defaults.  Host only. */

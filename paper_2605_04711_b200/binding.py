@@ -81,7 +81,7 @@ class Sample(C.Structure):
 class Info(C.Structure):
     _fields_ = [("n_blocks", C.c_int32), ("n_cfg", C.c_int32), ("numel", C.c_int64), ("n_tiles", C.c_int64),
                 ("stats_steps", C.c_int64), ("state_bytes", C.c_int64), ("kernel_launches", C.c_int64),
-                ("stats_bytes_per_call", C.c_int64), ("step_bytes_per_call", C.c_int64)]
+                ("stats_bytes_per_call", C.c_int64), ("step_bytes_per_call", C.c_int64), ("select_retries", C.c_int64)]
 
 
 EXPORTS = ["baoc_default_opts", "baoc_create", "baoc_destroy", "baoc_last_error", "baoc_query",

@@ -383,7 +383,7 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
         h->launches += 1;
     }
     LAUNCH(launch_final_sums(blocks, tiles, dparams, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<uint32_t>(ws, L.hist),
-                             at<RankSel>(ws, L.sel), h->n_stat_tiles, n, h->opts.eps, float(h->opts.eps_adam),
+                             at<RankSel>(ws, L.sel), at<SelKey>(ws, L.selkey), h->n_stat_tiles, n, h->opts.eps, float(h->opts.eps_adam),
                              h->opts.quantizer8, ws_ctx(h, h->n_stat_tiles), s),
            "final_sums_kernel");
     h->launches += 5;
@@ -393,14 +393,33 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
         h->launches += 3;
     }
     LAUNCH(launch_final_resid_select(blocks, tiles, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<RankSel>(ws, L.sel),
-                                     at<uint32_t>(ws, L.hist), at<uint32_t>(ws, L.surv), at<uint32_t>(ws, L.surv_cnt),
-                                     at<double>(ws, L.acc), h->n_stat_tiles, n, ws_ctx(h, h->n_stat_tiles), s),
+                                     at<SelKey>(ws, L.selkey), at<uint32_t>(ws, L.hist), at<uint32_t>(ws, L.surv),
+                                     at<uint32_t>(ws, L.surv_cnt), at<double>(ws, L.acc), h->n_stat_tiles, n,
+                                     ws_ctx(h, h->n_stat_tiles), s),
            "final_resid_hist_kernel");
     h->launches += 6;
 
     std::vector<double> out(size_t(kFinOut) * n);
     CU(cudaMemcpyAsync(out.data(), ws + L.fin_out, 8 * out.size(), cudaMemcpyDeviceToHost, s), "baoc_risk (copy back)");
     CU(cudaStreamSynchronize(s), "baoc_risk (wait)");
+    // The select orders each block by a key fitted to a sample of it.  A block whose order statistic came out at an end
+    // of that key range holds elements outside the sample's range there: it is selected again over the full range.
+    h->select_retries = 0;
+    h->selkey_staging.assign(size_t(n), SelKey{0, -1});
+    for (int i = 0; i < n; ++i)
+        if (out[size_t(i) * kFinOut + kFinFlag] != 0.0) { h->selkey_staging[i] = SelKey{-1, kSelFullS}; ++h->select_retries; }
+    if (h->select_retries > 0) {
+        CU(cudaMemcpyAsync(ws + L.selkey, h->selkey_staging.data(), sizeof(SelKey) * size_t(n), cudaMemcpyHostToDevice, s),
+           "baoc_risk (select keys)");
+        LAUNCH(launch_select_again(blocks, tiles, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<RankSel>(ws, L.sel),
+                                   at<SelKey>(ws, L.selkey), at<uint32_t>(ws, L.hist), at<uint32_t>(ws, L.surv),
+                                   at<uint32_t>(ws, L.surv_cnt), at<double>(ws, L.acc), h->n_stat_tiles, n,
+                                   ws_ctx(h, h->n_stat_tiles), s),
+               "select_first_kernel");
+        h->launches += 8;
+        CU(cudaMemcpyAsync(out.data(), ws + L.fin_out, 8 * out.size(), cudaMemcpyDeviceToHost, s), "baoc_risk (copy back)");
+        CU(cudaStreamSynchronize(s), "baoc_risk (wait)");
+    }
 
     std::vector<baoc_block_stats_t> tmp;
     baoc_block_stats_t* st = stats_out;

@@ -25,18 +25,54 @@ namespace baoc {
 // ============================================================================
 __device__ __forceinline__ float precond_of(float v, float eps) { return rcp_approx(sqrt_approx(v) + eps); }
 
+// ---- the key of the quantile select (see SelKey) --------------------------------
+// clamp(pattern - lo, 0, wmax) in two instructions; lo >= -1, and a pattern with the sign bit set (no second moment has
+// one) counts as below everything.
+__device__ __forceinline__ uint32_t sel_key(uint32_t pattern, int lo, int wmax) {
+    return uint32_t(min(__viaddmax_s32_relu(int(pattern), -lo, 0), wmax));
+}
+__device__ __forceinline__ int sel_wmax(int s) { return int((uint32_t(kSelBins) << s) - 1u); }
+// lowest bit and width of the digit of pass 0, 1, 2
+__device__ __forceinline__ void sel_digit(int s, int pass, int& shift, int& bits) {
+    const int b2 = s < kSelBits ? s : kSelBits;
+    if (pass == 0) { shift = s; bits = kSelBits; }
+    else if (pass == 1) { shift = s - b2; bits = b2; }
+    else { shift = 0; bits = s - b2; }
+}
+
+// Also the key of the block's select: lo one below the smallest pattern of the sample, s the smallest shift for which
+// the largest pattern of the sample stays below the top of the key range.
 __global__ void __launch_bounds__(kThreads)
-final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, double* __restrict__ fin_out) {
+final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, double* __restrict__ fin_out, SelKey* __restrict__ selkey) {
     __shared__ double total[1];
+    __shared__ int s_min, s_max;
     const StatBlock* b = blocks + blockIdx.x;
     const int64_t numel = b->numel;
     const int64_t n = min64(numel, 1024);
     const int64_t stride = numel / n;
+    if (threadIdx.x == 0) { s_min = 0x7f800000; s_max = 0; }
+    __syncthreads();
     double acc[1] = {0.0};
-    for (int64_t k = threadIdx.x; k < n; k += kThreads) acc[0] += double(precond_of(b->v[k * stride], eps));
+    int lo = 0x7f800000, hi = 0;
+    for (int64_t k = threadIdx.x; k < n; k += kThreads) {
+        const float x = b->v[k * stride];
+        acc[0] += double(precond_of(x, eps));
+        const int pat = min(max(__float_as_int(x), 0), 0x7f800000);
+        lo = min(lo, pat); hi = max(hi, pat);
+    }
+    lo = __reduce_min_sync(0xffffffffu, lo); hi = __reduce_max_sync(0xffffffffu, hi);
+    if ((threadIdx.x & 31) == 0) { atomicMin(&s_min, lo); atomicMax(&s_max, hi); }
     cta_reduce_store<1>(acc, total);
     // n identical fp32 values sum exactly in double, and the correctly rounded quotient is that value again
-    if (threadIdx.x == 0) fin_out[size_t(blockIdx.x) * kFinOut + kFinPilot] = double(float(total[0] / double(n)));
+    if (threadIdx.x == 0) {
+        fin_out[size_t(blockIdx.x) * kFinOut + kFinPilot] = double(float(total[0] / double(n)));
+        SelKey key;
+        key.lo = s_min - 1;
+        const int64_t top = int64_t(s_max) - key.lo + 2;       // the sample's largest key, and one value above it, below wmax
+        key.s = 0;
+        while (key.s < kSelFullS && (int64_t(kSelBins) << key.s) < top) ++key.s;
+        selkey[blockIdx.x] = key;
+    }
 }
 
 // ============================================================================
@@ -92,7 +128,7 @@ __device__ __forceinline__ float rsqrt_approx(float x) {
 template <bool kFull, bool kDyn>
 __device__ __forceinline__ void fs_slice(const float (&mm)[8], const float (&vv)[8], const float (&tt)[8], int cnt,
                                          float p0, float eps_f, float eps_adam, f32x2 (&F)[kFinalSums], uint32_t* hist1,
-                                         const float* dyn) {
+                                         int key_lo, int key_s, const float* dyn) {
     const f32x2 P0 = splat2(p0), MAGIC = splat2(12582912.0f), C16 = splat2(65537.0f), EA = splat2(eps_adam), EPS = splat2(eps_f),
                 ONE = splat2(1.0f), MONE = splat2(-1.0f);
     // ---- absmax of the warp's quantisation block, code scales
@@ -160,20 +196,21 @@ __device__ __forceinline__ void fs_slice(const float (&mm)[8], const float (&vv)
         F[10] = fma2(E0, E0, F[10]); F[11] = fma2(E1, E1, F[11]); F[12] = fma2(E2, E2, F[12]); F[13] = fma2(E3, E3, F[13]);
     }
 
-    // ---- first radix pass of the quantile select: the top 12 bits of v's bit pattern (sign, exponent, three mantissa
-    // bits).  The second moments of a block spread over many of these bins, so a plain shared-memory histogram with one
-    // atomic per element meets few collisions.
+    // ---- first radix pass of the quantile select: the top 12 bits of the block's key (see SelKey).  The key range is
+    // fitted to the block, so its second moments spread over most of the 4096 bins and a plain shared-memory histogram
+    // with one atomic per element meets few collisions.
 #pragma unroll
     for (int j = 0; j < 8; ++j)
-        if (kFull || j < cnt) atomicAdd(hist1 + (__float_as_uint(vv[j]) >> (32 - kSelBits)), 1u);
+        if (kFull || j < cnt)
+            atomicAdd(hist1 + min(__viaddmax_s32_relu(__float_as_int(vv[j]), -key_lo, 0) >> key_s, kSelBins - 1), 1u);
 }
 
 template <bool kDyn>
 __global__ void __launch_bounds__(kThreads, 2)
 final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
                   const float* const* __restrict__ params, double* __restrict__ fin,
-                  const double* __restrict__ fin_out, uint32_t* __restrict__ hist, int64_t n_tiles,
-                  int tiles_per_cta, float eps_f, float eps_adam BAOC_CHECK_PARAM) {
+                  const double* __restrict__ fin_out, uint32_t* __restrict__ hist, const SelKey* __restrict__ selkey,
+                  int64_t n_tiles, int tiles_per_cta, float eps_f, float eps_adam BAOC_CHECK_PARAM) {
 #ifdef BAOC_CHECKED
     {   // validate every tile of this CTA's run, and the ranges of the workspace it will touch, before touching anything
         const int64_t c0 = int64_t(blockIdx.x) * tiles_per_cta, c1 = min64(c0 + tiles_per_cta, n_tiles);
@@ -263,6 +300,7 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
     int cur_block = -1;
     int64_t run_first = first;
     float p0 = 0.f;
+    int key_lo = 0, key_s = 0;
 #pragma unroll 1
     for (int k = 0; k < nsl; ++k) {
         prefetch(k + kFsStages - 1);
@@ -274,6 +312,8 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
             cur_block = int(t.block);
             run_first = ti;
             p0 = float(fin_out[size_t(t.block) * kFinOut + kFinPilot]);
+            const SelKey key = selkey[t.block];
+            key_lo = key.lo; key_s = key.s;
         }
         const unsigned char* mine = stage + take;
         take = take == (kFsStages - 1) * kFsStageBytes ? 0u : take + kFsStageBytes;
@@ -285,7 +325,7 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
         f4_to8(*reinterpret_cast<const float4*>(mine + ov), *reinterpret_cast<const float4*>(mine + ov + kHalf), vv);
         if (w0 + kQBlock <= numel) {                         // uniform over the warp
             f4_to8(*reinterpret_cast<const float4*>(mine + ot), *reinterpret_cast<const float4*>(mine + ot + kHalf), tt);
-            fs_slice<true, kDyn>(mm, vv, tt, 8, p0, eps_f, eps_adam, F, hist1, dyn_tables);
+            fs_slice<true, kDyn>(mm, vv, tt, 8, p0, eps_f, eps_adam, F, hist1, key_lo, key_s, dyn_tables);
         } else {
             const int64_t e = w0 + lane * 8;
             const int cnt = int(max64(0, min64(8, numel - e)));
@@ -296,7 +336,7 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
 #pragma unroll
                 for (int j = 0; j < 8; ++j) tt[j] = j < cnt ? th[e + j] : 0.f;
             }
-            fs_slice<false, kDyn>(mm, vv, tt, cnt, p0, eps_f, eps_adam, F, hist1, dyn_tables);
+            fs_slice<false, kDyn>(mm, vv, tt, cnt, p0, eps_f, eps_adam, F, hist1, key_lo, key_s, dyn_tables);
         }
     }
     cp_async_wait<0>();
@@ -394,13 +434,15 @@ __device__ __forceinline__ Leaders leaders_of(const RankSel* __restrict__ sel, i
     return L;
 }
 
-// bit j set: element j of the thread (8 h + i: slice h, element i) is in range and its key is a leader's
-template <int kL, bool kFull, int kKeyShift>
-__device__ __forceinline__ uint32_t match_mask(const uint32_t (&u)[16], const int (&valid)[2], const Leaders& L) {
+// Replaces the thread's 16 patterns by their keys; bit j of the result set: element j (8 h + i: slice h, element i) is
+// in range and the resolved part of its key is a leader's.
+template <int kL, bool kFull>
+__device__ __forceinline__ uint32_t match_mask(uint32_t (&u)[16], const int (&valid)[2], const Leaders& L, int lo, int wmax, int s) {
     uint32_t mask = 0u;
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-        const uint32_t key = u[j] >> kKeyShift;
+        u[j] = sel_key(u[j], lo, wmax);
+        const uint32_t key = u[j] >> s;
         bool p = (key == L.key[0]) | (key == L.key[1]);
         if (kL > 2) p |= (key == L.key[2]) | (key == L.key[3]);
         if (!kFull) p &= (j & 7) < valid[j >> 3];
@@ -411,8 +453,9 @@ __device__ __forceinline__ uint32_t match_mask(const uint32_t (&u)[16], const in
 
 __global__ void __launch_bounds__(kThreads, 3)
 final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const RankSel* __restrict__ sel,
-                        double* __restrict__ fin, uint32_t* __restrict__ hist, uint32_t* __restrict__ surv,
-                        uint32_t* __restrict__ surv_cnt, int64_t n_tiles, int tiles_per_cta BAOC_CHECK_PARAM) {
+                        const SelKey* __restrict__ selkey, double* __restrict__ fin, uint32_t* __restrict__ hist,
+                        uint32_t* __restrict__ surv, uint32_t* __restrict__ surv_cnt, int64_t n_tiles, int tiles_per_cta,
+                        int with_resid BAOC_CHECK_PARAM) {
 #ifdef BAOC_CHECKED
     {
         const int64_t c0 = int64_t(blockIdx.x) * tiles_per_cta, c1 = min64(c0 + tiles_per_cta, n_tiles);
@@ -441,13 +484,13 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __rest
     uint32_t* stage = reinterpret_cast<uint32_t*>(dyn + kRhHistBytes);
     __shared__ int wcnt[kThreads / 32];                       // survivors a warp has staged of its current tile
     __shared__ int run_cnt, run_over;                         // survivors of the run written so far; the run outgrew its slots
-    constexpr int kKeyShift = 32 - kSelBits;                  // the first digit
     constexpr int kSl = kTile / (kThreads * 8);
     static_assert(kSl == 2, "a tile is two slices of eight elements per thread");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
     Leaders L;
     L.n = 0;
+    int key_lo = 0, key_s = -1, key_max = 0, d_shift = 0, d_bits = 0;   // the block's key; this pass's digit (s < 0: the block sits this round out)
     // what the tiles of one block share, fetched once when the CTA enters the block (nothing a tile needs then hangs on
     // a chain of dependent loads): its extent in the tile table, v, the row/column sums, 1 / total
     int cur_block = -1;
@@ -466,15 +509,20 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __rest
     int64_t next_base = -1;
 
     auto flush = [&](int blk, int64_t t_begin) {
-        cta_reduce_store<kResidSums>(acc, fin + size_t(t_begin) * kResidSums);   // (every warp has drained its last tile)
-        acc[0] = 0.0;
-        if (threadIdx.x == 0) {
+        if (key_s < 0) return;                                // uniform over the CTA: nothing was done for this block
+        if (with_resid) {
+            cta_reduce_store<kResidSums>(acc, fin + size_t(t_begin) * kResidSums);
+            acc[0] = 0.0;
+        } else {
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) {                               // (every warp has drained its last tile)
             surv_cnt[t_begin] = run_over ? kSurvOverflow : uint32_t(run_cnt);
             run_cnt = 0; run_over = 0;
         }
 #pragma unroll
         for (int k = 0; k < kRanks; ++k) {
-            if (k >= L.n) continue;                           // uniform over the CTA
+            if (k >= L.n || d_bits == 0) continue;            // uniform over the CTA
             uint32_t* out = hist + (size_t(blk) * kRanks + L.slot[k]) * kSelBins;
             for (int w = threadIdx.x; w < kRhHistWords; w += kThreads) {
                 const uint32_t x = sh[k][w];
@@ -513,10 +561,13 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __rest
             blk_end = min64(last, tile0 + b->ntiles);
             numel = b->numel;
             v = reinterpret_cast<const uint32_t*>(b->v);
-            L = leaders_of(sel + size_t(t.block) * kRanks, kKeyShift);
+            const SelKey key = selkey[t.block];
+            key_lo = key.lo; key_s = key.s; key_max = sel_wmax(max(key.s, 0));
+            sel_digit(key.s, 1, d_shift, d_bits);
+            L = leaders_of(sel + size_t(t.block) * kRanks, max(key.s, 0));
             cap = int(blk_end - ti) * kSurvTile;
             surv_run = surv + size_t(ti) * kSurvTile;
-            cols_u = uint32_t(b->cols);
+            cols_u = with_resid ? uint32_t(b->cols) : 1u;
             magic = 0xffffffffu / cols_u;
             next_base = -1;
             if (cols_u > 1u) {
@@ -525,6 +576,7 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __rest
                 inv_total = total > 0.0 ? 1.0 / total : 0.0;
             }
         }
+        if (key_s < 0) continue;                              // uniform over the CTA
         const int64_t base = (ti - tile0) * kTile;
         if (cols_u > 1u) {
             if (base == next_base) {                          // the next piece of the same matrix: advance by one tile
@@ -592,58 +644,58 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __rest
         }
 
         // ---- the survivors of this tile: noted, staged by warp, counted, listed
+        if (d_bits == 0) continue;                            // uniform over the CTA: the first pass resolved the whole key
         uint32_t mask;
-        if (tile_full) mask = L.n <= 2 ? match_mask<2, true, kKeyShift>(u, valid, L) : match_mask<4, true, kKeyShift>(u, valid, L);
-        else mask = match_mask<4, false, kKeyShift>(u, valid, L);
+        if (tile_full) mask = L.n <= 2 ? match_mask<2, true>(u, valid, L, key_lo, key_max, key_s) : match_mask<4, true>(u, valid, L, key_lo, key_max, key_s);
+        else mask = match_mask<4, false>(u, valid, L, key_lo, key_max, key_s);
+        if (!__any_sync(0xffffffffu, mask != 0u)) continue;   // the usual case: a bin of the first digit holds few elements
         uint32_t* seg = stage + warp * kRhSegWords;
-        const int mine = __popc(mask);
-        int pos = mine ? atomicAdd(&wcnt[warp], mine) : 0;
+        const int found = __popc(mask);
+        int pos = found ? atomicAdd(&wcnt[warp], found) : 0;
 #pragma unroll
         for (int j = 0; j < 8 * kSl; ++j)
             if (mask & (1u << j)) seg[pos++] = u[j];
         __syncwarp();
         const int staged = wcnt[warp];                        // uniform over the warp
-        if (staged > 0) {
-            int off = 0;
-            if (lane == 0) {
-                off = atomicAdd(&run_cnt, staged);
-                if (off + staged > cap) run_over = 1;
-            }
-            off = __shfl_sync(0xffffffffu, off, 0);
-            const bool fits = off + staged <= cap;
-            for (int i0 = 0; i0 < staged; i0 += 32) {
-                const int i = i0 + lane;
-                const bool on = i < staged;
-                const unsigned act = __ballot_sync(0xffffffffu, on);
-                if (on) {
-                    const uint32_t x = seg[i];
-                    if (fits) surv_run[off + i] = x;
-                    const unsigned same = __match_any_sync(act, x);
-                    if (lane == __ffs(int(same)) - 1) {       // one lane per distinct value adds for all of them
-                        const uint32_t key = x >> kKeyShift, d = (x >> kSel3Bits) & uint32_t(kSelBins - 1);
-                        const uint32_t n = uint32_t(__popc(same)) << ((d & 1u) * 16u);
+        int off = 0;
+        if (lane == 0) {
+            off = atomicAdd(&run_cnt, staged);
+            if (off + staged > cap) run_over = 1;
+        }
+        off = __shfl_sync(0xffffffffu, off, 0);
+        const bool fits = off + staged <= cap;
+        for (int i0 = 0; i0 < staged; i0 += 32) {
+            const int i = i0 + lane;
+            const bool on = i < staged;
+            const unsigned act = __ballot_sync(0xffffffffu, on);
+            if (on) {
+                const uint32_t x = seg[i];
+                if (fits) surv_run[off + i] = x;
+                const unsigned same = __match_any_sync(act, x);
+                if (lane == __ffs(int(same)) - 1) {           // one lane per distinct key adds for all of them
+                    const uint32_t key = x >> key_s, d = (x >> d_shift) & ((1u << d_bits) - 1u);
+                    const uint32_t n = uint32_t(__popc(same)) << ((d & 1u) * 16u);
 #pragma unroll
-                        for (int k = 0; k < kRanks; ++k)
-                            if (key == L.key[k]) atomicAdd(&sh[k][d >> 1], n);
-                    }
+                    for (int k = 0; k < kRanks; ++k)
+                        if (key == L.key[k]) atomicAdd(&sh[k][d >> 1], n);
                 }
             }
-            __syncwarp();
-            if (lane == 0) wcnt[warp] = 0;
-            __syncwarp();
         }
+        __syncwarp();
+        if (lane == 0) wcnt[warp] = 0;
+        __syncwarp();
     }
     if (cur_block >= 0) flush(cur_block, run_first);
 }
 
-// Sweep 3: the last 8 bits.  Same partition of the tiles into runs as sweep 2; per run either its survivors list or, for
+// Sweep 3: the last bits of the key (at most 7).  Same partition of the tiles into runs as sweep 2; per run either its survivors list or, for
 // a run that was marked, the tiles of v themselves.  The histogram (256 bins of 32 bits per leader) is handed over per run.
 constexpr int kLastBins = 1 << kSel3Bits;
 
 __global__ void __launch_bounds__(kThreads)
 final_last_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const RankSel* __restrict__ sel,
-                  uint32_t* __restrict__ hist, const uint32_t* __restrict__ surv, const uint32_t* __restrict__ surv_cnt,
-                  int64_t n_tiles, int tiles_per_cta BAOC_CHECK_PARAM) {
+                  const SelKey* __restrict__ selkey, uint32_t* __restrict__ hist, const uint32_t* __restrict__ surv,
+                  const uint32_t* __restrict__ surv_cnt, int64_t n_tiles, int tiles_per_cta BAOC_CHECK_PARAM) {
     __shared__ uint32_t sh[kRanks][kLastBins];
     const int lane = threadIdx.x & 31;
     const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
@@ -653,11 +705,11 @@ final_last_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
     for (int i = threadIdx.x; i < kRanks * kLastBins; i += kThreads) (&sh[0][0])[i] = 0u;
     __syncthreads();
 
-    // one lane per distinct value among the lanes `act` adds for all of them
-    auto count_same = [&](unsigned act, uint32_t x, const Leaders& L) {
+    // one lane per distinct key among the lanes `act` adds for all of them
+    auto count_same = [&](unsigned act, uint32_t x, const Leaders& L, int bits) {
         const unsigned same = __match_any_sync(act, x);
         if (lane == __ffs(int(same)) - 1) {
-            const uint32_t key = x >> kSel3Bits, d = x & uint32_t(kLastBins - 1);
+            const uint32_t key = x >> bits, d = x & ((1u << bits) - 1u);
 #pragma unroll
             for (int k = 0; k < kRanks; ++k)
                 if (key == L.key[k]) atomicAdd(&sh[k][d], uint32_t(__popc(same)));
@@ -672,7 +724,11 @@ final_last_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
 #endif
         const StatBlock* b = blocks + t.block;
         const int64_t t_end = min64(last, b->tile0 + b->ntiles);     // the run: this CTA's tiles of the block
-        const Leaders L = leaders_of(sel + size_t(t.block) * kRanks, kSel3Bits);
+        const SelKey key = selkey[t.block];
+        int d_shift, d_bits;
+        sel_digit(key.s, 2, d_shift, d_bits);
+        if (key.s < 0 || d_bits == 0) { t_begin = t_end; continue; }   // uniform over the CTA: not in this round, or nothing left to find
+        const Leaders L = leaders_of(sel + size_t(t.block) * kRanks, d_bits);
         const uint32_t cnt = surv_cnt[t_begin];
 #ifdef BAOC_CHECKED
         if (!check_range(ck, kKerFinalLast, surv_cnt + t_begin, 4, 0) ||
@@ -688,7 +744,7 @@ final_last_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
                 const uint32_t i = i0 + threadIdx.x;
                 const bool on = i < cnt;
                 const unsigned act = __ballot_sync(0xffffffffu, on);
-                if (on) count_same(act, list[i], L);
+                if (on) count_same(act, list[i], L, d_bits);
             }
         } else {
             const uint32_t* __restrict__ v = reinterpret_cast<const uint32_t*>(b->v);
@@ -702,12 +758,12 @@ final_last_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
                 uint32_t x = 0u;
                 bool hit = false;
                 if (on) {
-                    x = v[i];
-                    const uint32_t key = x >> kSel3Bits;
-                    hit = (key == L.key[0]) | (key == L.key[1]) | (key == L.key[2]) | (key == L.key[3]);
+                    x = sel_key(v[i], key.lo, sel_wmax(key.s));
+                    const uint32_t upper = x >> d_bits;
+                    hit = (upper == L.key[0]) | (upper == L.key[1]) | (upper == L.key[2]) | (upper == L.key[3]);
                 }
                 const unsigned act = __ballot_sync(0xffffffffu, hit);
-                if (hit) count_same(act, x, L);
+                if (hit) count_same(act, x, L, d_bits);
             }
         }
         __syncthreads();
@@ -726,15 +782,20 @@ final_last_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
 }
 
 // One CTA per block: for each of the four ranks find the bin of its leader's
-// histogram that holds the rank (a scan over the CTA), extend the prefix,
-// recompute which ranks still share a prefix, and clear the histograms for the
-// next pass.
+// histogram that holds the rank (a scan over the CTA), extend the prefix by this
+// pass's digit, recompute which ranks still share a prefix, and clear the
+// histograms for the next pass.
 __global__ void __launch_bounds__(kThreads)
-select_pick_kernel(RankSel* __restrict__ sel, uint32_t* __restrict__ hist, int shift, int bins) {
+select_pick_kernel(RankSel* __restrict__ sel, uint32_t* __restrict__ hist, const SelKey* __restrict__ selkey, int pass) {
     __shared__ unsigned long long warp_tot[kThreads / 32];
     __shared__ int res_d[kRanks];
     __shared__ long long res_rem[kRanks];
     const int blk = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const SelKey key = selkey[blk];
+    int shift, bits;
+    sel_digit(key.s, pass, shift, bits);
+    if (key.s < 0 || bits == 0) return;                       // uniform over the CTA: not in this round, or no digit left (nothing was counted)
+    const int bins = pass < 2 ? kSelBins : kLastBins;
     RankSel s[kRanks];
 #pragma unroll
     for (int r = 0; r < kRanks; ++r) s[r] = sel[size_t(blk) * kRanks + r];
@@ -786,9 +847,10 @@ select_pick_kernel(RankSel* __restrict__ sel, uint32_t* __restrict__ hist, int s
 }
 
 // Start of a select: ranks floor(q (n-1)) and the next one for q = 0.1, 0.9; all four share the empty prefix.
-__global__ void select_init_kernel(const StatBlock* __restrict__ blocks, RankSel* __restrict__ sel, int n_blocks) {
+__global__ void select_init_kernel(const StatBlock* __restrict__ blocks, RankSel* __restrict__ sel,
+                                   const SelKey* __restrict__ selkey, int n_blocks) {
     const int blk = blockIdx.x * blockDim.x + threadIdx.x;
-    if (blk >= n_blocks) return;
+    if (blk >= n_blocks || (selkey != nullptr && selkey[blk].s < 0)) return;
     const int64_t n = blocks[blk].numel;
     const double qs[2] = {0.1, 0.9};
     for (int k = 0; k < 2; ++k) {
@@ -802,14 +864,56 @@ __global__ void select_init_kernel(const StatBlock* __restrict__ blocks, RankSel
 
 // End of the window: gather what the host needs into fin_out[block]:
 //   [0..15] sweep-1 sums, [16..19] the four order statistics (as doubles),
-//   [20..27] the running window values, [28] the Eq. 7 numerator, [29] the pilot value.
-__global__ void stats_gather_kernel(const RankSel* __restrict__ sel, const double* __restrict__ acc,
-                                    double* __restrict__ fin_out, int n_blocks) {
+//   [20..27] the running window values, [28] the Eq. 7 numerator, [29] the pilot value,
+//   [30] whether an order statistic came out at an end of the key range (a clamped element: to be found again).
+__global__ void stats_gather_kernel(const RankSel* __restrict__ sel, const SelKey* __restrict__ selkey,
+                                    const double* __restrict__ acc, double* __restrict__ fin_out, int n_blocks) {
     const int blk = blockIdx.x * blockDim.x + threadIdx.x;
     if (blk >= n_blocks) return;
+    const SelKey key = selkey[blk];
+    if (key.s < 0) return;
     double* o = fin_out + size_t(blk) * kFinOut;
-    for (int r = 0; r < kRanks; ++r) o[kFinRanks + r] = double(__uint_as_float(sel[size_t(blk) * kRanks + r].prefix));
+    const uint32_t wmax = uint32_t(sel_wmax(key.s));
+    bool clamped = false;
+    for (int r = 0; r < kRanks; ++r) {
+        const uint32_t w = sel[size_t(blk) * kRanks + r].prefix;
+        clamped |= w == 0u || w == wmax;
+        o[kFinRanks + r] = double(__int_as_float(int(w) + key.lo));
+    }
+    o[kFinFlag] = clamped ? 1.0 : 0.0;
     for (int k = 0; k < kBlockAcc; ++k) o[kFinAcc + k] = acc[size_t(blk) * kBlockAcc + k];
+}
+
+// First pass of the select on its own (the first sweep does it for the first round): the top 12 bits of the key of
+// every element of the blocks that take part.
+__global__ void __launch_bounds__(kThreads)
+select_first_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const SelKey* __restrict__ selkey,
+                    uint32_t* __restrict__ hist, int64_t n_tiles, int tiles_per_cta) {
+    __shared__ uint32_t sh[kSelBins];
+    const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
+    for (int i = threadIdx.x; i < kSelBins; i += kThreads) sh[i] = 0u;
+    __syncthreads();
+#pragma unroll 1
+    for (int64_t t_begin = first; t_begin < last;) {
+        const Tile t = tiles[t_begin];
+        const StatBlock* b = blocks + t.block;
+        const int64_t t_end = min64(last, b->tile0 + b->ntiles);
+        const SelKey key = selkey[t.block];
+        if (key.s >= 0) {                                     // uniform over the CTA
+            const uint32_t* __restrict__ v = reinterpret_cast<const uint32_t*>(b->v);
+            const int64_t e0 = int64_t(t.piece) * kTile, e1 = min64(b->numel, e0 + (t_end - t_begin) * int64_t(kTile));
+            const int wmax = sel_wmax(key.s);
+            for (int64_t i = e0 + threadIdx.x; i < e1; i += kThreads) atomicAdd(&sh[sel_key(v[i], key.lo, wmax) >> key.s], 1u);
+            __syncthreads();
+            uint32_t* out = hist + size_t(t.block) * kRanks * kSelBins;          // all four ranks still share one histogram
+            for (int d = threadIdx.x; d < kSelBins; d += kThreads) {
+                const uint32_t c = sh[d];
+                if (c) { atomicAdd(out + d, c); sh[d] = 0u; }
+            }
+            __syncthreads();
+        }
+        t_begin = t_end;
+    }
 }
 
 // ---- launchers ------------------------------------------------------------------
@@ -828,15 +932,15 @@ static int run_tiles(int64_t n_tiles, int most) {
 }
 
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
-                      double* fin_out, uint32_t* hist, RankSel* sel, int64_t n_tiles, int n_blocks, double eps,
+                      double* fin_out, uint32_t* hist, RankSel* sel, SelKey* selkey, int64_t n_tiles, int n_blocks, double eps,
                       float eps_adam, int quantizer8, const CheckCtx& ck, cudaStream_t s) {
     (void)ck;
     const int tb = 128, gb = (n_blocks + tb - 1) / tb;
     cudaError_t e = cudaMemsetAsync(hist, 0, size_t(n_blocks) * kRanks * kSelBins * sizeof(uint32_t), s);
     if (e != cudaSuccess) return int(e);
-    select_init_kernel<<<gb, tb, 0, s>>>(blocks, sel, n_blocks);
+    select_init_kernel<<<gb, tb, 0, s>>>(blocks, sel, nullptr, n_blocks);
     BAOC_LAUNCH_CHECK();
-    final_pilot_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, float(eps), fin_out);
+    final_pilot_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, float(eps), fin_out, selkey);
     BAOC_LAUNCH_CHECK();
     e = cudaFuncSetAttribute(final_sums_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(final_sums_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes);
@@ -844,42 +948,66 @@ int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* c
     const int per = run_tiles(n_tiles, kFinRunTiles);
     const unsigned grid = unsigned((n_tiles + per - 1) / per);
     if (quantizer8)
-        final_sums_kernel<true><<<grid, kThreads, kFsSmemBytes, s>>>(blocks, tiles, params, fin, fin_out, hist, n_tiles, per,
-                                                                       float(eps), eps_adam BAOC_CHECK_ARG(ck));
+        final_sums_kernel<true><<<grid, kThreads, kFsSmemBytes, s>>>(blocks, tiles, params, fin, fin_out, hist, selkey, n_tiles,
+                                                                       per, float(eps), eps_adam BAOC_CHECK_ARG(ck));
     else
-        final_sums_kernel<false><<<grid, kThreads, kFsSmemBytes, s>>>(blocks, tiles, params, fin, fin_out, hist, n_tiles, per,
-                                                                        float(eps), eps_adam BAOC_CHECK_ARG(ck));
+        final_sums_kernel<false><<<grid, kThreads, kFsSmemBytes, s>>>(blocks, tiles, params, fin, fin_out, hist, selkey, n_tiles,
+                                                                        per, float(eps), eps_adam BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     final_sums_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
     BAOC_LAUNCH_CHECK();
-    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, 32 - kSelBits, kSelBins);
+    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, selkey, 0);
     BAOC_LAUNCH_CHECK();
     return 0;
 }
 
-int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                              uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc, int64_t n_tiles,
-                              int n_blocks, const CheckCtx& ck, cudaStream_t s) {
+// The second and third pass of the select (with the Eq. 7 residual in the second sweep if with_resid), and the gather.
+static int select_rest(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
+                       const SelKey* selkey, uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc,
+                       int64_t n_tiles, int n_blocks, int with_resid, const CheckCtx& ck, cudaStream_t s) {
     (void)ck;
     cudaError_t e = cudaFuncSetAttribute(final_resid_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRhSmemBytes);
     if (e != cudaSuccess) return int(e);
     const int per = run_tiles(n_tiles, kSelRunTiles);
     const unsigned grid = unsigned((n_tiles + per - 1) / per);
-    final_resid_hist_kernel<<<grid, kThreads, kRhSmemBytes, s>>>(blocks, tiles, sel, fin, hist, surv, surv_cnt, n_tiles,
-                                                                per BAOC_CHECK_ARG(ck));
+    final_resid_hist_kernel<<<grid, kThreads, kRhSmemBytes, s>>>(blocks, tiles, sel, selkey, fin, hist, surv, surv_cnt, n_tiles,
+                                                                per, with_resid BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
-    final_resid_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
+    if (with_resid) {
+        final_resid_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
+        BAOC_LAUNCH_CHECK();
+    }
+    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, selkey, 1);
     BAOC_LAUNCH_CHECK();
-    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, kSel3Bits, kSelBins);
+    final_last_kernel<<<grid, kThreads, 0, s>>>(blocks, tiles, sel, selkey, hist, surv, surv_cnt, n_tiles, per BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
-    final_last_kernel<<<grid, kThreads, 0, s>>>(blocks, tiles, sel, hist, surv, surv_cnt, n_tiles, per BAOC_CHECK_ARG(ck));
-    BAOC_LAUNCH_CHECK();
-    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, 0, 1 << kSel3Bits);
+    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, selkey, 2);
     BAOC_LAUNCH_CHECK();
     const int tb = 128, gb = (n_blocks + tb - 1) / tb;
-    stats_gather_kernel<<<gb, tb, 0, s>>>(sel, acc, fin_out, n_blocks);
+    stats_gather_kernel<<<gb, tb, 0, s>>>(sel, selkey, acc, fin_out, n_blocks);
     BAOC_LAUNCH_CHECK();
     return 0;
+}
+
+int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
+                              const SelKey* selkey, uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc,
+                              int64_t n_tiles, int n_blocks, const CheckCtx& ck, cudaStream_t s) {
+    return select_rest(blocks, tiles, fin, fin_out, sel, selkey, hist, surv, surv_cnt, acc, n_tiles, n_blocks, 1, ck, s);
+}
+
+int launch_select_again(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
+                        const SelKey* selkey, uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc,
+                        int64_t n_tiles, int n_blocks, const CheckCtx& ck, cudaStream_t s) {
+    const int tb = 128, gb = (n_blocks + tb - 1) / tb;
+    select_init_kernel<<<gb, tb, 0, s>>>(blocks, sel, selkey, n_blocks);
+    BAOC_LAUNCH_CHECK();
+    const int per = run_tiles(n_tiles, kSelRunTiles);
+    const unsigned grid = unsigned((n_tiles + per - 1) / per);
+    select_first_kernel<<<grid, kThreads, 0, s>>>(blocks, tiles, selkey, hist, n_tiles, per);
+    BAOC_LAUNCH_CHECK();
+    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, selkey, 0);
+    BAOC_LAUNCH_CHECK();
+    return select_rest(blocks, tiles, fin, fin_out, sel, selkey, hist, surv, surv_cnt, acc, n_tiles, n_blocks, 0, ck, s);
 }
 
 }  // namespace baoc

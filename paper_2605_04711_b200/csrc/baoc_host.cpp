@@ -140,6 +140,7 @@ void compute_stat_layout(Handle* h) {
     L.fin_out = take(&cur, 8 * size_t(kFinOut) * n);
     L.hist = take(&cur, 4 * size_t(kSelBins) * kRanks * n);
     L.sel = take(&cur, sizeof(RankSel) * size_t(kRanks) * n);
+    L.selkey = take(&cur, sizeof(SelKey) * size_t(n));
     L.surv = take(&cur, 4 * size_t(kSurvTile) * size_t(tiles));
     L.surv_cnt = take(&cur, 4 * size_t(tiles));
     L.rowsum = take(&cur, 8 * size_t(std::max<int64_t>(sum_rows, 1)));
@@ -627,6 +628,7 @@ int baoc_query(const baoc_t* h, baoc_info_t* info) {
     info->n_tiles = h->n_stat_tiles; info->stats_steps = h->stats_steps;
     info->state_bytes = h->configured ? h->state_mem : 0;
     info->kernel_launches = h->launches;
+    info->select_retries = h->select_retries;
     {   // g_t, g_{t-1}, m, v read; m, v, g_{t-1} written, over what the statistics see (+ the gather of a sample)
         int64_t seen = 0;
         for (const baoc_block_t& b : (h->sampled ? h->stat_shapes : h->blocks)) seen += b.numel;

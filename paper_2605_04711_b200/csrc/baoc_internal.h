@@ -34,7 +34,8 @@ constexpr int kFinOut = 32;           // doubles per block copied to the host at
 constexpr int kFinRanks = 16;         //   [0..15] first-sweep sums, [16..19] the four order statistics,
 constexpr int kFinAcc = 20;           //   [20..27] the running window values,
 constexpr int kFinResid = 28;         //   [28] the Eq. 7 numerator,
-constexpr int kFinPilot = 29;         //   [29] the pilot value of the Eq. 6 preconditioner
+constexpr int kFinPilot = 29;         //   [29] the pilot value of the Eq. 6 preconditioner,
+constexpr int kFinFlag = 30;          //   [30] non-zero: an order statistic lies outside the key range of the select
 constexpr int kSelBits = 12;          // bits of the first and of the second radix pass of the quantile select
 constexpr int kSelBins = 1 << kSelBits;
 constexpr int kSel3Bits = 32 - 2 * kSelBits;   // bits of the third and last pass
@@ -204,6 +205,18 @@ struct RankSel {
     int64_t remaining;
 };
 
+// The key the select orders a block's second moments by: w = clamp(pattern - lo, 0, (4096 << s) - 1) for the fp32 bit
+// pattern of an element (v >= 0, so patterns order like values): 12 + s bits, found in passes of 12, min(12, s) and
+// s - 12 bits.  lo and s come from the smallest and largest pattern of a sample of the block, so that the first digit
+// already spreads the block over most of its 4096 bins; an order statistic that comes out at either end of the key
+// range (an element outside the sample's range) is found again with lo = -1, s = 19, which covers every finite value.
+// s < 0: the block takes no part in this round of the select.
+struct SelKey {
+    int32_t lo;
+    int32_t s;
+};
+constexpr int kSelFullS = 31 - kSelBits;   // with lo = -1 the key pattern + 1 of every finite non-negative value fits
+
 // One CTA of the row/column reduction: a kRedRows x kRedCols piece of a matrix block.
 struct RedTile {
     uint32_t block;
@@ -263,8 +276,10 @@ struct Handle {
     std::vector<const void*> sample_tables;
     std::vector<const void*> last_stat_grads;
     std::vector<const void*> last_stat_params;
+    std::vector<SelKey> selkey_staging;                    // keys of a repeated select (must outlive the async copy)
+    int64_t select_retries = 0;                            // blocks whose select was repeated in the last baoc_risk
     struct StatLayout {
-        size_t blocks, tiles, red_tiles, matrix_ids, grads, params, m, v, gprev, partials, acc, fin, fin_out, hist, sel, surv, surv_cnt,
+        size_t blocks, tiles, red_tiles, matrix_ids, grads, params, m, v, gprev, partials, acc, fin, fin_out, hist, sel, selkey, surv, surv_cnt,
                rowsum, colsum, redpart, ridx, cidx, gsample, psample, sgrads, sparams, total;
     } sl{};
 
@@ -348,11 +363,15 @@ int launch_stats_combine(const StatBlock* blocks, const double* partials, double
 // First finalize sweep (with the pilot values, the start of the select and its first radix pass), then, after the
 // row/column sums of the matrix blocks, the second and third sweep and the gather of the per-block results.
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
-                      double* fin_out, uint32_t* hist, RankSel* sel, int64_t n_tiles, int n_blocks, double eps,
+                      double* fin_out, uint32_t* hist, RankSel* sel, SelKey* selkey, int64_t n_tiles, int n_blocks, double eps,
                       float eps_adam, int quantizer8, const CheckCtx& ck, cudaStream_t s);
 int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                              uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc, int64_t n_tiles,
-                              int n_blocks, const CheckCtx& ck, cudaStream_t s);
+                              const SelKey* selkey, uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc,
+                              int64_t n_tiles, int n_blocks, const CheckCtx& ck, cudaStream_t s);
+// The select once more, from its first pass, for the blocks whose selkey has s >= 0 (the others keep their results).
+int launch_select_again(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
+                        const SelKey* selkey, uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc,
+                        int64_t n_tiles, int n_blocks, const CheckCtx& ck, cudaStream_t s);
 int launch_sample_gather(const StatBlock* blocks, const Tile* tiles, const void* const* src, int64_t n_tiles, int fp32,
                          const CheckCtx& ck, cudaStream_t s);
 int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const int32_t* ids, int64_t n_red, int n_matrix,

@@ -138,6 +138,7 @@ def test_stats_window_odd_sizes(B, H):
     _check_stats(sess, states)
     info = sess.h.query()
     assert info.stats_steps == wl.window and info.kernel_launches > 0
+    assert info.select_retries == 0                                 # every quantile lay inside its block's sampled range
 
 
 def test_finalize_from_shared_moments_holds_every_diagnostic_to_1e_4(B, H):
@@ -202,6 +203,49 @@ def test_stats_invariants_identical_zero_and_flipped_gradients(B, H):
         assert abs(st2[i]["C"]) < 1e-9                               # constant preconditioner: no distortion
         if wl2.blocks[i].cols > 1:
             assert st2[i]["F"] < 1e-6                                # constant matrix is rank one
+
+
+def test_quantile_select_repeats_over_the_full_range_when_the_sample_misses_the_tails(B, H):
+    """The select orders a block by a key fitted to 1024 evenly spaced elements of it.  Here those elements all lie in
+    [1, 2) while 30 % of the others are a million times smaller and 20 % a thousand times larger, so both quantiles of
+    Eq. 4 fall outside the fitted range: the library must notice (an order statistic at an end of the key range) and
+    find them again over the full range.  Moments are written oracle -> device, as in the shared-state test."""
+    wl = _odd_workload(seed=12, window=3)
+    sess = H.Session(wl, n_grad_sets=2)
+    sess.init_params()
+    o = O.Opts()
+    states = _oracle_window(sess, wl.window, o)
+    rng = np.random.default_rng(5)
+    crafted = [5, 9, 10, 14]                                        # (4097,), (300, 520), (5000, 8), (8200,)
+    for i, b in enumerate(wl.blocks):
+        states[i].m = states[i].m.astype(np.float32).astype(np.float64)
+        v = states[i].v.astype(np.float32).astype(np.float64)
+        if i in crafted:
+            n = b.numel
+            v = rng.uniform(1.0, 2.0, n)
+            kind = rng.uniform(0.0, 1.0, n)
+            v[kind < 0.3] *= 1e-6
+            v[kind > 0.8] *= 1e3
+            stride = n // min(n, 1024)
+            seen = np.arange(min(n, 1024)) * stride
+            v[seen] = rng.uniform(1.0, 2.0, seen.size)
+            v = v.astype(np.float32).astype(np.float64)
+        states[i].v = v
+        sess.h.view_tensor(i, 0, torch.float32).copy_(torch.from_numpy(states[i].m.astype(np.float32)).to(sess.device))
+        sess.h.view_tensor(i, 1, torch.float32).copy_(torch.from_numpy(states[i].v.astype(np.float32)).to(sess.device))
+    _, st = sess.risk()
+    assert sess.h.query().select_retries == len(crafted)
+    for i, b in enumerate(wl.blocks):
+        raw = O.stats_finalize(states[i], sess.block_param_host(i), b.rows, b.cols, o)
+        for k in ("A", "q10", "q90"):
+            assert abs(st[i][k] - raw[k]) <= 1e-6 * max(abs(raw[k]), 1e-30), (b.name, k, st[i][k], raw[k])
+        for k in STAT_KEYS:
+            if k in ("rho_bar", "rho_mom"):
+                continue
+            assert abs(st[i][k] - raw[k]) <= 1e-4 * max(abs(raw[k]), 1e-3), (b.name, k, st[i][k], raw[k])
+    _, st2 = sess.risk()                                            # and again: the repeated round leaves nothing behind
+    for i in range(len(wl.blocks)):
+        assert st2[i]["q10"] == st[i]["q10"] and st2[i]["q90"] == st[i]["q90"]
 
 
 def test_quantile_select_with_long_stretches_of_equal_values(B, H):
