@@ -303,6 +303,9 @@ static int bind_stats(baoc_t* h, void* dev, size_t bytes, baoc_stream_t stream, 
         }
     }
     h->n_matrix = int(ids.size());
+    std::vector<SelPiece> pieces;
+    uint64_t surv_words = 0;
+    build_sel_pieces(h, &pieces, &sb, &surv_words);
     if (h->sampled) {
         // index lists and the tables of sample-buffer pointers (the host vectors outlive the copies: they belong to the handle)
         h->sample_tables.clear();
@@ -321,6 +324,7 @@ static int bind_stats(baoc_t* h, void* dev, size_t bytes, baoc_stream_t stream, 
     }
     CU(cudaMemcpyAsync(ws + L.blocks, sb.data(), sizeof(StatBlock) * n, cudaMemcpyHostToDevice, s), "upload block table");
     CU(cudaMemcpyAsync(ws + L.tiles, tiles.data(), sizeof(Tile) * tiles.size(), cudaMemcpyHostToDevice, s), "upload tile table");
+    CU(cudaMemcpyAsync(ws + L.pieces, pieces.data(), sizeof(SelPiece) * pieces.size(), cudaMemcpyHostToDevice, s), "upload piece table");
     if (!red.empty())
         CU(cudaMemcpyAsync(ws + L.red_tiles, red.data(), sizeof(RedTile) * red.size(), cudaMemcpyHostToDevice, s), "upload reduction table");
     if (!ids.empty())
@@ -392,11 +396,10 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
                                     h->n_matrix, ws_ctx(h, h->n_red_tiles), s), "moment_reduce_kernel");
         h->launches += 3;
     }
-    LAUNCH(launch_final_resid_select(blocks, tiles, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<RankSel>(ws, L.sel),
-                                     at<SelKey>(ws, L.selkey), at<uint32_t>(ws, L.hist), at<uint32_t>(ws, L.surv),
-                                     at<uint32_t>(ws, L.surv_cnt), at<double>(ws, L.acc), h->n_stat_tiles, n,
-                                     ws_ctx(h, h->n_stat_tiles), s),
-           "final_resid_hist_kernel");
+    SelectArgs sa{blocks, tiles, at<SelPiece>(ws, L.pieces), at<RankSel>(ws, L.sel), at<SelKey>(ws, L.selkey),
+                  at<uint32_t>(ws, L.hist), at<uint32_t>(ws, L.surv), at<uint32_t>(ws, L.surv_cnt), at<double>(ws, L.resid_part),
+                  at<double>(ws, L.fin_out), at<double>(ws, L.acc), h->n_stat_tiles, h->n_sel_pieces, n};
+    LAUNCH(launch_final_resid_select(sa, ws_ctx(h, h->n_sel_pieces), s), "final_resid_hist_kernel");
     h->launches += 6;
 
     std::vector<double> out(size_t(kFinOut) * n);
@@ -411,11 +414,7 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
     if (h->select_retries > 0) {
         CU(cudaMemcpyAsync(ws + L.selkey, h->selkey_staging.data(), sizeof(SelKey) * size_t(n), cudaMemcpyHostToDevice, s),
            "baoc_risk (select keys)");
-        LAUNCH(launch_select_again(blocks, tiles, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<RankSel>(ws, L.sel),
-                                   at<SelKey>(ws, L.selkey), at<uint32_t>(ws, L.hist), at<uint32_t>(ws, L.surv),
-                                   at<uint32_t>(ws, L.surv_cnt), at<double>(ws, L.acc), h->n_stat_tiles, n,
-                                   ws_ctx(h, h->n_stat_tiles), s),
-               "select_first_kernel");
+        LAUNCH(launch_select_again(sa, ws_ctx(h, h->n_sel_pieces), s), "select_first_kernel");
         h->launches += 8;
         CU(cudaMemcpyAsync(out.data(), ws + L.fin_out, 8 * out.size(), cudaMemcpyDeviceToHost, s), "baoc_risk (copy back)");
         CU(cudaStreamSynchronize(s), "baoc_risk (wait)");

@@ -10,6 +10,7 @@
 // histograms on chip while the tiles belong to one block, and hands them over
 // once per block (a deterministic, fixed partition of the work).
 #include <cstring>
+#include <type_traits>
 
 #include "baoc_device.cuh"
 
@@ -369,46 +370,50 @@ final_sums_combine_kernel(const StatBlock* __restrict__ blocks, const double* __
 }
 
 __global__ void __launch_bounds__(kThreads)
-final_resid_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ fin, double* __restrict__ fin_out, int per) {
+final_resid_combine_kernel(const StatBlock* __restrict__ blocks, const double* __restrict__ resid_part, double* __restrict__ fin_out) {
     const StatBlock* b = blocks + blockIdx.x;
-    block_runs_sum<kResidSums>(fin, b->tile0, b->ntiles, per, fin_out + size_t(blockIdx.x) * kFinOut + kFinResid);
+    block_tiles_sum<kResidSums>(resid_part, b->piece0, b->npieces, fin_out + size_t(blockIdx.x) * kFinOut + kFinResid);
 }
 
 // ============================================================================
 // Sweeps 2 and 3: the remaining radix passes of the exact quantile select over
-// the fp32 bit patterns of v (v >= 0, so the unsigned order of the patterns is
-// the numeric order): four ranks per block (the two order statistics around each
-// of the two quantile positions); ranks that still share a prefix share one
-// histogram (the "leader" rank's).  The first pass (top 12 bits) is part of the
-// first sweep.
+// the keys of v (see SelKey): four ranks per block (the two order statistics
+// around each of the two quantile positions); ranks that still share a prefix
+// share one histogram (the "leader" rank's).  The first pass (top 12 bits of the
+// key) is part of the first sweep.
 //
-// Sweep 2 (final_resid_hist_kernel) reads v: the second pass, bits [8, 20) of the
-// elements whose top 12 bits are a rank's prefix (the "survivors"), and in the
-// same sweep the Eq. 7 numerator
+// Sweep 2 (final_resid_hist_kernel) reads v once more, piece by piece (SelPiece:
+// a run of rows of a strip of at most 512 columns): the second pass, the next
+// min(12, s) bits of the elements whose first digit is a rank's (the "survivors"),
+// and in the same sweep the Eq. 7 numerator
 //     sum (S_ij - a_i b_j / mu)^2 = sum (v_ij - rowsum_i colsum_j / total)^2
-// of matrix blocks, in double (a difference of nearly equal numbers).
-// Survivors are few (one bin of the first digit is an eighth of an octave), so
-// they are not counted where they are found, which would leave most lanes idle
-// around every atomic: a thread notes which of its 16 elements survive in a bit
-// mask and copies them to its warp's staging segment; the warp then counts the
-// staged values with all lanes busy (lanes holding equal values add once).  The
-// staged values also go to a survivors list in global memory, kSurvTile slots per
-// tile of the CTA's run of tiles of one block.
+// of matrix blocks, in double (a difference of nearly equal numbers).  A thread
+// keeps eight adjacent columns for all rows of the piece, so the column sums sit
+// in registers and a row costs one row sum per thread.
+// Survivors are few (the key range is fitted to the block, a bin of the first
+// digit holds a fraction of a percent of it), so they are not counted where they
+// are found, which would leave most lanes idle around every atomic: a thread
+// copies its survivors to its warp's staging segment, and the warp counts the
+// staged keys with all lanes busy (lanes holding equal keys add once) when the
+// segment runs full or the piece ends.  The staged keys also go to the piece's
+// survivors list in global memory.
 //
-// Sweep 3 (final_last_kernel) reads that list instead of v: the third pass, bits
-// [0, 8) of the survivors whose upper 24 bits are a rank's prefix.  A run whose
-// survivors did not fit its slots (more than one element in eight: a constant or
-// nearly constant tensor) is marked, and the third pass reads v for that run.
+// Sweep 3 (final_last_kernel) reads those lists instead of v: the third pass, the
+// last s - 12 bits of the survivors whose upper bits are a rank's prefix.  A piece
+// whose survivors did not fit its slots (more than one element in eight: a
+// constant or nearly constant tensor) is marked, and the third pass reads v for it.
 //
-// The second pass counts in 16 bits, two bins per word (32 KB of histograms, 16 KB
-// of staging); a CTA therefore hands its histograms over after at most
-// kSelRunTiles = 15 tiles (61440 elements, below 2^16).
+// The second pass counts in 16 bits, two bins per word (32 KB of histograms for a
+// piece of at most 49152 elements), next to 32 KB of staging.
 // ============================================================================
 constexpr int kRhHistWords = kSelBins / 2;
 constexpr int kRhHistBytes = kRanks * kRhHistWords * 4;
-constexpr int kRhSegWords = kTile / (kThreads / 32);          // a warp's 512 elements of a tile, should all survive
-constexpr int kRhSmemBytes = kRhHistBytes + kTile * 4;
-static_assert(kSelRunTiles * kTile < 65536, "a 16-bit bin must hold a whole run of tiles");
+constexpr int kRhSegWords = 1024;                             // a warp's staging segment
+constexpr int kRhBatch = 2;                                   // rows a thread requests before it uses the first
+constexpr int kRhDrainAt = kRhSegWords - kRhBatch * 32 * 8;   // staged keys above which the segment may not hold another batch
+constexpr int kRhSmemBytes = kRhHistBytes + (kThreads / 32) * kRhSegWords * 4;
+static_assert(kPieceElems < 65536, "a 16-bit bin must hold a whole piece");
+static_assert(kRhDrainAt >= 0, "a batch of rows must fit the staging segment");
 
 // The distinct prefixes the ranks of a block still have (one per leader), padded with a value no key takes.
 struct Leaders {
@@ -434,350 +439,327 @@ __device__ __forceinline__ Leaders leaders_of(const RankSel* __restrict__ sel, i
     return L;
 }
 
-// Replaces the thread's 16 patterns by their keys; bit j of the result set: element j (8 h + i: slice h, element i) is
-// in range and the resolved part of its key is a leader's.
-template <int kL, bool kFull>
-__device__ __forceinline__ uint32_t match_mask(uint32_t (&u)[16], const int (&valid)[2], const Leaders& L, int lo, int wmax, int s) {
-    uint32_t mask = 0u;
+// Geometry of a piece for the CTA: threads across (8 columns each), rows per step.
+struct PieceGeom {
+    int cols;        // row length of the block (kPieceCols for a vector block)
+    int width;       // columns of the piece
+    int tx, ty;      // this thread's place: columns col0 + 8 tx .. + 7 of rows row0 + ty, row0 + ty + step, ...
+    int step;
+    int nc;          // columns of this thread that exist (0..8)
+    bool vec;        // rows start 16-byte aligned: 16-byte loads
+};
+__device__ __forceinline__ PieceGeom piece_geom(const SelPiece& pc, const StatBlock* b) {
+    PieceGeom g;
+    g.cols = b->cols > 1 ? b->cols : kPieceCols;
+    g.width = min(kPieceCols, g.cols - int(pc.col0));
+    int across = 1, sh = 0;
+    while (across * 8 < g.width) { across <<= 1; ++sh; }
+    g.tx = threadIdx.x & (across - 1); g.ty = threadIdx.x >> sh;
+    g.step = kThreads >> sh;
+    g.nc = max(0, min(8, g.width - g.tx * 8));
+    g.vec = (g.cols & 3) == 0;
+    return g;
+}
+// The thread's eight patterns of row r (zeros where there is no element); returns how many exist.
+__device__ __forceinline__ int piece_load(const uint32_t* __restrict__ v, const SelPiece& pc, const PieceGeom& g, int64_t numel,
+                                          int64_t r, uint32_t (&u)[8]) {
+    const int64_t e = r * g.cols + pc.col0 + g.tx * 8;
+    const int n = int(max64(0, min64(g.nc, numel - e)));          // (a vector block's last row may be short)
+    if (g.vec && n == 8) {
+        const uint4 a = ld_stream_u4(v + e), c = ld_stream_u4(v + e + 4);
+        u[0] = a.x; u[1] = a.y; u[2] = a.z; u[3] = a.w; u[4] = c.x; u[5] = c.y; u[6] = c.z; u[7] = c.w;
+    } else {
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-        u[j] = sel_key(u[j], lo, wmax);
-        const uint32_t key = u[j] >> s;
-        bool p = (key == L.key[0]) | (key == L.key[1]);
-        if (kL > 2) p |= (key == L.key[2]) | (key == L.key[3]);
-        if (!kFull) p &= (j & 7) < valid[j >> 3];
-        if (p) mask |= 1u << j;
+        for (int j = 0; j < 8; ++j) u[j] = j < n ? v[e + j] : 0u;
     }
-    return mask;
+    return n;
 }
 
 __global__ void __launch_bounds__(kThreads, 3)
-final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const RankSel* __restrict__ sel,
-                        const SelKey* __restrict__ selkey, double* __restrict__ fin, uint32_t* __restrict__ hist,
-                        uint32_t* __restrict__ surv, uint32_t* __restrict__ surv_cnt, int64_t n_tiles, int tiles_per_cta,
-                        int with_resid BAOC_CHECK_PARAM) {
+final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const SelPiece* __restrict__ pieces, const RankSel* __restrict__ sel,
+                        const SelKey* __restrict__ selkey, double* __restrict__ resid_part, uint32_t* __restrict__ hist,
+                        uint32_t* __restrict__ surv, uint32_t* __restrict__ surv_cnt, int64_t n_pieces, int with_resid BAOC_CHECK_PARAM) {
+    const SelPiece pc = pieces[blockIdx.x];
 #ifdef BAOC_CHECKED
     {
-        const int64_t c0 = int64_t(blockIdx.x) * tiles_per_cta, c1 = min64(c0 + tiles_per_cta, n_tiles);
-        if (c0 >= ck.n_tiles || n_tiles != ck.n_tiles) { check_fail(kChkTileIndex, kKerFinalHist, c0, ck.n_tiles, n_tiles, 0); return; }
-        for (int64_t ti = c0; ti < c1; ++ti) {
-            const Tile ct = tiles[ti];
-            if (ct.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerFinalHist, ct.block, ck.n_blocks, ti, 0); return; }
-            const StatBlock* cb = blocks + ct.block;
-            const int64_t cbase = int64_t(ct.piece) * kTile;
-            const int64_t cpad = (cb->numel + kQBlock - 1) / kQBlock * kQBlock, cn = min64(kTile, cpad - cbase);
-            if (!check_tile(ck, kKerFinalHist, ti, ct.block, cbase, cb->numel) ||
-                !check_range(ck, kKerFinalHist, cb->v + cbase, 4 * cn, 0) ||
-                !check_range(ck, kKerFinalHist, hist + size_t(ct.block) * kRanks * kSelBins, 4ll * kRanks * kSelBins, 1) ||
-                !check_range(ck, kKerFinalHist, sel + size_t(ct.block) * kRanks, int64_t(sizeof(RankSel)) * kRanks, 2) ||
-                !check_range(ck, kKerFinalHist, fin + size_t(ti) * kResidSums, 8 * kResidSums, 3) ||
-                !check_range(ck, kKerFinalHist, surv + size_t(ti) * kSurvTile, 4ll * kSurvTile, 6) ||
-                !check_range(ck, kKerFinalHist, surv_cnt + ti, 4, 7) ||
-                (cb->cols > 1 && (!check_range(ck, kKerFinalHist, cb->rowsum, 8ll * (cb->rows + 1), 4) ||
-                                  !check_range(ck, kKerFinalHist, cb->colsum, 8ll * cb->cols, 5))))
-                return;
-        }
+        if (int64_t(blockIdx.x) >= ck.n_tiles || n_pieces != ck.n_tiles) { check_fail(kChkTileIndex, kKerFinalHist, blockIdx.x, ck.n_tiles, n_pieces, 0); return; }
+        if (pc.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerFinalHist, pc.block, ck.n_blocks, blockIdx.x, 0); return; }
+        const StatBlock* cb = blocks + pc.block;
+        const int64_t ccols = cb->cols > 1 ? cb->cols : kPieceCols, crows = cb->cols > 1 ? cb->rows : (cb->numel + kPieceCols - 1) / kPieceCols;
+        if (int64_t(pc.col0) >= ccols || int64_t(pc.row0) + pc.nrows > crows || pc.nrows == 0) { check_fail(kChkTileStart, kKerFinalHist, pc.col0, ccols, pc.row0 + pc.nrows, crows); return; }
+        const int64_t cpad = (cb->numel + kQBlock - 1) / kQBlock * kQBlock;
+        if (!check_range(ck, kKerFinalHist, cb->v, 4 * cpad, 0) ||
+            !check_range(ck, kKerFinalHist, hist + size_t(pc.block) * kRanks * kSelBins, 4ll * kRanks * kSelBins, 1) ||
+            !check_range(ck, kKerFinalHist, sel + size_t(pc.block) * kRanks, int64_t(sizeof(RankSel)) * kRanks, 2) ||
+            !check_range(ck, kKerFinalHist, resid_part + blockIdx.x, 8, 3) ||
+            !check_range(ck, kKerFinalHist, surv + pc.surv_off, 4ll * pc.slots, 6) ||
+            !check_range(ck, kKerFinalHist, surv_cnt + blockIdx.x, 4, 7) ||
+            (cb->cols > 1 && (!check_range(ck, kKerFinalHist, cb->rowsum, 8ll * (cb->rows + 1), 4) ||
+                              !check_range(ck, kKerFinalHist, cb->colsum, 8ll * cb->cols, 5))))
+            return;
     }
 #endif
     extern __shared__ __align__(16) unsigned char dyn[];
     uint32_t (*sh)[kRhHistWords] = reinterpret_cast<uint32_t (*)[kRhHistWords]>(dyn);
     uint32_t* stage = reinterpret_cast<uint32_t*>(dyn + kRhHistBytes);
-    __shared__ int wcnt[kThreads / 32];                       // survivors a warp has staged of its current tile
-    __shared__ int run_cnt, run_over;                         // survivors of the run written so far; the run outgrew its slots
-    constexpr int kSl = kTile / (kThreads * 8);
-    static_assert(kSl == 2, "a tile is two slices of eight elements per thread");
+    __shared__ int wcnt[kThreads / 32];                       // keys a warp has staged
+    __shared__ int run_cnt, run_over;                         // survivors of the piece listed so far; the piece outgrew its slots
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
-    Leaders L;
-    L.n = 0;
-    int key_lo = 0, key_s = -1, key_max = 0, d_shift = 0, d_bits = 0;   // the block's key; this pass's digit (s < 0: the block sits this round out)
-    // what the tiles of one block share, fetched once when the CTA enters the block (nothing a tile needs then hangs on
-    // a chain of dependent loads): its extent in the tile table, v, the row/column sums, 1 / total
-    int cur_block = -1;
-    int64_t blk_end = first, tile0 = 0, numel = 0;
-    const uint32_t* __restrict__ v = nullptr;
-    const double* __restrict__ rowsum = nullptr;
-    const double* __restrict__ colsum = nullptr;
-    double inv_total = 0.0;
-    int64_t run_first = first;
-    int cap = 0;                                              // slots of the current run
-    uint32_t* surv_run = surv;
-    double acc[kResidSums] = {0.0};
-    // position of the current tile's first element in its matrix, kept by 32-bit arithmetic from tile to tile
-    int64_t row0 = 0;
-    uint32_t col0 = 0, cols_u = 1, magic = 0;
-    int64_t next_base = -1;
+    const StatBlock* b = blocks + pc.block;
+    const SelKey key = selkey[pc.block];
+    if (key.s < 0) return;                                    // uniform over the CTA: the block sits this round out
+    int d_shift, d_bits;
+    sel_digit(key.s, 1, d_shift, d_bits);
+    const int wmax = sel_wmax(key.s);
+    const bool resid = with_resid != 0 && b->cols > 1;
+    if (!resid && d_bits == 0) {                              // nothing to do here (uniform)
+        if (threadIdx.x == 0) { surv_cnt[blockIdx.x] = 0u; if (with_resid) resid_part[blockIdx.x] = 0.0; }
+        return;
+    }
+    const Leaders L = leaders_of(sel + size_t(pc.block) * kRanks, key.s);
+    const PieceGeom g = piece_geom(pc, b);
+    const int64_t numel = b->numel;
+    const uint32_t* __restrict__ v = reinterpret_cast<const uint32_t*>(b->v);
+    uint32_t* seg = stage + warp * kRhSegWords;
+    uint32_t* list = surv + pc.surv_off;
 
-    auto flush = [&](int blk, int64_t t_begin) {
-        if (key_s < 0) return;                                // uniform over the CTA: nothing was done for this block
-        if (with_resid) {
-            cta_reduce_store<kResidSums>(acc, fin + size_t(t_begin) * kResidSums);
-            acc[0] = 0.0;
-        } else {
-            __syncthreads();
-        }
-        if (threadIdx.x == 0) {                               // (every warp has drained its last tile)
-            surv_cnt[t_begin] = run_over ? kSurvOverflow : uint32_t(run_cnt);
-            run_cnt = 0; run_over = 0;
-        }
-#pragma unroll
-        for (int k = 0; k < kRanks; ++k) {
-            if (k >= L.n || d_bits == 0) continue;            // uniform over the CTA
-            uint32_t* out = hist + (size_t(blk) * kRanks + L.slot[k]) * kSelBins;
-            for (int w = threadIdx.x; w < kRhHistWords; w += kThreads) {
-                const uint32_t x = sh[k][w];
-                if (x) {
-                    if (x & 0xffffu) atomicAdd(out + 2 * w, x & 0xffffu);
-                    if (x >> 16) atomicAdd(out + 2 * w + 1, x >> 16);
-                    sh[k][w] = 0u;
-                }
-            }
-        }
-        __syncthreads();
-    };
-    // floor(x / cols_u) for x < 2^32 from the precomputed floor((2^32 - 1) / cols_u): the estimate is at most 2 short
-    auto divmod = [&](uint32_t x, uint32_t& rem) {
-        uint32_t q = __umulhi(x, magic);
-        rem = x - q * cols_u;
-        if (rem >= cols_u) { rem -= cols_u; ++q; }
-        if (rem >= cols_u) { rem -= cols_u; ++q; }
-        return q;
-    };
-
-    for (int i = threadIdx.x; i < kRanks * kRhHistWords; i += kThreads) (&sh[0][0])[i] = 0u;
+    if (d_bits > 0)
+        for (int i = threadIdx.x; i < kRanks * kRhHistWords; i += kThreads) (&sh[0][0])[i] = 0u;
     if (threadIdx.x < kThreads / 32) wcnt[threadIdx.x] = 0;
     if (threadIdx.x == 0) { run_cnt = 0; run_over = 0; }
+    // the thread's column sums, and 1 / total
+    double cs[8];
+    double inv_total = 0.0;
+    const double* __restrict__ rowsum = b->rowsum;
+    if (resid) {
+        const double total = rowsum[b->rows];                 // the block's sum of v, left there by the row/column combine
+        inv_total = total > 0.0 ? 1.0 / total : 0.0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cs[j] = j < g.nc ? b->colsum[pc.col0 + g.tx * 8 + j] : 0.0;
+    }
     __syncthreads();
 
-#pragma unroll 1
-    for (int64_t ti = first; ti < last; ++ti) {
-        if (ti == blk_end) {                                  // uniform over the CTA: the first tile of the next block
-            if (cur_block >= 0) flush(cur_block, run_first);
-            const Tile t = tiles[ti];
-            const StatBlock* b = blocks + t.block;
-            cur_block = int(t.block);
-            run_first = ti;
-            tile0 = b->tile0;                                 // the block's tiles are tile0 + piece, piece = 0, 1, ...
-            blk_end = min64(last, tile0 + b->ntiles);
-            numel = b->numel;
-            v = reinterpret_cast<const uint32_t*>(b->v);
-            const SelKey key = selkey[t.block];
-            key_lo = key.lo; key_s = key.s; key_max = sel_wmax(max(key.s, 0));
-            sel_digit(key.s, 1, d_shift, d_bits);
-            L = leaders_of(sel + size_t(t.block) * kRanks, max(key.s, 0));
-            cap = int(blk_end - ti) * kSurvTile;
-            surv_run = surv + size_t(ti) * kSurvTile;
-            cols_u = with_resid ? uint32_t(b->cols) : 1u;
-            magic = 0xffffffffu / cols_u;
-            next_base = -1;
-            if (cols_u > 1u) {
-                rowsum = b->rowsum; colsum = b->colsum;
-                const double total = rowsum[b->rows];         // the block's sum of v, left there by the row/column combine
-                inv_total = total > 0.0 ? 1.0 / total : 0.0;
-            }
-        }
-        if (key_s < 0) continue;                              // uniform over the CTA
-        const int64_t base = (ti - tile0) * kTile;
-        if (cols_u > 1u) {
-            if (base == next_base) {                          // the next piece of the same matrix: advance by one tile
-                uint32_t rem;
-                row0 += divmod(col0 + uint32_t(kTile), rem);
-                col0 = rem;
-            } else {
-                row0 = base / int64_t(cols_u);
-                col0 = uint32_t(base - row0 * int64_t(cols_u));
-            }
-            next_base = base + kTile;
-        }
-        const bool tile_full = base + kTile <= numel;         // uniform over the CTA
-        const uint32_t* __restrict__ vt = v + base + threadIdx.x * 8;
-        uint32_t u[8 * kSl];
-        int valid[kSl];
-        if (tile_full) {
-#pragma unroll
-            for (int h = 0; h < kSl; ++h) {
-                const uint4 a = ld_stream_u4(vt + h * (kThreads * 8)), c = ld_stream_u4(vt + h * (kThreads * 8) + 4);
-                valid[h] = 8;
-                u[8 * h + 0] = a.x; u[8 * h + 1] = a.y; u[8 * h + 2] = a.z; u[8 * h + 3] = a.w;
-                u[8 * h + 4] = c.x; u[8 * h + 5] = c.y; u[8 * h + 6] = c.z; u[8 * h + 7] = c.w;
-            }
-        } else {
-#pragma unroll
-            for (int h = 0; h < kSl; ++h) {                   // v is padded to whole quantisation blocks: in bounds whenever e < numel
-                const int64_t e = base + int64_t(h) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
-                valid[h] = e < numel ? int(min64(8, numel - e)) : 0;
-                uint4 a = make_uint4(0u, 0u, 0u, 0u), c = a;
-                if (valid[h] > 0) { a = ld_stream_u4(vt + h * (kThreads * 8)); c = ld_stream_u4(vt + h * (kThreads * 8) + 4); }
-                u[8 * h + 0] = a.x; u[8 * h + 1] = a.y; u[8 * h + 2] = a.z; u[8 * h + 3] = a.w;
-                u[8 * h + 4] = c.x; u[8 * h + 5] = c.y; u[8 * h + 6] = c.z; u[8 * h + 7] = c.w;
-            }
-        }
-
-        if (cols_u > 1u) {
-#pragma unroll
-            for (int h = 0; h < kSl; ++h) {
-                if (valid[h] == 0) continue;
-                uint32_t c;
-                int64_t r = row0 + divmod(col0 + uint32_t(h * (kThreads * 8) + threadIdx.x * 8), c);
-                double rs = __ldg(rowsum + r) * inv_total;
-                if (valid[h] == 8 && (cols_u & 7u) == 0u) {
-                    // the eight elements lie in one row: one row sum, four 16-byte loads of column sums
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const double2 w = __ldg(reinterpret_cast<const double2*>(colsum + c) + q);
-                        const double d0 = fma(-rs, w.x, double(__uint_as_float(u[8 * h + 2 * q])));
-                        const double d1 = fma(-rs, w.y, double(__uint_as_float(u[8 * h + 2 * q + 1])));
-                        acc[0] = fma(d0, d0, acc[0]);
-                        acc[0] = fma(d1, d1, acc[0]);
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (j < valid[h]) {
-                            const double diff = fma(-rs, __ldg(colsum + c), double(__uint_as_float(u[8 * h + j])));
-                            acc[0] = fma(diff, diff, acc[0]);
-                            if (++c == cols_u) { c = 0u; ++r; if (j + 1 < valid[h]) rs = __ldg(rowsum + r) * inv_total; }
-                        }
-                    }
-                }
-            }
-        }
-
-        // ---- the survivors of this tile: noted, staged by warp, counted, listed
-        if (d_bits == 0) continue;                            // uniform over the CTA: the first pass resolved the whole key
-        uint32_t mask;
-        if (tile_full) mask = L.n <= 2 ? match_mask<2, true>(u, valid, L, key_lo, key_max, key_s) : match_mask<4, true>(u, valid, L, key_lo, key_max, key_s);
-        else mask = match_mask<4, false>(u, valid, L, key_lo, key_max, key_s);
-        if (!__any_sync(0xffffffffu, mask != 0u)) continue;   // the usual case: a bin of the first digit holds few elements
-        uint32_t* seg = stage + warp * kRhSegWords;
-        const int found = __popc(mask);
-        int pos = found ? atomicAdd(&wcnt[warp], found) : 0;
-#pragma unroll
-        for (int j = 0; j < 8 * kSl; ++j)
-            if (mask & (1u << j)) seg[pos++] = u[j];
-        __syncwarp();
+    // the warp's staged keys: listed, and counted into the histograms of this pass's digit
+    auto drain = [&]() {
         const int staged = wcnt[warp];                        // uniform over the warp
+        if (staged == 0) return;
         int off = 0;
         if (lane == 0) {
             off = atomicAdd(&run_cnt, staged);
-            if (off + staged > cap) run_over = 1;
+            if (off + staged > int(pc.slots)) run_over = 1;
         }
         off = __shfl_sync(0xffffffffu, off, 0);
-        const bool fits = off + staged <= cap;
+        const bool fits = off + staged <= int(pc.slots);
         for (int i0 = 0; i0 < staged; i0 += 32) {
             const int i = i0 + lane;
             const bool on = i < staged;
             const unsigned act = __ballot_sync(0xffffffffu, on);
             if (on) {
                 const uint32_t x = seg[i];
-                if (fits) surv_run[off + i] = x;
+                if (fits) list[off + i] = x;
                 const unsigned same = __match_any_sync(act, x);
                 if (lane == __ffs(int(same)) - 1) {           // one lane per distinct key adds for all of them
-                    const uint32_t key = x >> key_s, d = (x >> d_shift) & ((1u << d_bits) - 1u);
+                    const uint32_t top = x >> key.s, d = (x >> d_shift) & ((1u << d_bits) - 1u);
                     const uint32_t n = uint32_t(__popc(same)) << ((d & 1u) * 16u);
 #pragma unroll
                     for (int k = 0; k < kRanks; ++k)
-                        if (key == L.key[k]) atomicAdd(&sh[k][d >> 1], n);
+                        if (top == L.key[k]) atomicAdd(&sh[k][d >> 1], n);
                 }
             }
         }
         __syncwarp();
         if (lane == 0) wcnt[warp] = 0;
         __syncwarp();
-    }
-    if (cur_block >= 0) flush(cur_block, run_first);
-}
+    };
 
-// Sweep 3: the last bits of the key (at most 7).  Same partition of the tiles into runs as sweep 2; per run either its survivors list or, for
-// a run that was marked, the tiles of v themselves.  The histogram (256 bins of 32 bits per leader) is handed over per run.
-constexpr int kLastBins = 1 << kSel3Bits;
+    double acc[kResidSums] = {0.0};
+    const int64_t r_end = int64_t(pc.row0) + pc.nrows;
+    // Which elements survive.  A leader whose first digit is neither the lowest nor the highest bin covers the patterns
+    // [lo + (digit << s), lo + ((digit + 1) << s)): one subtraction and one unsigned comparison per element and leader,
+    // no key.  The two end bins also hold the clamped elements, so a block with a leader there takes the general test
+    // on the key itself.
+    const bool inner = L.n <= 2 && L.key[0] - 1u < uint32_t(kSelBins - 2) && (L.n < 2 || L.key[1] - 1u < uint32_t(kSelBins - 2));
+    const uint32_t span = 1u << key.s;
+    const uint32_t base0 = uint32_t(key.lo) + (L.key[0] << key.s);
+    const uint32_t base1 = L.n > 1 ? uint32_t(key.lo) + (L.key[1] << key.s) : base0;
+    // a vector block's last row may be short; every other row of a piece holds the thread's nc columns
+    const int64_t short_row = (b->cols > 1 || (numel % kPieceCols) == 0) ? -1 : numel / kPieceCols;
+    const bool wide = g.vec && g.nc == 8;                     // the thread's usual row: eight elements, two 16-byte loads
+    const uint32_t* __restrict__ vp = v + (int64_t(pc.row0) + g.ty) * g.cols + pc.col0 + g.tx * 8;
+    const int64_t v_step = int64_t(g.step) * g.cols;
 
-__global__ void __launch_bounds__(kThreads)
-final_last_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const RankSel* __restrict__ sel,
-                  const SelKey* __restrict__ selkey, uint32_t* __restrict__ hist, const uint32_t* __restrict__ surv,
-                  const uint32_t* __restrict__ surv_cnt, int64_t n_tiles, int tiles_per_cta BAOC_CHECK_PARAM) {
-    __shared__ uint32_t sh[kRanks][kLastBins];
-    const int lane = threadIdx.x & 31;
-    const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
-#ifdef BAOC_CHECKED
-    if (first >= ck.n_tiles || n_tiles != ck.n_tiles) { check_fail(kChkTileIndex, kKerFinalLast, first, ck.n_tiles, n_tiles, 0); return; }
-#endif
-    for (int i = threadIdx.x; i < kRanks * kLastBins; i += kThreads) (&sh[0][0])[i] = 0u;
-    __syncthreads();
-
-    // one lane per distinct key among the lanes `act` adds for all of them
-    auto count_same = [&](unsigned act, uint32_t x, const Leaders& L, int bits) {
-        const unsigned same = __match_any_sync(act, x);
-        if (lane == __ffs(int(same)) - 1) {
-            const uint32_t key = x >> bits, d = x & ((1u << bits) - 1u);
+    // one row of the thread: kWide: all eight elements exist
+    auto row = [&](auto wide_tag, uint32_t (&u)[8], int n, double rsum) {
+        constexpr bool kWide = decltype(wide_tag)::value;
+        if (resid) {
+            const double a = rsum * inv_total;
 #pragma unroll
-            for (int k = 0; k < kRanks; ++k)
-                if (key == L.key[k]) atomicAdd(&sh[k][d], uint32_t(__popc(same)));
+            for (int j = 0; j < 8; ++j) {
+                if (kWide || j < n) {
+                    const double d = fma(-a, cs[j], double(__uint_as_float(u[j])));
+                    acc[0] = fma(d, d, acc[0]);
+                }
+            }
+        }
+        if (d_bits == 0) return;
+        uint32_t mask = 0u;
+        if (inner) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const bool p = (kWide || j < n) & ((u[j] - base0 < span) | (u[j] - base1 < span));
+                if (p) mask |= 1u << j;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t top = sel_key(u[j], key.lo, wmax) >> key.s;
+                const bool p = (kWide || j < n) & ((top == L.key[0]) | (top == L.key[1]) | (top == L.key[2]) | (top == L.key[3]));
+                if (p) mask |= 1u << j;
+            }
+        }
+        if (mask) {                                           // few threads
+            int pos = atomicAdd(&wcnt[warp], __popc(mask));
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (mask & (1u << j)) seg[pos++] = sel_key(u[j], key.lo, wmax);
         }
     };
 
 #pragma unroll 1
-    for (int64_t t_begin = first; t_begin < last;) {
-        const Tile t = tiles[t_begin];
-#ifdef BAOC_CHECKED
-        if (t.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerFinalLast, t.block, ck.n_blocks, t_begin, 0); return; }
-#endif
-        const StatBlock* b = blocks + t.block;
-        const int64_t t_end = min64(last, b->tile0 + b->ntiles);     // the run: this CTA's tiles of the block
-        const SelKey key = selkey[t.block];
-        int d_shift, d_bits;
-        sel_digit(key.s, 2, d_shift, d_bits);
-        if (key.s < 0 || d_bits == 0) { t_begin = t_end; continue; }   // uniform over the CTA: not in this round, or nothing left to find
-        const Leaders L = leaders_of(sel + size_t(t.block) * kRanks, d_bits);
-        const uint32_t cnt = surv_cnt[t_begin];
-#ifdef BAOC_CHECKED
-        if (!check_range(ck, kKerFinalLast, surv_cnt + t_begin, 4, 0) ||
-            !check_range(ck, kKerFinalLast, surv + size_t(t_begin) * kSurvTile, 4ll * kSurvTile * (t_end - t_begin), 1) ||
-            !check_range(ck, kKerFinalLast, hist + size_t(t.block) * kRanks * kSelBins, 4ll * kRanks * kSelBins, 2) ||
-            (cnt != kSurvOverflow && int64_t(cnt) > int64_t(kSurvTile) * (t_end - t_begin) &&
-             !check_fail(kChkRange, kKerFinalLast, 3, cnt, t_begin, t_end)))
-            return;
-#endif
-        if (cnt != kSurvOverflow) {
-            const uint32_t* __restrict__ list = surv + size_t(t_begin) * kSurvTile;
-            for (uint32_t i0 = 0; i0 < cnt; i0 += kThreads) {             // uniform over the CTA
-                const uint32_t i = i0 + threadIdx.x;
-                const bool on = i < cnt;
-                const unsigned act = __ballot_sync(0xffffffffu, on);
-                if (on) count_same(act, list[i], L, d_bits);
-            }
-        } else {
-            const uint32_t* __restrict__ v = reinterpret_cast<const uint32_t*>(b->v);
-            const int64_t e0 = int64_t(t.piece) * kTile, e1 = min64(b->numel, e0 + (t_end - t_begin) * int64_t(kTile));
-#ifdef BAOC_CHECKED
-            if (!check_range(ck, kKerFinalLast, v + e0, 4 * (e1 - e0), 4)) return;
-#endif
-            for (int64_t i0 = e0; i0 < e1; i0 += kThreads) {              // uniform over the CTA
-                const int64_t i = i0 + threadIdx.x;
-                const bool on = i < e1;
-                uint32_t x = 0u;
-                bool hit = false;
-                if (on) {
-                    x = sel_key(v[i], key.lo, sel_wmax(key.s));
-                    const uint32_t upper = x >> d_bits;
-                    hit = (upper == L.key[0]) | (upper == L.key[1]) | (upper == L.key[2]) | (upper == L.key[3]);
-                }
-                const unsigned act = __ballot_sync(0xffffffffu, hit);
-                if (hit) count_same(act, x, L, d_bits);
-            }
-        }
-        __syncthreads();
+    for (int64_t r0 = int64_t(pc.row0); r0 < r_end; r0 += int64_t(kRhBatch) * g.step) {   // the same trips for every thread
+        uint32_t u[kRhBatch][8];
+        int n[kRhBatch];
+        double rs[kRhBatch];
 #pragma unroll
-        for (int k = 0; k < kRanks; ++k) {
-            if (k >= L.n) continue;                           // uniform over the CTA
-            uint32_t* out = hist + (size_t(t.block) * kRanks + L.slot[k]) * kSelBins;
-            for (int w = threadIdx.x; w < kLastBins; w += kThreads) {
-                const uint32_t x = sh[k][w];
-                if (x) { atomicAdd(out + w, x); sh[k][w] = 0u; }
+        for (int k = 0; k < kRhBatch; ++k) {
+            const int64_t r = r0 + g.ty + int64_t(k) * g.step;
+            n[k] = 0;
+            rs[k] = 0.0;
+            if (r < r_end) {
+                if (wide && r != short_row) {
+                    const uint4 a = ld_stream_u4(vp + k * v_step), c = ld_stream_u4(vp + k * v_step + 4);
+                    u[k][0] = a.x; u[k][1] = a.y; u[k][2] = a.z; u[k][3] = a.w; u[k][4] = c.x; u[k][5] = c.y; u[k][6] = c.z; u[k][7] = c.w;
+                    n[k] = 8;
+                } else {
+                    n[k] = piece_load(v, pc, g, numel, r, u[k]);
+                }
+                if (resid) rs[k] = __ldg(rowsum + r);
             }
         }
-        __syncthreads();
-        t_begin = t_end;
+        vp += kRhBatch * v_step;
+#pragma unroll
+        for (int k = 0; k < kRhBatch; ++k) {
+            if (n[k] == 8) row(std::true_type{}, u[k], 8, rs[k]);
+            else if (n[k] > 0) row(std::false_type{}, u[k], n[k], rs[k]);
+        }
+        __syncwarp();
+        if (wcnt[warp] > kRhDrainAt) drain();                 // uniform over the warp: room for the next batch
+    }
+    __syncwarp();
+    drain();
+    if (with_resid) cta_reduce_store<kResidSums>(acc, resid_part + blockIdx.x);
+    else __syncthreads();
+    if (threadIdx.x == 0) surv_cnt[blockIdx.x] = run_over ? kSurvOverflow : uint32_t(run_cnt);
+    if (d_bits == 0 || (run_cnt == 0 && run_over == 0)) return;   // uniform over the CTA: nothing was counted
+#pragma unroll
+    for (int k = 0; k < kRanks; ++k) {
+        if (k >= L.n) continue;                               // uniform over the CTA
+        uint32_t* out = hist + (size_t(pc.block) * kRanks + L.slot[k]) * kSelBins;
+        for (int w = threadIdx.x; w < kRhHistWords; w += kThreads) {
+            const uint32_t x = sh[k][w];
+            if (x) {
+                if (x & 0xffffu) atomicAdd(out + 2 * w, x & 0xffffu);
+                if (x >> 16) atomicAdd(out + 2 * w + 1, x >> 16);
+            }
+        }
+    }
+}
+
+// Sweep 3: the last bits of the key (at most 7), one CTA per piece: its survivors list or, for a piece that was
+// marked, its elements of v.  The histogram (256 bins of 32 bits per leader) is handed over per piece.
+constexpr int kLastBins = 1 << kSel3Bits;
+
+__global__ void __launch_bounds__(kThreads)
+final_last_kernel(const StatBlock* __restrict__ blocks, const SelPiece* __restrict__ pieces, const RankSel* __restrict__ sel,
+                  const SelKey* __restrict__ selkey, uint32_t* __restrict__ hist, const uint32_t* __restrict__ surv,
+                  const uint32_t* __restrict__ surv_cnt, int64_t n_pieces BAOC_CHECK_PARAM) {
+    __shared__ uint32_t sh[kRanks][kLastBins];
+    __shared__ int counted;
+    const int lane = threadIdx.x & 31;
+    const SelPiece pc = pieces[blockIdx.x];
+#ifdef BAOC_CHECKED
+    if (int64_t(blockIdx.x) >= ck.n_tiles || n_pieces != ck.n_tiles) { check_fail(kChkTileIndex, kKerFinalLast, blockIdx.x, ck.n_tiles, n_pieces, 0); return; }
+    if (pc.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerFinalLast, pc.block, ck.n_blocks, blockIdx.x, 0); return; }
+#endif
+    const StatBlock* b = blocks + pc.block;
+    const SelKey key = selkey[pc.block];
+    int d_shift, d_bits;
+    sel_digit(key.s, 2, d_shift, d_bits);
+    if (key.s < 0 || d_bits == 0) return;                     // uniform over the CTA: not in this round, or nothing left to find
+    const uint32_t cnt = surv_cnt[blockIdx.x];
+    if (cnt == 0u) return;
+#ifdef BAOC_CHECKED
+    if (!check_range(ck, kKerFinalLast, surv_cnt + blockIdx.x, 4, 0) ||
+        !check_range(ck, kKerFinalLast, surv + pc.surv_off, 4ll * pc.slots, 1) ||
+        !check_range(ck, kKerFinalLast, hist + size_t(pc.block) * kRanks * kSelBins, 4ll * kRanks * kSelBins, 2) ||
+        (cnt != kSurvOverflow && cnt > pc.slots && !check_fail(kChkRange, kKerFinalLast, 3, cnt, pc.slots, blockIdx.x)))
+        return;
+#endif
+    const Leaders L = leaders_of(sel + size_t(pc.block) * kRanks, d_bits);
+    for (int i = threadIdx.x; i < kRanks * kLastBins; i += kThreads) (&sh[0][0])[i] = 0u;
+    if (threadIdx.x == 0) counted = 0;
+    __syncthreads();
+
+    // one lane per distinct key among the lanes `act` adds for all of them
+    auto count_same = [&](unsigned act, uint32_t x) {
+        const unsigned same = __match_any_sync(act, x);
+        if (lane == __ffs(int(same)) - 1) {
+            const uint32_t upper = x >> d_bits, d = x & ((1u << d_bits) - 1u);
+#pragma unroll
+            for (int k = 0; k < kRanks; ++k)
+                if (upper == L.key[k]) { atomicAdd(&sh[k][d], uint32_t(__popc(same))); counted = 1; }
+        }
+    };
+
+    if (cnt != kSurvOverflow) {
+        const uint32_t* __restrict__ list = surv + pc.surv_off;
+        for (uint32_t i0 = 0; i0 < cnt; i0 += kThreads) {     // uniform over the CTA
+            const uint32_t i = i0 + threadIdx.x;
+            const bool on = i < cnt;
+            const unsigned act = __ballot_sync(0xffffffffu, on);
+            if (on) count_same(act, list[i]);
+        }
+    } else {
+        const PieceGeom g = piece_geom(pc, b);
+        const uint32_t* __restrict__ v = reinterpret_cast<const uint32_t*>(b->v);
+        const int wmax = sel_wmax(key.s);
+#ifdef BAOC_CHECKED
+        if (!check_range(ck, kKerFinalLast, v, 4 * ((b->numel + kQBlock - 1) / kQBlock * kQBlock), 4)) return;
+#endif
+        const int64_t r_end = int64_t(pc.row0) + pc.nrows;
+        for (int64_t r0 = int64_t(pc.row0); r0 < r_end; r0 += g.step) {   // uniform over the CTA
+            const int64_t r = r0 + g.ty;
+            uint32_t u[8];
+            const int n = r < r_end ? piece_load(v, pc, g, b->numel, r, u) : 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t x = sel_key(u[j], key.lo, wmax), upper = x >> d_bits;
+                const bool hit = (j < n) & ((upper == L.key[0]) | (upper == L.key[1]) | (upper == L.key[2]) | (upper == L.key[3]));
+                const unsigned act = __ballot_sync(0xffffffffu, hit);
+                if (hit) count_same(act, x);
+            }
+        }
+    }
+    __syncthreads();
+    if (!counted) return;                                     // uniform over the CTA
+#pragma unroll
+    for (int k = 0; k < kRanks; ++k) {
+        if (k >= L.n) continue;                               // uniform over the CTA
+        uint32_t* out = hist + (size_t(pc.block) * kRanks + L.slot[k]) * kSelBins;
+        for (int w = threadIdx.x; w < kLastBins; w += kThreads) {
+            const uint32_t x = sh[k][w];
+            if (x) atomicAdd(out + w, x);
+        }
     }
 }
 
@@ -962,52 +944,43 @@ int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* c
 }
 
 // The second and third pass of the select (with the Eq. 7 residual in the second sweep if with_resid), and the gather.
-static int select_rest(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                       const SelKey* selkey, uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc,
-                       int64_t n_tiles, int n_blocks, int with_resid, const CheckCtx& ck, cudaStream_t s) {
+static int select_rest(const SelectArgs& a, int with_resid, const CheckCtx& ck, cudaStream_t s) {
     (void)ck;
     cudaError_t e = cudaFuncSetAttribute(final_resid_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRhSmemBytes);
     if (e != cudaSuccess) return int(e);
-    const int per = run_tiles(n_tiles, kSelRunTiles);
-    const unsigned grid = unsigned((n_tiles + per - 1) / per);
-    final_resid_hist_kernel<<<grid, kThreads, kRhSmemBytes, s>>>(blocks, tiles, sel, selkey, fin, hist, surv, surv_cnt, n_tiles,
-                                                                per, with_resid BAOC_CHECK_ARG(ck));
+    const unsigned grid = unsigned(a.n_pieces);
+    final_resid_hist_kernel<<<grid, kThreads, kRhSmemBytes, s>>>(a.blocks, a.pieces, a.sel, a.selkey, a.resid_part, a.hist, a.surv,
+                                                                a.surv_cnt, a.n_pieces, with_resid BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
     if (with_resid) {
-        final_resid_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
+        final_resid_combine_kernel<<<a.n_blocks, kThreads, 0, s>>>(a.blocks, a.resid_part, a.fin_out);
         BAOC_LAUNCH_CHECK();
     }
-    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, selkey, 1);
+    select_pick_kernel<<<a.n_blocks, kThreads, 0, s>>>(a.sel, a.hist, a.selkey, 1);
     BAOC_LAUNCH_CHECK();
-    final_last_kernel<<<grid, kThreads, 0, s>>>(blocks, tiles, sel, selkey, hist, surv, surv_cnt, n_tiles, per BAOC_CHECK_ARG(ck));
+    final_last_kernel<<<grid, kThreads, 0, s>>>(a.blocks, a.pieces, a.sel, a.selkey, a.hist, a.surv, a.surv_cnt, a.n_pieces BAOC_CHECK_ARG(ck));
     BAOC_LAUNCH_CHECK();
-    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, selkey, 2);
+    select_pick_kernel<<<a.n_blocks, kThreads, 0, s>>>(a.sel, a.hist, a.selkey, 2);
     BAOC_LAUNCH_CHECK();
-    const int tb = 128, gb = (n_blocks + tb - 1) / tb;
-    stats_gather_kernel<<<gb, tb, 0, s>>>(sel, selkey, acc, fin_out, n_blocks);
+    const int tb = 128, gb = (a.n_blocks + tb - 1) / tb;
+    stats_gather_kernel<<<gb, tb, 0, s>>>(a.sel, a.selkey, a.acc, a.fin_out, a.n_blocks);
     BAOC_LAUNCH_CHECK();
     return 0;
 }
 
-int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                              const SelKey* selkey, uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc,
-                              int64_t n_tiles, int n_blocks, const CheckCtx& ck, cudaStream_t s) {
-    return select_rest(blocks, tiles, fin, fin_out, sel, selkey, hist, surv, surv_cnt, acc, n_tiles, n_blocks, 1, ck, s);
-}
+int launch_final_resid_select(const SelectArgs& a, const CheckCtx& ck, cudaStream_t s) { return select_rest(a, 1, ck, s); }
 
-int launch_select_again(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                        const SelKey* selkey, uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc,
-                        int64_t n_tiles, int n_blocks, const CheckCtx& ck, cudaStream_t s) {
-    const int tb = 128, gb = (n_blocks + tb - 1) / tb;
-    select_init_kernel<<<gb, tb, 0, s>>>(blocks, sel, selkey, n_blocks);
+int launch_select_again(const SelectArgs& a, const CheckCtx& ck, cudaStream_t s) {
+    const int tb = 128, gb = (a.n_blocks + tb - 1) / tb;
+    select_init_kernel<<<gb, tb, 0, s>>>(a.blocks, a.sel, a.selkey, a.n_blocks);
     BAOC_LAUNCH_CHECK();
-    const int per = run_tiles(n_tiles, kSelRunTiles);
-    const unsigned grid = unsigned((n_tiles + per - 1) / per);
-    select_first_kernel<<<grid, kThreads, 0, s>>>(blocks, tiles, selkey, hist, n_tiles, per);
+    const int per = run_tiles(a.n_tiles, kSelRunTiles);
+    const unsigned grid = unsigned((a.n_tiles + per - 1) / per);
+    select_first_kernel<<<grid, kThreads, 0, s>>>(a.blocks, a.tiles, a.selkey, a.hist, a.n_tiles, per);
     BAOC_LAUNCH_CHECK();
-    select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, selkey, 0);
+    select_pick_kernel<<<a.n_blocks, kThreads, 0, s>>>(a.sel, a.hist, a.selkey, 0);
     BAOC_LAUNCH_CHECK();
-    return select_rest(blocks, tiles, fin, fin_out, sel, selkey, hist, surv, surv_cnt, acc, n_tiles, n_blocks, 0, ck, s);
+    return select_rest(a, 0, ck, s);
 }
 
 }  // namespace baoc

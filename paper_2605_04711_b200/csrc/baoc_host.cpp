@@ -76,6 +76,32 @@ static size_t take(size_t* cur, size_t bytes) {
     return at;
 }
 
+// Pieces of the select's second sweep, block by block: strips of at most kPieceCols columns, cut into runs of rows of at
+// most kPieceElems elements (a multiple of 16 rows: the CTA's row step at full width).  Sets piece0 / npieces of the
+// blocks and returns the words of the survivors list: one slot per eight elements of a piece.
+void build_sel_pieces(const Handle* h, std::vector<SelPiece>* out, std::vector<StatBlock>* blocks, uint64_t* surv_words) {
+    out->clear();
+    uint64_t off = 0;
+    for (int i = 0; i < h->n_blocks; ++i) {
+        const baoc_block_t& b = h->stat_shapes[i];
+        const int64_t C = b.cols > 1 ? b.cols : kPieceCols;
+        const int64_t R = b.cols > 1 ? b.rows : ceil_div(b.numel, kPieceCols);
+        (*blocks)[i].piece0 = int64_t(out->size());
+        for (int64_t c0 = 0; c0 < C; c0 += kPieceCols) {
+            const int64_t width = std::min<int64_t>(kPieceCols, C - c0);
+            const int64_t rows_per = std::max<int64_t>(16, kPieceElems / width / 16 * 16);
+            for (int64_t r0 = 0; r0 < R; r0 += rows_per) {
+                const int64_t nr = std::min(rows_per, R - r0);
+                const uint32_t slots = uint32_t(round_up(ceil_div(nr * width, 8), 32));
+                out->push_back(SelPiece{uint32_t(i), uint32_t(c0), uint32_t(r0), uint32_t(nr), off, slots, 0u});
+                off += slots;
+            }
+        }
+        (*blocks)[i].npieces = int32_t(int64_t(out->size()) - (*blocks)[i].piece0);
+    }
+    *surv_words = off;
+}
+
 // Statistics workspace: tables, moments, previous gradient, partial sums,
 // per-block accumulators and the scratch of the finalize pass.  Pointers in
 // h_stat_blocks are offsets from a null base until a workspace is bound.
@@ -123,6 +149,10 @@ void compute_stat_layout(Handle* h) {
         }
     }
     h->n_stat_tiles = tiles; h->n_red_tiles = red;
+    std::vector<SelPiece> pieces;
+    uint64_t surv_words = 0;
+    build_sel_pieces(h, &pieces, &h->h_stat_blocks, &surv_words);
+    h->n_sel_pieces = int64_t(pieces.size());
     auto& L = h->sl;
     size_t cur = 0;
     L.blocks = take(&cur, sizeof(StatBlock) * n);
@@ -141,8 +171,10 @@ void compute_stat_layout(Handle* h) {
     L.hist = take(&cur, 4 * size_t(kSelBins) * kRanks * n);
     L.sel = take(&cur, sizeof(RankSel) * size_t(kRanks) * n);
     L.selkey = take(&cur, sizeof(SelKey) * size_t(n));
-    L.surv = take(&cur, 4 * size_t(kSurvTile) * size_t(tiles));
-    L.surv_cnt = take(&cur, 4 * size_t(tiles));
+    L.pieces = take(&cur, sizeof(SelPiece) * pieces.size());
+    L.resid_part = take(&cur, 8 * pieces.size());
+    L.surv = take(&cur, 4 * size_t(surv_words));
+    L.surv_cnt = take(&cur, 4 * pieces.size());
     L.rowsum = take(&cur, 8 * size_t(std::max<int64_t>(sum_rows, 1)));
     L.colsum = take(&cur, 8 * size_t(std::max<int64_t>(sum_cols, 1)));
     L.redpart = take(&cur, 8 * size_t(std::max<int64_t>(redpart, 1)));

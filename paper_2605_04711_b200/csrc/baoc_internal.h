@@ -41,7 +41,8 @@ constexpr int kSelBins = 1 << kSelBits;
 constexpr int kSel3Bits = 32 - 2 * kSelBits;   // bits of the third and last pass
 constexpr int kFinRunTiles = 8;       // most tiles a CTA of the first finalize sweep works through (its partial sums stay in fp32 that long)
 constexpr int kSelRunTiles = 15;      // most tiles a CTA of the other two sweeps works through (their histograms count in 16 bits)
-constexpr int kSurvTile = 512;        // slots per tile in the list of the select's survivors (elements that share a rank's first digit)
+constexpr int kPieceCols = 512;       // widest piece of the select's second sweep, in columns
+constexpr int kPieceElems = 49152;    // most elements of a piece (its histograms count in 16 bits)
 constexpr uint32_t kSurvOverflow = 0xffffffffu;   // count of a run whose survivors did not fit: the last pass reads v instead
 constexpr int kRedRows = 64;          // rows per CTA of the row/column reduction kernel
 constexpr int kRedCols = 512;         // columns per CTA of the row/column reduction kernel
@@ -146,7 +147,7 @@ struct StatBlock {
     int64_t numel;
     int64_t tile0;       // index of the block's first tile
     int32_t rows, cols;
-    int32_t ntiles, pad;
+    int32_t ntiles, npieces;   // tiles of the block; pieces of the select's second sweep (see SelPiece)
     RedGeom red;
     // coordinate sampling: the statistics see the sub-grid rows[ridx] x cols[cidx] of the block (null: the whole block)
     const int64_t* ridx;
@@ -154,6 +155,7 @@ struct StatBlock {
     uint16_t* gsample;   // gathered gradient of the current step, bf16 bits
     float* psample;      // gathered parameters (finalize)
     int64_t full_cols;   // row length of the whole block
+    int64_t piece0;      // index of the block's first piece
 };
 
 // Per-block record of the fused step (device copy lives in the state buffer).
@@ -217,6 +219,19 @@ struct SelKey {
 };
 constexpr int kSelFullS = 31 - kSelBits;   // with lo = -1 the key pattern + 1 of every finite non-negative value fits
 
+// One CTA of the select's second sweep: rows [row0, row0 + nrows) x columns [col0, col0 + min(kPieceCols, cols - col0))
+// of a matrix block; a vector block counts as a matrix of kPieceCols columns (its last row may be short).  The piece's
+// survivors (elements that share a rank's first digit) are listed in surv[surv_off, surv_off + slots).
+struct SelPiece {
+    uint32_t block;
+    uint32_t col0;
+    uint32_t row0;
+    uint32_t nrows;
+    uint64_t surv_off;
+    uint32_t slots;
+    uint32_t pad;
+};
+
 // One CTA of the row/column reduction: a kRedRows x kRedCols piece of a matrix block.
 struct RedTile {
     uint32_t block;
@@ -277,9 +292,10 @@ struct Handle {
     std::vector<const void*> last_stat_grads;
     std::vector<const void*> last_stat_params;
     std::vector<SelKey> selkey_staging;                    // keys of a repeated select (must outlive the async copy)
+    int64_t n_sel_pieces = 0;                              // pieces of the select's second sweep
     int64_t select_retries = 0;                            // blocks whose select was repeated in the last baoc_risk
     struct StatLayout {
-        size_t blocks, tiles, red_tiles, matrix_ids, grads, params, m, v, gprev, partials, acc, fin, fin_out, hist, sel, selkey, surv, surv_cnt,
+        size_t blocks, tiles, red_tiles, matrix_ids, grads, params, m, v, gprev, partials, acc, fin, fin_out, hist, sel, selkey, pieces, resid_part, surv, surv_cnt,
                rowsum, colsum, redpart, ridx, cidx, gsample, psample, sgrads, sparams, total;
     } sl{};
 
@@ -354,6 +370,7 @@ int64_t state_mem_bytes(const baoc_config_t& c, const baoc_block_t& b);
 double step_traffic_bytes(const baoc_config_t& c, const baoc_block_t& b);
 
 void compute_stat_layout(Handle* h);
+void build_sel_pieces(const Handle* h, std::vector<SelPiece>* out, std::vector<StatBlock>* blocks, uint64_t* surv_words);
 
 // Kernel launchers (defined in the .cu files).  Each returns 0 or a cudaError_t value.
 int launch_stats_step(const StatBlock* blocks, const Tile* tiles, const void* const* grads, double* partials,
@@ -365,13 +382,25 @@ int launch_stats_combine(const StatBlock* blocks, const double* partials, double
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
                       double* fin_out, uint32_t* hist, RankSel* sel, SelKey* selkey, int64_t n_tiles, int n_blocks, double eps,
                       float eps_adam, int quantizer8, const CheckCtx& ck, cudaStream_t s);
-int launch_final_resid_select(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                              const SelKey* selkey, uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc,
-                              int64_t n_tiles, int n_blocks, const CheckCtx& ck, cudaStream_t s);
+// The buffers of the select's second and third sweep.
+struct SelectArgs {
+    const StatBlock* blocks;
+    const Tile* tiles;
+    const SelPiece* pieces;
+    RankSel* sel;
+    const SelKey* selkey;
+    uint32_t* hist;
+    uint32_t* surv;
+    uint32_t* surv_cnt;      // per piece: survivors listed, or kSurvOverflow
+    double* resid_part;      // per piece: its part of the Eq. 7 numerator
+    double* fin_out;
+    const double* acc;
+    int64_t n_tiles, n_pieces;
+    int n_blocks;
+};
+int launch_final_resid_select(const SelectArgs& a, const CheckCtx& ck, cudaStream_t s);
 // The select once more, from its first pass, for the blocks whose selkey has s >= 0 (the others keep their results).
-int launch_select_again(const StatBlock* blocks, const Tile* tiles, double* fin, double* fin_out, RankSel* sel,
-                        const SelKey* selkey, uint32_t* hist, uint32_t* surv, uint32_t* surv_cnt, const double* acc,
-                        int64_t n_tiles, int n_blocks, const CheckCtx& ck, cudaStream_t s);
+int launch_select_again(const SelectArgs& a, const CheckCtx& ck, cudaStream_t s);
 int launch_sample_gather(const StatBlock* blocks, const Tile* tiles, const void* const* src, int64_t n_tiles, int fp32,
                          const CheckCtx& ck, cudaStream_t s);
 int launch_moment_reduce(const StatBlock* blocks, const RedTile* rtiles, const int32_t* ids, int64_t n_red, int n_matrix,
