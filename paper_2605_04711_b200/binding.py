@@ -324,13 +324,14 @@ class Baoc:
         self._check(_lib.baoc_read_stats(self._h, out, _stream()))
         return [s.as_dict() for s in out]
 
-    def risk(self, params):
-        """Returns (risk [n_blocks, n_cfg] float64, list of per-block stats dicts)."""
+    def risk(self, params, as_dicts: bool = True):
+        """Returns (risk [n_blocks, n_cfg] float64, list of per-block stats dicts); with as_dicts=False the second item is
+        the array of BlockStats structures as the library filled it (no per-field conversion)."""
         tab = params if isinstance(params, C.Array) else pointer_table(params)
         risk = np.zeros((self.n_blocks, self.n_cfg), np.float64)
         st = (BlockStats * self.n_blocks)()
         self._check(_lib.baoc_risk(self._h, tab, risk.ctypes.data, st, _stream()))
-        return risk, [s.as_dict() for s in st]
+        return risk, ([s.as_dict() for s in st] if as_dicts else st)
 
     def risk_from_raw(self, raw: Sequence[dict]):
         st = (BlockStats * self.n_blocks)()

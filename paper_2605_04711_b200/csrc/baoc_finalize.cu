@@ -102,7 +102,7 @@ final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, double* __re
 // slices ahead (96 bytes per thread and slice: m, v, theta), so loads in flight
 // hold no registers during the long arithmetic of the current slice.
 // ============================================================================
-constexpr int kFsStageBytes = kThreads * 96;                 // m 32 B/thread at 0, v at 8192, theta at 16384
+constexpr int kFsStageBytes = kThreads * 96;                 // m (32 B/thread) at 0, v at 8192, theta at 16384
 constexpr int kFsStages = 3;
 constexpr int kFsSmemBytes = kFsStages * kFsStageBytes + kSelBins * 4 + 4096;   // the staging ring, the histogram of the first digit, the codebook
 
@@ -241,8 +241,10 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
     const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
     const int nsl = int(last - first) * (kTile / (kThreads * 8));     // slices of this CTA
     const uint32_t sm0 = smem_addr(stage);
-    const uint32_t om = threadIdx.x * 32, ov = 8192 + om, ot = 16384 + om;
-    constexpr uint32_t kHalf = 16;                           // a thread's 32 bytes per array are contiguous
+    // a thread's 32 bytes per array as two 16-byte pieces: the lanes' first pieces lie side by side, then their second
+    // pieces, so that a quarter warp's 16-byte accesses cover 128 contiguous bytes (no bank conflicts)
+    const uint32_t om = uint32_t(warp) * 1024u + uint32_t(lane) * 16u, ov = 8192 + om, ot = 16384 + om;
+    constexpr uint32_t kHalf = 512;
 
     for (int i = threadIdx.x; i < kSelBins; i += kThreads) hist1[i] = 0u;
     __syncthreads();
