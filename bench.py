@@ -307,6 +307,7 @@ def run_ours(args):
     ev = lambda: torch.cuda.Event(enable_timing=True)
     for t in range(1, args.window + 1):
         sess.sample_stats(t % 2)
+    sess.h.risk(sess.param_table, as_dicts=False)                    # untimed: the first call also loads the finalize kernels
     e0, e1 = ev(), ev()
     e0.record()
     risk, stats = sess.h.risk(sess.param_table, as_dicts=False)      # the C call alone: it returns after its own copy back

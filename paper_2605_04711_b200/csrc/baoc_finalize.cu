@@ -2,13 +2,15 @@
 // signal-to-noise ratio (Eq. 5), the distortion (Eq. 6), the structure residual
 // (Eq. 7) and the precision cosines (Eq. 8), and the exact quantiles behind the
 // anisotropy (Eq. 4).  Three sweeps over the window's moments:
-//   1. final_sums_kernel   reads m, v, theta: 16 sums per block, and the histogram of the top 12 bits of v
-//   2. final_resid_hist_kernel   reads v: Eq. 7 residual (after the row/column sums), histogram of the next 12 bits of
-//                                the elements that share a rank's top 12 bits, and the list of those elements
-//   3. final_last_kernel         reads that list (a tenth of v or less): histogram of the last 8 bits
-// A CTA works through a run of consecutive tiles, keeps its partial sums and
-// histograms on chip while the tiles belong to one block, and hands them over
-// once per block (a deterministic, fixed partition of the work).
+//   1. final_sums_kernel         reads m, v, theta: 16 sums per block, and the histogram of the top 12 bits of the
+//                                select's key (SelKey: fitted per block to a sample of v by final_pilot_kernel)
+//   2. final_resid_hist_kernel   reads v by pieces (rows of a strip of columns): Eq. 7 residual (after the row/column
+//                                sums), histogram of the next digit of the elements that share a rank's first digit,
+//                                and the list of those elements
+//   3. final_last_kernel         reads those lists (well under a percent of v): histogram of the last digit
+// A CTA of the first sweep works through a run of consecutive tiles, keeps its
+// partial sums and histogram on chip while the tiles belong to one block, and
+// hands them over once per block (a deterministic, fixed partition of the work).
 #include <cstring>
 #include <type_traits>
 

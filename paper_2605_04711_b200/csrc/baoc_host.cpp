@@ -50,12 +50,15 @@ double step_traffic_bytes(const baoc_config_t& c, const baoc_block_t& b) {
     return bytes;
 }
 
-// About 16 * refine row chunks per matrix (never finer than one group of 64 rows).
+// About 16 * refine row chunks per matrix (never finer than one group of 64 rows), and more for a tall matrix: a CTA
+// walks its chunk one group after the other, so a chunk of more than eight groups (an embedding table of tens of
+// thousands of rows cut into 16) would leave a few CTAs running long after the rest of the grid has finished.
 RedGeom red_geometry(int32_t rows, int32_t cols, int refine) {
     RedGeom g{};
     g.rowpart = nullptr; g.colpart = nullptr; g.red0 = -1;
     const int64_t groups = ceil_div(rows, kRedRows);
     g.L = int32_t(std::max<int64_t>(1, ceil_div(groups, std::min<int64_t>(16 * int64_t(refine), groups))));
+    g.L = std::min<int32_t>(g.L, 8);
     g.chunks = int32_t(ceil_div(rows, int64_t(kRedRows) * g.L));
     g.strips = int32_t(ceil_div(cols, kRedCols));
     return g;

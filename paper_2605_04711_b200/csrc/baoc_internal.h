@@ -36,11 +36,11 @@ constexpr int kFinAcc = 20;           //   [20..27] the running window values,
 constexpr int kFinResid = 28;         //   [28] the Eq. 7 numerator,
 constexpr int kFinPilot = 29;         //   [29] the pilot value of the Eq. 6 preconditioner,
 constexpr int kFinFlag = 30;          //   [30] non-zero: an order statistic lies outside the key range of the select
-constexpr int kSelBits = 12;          // bits of the first and of the second radix pass of the quantile select
+constexpr int kSelBits = 12;          // bits of the first and (at most) of the second radix pass of the quantile select
 constexpr int kSelBins = 1 << kSelBits;
-constexpr int kSel3Bits = 32 - 2 * kSelBits;   // bits of the third and last pass
+constexpr int kSel3Bits = 32 - 2 * kSelBits;   // bins of the third and last pass: 2^8 (a key has at most 31 bits: 12 + 12 + 7)
 constexpr int kFinRunTiles = 8;       // most tiles a CTA of the first finalize sweep works through (its partial sums stay in fp32 that long)
-constexpr int kSelRunTiles = 15;      // most tiles a CTA of the other two sweeps works through (their histograms count in 16 bits)
+constexpr int kSelRunTiles = 15;      // tiles a CTA of the stand-alone first pass (a repeated select) works through
 constexpr int kPieceCols = 512;       // widest piece of the select's second sweep, in columns
 constexpr int kPieceElems = 49152;    // most elements of a piece (its histograms count in 16 bits)
 constexpr uint32_t kSurvOverflow = 0xffffffffu;   // count of a run whose survivors did not fit: the last pass reads v instead
