@@ -22,7 +22,7 @@ namespace baoc {
 enum CheckCode : unsigned int { kChkNone = 0, kChkTileIndex = 1, kChkBlockIndex = 2, kChkTileStart = 3, kChkRange = 4, kChkNull = 5 };
 enum CheckKernel : unsigned int {
     kKerStatsStep = 1, kKerStatsCombine = 2, kKerSampleGather = 3, kKerFinalSums = 4, kKerFinalHist = 5, kKerMomentReduce = 6,
-    kKerFactoredReduce = 7, kKerFactoredCombine = 8, kKerFusedStep = 9, kKerSelfTest = 10, kKerFactoredNorms = 11, kKerFinalLast = 12
+    kKerFactoredReduce = 7, kKerFactoredCombine = 8, kKerFusedStep = 9, kKerSelfTest = 10, kKerFactoredNorms = 11, kKerFinalLast = 12, kKerSelectFirst = 13
 };
 #ifdef BAOC_CHECKED
 #define BAOC_CHECK_PARAM , const CheckCtx ck

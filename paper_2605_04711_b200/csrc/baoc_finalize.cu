@@ -874,9 +874,26 @@ __global__ void stats_gather_kernel(const RankSel* __restrict__ sel, const SelKe
 // every element of the blocks that take part.
 __global__ void __launch_bounds__(kThreads)
 select_first_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles, const SelKey* __restrict__ selkey,
-                    uint32_t* __restrict__ hist, int64_t n_tiles, int tiles_per_cta) {
+                    uint32_t* __restrict__ hist, int64_t n_tiles, int tiles_per_cta BAOC_CHECK_PARAM) {
     __shared__ uint32_t sh[kSelBins];
     const int64_t first = int64_t(blockIdx.x) * tiles_per_cta, last = min64(first + tiles_per_cta, n_tiles);
+#ifdef BAOC_CHECKED
+    {
+        if (first >= ck.n_tiles || n_tiles != ck.n_tiles) { check_fail(kChkTileIndex, kKerSelectFirst, first, ck.n_tiles, n_tiles, 0); return; }
+        for (int64_t ti = first; ti < last; ++ti) {
+            const Tile ct = tiles[ti];
+            if (ct.block >= unsigned(ck.n_blocks)) { check_fail(kChkBlockIndex, kKerSelectFirst, ct.block, ck.n_blocks, ti, 0); return; }
+            const StatBlock* cb = blocks + ct.block;
+            const int64_t cbase = int64_t(ct.piece) * kTile;
+            const int64_t cpad = (cb->numel + kQBlock - 1) / kQBlock * kQBlock, cn = min64(kTile, cpad - cbase);
+            if (!check_tile(ck, kKerSelectFirst, ti, ct.block, cbase, cb->numel) ||
+                !check_range(ck, kKerSelectFirst, cb->v + cbase, 4 * cn, 0) ||
+                !check_range(ck, kKerSelectFirst, hist + size_t(ct.block) * kRanks * kSelBins, 4ll * kSelBins, 1) ||
+                !check_range(ck, kKerSelectFirst, selkey + ct.block, int64_t(sizeof(SelKey)), 2))
+                return;
+        }
+    }
+#endif
     for (int i = threadIdx.x; i < kSelBins; i += kThreads) sh[i] = 0u;
     __syncthreads();
 #pragma unroll 1
@@ -980,7 +997,11 @@ int launch_select_again(const SelectArgs& a, const CheckCtx& ck, cudaStream_t s)
     BAOC_LAUNCH_CHECK();
     const int per = run_tiles(a.n_tiles, kSelRunTiles);
     const unsigned grid = unsigned((a.n_tiles + per - 1) / per);
-    select_first_kernel<<<grid, kThreads, 0, s>>>(a.blocks, a.tiles, a.selkey, a.hist, a.n_tiles, per);
+#ifdef BAOC_CHECKED
+    CheckCtx ck_tiles = ck;                                   // this kernel walks tiles, the later sweeps pieces
+    ck_tiles.n_tiles = a.n_tiles;
+#endif
+    select_first_kernel<<<grid, kThreads, 0, s>>>(a.blocks, a.tiles, a.selkey, a.hist, a.n_tiles, per BAOC_CHECK_ARG(ck_tiles));
     BAOC_LAUNCH_CHECK();
     select_pick_kernel<<<a.n_blocks, kThreads, 0, s>>>(a.sel, a.hist, a.selkey, 0);
     BAOC_LAUNCH_CHECK();
