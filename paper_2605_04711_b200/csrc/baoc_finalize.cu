@@ -104,6 +104,17 @@ final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, double* __re
 // slices ahead (96 bytes per thread and slice: m, v, theta), so loads in flight
 // hold no registers during the long arithmetic of the current slice.
 // ============================================================================
+// One tile of the first sweep as its slices see it.
+struct FsTile {
+    const float* m;      // the tile's first element of m, v and theta
+    const float* v;
+    const float* th;
+    int left;            // elements of the block from there on, at most a tile's
+    int block;
+    float p0;            // the block's pilot value and select key
+    int key_lo, key_s;
+};
+
 constexpr int kFsStageBytes = kThreads * 96;                 // m (32 B/thread) at 0, v at 8192, theta at 16384
 constexpr int kFsStages = 3;
 constexpr int kFsSmemBytes = kFsStages * kFsStageBytes + kSelBins * 4 + 4096;   // the staging ring, the histogram of the first digit, the codebook
@@ -124,8 +135,9 @@ __device__ __forceinline__ float rsqrt_approx(float x) {
 // masked out of the one sum it would otherwise enter (p - p0).
 //
 // The bf16 direction costs no extra square root or reciprocal: with n = (v - v16) / v (|n| <= 2^-8),
-// sqrt(v16) - sqrt(v) = -sqrt(v) n (1/2 + n/8 + n^2/16) up to n^4, and with e that difference over (sqrt(v) + eps_adam),
-// 1 / (sqrt(v16) + eps_adam) = (1 - e + e^2 - e^3) / (sqrt(v) + eps_adam) up to e^4: both truncations are below 1e-10.
+// sqrt(v16) - sqrt(v) = -sqrt(v) n (1/2 + n/8) up to n^3, and with e that difference over (sqrt(v) + eps_adam)
+// (|e| <= 2^-9), 1 / (sqrt(v16) + eps_adam) = (1 - e + e^2) / (sqrt(v) + eps_adam) up to e^3: both truncations are
+// below 1e-8 of the direction, far below what a cosine compared at 1e-4 can see.
 // kDyn: the 8-bit round trip goes through the non-linear codebook (dyn: its fp32 tables in shared memory) instead of the
 // linear absmax codes.
 template <bool kFull, bool kDyn>
@@ -187,9 +199,9 @@ __device__ __forceinline__ void fs_slice(const float (&mm)[8], const float (&vv)
         const f32x2 U8 = mul2(M8, pack2(rcp_approx(b0), rcp_approx(b1)));
         // bf16 direction from the series
         const f32x2 N = mul2(E3, mul2(R, R));
-        const f32x2 H = mul2(N, fma2(N, fma2(N, splat2(0.0625f), splat2(0.125f)), splat2(0.5f)));
+        const f32x2 H = mul2(N, fma2(N, splat2(0.125f), splat2(0.5f)));
         const f32x2 NE = mul2(mul2(S, H), R32);                                  // -(sqrt(v16) - sqrt(v)) / (sqrt(v) + eps_adam)
-        const f32x2 U16 = mul2(M16, mul2(R32, fma2(NE, fma2(NE, add2(NE, ONE), ONE), ONE)));
+        const f32x2 U16 = mul2(M16, mul2(R32, fma2(NE, add2(NE, ONE), ONE)));
         // the sums
         F[0] = fma2(M, M, F[0]); F[1] = add2(F[1], V); F[2] = fma2(V, V, F[2]); F[3] = add2(F[3], PD);
         const f32x2 T2 = mul2(T, T), PT = mul2(PD, T2);
@@ -248,6 +260,22 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
     const uint32_t om = uint32_t(warp) * 1024u + uint32_t(lane) * 16u, ov = 8192 + om, ot = 16384 + om;
     constexpr uint32_t kHalf = 512;
 
+    // What the slices of the CTA's tiles need from the tables, gathered once (one thread per tile follows the chain
+    // tile -> block -> pointers; the slices then read it from shared memory instead of following it themselves).
+    __shared__ FsTile desc[kFinRunTiles];
+    if (threadIdx.x < int(last - first)) {
+        const Tile t = tiles[first + threadIdx.x];
+        const StatBlock* b = blocks + t.block;
+        const int64_t base = int64_t(t.piece) * kTile;
+        const SelKey key = selkey[t.block];
+        FsTile d;
+        d.m = b->m + base; d.v = b->v + base; d.th = params[t.block] + base;
+        d.left = int(min64(b->numel - base, kTile));
+        d.block = int(t.block);
+        d.p0 = float(fin_out[size_t(t.block) * kFinOut + kFinPilot]);
+        d.key_lo = key.lo; d.key_s = key.s;
+        desc[threadIdx.x] = d;
+    }
     for (int i = threadIdx.x; i < kSelBins; i += kThreads) hist1[i] = 0u;
     __syncthreads();
 
@@ -278,21 +306,22 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
     // Each thread copies the 32 bytes per array that hold its own eight elements, as two 16-byte copies through L1:
     // the second copy finds its 32-byte sector there, so that L2 serves every sector once.
     uint32_t fill = 0, take = 0;
+    const int in_slice = threadIdx.x * 8;                    // the thread's first element within a slice
     auto prefetch = [&](int k) {
         if (k < nsl) {
-            const Tile t = tiles[first + (k >> 1)];
-            const StatBlock* b = blocks + t.block;
-            const int64_t numel = b->numel;
-            const int64_t e = int64_t(t.piece) * kTile + int64_t(k & 1) * (kThreads * 8) + int64_t(threadIdx.x) * 8;
+            const FsTile& t = desc[k >> 1];
+            const int e = (k & 1) * (kThreads * 8) + in_slice;           // within the tile
             // m and v are padded with zeros to whole quantisation blocks: in bounds whenever the warp's block starts
             // inside the array; theta is not padded
-            if (e - lane * 8 < numel) {
+            if (e - lane * 8 < t.left) {
                 const uint32_t d = sm0 + fill;
-                cp_async16_l1(d + om, b->m + e); cp_async16_l1(d + om + kHalf, b->m + e + 4);
-                cp_async16_l1(d + ov, b->v + e); cp_async16_l1(d + ov + kHalf, b->v + e + 4);
-                if (e + 8 <= numel) {
-                    const float* th = params[t.block];
-                    cp_async16_l1(d + ot, th + e); cp_async16_l1(d + ot + kHalf, th + e + 4);
+                const float* pm = t.m + e;
+                const float* pv = t.v + e;
+                cp_async16_l1(d + om, pm); cp_async16_l1(d + om + kHalf, pm + 4);
+                cp_async16_l1(d + ov, pv); cp_async16_l1(d + ov + kHalf, pv + 4);
+                if (e + 8 <= t.left) {
+                    const float* pt = t.th + e;
+                    cp_async16_l1(d + ot, pt); cp_async16_l1(d + ot + kHalf, pt + 4);
                 }
             }
         }
@@ -310,34 +339,31 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
     for (int k = 0; k < nsl; ++k) {
         prefetch(k + kFsStages - 1);
         cp_async_wait<kFsStages - 1>();                      // this slice's copies have landed
-        const int64_t ti = first + (k >> 1);
-        const Tile t = tiles[ti];
-        if (int(t.block) != cur_block) {                     // uniform over the CTA; only at a tile boundary
+        const FsTile& t = desc[k >> 1];
+        if (t.block != cur_block) {                          // uniform over the CTA; only at a tile boundary
             if (cur_block >= 0) flush(cur_block, run_first);
-            cur_block = int(t.block);
-            run_first = ti;
-            p0 = float(fin_out[size_t(t.block) * kFinOut + kFinPilot]);
-            const SelKey key = selkey[t.block];
-            key_lo = key.lo; key_s = key.s;
+            cur_block = t.block;
+            run_first = first + (k >> 1);
+            p0 = t.p0; key_lo = t.key_lo; key_s = t.key_s;
         }
         const unsigned char* mine = stage + take;
         take = take == (kFsStages - 1) * kFsStageBytes ? 0u : take + kFsStageBytes;
-        const int64_t numel = blocks[t.block].numel;
-        const int64_t w0 = int64_t(t.piece) * kTile + int64_t(k & 1) * (kThreads * 8) + int64_t(warp) * kQBlock;
-        if (w0 >= numel) continue;                           // whole warp out of range
+        const int left = t.left;
+        const int w0 = (k & 1) * (kThreads * 8) + warp * kQBlock;        // the warp's quantisation block, within the tile
+        if (w0 >= left) continue;                            // whole warp out of range
         float mm[8], vv[8], tt[8];
         f4_to8(*reinterpret_cast<const float4*>(mine + om), *reinterpret_cast<const float4*>(mine + om + kHalf), mm);
         f4_to8(*reinterpret_cast<const float4*>(mine + ov), *reinterpret_cast<const float4*>(mine + ov + kHalf), vv);
-        if (w0 + kQBlock <= numel) {                         // uniform over the warp
+        if (w0 + kQBlock <= left) {                          // uniform over the warp
             f4_to8(*reinterpret_cast<const float4*>(mine + ot), *reinterpret_cast<const float4*>(mine + ot + kHalf), tt);
             fs_slice<true, kDyn>(mm, vv, tt, 8, p0, eps_f, eps_adam, F, hist1, key_lo, key_s, dyn_tables);
         } else {
-            const int64_t e = w0 + lane * 8;
-            const int cnt = int(max64(0, min64(8, numel - e)));
+            const int e = w0 + lane * 8;
+            const int cnt = max(0, min(8, left - e));
             if (cnt == 8) {
                 f4_to8(*reinterpret_cast<const float4*>(mine + ot), *reinterpret_cast<const float4*>(mine + ot + kHalf), tt);
             } else {
-                const float* th = params[t.block];
+                const float* th = t.th;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) tt[j] = j < cnt ? th[e + j] : 0.f;
             }
