@@ -618,72 +618,86 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const SelPiece* __
     const uint32_t* __restrict__ vp = v + (int64_t(pc.row0) + g.ty) * g.cols + pc.col0 + g.tx * 8;
     const int64_t v_step = int64_t(g.step) * g.cols;
 
-    // one row of the thread: kWide: all eight elements exist
-    auto row = [&](auto wide_tag, uint32_t (&u)[8], int n, double rsum) {
-        constexpr bool kWide = decltype(wide_tag)::value;
-        if (resid) {
-            const double a = rsum * inv_total;
+    // The walk over the piece's rows, compiled once per combination of what the whole CTA does or does not do
+    // (kResid: Eq. 7; kKeys: this pass has a digit to find; kInner: the cheap survivor test applies), so that none of
+    // it is decided again for every row.
+    auto rows = [&](auto resid_tag, auto keys_tag, auto inner_tag) {
+        constexpr bool kResid = decltype(resid_tag)::value, kKeys = decltype(keys_tag)::value, kInner = decltype(inner_tag)::value;
+        // one row of the thread: kWide: all eight elements exist
+        auto row = [&](auto wide_tag, uint32_t (&u)[8], int n, double rsum) {
+            constexpr bool kWide = decltype(wide_tag)::value;
+            if (kResid) {
+                const double a = rsum * inv_total;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (kWide || j < n) {
-                    const double d = fma(-a, cs[j], double(__uint_as_float(u[j])));
-                    acc[0] = fma(d, d, acc[0]);
+                for (int j = 0; j < 8; ++j) {
+                    if (kWide || j < n) {
+                        const double d = fma(-a, cs[j], double(__uint_as_float(u[j])));
+                        acc[0] = fma(d, d, acc[0]);
+                    }
                 }
             }
-        }
-        if (d_bits == 0) return;
-        uint32_t mask = 0u;
-        if (inner) {
+            if (!kKeys) return;
+            uint32_t mask = 0u;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const bool p = (kWide || j < n) & ((u[j] - base0 < span) | (u[j] - base1 < span));
-                if (p) mask |= 1u << j;
+                bool p;
+                if (kInner) {
+                    p = (u[j] - base0 < span) | (u[j] - base1 < span);
+                } else {
+                    const uint32_t top = sel_key(u[j], key.lo, wmax) >> key.s;
+                    p = (top == L.key[0]) | (top == L.key[1]) | (top == L.key[2]) | (top == L.key[3]);
+                }
+                if ((kWide || j < n) && p) mask |= 1u << j;
             }
-        } else {
+            if (mask) {                                       // few threads
+                int pos = atomicAdd(&wcnt[warp], __popc(mask));
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint32_t top = sel_key(u[j], key.lo, wmax) >> key.s;
-                const bool p = (kWide || j < n) & ((top == L.key[0]) | (top == L.key[1]) | (top == L.key[2]) | (top == L.key[3]));
-                if (p) mask |= 1u << j;
+                for (int j = 0; j < 8; ++j)
+                    if (mask & (1u << j)) seg[pos++] = sel_key(u[j], key.lo, wmax);
             }
-        }
-        if (mask) {                                           // few threads
-            int pos = atomicAdd(&wcnt[warp], __popc(mask));
+        };
+#pragma unroll 1
+        for (int64_t r0 = int64_t(pc.row0); r0 < r_end; r0 += int64_t(kRhBatch) * g.step) {   // the same trips for every thread
+            uint32_t u[kRhBatch][8];
+            int n[kRhBatch];
+            double rs[kRhBatch];
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (mask & (1u << j)) seg[pos++] = sel_key(u[j], key.lo, wmax);
+            for (int k = 0; k < kRhBatch; ++k) {
+                const int64_t r = r0 + g.ty + int64_t(k) * g.step;
+                n[k] = 0;
+                rs[k] = 0.0;
+                if (r < r_end) {
+                    if (wide && r != short_row) {
+                        const uint4 a = ld_stream_u4(vp + k * v_step), c = ld_stream_u4(vp + k * v_step + 4);
+                        u[k][0] = a.x; u[k][1] = a.y; u[k][2] = a.z; u[k][3] = a.w; u[k][4] = c.x; u[k][5] = c.y; u[k][6] = c.z; u[k][7] = c.w;
+                        n[k] = 8;
+                    } else {
+                        n[k] = piece_load(v, pc, g, numel, r, u[k]);
+                    }
+                    if (kResid) rs[k] = __ldg(rowsum + r);
+                }
+            }
+            vp += kRhBatch * v_step;
+#pragma unroll
+            for (int k = 0; k < kRhBatch; ++k) {
+                if (n[k] == 8) row(std::true_type{}, u[k], 8, rs[k]);
+                else if (n[k] > 0) row(std::false_type{}, u[k], n[k], rs[k]);
+            }
+            if (kKeys) {
+                __syncwarp();
+                if (wcnt[warp] > kRhDrainAt) drain();         // uniform over the warp: room for the next batch
+            }
         }
     };
-
-#pragma unroll 1
-    for (int64_t r0 = int64_t(pc.row0); r0 < r_end; r0 += int64_t(kRhBatch) * g.step) {   // the same trips for every thread
-        uint32_t u[kRhBatch][8];
-        int n[kRhBatch];
-        double rs[kRhBatch];
-#pragma unroll
-        for (int k = 0; k < kRhBatch; ++k) {
-            const int64_t r = r0 + g.ty + int64_t(k) * g.step;
-            n[k] = 0;
-            rs[k] = 0.0;
-            if (r < r_end) {
-                if (wide && r != short_row) {
-                    const uint4 a = ld_stream_u4(vp + k * v_step), c = ld_stream_u4(vp + k * v_step + 4);
-                    u[k][0] = a.x; u[k][1] = a.y; u[k][2] = a.z; u[k][3] = a.w; u[k][4] = c.x; u[k][5] = c.y; u[k][6] = c.z; u[k][7] = c.w;
-                    n[k] = 8;
-                } else {
-                    n[k] = piece_load(v, pc, g, numel, r, u[k]);
-                }
-                if (resid) rs[k] = __ldg(rowsum + r);
-            }
-        }
-        vp += kRhBatch * v_step;
-#pragma unroll
-        for (int k = 0; k < kRhBatch; ++k) {
-            if (n[k] == 8) row(std::true_type{}, u[k], 8, rs[k]);
-            else if (n[k] > 0) row(std::false_type{}, u[k], n[k], rs[k]);
-        }
-        __syncwarp();
-        if (wcnt[warp] > kRhDrainAt) drain();                 // uniform over the warp: room for the next batch
+    const std::true_type yes{};
+    const std::false_type no{};
+    if (resid) {                                              // all uniform over the CTA
+        if (d_bits == 0) rows(yes, no, no);
+        else if (inner) rows(yes, yes, yes);
+        else rows(yes, yes, no);
+    } else {
+        if (inner) rows(no, yes, yes);
+        else rows(no, yes, no);
     }
     __syncwarp();
     drain();
