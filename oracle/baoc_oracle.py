@@ -66,6 +66,8 @@ class Opts:
     eps_adam: float = 1e-8         # epsilon of the update direction in Eq. 8
     qblock: int = 256              # elements per quantisation block
     quantizer8: str = "linear"     # the 8-bit quantiser of Eq. 8: "linear" absmax codes or the "dynamic" codebook
+    debias: bool = False           # alternative reading of the hats in Eq. 3: the diagnostics of Eq. 4-8 are taken from
+                                   # the bias-corrected moments m / (1 - beta_m^T), v / (1 - beta_v^T) after T steps
 
 
 @dataclass
@@ -348,24 +350,33 @@ def quant_rel_error(x: np.ndarray, bits: int, signed: bool, o: Opts) -> float:
     return float(np.linalg.norm(x - xq)) / n if n > 0.0 else 0.0
 
 
+def window_moments(st: StatsState, o: Opts) -> Tuple[np.ndarray, np.ndarray]:
+    """The moments the end-of-window diagnostics are taken from: the recursion of Eq. 3 as it stands, or (o.debias) with
+    Adam's bias correction for the st.t steps observed, m / (1 - beta_m^t) and v / (1 - beta_v^t)."""
+    if o.debias and st.t > 0:
+        return st.m / (1.0 - o.beta_m ** st.t), st.v / (1.0 - o.beta_v ** st.t)
+    return st.m, st.v
+
+
 def stats_finalize(st: StatsState, theta: np.ndarray, rows: int, cols: int, o: Opts) -> Dict[str, float]:
     """Raw diagnostics z_i of one block at the end of the window."""
+    m, v = window_moments(st, o)
     return {
-        "A": anisotropy(st.v, o.eps),
+        "A": anisotropy(v, o.eps),
         "rho_bar": st.rho_bar,
-        "snr": snr(st.m, st.v, o.eps),
-        "C": distortion(st.v, theta, o.eps),
-        "F": structure_residual(st.v, rows, cols, o.eps),
-        "Q32": precision_cosine(st.m, st.v, 32, o),
-        "Q16": precision_cosine(st.m, st.v, 16, o),
-        "Q8": precision_cosine(st.m, st.v, 8, o),
-        "q10": quantile_linear(st.v, 0.1),
-        "q90": quantile_linear(st.v, 0.9),
+        "snr": snr(m, v, o.eps),
+        "C": distortion(v, theta, o.eps),
+        "F": structure_residual(v, rows, cols, o.eps),
+        "Q32": precision_cosine(m, v, 32, o),
+        "Q16": precision_cosine(m, v, 16, o),
+        "Q8": precision_cosine(m, v, 8, o),
+        "q10": quantile_linear(v, 0.1),
+        "q90": quantile_linear(v, 0.9),
         "rho_mom": st.rho_mom,
-        "err_m8": quant_rel_error(st.m, 8, True, o),
-        "err_v8": quant_rel_error(st.v, 8, False, o),
-        "err_m16": quant_rel_error(st.m, 16, True, o),
-        "err_v16": quant_rel_error(st.v, 16, False, o),
+        "err_m8": quant_rel_error(m, 8, True, o),
+        "err_v8": quant_rel_error(v, 8, False, o),
+        "err_m16": quant_rel_error(m, 16, True, o),
+        "err_v16": quant_rel_error(v, 16, False, o),
     }
 
 

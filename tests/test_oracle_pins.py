@@ -110,6 +110,45 @@ def test_constant_gradient_closed_forms(T):
     assert abs(O.snr(st.m, st.v, o.eps) / want - 1.0) < 1e-9
 
 
+@pytest.mark.parametrize("T", [1, 5, 32])
+def test_debiased_window_moments_closed_forms(T):
+    """The alternative reading of the hats in Eq. 3 (Opts.debias): a constant gradient g gives m / (1 - beta_m^T) = g and
+    v / (1 - beta_v^T) = g^2 exactly, so the diagnostics are those of (g, g^2): SNR = sum g^2 / (sum g^2 + eps), every
+    element of the direction has modulus |g| / (|g| + eps_adam), and the quantiles are those of g^2.  With the option
+    off the same window gives the raw closed forms of the test above: the two readings differ."""
+    o = O.Opts(debias=True)
+    g = RNG.standard_normal(257)
+    st = _run_window([g] * T, o)
+    m, v = O.window_moments(st, o)
+    np.testing.assert_allclose(m, g, rtol=1e-12)
+    np.testing.assert_allclose(v, g * g, rtol=1e-12)
+    raw = O.stats_finalize(st, np.ones(257), 257, 1, o)
+    s2 = float(np.sum(g * g))
+    assert abs(raw["snr"] / (s2 / (s2 + o.eps)) - 1.0) < 1e-9
+    assert abs(raw["q10"] / np.quantile(g * g, 0.1) - 1.0) < 1e-9 and abs(raw["q90"] / np.quantile(g * g, 0.9) - 1.0) < 1e-9
+    assert abs(raw["A"] - math.log((np.quantile(g * g, 0.9) + o.eps) / (np.quantile(g * g, 0.1) + o.eps))) < 1e-9
+    off = O.stats_finalize(st, np.ones(257), 257, 1, O.Opts())
+    want_off = (1 - o.beta_m ** T) ** 2 / (1 - o.beta_v ** T)
+    assert abs(off["snr"] / want_off - 1.0) < 1e-9
+    if T > 1:
+        assert abs(off["snr"] - raw["snr"]) > 1e-3
+    # the correction is a positive rescaling of each moment: the anisotropy of Eq. 4 changes only through eps
+    assert abs(off["A"] - raw["A"]) < 1e-6
+
+
+def test_debias_uses_the_steps_observed_and_leaves_an_empty_window_alone():
+    o = O.Opts(debias=True)
+    st = O.stats_init(4)
+    m, v = O.window_moments(st, o)
+    assert np.all(m == 0.0) and np.all(v == 0.0)                 # no step, no division by 1 - beta^0 = 0
+    g1, g2 = np.array([1.0, -2.0, 0.5, 4.0]), np.array([0.0, 1.0, -1.0, 2.0])
+    O.stats_step(st, g1, o); O.stats_step(st, g2, o)
+    m, v = O.window_moments(st, o)
+    bm, bv = o.beta_m, o.beta_v
+    np.testing.assert_allclose(m, ((1 - bm) * bm * g1 + (1 - bm) * g2) / (1 - bm ** 2), rtol=1e-14)
+    np.testing.assert_allclose(v, ((1 - bv) * bv * g1 ** 2 + (1 - bv) * g2 ** 2) / (1 - bv ** 2), rtol=1e-14)
+
+
 def test_moments_match_explicit_weighted_sums():
     o = O.Opts()
     gs = [RNG.standard_normal(50) for _ in range(7)]
