@@ -134,7 +134,9 @@ typedef struct {
     int32_t qblock;               /* elements per 8-bit quantisation block */
     int64_t node_limit;           /* allocator search-node limit (0 = default) */
     int32_t quantizer8;           /* the 8-bit quantiser of Eq. 8: BAOC_Q_LINEAR (default) or BAOC_Q_DYNAMIC */
-    int32_t reserved;             /* 0 */
+    int32_t debias;               /* 0 (default): the diagnostics of Eq. 4-8 are taken from the recursion of Eq. 3 as it
+                                   * stands; 1: from the bias-corrected moments m / (1 - beta_m^T), v / (1 - beta_v^T)
+                                   * after the T gradients observed (the alternative reading of the hats in Eq. 3) */
 } baoc_opts_t;
 
 /* Per-block diagnostics z_i: raw (Eq. 4-8), normalised (Eq. 10-20) and a few

@@ -55,7 +55,7 @@ class Opts(C.Structure):
                 ("a_lo", C.c_double), ("a_hi", C.c_double), ("rho_lo", C.c_double), ("rho_hi", C.c_double),
                 ("snr_lo", C.c_double), ("snr_hi", C.c_double), ("w", C.c_double * 5), ("gamma", C.c_double),
                 ("eps_adam", C.c_double), ("use_snr", C.c_int32), ("qblock", C.c_int32), ("node_limit", C.c_int64),
-                ("quantizer8", C.c_int32), ("reserved", C.c_int32)]
+                ("quantizer8", C.c_int32), ("debias", C.c_int32)]
 
 
 class BlockStats(C.Structure):

@@ -386,9 +386,14 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
                "sample_gather_kernel");
         h->launches += 1;
     }
+    // The alternative reading of the hats in Eq. 3: Adam's bias correction for the steps observed.  A positive factor per
+    // moment: the first sweep applies it as it loads m and v; the order statistics and the Eq. 7 residual, which are
+    // taken from v as stored, are scaled on the host.
+    const double m_scale = h->opts.debias ? 1.0 / (1.0 - std::pow(h->opts.beta_m, double(h->stats_steps))) : 1.0;
+    const double v_scale = h->opts.debias ? 1.0 / (1.0 - std::pow(h->opts.beta_v, double(h->stats_steps))) : 1.0;
     LAUNCH(launch_final_sums(blocks, tiles, dparams, at<double>(ws, L.fin), at<double>(ws, L.fin_out), at<uint32_t>(ws, L.hist),
                              at<RankSel>(ws, L.sel), at<SelKey>(ws, L.selkey), h->n_stat_tiles, n, h->opts.eps, float(h->opts.eps_adam),
-                             h->opts.quantizer8, ws_ctx(h, h->n_stat_tiles), s),
+                             h->opts.quantizer8, h->opts.debias, float(m_scale), float(v_scale), ws_ctx(h, h->n_stat_tiles), s),
            "final_sums_kernel");
     h->launches += 5;
     if (h->n_matrix > 0) {
@@ -440,7 +445,7 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
         for (int k = 0; k < 2; ++k) {
             const double pos = qs[k] * double(b.numel - 1);
             const double frac = pos - std::floor(pos);
-            const double lo = o[kFinRanks + 2 * k], hi = o[kFinRanks + 2 * k + 1];
+            const double lo = o[kFinRanks + 2 * k] * v_scale, hi = o[kFinRanks + 2 * k + 1] * v_scale;   // the select ran on v as stored
             qv[k] = lo + frac * (hi - lo);
         }
         z.q10 = qv[0]; z.q90 = qv[1];
@@ -453,7 +458,7 @@ int baoc_risk(baoc_t* h, const float* const* params, double* risk_out, baoc_bloc
             const double num2 = std::max(0.0, o[15] - 2.0 * delta * o[14] + delta * delta * o[4]);
             z.C = pbar > 0.0 ? (std::sqrt(num2) / pbar) / (std::sqrt(o[4]) + eps) : 0.0;
         }
-        z.F = b.cols > 1 ? std::sqrt(o[kFinResid]) / (std::sqrt(o[2]) + eps) : 1.0;   // Eq. 7
+        z.F = b.cols > 1 ? (std::sqrt(o[kFinResid]) * v_scale) / (std::sqrt(o[2]) + eps) : 1.0;   // Eq. 7 (the residual sweep ran on v as stored)
         z.Q32 = cosine(o[5], o[5], o[5]);                                   // Eq. 8
         z.Q16 = cosine(o[9], o[5], o[8]);
         z.Q8 = cosine(o[7], o[5], o[6]);

@@ -46,7 +46,8 @@ __device__ __forceinline__ void sel_digit(int s, int pass, int& shift, int& bits
 // Also the key of the block's select: lo one below the smallest pattern of the sample, s the smallest shift for which
 // the largest pattern of the sample stays below the top of the key range.
 __global__ void __launch_bounds__(kThreads)
-final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, double* __restrict__ fin_out, SelKey* __restrict__ selkey) {
+final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, float v_scale, double* __restrict__ fin_out,
+                   SelKey* __restrict__ selkey) {
     __shared__ double total[1];
     __shared__ int s_min, s_max;
     const StatBlock* b = blocks + blockIdx.x;
@@ -59,7 +60,7 @@ final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, double* __re
     int lo = 0x7f800000, hi = 0;
     for (int64_t k = threadIdx.x; k < n; k += kThreads) {
         const float x = b->v[k * stride];
-        acc[0] += double(precond_of(x, eps));
+        acc[0] += double(precond_of(x * v_scale, eps));          // (the key is fitted to v as stored: a positive factor keeps the order)
         const int pat = min(max(__float_as_int(x), 0), 0x7f800000);
         lo = min(lo, pat); hi = max(hi, pat);
     }
@@ -140,10 +141,22 @@ __device__ __forceinline__ float rsqrt_approx(float x) {
 // below 1e-8 of the direction, far below what a cosine compared at 1e-4 can see.
 // kDyn: the 8-bit round trip goes through the non-linear codebook (dyn: its fp32 tables in shared memory) instead of the
 // linear absmax codes.
-template <bool kFull, bool kDyn>
-__device__ __forceinline__ void fs_slice(const float (&mm)[8], const float (&vv)[8], const float (&tt)[8], int cnt,
+// kDebias: m and v are multiplied by m_scale and v_scale first (the select's digit is taken from v as stored).
+template <bool kFull, bool kDyn, bool kDebias>
+__device__ __forceinline__ void fs_slice(float (&mm)[8], float (&vv)[8], const float (&tt)[8], int cnt,
                                          float p0, float eps_f, float eps_adam, f32x2 (&F)[kFinalSums], uint32_t* hist1,
-                                         int key_lo, int key_s, const float* dyn) {
+                                         int key_lo, int key_s, float m_scale, float v_scale, const float* dyn) {
+    // ---- first radix pass of the quantile select: the top 12 bits of the block's key (see SelKey).  The key range is
+    // fitted to the block, so its second moments spread over most of the 4096 bins and a plain shared-memory histogram
+    // with one atomic per element meets few collisions.
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        if (kFull || j < cnt)
+            atomicAdd(hist1 + min(__viaddmax_s32_relu(__float_as_int(vv[j]), -key_lo, 0) >> key_s, kSelBins - 1), 1u);
+    if (kDebias) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { mm[j] *= m_scale; vv[j] *= v_scale; }
+    }
     const f32x2 P0 = splat2(p0), MAGIC = splat2(12582912.0f), C16 = splat2(65537.0f), EA = splat2(eps_adam), EPS = splat2(eps_f),
                 ONE = splat2(1.0f), MONE = splat2(-1.0f);
     // ---- absmax of the warp's quantisation block, code scales
@@ -210,22 +223,14 @@ __device__ __forceinline__ void fs_slice(const float (&mm)[8], const float (&vv)
         F[8] = fma2(U16, U16, F[8]); F[9] = fma2(U32, U16, F[9]);
         F[10] = fma2(E0, E0, F[10]); F[11] = fma2(E1, E1, F[11]); F[12] = fma2(E2, E2, F[12]); F[13] = fma2(E3, E3, F[13]);
     }
-
-    // ---- first radix pass of the quantile select: the top 12 bits of the block's key (see SelKey).  The key range is
-    // fitted to the block, so its second moments spread over most of the 4096 bins and a plain shared-memory histogram
-    // with one atomic per element meets few collisions.
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-        if (kFull || j < cnt)
-            atomicAdd(hist1 + min(__viaddmax_s32_relu(__float_as_int(vv[j]), -key_lo, 0) >> key_s, kSelBins - 1), 1u);
 }
 
-template <bool kDyn>
+template <bool kDyn, bool kDebias>
 __global__ void __launch_bounds__(kThreads, 2)
 final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__ tiles,
                   const float* const* __restrict__ params, double* __restrict__ fin,
                   const double* __restrict__ fin_out, uint32_t* __restrict__ hist, const SelKey* __restrict__ selkey,
-                  int64_t n_tiles, int tiles_per_cta, float eps_f, float eps_adam BAOC_CHECK_PARAM) {
+                  int64_t n_tiles, int tiles_per_cta, float eps_f, float eps_adam, float m_scale, float v_scale BAOC_CHECK_PARAM) {
 #ifdef BAOC_CHECKED
     {   // validate every tile of this CTA's run, and the ranges of the workspace it will touch, before touching anything
         const int64_t c0 = int64_t(blockIdx.x) * tiles_per_cta, c1 = min64(c0 + tiles_per_cta, n_tiles);
@@ -356,7 +361,7 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
         f4_to8(*reinterpret_cast<const float4*>(mine + ov), *reinterpret_cast<const float4*>(mine + ov + kHalf), vv);
         if (w0 + kQBlock <= left) {                          // uniform over the warp
             f4_to8(*reinterpret_cast<const float4*>(mine + ot), *reinterpret_cast<const float4*>(mine + ot + kHalf), tt);
-            fs_slice<true, kDyn>(mm, vv, tt, 8, p0, eps_f, eps_adam, F, hist1, key_lo, key_s, dyn_tables);
+            fs_slice<true, kDyn, kDebias>(mm, vv, tt, 8, p0, eps_f, eps_adam, F, hist1, key_lo, key_s, m_scale, v_scale, dyn_tables);
         } else {
             const int e = w0 + lane * 8;
             const int cnt = max(0, min(8, left - e));
@@ -367,7 +372,7 @@ final_sums_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
 #pragma unroll
                 for (int j = 0; j < 8; ++j) tt[j] = j < cnt ? th[e + j] : 0.f;
             }
-            fs_slice<false, kDyn>(mm, vv, tt, cnt, p0, eps_f, eps_adam, F, hist1, key_lo, key_s, dyn_tables);
+            fs_slice<false, kDyn, kDebias>(mm, vv, tt, cnt, p0, eps_f, eps_adam, F, hist1, key_lo, key_s, m_scale, v_scale, dyn_tables);
         }
     }
     cp_async_wait<0>();
@@ -974,29 +979,38 @@ static int run_tiles(int64_t n_tiles, int most) {
     return int(want < 1 ? 1 : (want > most ? most : want));
 }
 
+template <bool kDyn, bool kDebias>
+static cudaError_t launch_sums_instance(unsigned grid, const StatBlock* blocks, const Tile* tiles, const float* const* params,
+                                        double* fin, const double* fin_out, uint32_t* hist, const SelKey* selkey, int64_t n_tiles,
+                                        int per, float eps, float eps_adam, float m_scale, float v_scale, const CheckCtx& ck,
+                                        cudaStream_t s) {
+    (void)ck;
+    cudaError_t e = cudaFuncSetAttribute(final_sums_kernel<kDyn, kDebias>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes);
+    if (e != cudaSuccess) return e;
+    final_sums_kernel<kDyn, kDebias><<<grid, kThreads, kFsSmemBytes, s>>>(blocks, tiles, params, fin, fin_out, hist, selkey, n_tiles,
+                                                                            per, eps, eps_adam, m_scale, v_scale BAOC_CHECK_ARG(ck));
+    return cudaGetLastError();
+}
+
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
                       double* fin_out, uint32_t* hist, RankSel* sel, SelKey* selkey, int64_t n_tiles, int n_blocks, double eps,
-                      float eps_adam, int quantizer8, const CheckCtx& ck, cudaStream_t s) {
-    (void)ck;
+                      float eps_adam, int quantizer8, int debias, float m_scale, float v_scale, const CheckCtx& ck, cudaStream_t s) {
     const int tb = 128, gb = (n_blocks + tb - 1) / tb;
     cudaError_t e = cudaMemsetAsync(hist, 0, size_t(n_blocks) * kRanks * kSelBins * sizeof(uint32_t), s);
     if (e != cudaSuccess) return int(e);
     select_init_kernel<<<gb, tb, 0, s>>>(blocks, sel, nullptr, n_blocks);
     BAOC_LAUNCH_CHECK();
-    final_pilot_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, float(eps), fin_out, selkey);
+    final_pilot_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, float(eps), debias ? v_scale : 1.0f, fin_out, selkey);
     BAOC_LAUNCH_CHECK();
-    e = cudaFuncSetAttribute(final_sums_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(final_sums_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes);
-    if (e != cudaSuccess) return int(e);
     const int per = run_tiles(n_tiles, kFinRunTiles);
     const unsigned grid = unsigned((n_tiles + per - 1) / per);
     if (quantizer8)
-        final_sums_kernel<true><<<grid, kThreads, kFsSmemBytes, s>>>(blocks, tiles, params, fin, fin_out, hist, selkey, n_tiles,
-                                                                       per, float(eps), eps_adam BAOC_CHECK_ARG(ck));
+        e = debias ? launch_sums_instance<true, true>(grid, blocks, tiles, params, fin, fin_out, hist, selkey, n_tiles, per, float(eps), eps_adam, m_scale, v_scale, ck, s)
+                   : launch_sums_instance<true, false>(grid, blocks, tiles, params, fin, fin_out, hist, selkey, n_tiles, per, float(eps), eps_adam, 1.f, 1.f, ck, s);
     else
-        final_sums_kernel<false><<<grid, kThreads, kFsSmemBytes, s>>>(blocks, tiles, params, fin, fin_out, hist, selkey, n_tiles,
-                                                                        per, float(eps), eps_adam BAOC_CHECK_ARG(ck));
-    BAOC_LAUNCH_CHECK();
+        e = debias ? launch_sums_instance<false, true>(grid, blocks, tiles, params, fin, fin_out, hist, selkey, n_tiles, per, float(eps), eps_adam, m_scale, v_scale, ck, s)
+                   : launch_sums_instance<false, false>(grid, blocks, tiles, params, fin, fin_out, hist, selkey, n_tiles, per, float(eps), eps_adam, 1.f, 1.f, ck, s);
+    if (e != cudaSuccess) return int(e);
     final_sums_combine_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, fin, fin_out, per);
     BAOC_LAUNCH_CHECK();
     select_pick_kernel<<<n_blocks, kThreads, 0, s>>>(sel, hist, selkey, 0);

@@ -587,7 +587,7 @@ int baoc_create(baoc_t** out, int n_blocks, const baoc_block_t* blocks, int n_cf
     if (!blocks || !cfgs || n_blocks <= 0 || n_cfg <= 0 || n_cfg > kMaxCfg) return BAOC_E_INVALID;
     baoc_opts_t o;
     if (opts) o = *opts; else baoc_default_opts(&o);
-    if (o.qblock != kQBlock || o.quantizer8 < 0 || o.quantizer8 > 1 || o.reserved != 0) return BAOC_E_INVALID;
+    if (o.qblock != kQBlock || o.quantizer8 < 0 || o.quantizer8 > 1 || o.debias < 0 || o.debias > 1) return BAOC_E_INVALID;
     if (!(o.beta_m >= 0 && o.beta_m < 1 && o.beta_v >= 0 && o.beta_v < 1 && o.beta_rho >= 0 && o.beta_rho < 1)) return BAOC_E_INVALID;
     if (!(o.a_hi > o.a_lo && o.rho_hi > o.rho_lo && o.snr_hi > o.snr_lo && o.eps >= 0)) return BAOC_E_INVALID;
     int64_t total = 0;

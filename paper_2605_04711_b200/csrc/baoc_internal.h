@@ -381,7 +381,7 @@ int launch_stats_combine(const StatBlock* blocks, const double* partials, double
 // row/column sums of the matrix blocks, the second and third sweep and the gather of the per-block results.
 int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* const* params, double* fin,
                       double* fin_out, uint32_t* hist, RankSel* sel, SelKey* selkey, int64_t n_tiles, int n_blocks, double eps,
-                      float eps_adam, int quantizer8, const CheckCtx& ck, cudaStream_t s);
+                      float eps_adam, int quantizer8, int debias, float m_scale, float v_scale, const CheckCtx& ck, cudaStream_t s);
 // The buffers of the select's second and third sweep.
 struct SelectArgs {
     const StatBlock* blocks;

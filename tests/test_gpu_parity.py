@@ -748,6 +748,26 @@ def test_precision_cosine_with_the_dynamic_codebook_on_the_device(B, H):
     assert differs >= len(wl.blocks) // 2                           # the codebook is really in use
 
 
+def test_diagnostics_from_bias_corrected_moments(B, H):
+    """debias = 1 (the alternative reading of the hats in Eq. 3): every diagnostic of Eq. 4-8, the quantiles and the
+    quantisation errors from m / (1 - beta_m^T), v / (1 - beta_v^T); the window itself (Eq. 3, Eq. 5 left) is unchanged."""
+    wl = _odd_workload(seed=77, window=5)
+    opts = B.default_opts()
+    opts.debias = 1
+    sess = H.Session(wl, opts=opts, n_grad_sets=2)
+    sess.init_params()
+    o = O.Opts(debias=True)
+    states = _oracle_window(sess, wl.window, o)
+    _, st, _ = _check_stats(sess, states, o)
+    plain = O.Opts()
+    moved = 0
+    for i, b in enumerate(wl.blocks):
+        raw_off = O.stats_finalize(states[i], sess.block_param_host(i), b.rows, b.cols, plain)
+        moved += abs(st[i]["snr"] - raw_off["snr"]) > 1e-3 * abs(raw_off["snr"])
+        assert abs(st[i]["q90"] - raw_off["q90"] / (1.0 - plain.beta_v ** wl.window)) <= 1e-6 * abs(st[i]["q90"])
+    assert moved >= len(wl.blocks) - 1                              # the correction is really applied
+
+
 def test_nonfinite_gradient_is_flagged_not_fatal(B, H):
     wl = _odd_workload(seed=31)
     sess = H.Session(wl, n_grad_sets=1)
