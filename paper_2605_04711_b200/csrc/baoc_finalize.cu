@@ -619,7 +619,6 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const SelPiece* __
     const uint32_t base1 = L.n > 1 ? uint32_t(key.lo) + (L.key[1] << key.s) : base0;
     // a vector block's last row may be short; every other row of a piece holds the thread's nc columns
     const int64_t short_row = (b->cols > 1 || (numel % kPieceCols) == 0) ? -1 : numel / kPieceCols;
-    const bool wide = g.vec && g.nc == 8;                     // the thread's usual row: eight elements, two 16-byte loads
     const uint32_t* __restrict__ vp = v + (int64_t(pc.row0) + g.ty) * g.cols + pc.col0 + g.tx * 8;
     const int64_t v_step = int64_t(g.step) * g.cols;
 
@@ -661,8 +660,34 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const SelPiece* __
                     if (mask & (1u << j)) seg[pos++] = sel_key(u[j], key.lo, wmax);
             }
         };
+        // whole batches of full rows first (no per-row decisions), then what is left, row by row
+        // (uniform over the CTA) every row of a thread is eight elements, two 16-byte loads, or the thread has no column at all
+        const bool plain = g.vec && (g.width & 7) == 0 && short_row < 0;
+        const int64_t batch = int64_t(kRhBatch) * g.step;
+        const int64_t r_full = plain ? int64_t(pc.row0) + (int64_t(pc.nrows) / batch) * batch : int64_t(pc.row0);
+        int64_t r0 = int64_t(pc.row0);
 #pragma unroll 1
-        for (int64_t r0 = int64_t(pc.row0); r0 < r_end; r0 += int64_t(kRhBatch) * g.step) {   // the same trips for every thread
+        for (; r0 < r_full; r0 += batch) {                    // the same trips for every thread
+            if (g.nc == 8) {
+                uint32_t u[kRhBatch][8];
+                double rs[kRhBatch];
+#pragma unroll
+                for (int k = 0; k < kRhBatch; ++k) {
+                    const uint4 a = ld_stream_u4(vp + k * v_step), c = ld_stream_u4(vp + k * v_step + 4);
+                    u[k][0] = a.x; u[k][1] = a.y; u[k][2] = a.z; u[k][3] = a.w; u[k][4] = c.x; u[k][5] = c.y; u[k][6] = c.z; u[k][7] = c.w;
+                    rs[k] = kResid ? __ldg(rowsum + (r0 + g.ty + int64_t(k) * g.step)) : 0.0;
+                }
+#pragma unroll
+                for (int k = 0; k < kRhBatch; ++k) row(std::true_type{}, u[k], 8, rs[k]);
+            }
+            vp += kRhBatch * v_step;
+            if (kKeys) {
+                __syncwarp();
+                if (wcnt[warp] > kRhDrainAt) drain();         // uniform over the warp: room for the next batch
+            }
+        }
+#pragma unroll 1
+        for (; r0 < r_end; r0 += batch) {                     // the same trips for every thread
             uint32_t u[kRhBatch][8];
             int n[kRhBatch];
             double rs[kRhBatch];
@@ -672,17 +697,10 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const SelPiece* __
                 n[k] = 0;
                 rs[k] = 0.0;
                 if (r < r_end) {
-                    if (wide && r != short_row) {
-                        const uint4 a = ld_stream_u4(vp + k * v_step), c = ld_stream_u4(vp + k * v_step + 4);
-                        u[k][0] = a.x; u[k][1] = a.y; u[k][2] = a.z; u[k][3] = a.w; u[k][4] = c.x; u[k][5] = c.y; u[k][6] = c.z; u[k][7] = c.w;
-                        n[k] = 8;
-                    } else {
-                        n[k] = piece_load(v, pc, g, numel, r, u[k]);
-                    }
+                    n[k] = piece_load(v, pc, g, numel, r, u[k]);
                     if (kResid) rs[k] = __ldg(rowsum + r);
                 }
             }
-            vp += kRhBatch * v_step;
 #pragma unroll
             for (int k = 0; k < kRhBatch; ++k) {
                 if (n[k] == 8) row(std::true_type{}, u[k], 8, rs[k]);
@@ -690,7 +708,7 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const SelPiece* __
             }
             if (kKeys) {
                 __syncwarp();
-                if (wcnt[warp] > kRhDrainAt) drain();         // uniform over the warp: room for the next batch
+                if (wcnt[warp] > kRhDrainAt) drain();
             }
         }
     };
