@@ -151,6 +151,8 @@ __device__ __forceinline__ void block_tiles_sum(const double* __restrict__ part,
     double acc[K];
 #pragma unroll
     for (int k = 0; k < K; ++k) acc[k] = 0.0;
+    // (four slots requested before the first is added: the order of the additions is unchanged)
+#pragma unroll 4
     for (int i = threadIdx.x; i < ntiles; i += kThreads) {
         const double* p = part + size_t(tile0 + i) * K;
 #pragma unroll
