@@ -205,6 +205,24 @@ def test_stats_invariants_identical_zero_and_flipped_gradients(B, H):
             assert st2[i]["F"] < 1e-6                                # constant matrix is rank one
 
 
+def test_finalize_on_extreme_shapes(B, H):
+    """The second finalize sweep walks a block by pieces (rows of a strip of at most 512 columns; a vector as rows of
+    512): a long vector with a ragged last row, a matrix of three very long rows whose length is no multiple of four
+    (scalar loads, thousands of strips, a last strip of a few columns), a very tall matrix of three columns (one
+    thread per row), and a matrix whose strips end in a narrow one.  Every diagnostic against the oracle."""
+    shapes = [(2_500_017, 1), (3, 700_003), (700_003, 3), (1500, 1032), (513, 1), (2, 5)]
+    blocks = [W.Block(f"x{i}", r, c) for i, (r, c) in enumerate(shapes)]
+    rng = np.random.default_rng(21)
+    for b in blocks:
+        b.stability = float(rng.uniform(0.2, 0.8)); b.tau = float(rng.uniform(0.0, 1.5)); b.scale = float(10.0 ** rng.uniform(-3, -1))
+    wl = W.Workload("shapes", blocks, window=3, mem_budget_frac=0.4, time_budget=1.3, seed=21)
+    sess = H.Session(wl, n_grad_sets=2)
+    sess.init_params()
+    states = _oracle_window(sess, wl.window)
+    _check_stats(sess, states)
+    assert sess.h.query().select_retries == 0
+
+
 def test_quantile_select_repeats_over_the_full_range_when_the_sample_misses_the_tails(B, H):
     """The select orders a block by a key fitted to 1024 evenly spaced elements of it.  Here those elements all lie in
     [1, 2) while 30 % of the others are a million times smaller and 20 % a thousand times larger, so both quantiles of
