@@ -44,7 +44,7 @@ def build(force: bool = False, verbose: bool = False, checked: bool = False) -> 
     nvcc = _nvcc()
     bdir = os.path.join(HERE, "_build", "checked" if checked else "plain")
     os.makedirs(bdir, exist_ok=True)
-    common = ["-std=c++17", "-O3", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
+    common = ["-std=c++17", "-O3", "-Wno-deprecated-gpu-targets", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
               "-Xcompiler", "-fPIC,-ffp-contract=off,-Wall"] + (["-DBAOC_CHECKED"] if checked else [])
     cuda_flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo"]
     if verbose:
@@ -58,7 +58,7 @@ def build(force: bool = False, verbose: bool = False, checked: bool = False) -> 
             print(" ".join(cmd), flush=True)
         subprocess.run(cmd, check=True)
         objs.append(obj)
-    subprocess.run([nvcc, "-shared", "-o", lib] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"], check=True)
+    subprocess.run([nvcc, "-shared", "-Wno-deprecated-gpu-targets", "-o", lib] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"], check=True)
     return lib
 
 
