@@ -766,15 +766,18 @@ def test_precision_cosine_with_the_dynamic_codebook_on_the_device(B, H):
     assert differs >= len(wl.blocks) // 2                           # the codebook is really in use
 
 
-def test_diagnostics_from_bias_corrected_moments(B, H):
+@pytest.mark.parametrize("dynamic", [False, True])
+def test_diagnostics_from_bias_corrected_moments(B, H, dynamic):
     """debias = 1 (the alternative reading of the hats in Eq. 3): every diagnostic of Eq. 4-8, the quantiles and the
-    quantisation errors from m / (1 - beta_m^T), v / (1 - beta_v^T); the window itself (Eq. 3, Eq. 5 left) is unchanged."""
+    quantisation errors from m / (1 - beta_m^T), v / (1 - beta_v^T); the window itself (Eq. 3, Eq. 5 left) is unchanged.
+    Also together with the other alternative reading of Eq. 8, the non-linear 8-bit codebook."""
     wl = _odd_workload(seed=77, window=5)
     opts = B.default_opts()
     opts.debias = 1
+    opts.quantizer8 = B.Q_DYNAMIC if dynamic else B.Q_LINEAR
     sess = H.Session(wl, opts=opts, n_grad_sets=2)
     sess.init_params()
-    o = O.Opts(debias=True)
+    o = O.Opts(debias=True, quantizer8="dynamic" if dynamic else "linear")
     states = _oracle_window(sess, wl.window, o)
     _, st, _ = _check_stats(sess, states, o)
     plain = O.Opts()

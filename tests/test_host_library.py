@@ -231,6 +231,20 @@ def test_export_import_blob_without_device_state(B):
         assert e.value.code == B.E_INVALID
 
 
+def test_options_default_to_the_literal_readings_and_are_validated(B):
+    o = B.default_opts()
+    assert (o.debias, o.quantizer8, o.use_snr, o.qblock) == (0, B.Q_LINEAR, 1, 256)
+    for field, bad in (("debias", 2), ("debias", -1), ("quantizer8", 7), ("qblock", 128)):
+        o = B.default_opts()
+        setattr(o, field, bad)
+        with pytest.raises(B.BaocError) as e:
+            B.Baoc([(64, 8, 8)], B.default_configs(), o)
+        assert e.value.code == B.E_INVALID
+    o = B.default_opts()
+    o.debias = 1
+    B.Baoc([(64, 8, 8)], B.default_configs(), o)
+
+
 def test_set_sampling_validates_indices_and_shrinks_the_workspace(B):
     blocks = [(4096 * 8, 256, 128), (1000, 1000, 1)]
     h = B.Baoc(blocks, B.default_configs())
