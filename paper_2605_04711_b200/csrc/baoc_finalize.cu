@@ -98,7 +98,7 @@ final_pilot_kernel(const StatBlock* __restrict__ blocks, float eps, float v_scal
 // Veltkamp split (x*(2^16+1) - (x*(2^16+1) - x) keeps the upper 8 significant
 // bits, rounded to nearest), which runs on the FMA pipe instead of the narrow
 // conversion pipe.  A thread keeps its partial sums in fp32 for at most
-// kFinRunTiles tiles (128 elements per thread) and widens them to double for the
+// kFinRunTiles tiles (512 elements per thread) and widens them to double for the
 // reduction across the CTA.
 //
 // The slices are staged through shared memory by per-thread cp.async copies two
@@ -992,8 +992,8 @@ select_first_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict
 BAOC_DEFINE_CHECK_FETCH(finalize_check_fetch)
 
 // Tiles per CTA of a sweep: as many as `most`, fewer when the workload would then not give every SM a few CTAs.
-static int run_tiles(int64_t n_tiles, int most) {
-    const int64_t want = n_tiles / (int64_t(148) * 6);
+static int run_tiles(int64_t n_tiles, int most, int ctas_per_sm = 6) {
+    const int64_t want = n_tiles / (int64_t(148) * ctas_per_sm);
     return int(want < 1 ? 1 : (want > most ? most : want));
 }
 
@@ -1020,7 +1020,7 @@ int launch_final_sums(const StatBlock* blocks, const Tile* tiles, const float* c
     BAOC_LAUNCH_CHECK();
     final_pilot_kernel<<<n_blocks, kThreads, 0, s>>>(blocks, float(eps), debias ? v_scale : 1.0f, fin_out, selkey);
     BAOC_LAUNCH_CHECK();
-    const int per = run_tiles(n_tiles, kFinRunTiles);
+    const int per = run_tiles(n_tiles, kFinRunTiles, 12);     // long runs (a run's hand-over costs a tenth of eight tiles' work), but six waves of CTAs at least
     const unsigned grid = unsigned((n_tiles + per - 1) / per);
     if (quantizer8)
         e = debias ? launch_sums_instance<true, true>(grid, blocks, tiles, params, fin, fin_out, hist, selkey, n_tiles, per, float(eps), eps_adam, m_scale, v_scale, ck, s)

@@ -39,7 +39,7 @@ constexpr int kFinFlag = 30;          //   [30] non-zero: an order statistic lie
 constexpr int kSelBits = 12;          // bits of the first and (at most) of the second radix pass of the quantile select
 constexpr int kSelBins = 1 << kSelBits;
 constexpr int kSel3Bits = 32 - 2 * kSelBits;   // bins of the third and last pass: 2^8 (a key has at most 31 bits: 12 + 12 + 7)
-constexpr int kFinRunTiles = 8;       // most tiles a CTA of the first finalize sweep works through (its partial sums stay in fp32 that long)
+constexpr int kFinRunTiles = 32;      // most tiles a CTA of the first finalize sweep works through (its partial sums stay in fp32 that long)
 constexpr int kSelRunTiles = 15;      // tiles a CTA of the stand-alone first pass (a repeated select) works through
 constexpr int kPieceCols = 512;       // widest piece of the select's second sweep, in columns
 constexpr int kPieceElems = 49152;    // most elements of a piece (its histograms count in 16 bits)
