@@ -30,6 +30,17 @@ __device__ __forceinline__ float4 ld_stream_f4(const void* p) {
                  : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(p));
     return r;
 }
+// 256-bit forms (sm_100): one request for a thread's eight fp32 values.  The address must be 32-byte aligned: true for
+// every tensor of the bound workspace and state buffer at an element index that is a multiple of eight; caller-owned
+// arrays promise 16 bytes only.
+__device__ __forceinline__ void ld_stream_f8(const void* p, float4& a, float4& b) {
+    asm volatile("ld.global.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w), "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w) : "l"(p));
+}
+__device__ __forceinline__ void st_stream_f8(void* p, const float (&x)[8]) {
+    asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]),
+                 "f"(x[4]), "f"(x[5]), "f"(x[6]), "f"(x[7]) : "memory");
+}
 __device__ __forceinline__ uint2 ld_stream_u2(const void* p) {
     uint2 r;
     asm volatile("ld.global.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(r.x), "=r"(r.y) : "l"(p));

@@ -57,8 +57,8 @@ stats_step_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
         if (full[s]) {
             wg[s] = ld_stream_u4(g + e);
             wp[s] = ld_stream_u4(gp + e);
-            m0[s] = ld_stream_f4(m + e); m1[s] = ld_stream_f4(m + e + 4);
-            v0[s] = ld_stream_f4(v + e); v1[s] = ld_stream_f4(v + e + 4);
+            ld_stream_f8(m + e, m0[s], m1[s]);                // (workspace tensors: 32-byte aligned at multiples of eight elements)
+            ld_stream_f8(v + e, v0[s], v1[s]);
         }
     }
 #pragma unroll
@@ -78,10 +78,8 @@ stats_step_kernel(const StatBlock* __restrict__ blocks, const Tile* __restrict__
                 mm[j] = ema(mm[j], x[j], om);
                 vv[j] = ema(vv[j], x[j] * x[j], ov);
             }
-            st_stream_f4(m + e, make_float4(mm[0], mm[1], mm[2], mm[3]));
-            st_stream_f4(m + e + 4, make_float4(mm[4], mm[5], mm[6], mm[7]));
-            st_stream_f4(v + e, make_float4(vv[0], vv[1], vv[2], vv[3]));
-            st_stream_f4(v + e + 4, make_float4(vv[4], vv[5], vv[6], vv[7]));
+            st_stream_f8(m + e, mm);
+            st_stream_f8(v + e, vv);
             st_stream_u4(gp + e, wg[s]);
         } else if (e < numel) {
             const int cnt = int(numel - e);

@@ -396,6 +396,12 @@ __device__ __forceinline__ void st8(float* p, const float (&x)[8]) {
     st_stream_f4(p, make_float4(x[0], x[1], x[2], x[3]));
     st_stream_f4(p + 4, make_float4(x[4], x[5], x[6], x[7]));
 }
+// Eight fp32 values to a caller-owned array (parameters): one 256-bit store where the array happens to be 32-byte
+// aligned (the interface promises 16), else two 128-bit ones.  wide is uniform over the CTA.
+__device__ __forceinline__ void st8_param(float* p, const float (&x)[8], bool wide) {
+    if (wide) st_stream_f8(p, x); else st8(p, x);
+}
+__device__ __forceinline__ bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0u; }
 // 0 * x is 0 for a finite x and NaN otherwise: one FMA per value folds a
 // non-finite test of many values into one accumulator.
 __device__ __forceinline__ float poison(float acc, float x) { return fmaf(x, 0.0f, acc); }
@@ -471,6 +477,7 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
     uint16_t* __restrict__ mh = static_cast<uint16_t*>(mp);
     uint16_t* __restrict__ vh = static_cast<uint16_t*>(vp);
     float chk = 0.f;
+    const bool th_wide = aligned32(th);                              // uniform over the CTA
     uint4 wg[kSlices];
     float4 t0[kSlices], t1[kSlices], m0[kSlices], m1[kSlices], v0[kSlices], v1[kSlices];
     uint4 mw[kSlices], vw[kSlices];
@@ -481,13 +488,14 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
         full[s] = e + 8 <= numel;
         if (full[s]) {
             wg[s] = ld_stream_u4(g + e);
-            t0[s] = ld_stream_f4(th + e); t1[s] = ld_stream_f4(th + e + 4);
+            if (th_wide) ld_stream_f8(th + e, t0[s], t1[s]);
+            else { t0[s] = ld_stream_f4(th + e); t1[s] = ld_stream_f4(th + e + 4); }
             if (kB16) {
                 if (kM) mw[s] = ld_stream_u4(mh + e);
                 if (kV) vw[s] = ld_stream_u4(vh + e);
-            } else {
-                if (kM) { m0[s] = ld_stream_f4(m + e); m1[s] = ld_stream_f4(m + e + 4); }
-                if (kV) { v0[s] = ld_stream_f4(v + e); v1[s] = ld_stream_f4(v + e + 4); }
+            } else {                                                 // state tensors: 32-byte aligned at multiples of eight elements
+                if (kM) ld_stream_f8(m + e, m0[s], m1[s]);
+                if (kV) ld_stream_f8(v + e, v0[s], v1[s]);
             }
         }
     }
@@ -510,15 +518,15 @@ __device__ __forceinline__ unsigned tile_dense(const StepBlock* b, const CfgStep
                 DenseElem<kM, kV, kB16>::upd(x[j], t[j], mm[j], vv[j], mb[j], vb[j], P);
                 chk = poison(chk, t[j]);
             }
-            st8(th + e, t);
+            st8_param(th + e, t, th_wide);
             if (kB16) {
                 if (kM) st_stream_u4(mh + e, make_uint4(pack_bf16x2_rne(mb[0], mb[1]), pack_bf16x2_rne(mb[2], mb[3]),
                                                         pack_bf16x2_rne(mb[4], mb[5]), pack_bf16x2_rne(mb[6], mb[7])));
                 if (kV) st_stream_u4(vh + e, make_uint4(pack_bf16x2_rne(vb[0], vb[1]), pack_bf16x2_rne(vb[2], vb[3]),
                                                         pack_bf16x2_rne(vb[4], vb[5]), pack_bf16x2_rne(vb[6], vb[7])));
             } else {
-                if (kM) st8(m + e, mm);
-                if (kV) st8(v + e, vv);
+                if (kM) st_stream_f8(m + e, mm);
+                if (kV) st_stream_f8(v + e, vv);
             }
         } else if (e < numel) {
             const int cnt = int(numel - e);
@@ -583,6 +591,7 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
         const int left = int(min64(numel - base, kTileF));          // a multiple of 8 here
         const uint16_t* __restrict__ gt = g + base;
         float* __restrict__ tht = th + base;
+        const bool th_wide = aligned32(tht);                          // uniform over the CTA
         const float* __restrict__ rt = r + row0;
         const int toff = threadIdx.x * 8;
         const uint32_t sm0 = smem_addr(stage), sg = threadIdx.x * 16, st_ = 4096 + threadIdx.x * 32;
@@ -623,7 +632,7 @@ __device__ __forceinline__ unsigned tile_factored(const StepBlock* b, const CfgS
                 t[j] = adaptive_apply(t[j], x[j], rs * cj[j], step, P);
                 chk = poison(chk, t[j]);
             }
-            st8(tht + e, t);
+            st8_param(tht + e, t, th_wide);
         }
         cp_async_wait<0>();
         return chk != 0.f;
@@ -759,6 +768,7 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
     const int left = int(min64(numel - base, kTileQ));              // elements of the block in this tile (>= 1)
     const uint16_t* __restrict__ gt = g + base;
     float* __restrict__ tht = th + base;
+    const bool th_wide = aligned32(tht);                             // uniform over the CTA
     int8_t* __restrict__ qmt = qm + base;
     uint8_t* __restrict__ qvt = qv + base;
     float* __restrict__ amt = am + base / kQBlock;                   // base is a multiple of the quantisation block
@@ -951,7 +961,7 @@ __device__ __forceinline__ unsigned tile_int8(const StepBlock* b, const CfgStep&
         }
 
         if (cnt == 8) {
-            st8(tht + e, t);
+            st8_param(tht + e, t, th_wide);
             if (kM) st_stream_u2(qmt + e, om);
             if (kV) st_stream_u2(qvt + e, ov);
         } else {
