@@ -663,6 +663,7 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const SelPiece* __
         // whole batches of full rows first (no per-row decisions), then what is left, row by row
         // (uniform over the CTA) every row of a thread is eight elements, two 16-byte loads, or the thread has no column at all
         const bool plain = g.vec && (g.width & 7) == 0 && short_row < 0;
+        const bool rows32 = (g.cols & 7) == 0;                // every row of the thread starts 32-byte aligned: one 256-bit load
         const int64_t batch = int64_t(kRhBatch) * g.step;
         const int64_t r_full = plain ? int64_t(pc.row0) + (int64_t(pc.nrows) / batch) * batch : int64_t(pc.row0);
         int64_t r0 = int64_t(pc.row0);
@@ -673,8 +674,12 @@ final_resid_hist_kernel(const StatBlock* __restrict__ blocks, const SelPiece* __
                 double rs[kRhBatch];
 #pragma unroll
                 for (int k = 0; k < kRhBatch; ++k) {
-                    const uint4 a = ld_stream_u4(vp + k * v_step), c = ld_stream_u4(vp + k * v_step + 4);
-                    u[k][0] = a.x; u[k][1] = a.y; u[k][2] = a.z; u[k][3] = a.w; u[k][4] = c.x; u[k][5] = c.y; u[k][6] = c.z; u[k][7] = c.w;
+                    if (rows32) {
+                        ld_stream_u8(vp + k * v_step, u[k]);
+                    } else {
+                        const uint4 a = ld_stream_u4(vp + k * v_step), c = ld_stream_u4(vp + k * v_step + 4);
+                        u[k][0] = a.x; u[k][1] = a.y; u[k][2] = a.z; u[k][3] = a.w; u[k][4] = c.x; u[k][5] = c.y; u[k][6] = c.z; u[k][7] = c.w;
+                    }
                     rs[k] = kResid ? __ldg(rowsum + (r0 + g.ty + int64_t(k) * g.step)) : 0.0;
                 }
 #pragma unroll
