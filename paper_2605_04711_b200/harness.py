@@ -100,7 +100,7 @@ class Session:
 
     def __init__(self, wl: W.Workload, configs: Optional[Sequence[B.Config]] = None, opts: Optional[B.Opts] = None,
                  n_grad_sets: int = 2, device: str = "cuda:0", pinned_host_grads: bool = False, samples=None,
-                 param_capacity: int = 0, factored_group_bytes: int = 0):
+                 param_capacity: int = 0, factored_group_bytes: int = 0, param_skew_elems: int = 0):
         global LIVE_SESSIONS
         if LIVE_SESSIONS is None:
             import weakref
@@ -123,7 +123,9 @@ class Session:
             return view
 
         self._alloc = alloc
-        self.params = alloc(4 * max(self.total, int(param_capacity)), True).view(torch.float32)
+        # param_skew_elems: start the parameter buffer this many elements into its allocation (4: every block pointer is
+        # then 16-byte but not 32-byte aligned, the least the interface accepts)
+        self.params = alloc(4 * (max(self.total, int(param_capacity)) + int(param_skew_elems)), True).view(torch.float32)[int(param_skew_elems):]
         self.grads = [alloc(2 * self.total, True).view(torch.bfloat16) for _ in range(n_grad_sets)]
         self.param_views = [self.params[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)]
         self.grad_views = [[g[o:o + b.numel] for o, b in zip(self.offs, wl.blocks)] for g in self.grads]

@@ -15,7 +15,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 # update path, ragged tails, one-element blocks, sampling, re-configuration, both routes of the select's last pass and
 # the repeated select
 CASES = ("odd_sizes or each_configuration or stateless_bf16 or factored_with or finalize_from_shared or sampled_statistics "
-         "or quantile_select or bias_corrected or extreme_shapes "
+         "or quantile_select or bias_corrected or extreme_shapes or least_alignment "
          "or reconfigure or configure_from_window or toy_pipeline or grouped_factored or nonfinite or coupled_decay "
          "or dynamic_codebook or adafactor")
 

@@ -920,6 +920,32 @@ def test_step_from_host_equals_separate_calls_bit_for_bit(B, H, extended):
     assert res[0][4] == res[1][4] == 0
 
 
+def test_parameters_at_the_least_alignment_the_interface_accepts(B, H):
+    """Parameter arrays need 16-byte alignment only; where one is 32-byte aligned the step uses 256-bit accesses on it.
+    Both routes must leave the same bits: every tuple on the ResNet-50-shaped workload, three steps, parameter
+    pointers at 16 (mod 32) against the harness's usual 512-byte alignment."""
+    wl = W.make_workload("resnet50", seed=5)
+    vec = {3: 1, 11: 7, 12: 9, 14: 2}
+    assign = [(vec[i % 15] if ((i % 15) in vec and b.cols <= 1) else i % 15) for i, b in enumerate(wl.blocks)]
+    res = []
+    for skew in (0, 4):
+        sess = H.Session(wl, configs=B.extended_configs(), n_grad_sets=2, param_skew_elems=skew)
+        assert all((v.data_ptr() % 32) == (16 if skew else 0) for v in sess.param_views)
+        sess.init_params()
+        sess.configure(assign)
+        for t in (1, 2, 3):
+            k = sess.fill_grads(t)
+            sess.sample_stats(k)
+            sess.step(k, t)
+        torch.cuda.synchronize()
+        res.append((sess.params.clone(), _state_tensors(sess, B), sess.h.nonfinite()[0]))
+    assert torch.equal(res[0][0], res[1][0])
+    assert len(res[0][1]) == len(res[1][1]) > 0
+    for x, y in zip(res[0][1], res[1][1]):
+        assert torch.equal(x, y)
+    assert res[0][2] == res[1][2] == 0
+
+
 @pytest.mark.parametrize("variant", [0, 1])
 @pytest.mark.parametrize("inherit", [True, False])
 def test_reconfigure_migrates_states_like_the_oracle(B, H, inherit, variant):
